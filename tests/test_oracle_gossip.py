@@ -1,0 +1,172 @@
+"""Pins for the oracle's gossip/top-k step and glue ops (no GPU)."""
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def ring(n):
+    W = np.zeros((n, n), np.float32)
+    for i in range(n):
+        for j in (i - 1, i, i + 1):
+            W[i, j % n] += np.float32(1.0 / 3.0)
+    return W
+
+
+def test_ring4_hand_case():
+    rows = {l.split()[0]: np.array(l.split()[1:], np.float32)
+            for l in open(os.path.join(GOLD, "gossip_ring4_hand_case.txt"))
+            if l.strip() and not l.startswith("#")}
+    xh = rows["x_half"].reshape(4, 1)
+    x, xhat, q = oracle.gossip_mix(xh, np.zeros((4, 1), np.float32), ring(4), 1.0)
+    assert np.allclose(x.ravel(), rows["x_out"], atol=1e-6)
+    assert np.array_equal(xhat.ravel(), rows["x_hat_new"])
+    assert np.array_equal(q, xh)
+
+
+@pytest.mark.parametrize("k_frac", [1.0, 0.1, 0.01])
+def test_average_is_preserved(k_frac):
+    # doubly-stochastic W: sum_i x_i = sum_i x_half_i for any x_hat, gamma, k
+    rng = np.random.default_rng(0)
+    n, d = 8, 1000
+    xh = rng.standard_normal((n, d)).astype(np.float32)
+    xhat = rng.standard_normal((n, d)).astype(np.float32)
+    k = max(1, int(k_frac * d))
+    x, _, _ = oracle.gossip_mix(xh, xhat, ring(n), 0.37, [0, d], [k])
+    assert np.allclose(x.astype(np.float64).sum(0), xh.astype(np.float64).sum(0),
+                       atol=1e-6 * n * np.abs(xh).max())
+
+
+def test_no_compression_is_plain_mixing():
+    # k = d, gamma = 1, x_hat = anything: x_hat_new = x_half, and x = W @ x_half (D-PSGD)
+    rng = np.random.default_rng(1)
+    n, d = 6, 257
+    xh = rng.standard_normal((n, d)).astype(np.float32)
+    xhat0 = np.zeros((n, d), np.float32)
+    W = ring(n)
+    x, xhat, q = oracle.gossip_mix(xh, xhat0, W, 1.0)
+    assert np.array_equal(xhat, xh)
+    assert np.allclose(x, W.astype(np.float64) @ xh.astype(np.float64), atol=1e-6)
+    # asymmetric row-stochastic W: row i holds the weights node i applies (not the transpose)
+    Wa = rng.uniform(0, 1, (n, n)); Wa /= Wa.sum(1, keepdims=True)
+    x, _, _ = oracle.gossip_mix(xh, xhat0, Wa.astype(np.float32), 1.0)
+    assert np.allclose(x, Wa.astype(np.float32).astype(np.float64) @ xh, atol=2e-6)
+
+
+def test_consensus_fixed_point_and_gamma():
+    n, d = 5, 33
+    row = np.linspace(-1, 1, d, dtype=np.float32)
+    xh = np.tile(row, (n, 1))
+    x, xhat, _ = oracle.gossip_mix(xh, xh.copy(), ring(n), 0.7)
+    assert np.array_equal(x, xh) and np.array_equal(xhat, xh)
+    # gamma scales the consensus term linearly
+    rng = np.random.default_rng(2)
+    xh = rng.standard_normal((n, d)).astype(np.float32)
+    xhat = rng.standard_normal((n, d)).astype(np.float32)
+    x1, _, _ = oracle.gossip_mix(xh, xhat, ring(n), 1.0, [0, d], [3])
+    x2, _, _ = oracle.gossip_mix(xh, xhat, ring(n), 0.25, [0, d], [3])
+    assert np.allclose((x2 - xh), 0.25 * (x1 - xh).astype(np.float64), atol=1e-6)
+
+
+def test_topk_selection_rules():
+    rng = np.random.default_rng(3)
+    n, d, k = 3, 500, 17
+    xh = rng.standard_normal((n, d)).astype(np.float32)
+    xhat0 = rng.standard_normal((n, d)).astype(np.float32)
+    _, xhat, q = oracle.gossip_mix(xh, xhat0, ring(n), 0.5, [0, d], [k])
+    delta = xh - xhat0
+    for i in range(n):
+        nz = np.flatnonzero(q[i])
+        assert len(nz) == k
+        assert np.array_equal(q[i, nz], delta[i, nz])
+        dropped = np.setdiff1d(np.arange(d), nz)
+        assert np.abs(delta[i, nz]).min() >= np.abs(delta[i, dropped]).max()
+    assert np.array_equal(xhat, xhat0 + q)                       # error feedback update
+    # brute force: the kept set equals the k largest by (|delta| desc, index asc)
+    for i in range(n):
+        order = sorted(range(d), key=lambda e: (-abs(float(delta[i, e])), e))
+        assert sorted(order[:k]) == np.flatnonzero(q[i]).tolist()
+
+
+def test_topk_ties_keep_lower_index_and_segments():
+    xh = np.array([[1, -1, 1, -1, 0.5, 2, 2, 2]], np.float32)
+    xhat0 = np.zeros_like(xh)
+    W1 = np.ones((1, 1), np.float32)
+    _, _, q = oracle.gossip_mix(xh, xhat0, W1, 1.0, [0, 8], [3])
+    assert q.tolist() == [[0, 0, 0, 0, 0, 2, 2, 2]]
+    _, _, q = oracle.gossip_mix(xh, xhat0, W1, 1.0, [0, 5, 8], [2, 1])   # layer-wise top-k
+    assert q.tolist() == [[1, -1, 0, 0, 0, 2, 0, 0]]
+    _, _, q = oracle.gossip_mix(xh, xhat0, W1, 1.0, [0, 5, 8], [5, 2])   # k == len: dense segment
+    assert q.tolist() == [[1, -1, 1, -1, 0.5, 2, 2, 0]]
+
+
+def test_uses_updated_public_copies():
+    # 2 nodes, W = 1/2 everywhere, k = d: x_i = xh_i + (1/2)(xh_j - xh_i) needs x_hat AFTER the update
+    xh = np.array([[2.0], [6.0]], np.float32)
+    W = np.full((2, 2), 0.5, np.float32)
+    x, _, _ = oracle.gossip_mix(xh, np.array([[100.0], [-50.0]], np.float32), W, 1.0)
+    assert x.ravel().tolist() == [4.0, 4.0]
+
+
+def test_sgd_update():
+    x = np.array([1.0, 2.0, -3.0], np.float32); g = np.array([0.5, -4.0, 0.25], np.float32)
+    assert oracle.sgd_update(x, g, 0.1).tolist() == [np.float32(1.0) - np.float32(0.1) * np.float32(0.5),
+                                                      np.float32(2.0) + np.float32(0.1) * np.float32(4.0),
+                                                      np.float32(-3.0) - np.float32(0.1) * np.float32(0.25)]
+
+
+def test_residual_add_and_adjoint():
+    rng = np.random.default_rng(4)
+    a = rng.standard_normal((2, 2, 4, 4, 3)).astype(np.float32)
+    r = rng.standard_normal((2, 2, 4, 4, 3)).astype(np.float32)
+    assert np.array_equal(oracle.residual_add(r, a), r + a)
+    # projection shortcut: spatial subsample by 2, channels placed at offset 2 of 7
+    r2 = rng.standard_normal((2, 2, 2, 2, 7)).astype(np.float32)
+    y = oracle.residual_add(r2, a, stride=2, ch_off=2)
+    want = r2.copy(); want[..., 2:5] += a[:, :, ::2, ::2, :]
+    assert np.array_equal(y, want)
+    dy = rng.standard_normal(r2.shape).astype(np.float32)
+    gm = rng.standard_normal(a.shape).astype(np.float32)
+    da = oracle.residual_add_bwd(dy, gm, stride=2, ch_off=2)
+    want = gm.copy(); want[:, :, ::2, ::2, :] += dy[..., 2:5]
+    assert np.array_equal(da, want)
+
+
+def test_pools():
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((2, 3, 4, 6, 5)).astype(np.float32)
+    assert np.allclose(oracle.avgpool(x), x.astype(np.float64).mean(axis=(2, 3)), atol=1e-7)
+    dy = rng.standard_normal((2, 3, 5)).astype(np.float32)
+    dx = oracle.avgpool_bwd(dy, 4, 6)
+    assert np.array_equal(dx, np.broadcast_to((dy / np.float32(24))[:, :, None, None, :], dx.shape))
+    y, idx = oracle.maxpool2x2(x)
+    want = x.reshape(2, 3, 2, 2, 3, 2, 5).max(axis=(3, 5))
+    assert np.array_equal(y, want)
+    g = rng.standard_normal(y.shape).astype(np.float32)
+    dxm = oracle.maxpool2x2_bwd(g, idx, 4, 6)
+    assert np.allclose(dxm.sum(), g.sum(), atol=1e-4)
+    assert np.array_equal(dxm.reshape(2, 3, 2, 2, 3, 2, 5).sum(axis=(3, 5)), g)
+    assert np.all((dxm != 0) <= (x == np.repeat(np.repeat(y, 2, 2), 2, 3)))
+
+
+def test_softmax_ce():
+    from scipy.special import log_softmax, softmax
+    rng = np.random.default_rng(6)
+    z = (3 * rng.standard_normal((2, 5, 10))).astype(np.float32)
+    lab = rng.integers(0, 10, (2, 5)).astype(np.int32)
+    loss, dz = oracle.softmax_ce(z, lab)
+    ls = log_softmax(z.astype(np.float64), axis=-1)
+    want_loss = -np.take_along_axis(ls, lab[..., None].astype(np.int64), -1).mean(axis=(1, 2))
+    assert np.allclose(loss, want_loss, atol=1e-6)
+    onehot = np.eye(10)[lab]
+    assert np.allclose(dz, (softmax(z.astype(np.float64), axis=-1) - onehot) / 5, atol=1e-7)
+    assert np.allclose(dz.sum(-1), 0, atol=1e-6)
+
+
+def test_colsum():
+    x = np.arange(24, dtype=np.float32).reshape(2, 3, 4)
+    assert np.array_equal(oracle.colsum(x), x.sum(1))
