@@ -1,0 +1,237 @@
+/*
+ * lpdt.h — C ABI of the low-precision decentralized training step library
+ * (8-bit training step of arXiv 2111.09389 on NVIDIA B200, sm_100a).
+ *
+ * Conventions (all entry points)
+ *   - Every data pointer is a DEVICE pointer owned by the caller unless the
+ *     argument is marked "host".  The library allocates no device memory;
+ *     scratch comes from the caller's workspace `ws` (`ws_bytes` long, 256-byte
+ *     aligned), whose required size the matching *_workspace_size call returns.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *     Calls only enqueue work; they never synchronise.  A workspace may be
+ *     reused by the next call on the same stream.
+ *   - The N simulated decentralized nodes are the leading dimension of every
+ *     tensor; each node has its own values and its own quantization scale.
+ *       activations  NHWC  [nodes][B][H][W][C]
+ *       weights      KRSC  [nodes][Cout][R][S][Cin]
+ *       parameters   flat  [nodes][d]; a tensor that lives inside the flat
+ *                    parameter (or gradient) vector is addressed by a base
+ *                    pointer plus a `*_node_stride` in elements.
+ *   - Return value: LPDT_OK or an error code.  Argument errors are detected on
+ *     the host before anything is enqueued.  Kernels never trap or spin
+ *     without bound: a device-side wait that runs out writes a non-zero code
+ *     into `dev_status` (one int32, caller-zeroed, nullable) and the kernel
+ *     returns.
+ *   - Integer accumulators are int32 and wrap modulo 2^32 like the hardware.
+ *   - Floating point: element-wise arithmetic is a fixed sequence of
+ *     individually rounded fp32 operations (no fused multiply-add, no fast
+ *     math); every reduction is accumulated in fp64 and rounded once.
+ */
+#ifndef LPDT_H
+#define LPDT_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t lpdt_status;
+enum {
+    LPDT_OK = 0,
+    LPDT_ERR_INVALID_ARG = 1,   /* null pointer, bad size, misalignment */
+    LPDT_ERR_UNSUPPORTED = 2,   /* valid request this build has no kernel for */
+    LPDT_ERR_WORKSPACE = 3,     /* workspace missing or too small */
+    LPDT_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed */
+    LPDT_ERR_TIMEOUT = 5,       /* a bounded device-side wait expired */
+    LPDT_ERR_OVERFLOW = 6
+};
+
+typedef enum { LPDT_SYM_S8 = 0, LPDT_AFFINE_U8 = 1 } lpdt_qmode;
+typedef enum { LPDT_ROUND_NEAREST_EVEN = 0, LPDT_ROUND_STOCHASTIC = 1 } lpdt_round;
+
+/* Convolution geometry.  Ho = (H + 2*pad - R)/stride + 1, likewise Wo.
+ * A linear layer is R = S = H = W = 1, stride 1, pad 0 (B rows, Cin -> Cout). */
+typedef struct {
+    int32_t nodes, B, H, W, Cin, Cout, R, S, stride, pad;
+} lpdt_conv_desc;
+
+const char *lpdt_version(void);
+const char *lpdt_status_string(lpdt_status s);
+
+/* ---------------------------------------------------------------------------
+ * lpdt_quantize — per-tensor, per-node 8-bit quantization.
+ * Paper: Section 3, "Low Precision Training" (weights, activations and layer
+ * gradients are quantized to 8 bits in every iteration; the scheme is named by
+ * citation only, the formulas below are this library's reading).
+ *
+ *   LPDT_SYM_S8 :  amax = max|x|; scale = amax/127; inv = 127/amax
+ *       nearest-even : q = clamp(rne(x*inv), -127, 127)
+ *       stochastic   : t = x*inv; q = floor(t) + [u < t - floor(t)], with u the
+ *                      24-bit uniform from word (i mod 4) of Philox4x32-10 at
+ *                      counter (i/4 low, i/4 high, node, ctr_offset), key = seed
+ *       amax == 0 gives scale = 1 and q = 0.
+ *   LPDT_AFFINE_U8 (nearest-even only): lo = min(0,min x), hi = max(0,max x),
+ *       scale = (hi-lo)/255 (1 if hi == lo), zp = clamp(rne(-lo/scale),0,255),
+ *       q = clamp(rne(x/scale) + zp, 0, 255), stored in the same byte array.
+ *
+ * x     : fp32, node n starts at x + n*x_node_stride, n_per_node elements each
+ * q     : 8-bit codes, contiguous [nodes][n_per_node]
+ * scale : fp32 [nodes];  zero_point : int32 [nodes], required for AFFINE_U8 only
+ * ws    : lpdt_quantize_workspace_size(nodes) bytes
+ * Errors: INVALID_ARG (null/negative/misaligned), WORKSPACE, CUDA.
+ * n_per_node == 0 or nodes == 0 is a no-op returning LPDT_OK.
+ */
+size_t lpdt_quantize_workspace_size(int32_t nodes);
+lpdt_status lpdt_quantize(const float *x, int32_t nodes, int64_t n_per_node, int64_t x_node_stride,
+                          lpdt_qmode mode, lpdt_round rounding, uint64_t seed, uint32_t ctr_offset,
+                          int8_t *q, float *scale, int32_t *zero_point,
+                          void *ws, size_t ws_bytes, void *stream);
+
+/* y = scale[n] * (q - zp[n]); zero_point == NULL means symmetric signed codes.
+ * q is contiguous [nodes][n_per_node]; node n of y starts at y + n*y_node_stride. */
+lpdt_status lpdt_dequantize(const int8_t *q, int32_t nodes, int64_t n_per_node,
+                            const float *scale, const int32_t *zero_point,
+                            float *y, int64_t y_node_stride, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * Quantized contractions on symmetric int8 operands (Section 3: the forward
+ * product and both backward products run on 8-bit operands; the operation
+ * count table's Conv and Linear rows count the three alike).  int32
+ * accumulation; the fp32 result is (float)acc * (s1[n]*s2[n]) (+ bias).
+ *
+ * fwd        acc[n,b,oh,ow,co] = sum_{r,s,ci} A[n,b,oh*st+r-p,ow*st+s-p,ci] * W[n,co,r,s,ci]
+ * bwd_data   dA[n,b,ih,iw,ci]  = sum_{r,s,co} E[n,b,oh,ow,co] * W[n,co,r,s,ci]
+ *                                over (oh,ow) with ih = oh*st+r-p, iw = ow*st+s-p
+ * bwd_weight dW[n,co,r,s,ci]   = sum_{b,oh,ow} E[n,b,oh,ow,co] * A[n,b,oh*st+r-p,ow*st+s-p,ci]
+ * Taps that fall outside the image read zero.
+ *
+ * A, E, Wq : int8, contiguous in the layouts above;  sA, sE, sW : fp32 [nodes]
+ * Y/dA/dW  : fp32 output (nullable);  Yacc/dAacc/dWacc : raw int32 accumulators
+ *            (nullable; same shape, contiguous).  At least one must be given.
+ * bias     : fp32, node n at bias + n*bias_node_stride, Cout entries (nullable)
+ * dW       : node n at dW + n*dw_node_stride (weight gradients stay fp32:
+ *            "gradient bifurcation"); dWacc is contiguous.
+ * ws       : lpdt_qconv_workspace_size(desc, which) bytes, which = 0 fwd,
+ *            1 bwd_data, 2 bwd_weight.
+ * Errors: INVALID_ARG, UNSUPPORTED (shape outside every kernel's range),
+ *         WORKSPACE, CUDA; TIMEOUT is reported through dev_status.
+ */
+size_t lpdt_qconv_workspace_size(const lpdt_conv_desc *d, int32_t which);
+lpdt_status lpdt_qconv_fwd(const lpdt_conv_desc *d, const int8_t *A, const float *sA,
+                           const int8_t *Wq, const float *sW,
+                           const float *bias, int64_t bias_node_stride,
+                           float *Y, int32_t *Yacc,
+                           void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
+lpdt_status lpdt_qconv_bwd_data(const lpdt_conv_desc *d, const int8_t *E, const float *sE,
+                                const int8_t *Wq, const float *sW,
+                                float *dA, int32_t *dAacc,
+                                void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
+lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8_t *E, const float *sE,
+                                  const int8_t *A, const float *sA,
+                                  float *dW, int64_t dw_node_stride, int32_t *dWacc,
+                                  void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * Range-EvoNorm (Eq. "ren"), forward and backward.
+ * For node n, sample b, group G of cpg = C/groups consecutive channels:
+ *   mx, mn = max/min of x over (h, w, c in G);  D = Cst*(mx-mn) + eps,
+ *   Cst = 1/sqrt(2 ln cpg);  u = v_c*x;  hs = clamp((u+3)/6, 0, 1);  m = x*hs;
+ *   y = (gamma_c*m)*(1/D) + beta_c
+ * Backward (t = dy*gamma_c, hp = 1/6 on -3<u<3 else 0, S = sum_G t*m):
+ *   dx = (t*(hs + u*hp))*(1/D), then dx[argmax] -= Cst*S/D^2, dx[argmin] += Cst*S/D^2
+ *   (skipped when argmax == argmin);  dbeta_c = sum dy;  dgamma_c = sum dy*(m/D);
+ *   dv_c = sum t*x*x*hp/D, sums over the node's (b,h,w).
+ * argmax/argmin: lowest (h*W+w)*C+c index attaining the extremum.
+ *
+ * x, y, dy, dx : fp32 NHWC;  v, gamma, beta : fp32, node n at p + n*param_node_stride
+ * gmin, gmax : fp32 [nodes][B][groups];  argmin, argmax : int32, same shape
+ * dv, dgamma, dbeta : fp32, node n at p + n*grad_node_stride, C entries
+ * Requires C % groups == 0 and cpg >= 2 (Cst is infinite for cpg = 1).
+ * Errors: INVALID_ARG, UNSUPPORTED (C beyond the kernels' range), WORKSPACE, CUDA.
+ */
+lpdt_status lpdt_range_evonorm_fwd(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C,
+                                   int32_t groups, float eps, const float *x,
+                                   const float *v, const float *gamma, const float *beta,
+                                   int64_t param_node_stride, float *y,
+                                   float *gmin, float *gmax, int32_t *argmin, int32_t *argmax,
+                                   void *stream);
+size_t lpdt_range_evonorm_bwd_workspace_size(int32_t nodes, int32_t C);
+lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C,
+                                   int32_t groups, float eps, const float *dy, const float *x,
+                                   const float *v, const float *gamma, int64_t param_node_stride,
+                                   const float *gmin, const float *gmax,
+                                   const int32_t *argmin, const int32_t *argmax,
+                                   float *dx, float *dv, float *dgamma, float *dbeta,
+                                   int64_t grad_node_stride,
+                                   void *ws, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * lpdt_gossip_mix — compression, public-copy update and gossip averaging of
+ * CHOCO-SGD (Algorithm 3: "compute and compress", the x_hat update, and the
+ * gossip update), for all nodes at once:
+ *   delta_i = x_half_i - x_hat_i
+ *   q_i     = delta_i on the seg_k[s] largest |delta_i| of every segment s
+ *             (equal magnitudes: lower index kept), 0 elsewhere;
+ *             seg_k[s] >= segment length means no compression
+ *   x_hat_i <- x_hat_i + q_i
+ *   x_out_i = x_half_i + gamma * sum_j Wmix[i][j] * (x_hat_j - x_hat_i)   (updated x_hat)
+ * x_half, x_hat (in/out), x_out : fp32 [nodes][d];  x_out may alias x_half.
+ * Wmix : fp32 [nodes][nodes] row-major, row i = the weights node i applies.
+ * seg_offsets (n_segments+1 entries) and seg_k (n_segments) are HOST arrays;
+ * segments must tile [0,d).  n_segments = 1 is the flattened vector.
+ * Errors: INVALID_ARG, UNSUPPORTED (nodes > 64), WORKSPACE, CUDA.
+ */
+size_t lpdt_gossip_mix_workspace_size(int32_t nodes, int64_t d, int32_t n_segments);
+lpdt_status lpdt_gossip_mix(int32_t nodes, int64_t d, const float *x_half, float *x_hat,
+                            float *x_out, const float *Wmix, float gamma,
+                            int32_t n_segments, const int64_t *seg_offsets, const int64_t *seg_k,
+                            void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
+
+/* ---------------------------------------------------------------------------
+ * Glue around the layers of one training step.
+ */
+
+/* Local SGD update (Algorithm 1, "update the model"): out = x - lr*g on the
+ * fp32 master weights.  out may alias x. */
+lpdt_status lpdt_sgd_update(int64_t n, const float *x, const float *g, float lr, float *out,
+                            void *stream);
+
+/* Residual connection y = r + P(a): P subsamples a [nodes*B][H][W][Ca]
+ * spatially by `stride` and places its channels at ch_off within C channels
+ * (identity shortcut: stride 1, Ca = C, ch_off 0).  y may alias r. */
+lpdt_status lpdt_residual_add(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t Ca,
+                              int32_t C, int32_t stride, int32_t ch_off,
+                              const float *r, const float *a, float *y, void *stream);
+/* Adjoint: da = g_main + P^T(dy).  da may alias g_main. */
+lpdt_status lpdt_residual_add_bwd(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t Ca,
+                                  int32_t C, int32_t stride, int32_t ch_off,
+                                  const float *dy, const float *g_main, float *da, void *stream);
+
+/* Global average pool over HW positions and its adjoint (dx = dy/HW). */
+lpdt_status lpdt_avgpool(int32_t nodes, int32_t B, int32_t HW, int32_t C,
+                         const float *x, float *y, void *stream);
+lpdt_status lpdt_avgpool_bwd(int32_t nodes, int32_t B, int32_t HW, int32_t C,
+                             const float *dy, float *dx, void *stream);
+
+/* 2x2/stride-2 max-pool on fp32 NHWC; idx (int8, output shape) records the
+ * winning tap 0..3 (row-major, first maximum wins).  H and W must be even. */
+lpdt_status lpdt_maxpool2x2(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C,
+                            const float *x, float *y, int8_t *idx, void *stream);
+lpdt_status lpdt_maxpool2x2_bwd(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C,
+                                const float *dy, const int8_t *idx, float *dx, void *stream);
+
+/* Softmax cross-entropy per node (mean over the node's batch):
+ * loss[n], dlogits = (softmax - onehot)/B.  logits fp32 [nodes][B][K], labels int32. */
+lpdt_status lpdt_softmax_ce(int32_t nodes, int32_t B, int32_t K, const float *logits,
+                            const int32_t *labels, float *loss, float *dlogits, void *stream);
+
+/* out[n][c] = sum_b x[n][b][c] (bias gradient); node n of out at out + n*out_node_stride. */
+lpdt_status lpdt_colsum(int32_t nodes, int32_t B, int32_t C, const float *x,
+                        float *out, int64_t out_node_stride, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LPDT_H */

@@ -1,0 +1,166 @@
+"""Python binding of the lpdt C ABI: argument marshalling only.
+
+Every function has the name of the C entry point it calls (include/lpdt.h),
+takes torch CUDA tensors as device memory, and launches on torch's current
+stream.  No arithmetic happens here.
+"""
+import ctypes as C
+
+import torch
+
+from ._lib import ConvDesc, lib
+
+
+class LpdtError(RuntimeError):
+    def __init__(self, fn, code):
+        self.code = code
+        super().__init__(f"{fn} failed: {lib().lpdt_status_string(code).decode()} ({code})")
+
+
+def _check(fn, code):
+    if code != 0:
+        raise LpdtError(fn, code)
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    assert t.is_cuda, "device tensor expected"
+    return t.data_ptr()
+
+
+def _stream():
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _ws(ws):
+    return (_ptr(ws), 0 if ws is None else ws.numel() * ws.element_size())
+
+
+def lpdt_version():
+    return lib().lpdt_version().decode()
+
+
+def conv_desc(nodes, B, H, W, Cin, Cout, R=3, S=3, stride=1, pad=1):
+    return ConvDesc(nodes, B, H, W, Cin, Cout, R, S, stride, pad)
+
+
+def lpdt_quantize_workspace_size(nodes):
+    return lib().lpdt_quantize_workspace_size(nodes)
+
+
+def lpdt_quantize(x, nodes, n_per_node, x_node_stride, q, scale, ws, mode=0, rounding=0, seed=0,
+                  ctr_offset=0, zero_point=None):
+    p, nb = _ws(ws)
+    _check("lpdt_quantize", lib().lpdt_quantize(_ptr(x), nodes, n_per_node, x_node_stride, mode, rounding,
+                                                seed, ctr_offset, _ptr(q), _ptr(scale), _ptr(zero_point),
+                                                p, nb, _stream()))
+
+
+def lpdt_dequantize(q, nodes, n_per_node, scale, y, y_node_stride=None, zero_point=None):
+    ys = n_per_node if y_node_stride is None else y_node_stride
+    _check("lpdt_dequantize", lib().lpdt_dequantize(_ptr(q), nodes, n_per_node, _ptr(scale),
+                                                    _ptr(zero_point), _ptr(y), ys, _stream()))
+
+
+def lpdt_qconv_workspace_size(desc, which):
+    return lib().lpdt_qconv_workspace_size(C.byref(desc), which)
+
+
+def lpdt_qconv_fwd(desc, A, sA, Wq, sW, Y=None, Yacc=None, bias=None, bias_node_stride=0, ws=None,
+                   dev_status=None):
+    p, nb = _ws(ws)
+    _check("lpdt_qconv_fwd", lib().lpdt_qconv_fwd(C.byref(desc), _ptr(A), _ptr(sA), _ptr(Wq), _ptr(sW),
+                                                  _ptr(bias), bias_node_stride, _ptr(Y), _ptr(Yacc), p, nb,
+                                                  _ptr(dev_status), _stream()))
+
+
+def lpdt_qconv_bwd_data(desc, E, sE, Wq, sW, dA=None, dAacc=None, ws=None, dev_status=None):
+    p, nb = _ws(ws)
+    _check("lpdt_qconv_bwd_data", lib().lpdt_qconv_bwd_data(C.byref(desc), _ptr(E), _ptr(sE), _ptr(Wq),
+                                                            _ptr(sW), _ptr(dA), _ptr(dAacc), p, nb,
+                                                            _ptr(dev_status), _stream()))
+
+
+def lpdt_qconv_bwd_weight(desc, E, sE, A, sA, dW=None, dw_node_stride=0, dWacc=None, ws=None,
+                          dev_status=None):
+    p, nb = _ws(ws)
+    _check("lpdt_qconv_bwd_weight", lib().lpdt_qconv_bwd_weight(C.byref(desc), _ptr(E), _ptr(sE), _ptr(A),
+                                                                _ptr(sA), _ptr(dW), dw_node_stride,
+                                                                _ptr(dWacc), p, nb, _ptr(dev_status),
+                                                                _stream()))
+
+
+def lpdt_range_evonorm_fwd(nodes, B, H, W, Cc, groups, eps, x, v, gamma, beta, param_node_stride, y,
+                           gmin, gmax, argmin, argmax):
+    _check("lpdt_range_evonorm_fwd", lib().lpdt_range_evonorm_fwd(
+        nodes, B, H, W, Cc, groups, eps, _ptr(x), _ptr(v), _ptr(gamma), _ptr(beta), param_node_stride,
+        _ptr(y), _ptr(gmin), _ptr(gmax), _ptr(argmin), _ptr(argmax), _stream()))
+
+
+def lpdt_range_evonorm_bwd_workspace_size(nodes, Cc):
+    return lib().lpdt_range_evonorm_bwd_workspace_size(nodes, Cc)
+
+
+def lpdt_range_evonorm_bwd(nodes, B, H, W, Cc, groups, eps, dy, x, v, gamma, param_node_stride, gmin,
+                           gmax, argmin, argmax, dx, dv, dgamma, dbeta, grad_node_stride, ws):
+    p, nb = _ws(ws)
+    _check("lpdt_range_evonorm_bwd", lib().lpdt_range_evonorm_bwd(
+        nodes, B, H, W, Cc, groups, eps, _ptr(dy), _ptr(x), _ptr(v), _ptr(gamma), param_node_stride,
+        _ptr(gmin), _ptr(gmax), _ptr(argmin), _ptr(argmax), _ptr(dx), _ptr(dv), _ptr(dgamma), _ptr(dbeta),
+        grad_node_stride, p, nb, _stream()))
+
+
+def lpdt_gossip_mix_workspace_size(nodes, d, n_segments):
+    return lib().lpdt_gossip_mix_workspace_size(nodes, d, n_segments)
+
+
+def lpdt_gossip_mix(nodes, d, x_half, x_hat, x_out, Wmix, gamma, seg_offsets, seg_k, ws, dev_status=None):
+    """seg_offsets / seg_k: host sequences of Python ints."""
+    ns = len(seg_k)
+    so = (C.c_int64 * (ns + 1))(*[int(v) for v in seg_offsets])
+    sk = (C.c_int64 * ns)(*[int(v) for v in seg_k])
+    p, nb = _ws(ws)
+    _check("lpdt_gossip_mix", lib().lpdt_gossip_mix(nodes, d, _ptr(x_half), _ptr(x_hat), _ptr(x_out),
+                                                    _ptr(Wmix), gamma, ns, C.addressof(so), C.addressof(sk),
+                                                    p, nb, _ptr(dev_status), _stream()))
+
+
+def lpdt_sgd_update(n, x, g, lr, out):
+    _check("lpdt_sgd_update", lib().lpdt_sgd_update(n, _ptr(x), _ptr(g), lr, _ptr(out), _stream()))
+
+
+def lpdt_residual_add(nodes, B, H, W, Ca, Cc, stride, ch_off, r, a, y):
+    _check("lpdt_residual_add", lib().lpdt_residual_add(nodes, B, H, W, Ca, Cc, stride, ch_off, _ptr(r),
+                                                        _ptr(a), _ptr(y), _stream()))
+
+
+def lpdt_residual_add_bwd(nodes, B, H, W, Ca, Cc, stride, ch_off, dy, g_main, da):
+    _check("lpdt_residual_add_bwd", lib().lpdt_residual_add_bwd(nodes, B, H, W, Ca, Cc, stride, ch_off,
+                                                                _ptr(dy), _ptr(g_main), _ptr(da), _stream()))
+
+
+def lpdt_avgpool(nodes, B, HW, Cc, x, y):
+    _check("lpdt_avgpool", lib().lpdt_avgpool(nodes, B, HW, Cc, _ptr(x), _ptr(y), _stream()))
+
+
+def lpdt_avgpool_bwd(nodes, B, HW, Cc, dy, dx):
+    _check("lpdt_avgpool_bwd", lib().lpdt_avgpool_bwd(nodes, B, HW, Cc, _ptr(dy), _ptr(dx), _stream()))
+
+
+def lpdt_maxpool2x2(nodes, B, H, W, Cc, x, y, idx):
+    _check("lpdt_maxpool2x2", lib().lpdt_maxpool2x2(nodes, B, H, W, Cc, _ptr(x), _ptr(y), _ptr(idx), _stream()))
+
+
+def lpdt_maxpool2x2_bwd(nodes, B, H, W, Cc, dy, idx, dx):
+    _check("lpdt_maxpool2x2_bwd", lib().lpdt_maxpool2x2_bwd(nodes, B, H, W, Cc, _ptr(dy), _ptr(idx), _ptr(dx),
+                                                            _stream()))
+
+
+def lpdt_softmax_ce(nodes, B, K, logits, labels, loss, dlogits):
+    _check("lpdt_softmax_ce", lib().lpdt_softmax_ce(nodes, B, K, _ptr(logits), _ptr(labels), _ptr(loss),
+                                                    _ptr(dlogits), _stream()))
+
+
+def lpdt_colsum(nodes, B, Cc, x, out, out_node_stride):
+    _check("lpdt_colsum", lib().lpdt_colsum(nodes, B, Cc, _ptr(x), _ptr(out), out_node_stride, _stream()))

@@ -1,0 +1,332 @@
+// Range-EvoNorm (Eq. "ren") forward and backward.
+//
+// One CTA per (node, sample).  Every thread owns a fixed vector-column of V
+// channels and walks the pixels, so global accesses are fully coalesced 16-byte
+// loads and the thread's channel parameters and group live in registers.
+// Pass 1 finds the per-group extrema (and, backward, the group sum S and the
+// per-channel gradient sums); a warp-shuffle reduction with a
+// (value, lowest index) comparator merges the threads of a group.  Pass 2
+// re-reads the sample (an L2 hit: a sample is at most a few hundred KB) and
+// writes the output.  Both kernels are HBM-bound: forward moves 4 B in + 4 B
+// out per element, backward 8 B in + 4 B out.
+#include <math.h>
+#include "common.cuh"
+
+namespace lpdt {
+
+struct Ext { float v; int idx; };
+
+__device__ __forceinline__ Ext ext_max(Ext a, Ext b) {
+    return (b.v > a.v || (b.v == a.v && b.idx < a.idx)) ? b : a;
+}
+__device__ __forceinline__ Ext ext_min(Ext a, Ext b) {
+    return (b.v < a.v || (b.v == a.v && b.idx < a.idx)) ? b : a;
+}
+__device__ __forceinline__ Ext shfl_ext(Ext e, int o) {
+    Ext r; r.v = __shfl_xor_sync(0xffffffffu, e.v, o); r.idx = __shfl_xor_sync(0xffffffffu, e.idx, o);
+    return r;
+}
+
+template <int V> struct VecLoad;
+template <> struct VecLoad<4> {
+    static __device__ __forceinline__ void ld(const float *p, float (&o)[4]) {
+        float4 t = *reinterpret_cast<const float4 *>(p); o[0] = t.x; o[1] = t.y; o[2] = t.z; o[3] = t.w;
+    }
+    static __device__ __forceinline__ void st(float *p, const float (&o)[4]) {
+        *reinterpret_cast<float4 *>(p) = make_float4(o[0], o[1], o[2], o[3]);
+    }
+};
+template <> struct VecLoad<1> {
+    static __device__ __forceinline__ void ld(const float *p, float (&o)[1]) { o[0] = *p; }
+    static __device__ __forceinline__ void st(float *p, const float (&o)[1]) { *p = o[0]; }
+};
+
+// hard sigmoid and the normalised product, each operation rounded on its own
+__device__ __forceinline__ float hsig(float u) {
+    float h = __fdiv_rn(__fadd_rn(u, 3.f), 6.f);
+    return fminf(fmaxf(h, 0.f), 1.f);
+}
+
+// Reduce per-thread extrema to per-group extrema.  s_mn/s_mx hold one entry per
+// thread; members of group g are the threads whose column lies in the group.
+template <int V>
+__device__ void reduce_groups(Ext mn, Ext mx, Ext *s_mn, Ext *s_mx, Ext *g_mn, Ext *g_mx,
+                              int CV, int cpg, int groups) {
+    const int T = blockDim.x, t = threadIdx.x;
+    s_mn[t] = mn; s_mx[t] = mx;
+    __syncthreads();
+    const int lane = t & 31, warp = t >> 5, nw = T >> 5;
+    const int cols = cpg / V, rows = T / CV, members = cols * rows;
+    for (int g = warp; g < groups; g += nw) {
+        Ext a; a.v = INFINITY; a.idx = 0x7fffffff;
+        Ext b; b.v = -INFINITY; b.idx = 0x7fffffff;
+        for (int m = lane; m < members; m += 32) {
+            int th = (m / cols) * CV + g * cols + (m % cols);
+            a = ext_min(a, s_mn[th]); b = ext_max(b, s_mx[th]);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) { a = ext_min(a, shfl_ext(a, o)); b = ext_max(b, shfl_ext(b, o)); }
+        if (lane == 0) { g_mn[g] = a; g_mx[g] = b; }
+    }
+    __syncthreads();
+}
+
+template <int V>
+__global__ void __launch_bounds__(512)
+ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
+               const float *__restrict__ x, const float *__restrict__ v,
+               const float *__restrict__ gamma, const float *__restrict__ beta, int64_t pstride,
+               int B, float *__restrict__ y, float *__restrict__ gmin, float *__restrict__ gmax,
+               int32_t *__restrict__ argmin, int32_t *__restrict__ argmax) {
+    extern __shared__ unsigned char smem_raw[];
+    const int T = blockDim.x, t = threadIdx.x;
+    Ext *s_mn = reinterpret_cast<Ext *>(smem_raw);
+    Ext *s_mx = s_mn + T;
+    Ext *g_mn = s_mx + T;
+    Ext *g_mx = g_mn + groups;
+    const int CV = C / V, cpg = C / groups;
+    const int col = t % CV, row0 = t / CV, rstep = T / CV;
+    const int c0 = col * V, grp = c0 / cpg;
+    const int64_t sample = blockIdx.x;         // node*B + b
+    const int node = (int)(sample / B);
+    const float *xs = x + sample * (int64_t)HW * C;
+    float *ys = y + sample * (int64_t)HW * C;
+
+    Ext mn, mx; mn.v = INFINITY; mn.idx = 0x7fffffff; mx.v = -INFINITY; mx.idx = 0x7fffffff;
+    for (int p = row0; p < HW; p += rstep) {
+        float xv[V];
+        VecLoad<V>::ld(xs + (int64_t)p * C + c0, xv);
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            int idx = p * C + c0 + k;
+            if (xv[k] > mx.v) { mx.v = xv[k]; mx.idx = idx; }
+            if (xv[k] < mn.v) { mn.v = xv[k]; mn.idx = idx; }
+        }
+    }
+    reduce_groups<V>(mn, mx, s_mn, s_mx, g_mn, g_mx, CV, cpg, groups);
+    if (t < groups) {
+        int64_t sg = sample * groups + t;
+        gmin[sg] = g_mn[t].v; gmax[sg] = g_mx[t].v; argmin[sg] = g_mn[t].idx; argmax[sg] = g_mx[t].idx;
+    }
+    const float rng = __fsub_rn(g_mx[grp].v, g_mn[grp].v);
+    const float D = __fadd_rn(__fmul_rn(Cst, rng), eps);
+    const float invD = __fdiv_rn(1.f, D);
+    float vc[V], gc[V], bc[V];
+#pragma unroll
+    for (int k = 0; k < V; ++k) {
+        vc[k] = v[(int64_t)node * pstride + c0 + k];
+        gc[k] = gamma[(int64_t)node * pstride + c0 + k];
+        bc[k] = beta[(int64_t)node * pstride + c0 + k];
+    }
+    for (int p = row0; p < HW; p += rstep) {
+        float xv[V], yv[V];
+        VecLoad<V>::ld(xs + (int64_t)p * C + c0, xv);
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            float u = __fmul_rn(vc[k], xv[k]);
+            float m = __fmul_rn(xv[k], hsig(u));
+            yv[k] = __fadd_rn(__fmul_rn(__fmul_rn(gc[k], m), invD), bc[k]);
+        }
+        VecLoad<V>::st(ys + (int64_t)p * C + c0, yv);
+    }
+}
+
+template <int V>
+__global__ void __launch_bounds__(512)
+ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
+               const float *__restrict__ dy, const float *__restrict__ x,
+               const float *__restrict__ v, const float *__restrict__ gamma, int64_t pstride, int B,
+               const float *__restrict__ gmin, const float *__restrict__ gmax,
+               const int32_t *__restrict__ argmin, const int32_t *__restrict__ argmax,
+               float *__restrict__ dx, double *__restrict__ acc /*[nodes][3][C]*/) {
+    extern __shared__ unsigned char smem_raw[];
+    const int T = blockDim.x, t = threadIdx.x;
+    double *s_ch = reinterpret_cast<double *>(smem_raw);      // [3][C]
+    double *s_S = s_ch + 3 * C;                               // [T]
+    double *g_S = s_S + T;                                    // [groups]
+    const int CV = C / V, cpg = C / groups;
+    const int col = t % CV, row0 = t / CV, rstep = T / CV;
+    const int c0 = col * V, grp = c0 / cpg;
+    const int64_t sample = blockIdx.x;
+    const int node = (int)(sample / B);
+    const float *xs = x + sample * (int64_t)HW * C;
+    const float *dys = dy + sample * (int64_t)HW * C;
+    float *dxs = dx + sample * (int64_t)HW * C;
+    for (int i = t; i < 3 * C; i += T) s_ch[i] = 0.0;
+
+    const int64_t sg = sample * groups + grp;
+    const float rng = __fsub_rn(gmax[sg], gmin[sg]);
+    const float D = __fadd_rn(__fmul_rn(Cst, rng), eps);
+    const float invD = __fdiv_rn(1.f, D);
+    const float sixth = __fdiv_rn(1.f, 6.f);
+    float vc[V], gc[V];
+#pragma unroll
+    for (int k = 0; k < V; ++k) {
+        vc[k] = v[(int64_t)node * pstride + c0 + k];
+        gc[k] = gamma[(int64_t)node * pstride + c0 + k];
+    }
+    double S = 0.0, ab[V], ag[V], av[V];
+#pragma unroll
+    for (int k = 0; k < V; ++k) { ab[k] = 0.0; ag[k] = 0.0; av[k] = 0.0; }
+    for (int p = row0; p < HW; p += rstep) {
+        float xv[V], dv_[V];
+        VecLoad<V>::ld(xs + (int64_t)p * C + c0, xv);
+        VecLoad<V>::ld(dys + (int64_t)p * C + c0, dv_);
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            float u = __fmul_rn(vc[k], xv[k]);
+            float hs = hsig(u);
+            float hp = (u > -3.f && u < 3.f) ? sixth : 0.f;
+            float m = __fmul_rn(xv[k], hs);
+            float tt = __fmul_rn(dv_[k], gc[k]);
+            S += (double)__fmul_rn(tt, m);
+            ab[k] += (double)dv_[k];
+            ag[k] += (double)__fmul_rn(dv_[k], __fmul_rn(m, invD));
+            av[k] += (double)__fmul_rn(__fmul_rn(__fmul_rn(tt, __fmul_rn(xv[k], xv[k])), hp), invD);
+        }
+    }
+    __syncthreads();   // s_ch zeroed
+#pragma unroll
+    for (int k = 0; k < V; ++k) {
+        atomicAdd(&s_ch[0 * C + c0 + k], av[k]);
+        atomicAdd(&s_ch[1 * C + c0 + k], ag[k]);
+        atomicAdd(&s_ch[2 * C + c0 + k], ab[k]);
+    }
+    s_S[t] = S;
+    __syncthreads();
+    {   // fixed-order group sums: one warp per group, lanes stride the members
+        const int lane = t & 31, warp = t >> 5, nw = T >> 5;
+        const int cols = cpg / V, rows = T / CV, members = cols * rows;
+        for (int g = warp; g < groups; g += nw) {
+            double a = 0.0;
+            for (int m = lane; m < members; m += 32) a += s_S[(m / cols) * CV + g * cols + (m % cols)];
+            a = warp_sum(a);
+            if (lane == 0) g_S[g] = a;
+        }
+    }
+    for (int i = t; i < 3 * C; i += T) atomicAdd(&acc[(int64_t)node * 3 * C + i], s_ch[i]);
+    __syncthreads();
+    const int amx = argmax[sg], amn = argmin[sg];
+    float coef = __fmul_rn(Cst, (float)g_S[grp]);
+    coef = __fmul_rn(coef, invD);
+    coef = __fmul_rn(coef, invD);
+    if (amx == amn) coef = 0.f;
+    for (int p = row0; p < HW; p += rstep) {
+        float xv[V], dv_[V], o[V];
+        VecLoad<V>::ld(xs + (int64_t)p * C + c0, xv);
+        VecLoad<V>::ld(dys + (int64_t)p * C + c0, dv_);
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            float u = __fmul_rn(vc[k], xv[k]);
+            float hs = hsig(u);
+            float hp = (u > -3.f && u < 3.f) ? sixth : 0.f;
+            float tt = __fmul_rn(dv_[k], gc[k]);
+            float inner = __fadd_rn(hs, __fmul_rn(u, hp));
+            float r = __fmul_rn(__fmul_rn(tt, inner), invD);
+            int idx = p * C + c0 + k;
+            if (idx == amx) r = __fsub_rn(r, coef);
+            if (idx == amn) r = __fadd_rn(r, coef);
+            o[k] = r;
+        }
+        VecLoad<V>::st(dxs + (int64_t)p * C + c0, o);
+    }
+}
+
+__global__ void ren_bwd_finalize(const double *__restrict__ acc, int nodes, int C,
+                                 float *__restrict__ dv, float *__restrict__ dgamma,
+                                 float *__restrict__ dbeta, int64_t gstride) {
+    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= nodes * C) return;
+    int node = i / C, c = i % C;
+    const double *a = acc + (int64_t)node * 3 * C;
+    dv[(int64_t)node * gstride + c] = (float)a[c];
+    dgamma[(int64_t)node * gstride + c] = (float)a[C + c];
+    dbeta[(int64_t)node * gstride + c] = (float)a[2 * C + c];
+}
+
+struct RenPlan { int V, threads; };
+
+static bool plan(int C, int groups, bool aligned16, RenPlan *pl) {
+    const int cpg = C / groups;
+    int V = (aligned16 && C % 4 == 0 && cpg % 4 == 0) ? 4 : 1;
+    int CV = C / V;
+    if (CV > 512) return false;
+    pl->V = V;
+    pl->threads = CV * (512 / CV);
+    if (pl->threads % 32) {                      // keep whole warps: pad down to a multiple of lcm
+        int th = pl->threads;
+        while (th > 0 && (th % 32 || th % CV)) th -= CV;
+        if (th <= 0) return false;
+        pl->threads = th;
+    }
+    return true;
+}
+
+static float ren_const(int cpg) { return (float)(1.0 / sqrt(2.0 * log((double)cpg))); }
+
+}  // namespace lpdt
+
+using namespace lpdt;
+
+extern "C" lpdt_status lpdt_range_evonorm_fwd(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C,
+                                              int32_t groups, float eps, const float *x, const float *v,
+                                              const float *gamma, const float *beta, int64_t pstride,
+                                              float *y, float *gmin, float *gmax, int32_t *argmin,
+                                              int32_t *argmax, void *stream) {
+    LPDT_CHECK_ARG(nodes >= 0 && B >= 0 && H > 0 && W > 0 && C > 0 && groups > 0);
+    LPDT_CHECK_ARG(C % groups == 0 && C / groups >= 2);
+    if (nodes == 0 || B == 0) return LPDT_OK;
+    LPDT_CHECK_ARG(x && v && gamma && beta && y && gmin && gmax && argmin && argmax);
+    LPDT_CHECK_ARG(pstride >= C || nodes == 1);
+    if ((int64_t)H * W * C > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
+    RenPlan pl;
+    if (!plan(C, groups, aligned(x, 16) && aligned(y, 16), &pl)) return LPDT_ERR_UNSUPPORTED;
+    size_t smem = (size_t)(2 * pl.threads + 2 * groups) * sizeof(Ext);
+    if (smem > 48 * 1024) return LPDT_ERR_UNSUPPORTED;
+    const float Cst = ren_const(C / groups);
+    dim3 grid((unsigned)((int64_t)nodes * B));
+    if (pl.V == 4)
+        ren_fwd_kernel<4><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax);
+    else
+        ren_fwd_kernel<1><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax);
+    LPDT_LAUNCH_CHECK();
+    return LPDT_OK;
+}
+
+extern "C" size_t lpdt_range_evonorm_bwd_workspace_size(int32_t nodes, int32_t C) {
+    return align_up((size_t)(nodes > 0 ? nodes : 1) * 3 * (size_t)(C > 0 ? C : 1) * sizeof(double), 256);
+}
+
+extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C,
+                                              int32_t groups, float eps, const float *dy, const float *x,
+                                              const float *v, const float *gamma, int64_t pstride,
+                                              const float *gmin, const float *gmax,
+                                              const int32_t *argmin, const int32_t *argmax,
+                                              float *dx, float *dv, float *dgamma, float *dbeta,
+                                              int64_t gstride, void *ws, size_t ws_bytes, void *stream) {
+    LPDT_CHECK_ARG(nodes >= 0 && B >= 0 && H > 0 && W > 0 && C > 0 && groups > 0);
+    LPDT_CHECK_ARG(C % groups == 0 && C / groups >= 2);
+    if (nodes == 0 || B == 0) return LPDT_OK;
+    LPDT_CHECK_ARG(dy && x && v && gamma && gmin && gmax && argmin && argmax && dx && dv && dgamma && dbeta);
+    LPDT_CHECK_ARG((pstride >= C && gstride >= C) || nodes == 1);
+    if ((int64_t)H * W * C > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < lpdt_range_evonorm_bwd_workspace_size(nodes, C) || !aligned(ws, 8))
+        return LPDT_ERR_WORKSPACE;
+    RenPlan pl;
+    if (!plan(C, groups, aligned(x, 16) && aligned(dy, 16) && aligned(dx, 16), &pl)) return LPDT_ERR_UNSUPPORTED;
+    size_t smem = (size_t)(3 * C + pl.threads + groups) * sizeof(double);
+    if (smem > 48 * 1024) return LPDT_ERR_UNSUPPORTED;
+    cudaStream_t st = as_stream(stream);
+    double *acc = (double *)ws;
+    LPDT_CUDA(cudaMemsetAsync(acc, 0, (size_t)nodes * 3 * C * sizeof(double), st));
+    const float Cst = ren_const(C / groups);
+    dim3 grid((unsigned)((int64_t)nodes * B));
+    if (pl.V == 4)
+        ren_bwd_kernel<4><<<grid, pl.threads, smem, st>>>(H * W, C, groups, eps, Cst, dy, x, v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc);
+    else
+        ren_bwd_kernel<1><<<grid, pl.threads, smem, st>>>(H * W, C, groups, eps, Cst, dy, x, v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc);
+    LPDT_LAUNCH_CHECK();
+    ren_bwd_finalize<<<(nodes * C + 255) / 256, 256, 0, st>>>(acc, nodes, C, dv, dgamma, dbeta, gstride);
+    LPDT_LAUNCH_CHECK();
+    return LPDT_OK;
+}

@@ -1,0 +1,248 @@
+"""One whole 8-bit training step of all simulated nodes, as a fixed sequence of
+lpdt C-ABI calls on preallocated device buffers.
+
+TrainStep walks a network op list (see `workloads`) forward and backward:
+every conv/linear quantizes its input and weights per node, runs the int8
+contraction and dequantizes; Range-EvoNorm follows in fp32; backward quantizes
+each incoming layer gradient once and feeds both adjoint contractions, weight
+gradients staying fp32; then the SGD half-step and the CHOCO gossip mix
+(Section 3 and Algorithms 1 and 3 of the paper).  Python only orders the calls
+and owns the buffers; all arithmetic runs in the CUDA library.
+"""
+import torch
+
+from . import api
+
+
+class TrainStep:
+    def __init__(self, ops, d, nodes, batch, in_shape, ren_eps=1e-5, lr=0.1, gamma=1.0,
+                 seg_offsets=None, seg_k=None, has_labels=True, grad_rounding=0, seed=0,
+                 quantize_wgrad=False, input_grad=False, device="cuda"):
+        if not torch.cuda.is_available():
+            raise RuntimeError("TrainStep needs a CUDA device; there is no CPU path")
+        self.ops, self.d, self.N, self.B = ops, d, nodes, batch
+        self.eps, self.lr, self.gamma = float(ren_eps), float(lr), float(gamma)
+        self.seg_offsets = [0, d] if seg_offsets is None else [int(v) for v in seg_offsets]
+        self.seg_k = [d] if seg_k is None else [int(v) for v in seg_k]
+        self.grad_rounding, self.seed = grad_rounding, seed
+        self.quantize_wgrad, self.input_grad = quantize_wgrad, input_grad
+        dev = torch.device(device)
+        N, B = nodes, batch
+        f32 = dict(dtype=torch.float32, device=dev)
+        i8 = dict(dtype=torch.int8, device=dev)
+        i32 = dict(dtype=torch.int32, device=dev)
+        self.params = torch.zeros(N, d, **f32)
+        self.grads = torch.zeros(N, d, **f32)
+        self.x_half = torch.zeros(N, d, **f32)
+        self.x_hat = torch.zeros(N, d, **f32)
+        self.x_out = torch.zeros(N, d, **f32)
+        self.Wmix = torch.zeros(N, N, **f32)
+        self.x = torch.zeros((N, B) + tuple(in_shape), **f32)
+        self.labels = torch.zeros(N, B, **i32) if has_labels else None
+        self.loss = torch.zeros(N, **f32)
+        self.dev_status = torch.zeros(1, **i32)
+        ws_bytes = max(api.lpdt_quantize_workspace_size(N),
+                       api.lpdt_gossip_mix_workspace_size(N, d, len(self.seg_k)))
+        self.buf = []
+        shape = tuple(in_shape)
+        for op in ops:
+            k = op["op"]
+            b = {}
+            if k in ("conv", "linear"):
+                if k == "linear":
+                    H = W = 1; R = S = 1; stride = 1; pad = 0
+                else:
+                    H, W, R, S, stride, pad = op["H"], op["W"], op["R"], op["S"], op["stride"], op["pad"]
+                desc = api.conv_desc(N, B, H, W, op["cin"], op["cout"], R, S, stride, pad)
+                Ho = (H + 2 * pad - R) // stride + 1
+                Wo = (W + 2 * pad - S) // stride + 1
+                b.update(desc=desc, in_shape=(H, W, op["cin"]),
+                         qA=torch.empty(N, B, H, W, op["cin"], **i8), sA=torch.empty(N, **f32),
+                         qW=torch.empty(N, op["cout"], R, S, op["cin"], **i8), sW=torch.empty(N, **f32),
+                         out=torch.empty(N, B, Ho, Wo, op["cout"], **f32),
+                         E=torch.empty(N, B, Ho, Wo, op["cout"], **i8), sE=torch.empty(N, **f32),
+                         dx=torch.empty(N, B, H, W, op["cin"], **f32),
+                         wn=op["cout"] * R * S * op["cin"])
+                if quantize_wgrad:
+                    b.update(gq=torch.empty(N, b["wn"], **i8), gs=torch.empty(N, **f32),
+                             gw=torch.empty(N, b["wn"], **f32))
+                for which in (0, 1, 2):
+                    ws_bytes = max(ws_bytes, api.lpdt_qconv_workspace_size(desc, which))
+                shape = (Ho, Wo, op["cout"])
+            elif k == "ren":
+                H, W, Cc, G = op["H"], op["W"], op["C"], op["groups"]
+                b.update(out=torch.empty(N, B, H, W, Cc, **f32), dx=torch.empty(N, B, H, W, Cc, **f32),
+                         gmin=torch.empty(N, B, G, **f32), gmax=torch.empty(N, B, G, **f32),
+                         amin=torch.empty(N, B, G, **i32), amax=torch.empty(N, B, G, **i32))
+                ws_bytes = max(ws_bytes, api.lpdt_range_evonorm_bwd_workspace_size(N, Cc))
+            elif k == "add":
+                Ho, Wo = (op["H"] + op["stride"] - 1) // op["stride"], (op["W"] + op["stride"] - 1) // op["stride"]
+                b.update(out=torch.empty(N, B, Ho, Wo, op["C"], **f32))
+            elif k == "save":
+                b.update(dx=torch.empty(N, B, op["H"], op["W"], op["C"], **f32))
+            elif k == "maxpool":
+                H, W, Cc = op["H"], op["W"], op["C"]
+                b.update(out=torch.empty(N, B, H // 2, W // 2, Cc, **f32),
+                         idx=torch.empty(N, B, H // 2, W // 2, Cc, **i8),
+                         dx=torch.empty(N, B, H, W, Cc, **f32))
+                shape = (H // 2, W // 2, Cc)
+            elif k == "avgpool":
+                b.update(out=torch.empty(N, B, 1, 1, op["C"], **f32),
+                         dx=torch.empty(N, B, op["H"], op["W"], op["C"], **f32))
+                shape = (1, 1, op["C"])
+            else:
+                raise ValueError(k)
+            self.buf.append(b)
+        self.out_shape = shape
+        self.dy = torch.zeros((N, B) + tuple(shape), **f32)      # upstream gradient / dlogits
+        self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+
+    # ---- host -> device ------------------------------------------------------------
+    def load(self, wl):
+        self.params.copy_(torch.from_numpy(wl["params"]))
+        self.x_hat.copy_(torch.from_numpy(wl["x_hat"]))
+        self.Wmix.copy_(torch.from_numpy(wl["Wmix"]))
+        self.x.copy_(torch.from_numpy(wl["x"]))
+        if "labels" in wl and self.labels is not None:
+            self.labels.copy_(torch.from_numpy(wl["labels"]))
+        if "dy" in wl:
+            self.dy.copy_(torch.from_numpy(wl["dy"]))
+
+    @classmethod
+    def from_workload(cls, wl, **kw):
+        st = cls(wl["ops"], wl["d"], wl["nodes"], wl["batch"], wl["x"].shape[2:], wl["ren_eps"], wl["lr"],
+                 wl["gamma"], wl["seg_offsets"], wl["seg_k"], has_labels=("labels" in wl),
+                 input_grad=("dy" in wl), **kw)
+        st.load(wl)
+        return st
+
+    # ---- the step --------------------------------------------------------------------
+    def _p(self, off):
+        return self.params[:, off:]
+
+    def _g(self, off):
+        return self.grads[:, off:]
+
+    def forward(self):
+        N, B, d = self.N, self.B, self.d
+        cur = self.x
+        saved = []
+        for op, b in zip(self.ops, self.buf):
+            k = op["op"]
+            if k in ("conv", "linear"):
+                n_in = cur.numel() // N
+                api.lpdt_quantize(cur, N, n_in, n_in, b["qA"], b["sA"], self.ws)
+                api.lpdt_quantize(self._p(op["w_off"]), N, b["wn"], d, b["qW"], b["sW"], self.ws)
+                bias = self._p(op["b_off"]) if k == "linear" else None
+                api.lpdt_qconv_fwd(b["desc"], b["qA"], b["sA"], b["qW"], b["sW"], Y=b["out"], bias=bias,
+                                   bias_node_stride=d, ws=self.ws, dev_status=self.dev_status)
+                cur = b["out"]
+            elif k == "ren":
+                Cc = op["C"]
+                b["x"] = cur
+                api.lpdt_range_evonorm_fwd(N, B, op["H"], op["W"], Cc, op["groups"], self.eps, cur,
+                                           self._p(op["p_off"]), self._p(op["p_off"] + Cc),
+                                           self._p(op["p_off"] + 2 * Cc), d, b["out"], b["gmin"], b["gmax"],
+                                           b["amin"], b["amax"])
+                cur = b["out"]
+            elif k == "save":
+                saved.append(cur)
+            elif k == "add":
+                a = saved.pop()
+                api.lpdt_residual_add(N, B, op["H"], op["W"], op["Ca"], op["C"], op["stride"], op["ch_off"],
+                                      cur, a, b["out"])
+                cur = b["out"]
+            elif k == "maxpool":
+                api.lpdt_maxpool2x2(N, B, op["H"], op["W"], op["C"], cur, b["out"], b["idx"])
+                cur = b["out"]
+            elif k == "avgpool":
+                api.lpdt_avgpool(N, B, op["H"] * op["W"], op["C"], cur, b["out"])
+                cur = b["out"]
+        self.out = cur
+        return cur
+
+    def backward(self):
+        N, B, d = self.N, self.B, self.d
+        if self.labels is not None:
+            K = self.out.numel() // (N * B)
+            api.lpdt_softmax_ce(N, B, K, self.out, self.labels, self.loss, self.dy)
+        g = self.dy
+        sc = []
+        ctr = 0
+        for li in range(len(self.ops) - 1, -1, -1):
+            op, b = self.ops[li], self.buf[li]
+            k = op["op"]
+            if k in ("conv", "linear"):
+                if k == "linear":
+                    api.lpdt_colsum(N, B, op["cout"], g, self._g(op["b_off"]), d)
+                n_out = g.numel() // N
+                api.lpdt_quantize(g, N, n_out, n_out, b["E"], b["sE"], self.ws, rounding=self.grad_rounding,
+                                  seed=self.seed, ctr_offset=ctr)
+                ctr += 1
+                if self.quantize_wgrad:
+                    api.lpdt_qconv_bwd_weight(b["desc"], b["E"], b["sE"], b["qA"], b["sA"], dW=b["gw"],
+                                              dw_node_stride=b["wn"], ws=self.ws, dev_status=self.dev_status)
+                    api.lpdt_quantize(b["gw"], N, b["wn"], b["wn"], b["gq"], b["gs"], self.ws)
+                    api.lpdt_dequantize(b["gq"], N, b["wn"], b["gs"], self._g(op["w_off"]), d)
+                else:
+                    api.lpdt_qconv_bwd_weight(b["desc"], b["E"], b["sE"], b["qA"], b["sA"],
+                                              dW=self._g(op["w_off"]), dw_node_stride=d, ws=self.ws,
+                                              dev_status=self.dev_status)
+                if li > 0 or self.input_grad:
+                    api.lpdt_qconv_bwd_data(b["desc"], b["E"], b["sE"], b["qW"], b["sW"], dA=b["dx"],
+                                            ws=self.ws, dev_status=self.dev_status)
+                    g = b["dx"]
+                else:
+                    g = None
+            elif k == "ren":
+                Cc = op["C"]
+                api.lpdt_range_evonorm_bwd(N, B, op["H"], op["W"], Cc, op["groups"], self.eps, g, b["x"],
+                                           self._p(op["p_off"]), self._p(op["p_off"] + Cc), d, b["gmin"],
+                                           b["gmax"], b["amin"], b["amax"], b["dx"], self._g(op["p_off"]),
+                                           self._g(op["p_off"] + Cc), self._g(op["p_off"] + 2 * Cc), d, self.ws)
+                g = b["dx"]
+            elif k == "add":
+                sc.append((g, op))
+            elif k == "save":
+                dy_sc, aop = sc.pop()
+                api.lpdt_residual_add_bwd(N, B, aop["H"], aop["W"], aop["Ca"], aop["C"], aop["stride"],
+                                          aop["ch_off"], dy_sc, g, b["dx"])
+                g = b["dx"]
+            elif k == "maxpool":
+                api.lpdt_maxpool2x2_bwd(N, B, op["H"], op["W"], op["C"], g, b["idx"], b["dx"])
+                g = b["dx"]
+            elif k == "avgpool":
+                api.lpdt_avgpool_bwd(N, B, op["H"] * op["W"], op["C"], g, b["dx"])
+                g = b["dx"]
+        self.input_grad_out = g
+        return g
+
+    def update(self):
+        N, d = self.N, self.d
+        api.lpdt_sgd_update(N * d, self.params, self.grads, self.lr, self.x_half)
+        api.lpdt_gossip_mix(N, d, self.x_half, self.x_hat, self.x_out, self.Wmix, self.gamma,
+                            self.seg_offsets, self.seg_k, self.ws, self.dev_status)
+
+    def run(self):
+        self.forward()
+        self.backward()
+        self.update()
+
+    def launches_per_step(self):
+        """Kernel launches of one run(): counted from the op list (memsets excluded)."""
+        n = 0
+        for op in self.ops:
+            k = op["op"]
+            if k in ("conv", "linear"):
+                first = op is self.ops[0] and not self.input_grad
+                n += 2 * 2 + 1            # two quantizes (2 kernels each) + fwd
+                n += 2                    # quantize E
+                n += 2                    # bwd-weight + dequant (generic path upper bound)
+                n += 0 if first else 2    # transpose + bwd-data
+                n += 1 if k == "linear" else 0
+            elif k == "ren":
+                n += 1 + 2
+            elif k in ("add", "maxpool", "avgpool"):
+                n += 2
+        n += 1 if self.labels is not None else 0
+        return n + 1 + 2                  # sgd + select + mix

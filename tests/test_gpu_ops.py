@@ -1,0 +1,365 @@
+"""GPU parity: every lpdt entry point against the CPU oracle on the same seeded
+inputs, through the C ABI.  Integer results bit-exact; fp32 results within
+1e-5 relative / 1e-6 absolute."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2111_09389_b200 import api, workloads as wlmod
+
+pytestmark = pytest.mark.gpu
+
+RTOL, ATOL = 1e-5, 1e-6
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def close(got, want, rtol=RTOL, atol=ATOL):
+    got = got.cpu().numpy() if isinstance(got, torch.Tensor) else got
+    want = np.asarray(want, dtype=np.float64)
+    err = np.abs(got.astype(np.float64) - want)
+    ok = err <= atol + rtol * np.abs(want)
+    assert ok.all(), f"{(~ok).sum()} of {ok.size} outside tolerance, worst {err.max():.3e}"
+
+
+def ws_bytes(n):
+    return torch.empty(max(int(n), 256), dtype=torch.uint8, device="cuda")
+
+
+# ------------------------------------------------------------------ quantizer
+@pytest.mark.parametrize("nodes,n", [(1, 1), (3, 7), (4, 4096), (2, 100003), (16, 98304), (1, 1 << 22)])
+@pytest.mark.parametrize("rounding", [0, 1])
+def test_quantize_sym(nodes, n, rounding):
+    rng = np.random.default_rng(n + rounding)
+    x = (rng.standard_normal((nodes, n)) * rng.uniform(0.01, 100, (nodes, 1))).astype(np.float32)
+    q_ref, s_ref = oracle.quantize_sym_s8(x, rounding, seed=(9 << 32) | 77, ctr_offset=3)
+    xd = dev(x)
+    q = torch.empty(nodes, n, dtype=torch.int8, device="cuda")
+    s = torch.empty(nodes, dtype=torch.float32, device="cuda")
+    ws = ws_bytes(api.lpdt_quantize_workspace_size(nodes))
+    api.lpdt_quantize(xd, nodes, n, n, q, s, ws, mode=0, rounding=rounding, seed=(9 << 32) | 77, ctr_offset=3)
+    assert np.array_equal(s.cpu().numpy(), s_ref)
+    assert np.array_equal(q.cpu().numpy(), q_ref)
+    y = torch.empty(nodes, n, dtype=torch.float32, device="cuda")
+    api.lpdt_dequantize(q, nodes, n, s, y)
+    assert np.array_equal(y.cpu().numpy(), oracle.dequantize(q_ref, s_ref))
+
+
+def test_quantize_strided_rows_zero_tensor_and_ties():
+    # rows inside a wider flat vector (odd stride -> scalar path), an all-zero node, exact ties
+    rng = np.random.default_rng(0)
+    nodes, n, stride = 3, 432, 1001
+    flat = rng.standard_normal((nodes, stride)).astype(np.float32)
+    flat[1, 5:5 + n] = 0.0
+    flat[2, 5:5 + n] = np.round(flat[2, 5:5 + n] * 4) / 8      # many .5 ties once scaled
+    flat[2, 5] = 127.0 / 2
+    q_ref, s_ref = oracle.quantize_sym_s8(flat[:, 5:5 + n])
+    fd = dev(flat)
+    q = torch.empty(nodes, n, dtype=torch.int8, device="cuda")
+    s = torch.empty(nodes, dtype=torch.float32, device="cuda")
+    api.lpdt_quantize(fd[:, 5:], nodes, n, stride, q, s, ws_bytes(256))
+    assert np.array_equal(q.cpu().numpy(), q_ref) and np.array_equal(s.cpu().numpy(), s_ref)
+    assert s_ref[1] == 1.0 and not q_ref[1].any()
+
+
+@pytest.mark.parametrize("nodes,n", [(2, 1001), (3, 65536)])
+def test_quantize_affine(nodes, n):
+    rng = np.random.default_rng(n)
+    x = rng.uniform(-1, 3, (nodes, n)).astype(np.float32)
+    x[-1] = np.abs(x[-1]) + 0.5                                  # one-sided node
+    q_ref, s_ref, z_ref = oracle.quantize_affine_u8(x)
+    q = torch.empty(nodes, n, dtype=torch.int8, device="cuda")
+    s = torch.empty(nodes, dtype=torch.float32, device="cuda")
+    zp = torch.empty(nodes, dtype=torch.int32, device="cuda")
+    api.lpdt_quantize(dev(x), nodes, n, n, q, s, ws_bytes(256), mode=1, zero_point=zp)
+    assert np.array_equal(q.cpu().numpy().view(np.uint8), q_ref)
+    assert np.array_equal(s.cpu().numpy(), s_ref) and np.array_equal(zp.cpu().numpy(), z_ref)
+    y = torch.empty(nodes, n, dtype=torch.float32, device="cuda")
+    api.lpdt_dequantize(q, nodes, n, s, y, zero_point=zp)
+    assert np.array_equal(y.cpu().numpy(), oracle.dequantize(q_ref, s_ref, z_ref))
+
+
+def test_quantize_argument_errors():
+    x = torch.zeros(8, device="cuda")
+    q = torch.zeros(8, dtype=torch.int8, device="cuda")
+    s = torch.zeros(1, device="cuda")
+    with pytest.raises(api.LpdtError) as e:
+        api.lpdt_quantize(x, 1, 8, 8, q, s, None)
+    assert e.value.code == 3
+    with pytest.raises(api.LpdtError) as e:
+        api.lpdt_quantize(None, 1, 8, 8, q, s, ws_bytes(256))
+    assert e.value.code == 1
+    with pytest.raises(api.LpdtError) as e:
+        api.lpdt_quantize(x, 1, 8, 8, q, s, ws_bytes(256), mode=1)     # affine without zero_point
+    assert e.value.code == 1
+    api.lpdt_quantize(x, 0, 8, 8, q, s, None)                          # empty: no-op
+
+
+# ------------------------------------------------------------------ contractions
+CONV_CASES = [
+    # nodes, B, H, W, Cin, Cout, R, S, stride, pad
+    (4, 8, 16, 16, 16, 16, 3, 3, 1, 1),      # the single-layer workload
+    (2, 3, 32, 32, 3, 16, 3, 3, 1, 1),       # first layer of the networks
+    (2, 2, 16, 16, 16, 32, 3, 3, 2, 1),      # strided stage transition
+    (1, 2, 9, 7, 5, 6, 3, 3, 1, 1),          # ragged everything
+    (2, 4, 8, 8, 64, 64, 3, 3, 1, 1),
+    (1, 1, 12, 12, 32, 48, 1, 1, 1, 0),      # 1x1
+    (3, 32, 1, 1, 64, 10, 1, 1, 1, 0),       # classifier
+    (1, 5, 4, 4, 8, 8, 3, 3, 1, 0),          # no padding
+    (1, 2, 40, 24, 128, 64, 3, 3, 1, 1),
+]
+
+
+def _conv_inputs(case, seed=0):
+    nodes, B, H, W, Cin, Cout, R, S, stride, pad = case
+    rng = np.random.default_rng(seed)
+    A = wlmod.random_s8(rng, (nodes, B, H, W, Cin))
+    Wq = wlmod.random_s8(rng, (nodes, Cout, R, S, Cin))
+    Ho, Wo = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - S) // stride + 1
+    E = wlmod.random_s8(rng, (nodes, B, Ho, Wo, Cout))
+    s1 = rng.uniform(0.001, 0.1, nodes).astype(np.float32)
+    s2 = rng.uniform(0.001, 0.1, nodes).astype(np.float32)
+    return A, Wq, E, s1, s2
+
+
+@pytest.mark.parametrize("case", CONV_CASES)
+def test_qconv_all_three(case):
+    nodes, B, H, W, Cin, Cout, R, S, stride, pad = case
+    A, Wq, E, s1, s2 = _conv_inputs(case)
+    desc = api.conv_desc(*case)
+    ws = ws_bytes(max(api.lpdt_qconv_workspace_size(desc, w) for w in (0, 1, 2)))
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    Ad, Wd, Ed, s1d, s2d = dev(A), dev(Wq), dev(E), dev(s1), dev(s2)
+    # forward, with bias living in a strided parameter vector
+    acc_ref, ovf = oracle.qconv_fwd(A, Wq, stride, pad)
+    assert ovf == 0
+    bias = np.random.default_rng(1).standard_normal((nodes, Cout + 3)).astype(np.float32)
+    Y = torch.empty(acc_ref.shape, dtype=torch.float32, device="cuda")
+    Yacc = torch.empty(acc_ref.shape, dtype=torch.int32, device="cuda")
+    api.lpdt_qconv_fwd(desc, Ad, s1d, Wd, s2d, Y=Y, Yacc=Yacc, bias=dev(bias)[:, 3:], bias_node_stride=Cout + 3,
+                       ws=ws, dev_status=status)
+    assert np.array_equal(Yacc.cpu().numpy(), acc_ref)
+    assert np.array_equal(Y.cpu().numpy(), oracle.dequant_acc(acc_ref, s1, s2, bias[:, 3:]))
+    # backward data
+    dA_ref, _ = oracle.qconv_bwd_data(E, Wq, H, W, stride, pad)
+    dA = torch.empty(dA_ref.shape, dtype=torch.float32, device="cuda")
+    dAacc = torch.empty(dA_ref.shape, dtype=torch.int32, device="cuda")
+    api.lpdt_qconv_bwd_data(desc, Ed, s1d, Wd, s2d, dA=dA, dAacc=dAacc, ws=ws, dev_status=status)
+    assert np.array_equal(dAacc.cpu().numpy(), dA_ref)
+    assert np.array_equal(dA.cpu().numpy(), oracle.dequant_acc(dA_ref, s1, s2))
+    # backward weight, into a strided gradient vector
+    dW_ref, _ = oracle.qconv_bwd_weight(E, A, R, S, stride, pad)
+    wn = Cout * R * S * Cin
+    dW = torch.zeros(nodes, wn + 5, dtype=torch.float32, device="cuda")
+    dWacc = torch.empty(dW_ref.shape, dtype=torch.int32, device="cuda")
+    api.lpdt_qconv_bwd_weight(desc, Ed, s1d, Ad, s2d, dW=dW[:, 5:], dw_node_stride=wn + 5, dWacc=dWacc, ws=ws,
+                              dev_status=status)
+    assert np.array_equal(dWacc.cpu().numpy(), dW_ref)
+    assert np.array_equal(dW[:, 5:].cpu().numpy(), oracle.dequant_acc(dW_ref, s1, s2).reshape(nodes, wn))
+    assert float(dW[:, :5].abs().max()) == 0.0
+    # fp32-only outputs (workspace accumulators) give the same values
+    dW2 = torch.zeros(nodes, wn, dtype=torch.float32, device="cuda")
+    api.lpdt_qconv_bwd_weight(desc, Ed, s1d, Ad, s2d, dW=dW2, dw_node_stride=wn, ws=ws, dev_status=status)
+    assert torch.equal(dW2, dW[:, 5:])
+    assert int(status.item()) == 0
+
+
+def test_qconv_extreme_values_and_errors():
+    # all operands at +-127: the largest accumulators the shape can produce
+    case = (1, 2, 6, 6, 16, 16, 3, 3, 1, 1)
+    A = np.full((1, 2, 6, 6, 16), 127, np.int8); Wq = np.full((1, 16, 3, 3, 16), -127, np.int8)
+    desc = api.conv_desc(*case)
+    acc_ref, _ = oracle.qconv_fwd(A, Wq, 1, 1)
+    Yacc = torch.empty(acc_ref.shape, dtype=torch.int32, device="cuda")
+    api.lpdt_qconv_fwd(desc, dev(A), None, dev(Wq), None, Yacc=Yacc, ws=ws_bytes(256))
+    assert np.array_equal(Yacc.cpu().numpy(), acc_ref) and acc_ref.min() == -127 * 127 * 144
+    with pytest.raises(api.LpdtError) as e:
+        api.lpdt_qconv_fwd(desc, dev(A), None, dev(Wq), None, ws=ws_bytes(256))      # no output
+    assert e.value.code == 1
+    with pytest.raises(api.LpdtError) as e:
+        api.lpdt_qconv_bwd_data(desc, dev(A), None, dev(Wq), None, dAacc=Yacc, ws=None)
+    assert e.value.code == 3
+    bad = api.conv_desc(1, 1, 2, 2, 4, 4, 5, 5, 1, 0)                                 # kernel larger than image
+    with pytest.raises(api.LpdtError) as e:
+        api.lpdt_qconv_fwd(bad, dev(A), None, dev(Wq), None, Yacc=Yacc, ws=ws_bytes(256))
+    assert e.value.code == 1
+
+
+# ------------------------------------------------------------------ Range-EvoNorm
+REN_CASES = [(4, 8, 16, 16, 16, 4), (2, 3, 32, 32, 16, 2), (2, 2, 8, 8, 64, 8), (1, 3, 5, 7, 6, 3),
+             (1, 2, 4, 4, 12, 1), (2, 2, 32, 32, 64, 8), (1, 2, 2, 2, 512, 64), (1, 1, 1, 1, 8, 2)]
+
+
+def _ren_inputs(case, seed=0, ties=False):
+    nodes, B, H, W, C, groups = case
+    rng = np.random.default_rng(seed)
+    x = (2 * rng.standard_normal((nodes, B, H, W, C))).astype(np.float32)
+    if ties:
+        x = np.round(x * 2) / 2                # 8-bit-like grid: many tied extrema, hits u = +-3 exactly
+    pad = 7
+    P = rng.uniform(0.5, 1.5, (nodes, 3 * C + pad)).astype(np.float32)
+    P[:, 2 * C:3 * C] -= 1.0
+    if ties:
+        P[:, :C] = 1.0
+    dy = rng.standard_normal(x.shape).astype(np.float32)
+    return x, P, dy
+
+
+@pytest.mark.parametrize("case", REN_CASES)
+@pytest.mark.parametrize("ties", [False, True])
+def test_range_evonorm_fwd_bwd(case, ties):
+    nodes, B, H, W, C, groups = case
+    x, P, dy = _ren_inputs(case, ties=ties)
+    eps = 1e-5
+    v, g, b = P[:, :C], P[:, C:2 * C], P[:, 2 * C:3 * C]
+    y32, mn, mx, amn, amx = oracle.range_evonorm_fwd(x, v, g, b, groups, eps, "f32")
+    y64 = oracle.range_evonorm_fwd(x, v, g, b, groups, eps, "f64")[0]
+    xd, Pd = dev(x), dev(P)
+    stride = P.shape[1]
+    f = lambda *s: torch.empty(*s, dtype=torch.float32, device="cuda")
+    i = lambda *s: torch.empty(*s, dtype=torch.int32, device="cuda")
+    y, gmin, gmax, amin_, amax_ = f(*x.shape), f(nodes, B, groups), f(nodes, B, groups), i(nodes, B, groups), i(nodes, B, groups)
+    api.lpdt_range_evonorm_fwd(nodes, B, H, W, C, groups, eps, xd, Pd, Pd[:, C:], Pd[:, 2 * C:], stride, y, gmin, gmax,
+                               amin_, amax_)
+    assert np.array_equal(gmin.cpu().numpy(), mn) and np.array_equal(gmax.cpu().numpy(), mx)
+    assert np.array_equal(amin_.cpu().numpy(), amn) and np.array_equal(amax_.cpu().numpy(), amx)
+    assert np.array_equal(y.cpu().numpy(), y32)            # same fp32 operation sequence: bit-equal
+    close(y, y64)
+    dx32, dv32, dg32, db32 = oracle.range_evonorm_bwd(dy, x, v, g, mn, mx, amn, amx, groups, eps, "f32")
+    dx64, dv64, dg64, db64 = oracle.range_evonorm_bwd(dy, x, v, g, mn, mx, amn, amx, groups, eps, "f64")
+    G = torch.zeros(nodes, stride, dtype=torch.float32, device="cuda")
+    dx = f(*x.shape)
+    ws = ws_bytes(api.lpdt_range_evonorm_bwd_workspace_size(nodes, C))
+    api.lpdt_range_evonorm_bwd(nodes, B, H, W, C, groups, eps, dev(dy), xd, Pd, Pd[:, C:], stride, gmin, gmax, amin_, amax_,
+                               dx, G, G[:, C:], G[:, 2 * C:], stride, ws)
+    close(dx, dx32, 1e-6, 1e-7)
+    close(dx, dx64)
+    Gh = G.cpu().numpy()
+    scale = lambda r: 1e-6 * max(1.0, float(np.abs(r).max()))
+    close(Gh[:, :C], dv64, RTOL, scale(dv64))
+    close(Gh[:, C:2 * C], dg64, RTOL, scale(dg64))
+    close(Gh[:, 2 * C:3 * C], db64, RTOL, scale(db64))
+    assert not Gh[:, 3 * C:].any()
+
+
+def test_range_evonorm_errors():
+    t = torch.zeros(64, device="cuda"); ti = torch.zeros(64, dtype=torch.int32, device="cuda")
+    with pytest.raises(api.LpdtError) as e:      # one channel per group: the constant is infinite
+        api.lpdt_range_evonorm_fwd(1, 1, 2, 2, 4, 4, 1e-5, t, t, t, t, 4, t, t, t, ti, ti)
+    assert e.value.code == 1
+    with pytest.raises(api.LpdtError) as e:      # groups must divide C
+        api.lpdt_range_evonorm_fwd(1, 1, 2, 2, 6, 4, 1e-5, t, t, t, t, 6, t, t, t, ti, ti)
+    assert e.value.code == 1
+
+
+# ------------------------------------------------------------------ gossip
+def _gossip_case(nodes, d, seed, heavy=False):
+    rng = np.random.default_rng(seed)
+    xh = rng.standard_normal((nodes, d)).astype(np.float32)
+    resid = rng.standard_normal((nodes, d)) * (np.where(rng.random((nodes, d)) < 0.05, 1.0, 0.01) if heavy else 1.0)
+    xhat = (xh - resid).astype(np.float32)
+    return xh, xhat
+
+
+@pytest.mark.parametrize("nodes,d,segs", [
+    (4, 2736, None), (16, 10007, None), (8, 50000, [(0, 50000, 500)]), (40, 27041, [(0, 27041, 270)]),
+    (5, 3000, [(0, 1000, 10), (1000, 1001, 1), (1001, 3000, 1999)]), (3, 1000, [(0, 1000, 0)]),
+    (1, 777, [(0, 777, 5)]), (64, 300, [(0, 300, 3)]),
+])
+def test_gossip_mix(nodes, d, segs):
+    xh, xhat = _gossip_case(nodes, d, d, heavy=True)
+    W = wlmod.ring_matrix(nodes) if nodes >= 3 else np.full((nodes, nodes), 1.0 / nodes, np.float32)
+    so = [0, d] if segs is None else [s[0] for s in segs] + [d]
+    sk = [d] if segs is None else [s[2] for s in segs]
+    gamma = 1.0 if segs is None else 0.3
+    x_ref, xhat_ref, q_ref = oracle.gossip_mix(xh, xhat, W, gamma, so, sk)
+    xhd, xhatd = dev(xh), dev(xhat)
+    xo = torch.empty_like(xhd)
+    ws = ws_bytes(api.lpdt_gossip_mix_workspace_size(nodes, d, len(sk)))
+    api.lpdt_gossip_mix(nodes, d, xhd, xhatd, xo, dev(W), gamma, so, sk, ws)
+    assert np.array_equal(xhatd.cpu().numpy(), xhat_ref)          # selection + update: bit-exact
+    close(xo, x_ref)
+    # second call on the updated state (error feedback carried over)
+    x_ref2, xhat_ref2, _ = oracle.gossip_mix(x_ref, xhat_ref, W, gamma, so, sk)
+    xo2 = torch.empty_like(xhd)
+    api.lpdt_gossip_mix(nodes, d, dev(x_ref), xhatd, xo2, dev(W), gamma, so, sk, ws)
+    assert np.array_equal(xhatd.cpu().numpy(), xhat_ref2)
+    close(xo2, x_ref2)
+
+
+def test_gossip_topk_with_massive_ties_and_alias():
+    # magnitudes from a 4-value set: the tie cut decides almost every pick
+    nodes, d, k = 6, 9000, 1234
+    rng = np.random.default_rng(5)
+    xh = rng.choice(np.array([-2, -1, 1, 2, 0.5, -0.5], np.float32), size=(nodes, d))
+    xhat = np.zeros((nodes, d), np.float32)
+    W = wlmod.ring_matrix(nodes)
+    x_ref, xhat_ref, q_ref = oracle.gossip_mix(xh, xhat, W, 0.5, [0, d], [k])
+    assert all(np.count_nonzero(q_ref[i]) == k for i in range(nodes))
+    xhd, xhatd = dev(xh), dev(xhat)
+    ws = ws_bytes(api.lpdt_gossip_mix_workspace_size(nodes, d, 1))
+    api.lpdt_gossip_mix(nodes, d, xhd, xhatd, xhd, dev(W), 0.5, [0, d], [k], ws)   # x_out aliases x_half
+    assert np.array_equal(xhatd.cpu().numpy(), xhat_ref)
+    close(xhd, x_ref)
+
+
+def test_gossip_errors():
+    t = torch.zeros(4, 8, device="cuda"); W = torch.zeros(4, 4, device="cuda")
+    with pytest.raises(api.LpdtError) as e:
+        api.lpdt_gossip_mix(4, 8, t, t.clone(), t, W, 1.0, [0, 7], [7], ws_bytes(4096))   # segments don't tile
+    assert e.value.code == 1
+    with pytest.raises(api.LpdtError) as e:
+        api.lpdt_gossip_mix(4, 8, t, t, t, W, 1.0, [0, 8], [8], ws_bytes(4096))           # x_hat aliases x_half
+    assert e.value.code == 1
+    big = torch.zeros(65, 4, device="cuda")
+    with pytest.raises(api.LpdtError) as e:
+        api.lpdt_gossip_mix(65, 4, big, big.clone(), big.clone(), torch.zeros(65, 65, device="cuda"), 1.0, [0, 4], [4],
+                            ws_bytes(65536))
+    assert e.value.code == 2
+
+
+# ------------------------------------------------------------------ glue
+def test_glue_ops():
+    rng = np.random.default_rng(8)
+    f = lambda *s: torch.empty(*s, dtype=torch.float32, device="cuda")
+    x = rng.standard_normal(10007).astype(np.float32); g = rng.standard_normal(10007).astype(np.float32)
+    out = f(10007)
+    api.lpdt_sgd_update(10007, dev(x), dev(g), 0.1, out)
+    assert np.array_equal(out.cpu().numpy(), oracle.sgd_update(x, g, 0.1))
+    a = rng.standard_normal((2, 3, 8, 8, 16)).astype(np.float32)
+    r = rng.standard_normal((2, 3, 8, 8, 16)).astype(np.float32)
+    y = f(*r.shape)
+    api.lpdt_residual_add(2, 3, 8, 8, 16, 16, 1, 0, dev(r), dev(a), y)
+    assert np.array_equal(y.cpu().numpy(), oracle.residual_add(r, a))
+    r2 = rng.standard_normal((2, 3, 4, 4, 32)).astype(np.float32)
+    y2 = f(*r2.shape)
+    api.lpdt_residual_add(2, 3, 8, 8, 16, 32, 2, 8, dev(r2), dev(a), y2)
+    assert np.array_equal(y2.cpu().numpy(), oracle.residual_add(r2, a, 2, 8))
+    da = f(*a.shape)
+    api.lpdt_residual_add_bwd(2, 3, 8, 8, 16, 32, 2, 8, dev(r2), dev(a), da)
+    assert np.array_equal(da.cpu().numpy(), oracle.residual_add_bwd(r2, a, 2, 8))
+    p = f(2, 3, 16)
+    api.lpdt_avgpool(2, 3, 64, 16, dev(a), p)
+    assert np.array_equal(p.cpu().numpy(), oracle.avgpool(a))
+    dpx = f(*a.shape)
+    api.lpdt_avgpool_bwd(2, 3, 64, 16, p, dpx)
+    assert np.array_equal(dpx.cpu().numpy(), oracle.avgpool_bwd(oracle.avgpool(a), 8, 8))
+    m_ref, i_ref = oracle.maxpool2x2(a)
+    m = f(*m_ref.shape); idx = torch.empty(m_ref.shape, dtype=torch.int8, device="cuda")
+    api.lpdt_maxpool2x2(2, 3, 8, 8, 16, dev(a), m, idx)
+    assert np.array_equal(m.cpu().numpy(), m_ref) and np.array_equal(idx.cpu().numpy(), i_ref)
+    dm = f(*a.shape)
+    api.lpdt_maxpool2x2_bwd(2, 3, 8, 8, 16, m, idx, dm)
+    assert np.array_equal(dm.cpu().numpy(), oracle.maxpool2x2_bwd(m_ref, i_ref, 8, 8))
+    z = (3 * rng.standard_normal((3, 32, 10))).astype(np.float32)
+    lab = rng.integers(0, 10, (3, 32)).astype(np.int32)
+    loss_ref, dz_ref = oracle.softmax_ce(z, lab)
+    loss = f(3); dz = f(3, 32, 10)
+    api.lpdt_softmax_ce(3, 32, 10, dev(z), dev(lab), loss, dz)
+    close(loss, loss_ref); close(dz, dz_ref, 1e-6, 1e-8)
+    cs = torch.zeros(3, 14, device="cuda")
+    api.lpdt_colsum(3, 32, 10, dev(z), cs[:, 4:], 14)
+    close(cs[:, 4:], oracle.colsum(z), 1e-6, 1e-7)

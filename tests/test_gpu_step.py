@@ -1,0 +1,70 @@
+"""GPU parity of whole training steps against the oracle's step composition."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import step as ostep
+from paper_2111_09389_b200 import workloads as wlmod
+from paper_2111_09389_b200.step import TrainStep
+
+pytestmark = pytest.mark.gpu
+
+
+def close(got, want, rtol=1e-5, atol=1e-6, what=""):
+    got = got.cpu().numpy() if isinstance(got, torch.Tensor) else got
+    want = np.asarray(want, np.float64)
+    err = np.abs(got.astype(np.float64) - want)
+    ok = err <= atol + rtol * np.abs(want)
+    assert ok.all(), f"{what}: {(~ok).sum()} of {ok.size} outside tolerance, worst {err.max():.3e}"
+
+
+def _compare(wl, nodes_to_check=None, **kw):
+    keep = {}
+    ref = ostep.train_step(wl, keep=keep, **kw)
+    st = TrainStep.from_workload(wl, **kw)
+    st.run()
+    torch.cuda.synchronize()
+    assert int(st.dev_status.item()) == 0
+    # integer paths: every quantized layer gradient and accumulator-derived tensor, bit for bit
+    for li, (op, b) in enumerate(zip(wl["ops"], st.buf)):
+        if op["op"] in ("conv", "linear"):
+            assert np.array_equal(b["E"].cpu().numpy().reshape(keep[f"E{li}"].shape), keep[f"E{li}"]), f"E{li}"
+            assert np.array_equal(b["out"].cpu().numpy().reshape(keep[f"out{li}"].shape), keep[f"out{li}"]), f"out{li}"
+    if ref["loss"] is not None:
+        close(st.loss, ref["loss"], what="loss")
+    gscale = float(np.abs(ref["grads"]).max())
+    close(st.grads, ref["grads"], 1e-5, 1e-6 * max(1.0, gscale), "grads")
+    close(st.x_half, ref["x_half"], what="x_half")
+    close(st.x_hat, ref["x_hat"], what="x_hat")
+    close(st.x_out, ref["x"], what="x")
+    if ref["input_grad"] is not None:
+        close(st.input_grad_out, ref["input_grad"], what="input grad")
+    return st, ref
+
+
+def test_conv16_step():
+    _compare(wlmod.make_workload("conv16"))
+
+
+def test_conv16_step_stochastic_and_wgrad_quantized():
+    _compare(wlmod.make_workload("conv16"), grad_rounding=1, seed=1234)
+    _compare(wlmod.make_workload("conv16", nodes=2, batch=2), quantize_wgrad=True)
+
+
+def test_resnet20_step_small():
+    _compare(wlmod.make_workload("resnet20", nodes=3, batch=4))
+
+
+def test_resnet20_topk_step_small():
+    wl = wlmod.make_workload("resnet20_topk", nodes=5, batch=2)
+    st, ref = _compare(wl)
+    k = int(wl["seg_k"][0])
+    assert all(np.count_nonzero(ref["q"][i]) == k for i in range(5))
+
+
+def test_vgg11_step_small():
+    _compare(wlmod.make_workload("vgg11", nodes=2, batch=2))
+
+
+def test_resnet20_dirichlet_labels():
+    _compare(wlmod.make_workload("resnet20", nodes=2, batch=8, dirichlet_alpha=0.1))
