@@ -36,6 +36,10 @@ def _c(a, dt):
     return a
 
 
+def num_threads():
+    return int(lib().orc_num_threads())
+
+
 def philox4x32_10(ctr, key):
     ctr = _c(ctr, np.uint32)
     key = _c(key, np.uint32)

@@ -32,7 +32,21 @@
 #include <stdlib.h>
 #include <string.h>
 
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
 typedef long long i64;
+
+/* Threads the contraction loops will use (1 without OpenMP). */
+int orc_num_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
 
 /* ------------------------------------------------------------------------
  * Philox4x32-10 counter-based generator (Salmon, Moraes, Dror, Shaw:

@@ -11,6 +11,20 @@ import torch
 from ._lib import ConvDesc, lib
 
 
+# Kernels each entry point enqueues (memsets not counted); KERNEL_LAUNCHES accumulates them.
+KERNELS_PER_CALL = {
+    "lpdt_quantize": 2, "lpdt_dequantize": 1, "lpdt_qconv_fwd": 1, "lpdt_qconv_bwd_data": 2,
+    "lpdt_qconv_bwd_weight": 2, "lpdt_range_evonorm_fwd": 1, "lpdt_range_evonorm_bwd": 2,
+    "lpdt_gossip_mix": 2, "lpdt_sgd_update": 1, "lpdt_residual_add": 1, "lpdt_residual_add_bwd": 1,
+    "lpdt_avgpool": 1, "lpdt_avgpool_bwd": 1, "lpdt_maxpool2x2": 1, "lpdt_maxpool2x2_bwd": 1,
+    "lpdt_softmax_ce": 1, "lpdt_colsum": 1,
+}
+KERNEL_LAUNCHES = 0
+# Optional per-entry-point timing: {name: [(start_event, end_event), ...]} when TIMED holds names.
+TIMED = set()
+TIMINGS = {}
+
+
 class LpdtError(RuntimeError):
     def __init__(self, fn, code):
         self.code = code
@@ -18,8 +32,34 @@ class LpdtError(RuntimeError):
 
 
 def _check(fn, code):
+    global KERNEL_LAUNCHES
     if code != 0:
         raise LpdtError(fn, code)
+    KERNEL_LAUNCHES += KERNELS_PER_CALL.get(fn, 0)
+
+
+def timed(name):
+    """Context manager: brackets the enclosed call with CUDA events on the current
+    stream when `name` is in TIMED (used by the benchmark for the dominant kernel)."""
+    return _Timed(name)
+
+
+class _Timed:
+    def __init__(self, name):
+        self.on = name in TIMED
+        self.name = name
+
+    def __enter__(self):
+        if self.on:
+            self.a = torch.cuda.Event(enable_timing=True)
+            self.b = torch.cuda.Event(enable_timing=True)
+            self.a.record()
+
+    def __exit__(self, *exc):
+        if self.on:
+            self.b.record()
+            TIMINGS.setdefault(self.name, []).append((self.a, self.b))
+        return False
 
 
 def _ptr(t):
@@ -164,3 +204,22 @@ def lpdt_softmax_ce(nodes, B, K, logits, labels, loss, dlogits):
 
 def lpdt_colsum(nodes, B, Cc, x, out, out_node_stride):
     _check("lpdt_colsum", lib().lpdt_colsum(nodes, B, Cc, _ptr(x), _ptr(out), out_node_stride, _stream()))
+
+
+def _with_timing(fn):
+    name = fn.__name__
+
+    def call(*a, **kw):
+        if name in TIMED:
+            with timed(name):
+                return fn(*a, **kw)
+        return fn(*a, **kw)
+
+    call.__name__ = name
+    call.__doc__ = fn.__doc__
+    return call
+
+
+for _n in [n for n in list(globals()) if n.startswith("lpdt_") and n in KERNELS_PER_CALL]:
+    globals()[_n] = _with_timing(globals()[_n])
+del _n
