@@ -4,7 +4,19 @@
 #include "common.cuh"
 #include "qconv_internal.cuh"
 
+#include <stdlib.h>
+
 using namespace lpdt;
+
+// LPDT_DISABLE_TC=1 in the environment routes every shape to the CUDA-core kernels.
+static bool use_tc(const lpdt_conv_desc &d) {
+    static int disabled = -1;
+    if (disabled < 0) {
+        const char *e = getenv("LPDT_DISABLE_TC");
+        disabled = (e && e[0] == '1') ? 1 : 0;
+    }
+    return !disabled && tc::tc_supported(d);
+}
 
 static lpdt_status check_desc(const lpdt_conv_desc *d) {
     LPDT_CHECK_ARG(d != nullptr);
@@ -33,6 +45,8 @@ extern "C" lpdt_status lpdt_qconv_fwd(const lpdt_conv_desc *d, const int8_t *A, 
     LPDT_CHECK_ARG(A && Wq && (Y || Yacc));
     LPDT_CHECK_ARG(!Y || (sA && sW));
     LPDT_CHECK_ARG(!bias || bias_node_stride >= d->Cout || d->nodes == 1);
+    if (use_tc(*d) && aligned(A, 16) && aligned(Wq, 16) && (!Y || aligned(Y, 16)) && (!Yacc || aligned(Yacc, 16)))
+        return tc::tc_pix(*d, 0, A, sA, Wq, sW, bias, bias_node_stride, Y, Yacc, dev_status, as_stream(stream));
     return generic_fwd(*d, A, sA, Wq, sW, bias, bias_node_stride, Y, Yacc, as_stream(stream));
 }
 
@@ -46,6 +60,8 @@ extern "C" lpdt_status lpdt_qconv_bwd_data(const lpdt_conv_desc *d, const int8_t
     LPDT_CHECK_ARG(E && Wq && (dA || dAacc));
     LPDT_CHECK_ARG(!dA || (sE && sW));
     if (!ws || ws_bytes < lpdt_qconv_workspace_size(d, 1)) return LPDT_ERR_WORKSPACE;
+    if (use_tc(*d) && aligned(E, 16) && aligned(Wq, 16) && (!dA || aligned(dA, 16)) && (!dAacc || aligned(dAacc, 16)))
+        return tc::tc_pix(*d, 1, E, sE, Wq, sW, nullptr, 0, dA, dAacc, dev_status, as_stream(stream));
     return generic_bwd_data(*d, E, sE, Wq, sW, dA, dAacc, ws, as_stream(stream));
 }
 
@@ -62,5 +78,17 @@ extern "C" lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8
     LPDT_CHECK_ARG(!dW || dw_node_stride >= (int64_t)d->Cout * d->R * d->S * d->Cin || d->nodes == 1);
     if (!dWacc && (!ws || ws_bytes < lpdt_qconv_workspace_size(d, 2) || !aligned(ws, 4)))
         return LPDT_ERR_WORKSPACE;
+    if (use_tc(*d) && d->B > 0 && aligned(E, 16) && aligned(A, 16)) {
+        cudaStream_t st = as_stream(stream);
+        const int64_t per_node = (int64_t)d->Cout * d->R * d->S * d->Cin;
+        int32_t *acc = dWacc ? dWacc : (int32_t *)ws;
+        LPDT_CUDA(cudaMemsetAsync(acc, 0, (size_t)d->nodes * per_node * sizeof(int32_t), st));
+        lpdt_status r = tc::tc_wgrad(*d, E, A, acc, dev_status, st);
+        if (r == LPDT_OK) {
+            if (dW) return dequant_acc_launch(acc, d->nodes, per_node, sE, sA, dW, dw_node_stride, st);
+            return LPDT_OK;
+        }
+        if (r != LPDT_ERR_UNSUPPORTED) return r;
+    }
     return generic_bwd_weight(*d, E, sE, A, sA, dW, dw_node_stride, dWacc, ws, as_stream(stream));
 }

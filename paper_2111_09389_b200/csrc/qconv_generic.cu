@@ -149,6 +149,15 @@ __global__ void dequant_acc_kernel(const int32_t *__restrict__ acc, int nodes, i
     }
 }
 
+static unsigned grid_for(int64_t n);
+
+lpdt_status dequant_acc_launch(const int32_t *acc, int nodes, int64_t per_node, const float *s1,
+                               const float *s2, float *out, int64_t out_stride, cudaStream_t st) {
+    dequant_acc_kernel<<<grid_for(per_node * nodes), 256, 0, st>>>(acc, nodes, per_node, s1, s2, out, out_stride);
+    LPDT_LAUNCH_CHECK();
+    return LPDT_OK;
+}
+
 static unsigned grid_for(int64_t n) {
     int64_t b = ceil_div(n, 256), cap = (int64_t)kNumSMs * 32;
     return (unsigned)(b < 1 ? 1 : (b > cap ? cap : b));

@@ -16,4 +16,18 @@ lpdt_status generic_bwd_weight(const lpdt_conv_desc &d, const int8_t *E, const f
                                const float *sA, float *dW, int64_t dw_stride, int32_t *dWacc, void *ws,
                                cudaStream_t st);
 
+lpdt_status dequant_acc_launch(const int32_t *acc, int nodes, int64_t per_node, const float *s1,
+                               const float *s2, float *out, int64_t out_stride, cudaStream_t st);
+
+namespace tc {
+// Tensor-core engine (tcgen05 kind::i8): stride-1 convolutions and GEMMs whose
+// channel counts are multiples of 16.  mode 0 = forward, 1 = backward-data.
+bool tc_supported(const lpdt_conv_desc &d);
+lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const float *s1, const int8_t *Wq,
+                   const float *s2, const float *bias, int64_t bias_stride, float *Y, int32_t *Yacc,
+                   int32_t *dev_status, cudaStream_t st);
+lpdt_status tc_wgrad(const lpdt_conv_desc &d, const int8_t *E, const int8_t *A, int32_t *acc_out,
+                     int32_t *dev_status, cudaStream_t st);
+}  // namespace tc
+
 }  // namespace lpdt
