@@ -27,13 +27,26 @@ namespace tc {
 constexpr int kSliceBytes = 2048;     // 128 rows x 16 bytes
 constexpr int kThreads = 192;
 
+// A tile belongs to one "class" of M-space pixels.  Stride-1 problems have one
+// class holding every filter tap.  The stride-2 backward-data problem splits the
+// input pixels by the parity of (ih, iw): each parity class sees its own subset of
+// taps and is a stride-1 problem on the error image.
+constexpr int kMaxTaps = 64;
+struct TapTable {
+    int ntaps;
+    signed char wtap[kMaxTaps];   // tap index in the weight tensor (r*S + s)
+    signed char dh[kMaxTaps], dw[kMaxTaps];   // operand-A pixel offset of the tap
+};
 struct PixParams {
     int mode;                 // 0 forward, 1 backward-data
-    int nodes, B, Hm, Wm;     // M-space image (output pixels fwd, input pixels bwd-data)
+    int nodes, B, Hm, Wm;     // M-space grid of one class
+    int Hout, Wout;           // full output image; output pixel = out_mul*m + class parity
+    int out_mul, cmul;        // cmul scales tile origins into operand-A coordinates (forward stride)
+    int ncls, cls_ph[4], cls_pw[4], cls_iters[4];
+    TapTable tt[4];
     int Nc, Kc;               // N channels, K channels per tap
-    int R, S, pad, taps;
     int TB, TH, TW, tilesB, tilesH, tilesW, tilesN, BN;
-    int S_slices, iters, stages, tmem_cols;
+    int S_slices, stages, tmem_cols;
     int w_rows_per_node;      // Cout: rows of the weight map per node
     float *Y; int32_t *Yacc;
     const float *s1, *s2, *bias; long long bias_stride;
@@ -55,7 +68,7 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     const int stage_bytes = p.S_slices * (kSliceBytes + p.BN * 16);
     const int a_bytes = p.S_slices * kSliceBytes;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int total_tiles = p.nodes * p.tilesB * p.tilesH * p.tilesW * p.tilesN;
+    const int total_tiles = p.nodes * p.tilesB * p.tilesH * p.tilesW * p.tilesN * p.ncls;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.stages; ++i) { mbar_init(smem_u32(&ctl->full[i]), 1); mbar_init(smem_u32(&ctl->empty[i]), 1); }
@@ -76,12 +89,14 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             uint32_t g = 0;     // global stage counter
             for (int tile = blockIdx.x; tile < total_tiles && !ctl->abort_flag; tile += gridDim.x) {
                 int t = tile;
+                const int cls = t % p.ncls; t /= p.ncls;
                 const int nt = t % p.tilesN; t /= p.tilesN;
                 const int tw = t % p.tilesW; t /= p.tilesW;
                 const int th = t % p.tilesH; t /= p.tilesH;
                 const int tb = t % p.tilesB; const int node = t / p.tilesB;
-                const int n0 = nt * p.BN, w0 = tw * p.TW, h0 = th * p.TH, b0 = tb * p.TB;
-                for (int it = 0; it < p.iters; ++it, ++g) {
+                const int n0 = nt * p.BN, w0 = tw * p.TW * p.cmul, h0 = th * p.TH * p.cmul, b0 = tb * p.TB;
+                const TapTable &tt = p.tt[cls];
+                for (int it = 0; it < p.cls_iters[cls]; ++it, ++g) {
                     const int st = g % p.stages;
                     const uint32_t ph = (g / p.stages) & 1;
                     if (!mbar_wait(smem_u32(&ctl->empty[st]), ph ^ 1, &ctl->abort_flag, p.dev_status)) break;
@@ -91,13 +106,9 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                     const uint32_t b_st = a_st + a_bytes;
                     for (int sl = 0; sl < p.S_slices; ++sl) {
                         const int kap = it * p.S_slices + sl;
-                        const int tap = kap / cpt, chunk = kap % cpt;
-                        int hc = -(1 << 20), wc = 0;          // phantom slice: whole box out of range -> zeros
-                        if (tap < p.taps) {
-                            const int r = tap / p.S, s = tap % p.S;
-                            hc = h0 + (p.mode == 0 ? r - p.pad : p.pad - r);
-                            wc = w0 + (p.mode == 0 ? s - p.pad : p.pad - s);
-                        }
+                        const int ti = kap / cpt, chunk = kap % cpt;
+                        int hc = -(1 << 20), wc = 0, tap = 1 << 20;   // phantom slice: boxes out of range -> zeros
+                        if (ti < tt.ntaps) { hc = h0 + tt.dh[ti]; wc = w0 + tt.dw[ti]; tap = tt.wtap[ti]; }
                         tma_load_5d(a_st + sl * kSliceBytes, &mapA, full, chunk * 16, wc, hc, b0, node);
                         if (p.mode == 0) {
                             tma_load_3d(b_st + sl * p.BN * 16, &mapW, full, chunk * 16, tap,
@@ -122,7 +133,8 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * p.BN;
                 bool ok = true;
-                for (int it = 0; it < p.iters; ++it, ++g) {
+                const int iters = p.cls_iters[tile % p.ncls];
+                for (int it = 0; it < iters; ++it, ++g) {
                     const int st = g % p.stages;
                     const uint32_t ph = (g / p.stages) & 1;
                     if (!mbar_wait(smem_u32(&ctl->full[st]), ph, &ctl->abort_flag, p.dev_status)) { ok = false; break; }
@@ -149,18 +161,21 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         uint32_t tcount = 0;
         for (int tile = blockIdx.x; tile < total_tiles && !ctl->abort_flag; tile += gridDim.x, ++tcount) {
             int t = tile;
+            const int cls = t % p.ncls; t /= p.ncls;
             const int nt = t % p.tilesN; t /= p.tilesN;
             const int tw = t % p.tilesW; t /= p.tilesW;
             const int th = t % p.tilesH; t /= p.tilesH;
             const int tb = t % p.tilesB; const int node = t / p.tilesB;
             const int n0 = nt * p.BN;
-            const int w = tw * p.TW + pw, h = th * p.TH + phh, b = tb * p.TB + pb;
-            const bool valid = (w < p.Wm) && (h < p.Hm) && (b < p.B);
+            const int w = (tw * p.TW + pw) * p.out_mul + p.cls_pw[cls];
+            const int h = (th * p.TH + phh) * p.out_mul + p.cls_ph[cls];
+            const int b = tb * p.TB + pb;
+            const bool valid = (w < p.Wout) && (h < p.Hout) && (b < p.B);
             const int acc = tcount & 1;
             const uint32_t aph = (tcount >> 1) & 1;
             if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), aph, &ctl->abort_flag, p.dev_status)) break;
             tc_fence_after();
-            const long long pix = (((long long)node * p.B + b) * p.Hm + h) * p.Wm + w;
+            const long long pix = (((long long)node * p.B + b) * p.Hout + h) * p.Wout + w;
             const float sc = p.Y ? __fmul_rn(p.s1[node], p.s2[node]) : 0.f;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * p.BN;
             for (int c = 0; c < p.BN; c += 16) {
@@ -200,7 +215,7 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
 
 // ----------------------------------------------------------------------------------------------
 struct WgParams {
-    int nodes, B, Ho, Wo, Cin, Cout, R, S, pad, taps;
+    int nodes, B, Ho, Wo, Cin, Cout, R, S, pad, taps, stride;
     int TB, TH, TW, tilesB, tilesH, tilesW;       // pixel tiles = K blocks
     int kblocks, splits, kb_per_split;
     int mgroups, ngroups, mtiles, slicesA, BNc, total_slices;
@@ -259,7 +274,8 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                 for (int i = 0; i < nA; ++i) {
                     const int mu = mu0 + i, tap = mu / cpt, chunk = mu % cpt;
                     const int r = tap / p.S, s = tap % p.S;
-                    tma_load_5d(a_st + i * kSliceBytes, &mapX, full, chunk * 16, w0 + s - p.pad, h0 + r - p.pad, b0, node);
+                    tma_load_5d(a_st + i * kSliceBytes, &mapX, full, chunk * 16, w0 * p.stride + s - p.pad,
+                                h0 * p.stride + r - p.pad, b0, node);
                 }
             }
         }
@@ -335,12 +351,16 @@ static void pick_tile(int H, int W, int *TB, int *TH, int *TW) {
     *TW = bw; *TH = bh; *TB = 128 / (bw * bh);
 }
 
+// Activation map: box = one slice {16 channels, TW, TH, TB pixels}.  With estride 2 the
+// box samples every second pixel (the traversal stride of the tensor map), which is how
+// a stride-2 convolution reads its input.
 static bool act_map(CUtensorMap *m, const int8_t *base, int nodes, int B, int H, int W, int C,
-                    int TB, int TH, int TW) {
+                    int TB, int TH, int TW, int estride = 1) {
     uint64_t dims[5] = {(uint64_t)C, (uint64_t)W, (uint64_t)H, (uint64_t)B, (uint64_t)nodes};
     uint64_t strides[4] = {(uint64_t)C, (uint64_t)W * C, (uint64_t)H * W * C, (uint64_t)B * H * W * C};
-    uint32_t box[5] = {16, (uint32_t)TW, (uint32_t)TH, (uint32_t)TB, 1};
-    return make_map_u8(m, base, 5, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE);
+    uint32_t box[5] = {16, (uint32_t)(TW * estride), (uint32_t)(TH * estride), (uint32_t)TB, 1};
+    uint32_t es[5] = {1, (uint32_t)estride, (uint32_t)estride, 1, 1};
+    return make_map_u8(m, base, 5, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE, es);
 }
 
 static bool weight_map(CUtensorMap *m, const int8_t *base, int nodes, int Cout, int taps, int Cin, int box_rows) {
@@ -354,9 +374,9 @@ constexpr int kSmemBudget = 200 * 1024;
 constexpr int kMinSmem = 120 * 1024;      // keeps one CTA per SM, so TMEM allocation never waits
 
 bool tc_supported(const lpdt_conv_desc &d) {
-    if (d.stride != 1) return false;
+    if (d.stride != 1 && d.stride != 2) return false;
     if (d.Cin % 16 || d.Cout % 16) return false;
-    if (d.R * d.S > 64) return false;
+    if (d.R * d.S > kMaxTaps || d.R > 100 || d.S > 100 || d.pad > 100) return false;
     if (!encode_tiled_fn()) return false;
     return true;
 }
@@ -369,24 +389,63 @@ static int largest_div16(int C, int cap) {      // largest multiple of 16 dividi
 lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const float *s1, const int8_t *Wq,
                    const float *s2, const float *bias, int64_t bias_stride, float *Y, int32_t *Yacc,
                    int32_t *dev_status, cudaStream_t st) {
-    const int Ho = conv_out(d.H, d.pad, d.R, 1), Wo = conv_out(d.W, d.pad, d.S, 1);
+    const int Ho = conv_out(d.H, d.pad, d.R, d.stride), Wo = conv_out(d.W, d.pad, d.S, d.stride);
     PixParams p = {};
     p.mode = mode; p.nodes = d.nodes; p.B = d.B;
-    p.Hm = mode == 0 ? Ho : d.H; p.Wm = mode == 0 ? Wo : d.W;
     p.Nc = mode == 0 ? d.Cout : d.Cin; p.Kc = mode == 0 ? d.Cin : d.Cout;
-    p.R = d.R; p.S = d.S; p.pad = d.pad; p.taps = d.R * d.S;
+    p.out_mul = 1; p.cmul = 1; p.ncls = 1;
+    if (mode == 0) {
+        // output pixel (oh, ow) reads input (oh*stride + r - pad, ow*stride + s - pad)
+        p.Hout = Ho; p.Wout = Wo; p.Hm = Ho; p.Wm = Wo; p.cmul = d.stride;
+        TapTable &tt = p.tt[0];
+        for (int r = 0; r < d.R; ++r)
+            for (int s = 0; s < d.S; ++s) {
+                tt.wtap[tt.ntaps] = (signed char)(r * d.S + s);
+                tt.dh[tt.ntaps] = (signed char)(r - d.pad); tt.dw[tt.ntaps] = (signed char)(s - d.pad);
+                ++tt.ntaps;
+            }
+    } else {
+        // input pixel (ih, iw) = (stride*m + ph, ...) reads error pixel ((ih + pad - r)/stride, ...) for
+        // the taps whose offset is divisible by the stride
+        p.Hout = d.H; p.Wout = d.W; p.out_mul = d.stride;
+        p.Hm = (int)ceil_div(d.H, d.stride); p.Wm = (int)ceil_div(d.W, d.stride);
+        p.ncls = d.stride * d.stride;
+        for (int c = 0; c < p.ncls; ++c) {
+            const int ph = c / d.stride, pw = c % d.stride;
+            p.cls_ph[c] = ph; p.cls_pw[c] = pw;
+            TapTable &tt = p.tt[c];
+            for (int r = 0; r < d.R; ++r) {
+                if ((ph + d.pad - r) % d.stride) continue;
+                for (int s = 0; s < d.S; ++s) {
+                    if ((pw + d.pad - s) % d.stride) continue;
+                    tt.wtap[tt.ntaps] = (signed char)(r * d.S + s);
+                    // floor division; ph + pad - r may be negative
+                    const int nh = ph + d.pad - r, nw = pw + d.pad - s;
+                    tt.dh[tt.ntaps] = (signed char)(nh >= 0 ? nh / d.stride : -((-nh) / d.stride));
+                    tt.dw[tt.ntaps] = (signed char)(nw >= 0 ? nw / d.stride : -((-nw) / d.stride));
+                    ++tt.ntaps;
+                }
+            }
+        }
+    }
     pick_tile(p.Hm, p.Wm, &p.TB, &p.TH, &p.TW);
     p.tilesB = (int)ceil_div(d.B, p.TB); p.tilesH = (int)ceil_div(p.Hm, p.TH); p.tilesW = (int)ceil_div(p.Wm, p.TW);
     p.BN = largest_div16(p.Nc, 256);
     p.tilesN = p.Nc / p.BN;
-    int total = p.taps * (p.Kc / 16);
-    if (total & 1) total += 1;
-    int S = 2;
-    for (int s = 16; s >= 2; s -= 2) {
-        if (s * (kSliceBytes + p.BN * 16) > 48 * 1024) continue;
-        if (total % s == 0) { S = s; break; }
+    const int cpt = p.Kc / 16;
+    // slices per stage: even, <= 16, stage <= 48 KB, least padded work over the classes
+    int S = 2; long best = -1;
+    for (int s = 2; s <= 16; s += 2) {
+        if (s * (kSliceBytes + p.BN * 16) > 48 * 1024) break;
+        long work = 0;
+        for (int c = 0; c < p.ncls; ++c) work += ceil_div((long)p.tt[c].ntaps * cpt, s) * s;
+        if (best < 0 || work <= best) { best = work; S = s; }
     }
-    p.S_slices = S; p.iters = (int)ceil_div(total, S);
+    p.S_slices = S;
+    for (int c = 0; c < p.ncls; ++c) {
+        p.cls_iters[c] = (int)ceil_div((long)p.tt[c].ntaps * cpt, S);
+        if (p.cls_iters[c] < 1) p.cls_iters[c] = 1;      // a class without taps still writes zeros
+    }
     const int stage_bytes = S * (kSliceBytes + p.BN * 16);
     p.stages = (kSmemBudget - 1024) / stage_bytes;
     if (p.stages > 8) p.stages = 8;
@@ -396,10 +455,15 @@ lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const flo
     p.Y = Y; p.Yacc = Yacc; p.s1 = s1; p.s2 = s2; p.bias = bias; p.bias_stride = bias_stride;
     p.dev_status = dev_status;
     CUtensorMap mA, mW;
-    // operand A: activations (fwd, image H x W, Cin) or errors (bwd-data, image Ho x Wo, Cout)
-    if (!act_map(&mA, A, d.nodes, d.B, mode == 0 ? d.H : Ho, mode == 0 ? d.W : Wo, p.Kc, p.TB, p.TH, p.TW))
-        return LPDT_ERR_CUDA;
-    if (!weight_map(&mW, Wq, d.nodes, d.Cout, p.taps, d.Cin, mode == 0 ? p.BN : 16)) return LPDT_ERR_CUDA;
+    // operand A: activations (fwd: image H x W, Cin, sampled with the conv stride) or errors
+    // (bwd-data: image Ho x Wo, Cout, dense)
+    if (mode == 0) {
+        if (p.TW * d.stride > 256 || p.TH * d.stride > 256) return LPDT_ERR_UNSUPPORTED;
+        if (!act_map(&mA, A, d.nodes, d.B, d.H, d.W, p.Kc, p.TB, p.TH, p.TW, d.stride)) return LPDT_ERR_CUDA;
+    } else {
+        if (!act_map(&mA, A, d.nodes, d.B, Ho, Wo, p.Kc, p.TB, p.TH, p.TW, 1)) return LPDT_ERR_CUDA;
+    }
+    if (!weight_map(&mW, Wq, d.nodes, d.Cout, d.R * d.S, d.Cin, mode == 0 ? p.BN : 16)) return LPDT_ERR_CUDA;
     size_t smem = 1024 + (size_t)p.stages * stage_bytes;
     if (smem < kMinSmem) smem = kMinSmem;
     static bool attr = false;
@@ -407,7 +471,7 @@ lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const flo
         LPDT_CUDA(cudaFuncSetAttribute(conv_pix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr = true;
     }
-    const long long tiles = (long long)p.nodes * p.tilesB * p.tilesH * p.tilesW * p.tilesN;
+    const long long tiles = (long long)p.nodes * p.tilesB * p.tilesH * p.tilesW * p.tilesN * p.ncls;
     const int grid = (int)(tiles < kNumSMs ? tiles : kNumSMs);
     conv_pix_kernel<<<grid, kThreads, smem, st>>>(mA, mW, p);
     LPDT_LAUNCH_CHECK();
@@ -416,10 +480,10 @@ lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const flo
 
 lpdt_status tc_wgrad(const lpdt_conv_desc &d, const int8_t *E, const int8_t *A, int32_t *acc_out,
                      int32_t *dev_status, cudaStream_t st) {
-    const int Ho = conv_out(d.H, d.pad, d.R, 1), Wo = conv_out(d.W, d.pad, d.S, 1);
+    const int Ho = conv_out(d.H, d.pad, d.R, d.stride), Wo = conv_out(d.W, d.pad, d.S, d.stride);
     WgParams p = {};
     p.nodes = d.nodes; p.B = d.B; p.Ho = Ho; p.Wo = Wo; p.Cin = d.Cin; p.Cout = d.Cout;
-    p.R = d.R; p.S = d.S; p.pad = d.pad; p.taps = d.R * d.S;
+    p.R = d.R; p.S = d.S; p.pad = d.pad; p.taps = d.R * d.S; p.stride = d.stride;
     pick_tile(Ho, Wo, &p.TB, &p.TH, &p.TW);
     p.tilesB = (int)ceil_div(d.B, p.TB); p.tilesH = (int)ceil_div(Ho, p.TH); p.tilesW = (int)ceil_div(Wo, p.TW);
     p.kblocks = p.tilesB * p.tilesH * p.tilesW;
@@ -449,7 +513,8 @@ lpdt_status tc_wgrad(const lpdt_conv_desc &d, const int8_t *E, const int8_t *A, 
     p.splits = (int)ceil_div(p.kblocks, p.kb_per_split);
     p.acc_out = acc_out; p.dev_status = dev_status;
     CUtensorMap mX, mE;
-    if (!act_map(&mX, A, d.nodes, d.B, d.H, d.W, d.Cin, p.TB, p.TH, p.TW)) return LPDT_ERR_CUDA;
+    if (p.TW * d.stride > 256 || p.TH * d.stride > 256) return LPDT_ERR_UNSUPPORTED;
+    if (!act_map(&mX, A, d.nodes, d.B, d.H, d.W, d.Cin, p.TB, p.TH, p.TW, d.stride)) return LPDT_ERR_CUDA;
     if (!act_map(&mE, E, d.nodes, d.B, Ho, Wo, d.Cout, p.TB, p.TH, p.TW)) return LPDT_ERR_CUDA;
     size_t smem = 1024 + (size_t)p.stages * stage_bytes + 16 * 1024;   // slack: descriptors of a partial M tile read past it
     if (smem < kMinSmem) smem = kMinSmem;

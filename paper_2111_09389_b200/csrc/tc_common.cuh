@@ -187,12 +187,13 @@ static inline EncodeTiledFn encode_tiled_fn() {
 // Byte tensor, rank <= 5.  dims[0] is the contiguous dimension; strides[i] is the
 // byte stride of dims[i+1] (multiples of 16).  Out-of-range box elements read zero.
 static inline bool make_map_u8(CUtensorMap *map, const void *base, int rank, const uint64_t *dims,
-                               const uint64_t *strides, const uint32_t *box, CUtensorMapSwizzle swz) {
+                               const uint64_t *strides, const uint32_t *box, CUtensorMapSwizzle swz,
+                               const uint32_t *elem_strides = nullptr) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     cuuint64_t d[5], s[4];
     cuuint32_t b[5], e[5];
-    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; e[i] = 1; }
+    for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; e[i] = elem_strides ? elem_strides[i] : 1; }
     for (int i = 0; i + 1 < rank; ++i) s[i] = strides[i];
     CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void *>(base), d, s, b, e,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,

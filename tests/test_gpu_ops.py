@@ -110,6 +110,14 @@ CONV_CASES = [
     (3, 32, 1, 1, 64, 10, 1, 1, 1, 0),       # classifier
     (1, 5, 4, 4, 8, 8, 3, 3, 1, 0),          # no padding
     (1, 2, 40, 24, 128, 64, 3, 3, 1, 1),
+    (2, 3, 32, 32, 32, 64, 3, 3, 2, 1),      # strided, tensor-core path
+    (1, 2, 15, 13, 16, 16, 3, 3, 2, 1),      # strided with odd image sizes
+    (1, 2, 16, 16, 32, 32, 1, 1, 2, 0),      # strided 1x1: three of four input parities get no tap
+    (1, 1, 56, 56, 64, 64, 3, 3, 1, 1),      # image width that no power-of-two tile divides
+    (1, 3, 7, 7, 16, 32, 5, 5, 1, 2),        # 5x5 filter
+    (2, 40, 1, 1, 256, 128, 1, 1, 1, 0),     # linear layer on the tensor-core path
+    (1, 130, 1, 1, 512, 272, 1, 1, 1, 0),    # linear: ragged row tile, two N tiles (272 = 16*17)
+    (1, 1, 4, 4, 512, 512, 3, 3, 1, 1),      # wide channels on a tiny map
 ]
 
 
