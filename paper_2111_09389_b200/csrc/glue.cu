@@ -37,6 +37,54 @@ __global__ void residual_add_kernel(int64_t NB, int H, int W, int Ca, int C, int
     }
 }
 
+// Vector forms: 4 consecutive channels per thread (C, Ca and ch_off multiples of 4).
+__global__ void residual_add_v4_kernel(int NB, int H, int W, int Ca4, int C4, int stride, int ch_off4,
+                                       const float4 *__restrict__ r, const float4 *__restrict__ a,
+                                       float4 *__restrict__ y) {
+    const int Ho = (H + stride - 1) / stride, Wo = (W + stride - 1) / stride;
+    const long long total = (long long)NB * Ho * Wo * C4;
+    for (long long o = (long long)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(o % C4);
+        float4 v = r[o];
+        const int ca = c - ch_off4;
+        if (ca >= 0 && ca < Ca4) {
+            long long pix = o / C4;
+            const int ow = (int)(pix % Wo); pix /= Wo;
+            const int oh = (int)(pix % Ho);
+            const long long nb = pix / Ho;
+            const float4 u = a[((nb * H + (long long)oh * stride) * W + (long long)ow * stride) * Ca4 + ca];
+            v.x = __fadd_rn(v.x, u.x); v.y = __fadd_rn(v.y, u.y); v.z = __fadd_rn(v.z, u.z); v.w = __fadd_rn(v.w, u.w);
+        }
+        y[o] = v;
+    }
+}
+
+__global__ void residual_add_bwd_v4_kernel(int NB, int H, int W, int Ca4, int C4, int stride, int ch_off4,
+                                           const float4 *__restrict__ dy, const float4 *__restrict__ gm,
+                                           float4 *__restrict__ da) {
+    const int Ho = (H + stride - 1) / stride, Wo = (W + stride - 1) / stride;
+    const long long total = (long long)NB * H * W * Ca4;
+    for (long long o = (long long)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (long long)gridDim.x * blockDim.x) {
+        float4 v = gm[o];
+        bool hit = stride == 1;
+        long long src = o;
+        if (stride != 1 || Ca4 != C4) {
+            const int ca = (int)(o % Ca4);
+            long long pix = o / Ca4;
+            const int w = (int)(pix % W); pix /= W;
+            const int h = (int)(pix % H);
+            const long long nb = pix / H;
+            hit = (h % stride == 0) && (w % stride == 0);
+            src = ((nb * Ho + h / stride) * Wo + w / stride) * C4 + ca + ch_off4;
+        }
+        if (hit) {
+            const float4 u = dy[src];
+            v.x = __fadd_rn(v.x, u.x); v.y = __fadd_rn(v.y, u.y); v.z = __fadd_rn(v.z, u.z); v.w = __fadd_rn(v.w, u.w);
+        }
+        da[o] = v;
+    }
+}
+
 __global__ void residual_add_bwd_kernel(int64_t NB, int H, int W, int Ca, int C, int stride, int ch_off,
                                         const float *__restrict__ dy, const float *__restrict__ gm,
                                         float *__restrict__ da) {
@@ -172,6 +220,11 @@ extern "C" lpdt_status lpdt_residual_add(int32_t nodes, int32_t B, int32_t H, in
     if (nodes == 0 || B == 0) return LPDT_OK;
     LPDT_CHECK_ARG(r && a && y);
     const int Ho = (H + stride - 1) / stride, Wo = (W + stride - 1) / stride;
+    if (C % 4 == 0 && Ca % 4 == 0 && ch_off % 4 == 0 && aligned(r, 16) && aligned(a, 16) && aligned(y, 16) &&
+        (int64_t)nodes * B < 0x7fffffff)
+        residual_add_v4_kernel<<<grid1d((int64_t)nodes * B * Ho * Wo * C / 4), 256, 0, as_stream(stream)>>>(
+            nodes * B, H, W, Ca / 4, C / 4, stride, ch_off / 4, (const float4 *)r, (const float4 *)a, (float4 *)y);
+    else
     residual_add_kernel<<<grid1d((int64_t)nodes * B * Ho * Wo * C), 256, 0, as_stream(stream)>>>(
         (int64_t)nodes * B, H, W, Ca, C, stride, ch_off, r, a, y);
     LPDT_LAUNCH_CHECK();
@@ -185,6 +238,11 @@ extern "C" lpdt_status lpdt_residual_add_bwd(int32_t nodes, int32_t B, int32_t H
     LPDT_CHECK_ARG(ch_off >= 0 && ch_off + Ca <= C);
     if (nodes == 0 || B == 0) return LPDT_OK;
     LPDT_CHECK_ARG(dy && g_main && da);
+    if (C % 4 == 0 && Ca % 4 == 0 && ch_off % 4 == 0 && aligned(dy, 16) && aligned(g_main, 16) && aligned(da, 16) &&
+        (int64_t)nodes * B < 0x7fffffff)
+        residual_add_bwd_v4_kernel<<<grid1d((int64_t)nodes * B * H * W * Ca / 4), 256, 0, as_stream(stream)>>>(
+            nodes * B, H, W, Ca / 4, C / 4, stride, ch_off / 4, (const float4 *)dy, (const float4 *)g_main, (float4 *)da);
+    else
     residual_add_bwd_kernel<<<grid1d((int64_t)nodes * B * H * W * Ca), 256, 0, as_stream(stream)>>>(
         (int64_t)nodes * B, H, W, Ca, C, stride, ch_off, dy, g_main, da);
     LPDT_LAUNCH_CHECK();

@@ -1,21 +1,67 @@
 // Front end of the quantized contractions: argument validation, workspace
 // accounting and the choice between the tensor-core engine and the CUDA-core
-// kernels.
+// kernels.  Layers whose input channel count is not a multiple of 16 (the RGB
+// first layer) reach the tensor-core engine through zero-padded copies of the
+// activations and weights held in the workspace: zero channels add nothing to an
+// integer sum, so the result is unchanged.
+#include <stdlib.h>
 #include "common.cuh"
 #include "qconv_internal.cuh"
 
-#include <stdlib.h>
-
 using namespace lpdt;
 
+namespace lpdt {
+
+// dst[row][0..Cp) = src[row][0..C) followed by zeros.
+__global__ void pad_channels_kernel(const int8_t *__restrict__ src, int8_t *__restrict__ dst, int64_t rows,
+                                    int C, int Cp) {
+    const int64_t total = rows * Cp;
+    for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
+        const int c = (int)(o % Cp);
+        dst[o] = c < C ? src[(o / Cp) * C + c] : (int8_t)0;
+    }
+}
+
+// Drop the padded input channels of an accumulated weight gradient [rows][Cp] -> [rows][C],
+// writing raw accumulators and/or the dequantized fp32 gradient.
+__global__ void unpad_wgrad_kernel(const int32_t *__restrict__ acc_p, int nodes, int64_t rows_per_node, int C,
+                                   int Cp, const float *__restrict__ s1, const float *__restrict__ s2,
+                                   int32_t *__restrict__ acc_out, float *__restrict__ dW, int64_t dw_stride) {
+    const int64_t per_node = rows_per_node * C, total = per_node * nodes;
+    for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
+        const int n = (int)(o / per_node);
+        const int64_t i = o % per_node;
+        const int v = acc_p[((int64_t)n * rows_per_node + i / C) * Cp + i % C];
+        if (acc_out) acc_out[o] = v;
+        if (dW) dW[(int64_t)n * dw_stride + i] = __fmul_rn(__int2float_rn(v), __fmul_rn(s1[n], s2[n]));
+    }
+}
+
+}  // namespace lpdt
+
+static unsigned grid_for(int64_t n) {
+    int64_t b = ceil_div(n, 256), cap = (int64_t)kNumSMs * 32;
+    return (unsigned)(b < 1 ? 1 : (b > cap ? cap : b));
+}
+
 // LPDT_DISABLE_TC=1 in the environment routes every shape to the CUDA-core kernels.
-static bool use_tc(const lpdt_conv_desc &d) {
+static bool tc_enabled() {
     static int disabled = -1;
     if (disabled < 0) {
         const char *e = getenv("LPDT_DISABLE_TC");
         disabled = (e && e[0] == '1') ? 1 : 0;
     }
-    return !disabled && tc::tc_supported(d);
+    return !disabled;
+}
+static bool use_tc(const lpdt_conv_desc &d) { return tc_enabled() && tc::tc_supported(d); }
+
+static int pad16(int c) { return (c + 15) / 16 * 16; }
+// Input channels padded to a multiple of 16 make the shape eligible.
+static bool use_tc_padded(const lpdt_conv_desc &d, lpdt_conv_desc *dp) {
+    if (!tc_enabled() || d.Cin % 16 == 0) return false;
+    *dp = d;
+    dp->Cin = pad16(d.Cin);
+    return tc::tc_supported(*dp);
 }
 
 static lpdt_status check_desc(const lpdt_conv_desc *d) {
@@ -26,34 +72,62 @@ static lpdt_status check_desc(const lpdt_conv_desc *d) {
     return LPDT_OK;
 }
 
+struct PadPlan { size_t a_bytes, w_bytes, acc_bytes; };
+static PadPlan pad_plan(const lpdt_conv_desc &d) {
+    const size_t Cp = pad16(d.Cin);
+    PadPlan p;
+    p.a_bytes = align_up((size_t)d.nodes * d.B * d.H * d.W * Cp, 256);
+    p.w_bytes = align_up((size_t)d.nodes * d.Cout * d.R * d.S * Cp, 256);
+    p.acc_bytes = align_up((size_t)d.nodes * d.Cout * d.R * d.S * Cp * sizeof(int32_t), 256);
+    return p;
+}
+
 extern "C" size_t lpdt_qconv_workspace_size(const lpdt_conv_desc *d, int32_t which) {
-    if (!d || d->nodes <= 0) return 256;
+    if (!d || d->nodes <= 0 || check_desc(d) != LPDT_OK) return 256;
     const size_t wn = (size_t)d->nodes * d->Cout * d->R * d->S * d->Cin;
-    if (which == 1) return align_up(wn, 256);                       // transposed weights
-    if (which == 2) return align_up(wn * sizeof(int32_t), 256);     // int32 partial sums
-    return 256;
+    size_t need = 256;
+    if (which == 1) need = align_up(wn, 256);                       // transposed weights
+    if (which == 2) need = align_up(wn * sizeof(int32_t), 256);     // int32 partial sums
+    if (d->Cin % 16) {
+        const PadPlan p = pad_plan(*d);
+        if (which == 0 && p.a_bytes + p.w_bytes > need) need = p.a_bytes + p.w_bytes;
+        if (which == 2 && p.a_bytes + p.acc_bytes > need) need = p.a_bytes + p.acc_bytes;
+    }
+    return need;
 }
 
 extern "C" lpdt_status lpdt_qconv_fwd(const lpdt_conv_desc *d, const int8_t *A, const float *sA,
                                       const int8_t *Wq, const float *sW, const float *bias,
                                       int64_t bias_node_stride, float *Y, int32_t *Yacc, void *ws,
                                       size_t ws_bytes, int32_t *dev_status, void *stream) {
-    (void)ws; (void)ws_bytes; (void)dev_status;
     lpdt_status s = check_desc(d);
     if (s != LPDT_OK) return s;
     if (d->nodes == 0 || d->B == 0) return LPDT_OK;
     LPDT_CHECK_ARG(A && Wq && (Y || Yacc));
     LPDT_CHECK_ARG(!Y || (sA && sW));
     LPDT_CHECK_ARG(!bias || bias_node_stride >= d->Cout || d->nodes == 1);
-    if (use_tc(*d) && aligned(A, 16) && aligned(Wq, 16) && (!Y || aligned(Y, 16)) && (!Yacc || aligned(Yacc, 16)))
-        return tc::tc_pix(*d, 0, A, sA, Wq, sW, bias, bias_node_stride, Y, Yacc, dev_status, as_stream(stream));
-    return generic_fwd(*d, A, sA, Wq, sW, bias, bias_node_stride, Y, Yacc, as_stream(stream));
+    cudaStream_t st = as_stream(stream);
+    const bool out_ok = (!Y || aligned(Y, 16)) && (!Yacc || aligned(Yacc, 16));
+    if (use_tc(*d) && aligned(A, 16) && aligned(Wq, 16) && out_ok)
+        return tc::tc_pix(*d, 0, A, sA, Wq, sW, bias, bias_node_stride, Y, Yacc, dev_status, st);
+    lpdt_conv_desc dp;
+    if (use_tc_padded(*d, &dp) && out_ok && ws && aligned(ws, 256) &&
+        ws_bytes >= lpdt_qconv_workspace_size(d, 0)) {
+        const PadPlan pp = pad_plan(*d);
+        int8_t *Ap = (int8_t *)ws, *Wp = Ap + pp.a_bytes;
+        const int64_t arows = (int64_t)d->nodes * d->B * d->H * d->W, wrows = (int64_t)d->nodes * d->Cout * d->R * d->S;
+        pad_channels_kernel<<<grid_for(arows * dp.Cin), 256, 0, st>>>(A, Ap, arows, d->Cin, dp.Cin);
+        LPDT_LAUNCH_CHECK();
+        pad_channels_kernel<<<grid_for(wrows * dp.Cin), 256, 0, st>>>(Wq, Wp, wrows, d->Cin, dp.Cin);
+        LPDT_LAUNCH_CHECK();
+        return tc::tc_pix(dp, 0, Ap, sA, Wp, sW, bias, bias_node_stride, Y, Yacc, dev_status, st);
+    }
+    return generic_fwd(*d, A, sA, Wq, sW, bias, bias_node_stride, Y, Yacc, st);
 }
 
 extern "C" lpdt_status lpdt_qconv_bwd_data(const lpdt_conv_desc *d, const int8_t *E, const float *sE,
                                            const int8_t *Wq, const float *sW, float *dA, int32_t *dAacc,
                                            void *ws, size_t ws_bytes, int32_t *dev_status, void *stream) {
-    (void)dev_status;
     lpdt_status s = check_desc(d);
     if (s != LPDT_OK) return s;
     if (d->nodes == 0 || d->B == 0) return LPDT_OK;
@@ -69,7 +143,6 @@ extern "C" lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8
                                              const int8_t *A, const float *sA, float *dW,
                                              int64_t dw_node_stride, int32_t *dWacc, void *ws,
                                              size_t ws_bytes, int32_t *dev_status, void *stream) {
-    (void)dev_status;
     lpdt_status s = check_desc(d);
     if (s != LPDT_OK) return s;
     if (d->nodes == 0) return LPDT_OK;
@@ -78,8 +151,8 @@ extern "C" lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8
     LPDT_CHECK_ARG(!dW || dw_node_stride >= (int64_t)d->Cout * d->R * d->S * d->Cin || d->nodes == 1);
     if (!dWacc && (!ws || ws_bytes < lpdt_qconv_workspace_size(d, 2) || !aligned(ws, 4)))
         return LPDT_ERR_WORKSPACE;
+    cudaStream_t st = as_stream(stream);
     if (use_tc(*d) && d->B > 0 && aligned(E, 16) && aligned(A, 16)) {
-        cudaStream_t st = as_stream(stream);
         const int64_t per_node = (int64_t)d->Cout * d->R * d->S * d->Cin;
         int32_t *acc = dWacc ? dWacc : (int32_t *)ws;
         LPDT_CUDA(cudaMemsetAsync(acc, 0, (size_t)d->nodes * per_node * sizeof(int32_t), st));
@@ -90,5 +163,25 @@ extern "C" lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8
         }
         if (r != LPDT_ERR_UNSUPPORTED) return r;
     }
-    return generic_bwd_weight(*d, E, sE, A, sA, dW, dw_node_stride, dWacc, ws, as_stream(stream));
+    lpdt_conv_desc dp;
+    if (use_tc_padded(*d, &dp) && d->B > 0 && aligned(E, 16) && ws && aligned(ws, 256) &&
+        ws_bytes >= lpdt_qconv_workspace_size(d, 2)) {
+        const PadPlan pp = pad_plan(*d);
+        int8_t *Ap = (int8_t *)ws;
+        int32_t *accp = (int32_t *)(Ap + pp.a_bytes);
+        const int64_t arows = (int64_t)d->nodes * d->B * d->H * d->W;
+        const int64_t wrows_per_node = (int64_t)d->Cout * d->R * d->S;
+        pad_channels_kernel<<<grid_for(arows * dp.Cin), 256, 0, st>>>(A, Ap, arows, d->Cin, dp.Cin);
+        LPDT_LAUNCH_CHECK();
+        LPDT_CUDA(cudaMemsetAsync(accp, 0, (size_t)d->nodes * wrows_per_node * dp.Cin * sizeof(int32_t), st));
+        lpdt_status r = tc::tc_wgrad(dp, E, Ap, accp, dev_status, st);
+        if (r == LPDT_OK) {
+            unpad_wgrad_kernel<<<grid_for(d->nodes * wrows_per_node * d->Cin), 256, 0, st>>>(
+                accp, d->nodes, wrows_per_node, d->Cin, dp.Cin, sE, sA, dWacc, dW, dw_node_stride);
+            LPDT_LAUNCH_CHECK();
+            return LPDT_OK;
+        }
+        if (r != LPDT_ERR_UNSUPPORTED) return r;
+    }
+    return generic_bwd_weight(*d, E, sE, A, sA, dW, dw_node_stride, dWacc, ws, st);
 }

@@ -186,11 +186,25 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
         }
     }
     __syncthreads();   // s_ch zeroed
+    // Per-channel sums: when the column count divides the warp, lanes that share a
+    // column are first folded with shuffles, so only CV lanes per warp touch shared memory.
+    const bool fold = (CV <= 32) && (32 % CV == 0);
+    if (fold) {
 #pragma unroll
-    for (int k = 0; k < V; ++k) {
-        atomicAdd(&s_ch[0 * C + c0 + k], av[k]);
-        atomicAdd(&s_ch[1 * C + c0 + k], ag[k]);
-        atomicAdd(&s_ch[2 * C + c0 + k], ab[k]);
+        for (int k = 0; k < V; ++k)
+            for (int o = 16; o >= CV; o >>= 1) {
+                av[k] += __shfl_xor_sync(0xffffffffu, av[k], o);
+                ag[k] += __shfl_xor_sync(0xffffffffu, ag[k], o);
+                ab[k] += __shfl_xor_sync(0xffffffffu, ab[k], o);
+            }
+    }
+    if (!fold || (t & 31) < CV) {
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            atomicAdd(&s_ch[0 * C + c0 + k], av[k]);
+            atomicAdd(&s_ch[1 * C + c0 + k], ag[k]);
+            atomicAdd(&s_ch[2 * C + c0 + k], ab[k]);
+        }
     }
     s_S[t] = S;
     __syncthreads();

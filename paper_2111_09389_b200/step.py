@@ -228,6 +228,24 @@ class TrainStep:
         self.backward()
         self.update()
 
+    # ---- CUDA graph: the whole step as one replayable launch -------------------------------
+    def capture(self):
+        """Record run() into a CUDA graph (one warm-up run first so that every
+        one-time kernel attribute is set before capture)."""
+        self.run()
+        torch.cuda.synchronize()
+        before = api.KERNEL_LAUNCHES
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            self.run()
+        self.graph_launches = api.KERNEL_LAUNCHES - before
+        self.graph = g
+        return g
+
+    def replay(self):
+        self.graph.replay()
+        api.KERNEL_LAUNCHES += self.graph_launches
+
     def launches_per_step(self):
         """Kernel launches of one run(): counted from the op list (memsets excluded)."""
         n = 0

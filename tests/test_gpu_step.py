@@ -68,3 +68,16 @@ def test_vgg11_step_small():
 
 def test_resnet20_dirichlet_labels():
     _compare(wlmod.make_workload("resnet20", nodes=2, batch=8, dirichlet_alpha=0.1))
+
+
+def test_graph_replay_matches_eager():
+    wl = wlmod.make_workload("resnet20", nodes=2, batch=4)
+    a = TrainStep.from_workload(wl)
+    a.run()
+    b = TrainStep.from_workload(wl)
+    b.capture()                 # warm-up run + captured run executed eagerly... state advanced twice
+    b.load(wl)                  # restore the inputs, then replay once
+    b.replay()
+    torch.cuda.synchronize()
+    assert torch.equal(a.x_out, b.x_out) and torch.equal(a.x_hat, b.x_hat) and torch.equal(a.grads, b.grads)
+    assert b.graph_launches > 100
