@@ -1,42 +1,54 @@
 // Tensor-core engine of the quantized contractions: implicit-GEMM convolution
-// (stride 1) and GEMM on tcgen05.mma kind::i8 with TMA-staged operands, int32
-// accumulators in TMEM and a fused dequantize epilogue.
+// (stride 1 and 2) and GEMM on tcgen05.mma kind::i8 with TMA-staged operands,
+// int32 accumulators in TMEM and a fused dequantize epilogue.
 //
-// Data movement.  Activations stay NHWC int8 in HBM.  A TMA box of
-// {16 channels, TW, TH, TB pixels} lands in shared memory as 128 rows of 16
-// bytes, i.e. sixteen 8x16-byte core matrices of the no-swizzle canonical
-// layout.  One such box is a "slice" (16 bytes of the channel dimension at one
-// filter tap, shifted by the tap offset; out-of-image pixels are zero-filled by
-// TMA, which is exact for symmetric int8).  The same shared-memory image serves
+// Operand tiles.  Activations stay NHWC int8 in HBM.  A TMA box of
+// {RB channel bytes, TW, TH, TB pixels} (TB*TH*TW = 128) lands in shared memory
+// as 128 rows of RB bytes, RB = 128, 64, 32 or 16 chosen from the channel count.
+// Rows of 32..128 bytes use the matching TMA/UMMA swizzle; rows of 16 bytes are
+// the no-swizzle layout (sixteen contiguous 8x16-byte core matrices).  Each box is
+// read at the tap's pixel offset; out-of-image pixels are zero-filled by TMA,
+// which is exact for symmetric int8.  The same shared-memory image serves
 //   - as a K-major operand  (K = (tap, channel): forward and backward-data), and
-//   - as an MN-major operand (K = pixels: backward-weight),
-// only the descriptor's leading/stride offsets trade places.
+//   - as an MN-major operand (K = pixels: backward-weight);
+// only the descriptor changes.  When C = 16 and the stride is 1, the channel and
+// width dimensions are contiguous in memory and are fetched as one 256-byte row
+// per 16 pixels instead of sixteen 16-byte rows.
 //
 // Kernels.  conv_pix_kernel: M = 128 output pixels, N = channels, K = taps x
-// channels; persistent over tiles, double-buffered TMEM accumulator so the
-// epilogue of tile i overlaps the MMAs of tile i+1.  conv_wgrad_kernel: M = (tap,
-// input channel), N = output channels, K = pixels, split over CTAs with exact
-// int32 atomics.  Warp roles: warp 0 issues TMA, warp 1 owns TMEM and issues the
-// MMAs, warps 2-5 run the epilogue (one TMEM lane quarter each).
+// channels; each CTA walks a contiguous range of tiles with a double-buffered
+// TMEM accumulator, so the epilogue of tile i overlaps the MMAs of tile i+1.
+// conv_wgrad_kernel: M = (tap, input channel), N = output channels, K = pixels,
+// split over CTAs with exact int32 atomics.  Warp roles: warp 0 issues TMA,
+// warp 1 owns TMEM and issues the MMAs, warps 2-5 run the epilogue (one TMEM
+// lane quarter each).  Every wait is bounded (tc_common.cuh).
 #include "qconv_internal.cuh"
 #include "tc_common.cuh"
 
 namespace lpdt {
 namespace tc {
 
-constexpr int kSliceBytes = 2048;     // 128 rows x 16 bytes
 constexpr int kThreads = 192;
+constexpr int kMaxTaps = 64;
+
+// Row format of an operand tile: RB bytes per row and the UMMA layout code.
+__host__ __device__ inline uint32_t layout_code(int RB) { return RB == 128 ? 2u : RB == 64 ? 4u : RB == 32 ? 6u : 0u; }
+static int row_bytes_for(int C) { return C % 128 == 0 ? 128 : C % 64 == 0 ? 64 : C % 32 == 0 ? 32 : 16; }
+static CUtensorMapSwizzle swizzle_for(int RB) {
+    return RB == 128 ? CU_TENSOR_MAP_SWIZZLE_128B : RB == 64 ? CU_TENSOR_MAP_SWIZZLE_64B
+         : RB == 32 ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE;
+}
 
 // A tile belongs to one "class" of M-space pixels.  Stride-1 problems have one
 // class holding every filter tap.  The stride-2 backward-data problem splits the
 // input pixels by the parity of (ih, iw): each parity class sees its own subset of
 // taps and is a stride-1 problem on the error image.
-constexpr int kMaxTaps = 64;
 struct TapTable {
     int ntaps;
-    signed char wtap[kMaxTaps];   // tap index in the weight tensor (r*S + s)
+    signed char wtap[kMaxTaps];               // tap index in the weight tensor (r*S + s)
     signed char dh[kMaxTaps], dw[kMaxTaps];   // operand-A pixel offset of the tap
 };
+
 struct PixParams {
     int mode;                 // 0 forward, 1 backward-data
     int nodes, B, Hm, Wm;     // M-space grid of one class
@@ -45,8 +57,10 @@ struct PixParams {
     int ncls, cls_ph[4], cls_pw[4], cls_iters[4];
     TapTable tt[4];
     int Nc, Kc;               // N channels, K channels per tap
+    int RBa, RBn;             // row bytes of operand A (K side) and, backward-data, of the N side
+    int merged;               // operand A fetched through the merged (channel, width) map
     int TB, TH, TW, tilesB, tilesH, tilesW, tilesN, BN;
-    int S_slices, stages, tmem_cols;
+    int U, stages, tmem_cols; // K units (one A box each) per stage
     int w_rows_per_node;      // Cout: rows of the weight map per node
     float *Y; int32_t *Yacc;
     const float *s1, *s2, *bias; long long bias_stride;
@@ -59,16 +73,32 @@ struct SharedCtl {
     volatile int abort_flag;
 };
 
+struct TileCoord { int cls, tw, th, tb, nt, node; };
+// tile order: node, N tile, batch tile, row tile, column tile, class (fastest)
+__device__ __forceinline__ TileCoord decode_tile(const PixParams &p, int tile) {
+    TileCoord c; int t = tile;
+    c.cls = t % p.ncls; t /= p.ncls;
+    c.tw = t % p.tilesW; t /= p.tilesW;
+    c.th = t % p.tilesH; t /= p.tilesH;
+    c.tb = t % p.tilesB; t /= p.tilesB;
+    c.nt = t % p.tilesN; c.node = t / p.tilesN;
+    return c;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapW,
                 const PixParams p) {
     extern __shared__ __align__(1024) unsigned char smem[];
     SharedCtl *ctl = reinterpret_cast<SharedCtl *>(smem);
     unsigned char *data = smem + 1024;
-    const int stage_bytes = p.S_slices * (kSliceBytes + p.BN * 16);
-    const int a_bytes = p.S_slices * kSliceBytes;
+    const int a_unit = 128 * p.RBa;                        // bytes of one A box
+    const int b_unit = p.BN * p.RBa;                       // weight bytes that go with it
+    const int a_bytes = p.U * a_unit;
+    const int stage_bytes = p.U * (a_unit + b_unit);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int total_tiles = p.nodes * p.tilesB * p.tilesH * p.tilesW * p.tilesN * p.ncls;
+    const long long total_tiles = (long long)p.nodes * p.tilesN * p.tilesB * p.tilesH * p.tilesW * p.ncls;
+    const int tile_lo = (int)(total_tiles * blockIdx.x / gridDim.x);
+    const int tile_hi = (int)(total_tiles * (blockIdx.x + 1) / gridDim.x);
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.stages; ++i) { mbar_init(smem_u32(&ctl->full[i]), 1); mbar_init(smem_u32(&ctl->empty[i]), 1); }
@@ -81,22 +111,17 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
-    const int cpt = p.Kc / 16;
+    const int cpt = p.Kc / p.RBa;          // A boxes per tap
 
     if (warp == 0) {
         if (lane == 0) {
             tma_prefetch_desc(&mapA); tma_prefetch_desc(&mapW);
-            uint32_t g = 0;     // global stage counter
-            for (int tile = blockIdx.x; tile < total_tiles && !ctl->abort_flag; tile += gridDim.x) {
-                int t = tile;
-                const int cls = t % p.ncls; t /= p.ncls;
-                const int nt = t % p.tilesN; t /= p.tilesN;
-                const int tw = t % p.tilesW; t /= p.tilesW;
-                const int th = t % p.tilesH; t /= p.tilesH;
-                const int tb = t % p.tilesB; const int node = t / p.tilesB;
-                const int n0 = nt * p.BN, w0 = tw * p.TW * p.cmul, h0 = th * p.TH * p.cmul, b0 = tb * p.TB;
-                const TapTable &tt = p.tt[cls];
-                for (int it = 0; it < p.cls_iters[cls]; ++it, ++g) {
+            uint32_t g = 0;     // running stage counter
+            for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; ++tile) {
+                const TileCoord c = decode_tile(p, tile);
+                const int n0 = c.nt * p.BN, w0 = c.tw * p.TW * p.cmul, h0 = c.th * p.TH * p.cmul, b0 = c.tb * p.TB;
+                const TapTable &tt = p.tt[c.cls];
+                for (int it = 0; it < p.cls_iters[c.cls]; ++it, ++g) {
                     const int st = g % p.stages;
                     const uint32_t ph = (g / p.stages) & 1;
                     if (!mbar_wait(smem_u32(&ctl->empty[st]), ph ^ 1, &ctl->abort_flag, p.dev_status)) break;
@@ -104,19 +129,21 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                     mbar_expect_tx(full, stage_bytes);
                     const uint32_t a_st = smem_u32(data + (size_t)st * stage_bytes);
                     const uint32_t b_st = a_st + a_bytes;
-                    for (int sl = 0; sl < p.S_slices; ++sl) {
-                        const int kap = it * p.S_slices + sl;
+                    for (int u = 0; u < p.U; ++u) {
+                        const int kap = it * p.U + u;
                         const int ti = kap / cpt, chunk = kap % cpt;
-                        int hc = -(1 << 20), wc = 0, tap = 1 << 20;   // phantom slice: boxes out of range -> zeros
+                        int hc = -(1 << 20), wc = 0, tap = 1 << 20;   // phantom unit: boxes out of range -> zeros
                         if (ti < tt.ntaps) { hc = h0 + tt.dh[ti]; wc = w0 + tt.dw[ti]; tap = tt.wtap[ti]; }
-                        tma_load_5d(a_st + sl * kSliceBytes, &mapA, full, chunk * 16, wc, hc, b0, node);
+                        if (p.merged) tma_load_4d(a_st + u * a_unit, &mapA, full, wc * 16, hc, b0, c.node);
+                        else tma_load_5d(a_st + u * a_unit, &mapA, full, chunk * p.RBa, wc, hc, b0, c.node);
                         if (p.mode == 0) {
-                            tma_load_3d(b_st + sl * p.BN * 16, &mapW, full, chunk * 16, tap,
-                                        node * p.w_rows_per_node + n0);
+                            tma_load_3d(b_st + u * b_unit, &mapW, full, chunk * p.RBa, tap,
+                                        c.node * p.w_rows_per_node + n0);
                         } else {
-                            for (int j = 0; j < p.BN / 16; ++j)
-                                tma_load_3d(b_st + j * (p.S_slices * 256) + sl * 256, &mapW, full, n0 + j * 16, tap,
-                                            node * p.w_rows_per_node + chunk * 16);
+                            // N side in chunks of RBn bytes; this unit's RBa weight rows go at row u*RBa of each chunk
+                            for (int j = 0; j < p.BN / p.RBn; ++j)
+                                tma_load_3d(b_st + j * (p.U * p.RBa * p.RBn) + u * p.RBa * p.RBn, &mapW, full,
+                                            n0 + j * p.RBn, tap, c.node * p.w_rows_per_node + chunk * p.RBa);
                         }
                     }
                 }
@@ -125,8 +152,10 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = idesc_i8(128, p.BN, 0, p.mode == 0 ? 0 : 1);
+            const uint32_t la = layout_code(p.RBa), ln = layout_code(p.RBn);
+            const int n_mma = p.U * p.RBa / 32;
             uint32_t g = 0, tcount = 0;
-            for (int tile = blockIdx.x; tile < total_tiles && !ctl->abort_flag; tile += gridDim.x, ++tcount) {
+            for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; ++tile, ++tcount) {
                 const int acc = tcount & 1;
                 const uint32_t aph = (tcount >> 1) & 1;
                 if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), aph ^ 1, &ctl->abort_flag, p.dev_status)) break;
@@ -141,12 +170,20 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                     tc_fence_after();
                     const uint32_t a_st = smem_u32(data + (size_t)st * stage_bytes);
                     const uint32_t b_st = a_st + a_bytes;
-                    for (int j = 0; j < p.S_slices / 2; ++j) {
-                        const uint64_t ad = smem_desc(a_st + j * 2 * kSliceBytes, kSliceBytes, 128, 0);
-                        const uint64_t bd = (p.mode == 0)
-                            ? smem_desc(b_st + j * 2 * p.BN * 16, p.BN * 16, 128, 0)
-                            : smem_desc(b_st + j * 512, 128, p.S_slices * 256, 0);
-                        mma_i8(d_tmem, ad, bd, idesc, (it | j) != 0);
+                    for (int m = 0; m < n_mma; ++m) {
+                        const int kb = m * 32;                                   // K byte offset within the stage
+                        uint64_t ad, bd;
+                        if (p.RBa == 16) ad = smem_desc(a_st + (kb / 16) * a_unit, a_unit, 128, 0);
+                        else ad = smem_desc(a_st + (kb / p.RBa) * a_unit + kb % p.RBa, 16, 8 * p.RBa, la);
+                        if (p.mode == 0) {
+                            if (p.RBa == 16) bd = smem_desc(b_st + (kb / 16) * b_unit, b_unit, 128, 0);
+                            else bd = smem_desc(b_st + (kb / p.RBa) * b_unit + kb % p.RBa, 16, 8 * p.RBa, la);
+                        } else {
+                            // MN-major: K rows of RBn bytes; N chunks U*RBa rows apart
+                            if (p.RBn == 16) bd = smem_desc(b_st + kb * 16, 128, p.U * p.RBa * 16, 0);
+                            else bd = smem_desc(b_st + kb * p.RBn, p.U * p.RBa * p.RBn, 8 * p.RBn, ln);
+                        }
+                        mma_i8(d_tmem, ad, bd, idesc, (it | m) != 0);
                     }
                     mma_commit(smem_u32(&ctl->empty[st]));
                 }
@@ -159,31 +196,26 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         const int row = q * 32 + lane;                // tile row = pixel within the tile
         const int pw = row % p.TW, phh = (row / p.TW) % p.TH, pb = row / (p.TW * p.TH);
         uint32_t tcount = 0;
-        for (int tile = blockIdx.x; tile < total_tiles && !ctl->abort_flag; tile += gridDim.x, ++tcount) {
-            int t = tile;
-            const int cls = t % p.ncls; t /= p.ncls;
-            const int nt = t % p.tilesN; t /= p.tilesN;
-            const int tw = t % p.tilesW; t /= p.tilesW;
-            const int th = t % p.tilesH; t /= p.tilesH;
-            const int tb = t % p.tilesB; const int node = t / p.tilesB;
-            const int n0 = nt * p.BN;
-            const int w = (tw * p.TW + pw) * p.out_mul + p.cls_pw[cls];
-            const int h = (th * p.TH + phh) * p.out_mul + p.cls_ph[cls];
-            const int b = tb * p.TB + pb;
+        for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; ++tile, ++tcount) {
+            const TileCoord c = decode_tile(p, tile);
+            const int n0 = c.nt * p.BN;
+            const int w = (c.tw * p.TW + pw) * p.out_mul + p.cls_pw[c.cls];
+            const int h = (c.th * p.TH + phh) * p.out_mul + p.cls_ph[c.cls];
+            const int b = c.tb * p.TB + pb;
             const bool valid = (w < p.Wout) && (h < p.Hout) && (b < p.B);
             const int acc = tcount & 1;
             const uint32_t aph = (tcount >> 1) & 1;
             if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), aph, &ctl->abort_flag, p.dev_status)) break;
             tc_fence_after();
-            const long long pix = (((long long)node * p.B + b) * p.Hout + h) * p.Wout + w;
-            const float sc = p.Y ? __fmul_rn(p.s1[node], p.s2[node]) : 0.f;
+            const long long pix = (((long long)c.node * p.B + b) * p.Hout + h) * p.Wout + w;
+            const float sc = p.Y ? __fmul_rn(p.s1[c.node], p.s2[c.node]) : 0.f;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * p.BN;
-            for (int c = 0; c < p.BN; c += 16) {
+            for (int cc = 0; cc < p.BN; cc += 16) {
                 uint32_t v[16];
-                tmem_ld_32x16(t_row + c, v);
+                tmem_ld_32x16(t_row + cc, v);
                 tmem_ld_wait();
-                if (valid && n0 + c < p.Nc) {
-                    const long long o = pix * p.Nc + n0 + c;
+                if (valid) {
+                    const long long o = pix * p.Nc + n0 + cc;
                     if (p.Yacc) {
                         int4 *dst = reinterpret_cast<int4 *>(p.Yacc + o);
 #pragma unroll
@@ -195,7 +227,7 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
 #pragma unroll
                         for (int k = 0; k < 16; ++k) {
                             f[k] = __fmul_rn(__int2float_rn((int)v[k]), sc);
-                            if (p.bias) f[k] = __fadd_rn(f[k], p.bias[(long long)node * p.bias_stride + n0 + c + k]);
+                            if (p.bias) f[k] = __fadd_rn(f[k], p.bias[(long long)c.node * p.bias_stride + n0 + cc + k]);
                         }
                         float4 *dst = reinterpret_cast<float4 *>(p.Y + o);
 #pragma unroll
@@ -218,7 +250,8 @@ struct WgParams {
     int nodes, B, Ho, Wo, Cin, Cout, R, S, pad, taps, stride;
     int TB, TH, TW, tilesB, tilesH, tilesW;       // pixel tiles = K blocks
     int kblocks, splits, kb_per_split;
-    int mgroups, ngroups, mtiles, slicesA, BNc, total_slices;
+    int RBx, RBe, merged;                         // row bytes of the input tiles and of the error tiles
+    int mgroups, ngroups, mtiles, BNc, total_units;
     int stages, tmem_cols;
     int32_t *acc_out; int32_t *dev_status;
 };
@@ -232,14 +265,16 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int node = blockIdx.z;
     const int mg = blockIdx.y % p.mgroups, ng = blockIdx.y / p.mgroups;
-    const int mu0 = mg * p.mtiles * 8;
-    int nA = p.total_slices - mu0; if (nA > p.slicesA) nA = p.slicesA;
-    const int n0 = ng * p.BNc, nE = p.BNc / 16;
-    const int a_region = p.mtiles * 8 * kSliceBytes;
-    const int stage_bytes = a_region + nE * kSliceBytes;
+    const int G = 128 / p.RBx;                    // input boxes stacked in one 128-lane M tile
+    const int x_unit = 128 * p.RBx, e_unit = 128 * p.RBe;
+    const int mu0 = mg * p.mtiles * G;
+    int nX = p.total_units - mu0; if (nX > p.mtiles * G) nX = p.mtiles * G;
+    const int n0 = ng * p.BNc, nE = p.BNc / p.RBe;
+    const int x_region = p.mtiles * 16384;
+    const int stage_bytes = x_region + 128 * p.BNc;
     const int kb0 = blockIdx.x * p.kb_per_split;
     int kb1 = kb0 + p.kb_per_split; if (kb1 > p.kblocks) kb1 = p.kblocks;
-    const int cpt = p.Cin / 16;
+    const int cpt = p.Cin / p.RBx;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.stages; ++i) { mbar_init(smem_u32(&ctl->full[i]), 1); mbar_init(smem_u32(&ctl->empty[i]), 1); }
@@ -266,22 +301,24 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                 const uint32_t ph = (g / p.stages) & 1;
                 if (!mbar_wait(smem_u32(&ctl->empty[st]), ph ^ 1, &ctl->abort_flag, p.dev_status)) break;
                 const uint32_t full = smem_u32(&ctl->full[st]);
-                mbar_expect_tx(full, (nA + nE) * kSliceBytes);
-                const uint32_t a_st = smem_u32(data + (size_t)st * stage_bytes);
-                const uint32_t e_st = a_st + a_region;
+                mbar_expect_tx(full, nX * x_unit + nE * e_unit);
+                const uint32_t x_st = smem_u32(data + (size_t)st * stage_bytes);
+                const uint32_t e_st = x_st + x_region;
                 for (int c = 0; c < nE; ++c)
-                    tma_load_5d(e_st + c * kSliceBytes, &mapE, full, n0 + c * 16, w0, h0, b0, node);
-                for (int i = 0; i < nA; ++i) {
+                    tma_load_5d(e_st + c * e_unit, &mapE, full, n0 + c * p.RBe, w0, h0, b0, node);
+                for (int i = 0; i < nX; ++i) {
                     const int mu = mu0 + i, tap = mu / cpt, chunk = mu % cpt;
                     const int r = tap / p.S, s = tap % p.S;
-                    tma_load_5d(a_st + i * kSliceBytes, &mapX, full, chunk * 16, w0 * p.stride + s - p.pad,
-                                h0 * p.stride + r - p.pad, b0, node);
+                    const int wc = w0 * p.stride + s - p.pad, hc = h0 * p.stride + r - p.pad;
+                    if (p.merged) tma_load_4d(x_st + i * x_unit, &mapX, full, wc * 16, hc, b0, node);
+                    else tma_load_5d(x_st + i * x_unit, &mapX, full, chunk * p.RBx, wc, hc, b0, node);
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = idesc_i8(128, p.BNc, 1, 1);
+            const uint32_t lx = layout_code(p.RBx), le = layout_code(p.RBe);
             uint32_t g = 0;
             bool ok = true;
             for (int kb = kb0; kb < kb1; ++kb, ++g) {
@@ -289,12 +326,16 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                 const uint32_t ph = (g / p.stages) & 1;
                 if (!mbar_wait(smem_u32(&ctl->full[st]), ph, &ctl->abort_flag, p.dev_status)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t a_st = smem_u32(data + (size_t)st * stage_bytes);
-                const uint32_t e_st = a_st + a_region;
+                const uint32_t x_st = smem_u32(data + (size_t)st * stage_bytes);
+                const uint32_t e_st = x_st + x_region;
                 for (int t = 0; t < p.mtiles; ++t)
-                    for (int kk = 0; kk < 4; ++kk) {
-                        const uint64_t ad = smem_desc(a_st + t * 8 * kSliceBytes + kk * 512, 128, kSliceBytes, 0);
-                        const uint64_t bd = smem_desc(e_st + kk * 512, 128, kSliceBytes, 0);
+                    for (int kk = 0; kk < 4; ++kk) {       // 32 pixel rows per MMA
+                        const uint64_t ad = (p.RBx == 16)
+                            ? smem_desc(x_st + t * 16384 + kk * 512, 128, x_unit, 0)
+                            : smem_desc(x_st + t * 16384 + kk * 32 * p.RBx, x_unit, 8 * p.RBx, lx);
+                        const uint64_t bd = (p.RBe == 16)
+                            ? smem_desc(e_st + kk * 512, 128, e_unit, 0)
+                            : smem_desc(e_st + kk * 32 * p.RBe, e_unit, 8 * p.RBe, le);
                         mma_i8(tmem_base + t * p.BNc, ad, bd, idesc, (g | (uint32_t)kk) != 0);
                     }
                 mma_commit(smem_u32(&ctl->empty[st]));
@@ -307,10 +348,10 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         if (mbar_wait(smem_u32(&ctl->tmem_full[0]), 0, &ctl->abort_flag, p.dev_status)) {
             tc_fence_after();
             for (int t = 0; t < p.mtiles; ++t) {
-                const int i = t * 8 + row / 16;                 // slice within this CTA
+                const int i = t * G + row / p.RBx;                 // input box within this CTA
                 const int mu = mu0 + i;
-                const bool valid = (i < nA) && (mu < p.total_slices);
-                const int tap = mu / cpt, ci = (mu % cpt) * 16 + (row & 15);
+                const bool valid = (i < nX) && (mu < p.total_units);
+                const int tap = mu / cpt, ci = (mu % cpt) * p.RBx + row % p.RBx;
                 const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + t * p.BNc;
                 for (int c = 0; c < p.BNc; c += 16) {
                     uint32_t v[16];
@@ -337,9 +378,9 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
 static int pow2_at_least(int v) { int p = 32; while (p < v) p <<= 1; return p; }
 
 // Pixel tile {TB, TH, TW} with TB*TH*TW = 128 covering a W x H image with least waste.
-static void pick_tile(int H, int W, int *TB, int *TH, int *TW) {
+static void pick_tile(int H, int W, int max_tw, int *TB, int *TH, int *TW) {
     int bw = 1; long best = -1;
-    for (int t = 1; t <= 128; t <<= 1) {
+    for (int t = 1; t <= max_tw; t <<= 1) {
         long cover = (long)ceil_div(W, t) * t;
         if (best < 0 || cover <= best) { best = cover; bw = t; }
     }
@@ -351,23 +392,32 @@ static void pick_tile(int H, int W, int *TB, int *TH, int *TW) {
     *TW = bw; *TH = bh; *TB = 128 / (bw * bh);
 }
 
-// Activation map: box = one slice {16 channels, TW, TH, TB pixels}.  With estride 2 the
+// Activation map: box = {RB channel bytes, TW, TH, TB pixels, 1 node}.  With estride 2 the
 // box samples every second pixel (the traversal stride of the tensor map), which is how
 // a stride-2 convolution reads its input.
-static bool act_map(CUtensorMap *m, const int8_t *base, int nodes, int B, int H, int W, int C,
+static bool act_map(CUtensorMap *m, const int8_t *base, int nodes, int B, int H, int W, int C, int RB,
                     int TB, int TH, int TW, int estride = 1) {
     uint64_t dims[5] = {(uint64_t)C, (uint64_t)W, (uint64_t)H, (uint64_t)B, (uint64_t)nodes};
     uint64_t strides[4] = {(uint64_t)C, (uint64_t)W * C, (uint64_t)H * W * C, (uint64_t)B * H * W * C};
-    uint32_t box[5] = {16, (uint32_t)(TW * estride), (uint32_t)(TH * estride), (uint32_t)TB, 1};
+    uint32_t box[5] = {(uint32_t)RB, (uint32_t)(TW * estride), (uint32_t)(TH * estride), (uint32_t)TB, 1};
     uint32_t es[5] = {1, (uint32_t)estride, (uint32_t)estride, 1, 1};
-    return make_map_u8(m, base, 5, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE, es);
+    return make_map_u8(m, base, 5, dims, strides, box, swizzle_for(RB), es);
+}
+// C = 16, stride 1: (channel, width) is one contiguous row of 16*W bytes; a box row is TW pixels.
+static bool act_map_merged(CUtensorMap *m, const int8_t *base, int nodes, int B, int H, int W,
+                           int TB, int TH, int TW) {
+    uint64_t dims[4] = {(uint64_t)W * 16, (uint64_t)H, (uint64_t)B, (uint64_t)nodes};
+    uint64_t strides[3] = {(uint64_t)W * 16, (uint64_t)H * W * 16, (uint64_t)B * H * W * 16};
+    uint32_t box[4] = {(uint32_t)TW * 16, (uint32_t)TH, (uint32_t)TB, 1};
+    return make_map_u8(m, base, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE);
 }
 
-static bool weight_map(CUtensorMap *m, const int8_t *base, int nodes, int Cout, int taps, int Cin, int box_rows) {
+static bool weight_map(CUtensorMap *m, const int8_t *base, int nodes, int Cout, int taps, int Cin, int box_inner,
+                       int box_rows) {
     uint64_t dims[3] = {(uint64_t)Cin, (uint64_t)taps, (uint64_t)nodes * Cout};
     uint64_t strides[2] = {(uint64_t)Cin, (uint64_t)taps * Cin};
-    uint32_t box[3] = {16, 1, (uint32_t)box_rows};
-    return make_map_u8(m, base, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE);
+    uint32_t box[3] = {(uint32_t)box_inner, 1, (uint32_t)box_rows};
+    return make_map_u8(m, base, 3, dims, strides, box, swizzle_for(box_inner));
 }
 
 constexpr int kSmemBudget = 200 * 1024;
@@ -381,9 +431,9 @@ bool tc_supported(const lpdt_conv_desc &d) {
     return true;
 }
 
-static int largest_div16(int C, int cap) {      // largest multiple of 16 dividing C, <= cap
-    for (int v = cap - cap % 16; v >= 16; v -= 16) if (C % v == 0) return v;
-    return 16;
+static int largest_div(int C, int cap, int unit) {      // largest multiple of unit dividing C, <= cap
+    for (int v = cap - cap % unit; v >= unit; v -= unit) if (C % v == 0) return v;
+    return unit;
 }
 
 lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const float *s1, const int8_t *Wq,
@@ -419,34 +469,43 @@ lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const flo
                 for (int s = 0; s < d.S; ++s) {
                     if ((pw + d.pad - s) % d.stride) continue;
                     tt.wtap[tt.ntaps] = (signed char)(r * d.S + s);
-                    // floor division; ph + pad - r may be negative
-                    const int nh = ph + d.pad - r, nw = pw + d.pad - s;
-                    tt.dh[tt.ntaps] = (signed char)(nh >= 0 ? nh / d.stride : -((-nh) / d.stride));
-                    tt.dw[tt.ntaps] = (signed char)(nw >= 0 ? nw / d.stride : -((-nw) / d.stride));
+                    tt.dh[tt.ntaps] = (signed char)((ph + d.pad - r) / d.stride);   // exact: divisible
+                    tt.dw[tt.ntaps] = (signed char)((pw + d.pad - s) / d.stride);
                     ++tt.ntaps;
                 }
             }
         }
     }
-    pick_tile(p.Hm, p.Wm, &p.TB, &p.TH, &p.TW);
+    p.RBa = row_bytes_for(p.Kc);
+    p.RBn = row_bytes_for(p.Nc);
+    const int estride = mode == 0 ? d.stride : 1;
+    p.merged = (p.Kc == 16 && estride == 1) ? 1 : 0;
+    pick_tile(p.Hm, p.Wm, p.merged ? 16 : 128, &p.TB, &p.TH, &p.TW);
+    if (p.TW * estride > 256 || p.TH * estride > 256) return LPDT_ERR_UNSUPPORTED;
     p.tilesB = (int)ceil_div(d.B, p.TB); p.tilesH = (int)ceil_div(p.Hm, p.TH); p.tilesW = (int)ceil_div(p.Wm, p.TW);
-    p.BN = largest_div16(p.Nc, 256);
+    p.BN = largest_div(p.Nc, 256, mode == 0 ? 16 : p.RBn);
     p.tilesN = p.Nc / p.BN;
-    const int cpt = p.Kc / 16;
-    // slices per stage: even, <= 16, stage <= 48 KB, least padded work over the classes
-    int S = 2; long best = -1;
-    for (int s = 2; s <= 16; s += 2) {
-        if (s * (kSliceBytes + p.BN * 16) > 48 * 1024) break;
+    const int cpt = p.Kc / p.RBa;
+    const int unit_bytes = 128 * p.RBa + p.BN * p.RBa;
+    // K units per stage: stage <= 48 KB, at most 16 units, an even count for 16-byte rows (one MMA
+    // consumes two of them); the least padded work over the classes wins, ties go to the larger stage
+    int U = 0; long best = -1;
+    const int ustep = p.RBa == 16 ? 2 : 1;
+    for (int u = ustep; u <= 16; u += ustep) {
+        if (u * unit_bytes > 48 * 1024 && U) break;
         long work = 0;
-        for (int c = 0; c < p.ncls; ++c) work += ceil_div((long)p.tt[c].ntaps * cpt, s) * s;
-        if (best < 0 || work <= best) { best = work; S = s; }
+        for (int c = 0; c < p.ncls; ++c) {
+            long n = (long)p.tt[c].ntaps * cpt; if (n < 1) n = 1;
+            work += ceil_div(n, u) * u;
+        }
+        if (best < 0 || work <= best) { best = work; U = u; }
     }
-    p.S_slices = S;
+    p.U = U;
     for (int c = 0; c < p.ncls; ++c) {
-        p.cls_iters[c] = (int)ceil_div((long)p.tt[c].ntaps * cpt, S);
+        p.cls_iters[c] = (int)ceil_div((long)p.tt[c].ntaps * cpt, U);
         if (p.cls_iters[c] < 1) p.cls_iters[c] = 1;      // a class without taps still writes zeros
     }
-    const int stage_bytes = S * (kSliceBytes + p.BN * 16);
+    const int stage_bytes = U * unit_bytes;
     p.stages = (kSmemBudget - 1024) / stage_bytes;
     if (p.stages > 8) p.stages = 8;
     if (p.stages < 2) return LPDT_ERR_UNSUPPORTED;
@@ -457,13 +516,11 @@ lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const flo
     CUtensorMap mA, mW;
     // operand A: activations (fwd: image H x W, Cin, sampled with the conv stride) or errors
     // (bwd-data: image Ho x Wo, Cout, dense)
-    if (mode == 0) {
-        if (p.TW * d.stride > 256 || p.TH * d.stride > 256) return LPDT_ERR_UNSUPPORTED;
-        if (!act_map(&mA, A, d.nodes, d.B, d.H, d.W, p.Kc, p.TB, p.TH, p.TW, d.stride)) return LPDT_ERR_CUDA;
-    } else {
-        if (!act_map(&mA, A, d.nodes, d.B, Ho, Wo, p.Kc, p.TB, p.TH, p.TW, 1)) return LPDT_ERR_CUDA;
-    }
-    if (!weight_map(&mW, Wq, d.nodes, d.Cout, d.R * d.S, d.Cin, mode == 0 ? p.BN : 16)) return LPDT_ERR_CUDA;
+    const int Ha = mode == 0 ? d.H : Ho, Wa = mode == 0 ? d.W : Wo;
+    if (p.merged) { if (!act_map_merged(&mA, A, d.nodes, d.B, Ha, Wa, p.TB, p.TH, p.TW)) return LPDT_ERR_CUDA; }
+    else if (!act_map(&mA, A, d.nodes, d.B, Ha, Wa, p.Kc, p.RBa, p.TB, p.TH, p.TW, estride)) return LPDT_ERR_CUDA;
+    if (mode == 0) { if (!weight_map(&mW, Wq, d.nodes, d.Cout, d.R * d.S, d.Cin, p.RBa, p.BN)) return LPDT_ERR_CUDA; }
+    else if (!weight_map(&mW, Wq, d.nodes, d.Cout, d.R * d.S, d.Cin, p.RBn, p.RBa)) return LPDT_ERR_CUDA;
     size_t smem = 1024 + (size_t)p.stages * stage_bytes;
     if (smem < kMinSmem) smem = kMinSmem;
     static bool attr = false;
@@ -472,6 +529,7 @@ lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const flo
         attr = true;
     }
     const long long tiles = (long long)p.nodes * p.tilesB * p.tilesH * p.tilesW * p.tilesN * p.ncls;
+    if (tiles > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
     const int grid = (int)(tiles < kNumSMs ? tiles : kNumSMs);
     conv_pix_kernel<<<grid, kThreads, smem, st>>>(mA, mW, p);
     LPDT_LAUNCH_CHECK();
@@ -484,22 +542,25 @@ lpdt_status tc_wgrad(const lpdt_conv_desc &d, const int8_t *E, const int8_t *A, 
     WgParams p = {};
     p.nodes = d.nodes; p.B = d.B; p.Ho = Ho; p.Wo = Wo; p.Cin = d.Cin; p.Cout = d.Cout;
     p.R = d.R; p.S = d.S; p.pad = d.pad; p.taps = d.R * d.S; p.stride = d.stride;
-    pick_tile(Ho, Wo, &p.TB, &p.TH, &p.TW);
+    p.RBx = row_bytes_for(d.Cin); p.RBe = row_bytes_for(d.Cout);
+    p.merged = (d.Cin == 16 && d.stride == 1) ? 1 : 0;
+    pick_tile(Ho, Wo, p.merged ? 16 : 128, &p.TB, &p.TH, &p.TW);
+    if (p.TW * d.stride > 256 || p.TH * d.stride > 256) return LPDT_ERR_UNSUPPORTED;
     p.tilesB = (int)ceil_div(d.B, p.TB); p.tilesH = (int)ceil_div(Ho, p.TH); p.tilesW = (int)ceil_div(Wo, p.TW);
     p.kblocks = p.tilesB * p.tilesH * p.tilesW;
-    p.BNc = largest_div16(d.Cout, 256);
+    p.BNc = largest_div(d.Cout, 256, p.RBe);
     p.ngroups = d.Cout / p.BNc;
-    p.total_slices = p.taps * (d.Cin / 16);
-    const int all_tiles = (int)ceil_div(p.total_slices, 8);
-    int mt = 512 / p.BNc;                                   // accumulators that fit in TMEM
-    int mt_smem = ((96 * 1024) / kSliceBytes - p.BNc / 16) / 8;   // stage <= 96 KB -> at least two stages
+    const int G = 128 / p.RBx;
+    p.total_units = p.taps * (d.Cin / p.RBx);
+    const int all_tiles = (int)ceil_div(p.total_units, G);
+    int mt = 512 / p.BNc;                                        // accumulators that fit in TMEM
+    const int mt_smem = (96 * 1024 - 128 * p.BNc) / 16384;       // stage <= 96 KB -> at least two stages
     if (mt > mt_smem) mt = mt_smem;
     if (mt > all_tiles) mt = all_tiles;
     if (mt < 1) return LPDT_ERR_UNSUPPORTED;
     p.mtiles = mt;
     p.mgroups = (int)ceil_div(all_tiles, mt);
-    p.slicesA = mt * 8;
-    const int stage_bytes = (mt * 8 + p.BNc / 16) * kSliceBytes;
+    const int stage_bytes = mt * 16384 + 128 * p.BNc;
     p.stages = (kSmemBudget - 1024) / stage_bytes;
     if (p.stages > 8) p.stages = 8;
     if (p.stages < 2) return LPDT_ERR_UNSUPPORTED;
@@ -513,18 +574,18 @@ lpdt_status tc_wgrad(const lpdt_conv_desc &d, const int8_t *E, const int8_t *A, 
     p.splits = (int)ceil_div(p.kblocks, p.kb_per_split);
     p.acc_out = acc_out; p.dev_status = dev_status;
     CUtensorMap mX, mE;
-    if (p.TW * d.stride > 256 || p.TH * d.stride > 256) return LPDT_ERR_UNSUPPORTED;
-    if (!act_map(&mX, A, d.nodes, d.B, d.H, d.W, d.Cin, p.TB, p.TH, p.TW, d.stride)) return LPDT_ERR_CUDA;
-    if (!act_map(&mE, E, d.nodes, d.B, Ho, Wo, d.Cout, p.TB, p.TH, p.TW)) return LPDT_ERR_CUDA;
-    size_t smem = 1024 + (size_t)p.stages * stage_bytes + 16 * 1024;   // slack: descriptors of a partial M tile read past it
+    if (p.merged) { if (!act_map_merged(&mX, A, d.nodes, d.B, d.H, d.W, p.TB, p.TH, p.TW)) return LPDT_ERR_CUDA; }
+    else if (!act_map(&mX, A, d.nodes, d.B, d.H, d.W, d.Cin, p.RBx, p.TB, p.TH, p.TW, d.stride)) return LPDT_ERR_CUDA;
+    if (!act_map(&mE, E, d.nodes, d.B, Ho, Wo, d.Cout, p.RBe, p.TB, p.TH, p.TW)) return LPDT_ERR_CUDA;
+    size_t smem = 1024 + (size_t)p.stages * stage_bytes;
     if (smem < kMinSmem) smem = kMinSmem;
-    if (smem > 227 * 1024) { p.stages -= 1; smem = 1024 + (size_t)p.stages * stage_bytes + 16 * 1024; }
-    if (p.stages < 2 || smem > 227 * 1024) return LPDT_ERR_UNSUPPORTED;
+    if (smem > 227 * 1024) return LPDT_ERR_UNSUPPORTED;
     static bool attr = false;
     if (!attr) {
         LPDT_CUDA(cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr = true;
     }
+    if (d.nodes > 65535 || p.mgroups * p.ngroups > 65535) return LPDT_ERR_UNSUPPORTED;
     conv_wgrad_kernel<<<dim3(p.splits, p.mgroups * p.ngroups, d.nodes), kThreads, smem, st>>>(mX, mE, p);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
