@@ -74,7 +74,9 @@ struct SharedCtl {
 };
 
 struct TileCoord { int cls, tw, th, tb, nt, node; };
-// tile order: node, N tile, batch tile, row tile, column tile, class (fastest)
+// tile order: node, N tile, batch tile, row tile, column tile, class (fastest).  A CTA walks
+// consecutive tiles, so the coordinate is decoded once and then advanced like an odometer
+// (the single-thread roles are instruction-bound: no divisions in their loops).
 __device__ __forceinline__ TileCoord decode_tile(const PixParams &p, int tile) {
     TileCoord c; int t = tile;
     c.cls = t % p.ncls; t /= p.ncls;
@@ -83,6 +85,14 @@ __device__ __forceinline__ TileCoord decode_tile(const PixParams &p, int tile) {
     c.tb = t % p.tilesB; t /= p.tilesB;
     c.nt = t % p.tilesN; c.node = t / p.tilesN;
     return c;
+}
+__device__ __forceinline__ void next_tile(const PixParams &p, TileCoord &c) {
+    if (++c.cls < p.ncls) return; c.cls = 0;
+    if (++c.tw < p.tilesW) return; c.tw = 0;
+    if (++c.th < p.tilesH) return; c.th = 0;
+    if (++c.tb < p.tilesB) return; c.tb = 0;
+    if (++c.nt < p.tilesN) return; c.nt = 0;
+    ++c.node;
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -117,44 +127,62 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         if (lane == 0) {
             tma_prefetch_desc(&mapA); tma_prefetch_desc(&mapW);
             uint32_t g = 0;     // running stage counter
-            for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; ++tile) {
-                const TileCoord c = decode_tile(p, tile);
+            int st = 0; uint32_t ph = 0;
+            TileCoord c = decode_tile(p, tile_lo);
+            const int nj = p.BN / p.RBn, bj_stride = p.U * p.RBa * p.RBn, bu_stride = p.RBa * p.RBn;
+            for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; ++tile, next_tile(p, c)) {
                 const int n0 = c.nt * p.BN, w0 = c.tw * p.TW * p.cmul, h0 = c.th * p.TH * p.cmul, b0 = c.tb * p.TB;
+                const int wrow = c.node * p.w_rows_per_node;
                 const TapTable &tt = p.tt[c.cls];
+                int ti = 0, chunk = 0;                      // running (tap, channel chunk) of the next unit
                 for (int it = 0; it < p.cls_iters[c.cls]; ++it, ++g) {
-                    const int st = g % p.stages;
-                    const uint32_t ph = (g / p.stages) & 1;
                     if (!mbar_wait(smem_u32(&ctl->empty[st]), ph ^ 1, &ctl->abort_flag, p.dev_status)) break;
                     const uint32_t full = smem_u32(&ctl->full[st]);
                     mbar_expect_tx(full, stage_bytes);
-                    const uint32_t a_st = smem_u32(data + (size_t)st * stage_bytes);
-                    const uint32_t b_st = a_st + a_bytes;
+                    uint32_t a_dst = smem_u32(data + (size_t)st * stage_bytes);
+                    uint32_t b_dst = a_dst + a_bytes;
                     for (int u = 0; u < p.U; ++u) {
-                        const int kap = it * p.U + u;
-                        const int ti = kap / cpt, chunk = kap % cpt;
                         int hc = -(1 << 20), wc = 0, tap = 1 << 20;   // phantom unit: boxes out of range -> zeros
                         if (ti < tt.ntaps) { hc = h0 + tt.dh[ti]; wc = w0 + tt.dw[ti]; tap = tt.wtap[ti]; }
-                        if (p.merged) tma_load_4d(a_st + u * a_unit, &mapA, full, wc * 16, hc, b0, c.node);
-                        else tma_load_5d(a_st + u * a_unit, &mapA, full, chunk * p.RBa, wc, hc, b0, c.node);
+                        if (p.merged) tma_load_4d(a_dst, &mapA, full, wc * 16, hc, b0, c.node);
+                        else tma_load_5d(a_dst, &mapA, full, chunk * p.RBa, wc, hc, b0, c.node);
                         if (p.mode == 0) {
-                            tma_load_3d(b_st + u * b_unit, &mapW, full, chunk * p.RBa, tap,
-                                        c.node * p.w_rows_per_node + n0);
+                            tma_load_3d(b_dst, &mapW, full, chunk * p.RBa, tap, wrow + n0);
+                            b_dst += b_unit;
                         } else {
                             // N side in chunks of RBn bytes; this unit's RBa weight rows go at row u*RBa of each chunk
-                            for (int j = 0; j < p.BN / p.RBn; ++j)
-                                tma_load_3d(b_st + j * (p.U * p.RBa * p.RBn) + u * p.RBa * p.RBn, &mapW, full,
-                                            n0 + j * p.RBn, tap, c.node * p.w_rows_per_node + chunk * p.RBa);
+                            for (int j = 0; j < nj; ++j)
+                                tma_load_3d(b_dst + j * bj_stride, &mapW, full, n0 + j * p.RBn, tap,
+                                            wrow + chunk * p.RBa);
+                            b_dst += bu_stride;
                         }
+                        a_dst += a_unit;
+                        if (++chunk == cpt) { chunk = 0; ++ti; }
                     }
+                    if (++st == p.stages) { st = 0; ph ^= 1; }
                 }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = idesc_i8(128, p.BN, 0, p.mode == 0 ? 0 : 1);
-            const uint32_t la = layout_code(p.RBa), ln = layout_code(p.RBn);
-            const int n_mma = p.U * p.RBa / 32;
+            // Descriptor templates (start address 0); the loop only adds address increments.
+            const uint64_t a_tpl = (p.RBa == 16) ? smem_desc(0, a_unit, 128, 0)
+                                                 : smem_desc(0, 16, 8 * p.RBa, layout_code(p.RBa));
+            uint64_t b_tpl;
+            if (p.mode == 0) b_tpl = (p.RBa == 16) ? smem_desc(0, b_unit, 128, 0) : smem_desc(0, 16, 8 * p.RBa, layout_code(p.RBa));
+            else b_tpl = (p.RBn == 16) ? smem_desc(0, 128, p.U * p.RBa * 16, 0)
+                                       : smem_desc(0, p.U * p.RBa * p.RBn, 8 * p.RBn, layout_code(p.RBn));
+            // per-MMA (32 K bytes) and per-unit address steps, in 16-byte units
+            const int n_units = (p.RBa == 16) ? p.U / 2 : p.U;
+            const int steps = (p.RBa == 16) ? 1 : p.RBa / 32;
+            const uint32_t a_step = 2, a_unit_step = (p.RBa == 16) ? (2 * a_unit) >> 4 : (a_unit - p.RBa) >> 4;
+            uint32_t b_step, b_unit_step;
+            if (p.mode == 0) { b_step = 2; b_unit_step = (p.RBa == 16) ? (2 * b_unit) >> 4 : (b_unit - p.RBa) >> 4; }
+            else { b_step = (32 * p.RBn) >> 4; b_unit_step = (p.RBa == 16) ? b_step : 0; }
             uint32_t g = 0, tcount = 0;
+            int st = 0; uint32_t ph = 0;
+            int cls = tile_lo % p.ncls;
             for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; ++tile, ++tcount) {
                 const int acc = tcount & 1;
                 const uint32_t aph = (tcount >> 1) & 1;
@@ -162,30 +190,25 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * p.BN;
                 bool ok = true;
-                const int iters = p.cls_iters[tile % p.ncls];
+                const int iters = p.cls_iters[cls];
+                if (++cls == p.ncls) cls = 0;
+                uint32_t accum = 0;
                 for (int it = 0; it < iters; ++it, ++g) {
-                    const int st = g % p.stages;
-                    const uint32_t ph = (g / p.stages) & 1;
                     if (!mbar_wait(smem_u32(&ctl->full[st]), ph, &ctl->abort_flag, p.dev_status)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_st = smem_u32(data + (size_t)st * stage_bytes);
-                    const uint32_t b_st = a_st + a_bytes;
-                    for (int m = 0; m < n_mma; ++m) {
-                        const int kb = m * 32;                                   // K byte offset within the stage
-                        uint64_t ad, bd;
-                        if (p.RBa == 16) ad = smem_desc(a_st + (kb / 16) * a_unit, a_unit, 128, 0);
-                        else ad = smem_desc(a_st + (kb / p.RBa) * a_unit + kb % p.RBa, 16, 8 * p.RBa, la);
-                        if (p.mode == 0) {
-                            if (p.RBa == 16) bd = smem_desc(b_st + (kb / 16) * b_unit, b_unit, 128, 0);
-                            else bd = smem_desc(b_st + (kb / p.RBa) * b_unit + kb % p.RBa, 16, 8 * p.RBa, la);
-                        } else {
-                            // MN-major: K rows of RBn bytes; N chunks U*RBa rows apart
-                            if (p.RBn == 16) bd = smem_desc(b_st + kb * 16, 128, p.U * p.RBa * 16, 0);
-                            else bd = smem_desc(b_st + kb * p.RBn, p.U * p.RBa * p.RBn, 8 * p.RBn, ln);
+                    uint32_t a_lo = a_st >> 4, b_lo = (a_st + a_bytes) >> 4;
+                    for (int u = 0; u < n_units; ++u) {
+                        for (int k = 0; k < steps; ++k) {
+                            mma_i8(d_tmem, a_tpl | (a_lo & 0x3FFFu), b_tpl | (b_lo & 0x3FFFu), idesc, accum);
+                            accum = 1;
+                            a_lo += a_step; b_lo += b_step;
                         }
-                        mma_i8(d_tmem, ad, bd, idesc, (it | m) != 0);
+                        if (p.RBa == 16) { a_lo += a_unit_step - a_step; b_lo += b_unit_step - b_step; }
+                        else { a_lo += a_unit_step; b_lo += b_unit_step; }
                     }
                     mma_commit(smem_u32(&ctl->empty[st]));
+                    if (++st == p.stages) { st = 0; ph ^= 1; }
                 }
                 if (!ok) break;
                 mma_commit(smem_u32(&ctl->tmem_full[acc]));
@@ -196,19 +219,20 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         const int row = q * 32 + lane;                // tile row = pixel within the tile
         const int pw = row % p.TW, phh = (row / p.TW) % p.TH, pb = row / (p.TW * p.TH);
         uint32_t tcount = 0;
-        for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; ++tile, ++tcount) {
-            const TileCoord c = decode_tile(p, tile);
+        TileCoord c = decode_tile(p, tile_lo);
+        int sc_node = -1; float sc = 0.f;
+        for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; ++tile, ++tcount, next_tile(p, c)) {
             const int n0 = c.nt * p.BN;
             const int w = (c.tw * p.TW + pw) * p.out_mul + p.cls_pw[c.cls];
             const int h = (c.th * p.TH + phh) * p.out_mul + p.cls_ph[c.cls];
             const int b = c.tb * p.TB + pb;
             const bool valid = (w < p.Wout) && (h < p.Hout) && (b < p.B);
+            if (p.Y && c.node != sc_node) { sc_node = c.node; sc = __fmul_rn(p.s1[c.node], p.s2[c.node]); }
             const int acc = tcount & 1;
             const uint32_t aph = (tcount >> 1) & 1;
             if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), aph, &ctl->abort_flag, p.dev_status)) break;
             tc_fence_after();
             const long long pix = (((long long)c.node * p.B + b) * p.Hout + h) * p.Wout + w;
-            const float sc = p.Y ? __fmul_rn(p.s1[c.node], p.s2[c.node]) : 0.f;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * p.BN;
             for (int cc = 0; cc < p.BN; cc += 16) {
                 uint32_t v[16];
