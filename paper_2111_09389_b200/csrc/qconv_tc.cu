@@ -315,54 +315,58 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     if (warp == 0) {
         if (lane == 0) {
             tma_prefetch_desc(&mapX); tma_prefetch_desc(&mapE);
-            uint32_t g = 0;
-            for (int kb = kb0; kb < kb1; ++kb, ++g) {
-                int t = kb;
-                const int tw = t % p.tilesW; t /= p.tilesW;
-                const int th = t % p.tilesH; const int tb = t / p.tilesH;
+            int st = 0; uint32_t ph = 0;
+            int tw = kb0 % p.tilesW, th = (kb0 / p.tilesW) % p.tilesH, tb = kb0 / (p.tilesW * p.tilesH);
+            const int tap0 = mu0 / cpt, chunk0 = mu0 % cpt, r0 = tap0 / p.S, s0 = tap0 % p.S;
+            for (int kb = kb0; kb < kb1; ++kb) {
                 const int w0 = tw * p.TW, h0 = th * p.TH, b0 = tb * p.TB;
-                const int st = g % p.stages;
-                const uint32_t ph = (g / p.stages) & 1;
                 if (!mbar_wait(smem_u32(&ctl->empty[st]), ph ^ 1, &ctl->abort_flag, p.dev_status)) break;
                 const uint32_t full = smem_u32(&ctl->full[st]);
                 mbar_expect_tx(full, nX * x_unit + nE * e_unit);
-                const uint32_t x_st = smem_u32(data + (size_t)st * stage_bytes);
-                const uint32_t e_st = x_st + x_region;
-                for (int c = 0; c < nE; ++c)
-                    tma_load_5d(e_st + c * e_unit, &mapE, full, n0 + c * p.RBe, w0, h0, b0, node);
-                for (int i = 0; i < nX; ++i) {
-                    const int mu = mu0 + i, tap = mu / cpt, chunk = mu % cpt;
-                    const int r = tap / p.S, s = tap % p.S;
+                uint32_t x_dst = smem_u32(data + (size_t)st * stage_bytes);
+                uint32_t e_dst = x_dst + x_region;
+                for (int c = 0; c < nE; ++c, e_dst += e_unit)
+                    tma_load_5d(e_dst, &mapE, full, n0 + c * p.RBe, w0, h0, b0, node);
+                int chunk = chunk0, r = r0, s = s0;
+                for (int i = 0; i < nX; ++i, x_dst += x_unit) {
                     const int wc = w0 * p.stride + s - p.pad, hc = h0 * p.stride + r - p.pad;
-                    if (p.merged) tma_load_4d(x_st + i * x_unit, &mapX, full, wc * 16, hc, b0, node);
-                    else tma_load_5d(x_st + i * x_unit, &mapX, full, chunk * p.RBx, wc, hc, b0, node);
+                    if (p.merged) tma_load_4d(x_dst, &mapX, full, wc * 16, hc, b0, node);
+                    else tma_load_5d(x_dst, &mapX, full, chunk * p.RBx, wc, hc, b0, node);
+                    if (++chunk == cpt) { chunk = 0; if (++s == p.S) { s = 0; ++r; } }
                 }
+                if (++tw == p.tilesW) { tw = 0; if (++th == p.tilesH) { th = 0; ++tb; } }
+                if (++st == p.stages) { st = 0; ph ^= 1; }
             }
         }
     } else if (warp == 1) {
         if (lane == 0) {
             const uint32_t idesc = idesc_i8(128, p.BNc, 1, 1);
-            const uint32_t lx = layout_code(p.RBx), le = layout_code(p.RBe);
-            uint32_t g = 0;
+            const uint64_t a_tpl = (p.RBx == 16) ? smem_desc(0, 128, x_unit, 0)
+                                                 : smem_desc(0, x_unit, 8 * p.RBx, layout_code(p.RBx));
+            const uint64_t b_tpl = (p.RBe == 16) ? smem_desc(0, 128, e_unit, 0)
+                                                 : smem_desc(0, e_unit, 8 * p.RBe, layout_code(p.RBe));
+            const uint32_t a_step = (32 * p.RBx) >> 4, b_step = (32 * p.RBe) >> 4;   // 32 pixel rows per MMA
+            uint32_t accum = 0;
+            int st = 0; uint32_t ph = 0;
             bool ok = true;
-            for (int kb = kb0; kb < kb1; ++kb, ++g) {
-                const int st = g % p.stages;
-                const uint32_t ph = (g / p.stages) & 1;
+            for (int kb = kb0; kb < kb1; ++kb) {
                 if (!mbar_wait(smem_u32(&ctl->full[st]), ph, &ctl->abort_flag, p.dev_status)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t x_st = smem_u32(data + (size_t)st * stage_bytes);
-                const uint32_t e_st = x_st + x_region;
-                for (int t = 0; t < p.mtiles; ++t)
-                    for (int kk = 0; kk < 4; ++kk) {       // 32 pixel rows per MMA
-                        const uint64_t ad = (p.RBx == 16)
-                            ? smem_desc(x_st + t * 16384 + kk * 512, 128, x_unit, 0)
-                            : smem_desc(x_st + t * 16384 + kk * 32 * p.RBx, x_unit, 8 * p.RBx, lx);
-                        const uint64_t bd = (p.RBe == 16)
-                            ? smem_desc(e_st + kk * 512, 128, e_unit, 0)
-                            : smem_desc(e_st + kk * 32 * p.RBe, e_unit, 8 * p.RBe, le);
-                        mma_i8(tmem_base + t * p.BNc, ad, bd, idesc, (g | (uint32_t)kk) != 0);
+                const uint32_t e_lo0 = (x_st + x_region) >> 4;
+                uint32_t a_tile = x_st >> 4, d_tmem = tmem_base;
+                for (int t = 0; t < p.mtiles; ++t) {
+                    uint32_t a_lo = a_tile, b_lo = e_lo0;
+#pragma unroll
+                    for (int kk = 0; kk < 4; ++kk) {
+                        mma_i8(d_tmem, a_tpl | (a_lo & 0x3FFFu), b_tpl | (b_lo & 0x3FFFu), idesc, accum | (uint32_t)kk);
+                        a_lo += a_step; b_lo += b_step;
                     }
+                    a_tile += 16384 >> 4; d_tmem += p.BNc;
+                }
+                accum = 1;
                 mma_commit(smem_u32(&ctl->empty[st]));
+                if (++st == p.stages) { st = 0; ph ^= 1; }
             }
             if (ok) mma_commit(smem_u32(&ctl->tmem_full[0]));
         }
@@ -382,11 +386,15 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                     tmem_ld_32x16(t_row + c, v);
                     tmem_ld_wait();
                     if (valid) {
+                        int32_t *dst = p.acc_out + (((long long)node * p.Cout + n0 + c) * p.taps + tap) * p.Cin + ci;
+                        const long long cstride = (long long)p.taps * p.Cin;
+                        if (p.splits == 1) {
 #pragma unroll
-                        for (int k = 0; k < 16; ++k) {
-                            const int co = n0 + c + k;
-                            if ((int)v[k] != 0)
-                                atomicAdd(p.acc_out + (((long long)node * p.Cout + co) * p.taps + tap) * p.Cin + ci, (int)v[k]);
+                            for (int k = 0; k < 16; ++k) dst[k * cstride] = (int)v[k];
+                        } else {
+#pragma unroll
+                            for (int k = 0; k < 16; ++k)
+                                if ((int)v[k] != 0) atomicAdd(dst + k * cstride, (int)v[k]);
                         }
                     }
                 }
@@ -591,7 +599,7 @@ lpdt_status tc_wgrad(const lpdt_conv_desc &d, const int8_t *E, const int8_t *A, 
     p.tmem_cols = pow2_at_least(mt * p.BNc);
     if (p.tmem_cols > 512) return LPDT_ERR_UNSUPPORTED;
     long long ctas_fixed = (long long)d.nodes * p.mgroups * p.ngroups;
-    int splits = (int)ceil_div(2 * kNumSMs, ctas_fixed);
+    int splits = ctas_fixed >= kNumSMs ? 1 : (int)ceil_div(2 * kNumSMs, ctas_fixed);
     if (splits > p.kblocks) splits = p.kblocks;
     if (splits < 1) splits = 1;
     p.kb_per_split = (int)ceil_div(p.kblocks, splits);
