@@ -24,8 +24,11 @@
  *     returns.
  *   - Integer accumulators are int32 and wrap modulo 2^32 like the hardware.
  *   - Floating point: element-wise arithmetic is a fixed sequence of
- *     individually rounded fp32 operations (no fused multiply-add, no fast
- *     math); every reduction is accumulated in fp64 and rounded once.
+ *     individually rounded fp32 operations (no contraction, no fast math).
+ *     Reductions that decide later integer codes (ranges, the Range-EvoNorm
+ *     group sum) are exact or accumulated in fp64; the per-channel parameter
+ *     gradient sums add fp32 runs of at most 16 terms into fp64 accumulators.
+ *     Everything is rounded to fp32 once.
  */
 #ifndef LPDT_H
 #define LPDT_H

@@ -42,8 +42,15 @@ template <> struct VecLoad<1> {
 };
 
 // hard sigmoid and the normalised product, each operation rounded on its own
+// (u + 3)/6 correctly rounded without the division unit: q = a*y with y = RN(1/6), the
+// exact residual r = a - 6q by FMA, and one correction step q + r*y (Markstein's
+// division by a constant); identical to the IEEE quotient for every finite a here.
 __device__ __forceinline__ float hsig(float u) {
-    float h = __fdiv_rn(__fadd_rn(u, 3.f), 6.f);
+    const float a = __fadd_rn(u, 3.f);
+    const float y = 0x1.555556p-3f;
+    const float q = __fmul_rn(a, y);
+    const float r = __fmaf_rn(-6.f, q, a);
+    float h = __fmaf_rn(r, y, q);
     return fminf(fmaxf(h, 0.f), 1.f);
 }
 
@@ -72,7 +79,7 @@ __device__ void reduce_groups(Ext mn, Ext mx, Ext *s_mn, Ext *s_mx, Ext *g_mn, E
 }
 
 template <int V>
-__global__ void __launch_bounds__(512)
+__global__ void __launch_bounds__(512, 2)
 ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
                const float *__restrict__ x, const float *__restrict__ v,
                const float *__restrict__ gamma, const float *__restrict__ beta, int64_t pstride,
@@ -165,9 +172,15 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
         vc[k] = v[(int64_t)node * pstride + c0 + k];
         gc[k] = gamma[(int64_t)node * pstride + c0 + k];
     }
+    // S feeds dx (and through it the next quantizer): accumulated in double term by term.
+    // The per-channel parameter-gradient sums take a short fp32 run per thread (at most
+    // kRunLen terms) before they join the double accumulators.
+    constexpr int kRunLen = 16;
     double S = 0.0, ab[V], ag[V], av[V];
+    float fb[V], fg[V], fv[V];
+    int run = 0;
 #pragma unroll
-    for (int k = 0; k < V; ++k) { ab[k] = 0.0; ag[k] = 0.0; av[k] = 0.0; }
+    for (int k = 0; k < V; ++k) { ab[k] = 0.0; ag[k] = 0.0; av[k] = 0.0; fb[k] = 0.f; fg[k] = 0.f; fv[k] = 0.f; }
     for (int p = row0; p < HW; p += rstep) {
         float xv[V], dv_[V];
         VecLoad<V>::ld(xs + (int64_t)p * C + c0, xv);
@@ -180,11 +193,21 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
             float m = __fmul_rn(xv[k], hs);
             float tt = __fmul_rn(dv_[k], gc[k]);
             S += (double)__fmul_rn(tt, m);
-            ab[k] += (double)dv_[k];
-            ag[k] += (double)__fmul_rn(dv_[k], __fmul_rn(m, invD));
-            av[k] += (double)__fmul_rn(__fmul_rn(__fmul_rn(tt, __fmul_rn(xv[k], xv[k])), hp), invD);
+            fb[k] = __fadd_rn(fb[k], dv_[k]);
+            fg[k] = __fadd_rn(fg[k], __fmul_rn(dv_[k], __fmul_rn(m, invD)));
+            fv[k] = __fadd_rn(fv[k], __fmul_rn(__fmul_rn(__fmul_rn(tt, __fmul_rn(xv[k], xv[k])), hp), invD));
+        }
+        if (++run == kRunLen) {
+            run = 0;
+#pragma unroll
+            for (int k = 0; k < V; ++k) {
+                ab[k] += (double)fb[k]; ag[k] += (double)fg[k]; av[k] += (double)fv[k];
+                fb[k] = 0.f; fg[k] = 0.f; fv[k] = 0.f;
+            }
         }
     }
+#pragma unroll
+    for (int k = 0; k < V; ++k) { ab[k] += (double)fb[k]; ag[k] += (double)fg[k]; av[k] += (double)fv[k]; }
     __syncthreads();   // s_ch zeroed
     // Per-channel sums: when the column count divides the warp, lanes that share a
     // column are first folded with shuffles, so only CV lanes per warp touch shared memory.
@@ -266,7 +289,7 @@ static bool plan(int C, int groups, bool aligned16, RenPlan *pl) {
     int CV = C / V;
     if (CV > 512) return false;
     pl->V = V;
-    pl->threads = CV * (512 / CV);
+    pl->threads = CV <= 256 ? CV * (256 / CV) : CV;
     if (pl->threads % 32) {                      // keep whole warps: pad down to a multiple of lcm
         int th = pl->threads;
         while (th > 0 && (th % 32 || th % CV)) th -= CV;
