@@ -3,12 +3,13 @@
 // One CTA per (node, sample).  Every thread owns a fixed vector-column of V
 // channels and walks the pixels, so global accesses are fully coalesced 16-byte
 // loads and the thread's channel parameters and group live in registers.
-// Pass 1 finds the per-group extrema (and, backward, the group sum S and the
-// per-channel gradient sums); a warp-shuffle reduction with a
-// (value, lowest index) comparator merges the threads of a group.  Pass 2
-// re-reads the sample (an L2 hit: a sample is at most a few hundred KB) and
-// writes the output.  Both kernels are HBM-bound: forward moves 4 B in + 4 B
-// out per element, backward 8 B in + 4 B out.
+// Forward: pass 1 finds the per-group extrema; a warp-shuffle reduction with a
+// (value, lowest index) comparator merges the threads of a group; pass 2 re-reads
+// the sample (an L2 hit: a sample is at most a few hundred KB) and writes the
+// output.  Backward is a single pass: the local term of dx is written while the
+// group sum S and the per-channel gradient sums accumulate, and S is applied
+// afterwards at the two extremum positions of each group.  Both kernels are
+// HBM-bound: forward moves 4 B in + 4 B out per element, backward 8 B in + 4 B out.
 #include <math.h>
 #include "common.cuh"
 
@@ -182,7 +183,7 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
 #pragma unroll
     for (int k = 0; k < V; ++k) { ab[k] = 0.0; ag[k] = 0.0; av[k] = 0.0; fb[k] = 0.f; fg[k] = 0.f; fv[k] = 0.f; }
     for (int p = row0; p < HW; p += rstep) {
-        float xv[V], dv_[V];
+        float xv[V], dv_[V], o[V];
         VecLoad<V>::ld(xs + (int64_t)p * C + c0, xv);
         VecLoad<V>::ld(dys + (int64_t)p * C + c0, dv_);
 #pragma unroll
@@ -193,10 +194,12 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
             float m = __fmul_rn(xv[k], hs);
             float tt = __fmul_rn(dv_[k], gc[k]);
             S += (double)__fmul_rn(tt, m);
+            o[k] = __fmul_rn(__fmul_rn(tt, __fadd_rn(hs, __fmul_rn(u, hp))), invD);
             fb[k] = __fadd_rn(fb[k], dv_[k]);
             fg[k] = __fadd_rn(fg[k], __fmul_rn(dv_[k], __fmul_rn(m, invD)));
             fv[k] = __fadd_rn(fv[k], __fmul_rn(__fmul_rn(__fmul_rn(tt, __fmul_rn(xv[k], xv[k])), hp), invD));
         }
+        VecLoad<V>::st(dxs + (int64_t)p * C + c0, o);
         if (++run == kRunLen) {
             run = 0;
 #pragma unroll
@@ -243,29 +246,21 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
     }
     for (int i = t; i < 3 * C; i += T) atomicAdd(&acc[(int64_t)node * 3 * C + i], s_ch[i]);
     __syncthreads();
-    const int amx = argmax[sg], amn = argmin[sg];
-    float coef = __fmul_rn(Cst, (float)g_S[grp]);
-    coef = __fmul_rn(coef, invD);
-    coef = __fmul_rn(coef, invD);
-    if (amx == amn) coef = 0.f;
-    for (int p = row0; p < HW; p += rstep) {
-        float xv[V], dv_[V], o[V];
-        VecLoad<V>::ld(xs + (int64_t)p * C + c0, xv);
-        VecLoad<V>::ld(dys + (int64_t)p * C + c0, dv_);
-#pragma unroll
-        for (int k = 0; k < V; ++k) {
-            float u = __fmul_rn(vc[k], xv[k]);
-            float hs = hsig(u);
-            float hp = (u > -3.f && u < 3.f) ? sixth : 0.f;
-            float tt = __fmul_rn(dv_[k], gc[k]);
-            float inner = __fadd_rn(hs, __fmul_rn(u, hp));
-            float r = __fmul_rn(__fmul_rn(tt, inner), invD);
-            int idx = p * C + c0 + k;
-            if (idx == amx) r = __fsub_rn(r, coef);
-            if (idx == amn) r = __fadd_rn(r, coef);
-            o[k] = r;
+    // The group sum only enters dx at the two extremum positions: one thread per group
+    // applies the correction to the local term already stored there (same operation order
+    // as a fused evaluation: local term first, then -coef at argmax, +coef at argmin).
+    if (t < groups) {
+        const int64_t sgg = sample * groups + t;
+        const int amx = argmax[sgg], amn = argmin[sgg];
+        if (amx != amn) {
+            const float rng_g = __fsub_rn(gmax[sgg], gmin[sgg]);
+            const float invDg = __fdiv_rn(1.f, __fadd_rn(__fmul_rn(Cst, rng_g), eps));
+            float coef = __fmul_rn(Cst, (float)g_S[t]);
+            coef = __fmul_rn(coef, invDg);
+            coef = __fmul_rn(coef, invDg);
+            dxs[amx] = __fsub_rn(dxs[amx], coef);
+            dxs[amn] = __fadd_rn(dxs[amn], coef);
         }
-        VecLoad<V>::st(dxs + (int64_t)p * C + c0, o);
     }
 }
 
