@@ -99,6 +99,33 @@ lpdt_status lpdt_dequantize(const int8_t *q, int32_t nodes, int64_t n_per_node,
                             float *y, int64_t y_node_stride, void *stream);
 
 /* ---------------------------------------------------------------------------
+ * lpdt_quantize_static - lpdt_quantize without a caller workspace.
+ * (The paper has no counterpart: this entry point exists for integration only.)
+ *
+ * For callers that cannot hand the library any device scratch: a training loop
+ * on a device whose buffers were all fixed at start-up, or code called from a
+ * host application that owns the device memory pool and does not allow device
+ * allocation where this call sits.  The per-node range words live in an 8 KB
+ * array inside the library image instead (held by every GPU that loads the
+ * library, until the process exits).  The call allocates nothing.
+ *
+ * Arguments, results and rounding are those of lpdt_quantize; ws/ws_bytes are
+ * gone.  Limits and rules:
+ *   - nodes <= LPDT_QUANTIZE_STATIC_MAX_NODES, otherwise LPDT_ERR_WORKSPACE
+ *     (the built-in scratch is too small) and nothing is enqueued.
+ *   - The first call on each device looks up the array's device address (with
+ *     that device current); make that first call before any stream capture.
+ *   - All calls share the one array, so two calls whose kernels may overlap on
+ *     the GPU (different streams, no ordering between them) race; calls on one
+ *     stream, or otherwise ordered, are safe.  The words a call uses are cleared
+ *     at its start; it does not depend on what the previous call left behind.
+ */
+#define LPDT_QUANTIZE_STATIC_MAX_NODES 1024
+lpdt_status lpdt_quantize_static(const float *x, int32_t nodes, int64_t n_per_node, int64_t x_node_stride,
+                                 lpdt_qmode mode, lpdt_round rounding, uint64_t seed, uint32_t ctr_offset,
+                                 int8_t *q, float *scale, int32_t *zero_point, void *stream);
+
+/* ---------------------------------------------------------------------------
  * Quantized contractions on symmetric int8 operands (Section 3: the forward
  * product and both backward products run on 8-bit operands; the operation
  * count table's Conv and Linear rows count the three alike).  int32

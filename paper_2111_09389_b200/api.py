@@ -13,7 +13,7 @@ from ._lib import ConvDesc, lib
 
 # Kernels each entry point enqueues (memsets not counted); KERNEL_LAUNCHES accumulates them.
 KERNELS_PER_CALL = {
-    "lpdt_quantize": 2, "lpdt_dequantize": 1, "lpdt_qconv_fwd": 1, "lpdt_qconv_bwd_data": 2,
+    "lpdt_quantize": 2, "lpdt_quantize_static": 2, "lpdt_dequantize": 1, "lpdt_qconv_fwd": 1, "lpdt_qconv_bwd_data": 2,
     "lpdt_qconv_bwd_weight": 2, "lpdt_range_evonorm_fwd": 1, "lpdt_range_evonorm_bwd": 2,
     "lpdt_gossip_mix": 2, "lpdt_sgd_update": 1, "lpdt_residual_add": 1, "lpdt_residual_add_bwd": 1,
     "lpdt_avgpool": 1, "lpdt_avgpool_bwd": 1, "lpdt_maxpool2x2": 1, "lpdt_maxpool2x2_bwd": 1,
@@ -95,6 +95,15 @@ def lpdt_quantize(x, nodes, n_per_node, x_node_stride, q, scale, ws, mode=0, rou
     _check("lpdt_quantize", lib().lpdt_quantize(_ptr(x), nodes, n_per_node, x_node_stride, mode, rounding,
                                                 seed, ctr_offset, _ptr(q), _ptr(scale), _ptr(zero_point),
                                                 p, nb, _stream()))
+
+
+def lpdt_quantize_static(x, nodes, n_per_node, x_node_stride, q, scale, mode=0, rounding=0, seed=0,
+                         ctr_offset=0, zero_point=None):
+    """lpdt_quantize for callers without device scratch: the range words live inside the
+    library.  At most 1024 nodes; calls that may overlap on the GPU must be ordered."""
+    _check("lpdt_quantize_static", lib().lpdt_quantize_static(
+        _ptr(x), nodes, n_per_node, x_node_stride, mode, rounding, seed, ctr_offset, _ptr(q), _ptr(scale),
+        _ptr(zero_point), _stream()))
 
 
 def lpdt_dequantize(q, nodes, n_per_node, scale, y, y_node_stride=None, zero_point=None):

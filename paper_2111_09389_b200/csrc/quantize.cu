@@ -239,3 +239,56 @@ extern "C" lpdt_status lpdt_dequantize(const int8_t *q, int32_t nodes, int64_t n
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }
+
+// ---------------------------------------------------------------------------
+// Quantizer for callers that own no device scratch.
+//
+// lpdt_quantize needs a few bytes of caller-provided scratch for the per-node
+// range words.  Some users of this library cannot supply any: an edge-device
+// training loop that was given a fixed set of buffers at start-up and has no
+// allocator afterwards, or a plug-in called from a host application whose device
+// memory belongs to that application's own pool and which forbids device
+// allocation on its hot path (cudaMalloc also synchronises the whole device).
+// For them the range words live in the array below, which is part of the loaded
+// library image: every GPU that loads the library holds these 8 KB until the
+// process exits.
+//
+// In host code `g_static_range_words` is only a handle for the symbol, not a device
+// address, so its address on the current device is looked up once per device with
+// cudaGetSymbolAddress and that pointer is what the kernels receive.
+constexpr int kStaticMaxNodes = LPDT_QUANTIZE_STATIC_MAX_NODES;
+static __device__ __align__(256) uint32_t g_static_range_words[2 * kStaticMaxNodes];
+
+constexpr int kMaxDevices = 64;
+static uint32_t *g_static_range_ptr[kMaxDevices] = {};
+
+static lpdt_status static_range_words(uint32_t **out) {
+    int dev = -1;
+    LPDT_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return LPDT_ERR_UNSUPPORTED;
+    if (!g_static_range_ptr[dev]) {
+        uint32_t *p = nullptr;
+        if (cudaGetSymbolAddress((void **)&p, g_static_range_words) != cudaSuccess || !p) {
+            (void)cudaGetLastError();
+            return LPDT_ERR_CUDA;
+        }
+        g_static_range_ptr[dev] = p;
+    }
+    *out = g_static_range_ptr[dev];
+    return LPDT_OK;
+}
+
+extern "C" lpdt_status lpdt_quantize_static(const float *x, int32_t nodes, int64_t n_per_node,
+                                            int64_t x_node_stride, lpdt_qmode mode, lpdt_round rounding,
+                                            uint64_t seed, uint32_t ctr_offset, int8_t *q, float *scale,
+                                            int32_t *zero_point, void *stream) {
+    LPDT_CHECK_ARG(nodes >= 0);
+    if (nodes > kStaticMaxNodes) return LPDT_ERR_WORKSPACE;     // the built-in scratch holds 1024 nodes
+    uint32_t *words = nullptr;
+    lpdt_status s = static_range_words(&words);
+    if (s != LPDT_OK) return s;
+    // Same two passes as lpdt_quantize; it zeroes the words it uses before the range pass,
+    // so whatever the previous call left in the array does not matter.
+    return lpdt_quantize(x, nodes, n_per_node, x_node_stride, mode, rounding, seed, ctr_offset, q, scale,
+                         zero_point, words, sizeof(uint32_t) * 2 * kStaticMaxNodes, stream);
+}
