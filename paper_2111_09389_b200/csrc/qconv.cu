@@ -54,6 +54,21 @@ static bool tc_enabled() {
     return !disabled;
 }
 static bool use_tc(const lpdt_conv_desc &d) { return tc_enabled() && tc::tc_supported(d); }
+// LPDT_DISABLE_HALO=1 keeps 16-channel layers on the general tensor-core kernel.
+static bool use_halo(const lpdt_conv_desc &d, int mode) {
+    static int disabled = -1;
+    if (disabled < 0) {
+        const char *e = getenv("LPDT_DISABLE_HALO");
+        disabled = (e && e[0] == '1') ? 1 : 0;
+    }
+    return !disabled && tc::halo_supported(d, mode);
+}
+static lpdt_status run_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const float *s1, const int8_t *Wq,
+                           const float *s2, const float *bias, int64_t bias_stride, float *Y, int32_t *Yacc,
+                           int32_t *dev_status, cudaStream_t st) {
+    if (use_halo(d, mode)) return tc::tc_pix_halo(d, mode, A, s1, Wq, s2, bias, bias_stride, Y, Yacc, dev_status, st);
+    return tc::tc_pix(d, mode, A, s1, Wq, s2, bias, bias_stride, Y, Yacc, dev_status, st);
+}
 
 static int pad16(int c) { return (c + 15) / 16 * 16; }
 // Input channels padded to a multiple of 16 make the shape eligible.
@@ -109,7 +124,7 @@ extern "C" lpdt_status lpdt_qconv_fwd(const lpdt_conv_desc *d, const int8_t *A, 
     cudaStream_t st = as_stream(stream);
     const bool out_ok = (!Y || aligned(Y, 16)) && (!Yacc || aligned(Yacc, 16));
     if (use_tc(*d) && aligned(A, 16) && aligned(Wq, 16) && out_ok)
-        return tc::tc_pix(*d, 0, A, sA, Wq, sW, bias, bias_node_stride, Y, Yacc, dev_status, st);
+        return run_pix(*d, 0, A, sA, Wq, sW, bias, bias_node_stride, Y, Yacc, dev_status, st);
     lpdt_conv_desc dp;
     if (use_tc_padded(*d, &dp) && out_ok && ws && aligned(ws, 256) &&
         ws_bytes >= lpdt_qconv_workspace_size(d, 0)) {
@@ -120,7 +135,7 @@ extern "C" lpdt_status lpdt_qconv_fwd(const lpdt_conv_desc *d, const int8_t *A, 
         LPDT_LAUNCH_CHECK();
         pad_channels_kernel<<<grid_for(wrows * dp.Cin), 256, 0, st>>>(Wq, Wp, wrows, d->Cin, dp.Cin);
         LPDT_LAUNCH_CHECK();
-        return tc::tc_pix(dp, 0, Ap, sA, Wp, sW, bias, bias_node_stride, Y, Yacc, dev_status, st);
+        return run_pix(dp, 0, Ap, sA, Wp, sW, bias, bias_node_stride, Y, Yacc, dev_status, st);
     }
     return generic_fwd(*d, A, sA, Wq, sW, bias, bias_node_stride, Y, Yacc, st);
 }
@@ -135,7 +150,7 @@ extern "C" lpdt_status lpdt_qconv_bwd_data(const lpdt_conv_desc *d, const int8_t
     LPDT_CHECK_ARG(!dA || (sE && sW));
     if (!ws || ws_bytes < lpdt_qconv_workspace_size(d, 1)) return LPDT_ERR_WORKSPACE;
     if (use_tc(*d) && aligned(E, 16) && aligned(Wq, 16) && (!dA || aligned(dA, 16)) && (!dAacc || aligned(dAacc, 16)))
-        return tc::tc_pix(*d, 1, E, sE, Wq, sW, nullptr, 0, dA, dAacc, dev_status, as_stream(stream));
+        return run_pix(*d, 1, E, sE, Wq, sW, nullptr, 0, dA, dAacc, dev_status, as_stream(stream));
     return generic_bwd_data(*d, E, sE, Wq, sW, dA, dAacc, ws, as_stream(stream));
 }
 

@@ -1,0 +1,299 @@
+// Halo-tile variant of the pixel-M convolution kernel for 16-channel operands
+// (K = taps x 16 bytes, stride 1): forward with Cin = 16 and backward-data with
+// Cout = 16.
+//
+// With 16 channels a pixel is exactly one 16-byte row of the no-swizzle
+// core-matrix layout, and a filter tap is a shift by whole rows.  So instead of
+// one TMA box per tap, one box per tile fetches the 8 x 16 pixel tile together
+// with its halo ((8+S-1) x (16+R-1) pixels, out-of-image pixels zero-filled),
+// and each tap is reached through the matrix descriptor alone: start address =
+// the tap's offset inside the halo, stride between 8-row groups = the halo row
+// pitch, and the leading-dimension offset = the distance to the second tap of the
+// pair that shares a K = 32 MMA (an odd last tap is paired with a block of zeros).
+// The node's weights are loaded into shared memory once per node, not per tile.
+// Per tile this is 1 TMA request and ceil(taps/2) MMAs.
+#include "qconv_internal.cuh"
+#include "tc_common.cuh"
+
+namespace lpdt {
+namespace tc {
+
+constexpr int kHaloThreads = 192;
+constexpr int kHaloMaxTaps = 64;
+constexpr int kTileW = 8, kTileH = 16;
+constexpr int kZeroBytes = 4096;          // >= 15 halo rows of at most 256 bytes + one 8-row group
+
+struct HaloParams {
+    int mode;                  // 0 forward, 1 backward-data
+    int nodes, B, Hm, Wm;      // output image of this pass
+    int N;                     // output channels of this pass
+    int ntaps;
+    unsigned short off16[kHaloMaxTaps];   // tap offset inside the halo, in 16-byte rows, ascending
+    signed char wtap[kHaloMaxTaps];       // matching tap index in the weight tensor
+    int org_h, org_w;          // halo origin relative to the tile origin (smallest tap offsets)
+    int PH, PW;                // halo rows / pixels per row
+    int tilesH, tilesW;
+    int stages, halo_bytes, wres_bytes, tmem_cols;
+    int w_rows_per_node;
+    float *Y; int32_t *Yacc;
+    const float *s1, *s2, *bias; long long bias_stride;
+    int32_t *dev_status;
+};
+
+struct HaloCtl {
+    unsigned long long full[8], empty[8], tmem_full[2], tmem_empty[2], wfull;
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+
+struct HaloTile { int tw, th, b, node; };
+__device__ __forceinline__ HaloTile halo_decode(const HaloParams &p, int tile) {
+    HaloTile c; int t = tile;
+    c.tw = t % p.tilesW; t /= p.tilesW;
+    c.th = t % p.tilesH; t /= p.tilesH;
+    c.b = t % p.B; c.node = t / p.B;
+    return c;
+}
+__device__ __forceinline__ void halo_next(const HaloParams &p, HaloTile &c) {
+    if (++c.tw < p.tilesW) return; c.tw = 0;
+    if (++c.th < p.tilesH) return; c.th = 0;
+    if (++c.b < p.B) return; c.b = 0;
+    ++c.node;
+}
+
+__global__ void __launch_bounds__(kHaloThreads, 1)
+conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapW,
+                   const HaloParams p) {
+    extern __shared__ __align__(1024) unsigned char smem[];
+    HaloCtl *ctl = reinterpret_cast<HaloCtl *>(smem);
+    unsigned char *wres = smem + 1024;
+    unsigned char *stage0 = wres + p.wres_bytes;
+    unsigned char *zeros = stage0 + (size_t)p.stages * p.halo_bytes;     // above every tile: offsets to it are positive
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long total_tiles = (long long)p.nodes * p.B * p.tilesH * p.tilesW;
+    const int tile_lo = (int)(total_tiles * blockIdx.x / gridDim.x);
+    const int tile_hi = (int)(total_tiles * (blockIdx.x + 1) / gridDim.x);
+
+    for (int i = threadIdx.x; i < kZeroBytes / 4; i += blockDim.x) reinterpret_cast<uint32_t *>(zeros)[i] = 0u;
+    for (int i = threadIdx.x; i < p.wres_bytes / 4; i += blockDim.x) reinterpret_cast<uint32_t *>(wres)[i] = 0u;
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < p.stages; ++i) { mbar_init(smem_u32(&ctl->full[i]), 1); mbar_init(smem_u32(&ctl->empty[i]), 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&ctl->tmem_full[i]), 1); mbar_init(smem_u32(&ctl->tmem_empty[i]), 4); }
+        mbar_init(smem_u32(&ctl->wfull), 1);
+        ctl->abort_flag = 0;
+        mbar_fence_init();
+    }
+    if (warp == 1) { tmem_alloc(smem_u32(&ctl->tmem_base), p.tmem_cols); tmem_relinquish(); }
+    // the zero fills above are generic-proxy writes that the tensor core (async proxy) will read
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+    const int slot_bytes = p.mode == 0 ? p.N * 16 : 256;      // one tap of weights (backward: per 16-column chunk)
+    const int nchunk = p.N / 16;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            tma_prefetch_desc(&mapA); tma_prefetch_desc(&mapW);
+            int st = 0; uint32_t ph = 0;
+            int cur_node = -1;
+            HaloTile c = halo_decode(p, tile_lo);
+            for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; ++tile, halo_next(p, c)) {
+                if (c.node != cur_node) {
+                    // drain: every stage issued so far must have been consumed before the weights change
+                    int s2 = st; uint32_t ph2 = ph; bool ok = true;
+                    for (int i = 0; i < p.stages && ok; ++i) {
+                        ok = mbar_wait(smem_u32(&ctl->empty[s2]), ph2 ^ 1, &ctl->abort_flag, p.dev_status);
+                        if (++s2 == p.stages) { s2 = 0; ph2 ^= 1; }
+                    }
+                    if (!ok) break;
+                    cur_node = c.node;
+                    const uint32_t wfull = smem_u32(&ctl->wfull);
+                    mbar_expect_tx(wfull, p.ntaps * p.N * 16);
+                    const int wrow = c.node * p.w_rows_per_node;
+                    for (int i = 0; i < p.ntaps; ++i) {
+                        if (p.mode == 0) {
+                            tma_load_3d(smem_u32(wres) + i * slot_bytes, &mapW, wfull, 0, p.wtap[i], wrow);
+                        } else {
+                            for (int j = 0; j < nchunk; ++j)
+                                tma_load_3d(smem_u32(wres) + (j * (p.ntaps + 1) + i) * 256, &mapW, wfull, j * 16,
+                                            p.wtap[i], wrow);
+                        }
+                    }
+                }
+                if (!mbar_wait(smem_u32(&ctl->empty[st]), ph ^ 1, &ctl->abort_flag, p.dev_status)) break;
+                const uint32_t full = smem_u32(&ctl->full[st]);
+                mbar_expect_tx(full, p.PH * p.PW * 16);
+                tma_load_4d(smem_u32(stage0 + (size_t)st * p.halo_bytes), &mapA, full,
+                            (c.tw * kTileW + p.org_w) * 16, c.th * kTileH + p.org_h, c.b, c.node);
+                if (++st == p.stages) { st = 0; ph ^= 1; }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            const uint32_t idesc = idesc_i8(128, p.N, 0, p.mode == 0 ? 0 : 1);
+            const uint32_t sbo_a = p.PW * 16;                       // next 8-pixel row group = next halo row
+            const uint64_t a_fixed = ((uint64_t)((sbo_a >> 4) & 0x3FFFu) << 32) | ((uint64_t)1 << 46);
+            const uint64_t b_tpl = (p.mode == 0) ? smem_desc(0, p.N * 16, 128, 0)
+                                                 : smem_desc(0, 128, (p.ntaps + 1) * 256, 0);
+            const uint32_t w_lo0 = smem_u32(wres) >> 4;
+            const uint32_t b_pair_step = (2 * slot_bytes) >> 4;
+            const uint32_t zero_lo = smem_u32(zeros) >> 4;
+            const int npairs = (p.ntaps + 1) / 2;
+            int st = 0; uint32_t ph = 0, tcount = 0, wph = 0;
+            int cur_node = -1;
+            HaloTile c = halo_decode(p, tile_lo);
+            for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; ++tile, ++tcount, halo_next(p, c)) {
+                if (c.node != cur_node) {
+                    if (!mbar_wait(smem_u32(&ctl->wfull), wph, &ctl->abort_flag, p.dev_status)) break;
+                    wph ^= 1; cur_node = c.node;
+                }
+                const int acc = tcount & 1;
+                const uint32_t aph = (tcount >> 1) & 1;
+                if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), aph ^ 1, &ctl->abort_flag, p.dev_status)) break;
+                if (!mbar_wait(smem_u32(&ctl->full[st]), ph, &ctl->abort_flag, p.dev_status)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * p.N;
+                const uint32_t halo_lo = smem_u32(stage0 + (size_t)st * p.halo_bytes) >> 4;
+                uint32_t b_lo = w_lo0;
+                for (int i = 0; i < npairs; ++i) {
+                    const uint32_t s0 = halo_lo + p.off16[2 * i];
+                    const uint32_t lbo = (2 * i + 1 < p.ntaps) ? (uint32_t)(p.off16[2 * i + 1] - p.off16[2 * i])
+                                                               : (zero_lo - s0);
+                    const uint64_t ad = a_fixed | (uint64_t)(s0 & 0x3FFFu) | ((uint64_t)(lbo & 0x3FFFu) << 16);
+                    mma_i8(d_tmem, ad, b_tpl | (b_lo & 0x3FFFu), idesc, (uint32_t)i);
+                    b_lo += b_pair_step;
+                }
+                mma_commit(smem_u32(&ctl->empty[st]));
+                mma_commit(smem_u32(&ctl->tmem_full[acc]));
+                if (++st == p.stages) { st = 0; ph ^= 1; }
+            }
+        }
+    } else {
+        const int q = warp & 3;
+        const int row = q * 32 + lane;
+        const int pw = row % kTileW, phh = row / kTileW;
+        uint32_t tcount = 0;
+        HaloTile c = halo_decode(p, tile_lo);
+        int sc_node = -1; float sc = 0.f;
+        for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; ++tile, ++tcount, halo_next(p, c)) {
+            const int w = c.tw * kTileW + pw, h = c.th * kTileH + phh;
+            const bool valid = (w < p.Wm) && (h < p.Hm);
+            if (p.Y && c.node != sc_node) { sc_node = c.node; sc = __fmul_rn(p.s1[c.node], p.s2[c.node]); }
+            const int acc = tcount & 1;
+            const uint32_t aph = (tcount >> 1) & 1;
+            if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), aph, &ctl->abort_flag, p.dev_status)) break;
+            tc_fence_after();
+            const long long pix = (((long long)c.node * p.B + c.b) * p.Hm + h) * p.Wm + w;
+            const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * p.N;
+            for (int cc = 0; cc < p.N; cc += 16) {
+                uint32_t v[16];
+                tmem_ld_32x16(t_row + cc, v);
+                tmem_ld_wait();
+                if (valid) {
+                    const long long o = pix * p.N + cc;
+                    if (p.Yacc) {
+                        int4 *dst = reinterpret_cast<int4 *>(p.Yacc + o);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k)
+                            dst[k] = make_int4((int)v[4 * k], (int)v[4 * k + 1], (int)v[4 * k + 2], (int)v[4 * k + 3]);
+                    }
+                    if (p.Y) {
+                        float f[16];
+#pragma unroll
+                        for (int k = 0; k < 16; ++k) {
+                            f[k] = __fmul_rn(__int2float_rn((int)v[k]), sc);
+                            if (p.bias) f[k] = __fadd_rn(f[k], p.bias[(long long)c.node * p.bias_stride + cc + k]);
+                        }
+                        float4 *dst = reinterpret_cast<float4 *>(p.Y + o);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) dst[k] = make_float4(f[4 * k], f[4 * k + 1], f[4 * k + 2], f[4 * k + 3]);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, p.tmem_cols); }
+}
+
+static int halo_pow2(int v) { int p = 32; while (p < v) p <<= 1; return p; }
+
+bool halo_supported(const lpdt_conv_desc &d, int mode) {
+    if (d.stride != 1) return false;
+    const int Kc = mode == 0 ? d.Cin : d.Cout, N = mode == 0 ? d.Cout : d.Cin;
+    if (Kc != 16 || N % 16 || N > 256) return false;
+    if (d.S > 9 || d.R > 64 || d.R * d.S > kHaloMaxTaps) return false;
+    if ((d.R * d.S + 1) * N * 16 > 64 * 1024) return false;
+    if (d.pad > 100) return false;
+    return encode_tiled_fn() != nullptr;
+}
+
+lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, const float *s1, const int8_t *Wq,
+                        const float *s2, const float *bias, int64_t bias_stride, float *Y, int32_t *Yacc,
+                        int32_t *dev_status, cudaStream_t st) {
+    const int Ho = conv_out(d.H, d.pad, d.R, 1), Wo = conv_out(d.W, d.pad, d.S, 1);
+    HaloParams p = {};
+    p.mode = mode; p.nodes = d.nodes; p.B = d.B;
+    p.N = mode == 0 ? d.Cout : d.Cin;
+    p.Hm = mode == 0 ? Ho : d.H; p.Wm = mode == 0 ? Wo : d.W;
+    const int Ha = mode == 0 ? d.H : Ho, Wa = mode == 0 ? d.W : Wo;     // image of operand A
+    p.PH = kTileH + d.R - 1; p.PW = kTileW + d.S - 1;
+    // tap (r, s) reads operand pixel (m + dh, m + dw): dh = r - pad forward, pad - r backward
+    p.org_h = mode == 0 ? -d.pad : d.pad - (d.R - 1);
+    p.org_w = mode == 0 ? -d.pad : d.pad - (d.S - 1);
+    p.ntaps = d.R * d.S;
+    for (int i = 0; i < p.ntaps; ++i) {
+        // ascending halo offset: forward walks (r, s) up, backward walks them down
+        const int a = i / d.S, b = i % d.S;
+        const int r = mode == 0 ? a : d.R - 1 - a, s = mode == 0 ? b : d.S - 1 - b;
+        p.off16[i] = (unsigned short)(a * p.PW + b);
+        p.wtap[i] = (signed char)(r * d.S + s);
+    }
+    p.tilesH = (int)ceil_div(p.Hm, kTileH); p.tilesW = (int)ceil_div(p.Wm, kTileW);
+    p.halo_bytes = (int)align_up((size_t)p.PH * p.PW * 16, 128);
+    p.wres_bytes = (int)align_up((size_t)(p.ntaps + 1) * p.N * 16, 128);
+    if (15 * p.PW * 16 + 128 > kZeroBytes) return LPDT_ERR_UNSUPPORTED;
+    int stages = (196 * 1024 - p.wres_bytes - kZeroBytes) / p.halo_bytes;
+    if (stages > 8) stages = 8;
+    if (stages < 2) return LPDT_ERR_UNSUPPORTED;
+    p.stages = stages;
+    p.tmem_cols = halo_pow2(2 * p.N);
+    p.w_rows_per_node = d.Cout;
+    p.Y = Y; p.Yacc = Yacc; p.s1 = s1; p.s2 = s2; p.bias = bias; p.bias_stride = bias_stride;
+    p.dev_status = dev_status;
+    CUtensorMap mA, mW;
+    {   // operand A with (channel, width) merged into one contiguous row of 16*Wa bytes
+        uint64_t dims[4] = {(uint64_t)Wa * 16, (uint64_t)Ha, (uint64_t)d.B, (uint64_t)d.nodes};
+        uint64_t strides[3] = {(uint64_t)Wa * 16, (uint64_t)Ha * Wa * 16, (uint64_t)d.B * Ha * Wa * 16};
+        uint32_t box[4] = {(uint32_t)p.PW * 16, (uint32_t)p.PH, 1, 1};
+        if (!make_map_u8(&mA, A, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE)) return LPDT_ERR_CUDA;
+    }
+    {   // weights [nodes*Cout][taps][Cin]: forward box = N rows of one tap, backward = 16 rows x 16 columns
+        uint64_t dims[3] = {(uint64_t)d.Cin, (uint64_t)p.ntaps, (uint64_t)d.nodes * d.Cout};
+        uint64_t strides[2] = {(uint64_t)d.Cin, (uint64_t)p.ntaps * d.Cin};
+        uint32_t box[3] = {16, 1, (uint32_t)(mode == 0 ? p.N : 16)};
+        if (!make_map_u8(&mW, Wq, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE)) return LPDT_ERR_CUDA;
+    }
+    size_t smem = 1024 + (size_t)p.wres_bytes + (size_t)p.stages * p.halo_bytes + kZeroBytes;
+    if (smem < 120 * 1024) smem = 120 * 1024;        // one CTA per SM: TMEM allocation never waits
+    static bool attr = false;
+    if (!attr) {
+        LPDT_CUDA(cudaFuncSetAttribute(conv_halo16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        attr = true;
+    }
+    const long long tiles = (long long)p.nodes * p.B * p.tilesH * p.tilesW;
+    if (tiles > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
+    const int grid = (int)(tiles < kNumSMs ? tiles : kNumSMs);
+    conv_halo16_kernel<<<grid, kHaloThreads, smem, st>>>(mA, mW, p);
+    LPDT_LAUNCH_CHECK();
+    return LPDT_OK;
+}
+
+}  // namespace tc
+}  // namespace lpdt

@@ -118,6 +118,12 @@ CONV_CASES = [
     (2, 40, 1, 1, 256, 128, 1, 1, 1, 0),     # linear layer on the tensor-core path
     (1, 130, 1, 1, 512, 272, 1, 1, 1, 0),    # linear: ragged row tile, two N tiles (272 = 16*17)
     (1, 1, 4, 4, 512, 512, 3, 3, 1, 1),      # wide channels on a tiny map
+    (3, 5, 32, 32, 16, 16, 3, 3, 1, 1),      # 16-channel halo-tile path, several nodes per CTA range
+    (2, 3, 19, 13, 16, 48, 3, 3, 1, 1),      # halo path: ragged image, 16 -> 48 channels
+    (2, 2, 20, 20, 48, 16, 3, 3, 1, 1),      # halo path on the backward-data side (Cout = 16)
+    (1, 2, 17, 9, 16, 16, 5, 4, 1, 2),       # halo path: 5x4 filter (even tap count), asymmetric padding effect
+    (1, 2, 12, 12, 16, 32, 1, 1, 1, 0),      # halo path with a single tap
+    (2, 2, 10, 10, 16, 16, 3, 3, 1, 0),      # halo path without padding
 ]
 
 
