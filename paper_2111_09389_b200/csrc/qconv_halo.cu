@@ -69,7 +69,9 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
     unsigned char *wres = smem + 1024;
     unsigned char *stage0 = wres + p.wres_bytes;
     unsigned char *zeros = stage0 + (size_t)p.stages * p.halo_bytes;     // above every tile: offsets to it are positive
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // warp index and TMEM base are broadcast through a shuffle so that the compiler knows they are
+    // warp-uniform and keeps the role loops on the uniform datapath
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     const long long total_tiles = (long long)p.nodes * p.B * p.tilesH * p.tilesW;
     const int tile_lo = (int)(total_tiles * blockIdx.x / gridDim.x);
     const int tile_hi = (int)(total_tiles * (blockIdx.x + 1) / gridDim.x);
@@ -89,13 +91,13 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = ctl->tmem_base;
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, ctl->tmem_base, 0);
     const int slot_bytes = p.mode == 0 ? p.N * 16 : 256;      // one tap of weights (backward: per 16-column chunk)
     const int nchunk = p.N / 16;
 
     if (warp == 0) {
-        if (lane == 0) {
-            tma_prefetch_desc(&mapA); tma_prefetch_desc(&mapW);
+        {
+            if (elect_one()) { tma_prefetch_desc(&mapA); tma_prefetch_desc(&mapW); }
             int st = 0; uint32_t ph = 0;
             int cur_node = -1;
             HaloTile c = halo_decode(p, tile_lo);
@@ -110,28 +112,34 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
                     if (!ok) break;
                     cur_node = c.node;
                     const uint32_t wfull = smem_u32(&ctl->wfull);
-                    mbar_expect_tx(wfull, p.ntaps * p.N * 16);
                     const int wrow = c.node * p.w_rows_per_node;
-                    for (int i = 0; i < p.ntaps; ++i) {
-                        if (p.mode == 0) {
-                            tma_load_3d(smem_u32(wres) + i * slot_bytes, &mapW, wfull, 0, p.wtap[i], wrow);
-                        } else {
-                            for (int j = 0; j < nchunk; ++j)
-                                tma_load_3d(smem_u32(wres) + (j * (p.ntaps + 1) + i) * 256, &mapW, wfull, j * 16,
-                                            p.wtap[i], wrow);
+                    if (elect_one()) {
+                        mbar_expect_tx(wfull, p.ntaps * p.N * 16);
+                        for (int i = 0; i < p.ntaps; ++i) {
+                            if (p.mode == 0) {
+                                tma_load_3d(smem_u32(wres) + i * slot_bytes, &mapW, wfull, 0, p.wtap[i], wrow);
+                            } else {
+                                for (int j = 0; j < nchunk; ++j)
+                                    tma_load_3d(smem_u32(wres) + (j * (p.ntaps + 1) + i) * 256, &mapW, wfull, j * 16,
+                                                p.wtap[i], wrow);
+                            }
                         }
                     }
+                    __syncwarp();
                 }
                 if (!mbar_wait(smem_u32(&ctl->empty[st]), ph ^ 1, &ctl->abort_flag, p.dev_status)) break;
                 const uint32_t full = smem_u32(&ctl->full[st]);
-                mbar_expect_tx(full, p.PH * p.PW * 16);
-                tma_load_4d(smem_u32(stage0 + (size_t)st * p.halo_bytes), &mapA, full,
-                            (c.tw * kTileW + p.org_w) * 16, c.th * kTileH + p.org_h, c.b, c.node);
+                if (elect_one()) {
+                    mbar_expect_tx(full, p.PH * p.PW * 16);
+                    tma_load_4d(smem_u32(stage0 + (size_t)st * p.halo_bytes), &mapA, full,
+                                (c.tw * kTileW + p.org_w) * 16, c.th * kTileH + p.org_h, c.b, c.node);
+                }
+                __syncwarp();
                 if (++st == p.stages) { st = 0; ph ^= 1; }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        {
             const uint32_t idesc = idesc_i8(128, p.N, 0, p.mode == 0 ? 0 : 1);
             const uint32_t sbo_a = p.PW * 16;                       // next 8-pixel row group = next halo row
             const uint64_t a_fixed = ((uint64_t)((sbo_a >> 4) & 0x3FFFu) << 32) | ((uint64_t)1 << 46);
@@ -156,17 +164,20 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * p.N;
                 const uint32_t halo_lo = smem_u32(stage0 + (size_t)st * p.halo_bytes) >> 4;
-                uint32_t b_lo = w_lo0;
-                for (int i = 0; i < npairs; ++i) {
-                    const uint32_t s0 = halo_lo + p.off16[2 * i];
-                    const uint32_t lbo = (2 * i + 1 < p.ntaps) ? (uint32_t)(p.off16[2 * i + 1] - p.off16[2 * i])
-                                                               : (zero_lo - s0);
-                    const uint64_t ad = a_fixed | (uint64_t)(s0 & 0x3FFFu) | ((uint64_t)(lbo & 0x3FFFu) << 16);
-                    mma_i8(d_tmem, ad, b_tpl | (b_lo & 0x3FFFu), idesc, (uint32_t)i);
-                    b_lo += b_pair_step;
+                if (elect_one()) {
+                    uint32_t b_lo = w_lo0;
+                    for (int i = 0; i < npairs; ++i) {
+                        const uint32_t s0 = halo_lo + p.off16[2 * i];
+                        const uint32_t lbo = (2 * i + 1 < p.ntaps) ? (uint32_t)(p.off16[2 * i + 1] - p.off16[2 * i])
+                                                                   : (zero_lo - s0);
+                        const uint64_t ad = a_fixed | (uint64_t)(s0 & 0x3FFFu) | ((uint64_t)(lbo & 0x3FFFu) << 16);
+                        mma_i8(d_tmem, ad, b_tpl | (b_lo & 0x3FFFu), idesc, (uint32_t)i);
+                        b_lo += b_pair_step;
+                    }
+                    mma_commit(smem_u32(&ctl->empty[st]));
+                    mma_commit(smem_u32(&ctl->tmem_full[acc]));
                 }
-                mma_commit(smem_u32(&ctl->empty[st]));
-                mma_commit(smem_u32(&ctl->tmem_full[acc]));
+                __syncwarp();
                 if (++st == p.stages) { st = 0; ph ^= 1; }
             }
         }

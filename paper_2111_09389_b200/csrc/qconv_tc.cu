@@ -105,7 +105,9 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     const int b_unit = p.BN * p.RBa;                       // weight bytes that go with it
     const int a_bytes = p.U * a_unit;
     const int stage_bytes = p.U * (a_unit + b_unit);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // warp index (and below the TMEM base) go through a shuffle so that the compiler knows they are
+    // warp-uniform and keeps the single-issuer role loops on the uniform datapath
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     const long long total_tiles = (long long)p.nodes * p.tilesN * p.tilesB * p.tilesH * p.tilesW * p.ncls;
     const int tile_lo = (int)(total_tiles * blockIdx.x / gridDim.x);
     const int tile_hi = (int)(total_tiles * (blockIdx.x + 1) / gridDim.x);
@@ -120,12 +122,12 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = ctl->tmem_base;
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, ctl->tmem_base, 0);
     const int cpt = p.Kc / p.RBa;          // A boxes per tap
 
     if (warp == 0) {
-        if (lane == 0) {
-            tma_prefetch_desc(&mapA); tma_prefetch_desc(&mapW);
+        {
+            if (elect_one()) { tma_prefetch_desc(&mapA); tma_prefetch_desc(&mapW); }
             uint32_t g = 0;     // running stage counter
             int st = 0; uint32_t ph = 0;
             TileCoord c = decode_tile(p, tile_lo);
@@ -138,33 +140,36 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 for (int it = 0; it < p.cls_iters[c.cls]; ++it, ++g) {
                     if (!mbar_wait(smem_u32(&ctl->empty[st]), ph ^ 1, &ctl->abort_flag, p.dev_status)) break;
                     const uint32_t full = smem_u32(&ctl->full[st]);
-                    mbar_expect_tx(full, stage_bytes);
+                    const bool leader = elect_one();        // the whole warp walks the loop, one lane issues
+                    if (leader) mbar_expect_tx(full, stage_bytes);
                     uint32_t a_dst = smem_u32(data + (size_t)st * stage_bytes);
                     uint32_t b_dst = a_dst + a_bytes;
                     for (int u = 0; u < p.U; ++u) {
                         int hc = -(1 << 20), wc = 0, tap = 1 << 20;   // phantom unit: boxes out of range -> zeros
                         if (ti < tt.ntaps) { hc = h0 + tt.dh[ti]; wc = w0 + tt.dw[ti]; tap = tt.wtap[ti]; }
-                        if (p.merged) tma_load_4d(a_dst, &mapA, full, wc * 16, hc, b0, c.node);
-                        else tma_load_5d(a_dst, &mapA, full, chunk * p.RBa, wc, hc, b0, c.node);
-                        if (p.mode == 0) {
-                            tma_load_3d(b_dst, &mapW, full, chunk * p.RBa, tap, wrow + n0);
-                            b_dst += b_unit;
-                        } else {
-                            // N side in chunks of RBn bytes; this unit's RBa weight rows go at row u*RBa of each chunk
-                            for (int j = 0; j < nj; ++j)
-                                tma_load_3d(b_dst + j * bj_stride, &mapW, full, n0 + j * p.RBn, tap,
-                                            wrow + chunk * p.RBa);
-                            b_dst += bu_stride;
+                        if (leader) {
+                            if (p.merged) tma_load_4d(a_dst, &mapA, full, wc * 16, hc, b0, c.node);
+                            else tma_load_5d(a_dst, &mapA, full, chunk * p.RBa, wc, hc, b0, c.node);
+                            if (p.mode == 0) {
+                                tma_load_3d(b_dst, &mapW, full, chunk * p.RBa, tap, wrow + n0);
+                            } else {
+                                // N side in chunks of RBn bytes; this unit's RBa weight rows go at row u*RBa of each chunk
+                                for (int j = 0; j < nj; ++j)
+                                    tma_load_3d(b_dst + j * bj_stride, &mapW, full, n0 + j * p.RBn, tap,
+                                                wrow + chunk * p.RBa);
+                            }
                         }
+                        b_dst += (p.mode == 0) ? b_unit : bu_stride;
                         a_dst += a_unit;
                         if (++chunk == cpt) { chunk = 0; ++ti; }
                     }
+                    __syncwarp();
                     if (++st == p.stages) { st = 0; ph ^= 1; }
                 }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        {
             const uint32_t idesc = idesc_i8(128, p.BN, 0, p.mode == 0 ? 0 : 1);
             // Descriptor templates (start address 0); the loop only adds address increments.
             const uint64_t a_tpl = (p.RBa == 16) ? smem_desc(0, a_unit, 128, 0)
@@ -197,21 +202,25 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                     if (!mbar_wait(smem_u32(&ctl->full[st]), ph, &ctl->abort_flag, p.dev_status)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_st = smem_u32(data + (size_t)st * stage_bytes);
-                    uint32_t a_lo = a_st >> 4, b_lo = (a_st + a_bytes) >> 4;
-                    for (int u = 0; u < n_units; ++u) {
-                        for (int k = 0; k < steps; ++k) {
-                            mma_i8(d_tmem, a_tpl | (a_lo & 0x3FFFu), b_tpl | (b_lo & 0x3FFFu), idesc, accum);
-                            accum = 1;
-                            a_lo += a_step; b_lo += b_step;
+                    if (elect_one()) {
+                        uint32_t a_lo = a_st >> 4, b_lo = (a_st + a_bytes) >> 4, af = accum;
+                        for (int u = 0; u < n_units; ++u) {
+                            for (int k = 0; k < steps; ++k) {
+                                mma_i8(d_tmem, a_tpl | (a_lo & 0x3FFFu), b_tpl | (b_lo & 0x3FFFu), idesc, af);
+                                af = 1;
+                                a_lo += a_step; b_lo += b_step;
+                            }
+                            if (p.RBa == 16) { a_lo += a_unit_step - a_step; b_lo += b_unit_step - b_step; }
+                            else { a_lo += a_unit_step; b_lo += b_unit_step; }
                         }
-                        if (p.RBa == 16) { a_lo += a_unit_step - a_step; b_lo += b_unit_step - b_step; }
-                        else { a_lo += a_unit_step; b_lo += b_unit_step; }
+                        mma_commit(smem_u32(&ctl->empty[st]));
+                        if (it == iters - 1) mma_commit(smem_u32(&ctl->tmem_full[acc]));
                     }
-                    mma_commit(smem_u32(&ctl->empty[st]));
+                    __syncwarp();
+                    accum = 1;
                     if (++st == p.stages) { st = 0; ph ^= 1; }
                 }
                 if (!ok) break;
-                mma_commit(smem_u32(&ctl->tmem_full[acc]));
             }
         }
     } else {
@@ -286,7 +295,9 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     extern __shared__ __align__(1024) unsigned char smem[];
     SharedCtl *ctl = reinterpret_cast<SharedCtl *>(smem);
     unsigned char *data = smem + 1024;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // warp index (and below the TMEM base) go through a shuffle so that the compiler knows they are
+    // warp-uniform and keeps the single-issuer role loops on the uniform datapath
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     const int node = blockIdx.z;
     const int mg = blockIdx.y % p.mgroups, ng = blockIdx.y / p.mgroups;
     const int G = 128 / p.RBx;                    // input boxes stacked in one 128-lane M tile
@@ -310,11 +321,11 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
-    const uint32_t tmem_base = ctl->tmem_base;
+    const uint32_t tmem_base = __shfl_sync(0xffffffffu, ctl->tmem_base, 0);
 
     if (warp == 0) {
-        if (lane == 0) {
-            tma_prefetch_desc(&mapX); tma_prefetch_desc(&mapE);
+        {
+            if (elect_one()) { tma_prefetch_desc(&mapX); tma_prefetch_desc(&mapE); }
             int st = 0; uint32_t ph = 0;
             int tw = kb0 % p.tilesW, th = (kb0 / p.tilesW) % p.tilesH, tb = kb0 / (p.tilesW * p.tilesH);
             const int tap0 = mu0 / cpt, chunk0 = mu0 % cpt, r0 = tap0 / p.S, s0 = tap0 % p.S;
@@ -322,24 +333,28 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                 const int w0 = tw * p.TW, h0 = th * p.TH, b0 = tb * p.TB;
                 if (!mbar_wait(smem_u32(&ctl->empty[st]), ph ^ 1, &ctl->abort_flag, p.dev_status)) break;
                 const uint32_t full = smem_u32(&ctl->full[st]);
-                mbar_expect_tx(full, nX * x_unit + nE * e_unit);
+                const bool leader = elect_one();
+                if (leader) mbar_expect_tx(full, nX * x_unit + nE * e_unit);
                 uint32_t x_dst = smem_u32(data + (size_t)st * stage_bytes);
                 uint32_t e_dst = x_dst + x_region;
                 for (int c = 0; c < nE; ++c, e_dst += e_unit)
-                    tma_load_5d(e_dst, &mapE, full, n0 + c * p.RBe, w0, h0, b0, node);
+                    if (leader) tma_load_5d(e_dst, &mapE, full, n0 + c * p.RBe, w0, h0, b0, node);
                 int chunk = chunk0, r = r0, s = s0;
                 for (int i = 0; i < nX; ++i, x_dst += x_unit) {
                     const int wc = w0 * p.stride + s - p.pad, hc = h0 * p.stride + r - p.pad;
-                    if (p.merged) tma_load_4d(x_dst, &mapX, full, wc * 16, hc, b0, node);
-                    else tma_load_5d(x_dst, &mapX, full, chunk * p.RBx, wc, hc, b0, node);
+                    if (leader) {
+                        if (p.merged) tma_load_4d(x_dst, &mapX, full, wc * 16, hc, b0, node);
+                        else tma_load_5d(x_dst, &mapX, full, chunk * p.RBx, wc, hc, b0, node);
+                    }
                     if (++chunk == cpt) { chunk = 0; if (++s == p.S) { s = 0; ++r; } }
                 }
+                __syncwarp();
                 if (++tw == p.tilesW) { tw = 0; if (++th == p.tilesH) { th = 0; ++tb; } }
                 if (++st == p.stages) { st = 0; ph ^= 1; }
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        {
             const uint32_t idesc = idesc_i8(128, p.BNc, 1, 1);
             const uint64_t a_tpl = (p.RBx == 16) ? smem_desc(0, 128, x_unit, 0)
                                                  : smem_desc(0, x_unit, 8 * p.RBx, layout_code(p.RBx));
@@ -348,27 +363,29 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             const uint32_t a_step = (32 * p.RBx) >> 4, b_step = (32 * p.RBe) >> 4;   // 32 pixel rows per MMA
             uint32_t accum = 0;
             int st = 0; uint32_t ph = 0;
-            bool ok = true;
             for (int kb = kb0; kb < kb1; ++kb) {
-                if (!mbar_wait(smem_u32(&ctl->full[st]), ph, &ctl->abort_flag, p.dev_status)) { ok = false; break; }
+                if (!mbar_wait(smem_u32(&ctl->full[st]), ph, &ctl->abort_flag, p.dev_status)) break;
                 tc_fence_after();
                 const uint32_t x_st = smem_u32(data + (size_t)st * stage_bytes);
                 const uint32_t e_lo0 = (x_st + x_region) >> 4;
-                uint32_t a_tile = x_st >> 4, d_tmem = tmem_base;
-                for (int t = 0; t < p.mtiles; ++t) {
-                    uint32_t a_lo = a_tile, b_lo = e_lo0;
+                if (elect_one()) {
+                    uint32_t a_tile = x_st >> 4, d_tmem = tmem_base;
+                    for (int t = 0; t < p.mtiles; ++t) {
+                        uint32_t a_lo = a_tile, b_lo = e_lo0;
 #pragma unroll
-                    for (int kk = 0; kk < 4; ++kk) {
-                        mma_i8(d_tmem, a_tpl | (a_lo & 0x3FFFu), b_tpl | (b_lo & 0x3FFFu), idesc, accum | (uint32_t)kk);
-                        a_lo += a_step; b_lo += b_step;
+                        for (int kk = 0; kk < 4; ++kk) {
+                            mma_i8(d_tmem, a_tpl | (a_lo & 0x3FFFu), b_tpl | (b_lo & 0x3FFFu), idesc, accum | (uint32_t)kk);
+                            a_lo += a_step; b_lo += b_step;
+                        }
+                        a_tile += 16384 >> 4; d_tmem += p.BNc;
                     }
-                    a_tile += 16384 >> 4; d_tmem += p.BNc;
+                    mma_commit(smem_u32(&ctl->empty[st]));
+                    if (kb == kb1 - 1) mma_commit(smem_u32(&ctl->tmem_full[0]));
                 }
+                __syncwarp();
                 accum = 1;
-                mma_commit(smem_u32(&ctl->empty[st]));
                 if (++st == p.stages) { st = 0; ph ^= 1; }
             }
-            if (ok) mma_commit(smem_u32(&ctl->tmem_full[0]));
         }
     } else if (kb1 > kb0) {
         const int q = warp & 3;
