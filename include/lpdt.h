@@ -62,6 +62,8 @@ typedef struct {
 
 const char *lpdt_version(void);
 const char *lpdt_status_string(lpdt_status s);
+/* Enqueue a zero fill of `bytes` bytes at device pointer p (range accumulators, status words). */
+lpdt_status lpdt_fill_zero(void *p, size_t bytes, void *stream);
 
 /* ---------------------------------------------------------------------------
  * lpdt_quantize — per-tensor, per-node 8-bit quantization.
@@ -91,6 +93,16 @@ lpdt_status lpdt_quantize(const float *x, int32_t nodes, int64_t n_per_node, int
                           lpdt_qmode mode, lpdt_round rounding, uint64_t seed, uint32_t ctr_offset,
                           int8_t *q, float *scale, int32_t *zero_point,
                           void *ws, size_t ws_bytes, void *stream);
+
+/* Symmetric quantization when the per-node range is already known: only the
+ * scale-and-round pass of lpdt_quantize (LPDT_SYM_S8) runs.  amax : fp32 [nodes],
+ * max|x| of each node's tensor, as the producers below can emit while they write
+ * x (lpdt_range_evonorm_fwd/bwd, lpdt_residual_add: `amax_out`).  Same codes and
+ * scales as lpdt_quantize, bit for bit, because a maximum does not depend on the
+ * order it is taken in.  No workspace. */
+lpdt_status lpdt_quantize_with_range(const float *x, int32_t nodes, int64_t n_per_node, int64_t x_node_stride,
+                                     const float *amax, lpdt_round rounding, uint64_t seed,
+                                     uint32_t ctr_offset, int8_t *q, float *scale, void *stream);
 
 /* y = scale[n] * (q - zp[n]); zero_point == NULL means symmetric signed codes.
  * q is contiguous [nodes][n_per_node]; node n of y starts at y + n*y_node_stride. */
@@ -178,6 +190,8 @@ lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8_t *E, cons
  * x, y, dy, dx : fp32 NHWC;  v, gamma, beta : fp32, node n at p + n*param_node_stride
  * gmin, gmax : fp32 [nodes][B][groups];  argmin, argmax : int32, same shape
  * dv, dgamma, dbeta : fp32, node n at p + n*grad_node_stride, C entries
+ * amax_out (nullable) : fp32 [nodes], caller-zeroed; receives max|y| (forward) or max|dx|
+ *            (backward) per node by atomic maximum, for lpdt_quantize_with_range
  * Requires C % groups == 0 and cpg >= 2 (Cst is infinite for cpg = 1).
  * Errors: INVALID_ARG, UNSUPPORTED (C beyond the kernels' range), WORKSPACE, CUDA.
  */
@@ -186,7 +200,7 @@ lpdt_status lpdt_range_evonorm_fwd(int32_t nodes, int32_t B, int32_t H, int32_t 
                                    const float *v, const float *gamma, const float *beta,
                                    int64_t param_node_stride, float *y,
                                    float *gmin, float *gmax, int32_t *argmin, int32_t *argmax,
-                                   void *stream);
+                                   float *amax_out, void *stream);
 size_t lpdt_range_evonorm_bwd_workspace_size(int32_t nodes, int32_t C);
 lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C,
                                    int32_t groups, float eps, const float *dy, const float *x,
@@ -194,7 +208,7 @@ lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t H, int32_t 
                                    const float *gmin, const float *gmax,
                                    const int32_t *argmin, const int32_t *argmax,
                                    float *dx, float *dv, float *dgamma, float *dbeta,
-                                   int64_t grad_node_stride,
+                                   int64_t grad_node_stride, float *amax_out,
                                    void *ws, size_t ws_bytes, void *stream);
 
 /* ---------------------------------------------------------------------------
@@ -230,10 +244,11 @@ lpdt_status lpdt_sgd_update(int64_t n, const float *x, const float *g, float lr,
 
 /* Residual connection y = r + P(a): P subsamples a [nodes*B][H][W][Ca]
  * spatially by `stride` and places its channels at ch_off within C channels
- * (identity shortcut: stride 1, Ca = C, ch_off 0).  y may alias r. */
+ * (identity shortcut: stride 1, Ca = C, ch_off 0).  y may alias r.  amax_out (nullable,
+ * fp32 [nodes], caller-zeroed) receives max|y| per node. */
 lpdt_status lpdt_residual_add(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t Ca,
                               int32_t C, int32_t stride, int32_t ch_off,
-                              const float *r, const float *a, float *y, void *stream);
+                              const float *r, const float *a, float *y, float *amax_out, void *stream);
 /* Adjoint: da = g_main + P^T(dy).  da may alias g_main. */
 lpdt_status lpdt_residual_add_bwd(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t Ca,
                                   int32_t C, int32_t stride, int32_t ch_off,

@@ -21,21 +21,23 @@ class ConvDesc(C.Structure):
 SIGNATURES = {
     "lpdt_version": (C.c_char_p, []),
     "lpdt_status_string": (C.c_char_p, [_i32]),
+    "lpdt_fill_zero": (_i32, [_vp, _sz, _vp]),
     "lpdt_quantize_workspace_size": (_sz, [_i32]),
     "lpdt_quantize": (_i32, [_vp, _i32, _i64, _i64, _i32, _i32, _u64, _u32, _vp, _vp, _vp, _vp, _sz, _vp]),
     "lpdt_quantize_static": (_i32, [_vp, _i32, _i64, _i64, _i32, _i32, _u64, _u32, _vp, _vp, _vp, _vp]),
+    "lpdt_quantize_with_range": (_i32, [_vp, _i32, _i64, _i64, _vp, _i32, _u64, _u32, _vp, _vp, _vp]),
     "lpdt_dequantize": (_i32, [_vp, _i32, _i64, _vp, _vp, _vp, _i64, _vp]),
     "lpdt_qconv_workspace_size": (_sz, [C.POINTER(ConvDesc), _i32]),
     "lpdt_qconv_fwd": (_i32, [C.POINTER(ConvDesc), _vp, _vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _sz, _vp, _vp]),
     "lpdt_qconv_bwd_data": (_i32, [C.POINTER(ConvDesc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
     "lpdt_qconv_bwd_weight": (_i32, [C.POINTER(ConvDesc), _vp, _vp, _vp, _vp, _vp, _i64, _vp, _vp, _sz, _vp, _vp]),
-    "lpdt_range_evonorm_fwd": (_i32, [_i32] * 6 + [_f32] + [_vp] * 4 + [_i64] + [_vp] * 5 + [_vp]),
+    "lpdt_range_evonorm_fwd": (_i32, [_i32] * 6 + [_f32] + [_vp] * 4 + [_i64] + [_vp] * 6 + [_vp]),
     "lpdt_range_evonorm_bwd_workspace_size": (_sz, [_i32, _i32]),
-    "lpdt_range_evonorm_bwd": (_i32, [_i32] * 6 + [_f32] + [_vp] * 4 + [_i64] + [_vp] * 8 + [_i64, _vp, _sz, _vp]),
+    "lpdt_range_evonorm_bwd": (_i32, [_i32] * 6 + [_f32] + [_vp] * 4 + [_i64] + [_vp] * 8 + [_i64, _vp, _vp, _sz, _vp]),
     "lpdt_gossip_mix_workspace_size": (_sz, [_i32, _i64, _i32]),
     "lpdt_gossip_mix": (_i32, [_i32, _i64, _vp, _vp, _vp, _vp, _f32, _i32, _vp, _vp, _vp, _sz, _vp, _vp]),
     "lpdt_sgd_update": (_i32, [_i64, _vp, _vp, _f32, _vp, _vp]),
-    "lpdt_residual_add": (_i32, [_i32] * 8 + [_vp] * 4),
+    "lpdt_residual_add": (_i32, [_i32] * 8 + [_vp] * 5),
     "lpdt_residual_add_bwd": (_i32, [_i32] * 8 + [_vp] * 4),
     "lpdt_avgpool": (_i32, [_i32] * 4 + [_vp] * 3),
     "lpdt_avgpool_bwd": (_i32, [_i32] * 4 + [_vp] * 3),

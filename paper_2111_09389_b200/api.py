@@ -13,7 +13,7 @@ from ._lib import ConvDesc, lib
 
 # Kernels each entry point enqueues (memsets not counted); KERNEL_LAUNCHES accumulates them.
 KERNELS_PER_CALL = {
-    "lpdt_quantize": 2, "lpdt_quantize_static": 2, "lpdt_dequantize": 1, "lpdt_qconv_fwd": 1, "lpdt_qconv_bwd_data": 2,
+    "lpdt_quantize": 2, "lpdt_quantize_with_range": 1, "lpdt_quantize_static": 2, "lpdt_dequantize": 1, "lpdt_qconv_fwd": 1, "lpdt_qconv_bwd_data": 2,
     "lpdt_qconv_bwd_weight": 2, "lpdt_range_evonorm_fwd": 1, "lpdt_range_evonorm_bwd": 2,
     "lpdt_gossip_mix": 2, "lpdt_sgd_update": 1, "lpdt_residual_add": 1, "lpdt_residual_add_bwd": 1,
     "lpdt_avgpool": 1, "lpdt_avgpool_bwd": 1, "lpdt_maxpool2x2": 1, "lpdt_maxpool2x2_bwd": 1,
@@ -97,6 +97,16 @@ def lpdt_quantize(x, nodes, n_per_node, x_node_stride, q, scale, ws, mode=0, rou
                                                 p, nb, _stream()))
 
 
+def lpdt_quantize_with_range(x, nodes, n_per_node, x_node_stride, amax, q, scale, rounding=0, seed=0, ctr_offset=0):
+    _check("lpdt_quantize_with_range", lib().lpdt_quantize_with_range(
+        _ptr(x), nodes, n_per_node, x_node_stride, _ptr(amax), rounding, seed, ctr_offset, _ptr(q), _ptr(scale),
+        _stream()))
+
+
+def lpdt_fill_zero(t):
+    _check("lpdt_fill_zero", lib().lpdt_fill_zero(_ptr(t), t.numel() * t.element_size(), _stream()))
+
+
 def lpdt_quantize_static(x, nodes, n_per_node, x_node_stride, q, scale, mode=0, rounding=0, seed=0,
                          ctr_offset=0, zero_point=None):
     """lpdt_quantize for callers without device scratch: the range words live inside the
@@ -141,10 +151,10 @@ def lpdt_qconv_bwd_weight(desc, E, sE, A, sA, dW=None, dw_node_stride=0, dWacc=N
 
 
 def lpdt_range_evonorm_fwd(nodes, B, H, W, Cc, groups, eps, x, v, gamma, beta, param_node_stride, y,
-                           gmin, gmax, argmin, argmax):
+                           gmin, gmax, argmin, argmax, amax_out=None):
     _check("lpdt_range_evonorm_fwd", lib().lpdt_range_evonorm_fwd(
         nodes, B, H, W, Cc, groups, eps, _ptr(x), _ptr(v), _ptr(gamma), _ptr(beta), param_node_stride,
-        _ptr(y), _ptr(gmin), _ptr(gmax), _ptr(argmin), _ptr(argmax), _stream()))
+        _ptr(y), _ptr(gmin), _ptr(gmax), _ptr(argmin), _ptr(argmax), _ptr(amax_out), _stream()))
 
 
 def lpdt_range_evonorm_bwd_workspace_size(nodes, Cc):
@@ -152,12 +162,12 @@ def lpdt_range_evonorm_bwd_workspace_size(nodes, Cc):
 
 
 def lpdt_range_evonorm_bwd(nodes, B, H, W, Cc, groups, eps, dy, x, v, gamma, param_node_stride, gmin,
-                           gmax, argmin, argmax, dx, dv, dgamma, dbeta, grad_node_stride, ws):
+                           gmax, argmin, argmax, dx, dv, dgamma, dbeta, grad_node_stride, ws, amax_out=None):
     p, nb = _ws(ws)
     _check("lpdt_range_evonorm_bwd", lib().lpdt_range_evonorm_bwd(
         nodes, B, H, W, Cc, groups, eps, _ptr(dy), _ptr(x), _ptr(v), _ptr(gamma), param_node_stride,
         _ptr(gmin), _ptr(gmax), _ptr(argmin), _ptr(argmax), _ptr(dx), _ptr(dv), _ptr(dgamma), _ptr(dbeta),
-        grad_node_stride, p, nb, _stream()))
+        grad_node_stride, _ptr(amax_out), p, nb, _stream()))
 
 
 def lpdt_gossip_mix_workspace_size(nodes, d, n_segments):
@@ -179,9 +189,9 @@ def lpdt_sgd_update(n, x, g, lr, out):
     _check("lpdt_sgd_update", lib().lpdt_sgd_update(n, _ptr(x), _ptr(g), lr, _ptr(out), _stream()))
 
 
-def lpdt_residual_add(nodes, B, H, W, Ca, Cc, stride, ch_off, r, a, y):
+def lpdt_residual_add(nodes, B, H, W, Ca, Cc, stride, ch_off, r, a, y, amax_out=None):
     _check("lpdt_residual_add", lib().lpdt_residual_add(nodes, B, H, W, Ca, Cc, stride, ch_off, _ptr(r),
-                                                        _ptr(a), _ptr(y), _stream()))
+                                                        _ptr(a), _ptr(y), _ptr(amax_out), _stream()))
 
 
 def lpdt_residual_add_bwd(nodes, B, H, W, Ca, Cc, stride, ch_off, dy, g_main, da):

@@ -3,6 +3,13 @@
 
 extern "C" const char *lpdt_version(void) { return "lpdt 0.1 (sm_100a)"; }
 
+extern "C" lpdt_status lpdt_fill_zero(void *p, size_t bytes, void *stream) {
+    if (bytes == 0) return LPDT_OK;
+    LPDT_CHECK_ARG(p != nullptr);
+    LPDT_CUDA(cudaMemsetAsync(p, 0, bytes, lpdt::as_stream(stream)));
+    return LPDT_OK;
+}
+
 extern "C" const char *lpdt_status_string(lpdt_status s) {
     switch (s) {
         case LPDT_OK: return "ok";

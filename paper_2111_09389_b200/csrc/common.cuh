@@ -43,4 +43,20 @@ __device__ __forceinline__ double warp_sum(double v) {
     return v;
 }
 
+// Block-wide max of non-negative values, then one atomicMax on the float's bit pattern
+// (non-negative floats order like unsigned integers).  Every thread of the block must call.
+__device__ __forceinline__ void block_amax_to(float v, float *dst) {
+    __shared__ float s_blk_amax[32];
+    v = warp_max(v);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) s_blk_amax[warp] = v;
+    __syncthreads();
+    if (warp == 0) {
+        const int nw = (blockDim.x + 31) >> 5;
+        v = lane < nw ? s_blk_amax[lane] : 0.f;
+        v = warp_max(v);
+        if (lane == 0) atomicMax(reinterpret_cast<unsigned int *>(dst), __float_as_uint(v));
+    }
+}
+
 }  // namespace lpdt

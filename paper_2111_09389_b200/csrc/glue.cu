@@ -18,12 +18,16 @@ __global__ void sgd_kernel(int64_t n, const float *__restrict__ x, const float *
         out[i] = __fsub_rn(x[i], __fmul_rn(lr, g[i]));
 }
 
-__global__ void residual_add_kernel(int64_t NB, int H, int W, int Ca, int C, int stride, int ch_off,
+// grid.y = node; B = samples per node.  amax_out (nullable) receives max|y| per node.
+__global__ void residual_add_kernel(int B, int H, int W, int Ca, int C, int stride, int ch_off,
                                     const float *__restrict__ r, const float *__restrict__ a,
-                                    float *__restrict__ y) {
+                                    float *__restrict__ y, float *__restrict__ amax_out) {
     const int Ho = (H + stride - 1) / stride, Wo = (W + stride - 1) / stride;
-    const int64_t total = NB * Ho * Wo * C;
-    for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t per_node = (int64_t)B * Ho * Wo * C;
+    const int64_t base = (int64_t)blockIdx.y * per_node;
+    float ymax = 0.f;
+    for (int64_t ol = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; ol < per_node; ol += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t o = base + ol;
         int c = (int)(o % C);
         int64_t pix = o / C;
         int ow = (int)(pix % Wo); pix /= Wo;
@@ -34,16 +38,21 @@ __global__ void residual_add_kernel(int64_t NB, int H, int W, int Ca, int C, int
         if (ca >= 0 && ca < Ca)
             v = __fadd_rn(v, a[((nb * H + (int64_t)oh * stride) * W + (int64_t)ow * stride) * Ca + ca]);
         y[o] = v;
+        ymax = fmaxf(ymax, fabsf(v));
     }
+    if (amax_out) block_amax_to(ymax, amax_out + blockIdx.y);
 }
 
 // Vector forms: 4 consecutive channels per thread (C, Ca and ch_off multiples of 4).
-__global__ void residual_add_v4_kernel(int NB, int H, int W, int Ca4, int C4, int stride, int ch_off4,
+__global__ void residual_add_v4_kernel(int B, int H, int W, int Ca4, int C4, int stride, int ch_off4,
                                        const float4 *__restrict__ r, const float4 *__restrict__ a,
-                                       float4 *__restrict__ y) {
+                                       float4 *__restrict__ y, float *__restrict__ amax_out) {
     const int Ho = (H + stride - 1) / stride, Wo = (W + stride - 1) / stride;
-    const long long total = (long long)NB * Ho * Wo * C4;
-    for (long long o = (long long)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (long long)gridDim.x * blockDim.x) {
+    const long long per_node = (long long)B * Ho * Wo * C4;
+    const long long base = (long long)blockIdx.y * per_node;
+    float ymax = 0.f;
+    for (long long ol = (long long)blockIdx.x * blockDim.x + threadIdx.x; ol < per_node; ol += (long long)gridDim.x * blockDim.x) {
+        const long long o = base + ol;
         const int c = (int)(o % C4);
         float4 v = r[o];
         const int ca = c - ch_off4;
@@ -56,7 +65,9 @@ __global__ void residual_add_v4_kernel(int NB, int H, int W, int Ca4, int C4, in
             v.x = __fadd_rn(v.x, u.x); v.y = __fadd_rn(v.y, u.y); v.z = __fadd_rn(v.z, u.z); v.w = __fadd_rn(v.w, u.w);
         }
         y[o] = v;
+        ymax = fmaxf(ymax, fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w))));
     }
+    if (amax_out) block_amax_to(ymax, amax_out + blockIdx.y);
 }
 
 __global__ void residual_add_bwd_v4_kernel(int NB, int H, int W, int Ca4, int C4, int stride, int ch_off4,
@@ -214,19 +225,23 @@ extern "C" lpdt_status lpdt_sgd_update(int64_t n, const float *x, const float *g
 
 extern "C" lpdt_status lpdt_residual_add(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t Ca,
                                          int32_t C, int32_t stride, int32_t ch_off, const float *r,
-                                         const float *a, float *y, void *stream) {
+                                         const float *a, float *y, float *amax_out, void *stream) {
     LPDT_CHECK_ARG(nodes >= 0 && B >= 0 && H > 0 && W > 0 && Ca > 0 && C >= Ca && stride >= 1);
     LPDT_CHECK_ARG(ch_off >= 0 && ch_off + Ca <= C);
     if (nodes == 0 || B == 0) return LPDT_OK;
-    LPDT_CHECK_ARG(r && a && y);
+    LPDT_CHECK_ARG(r && a && y && nodes <= 65535);
     const int Ho = (H + stride - 1) / stride, Wo = (W + stride - 1) / stride;
-    if (C % 4 == 0 && Ca % 4 == 0 && ch_off % 4 == 0 && aligned(r, 16) && aligned(a, 16) && aligned(y, 16) &&
-        (int64_t)nodes * B < 0x7fffffff)
-        residual_add_v4_kernel<<<grid1d((int64_t)nodes * B * Ho * Wo * C / 4), 256, 0, as_stream(stream)>>>(
-            nodes * B, H, W, Ca / 4, C / 4, stride, ch_off / 4, (const float4 *)r, (const float4 *)a, (float4 *)y);
+    const int64_t per_node = (int64_t)B * Ho * Wo * C;
+    auto gx = [&](int64_t n) {
+        int64_t b = ceil_div(n, 256), cap = ceil_div((int64_t)kNumSMs * 16, nodes);
+        return (unsigned)(b < 1 ? 1 : (b > cap ? cap : b));
+    };
+    if (C % 4 == 0 && Ca % 4 == 0 && ch_off % 4 == 0 && aligned(r, 16) && aligned(a, 16) && aligned(y, 16))
+        residual_add_v4_kernel<<<dim3(gx(per_node / 4), nodes), 256, 0, as_stream(stream)>>>(
+            B, H, W, Ca / 4, C / 4, stride, ch_off / 4, (const float4 *)r, (const float4 *)a, (float4 *)y, amax_out);
     else
-    residual_add_kernel<<<grid1d((int64_t)nodes * B * Ho * Wo * C), 256, 0, as_stream(stream)>>>(
-        (int64_t)nodes * B, H, W, Ca, C, stride, ch_off, r, a, y);
+        residual_add_kernel<<<dim3(gx(per_node), nodes), 256, 0, as_stream(stream)>>>(
+            B, H, W, Ca, C, stride, ch_off, r, a, y, amax_out);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

@@ -92,19 +92,19 @@ template <int MODE /*0 sym rne, 1 sym stochastic, 2 affine*/, bool VEC>
 __global__ void quantize_kernel(const float *__restrict__ x, int64_t n, int64_t stride,
                                 const uint32_t *__restrict__ ws, int8_t *__restrict__ q,
                                 float *__restrict__ scale, int32_t *__restrict__ zero_point,
-                                uint2 key, uint32_t ctr_offset) {
+                                uint2 key, uint32_t ctr_offset, int wstride) {
     const int node = blockIdx.y;
     const float *xn = x + (int64_t)node * stride;
     int8_t *qn = q + (int64_t)node * n;
     float s, inv = 0.f, zf = 0.f;
     if (MODE == 2) {
-        const float hi = __uint_as_float(ws[2 * node]);
-        const float lo = -__uint_as_float(ws[2 * node + 1]);
+        const float hi = __uint_as_float(ws[wstride * node]);
+        const float lo = -__uint_as_float(ws[wstride * node + 1]);
         s = (hi == lo) ? 1.f : __fdiv_rn(__fsub_rn(hi, lo), 255.f);
         zf = rintf(__fdiv_rn(-lo, s));
         zf = fminf(fmaxf(zf, 0.f), 255.f);
     } else {
-        const float amax = __uint_as_float(ws[2 * node]);
+        const float amax = __uint_as_float(ws[wstride * node]);
         if (amax == 0.f) { s = 1.f; inv = 0.f; }
         else { s = __fdiv_rn(amax, 127.f); inv = __fdiv_rn(127.f, amax); }
     }
@@ -209,18 +209,18 @@ extern "C" lpdt_status lpdt_quantize(const float *x, int32_t nodes, int64_t n, i
         if (vec) range_kernel<true, true><<<grid, block, 0, st>>>(x, n, x_node_stride, w);
         else range_kernel<true, false><<<grid, block, 0, st>>>(x, n, x_node_stride, w);
         LPDT_LAUNCH_CHECK();
-        if (vec) quantize_kernel<2, true><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset);
-        else quantize_kernel<2, false><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset);
+        if (vec) quantize_kernel<2, true><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
+        else quantize_kernel<2, false><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
     } else {
         if (vec) range_kernel<false, true><<<grid, block, 0, st>>>(x, n, x_node_stride, w);
         else range_kernel<false, false><<<grid, block, 0, st>>>(x, n, x_node_stride, w);
         LPDT_LAUNCH_CHECK();
         if (rounding == LPDT_ROUND_NEAREST_EVEN) {
-            if (vec) quantize_kernel<0, true><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset);
-            else quantize_kernel<0, false><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset);
+            if (vec) quantize_kernel<0, true><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
+            else quantize_kernel<0, false><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
         } else {
-            if (vec) quantize_kernel<1, true><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset);
-            else quantize_kernel<1, false><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset);
+            if (vec) quantize_kernel<1, true><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
+            else quantize_kernel<1, false><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
         }
     }
     LPDT_LAUNCH_CHECK();
@@ -236,6 +236,32 @@ extern "C" lpdt_status lpdt_dequantize(const int8_t *q, int32_t nodes, int64_t n
     dim3 grid(blocks_for(n, nodes), nodes), block(256);
     if (zero_point) dequantize_kernel<true><<<grid, block, 0, as_stream(stream)>>>(q, n, scale, zero_point, y, y_node_stride);
     else dequantize_kernel<false><<<grid, block, 0, as_stream(stream)>>>(q, n, scale, zero_point, y, y_node_stride);
+    LPDT_LAUNCH_CHECK();
+    return LPDT_OK;
+}
+
+extern "C" lpdt_status lpdt_quantize_with_range(const float *x, int32_t nodes, int64_t n, int64_t x_node_stride,
+                                                const float *amax, lpdt_round rounding, uint64_t seed,
+                                                uint32_t ctr_offset, int8_t *q, float *scale, void *stream) {
+    LPDT_CHECK_ARG(nodes >= 0 && n >= 0);
+    if (nodes == 0 || n == 0) return LPDT_OK;
+    LPDT_CHECK_ARG(x && q && scale && amax);
+    LPDT_CHECK_ARG(x_node_stride >= n || nodes == 1);
+    LPDT_CHECK_ARG(rounding == LPDT_ROUND_NEAREST_EVEN || rounding == LPDT_ROUND_STOCHASTIC);
+    LPDT_CHECK_ARG(aligned(x, 4) && aligned(scale, 4) && aligned(amax, 4));
+    if (nodes > 65535) return LPDT_ERR_UNSUPPORTED;
+    cudaStream_t st = as_stream(stream);
+    const uint32_t *w = reinterpret_cast<const uint32_t *>(amax);      // non-negative floats, read as bit patterns
+    const bool vec = aligned(x, 16) && (x_node_stride % 4 == 0) && (n % 4 == 0) && aligned(q, 4);
+    dim3 grid(blocks_for(vec ? n / 4 : n, nodes), nodes), block(256);
+    const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
+    if (rounding == LPDT_ROUND_NEAREST_EVEN) {
+        if (vec) quantize_kernel<0, true><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, nullptr, key, ctr_offset, 1);
+        else quantize_kernel<0, false><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, nullptr, key, ctr_offset, 1);
+    } else {
+        if (vec) quantize_kernel<1, true><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, nullptr, key, ctr_offset, 1);
+        else quantize_kernel<1, false><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, nullptr, key, ctr_offset, 1);
+    }
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

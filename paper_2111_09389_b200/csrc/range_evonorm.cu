@@ -85,7 +85,7 @@ ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
                const float *__restrict__ x, const float *__restrict__ v,
                const float *__restrict__ gamma, const float *__restrict__ beta, int64_t pstride,
                int B, float *__restrict__ y, float *__restrict__ gmin, float *__restrict__ gmax,
-               int32_t *__restrict__ argmin, int32_t *__restrict__ argmax) {
+               int32_t *__restrict__ argmin, int32_t *__restrict__ argmax, float *__restrict__ amax_out) {
     extern __shared__ unsigned char smem_raw[];
     const int T = blockDim.x, t = threadIdx.x;
     Ext *s_mn = reinterpret_cast<Ext *>(smem_raw);
@@ -120,6 +120,7 @@ ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
     const float D = __fadd_rn(__fmul_rn(Cst, rng), eps);
     const float invD = __fdiv_rn(1.f, D);
     float vc[V], gc[V], bc[V];
+    float ymax = 0.f;
 #pragma unroll
     for (int k = 0; k < V; ++k) {
         vc[k] = v[(int64_t)node * pstride + c0 + k];
@@ -134,9 +135,11 @@ ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
             float u = __fmul_rn(vc[k], xv[k]);
             float m = __fmul_rn(xv[k], hsig(u));
             yv[k] = __fadd_rn(__fmul_rn(__fmul_rn(gc[k], m), invD), bc[k]);
+            ymax = fmaxf(ymax, fabsf(yv[k]));
         }
         VecLoad<V>::st(ys + (int64_t)p * C + c0, yv);
     }
+    if (amax_out) block_amax_to(ymax, amax_out + node);
 }
 
 template <int V>
@@ -146,7 +149,7 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
                const float *__restrict__ v, const float *__restrict__ gamma, int64_t pstride, int B,
                const float *__restrict__ gmin, const float *__restrict__ gmax,
                const int32_t *__restrict__ argmin, const int32_t *__restrict__ argmax,
-               float *__restrict__ dx, double *__restrict__ acc /*[nodes][3][C]*/) {
+               float *__restrict__ dx, double *__restrict__ acc /*[nodes][3][C]*/, float *__restrict__ amax_out) {
     extern __shared__ unsigned char smem_raw[];
     const int T = blockDim.x, t = threadIdx.x;
     double *s_ch = reinterpret_cast<double *>(smem_raw);      // [3][C]
@@ -177,6 +180,10 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
     // The per-channel parameter-gradient sums take a short fp32 run per thread (at most
     // kRunLen terms) before they join the double accumulators.
     constexpr int kRunLen = 16;
+    // max|dx| for the consumer's quantizer: the two extremum positions are left out here and
+    // added after their correction
+    const int g_amx = argmax[sg], g_amn = argmin[sg];
+    float dmax = 0.f;
     double S = 0.0, ab[V], ag[V], av[V];
     float fb[V], fg[V], fv[V];
     int run = 0;
@@ -195,6 +202,8 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
             float tt = __fmul_rn(dv_[k], gc[k]);
             S += (double)__fmul_rn(tt, m);
             o[k] = __fmul_rn(__fmul_rn(tt, __fadd_rn(hs, __fmul_rn(u, hp))), invD);
+            const int idx = p * C + c0 + k;
+            if (idx != g_amx && idx != g_amn) dmax = fmaxf(dmax, fabsf(o[k]));
             fb[k] = __fadd_rn(fb[k], dv_[k]);
             fg[k] = __fadd_rn(fg[k], __fmul_rn(dv_[k], __fmul_rn(m, invD)));
             fv[k] = __fadd_rn(fv[k], __fmul_rn(__fmul_rn(__fmul_rn(tt, __fmul_rn(xv[k], xv[k])), hp), invD));
@@ -258,10 +267,14 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
             float coef = __fmul_rn(Cst, (float)g_S[t]);
             coef = __fmul_rn(coef, invDg);
             coef = __fmul_rn(coef, invDg);
-            dxs[amx] = __fsub_rn(dxs[amx], coef);
-            dxs[amn] = __fadd_rn(dxs[amn], coef);
+            const float va = __fsub_rn(dxs[amx], coef), vb = __fadd_rn(dxs[amn], coef);
+            dxs[amx] = va; dxs[amn] = vb;
+            dmax = fmaxf(dmax, fmaxf(fabsf(va), fabsf(vb)));
+        } else {
+            dmax = fmaxf(dmax, fabsf(dxs[amx]));
         }
     }
+    if (amax_out) block_amax_to(dmax, amax_out + node);
 }
 
 __global__ void ren_bwd_finalize(const double *__restrict__ acc, int nodes, int C,
@@ -304,7 +317,7 @@ extern "C" lpdt_status lpdt_range_evonorm_fwd(int32_t nodes, int32_t B, int32_t 
                                               int32_t groups, float eps, const float *x, const float *v,
                                               const float *gamma, const float *beta, int64_t pstride,
                                               float *y, float *gmin, float *gmax, int32_t *argmin,
-                                              int32_t *argmax, void *stream) {
+                                              int32_t *argmax, float *amax_out, void *stream) {
     LPDT_CHECK_ARG(nodes >= 0 && B >= 0 && H > 0 && W > 0 && C > 0 && groups > 0);
     LPDT_CHECK_ARG(C % groups == 0 && C / groups >= 2);
     if (nodes == 0 || B == 0) return LPDT_OK;
@@ -318,9 +331,9 @@ extern "C" lpdt_status lpdt_range_evonorm_fwd(int32_t nodes, int32_t B, int32_t 
     const float Cst = ren_const(C / groups);
     dim3 grid((unsigned)((int64_t)nodes * B));
     if (pl.V == 4)
-        ren_fwd_kernel<4><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax);
+        ren_fwd_kernel<4><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out);
     else
-        ren_fwd_kernel<1><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax);
+        ren_fwd_kernel<1><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }
@@ -335,7 +348,8 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t 
                                               const float *gmin, const float *gmax,
                                               const int32_t *argmin, const int32_t *argmax,
                                               float *dx, float *dv, float *dgamma, float *dbeta,
-                                              int64_t gstride, void *ws, size_t ws_bytes, void *stream) {
+                                              int64_t gstride, float *amax_out, void *ws, size_t ws_bytes,
+                                              void *stream) {
     LPDT_CHECK_ARG(nodes >= 0 && B >= 0 && H > 0 && W > 0 && C > 0 && groups > 0);
     LPDT_CHECK_ARG(C % groups == 0 && C / groups >= 2);
     if (nodes == 0 || B == 0) return LPDT_OK;
@@ -354,9 +368,9 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t 
     const float Cst = ren_const(C / groups);
     dim3 grid((unsigned)((int64_t)nodes * B));
     if (pl.V == 4)
-        ren_bwd_kernel<4><<<grid, pl.threads, smem, st>>>(H * W, C, groups, eps, Cst, dy, x, v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc);
+        ren_bwd_kernel<4><<<grid, pl.threads, smem, st>>>(H * W, C, groups, eps, Cst, dy, x, v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc, amax_out);
     else
-        ren_bwd_kernel<1><<<grid, pl.threads, smem, st>>>(H * W, C, groups, eps, Cst, dy, x, v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc);
+        ren_bwd_kernel<1><<<grid, pl.threads, smem, st>>>(H * W, C, groups, eps, Cst, dy, x, v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc, amax_out);
     LPDT_LAUNCH_CHECK();
     ren_bwd_finalize<<<(nodes * C + 255) / 256, 256, 0, st>>>(acc, nodes, C, dv, dgamma, dbeta, gstride);
     LPDT_LAUNCH_CHECK();

@@ -94,6 +94,9 @@ class TrainStep:
                 raise ValueError(k)
             self.buf.append(b)
         self.out_shape = shape
+        # per-node ranges emitted by producers for the next quantizer: row li = forward output of op li,
+        # row len(ops)+li = layer gradient leaving op li; zeroed once per step
+        self.ranges = torch.zeros(2 * len(ops), N, **f32)
         self.dy = torch.zeros((N, B) + tuple(shape), **f32)      # upstream gradient / dlogits
         self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
 
@@ -126,38 +129,44 @@ class TrainStep:
     def forward(self):
         N, B, d = self.N, self.B, self.d
         cur = self.x
+        cur_range = None          # per-node max|cur| when the producer of cur emitted it
         saved = []
-        for op, b in zip(self.ops, self.buf):
+        api.lpdt_fill_zero(self.ranges)
+        for li, (op, b) in enumerate(zip(self.ops, self.buf)):
             k = op["op"]
             if k in ("conv", "linear"):
                 n_in = cur.numel() // N
-                api.lpdt_quantize(cur, N, n_in, n_in, b["qA"], b["sA"], self.ws)
+                if cur_range is not None:
+                    api.lpdt_quantize_with_range(cur, N, n_in, n_in, cur_range, b["qA"], b["sA"])
+                else:
+                    api.lpdt_quantize(cur, N, n_in, n_in, b["qA"], b["sA"], self.ws)
                 api.lpdt_quantize(self._p(op["w_off"]), N, b["wn"], d, b["qW"], b["sW"], self.ws)
                 bias = self._p(op["b_off"]) if k == "linear" else None
                 api.lpdt_qconv_fwd(b["desc"], b["qA"], b["sA"], b["qW"], b["sW"], Y=b["out"], bias=bias,
                                    bias_node_stride=d, ws=self.ws, dev_status=self.dev_status)
-                cur = b["out"]
+                cur, cur_range = b["out"], None
             elif k == "ren":
                 Cc = op["C"]
                 b["x"] = cur
                 api.lpdt_range_evonorm_fwd(N, B, op["H"], op["W"], Cc, op["groups"], self.eps, cur,
                                            self._p(op["p_off"]), self._p(op["p_off"] + Cc),
                                            self._p(op["p_off"] + 2 * Cc), d, b["out"], b["gmin"], b["gmax"],
-                                           b["amin"], b["amax"])
-                cur = b["out"]
+                                           b["amin"], b["amax"], amax_out=self.ranges[li])
+                cur, cur_range = b["out"], self.ranges[li]
             elif k == "save":
                 saved.append(cur)
             elif k == "add":
                 a = saved.pop()
                 api.lpdt_residual_add(N, B, op["H"], op["W"], op["Ca"], op["C"], op["stride"], op["ch_off"],
-                                      cur, a, b["out"])
-                cur = b["out"]
+                                      cur, a, b["out"], amax_out=self.ranges[li])
+                cur, cur_range = b["out"], self.ranges[li]
             elif k == "maxpool":
                 api.lpdt_maxpool2x2(N, B, op["H"], op["W"], op["C"], cur, b["out"], b["idx"])
-                cur = b["out"]
+                cur = b["out"]        # max-pooling keeps max|x| only for non-negative maxima: range recomputed
+                cur_range = None
             elif k == "avgpool":
                 api.lpdt_avgpool(N, B, op["H"] * op["W"], op["C"], cur, b["out"])
-                cur = b["out"]
+                cur, cur_range = b["out"], None
         self.out = cur
         return cur
 
@@ -167,6 +176,8 @@ class TrainStep:
             K = self.out.numel() // (N * B)
             api.lpdt_softmax_ce(N, B, K, self.out, self.labels, self.loss, self.dy)
         g = self.dy
+        g_range = None
+        L = len(self.ops)
         sc = []
         ctr = 0
         for li in range(len(self.ops) - 1, -1, -1):
@@ -176,8 +187,12 @@ class TrainStep:
                 if k == "linear":
                     api.lpdt_colsum(N, B, op["cout"], g, self._g(op["b_off"]), d)
                 n_out = g.numel() // N
-                api.lpdt_quantize(g, N, n_out, n_out, b["E"], b["sE"], self.ws, rounding=self.grad_rounding,
-                                  seed=self.seed, ctr_offset=ctr)
+                if g_range is not None:
+                    api.lpdt_quantize_with_range(g, N, n_out, n_out, g_range, b["E"], b["sE"],
+                                                 rounding=self.grad_rounding, seed=self.seed, ctr_offset=ctr)
+                else:
+                    api.lpdt_quantize(g, N, n_out, n_out, b["E"], b["sE"], self.ws, rounding=self.grad_rounding,
+                                      seed=self.seed, ctr_offset=ctr)
                 ctr += 1
                 if self.quantize_wgrad:
                     api.lpdt_qconv_bwd_weight(b["desc"], b["E"], b["sE"], b["qA"], b["sA"], dW=b["gw"],
@@ -191,7 +206,7 @@ class TrainStep:
                 if li > 0 or self.input_grad:
                     api.lpdt_qconv_bwd_data(b["desc"], b["E"], b["sE"], b["qW"], b["sW"], dA=b["dx"],
                                             ws=self.ws, dev_status=self.dev_status)
-                    g = b["dx"]
+                    g, g_range = b["dx"], None
                 else:
                     g = None
             elif k == "ren":
@@ -199,21 +214,22 @@ class TrainStep:
                 api.lpdt_range_evonorm_bwd(N, B, op["H"], op["W"], Cc, op["groups"], self.eps, g, b["x"],
                                            self._p(op["p_off"]), self._p(op["p_off"] + Cc), d, b["gmin"],
                                            b["gmax"], b["amin"], b["amax"], b["dx"], self._g(op["p_off"]),
-                                           self._g(op["p_off"] + Cc), self._g(op["p_off"] + 2 * Cc), d, self.ws)
-                g = b["dx"]
+                                           self._g(op["p_off"] + Cc), self._g(op["p_off"] + 2 * Cc), d, self.ws,
+                                           amax_out=self.ranges[L + li])
+                g, g_range = b["dx"], self.ranges[L + li]
             elif k == "add":
                 sc.append((g, op))
             elif k == "save":
                 dy_sc, aop = sc.pop()
                 api.lpdt_residual_add_bwd(N, B, aop["H"], aop["W"], aop["Ca"], aop["C"], aop["stride"],
                                           aop["ch_off"], dy_sc, g, b["dx"])
-                g = b["dx"]
+                g, g_range = b["dx"], None
             elif k == "maxpool":
                 api.lpdt_maxpool2x2_bwd(N, B, op["H"], op["W"], op["C"], g, b["idx"], b["dx"])
-                g = b["dx"]
+                g, g_range = b["dx"], None
             elif k == "avgpool":
                 api.lpdt_avgpool_bwd(N, B, op["H"] * op["W"], op["C"], g, b["dx"])
-                g = b["dx"]
+                g, g_range = b["dx"], None
         self.input_grad_out = g
         return g
 

@@ -259,6 +259,43 @@ def test_range_evonorm_fwd_bwd(case, ties):
     assert not Gh[:, 3 * C:].any()
 
 
+def test_fused_ranges_feed_the_quantizer_exactly():
+    # the producers' per-node max|x| must equal the range pass bit for bit, so that
+    # lpdt_quantize_with_range gives the same codes as lpdt_quantize
+    case = (3, 4, 16, 16, 16, 2)
+    nodes, B, H, W, C, groups = case
+    x, P, dy = _ren_inputs(case, seed=5, ties=True)
+    v, g, b = P[:, :C], P[:, C:2 * C], P[:, 2 * C:3 * C]
+    y32, mn, mx, amn, amx = oracle.range_evonorm_fwd(x, v, g, b, groups, 1e-5, "f32")
+    dx32 = oracle.range_evonorm_bwd(dy, x, v, g, mn, mx, amn, amx, groups, 1e-5, "f32")[0]
+    xd, Pd = dev(x), dev(P)
+    stride = P.shape[1]
+    f = lambda *s: torch.empty(*s, dtype=torch.float32, device="cuda")
+    i = lambda *s: torch.empty(*s, dtype=torch.int32, device="cuda")
+    ranges = torch.zeros(3, nodes, device="cuda")
+    y, gmin, gmax, amin_, amax_ = f(*x.shape), f(nodes, B, groups), f(nodes, B, groups), i(nodes, B, groups), i(nodes, B, groups)
+    api.lpdt_range_evonorm_fwd(nodes, B, H, W, C, groups, 1e-5, xd, Pd, Pd[:, C:], Pd[:, 2 * C:], stride, y, gmin, gmax,
+                               amin_, amax_, amax_out=ranges[0])
+    G = torch.zeros(nodes, stride, device="cuda")
+    dx = f(*x.shape)
+    ws = ws_bytes(api.lpdt_range_evonorm_bwd_workspace_size(nodes, C))
+    api.lpdt_range_evonorm_bwd(nodes, B, H, W, C, groups, 1e-5, dev(dy), xd, Pd, Pd[:, C:], stride, gmin, gmax, amin_, amax_,
+                               dx, G, G[:, C:], G[:, 2 * C:], stride, ws, amax_out=ranges[1])
+    r = f(*x.shape)
+    api.lpdt_residual_add(nodes, B, H, W, C, C, 1, 0, y, dx, r, amax_out=ranges[2])
+    rh = ranges.cpu().numpy()
+    assert np.array_equal(rh[0], np.abs(y32).reshape(nodes, -1).max(1))
+    assert np.array_equal(rh[1], np.abs(dx.cpu().numpy()).reshape(nodes, -1).max(1))
+    assert np.array_equal(rh[2], np.abs(r.cpu().numpy()).reshape(nodes, -1).max(1))
+    n = B * H * W * C
+    for t, row, rounding in ((y, 0, 0), (dx, 1, 1), (r, 2, 0)):
+        q1 = torch.empty(nodes, n, dtype=torch.int8, device="cuda"); s1 = f(nodes)
+        q2 = torch.empty(nodes, n, dtype=torch.int8, device="cuda"); s2 = f(nodes)
+        api.lpdt_quantize(t, nodes, n, n, q1, s1, ws_bytes(256), rounding=rounding, seed=5, ctr_offset=1)
+        api.lpdt_quantize_with_range(t, nodes, n, n, ranges[row], q2, s2, rounding=rounding, seed=5, ctr_offset=1)
+        assert torch.equal(q1, q2) and torch.equal(s1, s2)
+
+
 def test_range_evonorm_errors():
     t = torch.zeros(64, device="cuda"); ti = torch.zeros(64, dtype=torch.int32, device="cuda")
     with pytest.raises(api.LpdtError) as e:      # one channel per group: the constant is infinite
