@@ -201,7 +201,7 @@ lpdt_status lpdt_range_evonorm_fwd(int32_t nodes, int32_t B, int32_t H, int32_t 
                                    int64_t param_node_stride, float *y,
                                    float *gmin, float *gmax, int32_t *argmin, int32_t *argmax,
                                    float *amax_out, void *stream);
-size_t lpdt_range_evonorm_bwd_workspace_size(int32_t nodes, int32_t C);
+size_t lpdt_range_evonorm_bwd_workspace_size(int32_t nodes, int32_t B, int32_t C);
 lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C,
                                    int32_t groups, float eps, const float *dy, const float *x,
                                    const float *v, const float *gamma, int64_t param_node_stride,

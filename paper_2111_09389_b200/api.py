@@ -157,8 +157,8 @@ def lpdt_range_evonorm_fwd(nodes, B, H, W, Cc, groups, eps, x, v, gamma, beta, p
         _ptr(y), _ptr(gmin), _ptr(gmax), _ptr(argmin), _ptr(argmax), _ptr(amax_out), _stream()))
 
 
-def lpdt_range_evonorm_bwd_workspace_size(nodes, Cc):
-    return lib().lpdt_range_evonorm_bwd_workspace_size(nodes, Cc)
+def lpdt_range_evonorm_bwd_workspace_size(nodes, B, Cc):
+    return lib().lpdt_range_evonorm_bwd_workspace_size(nodes, B, Cc)
 
 
 def lpdt_range_evonorm_bwd(nodes, B, H, W, Cc, groups, eps, dy, x, v, gamma, param_node_stride, gmin,

@@ -149,7 +149,8 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
                const float *__restrict__ v, const float *__restrict__ gamma, int64_t pstride, int B,
                const float *__restrict__ gmin, const float *__restrict__ gmax,
                const int32_t *__restrict__ argmin, const int32_t *__restrict__ argmax,
-               float *__restrict__ dx, double *__restrict__ acc /*[nodes][3][C]*/, float *__restrict__ amax_out) {
+               float *__restrict__ dx, double *__restrict__ acc /*[nodes][B][3][C] per-sample partial sums*/,
+               float *__restrict__ amax_out) {
     extern __shared__ unsigned char smem_raw[];
     const int T = blockDim.x, t = threadIdx.x;
     double *s_ch = reinterpret_cast<double *>(smem_raw);      // [3][C]
@@ -253,7 +254,7 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
             if (lane == 0) g_S[g] = a;
         }
     }
-    for (int i = t; i < 3 * C; i += T) atomicAdd(&acc[(int64_t)node * 3 * C + i], s_ch[i]);
+    for (int i = t; i < 3 * C; i += T) acc[sample * 3 * C + i] = s_ch[i];      // summed over the batch by the finalize kernel
     __syncthreads();
     // The group sum only enters dx at the two extremum positions: one thread per group
     // applies the correction to the local term already stored there (same operation order
@@ -277,16 +278,18 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
     if (amax_out) block_amax_to(dmax, amax_out + node);
 }
 
-__global__ void ren_bwd_finalize(const double *__restrict__ acc, int nodes, int C,
+// Sum the per-sample partials of a node in sample order (deterministic) and round once.
+__global__ void ren_bwd_finalize(const double *__restrict__ acc, int nodes, int B, int C,
                                  float *__restrict__ dv, float *__restrict__ dgamma,
                                  float *__restrict__ dbeta, int64_t gstride) {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= nodes * C) return;
-    int node = i / C, c = i % C;
-    const double *a = acc + (int64_t)node * 3 * C;
-    dv[(int64_t)node * gstride + c] = (float)a[c];
-    dgamma[(int64_t)node * gstride + c] = (float)a[C + c];
-    dbeta[(int64_t)node * gstride + c] = (float)a[2 * C + c];
+    if (i >= nodes * 3 * C) return;
+    const int node = i / (3 * C), j = i % (3 * C), which = j / C, c = j % C;
+    const double *a = acc + (int64_t)node * B * 3 * C + j;
+    double s = 0.0;
+    for (int b = 0; b < B; ++b) s += a[(int64_t)b * 3 * C];
+    float *dst = which == 0 ? dv : which == 1 ? dgamma : dbeta;
+    dst[(int64_t)node * gstride + c] = (float)s;
 }
 
 struct RenPlan { int V, threads; };
@@ -338,8 +341,9 @@ extern "C" lpdt_status lpdt_range_evonorm_fwd(int32_t nodes, int32_t B, int32_t 
     return LPDT_OK;
 }
 
-extern "C" size_t lpdt_range_evonorm_bwd_workspace_size(int32_t nodes, int32_t C) {
-    return align_up((size_t)(nodes > 0 ? nodes : 1) * 3 * (size_t)(C > 0 ? C : 1) * sizeof(double), 256);
+extern "C" size_t lpdt_range_evonorm_bwd_workspace_size(int32_t nodes, int32_t B, int32_t C) {
+    return align_up((size_t)(nodes > 0 ? nodes : 1) * (size_t)(B > 0 ? B : 1) * 3 * (size_t)(C > 0 ? C : 1) *
+                    sizeof(double), 256);
 }
 
 extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C,
@@ -356,7 +360,7 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t 
     LPDT_CHECK_ARG(dy && x && v && gamma && gmin && gmax && argmin && argmax && dx && dv && dgamma && dbeta);
     LPDT_CHECK_ARG((pstride >= C && gstride >= C) || nodes == 1);
     if ((int64_t)H * W * C > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
-    if (!ws || ws_bytes < lpdt_range_evonorm_bwd_workspace_size(nodes, C) || !aligned(ws, 8))
+    if (!ws || ws_bytes < lpdt_range_evonorm_bwd_workspace_size(nodes, B, C) || !aligned(ws, 8))
         return LPDT_ERR_WORKSPACE;
     RenPlan pl;
     if (!plan(C, groups, aligned(x, 16) && aligned(dy, 16) && aligned(dx, 16), &pl)) return LPDT_ERR_UNSUPPORTED;
@@ -364,7 +368,6 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t 
     if (smem > 48 * 1024) return LPDT_ERR_UNSUPPORTED;
     cudaStream_t st = as_stream(stream);
     double *acc = (double *)ws;
-    LPDT_CUDA(cudaMemsetAsync(acc, 0, (size_t)nodes * 3 * C * sizeof(double), st));
     const float Cst = ren_const(C / groups);
     dim3 grid((unsigned)((int64_t)nodes * B));
     if (pl.V == 4)
@@ -372,7 +375,7 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t 
     else
         ren_bwd_kernel<1><<<grid, pl.threads, smem, st>>>(H * W, C, groups, eps, Cst, dy, x, v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc, amax_out);
     LPDT_LAUNCH_CHECK();
-    ren_bwd_finalize<<<(nodes * C + 255) / 256, 256, 0, st>>>(acc, nodes, C, dv, dgamma, dbeta, gstride);
+    ren_bwd_finalize<<<(nodes * 3 * C + 255) / 256, 256, 0, st>>>(acc, nodes, B, C, dv, dgamma, dbeta, gstride);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

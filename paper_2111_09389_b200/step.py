@@ -74,7 +74,7 @@ class TrainStep:
                 b.update(out=torch.empty(N, B, H, W, Cc, **f32), dx=torch.empty(N, B, H, W, Cc, **f32),
                          gmin=torch.empty(N, B, G, **f32), gmax=torch.empty(N, B, G, **f32),
                          amin=torch.empty(N, B, G, **i32), amax=torch.empty(N, B, G, **i32))
-                ws_bytes = max(ws_bytes, api.lpdt_range_evonorm_bwd_workspace_size(N, Cc))
+                ws_bytes = max(ws_bytes, api.lpdt_range_evonorm_bwd_workspace_size(N, B, Cc))
             elif k == "add":
                 Ho, Wo = (op["H"] + op["stride"] - 1) // op["stride"], (op["W"] + op["stride"] - 1) // op["stride"]
                 b.update(out=torch.empty(N, B, Ho, Wo, op["C"], **f32))

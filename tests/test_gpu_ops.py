@@ -246,7 +246,7 @@ def test_range_evonorm_fwd_bwd(case, ties):
     dx64, dv64, dg64, db64 = oracle.range_evonorm_bwd(dy, x, v, g, mn, mx, amn, amx, groups, eps, "f64")
     G = torch.zeros(nodes, stride, dtype=torch.float32, device="cuda")
     dx = f(*x.shape)
-    ws = ws_bytes(api.lpdt_range_evonorm_bwd_workspace_size(nodes, C))
+    ws = ws_bytes(api.lpdt_range_evonorm_bwd_workspace_size(nodes, B, C))
     api.lpdt_range_evonorm_bwd(nodes, B, H, W, C, groups, eps, dev(dy), xd, Pd, Pd[:, C:], stride, gmin, gmax, amin_, amax_,
                                dx, G, G[:, C:], G[:, 2 * C:], stride, ws)
     close(dx, dx32, 1e-6, 1e-7)
@@ -278,7 +278,7 @@ def test_fused_ranges_feed_the_quantizer_exactly():
                                amin_, amax_, amax_out=ranges[0])
     G = torch.zeros(nodes, stride, device="cuda")
     dx = f(*x.shape)
-    ws = ws_bytes(api.lpdt_range_evonorm_bwd_workspace_size(nodes, C))
+    ws = ws_bytes(api.lpdt_range_evonorm_bwd_workspace_size(nodes, B, C))
     api.lpdt_range_evonorm_bwd(nodes, B, H, W, C, groups, 1e-5, dev(dy), xd, Pd, Pd[:, C:], stride, gmin, gmax, amin_, amax_,
                                dx, G, G[:, C:], G[:, 2 * C:], stride, ws, amax_out=ranges[1])
     r = f(*x.shape)
