@@ -143,7 +143,7 @@ ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
 }
 
 template <int V>
-__global__ void __launch_bounds__(512)
+__global__ void __launch_bounds__(512, 2)
 ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
                const float *__restrict__ dy, const float *__restrict__ x,
                const float *__restrict__ v, const float *__restrict__ gamma, int64_t pstride, int B,
@@ -185,61 +185,56 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
     // added after their correction
     const int g_amx = argmax[sg], g_amn = argmin[sg];
     float dmax = 0.f;
-    double S = 0.0, ab[V], ag[V], av[V];
+    double S = 0.0;
     float fb[V], fg[V], fv[V];
-    int run = 0;
 #pragma unroll
-    for (int k = 0; k < V; ++k) { ab[k] = 0.0; ag[k] = 0.0; av[k] = 0.0; fb[k] = 0.f; fg[k] = 0.f; fv[k] = 0.f; }
-    for (int p = row0; p < HW; p += rstep) {
-        float xv[V], dv_[V], o[V];
-        VecLoad<V>::ld(xs + (int64_t)p * C + c0, xv);
-        VecLoad<V>::ld(dys + (int64_t)p * C + c0, dv_);
-#pragma unroll
-        for (int k = 0; k < V; ++k) {
-            float u = __fmul_rn(vc[k], xv[k]);
-            float hs = hsig(u);
-            float hp = (u > -3.f && u < 3.f) ? sixth : 0.f;
-            float m = __fmul_rn(xv[k], hs);
-            float tt = __fmul_rn(dv_[k], gc[k]);
-            S += (double)__fmul_rn(tt, m);
-            o[k] = __fmul_rn(__fmul_rn(tt, __fadd_rn(hs, __fmul_rn(u, hp))), invD);
-            const int idx = p * C + c0 + k;
-            if (idx != g_amx && idx != g_amn) dmax = fmaxf(dmax, fabsf(o[k]));
-            fb[k] = __fadd_rn(fb[k], dv_[k]);
-            fg[k] = __fadd_rn(fg[k], __fmul_rn(dv_[k], __fmul_rn(m, invD)));
-            fv[k] = __fadd_rn(fv[k], __fmul_rn(__fmul_rn(__fmul_rn(tt, __fmul_rn(xv[k], xv[k])), hp), invD));
-        }
-        VecLoad<V>::st(dxs + (int64_t)p * C + c0, o);
-        if (++run == kRunLen) {
-            run = 0;
+    for (int k = 0; k < V; ++k) { fb[k] = 0.f; fg[k] = 0.f; fv[k] = 0.f; }
+    __syncthreads();   // s_ch zeroed
+    // When the column count divides the warp, lanes that share a column are folded with
+    // shuffles first, so only CV lanes per warp touch the shared fp64 accumulators.
+    const bool fold = (CV <= 32) && (32 % CV == 0);
+    const int iters = (HW - 1) / rstep + 1;          // same trip count for every thread (rows are predicated)
+    for (int i = 0; i < iters; ++i) {
+        const int p = row0 + i * rstep;
+        if (p < HW) {
+            float xv[V], dv_[V], o[V];
+            VecLoad<V>::ld(xs + (int64_t)p * C + c0, xv);
+            VecLoad<V>::ld(dys + (int64_t)p * C + c0, dv_);
 #pragma unroll
             for (int k = 0; k < V; ++k) {
-                ab[k] += (double)fb[k]; ag[k] += (double)fg[k]; av[k] += (double)fv[k];
+                float u = __fmul_rn(vc[k], xv[k]);
+                float hs = hsig(u);
+                float hp = (u > -3.f && u < 3.f) ? sixth : 0.f;
+                float m = __fmul_rn(xv[k], hs);
+                float tt = __fmul_rn(dv_[k], gc[k]);
+                S += (double)__fmul_rn(tt, m);
+                o[k] = __fmul_rn(__fmul_rn(tt, __fadd_rn(hs, __fmul_rn(u, hp))), invD);
+                const int idx = p * C + c0 + k;
+                if (idx != g_amx && idx != g_amn) dmax = fmaxf(dmax, fabsf(o[k]));
+                fb[k] = __fadd_rn(fb[k], dv_[k]);
+                fg[k] = __fadd_rn(fg[k], __fmul_rn(dv_[k], __fmul_rn(m, invD)));
+                fv[k] = __fadd_rn(fv[k], __fmul_rn(__fmul_rn(__fmul_rn(tt, __fmul_rn(xv[k], xv[k])), hp), invD));
+            }
+            VecLoad<V>::st(dxs + (int64_t)p * C + c0, o);
+        }
+        if ((i + 1) % kRunLen == 0 || i == iters - 1) {      // uniform across the block
+#pragma unroll
+            for (int k = 0; k < V; ++k) {
+                double a = (double)fv[k], b = (double)fg[k], c = (double)fb[k];
+                if (fold) {
+                    for (int o = 16; o >= CV; o >>= 1) {
+                        a += __shfl_xor_sync(0xffffffffu, a, o);
+                        b += __shfl_xor_sync(0xffffffffu, b, o);
+                        c += __shfl_xor_sync(0xffffffffu, c, o);
+                    }
+                }
+                if (!fold || (t & 31) < CV) {
+                    atomicAdd(&s_ch[0 * C + c0 + k], a);
+                    atomicAdd(&s_ch[1 * C + c0 + k], b);
+                    atomicAdd(&s_ch[2 * C + c0 + k], c);
+                }
                 fb[k] = 0.f; fg[k] = 0.f; fv[k] = 0.f;
             }
-        }
-    }
-#pragma unroll
-    for (int k = 0; k < V; ++k) { ab[k] += (double)fb[k]; ag[k] += (double)fg[k]; av[k] += (double)fv[k]; }
-    __syncthreads();   // s_ch zeroed
-    // Per-channel sums: when the column count divides the warp, lanes that share a
-    // column are first folded with shuffles, so only CV lanes per warp touch shared memory.
-    const bool fold = (CV <= 32) && (32 % CV == 0);
-    if (fold) {
-#pragma unroll
-        for (int k = 0; k < V; ++k)
-            for (int o = 16; o >= CV; o >>= 1) {
-                av[k] += __shfl_xor_sync(0xffffffffu, av[k], o);
-                ag[k] += __shfl_xor_sync(0xffffffffu, ag[k], o);
-                ab[k] += __shfl_xor_sync(0xffffffffu, ab[k], o);
-            }
-    }
-    if (!fold || (t & 31) < CV) {
-#pragma unroll
-        for (int k = 0; k < V; ++k) {
-            atomicAdd(&s_ch[0 * C + c0 + k], av[k]);
-            atomicAdd(&s_ch[1 * C + c0 + k], ag[k]);
-            atomicAdd(&s_ch[2 * C + c0 + k], ab[k]);
         }
     }
     s_S[t] = S;
