@@ -284,6 +284,7 @@ struct WgParams {
     int TB, TH, TW, tilesB, tilesH, tilesW;       // pixel tiles = K blocks
     int kblocks, splits, kb_per_split;
     int RBx, RBe, merged;                         // row bytes of the input tiles and of the error tiles
+    int halo, PW, PH, halo_bytes;                 // 16-channel halo mode: one input box per pixel tile (see below)
     int mgroups, ngroups, mtiles, BNc, total_units;
     int stages, tmem_cols;
     int32_t *acc_out; int32_t *dev_status;
@@ -305,7 +306,7 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     const int mu0 = mg * p.mtiles * G;
     int nX = p.total_units - mu0; if (nX > p.mtiles * G) nX = p.mtiles * G;
     const int n0 = ng * p.BNc, nE = p.BNc / p.RBe;
-    const int x_region = p.mtiles * 16384;
+    const int x_region = p.halo ? p.halo_bytes : p.mtiles * 16384;
     const int stage_bytes = x_region + 128 * p.BNc;
     const int kb0 = blockIdx.x * p.kb_per_split;
     int kb1 = kb0 + p.kb_per_split; if (kb1 > p.kblocks) kb1 = p.kblocks;
@@ -334,13 +335,15 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                 if (!mbar_wait(smem_u32(&ctl->empty[st]), ph ^ 1, &ctl->abort_flag, p.dev_status)) break;
                 const uint32_t full = smem_u32(&ctl->full[st]);
                 const bool leader = elect_one();
-                if (leader) mbar_expect_tx(full, nX * x_unit + nE * e_unit);
+                if (leader) mbar_expect_tx(full, (p.halo ? p.PW * p.PH * 16 : nX * x_unit) + nE * e_unit);
                 uint32_t x_dst = smem_u32(data + (size_t)st * stage_bytes);
                 uint32_t e_dst = x_dst + x_region;
                 for (int c = 0; c < nE; ++c, e_dst += e_unit)
                     if (leader) tma_load_5d(e_dst, &mapE, full, n0 + c * p.RBe, w0, h0, b0, node);
+                // halo mode: the 8 x 16 pixel tile plus its filter halo in one box; taps are descriptor offsets
+                if (p.halo && leader) tma_load_4d(x_dst, &mapX, full, (w0 - p.pad) * 16, h0 - p.pad, b0, node);
                 int chunk = chunk0, r = r0, s = s0;
-                for (int i = 0; i < nX; ++i, x_dst += x_unit) {
+                for (int i = 0; i < (p.halo ? 0 : nX); ++i, x_dst += x_unit) {
                     const int wc = w0 * p.stride + s - p.pad, hc = h0 * p.stride + r - p.pad;
                     if (leader) {
                         if (p.merged) tma_load_4d(x_dst, &mapX, full, wc * 16, hc, b0, node);
@@ -356,11 +359,16 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     } else if (warp == 1) {
         {
             const uint32_t idesc = idesc_i8(128, p.BNc, 1, 1);
-            const uint64_t a_tpl = (p.RBx == 16) ? smem_desc(0, 128, x_unit, 0)
+            // halo mode: M tile r stacks the S taps of filter row r, one pixel (16 bytes) apart; 8-pixel
+            // K groups are one halo row apart
+            const uint64_t a_tpl = p.halo ? smem_desc(0, p.PW * 16, 16, 0)
+                                 : (p.RBx == 16) ? smem_desc(0, 128, x_unit, 0)
                                                  : smem_desc(0, x_unit, 8 * p.RBx, layout_code(p.RBx));
             const uint64_t b_tpl = (p.RBe == 16) ? smem_desc(0, 128, e_unit, 0)
                                                  : smem_desc(0, e_unit, 8 * p.RBe, layout_code(p.RBe));
-            const uint32_t a_step = (32 * p.RBx) >> 4, b_step = (32 * p.RBe) >> 4;   // 32 pixel rows per MMA
+            const uint32_t a_step = p.halo ? (uint32_t)(4 * p.PW) : (uint32_t)((32 * p.RBx) >> 4);   // 32 pixel rows per MMA
+            const uint32_t b_step = (32 * p.RBe) >> 4;
+            const uint32_t a_tile_step = p.halo ? (uint32_t)p.PW : (uint32_t)(16384 >> 4);
             uint32_t accum = 0;
             int st = 0; uint32_t ph = 0;
             for (int kb = kb0; kb < kb1; ++kb) {
@@ -377,7 +385,7 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                             mma_i8(d_tmem, a_tpl | (a_lo & 0x3FFFu), b_tpl | (b_lo & 0x3FFFu), idesc, accum | (uint32_t)kk);
                             a_lo += a_step; b_lo += b_step;
                         }
-                        a_tile += 16384 >> 4; d_tmem += p.BNc;
+                        a_tile += a_tile_step; d_tmem += p.BNc;
                     }
                     mma_commit(smem_u32(&ctl->empty[st]));
                     if (kb == kb1 - 1) mma_commit(smem_u32(&ctl->tmem_full[0]));
@@ -393,10 +401,15 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         if (mbar_wait(smem_u32(&ctl->tmem_full[0]), 0, &ctl->abort_flag, p.dev_status)) {
             tc_fence_after();
             for (int t = 0; t < p.mtiles; ++t) {
-                const int i = t * G + row / p.RBx;                 // input box within this CTA
-                const int mu = mu0 + i;
-                const bool valid = (i < nX) && (mu < p.total_units);
-                const int tap = mu / cpt, ci = (mu % cpt) * p.RBx + row % p.RBx;
+                int tap, ci; bool valid;
+                if (p.halo) {                                       // lane = (s, ci) of filter row t
+                    tap = t * p.S + (row >> 4); ci = row & 15; valid = (row >> 4) < p.S;
+                } else {
+                    const int i = t * G + row / p.RBx;             // input box within this CTA
+                    const int mu = mu0 + i;
+                    valid = (i < nX) && (mu < p.total_units);
+                    tap = mu / cpt; ci = (mu % cpt) * p.RBx + row % p.RBx;
+                }
                 const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + t * p.BNc;
                 for (int c = 0; c < p.BNc; c += 16) {
                     uint32_t v[16];
@@ -593,11 +606,13 @@ lpdt_status tc_wgrad(const lpdt_conv_desc &d, const int8_t *E, const int8_t *A, 
     p.R = d.R; p.S = d.S; p.pad = d.pad; p.taps = d.R * d.S; p.stride = d.stride;
     p.RBx = row_bytes_for(d.Cin); p.RBe = row_bytes_for(d.Cout);
     p.merged = (d.Cin == 16 && d.stride == 1) ? 1 : 0;
-    pick_tile(Ho, Wo, p.merged ? 16 : 128, &p.TB, &p.TH, &p.TW);
+    p.BNc = largest_div(d.Cout, 256, p.RBe);
+    p.halo = (p.merged && d.S <= 8 && d.R * p.BNc <= 512 && d.R <= 16) ? 1 : 0;
+    if (p.halo) { p.TW = 8; p.TH = 16; p.TB = 1; p.PW = 8 + d.S - 1; p.PH = 16 + d.R - 1; p.halo_bytes = (int)align_up((size_t)p.PW * p.PH * 16 + 256, 1024); }
+    else pick_tile(Ho, Wo, p.merged ? 16 : 128, &p.TB, &p.TH, &p.TW);
     if (p.TW * d.stride > 256 || p.TH * d.stride > 256) return LPDT_ERR_UNSUPPORTED;
     p.tilesB = (int)ceil_div(d.B, p.TB); p.tilesH = (int)ceil_div(Ho, p.TH); p.tilesW = (int)ceil_div(Wo, p.TW);
     p.kblocks = p.tilesB * p.tilesH * p.tilesW;
-    p.BNc = largest_div(d.Cout, 256, p.RBe);
     p.ngroups = d.Cout / p.BNc;
     const int G = 128 / p.RBx;
     p.total_units = p.taps * (d.Cin / p.RBx);
@@ -609,11 +624,12 @@ lpdt_status tc_wgrad(const lpdt_conv_desc &d, const int8_t *E, const int8_t *A, 
     if (mt < 1) return LPDT_ERR_UNSUPPORTED;
     p.mtiles = mt;
     p.mgroups = (int)ceil_div(all_tiles, mt);
-    const int stage_bytes = mt * 16384 + 128 * p.BNc;
+    if (p.halo) { p.mtiles = d.R; p.mgroups = 1; }
+    const int stage_bytes = (p.halo ? p.halo_bytes : mt * 16384) + 128 * p.BNc;
     p.stages = (kSmemBudget - 1024) / stage_bytes;
     if (p.stages > 8) p.stages = 8;
     if (p.stages < 2) return LPDT_ERR_UNSUPPORTED;
-    p.tmem_cols = pow2_at_least(mt * p.BNc);
+    p.tmem_cols = pow2_at_least(p.mtiles * p.BNc);
     if (p.tmem_cols > 512) return LPDT_ERR_UNSUPPORTED;
     long long ctas_fixed = (long long)d.nodes * p.mgroups * p.ngroups;
     int splits = ctas_fixed >= kNumSMs ? 1 : (int)ceil_div(2 * kNumSMs, ctas_fixed);
@@ -623,7 +639,12 @@ lpdt_status tc_wgrad(const lpdt_conv_desc &d, const int8_t *E, const int8_t *A, 
     p.splits = (int)ceil_div(p.kblocks, p.kb_per_split);
     p.acc_out = acc_out; p.dev_status = dev_status;
     CUtensorMap mX, mE;
-    if (p.merged) { if (!act_map_merged(&mX, A, d.nodes, d.B, d.H, d.W, p.TB, p.TH, p.TW)) return LPDT_ERR_CUDA; }
+    if (p.halo) {
+        uint64_t dims[4] = {(uint64_t)d.W * 16, (uint64_t)d.H, (uint64_t)d.B, (uint64_t)d.nodes};
+        uint64_t strides[3] = {(uint64_t)d.W * 16, (uint64_t)d.H * d.W * 16, (uint64_t)d.B * d.H * d.W * 16};
+        uint32_t box[4] = {(uint32_t)p.PW * 16, (uint32_t)p.PH, 1, 1};
+        if (!make_map_u8(&mX, A, 4, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE)) return LPDT_ERR_CUDA;
+    } else if (p.merged) { if (!act_map_merged(&mX, A, d.nodes, d.B, d.H, d.W, p.TB, p.TH, p.TW)) return LPDT_ERR_CUDA; }
     else if (!act_map(&mX, A, d.nodes, d.B, d.H, d.W, d.Cin, p.RBx, p.TB, p.TH, p.TW, d.stride)) return LPDT_ERR_CUDA;
     if (!act_map(&mE, E, d.nodes, d.B, Ho, Wo, d.Cout, p.RBe, p.TB, p.TH, p.TW)) return LPDT_ERR_CUDA;
     size_t smem = 1024 + (size_t)p.stages * stage_bytes;
