@@ -81,3 +81,80 @@ def test_graph_replay_matches_eager():
     torch.cuda.synchronize()
     assert torch.equal(a.x_out, b.x_out) and torch.equal(a.x_hat, b.x_hat) and torch.equal(a.grads, b.grads)
     assert b.graph_launches > 100
+
+
+def test_resnet20_full_size_step():
+    # the benchmark workload at its full size (16 nodes x batch 32): every node's codes, outputs,
+    # gradients and the gossip result against the oracle's whole step
+    _compare(wlmod.make_workload("resnet20"))
+
+
+def _subset(wl, sel):
+    """The same workload restricted to the nodes in sel (nodes are independent until the gossip step)."""
+    sub = dict(wl)
+    sub["nodes"] = len(sel)
+    for key in ("x", "labels", "dy", "params", "x_hat"):
+        if key in wl:
+            sub[key] = np.ascontiguousarray(wl[key][sel])
+    return sub
+
+
+def _compare_sampled_nodes(wl, sel):
+    """Full-size GPU step; the oracle recomputes the sampled nodes' gradients and half-steps, and the mix
+    is checked through what holds at any size (top-k count, x_hat update, average preservation)."""
+    st = TrainStep.from_workload(wl)
+    st.run()
+    torch.cuda.synchronize()
+    assert int(st.dev_status.item()) == 0
+    sub = _subset(wl, sel)
+    keep = {}
+    grads, loss, _ = ostep.forward_backward(sub["ops"], sub["params"], sub["x"], sub.get("labels"), None,
+                                            sub["ren_eps"], keep=keep)
+    for li, (op, b) in enumerate(zip(wl["ops"], st.buf)):
+        if op["op"] in ("conv", "linear"):
+            got = b["E"][sel].cpu().numpy()
+            assert np.array_equal(got.reshape(keep[f"E{li}"].shape), keep[f"E{li}"]), f"E{li}"
+    close(st.loss[sel], loss, what="loss")
+    gscale = float(np.abs(grads).max())
+    close(st.grads[sel], grads, 1e-5, 1e-6 * max(1.0, gscale), "grads")
+    import oracle
+    close(st.x_half[sel], oracle.sgd_update(sub["params"], grads, wl["lr"]), what="x_half")
+    # mix, from the GPU's own x_half (properties only)
+    xh = st.x_half.cpu().numpy(); xhat0 = wl["x_hat"]; xhat1 = st.x_hat.cpu().numpy()
+    q = xhat1 - xhat0
+    k = int(wl["seg_k"][0])
+    if k < wl["d"]:
+        delta = xh - xhat0
+        for i in range(wl["nodes"]):
+            nz = np.flatnonzero(q[i])
+            assert len(nz) <= k and len(nz) >= k - 8           # exact zeros among the kept deltas are possible
+            keptmin = np.abs(delta[i, nz]).min()
+            dropped = np.setdiff1d(np.arange(wl["d"]), nz)
+            assert keptmin >= np.abs(delta[i, dropped]).max()
+    else:
+        assert np.array_equal(xhat1, xh)
+    assert np.allclose(st.x_out.double().sum(0).cpu().numpy(), xh.astype(np.float64).sum(0),
+                       atol=1e-5 * wl["nodes"] * max(1.0, float(np.abs(xh).max())))
+
+
+def test_vgg11_full_size_sampled_nodes():
+    _compare_sampled_nodes(wlmod.make_workload("vgg11"), [0, 5])
+
+
+def test_resnet20_topk_full_size_sampled_nodes():
+    _compare_sampled_nodes(wlmod.make_workload("resnet20_topk"), [0, 17, 39])
+
+
+def test_resnet20_topk_40_nodes():
+    # 40-node ring with top-1% compression of the flattened update (batch reduced to keep the oracle short)
+    wl = wlmod.make_workload("resnet20_topk", batch=4)
+    st, ref = _compare(wl)
+    k = int(wl["seg_k"][0])
+    assert all(np.count_nonzero(ref["q"][i]) == k for i in range(wl["nodes"]))
+    # doubly-stochastic ring: the node average is preserved by the mix
+    assert np.allclose(st.x_out.double().sum(0).cpu().numpy(), st.x_half.double().sum(0).cpu().numpy(),
+                       atol=1e-4)
+
+
+def test_vgg11_8_nodes():
+    _compare(wlmod.make_workload("vgg11", batch=4))
