@@ -59,6 +59,7 @@ struct PixParams {
     int Nc, Kc;               // N channels, K channels per tap
     int RBa, RBn;             // row bytes of operand A (K side) and, backward-data, of the N side
     int merged;               // operand A fetched through the merged (channel, width) map
+    int raster;               // 1: CTAs take tiles round-robin in a blocked M x N order (long-K tiles, L2 reuse)
     int TB, TH, TW, tilesB, tilesH, tilesW, tilesN, BN;
     int U, stages, tmem_cols; // K units (one A box each) per stage
     int w_rows_per_node;      // Cout: rows of the weight map per node
@@ -95,6 +96,23 @@ __device__ __forceinline__ void next_tile(const PixParams &p, TileCoord &c) {
     ++c.node;
 }
 
+// Blocked order for long-K tiles: groups of kRasterM M tiles sweep all N tiles, so the tiles in flight
+// at any moment (consecutive indices, one per CTA) share a few operand panels that stay in L2.
+constexpr int kRasterM = 16;
+__device__ __forceinline__ TileCoord decode_raster(const PixParams &p, int tile) {
+    const int mtiles = p.nodes * p.tilesB * p.tilesH * p.tilesW;
+    const int per_group = kRasterM * p.tilesN;
+    const int mg = tile / per_group, rem = tile - mg * per_group;
+    int gsize = mtiles - mg * kRasterM; if (gsize > kRasterM) gsize = kRasterM;
+    TileCoord c; c.cls = 0;
+    c.nt = rem / gsize;
+    int m = mg * kRasterM + (rem - c.nt * gsize);
+    c.tw = m % p.tilesW; m /= p.tilesW;
+    c.th = m % p.tilesH; m /= p.tilesH;
+    c.tb = m % p.tilesB; c.node = m / p.tilesB;
+    return c;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapW,
                 const PixParams p) {
@@ -109,8 +127,9 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     // warp-uniform and keeps the single-issuer role loops on the uniform datapath
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
     const long long total_tiles = (long long)p.nodes * p.tilesN * p.tilesB * p.tilesH * p.tilesW * p.ncls;
-    const int tile_lo = (int)(total_tiles * blockIdx.x / gridDim.x);
-    const int tile_hi = (int)(total_tiles * (blockIdx.x + 1) / gridDim.x);
+    const int tile_lo = p.raster ? (int)blockIdx.x : (int)(total_tiles * blockIdx.x / gridDim.x);
+    const int tile_hi = p.raster ? (int)total_tiles : (int)(total_tiles * (blockIdx.x + 1) / gridDim.x);
+    const int tile_step = p.raster ? (int)gridDim.x : 1;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.stages; ++i) { mbar_init(smem_u32(&ctl->full[i]), 1); mbar_init(smem_u32(&ctl->empty[i]), 1); }
@@ -130,9 +149,10 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             if (elect_one()) { tma_prefetch_desc(&mapA); tma_prefetch_desc(&mapW); }
             uint32_t g = 0;     // running stage counter
             int st = 0; uint32_t ph = 0;
-            TileCoord c = decode_tile(p, tile_lo);
+            TileCoord c = decode_tile(p, p.raster ? 0 : tile_lo);
             const int nj = p.BN / p.RBn, bj_stride = p.U * p.RBa * p.RBn, bu_stride = p.RBa * p.RBn;
-            for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; ++tile, next_tile(p, c)) {
+            for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; tile += tile_step) {
+                if (p.raster) c = decode_raster(p, tile); else if (tile != tile_lo) next_tile(p, c);
                 const int n0 = c.nt * p.BN, w0 = c.tw * p.TW * p.cmul, h0 = c.th * p.TH * p.cmul, b0 = c.tb * p.TB;
                 const int wrow = c.node * p.w_rows_per_node;
                 const TapTable &tt = p.tt[c.cls];
@@ -188,7 +208,7 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             uint32_t g = 0, tcount = 0;
             int st = 0; uint32_t ph = 0;
             int cls = tile_lo % p.ncls;
-            for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; ++tile, ++tcount) {
+            for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; tile += tile_step, ++tcount) {
                 const int acc = tcount & 1;
                 const uint32_t aph = (tcount >> 1) & 1;
                 if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), aph ^ 1, &ctl->abort_flag, p.dev_status)) break;
@@ -228,9 +248,10 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         const int row = q * 32 + lane;                // tile row = pixel within the tile
         const int pw = row % p.TW, phh = (row / p.TW) % p.TH, pb = row / (p.TW * p.TH);
         uint32_t tcount = 0;
-        TileCoord c = decode_tile(p, tile_lo);
+        TileCoord c = decode_tile(p, p.raster ? 0 : tile_lo);
         int sc_node = -1; float sc = 0.f;
-        for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; ++tile, ++tcount, next_tile(p, c)) {
+        for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; tile += tile_step, ++tcount) {
+            if (p.raster) c = decode_raster(p, tile); else if (tile != tile_lo) next_tile(p, c);
             const int n0 = c.nt * p.BN;
             const int w = (c.tw * p.TW + pw) * p.out_mul + p.cls_pw[c.cls];
             const int h = (c.th * p.TH + phh) * p.out_mul + p.cls_ph[c.cls];
@@ -567,6 +588,8 @@ lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const flo
         p.cls_iters[c] = (int)ceil_div((long)p.tt[c].ntaps * cpt, U);
         if (p.cls_iters[c] < 1) p.cls_iters[c] = 1;      // a class without taps still writes zeros
     }
+    // long K loops (GEMM-like): blocked round-robin tile order; short ones: contiguous ranges
+    p.raster = (p.ncls == 1 && p.cls_iters[0] >= 8) ? 1 : 0;
     const int stage_bytes = U * unit_bytes;
     p.stages = (kSmemBudget - 1024) / stage_bytes;
     if (p.stages > 8) p.stages = 8;
