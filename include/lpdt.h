@@ -104,6 +104,19 @@ lpdt_status lpdt_quantize_with_range(const float *x, int32_t nodes, int64_t n_pe
                                      const float *amax, lpdt_round rounding, uint64_t seed,
                                      uint32_t ctr_offset, int8_t *q, float *scale, void *stream);
 
+/* lpdt_quantize_batch - symmetric nearest-even quantization (as lpdt_quantize, LPDT_SYM_S8) of
+ * n_tensors tensors that sit inside one flat per-node parameter vector, e.g. all layer
+ * weights of a network, in two launches.  Tensor t of node n is read from
+ * params + n*row_stride + src_offsets[t] (sizes[t] elements) and written as int8 to
+ * q + dst_offsets[t] + n*sizes[t]  (each tensor contiguous [nodes][sizes[t]], as the
+ * contractions expect); scales[t*nodes + n] receives its scale.  src_offsets, sizes and
+ * dst_offsets are HOST arrays; n_tensors <= 64 (LPDT_ERR_UNSUPPORTED beyond).
+ * ws : lpdt_quantize_batch_workspace_size(nodes, n_tensors) bytes. */
+size_t lpdt_quantize_batch_workspace_size(int32_t nodes, int32_t n_tensors);
+lpdt_status lpdt_quantize_batch(const float *params, int32_t nodes, int64_t row_stride, int32_t n_tensors,
+                                const int64_t *src_offsets, const int64_t *sizes, const int64_t *dst_offsets,
+                                int8_t *q, float *scales, void *ws, size_t ws_bytes, void *stream);
+
 /* y = scale[n] * (q - zp[n]); zero_point == NULL means symmetric signed codes.
  * q is contiguous [nodes][n_per_node]; node n of y starts at y + n*y_node_stride. */
 lpdt_status lpdt_dequantize(const int8_t *q, int32_t nodes, int64_t n_per_node,

@@ -26,6 +26,8 @@ SIGNATURES = {
     "lpdt_quantize": (_i32, [_vp, _i32, _i64, _i64, _i32, _i32, _u64, _u32, _vp, _vp, _vp, _vp, _sz, _vp]),
     "lpdt_quantize_static": (_i32, [_vp, _i32, _i64, _i64, _i32, _i32, _u64, _u32, _vp, _vp, _vp, _vp]),
     "lpdt_quantize_with_range": (_i32, [_vp, _i32, _i64, _i64, _vp, _i32, _u64, _u32, _vp, _vp, _vp]),
+    "lpdt_quantize_batch_workspace_size": (_sz, [_i32, _i32]),
+    "lpdt_quantize_batch": (_i32, [_vp, _i32, _i64, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp]),
     "lpdt_dequantize": (_i32, [_vp, _i32, _i64, _vp, _vp, _vp, _i64, _vp]),
     "lpdt_qconv_workspace_size": (_sz, [C.POINTER(ConvDesc), _i32]),
     "lpdt_qconv_fwd": (_i32, [C.POINTER(ConvDesc), _vp, _vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _sz, _vp, _vp]),

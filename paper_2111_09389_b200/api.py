@@ -13,7 +13,7 @@ from ._lib import ConvDesc, lib
 
 # Kernels each entry point enqueues (memsets not counted); KERNEL_LAUNCHES accumulates them.
 KERNELS_PER_CALL = {
-    "lpdt_quantize": 2, "lpdt_quantize_with_range": 1, "lpdt_quantize_static": 2, "lpdt_dequantize": 1, "lpdt_qconv_fwd": 1, "lpdt_qconv_bwd_data": 2,
+    "lpdt_quantize": 2, "lpdt_quantize_with_range": 1, "lpdt_quantize_static": 2, "lpdt_quantize_batch": 2, "lpdt_dequantize": 1, "lpdt_qconv_fwd": 1, "lpdt_qconv_bwd_data": 2,
     "lpdt_qconv_bwd_weight": 2, "lpdt_range_evonorm_fwd": 1, "lpdt_range_evonorm_bwd": 2,
     "lpdt_gossip_mix": 2, "lpdt_sgd_update": 1, "lpdt_residual_add": 1, "lpdt_residual_add_bwd": 1,
     "lpdt_avgpool": 1, "lpdt_avgpool_bwd": 1, "lpdt_maxpool2x2": 1, "lpdt_maxpool2x2_bwd": 1,
@@ -105,6 +105,22 @@ def lpdt_quantize_with_range(x, nodes, n_per_node, x_node_stride, amax, q, scale
 
 def lpdt_fill_zero(t):
     _check("lpdt_fill_zero", lib().lpdt_fill_zero(_ptr(t), t.numel() * t.element_size(), _stream()))
+
+
+def lpdt_quantize_batch_workspace_size(nodes, n_tensors):
+    return lib().lpdt_quantize_batch_workspace_size(nodes, n_tensors)
+
+
+def lpdt_quantize_batch(params, nodes, row_stride, src_offsets, sizes, dst_offsets, q, scales, ws):
+    """src_offsets / sizes / dst_offsets: host sequences of Python ints (one entry per tensor)."""
+    n = len(sizes)
+    so = (C.c_int64 * n)(*[int(v) for v in src_offsets])
+    sz = (C.c_int64 * n)(*[int(v) for v in sizes])
+    do = (C.c_int64 * n)(*[int(v) for v in dst_offsets])
+    p, nb = _ws(ws)
+    _check("lpdt_quantize_batch", lib().lpdt_quantize_batch(_ptr(params), nodes, row_stride, n, C.addressof(so),
+                                                            C.addressof(sz), C.addressof(do), _ptr(q), _ptr(scales),
+                                                            p, nb, _stream()))
 
 
 def lpdt_quantize_static(x, nodes, n_per_node, x_node_stride, q, scale, mode=0, rounding=0, seed=0,

@@ -318,3 +318,83 @@ extern "C" lpdt_status lpdt_quantize_static(const float *x, int32_t nodes, int64
     return lpdt_quantize(x, nodes, n_per_node, x_node_stride, mode, rounding, seed, ctr_offset, q, scale,
                          zero_point, words, sizeof(uint32_t) * 2 * kStaticMaxNodes, stream);
 }
+
+// ---------------------------------------------------------------------------
+// Batched symmetric quantization of many small tensors that live inside one flat
+// per-node parameter vector (all layer weights of a network): two launches in
+// total instead of two per tensor.
+namespace lpdt {
+
+constexpr int kMaxBatchTensors = 64;
+struct QuantBatch {
+    int count;
+    long long src_off[kMaxBatchTensors];    // element offset inside a node's parameter row
+    long long size[kMaxBatchTensors];       // elements per node
+    long long dst_off[kMaxBatchTensors];    // byte offset of the tensor's [nodes][size] block in q
+};
+
+// grid = (blocks, nodes, tensors); blocks beyond a tensor's length fall through
+__global__ void batch_range_kernel(const float *__restrict__ params, long long row_stride, QuantBatch qb,
+                                   uint32_t *__restrict__ ws) {
+    const int t = blockIdx.z, node = blockIdx.y;
+    const long long n = qb.size[t];
+    const float *x = params + (long long)node * row_stride + qb.src_off[t];
+    float m = 0.f;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+        m = fmaxf(m, fabsf(x[i]));
+    if ((long long)blockIdx.x * blockDim.x >= n) return;
+    block_amax_to(m, reinterpret_cast<float *>(ws + (size_t)t * gridDim.y + node));
+}
+
+__global__ void batch_quantize_kernel(const float *__restrict__ params, long long row_stride, QuantBatch qb,
+                                      const uint32_t *__restrict__ ws, int8_t *__restrict__ q,
+                                      float *__restrict__ scales) {
+    const int t = blockIdx.z, node = blockIdx.y, nodes = gridDim.y;
+    const long long n = qb.size[t];
+    const float *x = params + (long long)node * row_stride + qb.src_off[t];
+    int8_t *dst = q + qb.dst_off[t] + (long long)node * n;
+    const float amax = __uint_as_float(ws[(size_t)t * nodes + node]);
+    float s = 1.f, inv = 0.f;
+    if (amax != 0.f) { s = __fdiv_rn(amax, 127.f); inv = __fdiv_rn(127.f, amax); }
+    if (blockIdx.x == 0 && threadIdx.x == 0) scales[(size_t)t * nodes + node] = s;
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (long long)gridDim.x * blockDim.x)
+        dst[i] = (int8_t)q_sym_rne(x[i], inv);
+}
+
+}  // namespace lpdt
+
+extern "C" size_t lpdt_quantize_batch_workspace_size(int32_t nodes, int32_t n_tensors) {
+    return align_up((size_t)(nodes > 0 ? nodes : 1) * (size_t)(n_tensors > 0 ? n_tensors : 1) * sizeof(uint32_t), 256);
+}
+
+extern "C" lpdt_status lpdt_quantize_batch(const float *params, int32_t nodes, int64_t row_stride, int32_t n_tensors,
+                                           const int64_t *src_offsets, const int64_t *sizes,
+                                           const int64_t *dst_offsets, int8_t *q, float *scales, void *ws,
+                                           size_t ws_bytes, void *stream) {
+    LPDT_CHECK_ARG(nodes >= 0 && n_tensors >= 0);
+    if (nodes == 0 || n_tensors == 0) return LPDT_OK;
+    LPDT_CHECK_ARG(params && src_offsets && sizes && dst_offsets && q && scales);
+    if (n_tensors > kMaxBatchTensors || nodes > 65535) return LPDT_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < lpdt_quantize_batch_workspace_size(nodes, n_tensors)) return LPDT_ERR_WORKSPACE;
+    QuantBatch qb;
+    qb.count = n_tensors;
+    long long longest = 0;
+    for (int t = 0; t < n_tensors; ++t) {
+        LPDT_CHECK_ARG(src_offsets[t] >= 0 && sizes[t] >= 0 && dst_offsets[t] >= 0 && src_offsets[t] + sizes[t] <= row_stride);
+        qb.src_off[t] = src_offsets[t]; qb.size[t] = sizes[t]; qb.dst_off[t] = dst_offsets[t];
+        if (sizes[t] > longest) longest = sizes[t];
+    }
+    if (longest == 0) return LPDT_OK;
+    cudaStream_t st = as_stream(stream);
+    uint32_t *w = (uint32_t *)ws;
+    LPDT_CUDA(cudaMemsetAsync(w, 0, (size_t)nodes * n_tensors * sizeof(uint32_t), st));
+    int bx = (int)ceil_div(longest, 256 * 8);
+    if (bx > 64) bx = 64;
+    if (bx < 1) bx = 1;
+    dim3 grid(bx, nodes, n_tensors);
+    batch_range_kernel<<<grid, 256, 0, st>>>(params, row_stride, qb, w);
+    LPDT_LAUNCH_CHECK();
+    batch_quantize_kernel<<<grid, 256, 0, st>>>(params, row_stride, qb, w, q, scales);
+    LPDT_LAUNCH_CHECK();
+    return LPDT_OK;
+}

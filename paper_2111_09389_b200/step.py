@@ -45,6 +45,18 @@ class TrainStep:
                        api.lpdt_gossip_mix_workspace_size(N, d, len(self.seg_k)))
         self.buf = []
         shape = tuple(in_shape)
+        # all layer weights are quantized by one batched call into one int8 buffer (256-byte aligned blocks)
+        wlist = [op for op in ops if op["op"] in ("conv", "linear")]
+        self.w_src, self.w_size, self.w_dst = [], [], []
+        qbytes = 0
+        for op in wlist:
+            wn = op["cout"] * op["cin"] * (op["R"] * op["S"] if op["op"] == "conv" else 1)
+            self.w_src.append(op["w_off"]); self.w_size.append(wn); self.w_dst.append(qbytes)
+            qbytes += (N * wn + 255) // 256 * 256
+        self.qW_all = torch.empty(max(qbytes, 256), **i8)
+        self.sW_all = torch.empty(max(len(wlist), 1), N, **f32)
+        ws_bytes = max(ws_bytes, api.lpdt_quantize_batch_workspace_size(N, min(len(wlist), 64)))
+        wi = 0
         for op in ops:
             k = op["op"]
             b = {}
@@ -58,7 +70,8 @@ class TrainStep:
                 Wo = (W + 2 * pad - S) // stride + 1
                 b.update(desc=desc, in_shape=(H, W, op["cin"]),
                          qA=torch.empty(N, B, H, W, op["cin"], **i8), sA=torch.empty(N, **f32),
-                         qW=torch.empty(N, op["cout"], R, S, op["cin"], **i8), sW=torch.empty(N, **f32),
+                         qW=self.qW_all[self.w_dst[wi]:self.w_dst[wi] + N * self.w_size[wi]].view(N, op["cout"], R, S, op["cin"]),
+                         sW=self.sW_all[wi],
                          out=torch.empty(N, B, Ho, Wo, op["cout"], **f32),
                          E=torch.empty(N, B, Ho, Wo, op["cout"], **i8), sE=torch.empty(N, **f32),
                          dx=torch.empty(N, B, H, W, op["cin"], **f32),
@@ -66,6 +79,7 @@ class TrainStep:
                 if quantize_wgrad:
                     b.update(gq=torch.empty(N, b["wn"], **i8), gs=torch.empty(N, **f32),
                              gw=torch.empty(N, b["wn"], **f32))
+                wi += 1
                 for which in (0, 1, 2):
                     ws_bytes = max(ws_bytes, api.lpdt_qconv_workspace_size(desc, which))
                 shape = (Ho, Wo, op["cout"])
@@ -132,6 +146,10 @@ class TrainStep:
         cur_range = None          # per-node max|cur| when the producer of cur emitted it
         saved = []
         api.lpdt_fill_zero(self.ranges)
+        for lo in range(0, len(self.w_size), 64):        # every layer's weights, 64 tensors per call
+            hi = min(lo + 64, len(self.w_size))
+            api.lpdt_quantize_batch(self.params, N, d, self.w_src[lo:hi], self.w_size[lo:hi], self.w_dst[lo:hi],
+                                    self.qW_all, self.sW_all[lo:hi], self.ws)
         for li, (op, b) in enumerate(zip(self.ops, self.buf)):
             k = op["op"]
             if k in ("conv", "linear"):
@@ -140,7 +158,6 @@ class TrainStep:
                     api.lpdt_quantize_with_range(cur, N, n_in, n_in, cur_range, b["qA"], b["sA"])
                 else:
                     api.lpdt_quantize(cur, N, n_in, n_in, b["qA"], b["sA"], self.ws)
-                api.lpdt_quantize(self._p(op["w_off"]), N, b["wn"], d, b["qW"], b["sW"], self.ws)
                 bias = self._p(op["b_off"]) if k == "linear" else None
                 api.lpdt_qconv_fwd(b["desc"], b["qA"], b["sA"], b["qW"], b["sW"], Y=b["out"], bias=bias,
                                    bias_node_stride=d, ws=self.ws, dev_status=self.dev_status)

@@ -82,6 +82,27 @@ def test_quantize_affine(nodes, n):
     assert np.array_equal(y.cpu().numpy(), oracle.dequantize(q_ref, s_ref, z_ref))
 
 
+def test_quantize_batch_matches_per_tensor_calls():
+    rng = np.random.default_rng(11)
+    nodes, d = 5, 20011
+    params = (rng.standard_normal((nodes, d)) * rng.uniform(0.01, 3, (nodes, 1))).astype(np.float32)
+    src = [0, 432, 433, 5000, 15003]; size = [432, 1, 2304, 9216, 5008]
+    params[2, 432] = 0.0                                   # an all-zero single-element tensor on one node
+    dst, off = [], 0
+    for n in size:
+        dst.append(off); off += (nodes * n + 255) // 256 * 256
+    q = torch.full((off,), 99, dtype=torch.int8, device="cuda")
+    sc = torch.zeros(len(size), nodes, device="cuda")
+    ws = ws_bytes(api.lpdt_quantize_batch_workspace_size(nodes, len(size)))
+    api.lpdt_quantize_batch(dev(params), nodes, d, src, size, dst, q, sc, ws)
+    qh, sh = q.cpu().numpy(), sc.cpu().numpy()
+    for t, (o, n, do) in enumerate(zip(src, size, dst)):
+        q_ref, s_ref = oracle.quantize_sym_s8(params[:, o:o + n])
+        assert np.array_equal(sh[t], s_ref)
+        assert np.array_equal(qh[do:do + nodes * n].reshape(nodes, n), q_ref)
+    assert sh[1, 2] == 1.0
+
+
 def test_quantize_argument_errors():
     x = torch.zeros(8, device="cuda")
     q = torch.zeros(8, dtype=torch.int8, device="cuda")
