@@ -203,6 +203,8 @@ lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8_t *E, cons
  * x, y, dy, dx : fp32 NHWC;  v, gamma, beta : fp32, node n at p + n*param_node_stride
  * gmin, gmax : fp32 [nodes][B][groups];  argmin, argmax : int32, same shape
  * dv, dgamma, dbeta : fp32, node n at p + n*grad_node_stride, C entries
+ * res (forward, nullable) : fp32, shape of y; when given the identity shortcut of a residual
+ *            block is fused: y = RangeEvoNorm(x) + res (the sum is one more fp32 addition)
  * amax_out (nullable) : fp32 [nodes], caller-zeroed; receives max|y| (forward) or max|dx|
  *            (backward) per node by atomic maximum, for lpdt_quantize_with_range
  * Requires C % groups == 0 and cpg >= 2 (Cst is infinite for cpg = 1).
@@ -213,7 +215,7 @@ lpdt_status lpdt_range_evonorm_fwd(int32_t nodes, int32_t B, int32_t H, int32_t 
                                    const float *v, const float *gamma, const float *beta,
                                    int64_t param_node_stride, float *y,
                                    float *gmin, float *gmax, int32_t *argmin, int32_t *argmax,
-                                   float *amax_out, void *stream);
+                                   float *amax_out, const float *res, void *stream);
 size_t lpdt_range_evonorm_bwd_workspace_size(int32_t nodes, int32_t B, int32_t C);
 lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C,
                                    int32_t groups, float eps, const float *dy, const float *x,

@@ -33,7 +33,7 @@ SIGNATURES = {
     "lpdt_qconv_fwd": (_i32, [C.POINTER(ConvDesc), _vp, _vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _sz, _vp, _vp]),
     "lpdt_qconv_bwd_data": (_i32, [C.POINTER(ConvDesc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
     "lpdt_qconv_bwd_weight": (_i32, [C.POINTER(ConvDesc), _vp, _vp, _vp, _vp, _vp, _i64, _vp, _vp, _sz, _vp, _vp]),
-    "lpdt_range_evonorm_fwd": (_i32, [_i32] * 6 + [_f32] + [_vp] * 4 + [_i64] + [_vp] * 6 + [_vp]),
+    "lpdt_range_evonorm_fwd": (_i32, [_i32] * 6 + [_f32] + [_vp] * 4 + [_i64] + [_vp] * 7 + [_vp]),
     "lpdt_range_evonorm_bwd_workspace_size": (_sz, [_i32, _i32, _i32]),
     "lpdt_range_evonorm_bwd": (_i32, [_i32] * 6 + [_f32] + [_vp] * 4 + [_i64] + [_vp] * 8 + [_i64, _vp, _vp, _sz, _vp]),
     "lpdt_gossip_mix_workspace_size": (_sz, [_i32, _i64, _i32]),

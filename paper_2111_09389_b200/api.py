@@ -167,10 +167,10 @@ def lpdt_qconv_bwd_weight(desc, E, sE, A, sA, dW=None, dw_node_stride=0, dWacc=N
 
 
 def lpdt_range_evonorm_fwd(nodes, B, H, W, Cc, groups, eps, x, v, gamma, beta, param_node_stride, y,
-                           gmin, gmax, argmin, argmax, amax_out=None):
+                           gmin, gmax, argmin, argmax, amax_out=None, res=None):
     _check("lpdt_range_evonorm_fwd", lib().lpdt_range_evonorm_fwd(
         nodes, B, H, W, Cc, groups, eps, _ptr(x), _ptr(v), _ptr(gamma), _ptr(beta), param_node_stride,
-        _ptr(y), _ptr(gmin), _ptr(gmax), _ptr(argmin), _ptr(argmax), _ptr(amax_out), _stream()))
+        _ptr(y), _ptr(gmin), _ptr(gmax), _ptr(argmin), _ptr(argmax), _ptr(amax_out), _ptr(res), _stream()))
 
 
 def lpdt_range_evonorm_bwd_workspace_size(nodes, B, Cc):

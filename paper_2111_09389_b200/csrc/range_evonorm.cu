@@ -85,7 +85,8 @@ ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
                const float *__restrict__ x, const float *__restrict__ v,
                const float *__restrict__ gamma, const float *__restrict__ beta, int64_t pstride,
                int B, float *__restrict__ y, float *__restrict__ gmin, float *__restrict__ gmax,
-               int32_t *__restrict__ argmin, int32_t *__restrict__ argmax, float *__restrict__ amax_out) {
+               int32_t *__restrict__ argmin, int32_t *__restrict__ argmax, float *__restrict__ amax_out,
+               const float *__restrict__ res) {
     extern __shared__ unsigned char smem_raw[];
     const int T = blockDim.x, t = threadIdx.x;
     Ext *s_mn = reinterpret_cast<Ext *>(smem_raw);
@@ -130,11 +131,14 @@ ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
     for (int p = row0; p < HW; p += rstep) {
         float xv[V], yv[V];
         VecLoad<V>::ld(xs + (int64_t)p * C + c0, xv);
+        float rv[V];
+        if (res) VecLoad<V>::ld(res + sample * (int64_t)HW * C + (int64_t)p * C + c0, rv);
 #pragma unroll
         for (int k = 0; k < V; ++k) {
             float u = __fmul_rn(vc[k], xv[k]);
             float m = __fmul_rn(xv[k], hsig(u));
             yv[k] = __fadd_rn(__fmul_rn(__fmul_rn(gc[k], m), invD), bc[k]);
+            if (res) yv[k] = __fadd_rn(yv[k], rv[k]);           // fused identity shortcut: y = REN(x) + res
             ymax = fmaxf(ymax, fabsf(yv[k]));
         }
         VecLoad<V>::st(ys + (int64_t)p * C + c0, yv);
@@ -315,7 +319,7 @@ extern "C" lpdt_status lpdt_range_evonorm_fwd(int32_t nodes, int32_t B, int32_t 
                                               int32_t groups, float eps, const float *x, const float *v,
                                               const float *gamma, const float *beta, int64_t pstride,
                                               float *y, float *gmin, float *gmax, int32_t *argmin,
-                                              int32_t *argmax, float *amax_out, void *stream) {
+                                              int32_t *argmax, float *amax_out, const float *res, void *stream) {
     LPDT_CHECK_ARG(nodes >= 0 && B >= 0 && H > 0 && W > 0 && C > 0 && groups > 0);
     LPDT_CHECK_ARG(C % groups == 0 && C / groups >= 2);
     if (nodes == 0 || B == 0) return LPDT_OK;
@@ -323,15 +327,15 @@ extern "C" lpdt_status lpdt_range_evonorm_fwd(int32_t nodes, int32_t B, int32_t 
     LPDT_CHECK_ARG(pstride >= C || nodes == 1);
     if ((int64_t)H * W * C > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
     RenPlan pl;
-    if (!plan(C, groups, aligned(x, 16) && aligned(y, 16), &pl)) return LPDT_ERR_UNSUPPORTED;
+    if (!plan(C, groups, aligned(x, 16) && aligned(y, 16) && (!res || aligned(res, 16)), &pl)) return LPDT_ERR_UNSUPPORTED;
     size_t smem = (size_t)(2 * pl.threads + 2 * groups) * sizeof(Ext);
     if (smem > 48 * 1024) return LPDT_ERR_UNSUPPORTED;
     const float Cst = ren_const(C / groups);
     dim3 grid((unsigned)((int64_t)nodes * B));
     if (pl.V == 4)
-        ren_fwd_kernel<4><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out);
+        ren_fwd_kernel<4><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
     else
-        ren_fwd_kernel<1><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out);
+        ren_fwd_kernel<1><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

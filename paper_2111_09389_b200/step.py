@@ -165,15 +165,22 @@ class TrainStep:
             elif k == "ren":
                 Cc = op["C"]
                 b["x"] = cur
+                # an identity shortcut right after this layer is added inside the kernel
+                nxt = self.ops[li + 1] if li + 1 < len(self.ops) else None
+                fuse = nxt is not None and nxt["op"] == "add" and nxt["stride"] == 1 and nxt["Ca"] == nxt["C"]
+                res = saved[-1] if fuse else None
                 api.lpdt_range_evonorm_fwd(N, B, op["H"], op["W"], Cc, op["groups"], self.eps, cur,
                                            self._p(op["p_off"]), self._p(op["p_off"] + Cc),
                                            self._p(op["p_off"] + 2 * Cc), d, b["out"], b["gmin"], b["gmax"],
-                                           b["amin"], b["amax"], amax_out=self.ranges[li])
+                                           b["amin"], b["amax"], amax_out=self.ranges[li], res=res)
                 cur, cur_range = b["out"], self.ranges[li]
+                b["fused_add"] = fuse
             elif k == "save":
                 saved.append(cur)
             elif k == "add":
                 a = saved.pop()
+                if self.buf[li - 1].get("fused_add"):
+                    continue                        # already added by the Range-EvoNorm kernel before it
                 api.lpdt_residual_add(N, B, op["H"], op["W"], op["Ca"], op["C"], op["stride"], op["ch_off"],
                                       cur, a, b["out"], amax_out=self.ranges[li])
                 cur, cur_range = b["out"], self.ranges[li]
