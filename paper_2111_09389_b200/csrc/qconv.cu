@@ -66,7 +66,10 @@ static bool use_halo(const lpdt_conv_desc &d, int mode) {
 static lpdt_status run_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const float *s1, const int8_t *Wq,
                            const float *s2, const float *bias, int64_t bias_stride, float *Y, int32_t *Yacc,
                            int32_t *dev_status, cudaStream_t st) {
-    if (use_halo(d, mode)) return tc::tc_pix_halo(d, mode, A, s1, Wq, s2, bias, bias_stride, Y, Yacc, dev_status, st);
+    if (use_halo(d, mode)) {
+        lpdt_status r = tc::tc_pix_halo(d, mode, A, s1, Wq, s2, bias, bias_stride, Y, Yacc, dev_status, st);
+        if (r != LPDT_ERR_UNSUPPORTED) return r;
+    }
     return tc::tc_pix(d, mode, A, s1, Wq, s2, bias, bias_stride, Y, Yacc, dev_status, st);
 }
 

@@ -1,8 +1,8 @@
-// Halo-tile variant of the pixel-M convolution kernel for 16-channel operands
-// (K = taps x 16 bytes, stride 1): forward with Cin = 16 and backward-data with
-// Cout = 16.
+// Halo-tile variant of the pixel-M convolution kernel for narrow operands at
+// stride 1 (K channels = 16, 32, 64, 96 or 128): forward by Cin, backward-data by
+// Cout.
 //
-// With 16 channels a pixel is exactly one 16-byte row of the no-swizzle
+// A 16-channel chunk of a pixel is exactly one 16-byte row of the no-swizzle
 // core-matrix layout, and a filter tap is a shift by whole rows.  So instead of
 // one TMA box per tap, one box per tile fetches the 8 x 16 pixel tile together
 // with its halo ((8+S-1) x (16+R-1) pixels, out-of-image pixels zero-filled),
@@ -10,8 +10,11 @@
 // the tap's offset inside the halo, stride between 8-row groups = the halo row
 // pitch, and the leading-dimension offset = the distance to the second tap of the
 // pair that shares a K = 32 MMA (an odd last tap is paired with a block of zeros).
+// With more than 16 channels the box carries the 16-byte chunks as its outermost
+// dimension (one halo image per chunk) and an MMA pairs two chunks of the same tap.
 // The node's weights are loaded into shared memory once per node, not per tile.
-// Per tile this is 1 TMA request and ceil(taps/2) MMAs.
+// Per tile this is 1 TMA request and ceil(taps*chunks/2) MMAs.
+#include <stdlib.h>
 #include "qconv_internal.cuh"
 #include "tc_common.cuh"
 
@@ -20,6 +23,7 @@ namespace tc {
 
 constexpr int kHaloThreads = 192;
 constexpr int kHaloMaxTaps = 64;
+constexpr int kHaloMaxMma = 72;
 constexpr int kTileW = 8, kTileH = 16;
 constexpr int kZeroBytes = 4096;          // >= 15 halo rows of at most 256 bytes + one 8-row group
 
@@ -27,9 +31,11 @@ struct HaloParams {
     int mode;                  // 0 forward, 1 backward-data
     int nodes, B, Hm, Wm;      // output image of this pass
     int N;                     // output channels of this pass
-    int ntaps;
-    unsigned short off16[kHaloMaxTaps];   // tap offset inside the halo, in 16-byte rows, ascending
-    signed char wtap[kHaloMaxTaps];       // matching tap index in the weight tensor
+    int ntaps, cpt, nslices;   // taps, 16-channel chunks per tap, K slices = taps * chunks (order: tap, chunk)
+    signed char wtap[kHaloMaxTaps];       // tap index in the weight tensor of the i-th tap in halo order
+    int n_mma;                            // one MMA per pair of K slices
+    unsigned short a_off16[kHaloMaxMma];  // first slice of the pair: offset inside the stage, in 16-byte rows
+    unsigned short a_lbo16[kHaloMaxMma];  // distance to the second slice (0xFFFF: pair with the zero block)
     int org_h, org_w;          // halo origin relative to the tile origin (smallest tap offsets)
     int PH, PW;                // halo rows / pixels per row
     int tilesH, tilesW;
@@ -92,7 +98,7 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = __shfl_sync(0xffffffffu, ctl->tmem_base, 0);
-    const int slot_bytes = p.mode == 0 ? p.N * 16 : 256;      // one tap of weights (backward: per 16-column chunk)
+    const int slot_bytes = p.mode == 0 ? p.N * 16 : 256;      // one K slice of weights (backward: per 16-column chunk)
     const int nchunk = p.N / 16;
 
     if (warp == 0) {
@@ -114,25 +120,31 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
                     const uint32_t wfull = smem_u32(&ctl->wfull);
                     const int wrow = c.node * p.w_rows_per_node;
                     if (elect_one()) {
-                        mbar_expect_tx(wfull, p.ntaps * p.N * 16);
-                        for (int i = 0; i < p.ntaps; ++i) {
-                            if (p.mode == 0) {
-                                tma_load_3d(smem_u32(wres) + i * slot_bytes, &mapW, wfull, 0, p.wtap[i], wrow);
-                            } else {
-                                for (int j = 0; j < nchunk; ++j)
-                                    tma_load_3d(smem_u32(wres) + (j * (p.ntaps + 1) + i) * 256, &mapW, wfull, j * 16,
-                                                p.wtap[i], wrow);
+                        mbar_expect_tx(wfull, p.nslices * p.N * 16);
+                        int kap = 0;
+                        for (int i = 0; i < p.ntaps; ++i)
+                            for (int c2 = 0; c2 < p.cpt; ++c2, ++kap) {
+                                if (p.mode == 0) {      // N rows of 16 K bytes
+                                    tma_load_3d(smem_u32(wres) + kap * slot_bytes, &mapW, wfull, c2 * 16, p.wtap[i], wrow);
+                                } else {                // 16 K rows (output channels of the layer) of 16 N bytes
+                                    for (int j = 0; j < nchunk; ++j)
+                                        tma_load_3d(smem_u32(wres) + (j * (p.nslices + 1) + kap) * 256, &mapW, wfull,
+                                                    j * 16, p.wtap[i], wrow + c2 * 16);
+                                }
                             }
-                        }
                     }
                     __syncwarp();
                 }
                 if (!mbar_wait(smem_u32(&ctl->empty[st]), ph ^ 1, &ctl->abort_flag, p.dev_status)) break;
                 const uint32_t full = smem_u32(&ctl->full[st]);
                 if (elect_one()) {
-                    mbar_expect_tx(full, p.PH * p.PW * 16);
-                    tma_load_4d(smem_u32(stage0 + (size_t)st * p.halo_bytes), &mapA, full,
-                                (c.tw * kTileW + p.org_w) * 16, c.th * kTileH + p.org_h, c.b, c.node);
+                    mbar_expect_tx(full, p.PH * p.PW * 16 * p.cpt);
+                    if (p.cpt == 1)
+                        tma_load_4d(smem_u32(stage0 + (size_t)st * p.halo_bytes), &mapA, full,
+                                    (c.tw * kTileW + p.org_w) * 16, c.th * kTileH + p.org_h, c.b, c.node);
+                    else
+                        tma_load_5d(smem_u32(stage0 + (size_t)st * p.halo_bytes), &mapA, full, 0,
+                                    c.tw * kTileW + p.org_w, c.th * kTileH + p.org_h, c.node * p.B + c.b, 0);
                 }
                 __syncwarp();
                 if (++st == p.stages) { st = 0; ph ^= 1; }
@@ -144,11 +156,10 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
             const uint32_t sbo_a = p.PW * 16;                       // next 8-pixel row group = next halo row
             const uint64_t a_fixed = ((uint64_t)((sbo_a >> 4) & 0x3FFFu) << 32) | ((uint64_t)1 << 46);
             const uint64_t b_tpl = (p.mode == 0) ? smem_desc(0, p.N * 16, 128, 0)
-                                                 : smem_desc(0, 128, (p.ntaps + 1) * 256, 0);
+                                                 : smem_desc(0, 128, (p.nslices + 1) * 256, 0);
             const uint32_t w_lo0 = smem_u32(wres) >> 4;
             const uint32_t b_pair_step = (2 * slot_bytes) >> 4;
             const uint32_t zero_lo = smem_u32(zeros) >> 4;
-            const int npairs = (p.ntaps + 1) / 2;
             int st = 0; uint32_t ph = 0, tcount = 0, wph = 0;
             int cur_node = -1;
             HaloTile c = halo_decode(p, tile_lo);
@@ -166,10 +177,9 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
                 const uint32_t halo_lo = smem_u32(stage0 + (size_t)st * p.halo_bytes) >> 4;
                 if (elect_one()) {
                     uint32_t b_lo = w_lo0;
-                    for (int i = 0; i < npairs; ++i) {
-                        const uint32_t s0 = halo_lo + p.off16[2 * i];
-                        const uint32_t lbo = (2 * i + 1 < p.ntaps) ? (uint32_t)(p.off16[2 * i + 1] - p.off16[2 * i])
-                                                                   : (zero_lo - s0);
+                    for (int i = 0; i < p.n_mma; ++i) {
+                        const uint32_t s0 = halo_lo + p.a_off16[i];
+                        const uint32_t lbo = p.a_lbo16[i] != 0xFFFFu ? (uint32_t)p.a_lbo16[i] : (zero_lo - s0);
                         const uint64_t ad = a_fixed | (uint64_t)(s0 & 0x3FFFu) | ((uint64_t)(lbo & 0x3FFFu) << 16);
                         mma_i8(d_tmem, ad, b_tpl | (b_lo & 0x3FFFu), idesc, (uint32_t)i);
                         b_lo += b_pair_step;
@@ -233,14 +243,28 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
     if (warp == 1) { tc_fence_after(); tmem_dealloc(tmem_base, p.tmem_cols); }
 }
 
+// LPDT_FORCE_HALO=1 takes the halo kernel wherever it is valid (used by the parity tests).
+static bool halo_forced() {
+    static int forced = -1;
+    if (forced < 0) { const char *e = getenv("LPDT_FORCE_HALO"); forced = (e && e[0] == '1') ? 1 : 0; }
+    return forced == 1;
+}
+
 static int halo_pow2(int v) { int p = 32; while (p < v) p <<= 1; return p; }
 
 bool halo_supported(const lpdt_conv_desc &d, int mode) {
     if (d.stride != 1) return false;
     const int Kc = mode == 0 ? d.Cin : d.Cout, N = mode == 0 ? d.Cout : d.Cin;
-    if (Kc != 16 || N % 16 || N > 256) return false;
+    if (Kc % 16 || Kc > 128 || (Kc > 16 && Kc % 32) || N % 16 || N > 256) return false;
     if (d.S > 9 || d.R > 64 || d.R * d.S > kHaloMaxTaps) return false;
-    if ((d.R * d.S + 1) * N * 16 > 64 * 1024) return false;
+    // measured: with several chunks the 16-byte TMA rows only pay off for up to 64 channels on maps at
+    // least one tile (16 rows) high; elsewhere the general kernel is as fast or faster
+    const int Hm = mode == 0 ? conv_out(d.H, d.pad, d.R, 1) : d.H;
+    if (Kc > 16 && (Kc > 64 || Hm < 16) && !halo_forced()) return false;
+    const int nslices = d.R * d.S * (Kc / 16);
+    if ((nslices + 1) / 2 > kHaloMaxMma) return false;
+    if ((nslices + 1) * N * 16 > 72 * 1024) return false;
+    if ((8 + d.S - 1) * (16 + d.R - 1) >= 0x3FFF) return false;
     if (d.pad > 100) return false;
     return encode_tiled_fn() != nullptr;
 }
@@ -259,16 +283,28 @@ lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, cons
     p.org_h = mode == 0 ? -d.pad : d.pad - (d.R - 1);
     p.org_w = mode == 0 ? -d.pad : d.pad - (d.S - 1);
     p.ntaps = d.R * d.S;
+    const int Kc = mode == 0 ? d.Cin : d.Cout;
+    p.cpt = Kc / 16; p.nslices = p.ntaps * p.cpt;
+    const int chunk16 = p.PH * p.PW;                    // one chunk's halo image, in 16-byte rows
+    unsigned short off16[kHaloMaxTaps];
     for (int i = 0; i < p.ntaps; ++i) {
         // ascending halo offset: forward walks (r, s) up, backward walks them down
         const int a = i / d.S, b = i % d.S;
         const int r = mode == 0 ? a : d.R - 1 - a, s = mode == 0 ? b : d.S - 1 - b;
-        p.off16[i] = (unsigned short)(a * p.PW + b);
+        off16[i] = (unsigned short)(a * p.PW + b);
         p.wtap[i] = (signed char)(r * d.S + s);
     }
+    p.n_mma = (p.nslices + 1) / 2;
+    for (int m = 0; m < p.n_mma; ++m) {
+        const int k0 = 2 * m, k1 = 2 * m + 1;            // K slices (tap, chunk) of this MMA
+        const int o0 = (k0 % p.cpt) * chunk16 + off16[k0 / p.cpt];
+        p.a_off16[m] = (unsigned short)o0;
+        if (k1 < p.nslices) p.a_lbo16[m] = (unsigned short)((k1 % p.cpt) * chunk16 + off16[k1 / p.cpt] - o0);
+        else p.a_lbo16[m] = 0xFFFFu;
+    }
     p.tilesH = (int)ceil_div(p.Hm, kTileH); p.tilesW = (int)ceil_div(p.Wm, kTileW);
-    p.halo_bytes = (int)align_up((size_t)p.PH * p.PW * 16, 128);
-    p.wres_bytes = (int)align_up((size_t)(p.ntaps + 1) * p.N * 16, 128);
+    p.halo_bytes = (int)align_up((size_t)p.PH * p.PW * 16 * p.cpt, 128);
+    p.wres_bytes = (int)align_up((size_t)(p.nslices + 1) * p.N * 16, 128);
     if (15 * p.PW * 16 + 128 > kZeroBytes) return LPDT_ERR_UNSUPPORTED;
     int stages = (196 * 1024 - p.wres_bytes - kZeroBytes) / p.halo_bytes;
     if (stages > 8) stages = 8;
@@ -279,7 +315,12 @@ lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, cons
     p.Y = Y; p.Yacc = Yacc; p.s1 = s1; p.s2 = s2; p.bias = bias; p.bias_stride = bias_stride;
     p.dev_status = dev_status;
     CUtensorMap mA, mW;
-    {   // operand A with (channel, width) merged into one contiguous row of 16*Wa bytes
+    if (p.cpt > 1) {   // 16-byte chunk rows; the chunk index is the outermost box dimension
+        uint64_t dims[5] = {16, (uint64_t)Wa, (uint64_t)Ha, (uint64_t)d.nodes * d.B, (uint64_t)p.cpt};
+        uint64_t strides[4] = {(uint64_t)Kc, (uint64_t)Wa * Kc, (uint64_t)Ha * Wa * Kc, 16};
+        uint32_t box[5] = {16, (uint32_t)p.PW, (uint32_t)p.PH, 1, (uint32_t)p.cpt};
+        if (!make_map_u8(&mA, A, 5, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE)) return LPDT_ERR_UNSUPPORTED;
+    } else {   // operand A with (channel, width) merged into one contiguous row of 16*Wa bytes
         uint64_t dims[4] = {(uint64_t)Wa * 16, (uint64_t)Ha, (uint64_t)d.B, (uint64_t)d.nodes};
         uint64_t strides[3] = {(uint64_t)Wa * 16, (uint64_t)Ha * Wa * 16, (uint64_t)d.B * Ha * Wa * 16};
         uint32_t box[4] = {(uint32_t)p.PW * 16, (uint32_t)p.PH, 1, 1};

@@ -145,6 +145,10 @@ CONV_CASES = [
     (1, 2, 17, 9, 16, 16, 5, 4, 1, 2),       # halo path: 5x4 filter (even tap count), asymmetric padding effect
     (1, 2, 12, 12, 16, 32, 1, 1, 1, 0),      # halo path with a single tap
     (2, 2, 10, 10, 16, 16, 3, 3, 1, 0),      # halo path without padding
+    (2, 3, 16, 16, 32, 32, 3, 3, 1, 1),      # halo path with two 16-channel chunks
+    (2, 5, 8, 8, 64, 64, 3, 3, 1, 1),        # halo path: 8x8 maps (half of each tile is outside the image)
+    (1, 2, 13, 11, 96, 32, 3, 3, 1, 1),      # halo path: 6 chunks forward, 2 chunks backward
+    (1, 2, 9, 20, 128, 128, 3, 3, 1, 1),     # halo path at its channel limit
 ]
 
 
@@ -435,3 +439,19 @@ def test_glue_ops():
     cs = torch.zeros(3, 14, device="cuda")
     api.lpdt_colsum(3, 32, 10, dev(z), cs[:, 4:], 14)
     close(cs[:, 4:], oracle.colsum(z), 1e-6, 1e-7)
+
+
+@pytest.mark.parametrize("env", [{"LPDT_FORCE_HALO": "1"}, {"LPDT_DISABLE_HALO": "1"}, {"LPDT_DISABLE_TC": "1"}])
+def test_qconv_cases_on_every_kernel_family(env):
+    """The kernel choice is made once per process from the environment, so the contraction
+    cases are re-run in child processes with the halo kernels forced, with the halo kernels
+    off (general tensor-core kernels) and with the tensor-core engine off (CUDA-core kernels)."""
+    import os, subprocess, sys
+    if os.environ.get("LPDT_CHILD") == "1":
+        pytest.skip("already inside a child run")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    child_env = dict(os.environ, LPDT_CHILD="1", **env)
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_ops.py"), "-m", "gpu",
+                        "-q", "-x", "-k", "test_qconv_all_three or test_qconv_extreme"], env=child_env, cwd=root,
+                       capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
