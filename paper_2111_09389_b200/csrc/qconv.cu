@@ -22,21 +22,6 @@ __global__ void pad_channels_kernel(const int8_t *__restrict__ src, int8_t *__re
     }
 }
 
-// Drop the padded input channels of an accumulated weight gradient [rows][Cp] -> [rows][C],
-// writing raw accumulators and/or the dequantized fp32 gradient.
-__global__ void unpad_wgrad_kernel(const int32_t *__restrict__ acc_p, int nodes, int64_t rows_per_node, int C,
-                                   int Cp, const float *__restrict__ s1, const float *__restrict__ s2,
-                                   int32_t *__restrict__ acc_out, float *__restrict__ dW, int64_t dw_stride) {
-    const int64_t per_node = rows_per_node * C, total = per_node * nodes;
-    for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
-        const int n = (int)(o / per_node);
-        const int64_t i = o % per_node;
-        const int v = acc_p[((int64_t)n * rows_per_node + i / C) * Cp + i % C];
-        if (acc_out) acc_out[o] = v;
-        if (dW) dW[(int64_t)n * dw_stride + i] = __fmul_rn(__int2float_rn(v), __fmul_rn(s1[n], s2[n]));
-    }
-}
-
 }  // namespace lpdt
 
 static unsigned grid_for(int64_t n) {
@@ -109,7 +94,7 @@ extern "C" size_t lpdt_qconv_workspace_size(const lpdt_conv_desc *d, int32_t whi
     if (d->Cin % 16) {
         const PadPlan p = pad_plan(*d);
         if (which == 0 && p.a_bytes + p.w_bytes > need) need = p.a_bytes + p.w_bytes;
-        if (which == 2 && p.a_bytes + p.acc_bytes > need) need = p.a_bytes + p.acc_bytes;
+        if (which == 2) need += p.a_bytes;                              // + zero-padded copy of the input
     }
     return need;
 }
@@ -167,39 +152,22 @@ extern "C" lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8
     LPDT_CHECK_ARG(E && A && (dW || dWacc));
     LPDT_CHECK_ARG(!dW || (sE && sA));
     LPDT_CHECK_ARG(!dW || dw_node_stride >= (int64_t)d->Cout * d->R * d->S * d->Cin || d->nodes == 1);
-    if (!dWacc && (!ws || ws_bytes < lpdt_qconv_workspace_size(d, 2) || !aligned(ws, 4)))
-        return LPDT_ERR_WORKSPACE;
+    if (!ws || ws_bytes < lpdt_qconv_workspace_size(d, 2) || !aligned(ws, 256)) return LPDT_ERR_WORKSPACE;
     cudaStream_t st = as_stream(stream);
-    if (use_tc(*d) && d->B > 0 && aligned(E, 16) && aligned(A, 16)) {
-        const int64_t per_node = (int64_t)d->Cout * d->R * d->S * d->Cin;
-        int32_t *acc = dWacc ? dWacc : (int32_t *)ws;
-        LPDT_CUDA(cudaMemsetAsync(acc, 0, (size_t)d->nodes * per_node * sizeof(int32_t), st));
-        lpdt_status r = tc::tc_wgrad(*d, E, A, acc, dev_status, st);
-        if (r == LPDT_OK) {
-            if (dW) return dequant_acc_launch(acc, d->nodes, per_node, sE, sA, dW, dw_node_stride, st);
-            return LPDT_OK;
-        }
-        if (r != LPDT_ERR_UNSUPPORTED) return r;
-    }
+    // workspace: [int32 sums (used unless the caller gave dWacc) | zero-padded input copy]
+    const size_t acc_bytes = align_up((size_t)d->nodes * d->Cout * d->R * d->S * d->Cin * sizeof(int32_t), 256);
+    int32_t *acc_ws = (int32_t *)ws;
     lpdt_conv_desc dp;
-    if (use_tc_padded(*d, &dp) && d->B > 0 && aligned(E, 16) && ws && aligned(ws, 256) &&
-        ws_bytes >= lpdt_qconv_workspace_size(d, 2)) {
-        const PadPlan pp = pad_plan(*d);
-        int8_t *Ap = (int8_t *)ws;
-        int32_t *accp = (int32_t *)(Ap + pp.a_bytes);
+    if (use_tc(*d) && d->B > 0 && aligned(E, 16) && aligned(A, 16)) {
+        lpdt_status r = tc::tc_wgrad(*d, d->Cin, E, sE, A, sA, dWacc, acc_ws, dW, dw_node_stride, dev_status, st);
+        if (r != LPDT_ERR_UNSUPPORTED) return r;
+    } else if (use_tc_padded(*d, &dp) && d->B > 0 && aligned(E, 16)) {
+        int8_t *Ap = (int8_t *)((char *)ws + acc_bytes);
         const int64_t arows = (int64_t)d->nodes * d->B * d->H * d->W;
-        const int64_t wrows_per_node = (int64_t)d->Cout * d->R * d->S;
         pad_channels_kernel<<<grid_for(arows * dp.Cin), 256, 0, st>>>(A, Ap, arows, d->Cin, dp.Cin);
         LPDT_LAUNCH_CHECK();
-        LPDT_CUDA(cudaMemsetAsync(accp, 0, (size_t)d->nodes * wrows_per_node * dp.Cin * sizeof(int32_t), st));
-        lpdt_status r = tc::tc_wgrad(dp, E, Ap, accp, dev_status, st);
-        if (r == LPDT_OK) {
-            unpad_wgrad_kernel<<<grid_for(d->nodes * wrows_per_node * d->Cin), 256, 0, st>>>(
-                accp, d->nodes, wrows_per_node, d->Cin, dp.Cin, sE, sA, dWacc, dW, dw_node_stride);
-            LPDT_LAUNCH_CHECK();
-            return LPDT_OK;
-        }
+        lpdt_status r = tc::tc_wgrad(dp, d->Cin, E, sE, Ap, sA, dWacc, acc_ws, dW, dw_node_stride, dev_status, st);
         if (r != LPDT_ERR_UNSUPPORTED) return r;
     }
-    return generic_bwd_weight(*d, E, sE, A, sA, dW, dw_node_stride, dWacc, ws, st);
+    return generic_bwd_weight(*d, E, sE, A, sA, dW, dw_node_stride, dWacc, acc_ws, st);
 }

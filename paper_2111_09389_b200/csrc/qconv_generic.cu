@@ -196,7 +196,7 @@ lpdt_status generic_bwd_weight(const lpdt_conv_desc &d, const int8_t *E, const f
     int32_t *acc = dWacc ? dWacc : (int32_t *)ws;
     LPDT_CUDA(cudaMemsetAsync(acc, 0, (size_t)d.nodes * per_node * sizeof(int32_t), st));
     const int64_t npix = (int64_t)d.B * Ho * Wo;
-    int chunk = 64;
+    int chunk = 4;
     while (ceil_div(npix, chunk) * d.nodes > (int64_t)kNumSMs * 16) chunk *= 2;
     conv_bwd_weight_generic<<<dim3((unsigned)ceil_div(npix, chunk), d.nodes), 256, 0, st>>>(d, Ho, Wo, chunk, E, A, acc);
     LPDT_LAUNCH_CHECK();

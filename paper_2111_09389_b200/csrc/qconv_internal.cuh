@@ -31,7 +31,8 @@ bool halo_supported(const lpdt_conv_desc &d, int mode);
 lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, const float *s1, const int8_t *Wq,
                         const float *s2, const float *bias, int64_t bias_stride, float *Y, int32_t *Yacc,
                         int32_t *dev_status, cudaStream_t st);
-lpdt_status tc_wgrad(const lpdt_conv_desc &d, const int8_t *E, const int8_t *A, int32_t *acc_out,
+lpdt_status tc_wgrad(const lpdt_conv_desc &d, int cin_real, const int8_t *E, const float *sE, const int8_t *A,
+                     const float *sA, int32_t *acc_user, int32_t *acc_ws, float *dW, int64_t dw_stride,
                      int32_t *dev_status, cudaStream_t st);
 }  // namespace tc
 

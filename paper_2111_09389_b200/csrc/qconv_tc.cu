@@ -308,7 +308,11 @@ struct WgParams {
     int halo, PW, PH, halo_bytes;                 // 16-channel halo mode: one input box per pixel tile (see below)
     int mgroups, ngroups, mtiles, BNc, total_units;
     int stages, tmem_cols;
-    int32_t *acc_out; int32_t *dev_status;
+    int cin_real;                                 // channels of the caller's weight layout (< Cin when the input was zero-padded)
+    int32_t *acc_out;                             // int32 sums [nodes][Cout][taps][cin_real] (nullable if 1 split)
+    float *dW; long long dw_stride;               // fp32 result, written here only if 1 split (nullable)
+    const float *s1, *s2;                         // per-node scales of the two operands
+    int32_t *dev_status;
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -417,10 +421,15 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
             }
         }
     } else if (kb1 > kb0) {
+        // Epilogue.  One split: raw sums and/or the dequantized fp32 result go straight to their
+        // destinations.  Several splits: partial sums are added with exact int32 atomics into zeroed
+        // storage and the launcher converts them afterwards.
         const int q = warp & 3;
         const int row = q * 32 + lane;
         if (mbar_wait(smem_u32(&ctl->tmem_full[0]), 0, &ctl->abort_flag, p.dev_status)) {
             tc_fence_after();
+            const float sc = (p.dW && p.splits == 1) ? __fmul_rn(p.s1[node], p.s2[node]) : 0.f;
+            const long long cstride = (long long)p.taps * p.cin_real;
             for (int t = 0; t < p.mtiles; ++t) {
                 int tap, ci; bool valid;
                 if (p.halo) {                                       // lane = (s, ci) of filter row t
@@ -431,21 +440,28 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
                     valid = (i < nX) && (mu < p.total_units);
                     tap = mu / cpt; ci = (mu % cpt) * p.RBx + row % p.RBx;
                 }
+                valid = valid && (ci < p.cin_real);
                 const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + t * p.BNc;
                 for (int c = 0; c < p.BNc; c += 16) {
                     uint32_t v[16];
                     tmem_ld_32x16(t_row + c, v);
                     tmem_ld_wait();
-                    if (valid) {
-                        int32_t *dst = p.acc_out + (((long long)node * p.Cout + n0 + c) * p.taps + tap) * p.Cin + ci;
-                        const long long cstride = (long long)p.taps * p.Cin;
-                        if (p.splits == 1) {
+                    if (!valid) continue;
+                    const long long o = ((long long)(n0 + c) * p.taps + tap) * p.cin_real + ci;
+                    int32_t *acc = p.acc_out + (long long)node * p.Cout * cstride + o;
+                    if (p.splits > 1) {
 #pragma unroll
-                            for (int k = 0; k < 16; ++k) dst[k * cstride] = (int)v[k];
-                        } else {
+                        for (int k = 0; k < 16; ++k)
+                            if ((int)v[k] != 0) atomicAdd(acc + k * cstride, (int)v[k]);
+                    } else {
+                        if (p.acc_out) {
 #pragma unroll
-                            for (int k = 0; k < 16; ++k)
-                                if ((int)v[k] != 0) atomicAdd(dst + k * cstride, (int)v[k]);
+                            for (int k = 0; k < 16; ++k) acc[k * cstride] = (int)v[k];
+                        }
+                        if (p.dW) {
+                            float *dst = p.dW + (long long)node * p.dw_stride + o;
+#pragma unroll
+                            for (int k = 0; k < 16; ++k) dst[k * cstride] = __fmul_rn(__int2float_rn((int)v[k]), sc);
                         }
                     }
                 }
@@ -621,7 +637,11 @@ lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const flo
     return LPDT_OK;
 }
 
-lpdt_status tc_wgrad(const lpdt_conv_desc &d, const int8_t *E, const int8_t *A, int32_t *acc_out,
+// acc_user: the caller's raw-sum array or null; acc_ws: scratch of the same shape [nodes][Cout][taps][cin_real]
+// (the caller's weight layout); dW: fp32 result or null.  With one split the kernel writes both outputs
+// itself; with several it accumulates into zeroed int32 storage and a conversion launch follows.
+lpdt_status tc_wgrad(const lpdt_conv_desc &d, int cin_real, const int8_t *E, const float *sE, const int8_t *A,
+                     const float *sA, int32_t *acc_user, int32_t *acc_ws, float *dW, int64_t dw_stride,
                      int32_t *dev_status, cudaStream_t st) {
     const int Ho = conv_out(d.H, d.pad, d.R, d.stride), Wo = conv_out(d.W, d.pad, d.S, d.stride);
     WgParams p = {};
@@ -660,7 +680,9 @@ lpdt_status tc_wgrad(const lpdt_conv_desc &d, const int8_t *E, const int8_t *A, 
     if (splits < 1) splits = 1;
     p.kb_per_split = (int)ceil_div(p.kblocks, splits);
     p.splits = (int)ceil_div(p.kblocks, p.kb_per_split);
-    p.acc_out = acc_out; p.dev_status = dev_status;
+    p.cin_real = cin_real; p.dW = dW; p.dw_stride = dw_stride; p.s1 = sE; p.s2 = sA;
+    p.acc_out = p.splits == 1 ? acc_user : (acc_user ? acc_user : acc_ws);
+    p.dev_status = dev_status;
     CUtensorMap mX, mE;
     if (p.halo) {
         uint64_t dims[4] = {(uint64_t)d.W * 16, (uint64_t)d.H, (uint64_t)d.B, (uint64_t)d.nodes};
@@ -679,8 +701,14 @@ lpdt_status tc_wgrad(const lpdt_conv_desc &d, const int8_t *E, const int8_t *A, 
         attr = true;
     }
     if (d.nodes > 65535 || p.mgroups * p.ngroups > 65535) return LPDT_ERR_UNSUPPORTED;
+    const int64_t per_node = (int64_t)d.Cout * p.taps * cin_real;
+    if (p.splits > 1) {
+        if (!p.acc_out) return LPDT_ERR_WORKSPACE;
+        LPDT_CUDA(cudaMemsetAsync(p.acc_out, 0, (size_t)d.nodes * per_node * sizeof(int32_t), st));
+    }
     conv_wgrad_kernel<<<dim3(p.splits, p.mgroups * p.ngroups, d.nodes), kThreads, smem, st>>>(mX, mE, p);
     LPDT_LAUNCH_CHECK();
+    if (p.splits > 1 && dW) return dequant_acc_launch(p.acc_out, d.nodes, per_node, sE, sA, dW, dw_stride, st);
     return LPDT_OK;
 }
 

@@ -277,18 +277,23 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
     if (amax_out) block_amax_to(dmax, amax_out + node);
 }
 
-// Sum the per-sample partials of a node in sample order (deterministic) and round once.
+// Sum the per-sample partials of a node and round once.  One warp per output: lane l adds samples
+// l, l+32, ... in order and the lanes combine in a fixed shuffle tree, so the result is deterministic.
 __global__ void ren_bwd_finalize(const double *__restrict__ acc, int nodes, int B, int C,
                                  float *__restrict__ dv, float *__restrict__ dgamma,
                                  float *__restrict__ dbeta, int64_t gstride) {
-    int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (i >= nodes * 3 * C) return;
     const int node = i / (3 * C), j = i % (3 * C), which = j / C, c = j % C;
     const double *a = acc + (int64_t)node * B * 3 * C + j;
     double s = 0.0;
-    for (int b = 0; b < B; ++b) s += a[(int64_t)b * 3 * C];
-    float *dst = which == 0 ? dv : which == 1 ? dgamma : dbeta;
-    dst[(int64_t)node * gstride + c] = (float)s;
+    for (int b = lane; b < B; b += 32) s += a[(int64_t)b * 3 * C];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_down_sync(0xffffffffu, s, o);
+    if (lane == 0) {
+        float *dst = which == 0 ? dv : which == 1 ? dgamma : dbeta;
+        dst[(int64_t)node * gstride + c] = (float)s;
+    }
 }
 
 struct RenPlan { int V, threads; };
@@ -374,7 +379,7 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t 
     else
         ren_bwd_kernel<1><<<grid, pl.threads, smem, st>>>(H * W, C, groups, eps, Cst, dy, x, v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc, amax_out);
     LPDT_LAUNCH_CHECK();
-    ren_bwd_finalize<<<(nodes * 3 * C + 255) / 256, 256, 0, st>>>(acc, nodes, B, C, dv, dgamma, dbeta, gstride);
+    ren_bwd_finalize<<<(nodes * 3 * C + 7) / 8, 256, 0, st>>>(acc, nodes, B, C, dv, dgamma, dbeta, gstride);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }
