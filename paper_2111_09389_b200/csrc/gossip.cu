@@ -23,15 +23,28 @@ struct SelectOut {       // per (node, segment)
     int64_t cut;         // ties (== thr) are kept only below this index
 };
 
+template <int V> struct VecIO;
+template <> struct VecIO<4> {
+    static __device__ __forceinline__ void ld(const float *p, float (&o)[4]) {
+        float4 t = *reinterpret_cast<const float4 *>(p); o[0] = t.x; o[1] = t.y; o[2] = t.z; o[3] = t.w;
+    }
+    static __device__ __forceinline__ void st(float *p, const float (&o)[4]) {
+        *reinterpret_cast<float4 *>(p) = make_float4(o[0], o[1], o[2], o[3]);
+    }
+};
+template <> struct VecIO<1> {
+    static __device__ __forceinline__ void ld(const float *p, float (&o)[1]) { o[0] = *p; }
+    static __device__ __forceinline__ void st(float *p, const float (&o)[1]) { *p = o[0]; }
+};
+
 __device__ __forceinline__ uint32_t mag_bits(float xh, float xhat) {
     return __float_as_uint(__fsub_rn(xh, xhat)) & 0x7fffffffu;
 }
 
 // One CTA per (node, segment).  Four 8-bit radix passes, most significant
 // first, narrow the k-th largest key; a final ordered pass places the tie cut.
-__global__ void __launch_bounds__(1024)
-topk_select_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d,
-                   SegTable seg, SelectOut *__restrict__ out) {
+__device__ __forceinline__ void topk_select_body(const float *__restrict__ x_half, const float *__restrict__ x_hat,
+                                                 int64_t d, const SegTable &seg, SelectOut *__restrict__ out) {
     const int s = blockIdx.x, node = blockIdx.y;
     const int64_t lo = seg.off[s], hi = seg.off[s + 1], len = hi - lo;
     const int64_t k = seg.k[s];
@@ -110,48 +123,121 @@ topk_select_kernel(const float *__restrict__ x_half, const float *__restrict__ x
     if (threadIdx.x == 0) { o->thr = thr; o->dense = 0; o->cut = s_cut; }
 }
 
-// Fused public-copy update + mixing.  Block = TE consecutive parameters of all nodes.
-template <int TE>
-__global__ void __launch_bounds__(TE)
-gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float *__restrict__ x_hat,
-                  float *__restrict__ x_out, const float *__restrict__ Wmix, float gamma,
-                  SegTable seg, const SelectOut *__restrict__ sel) {
-    extern __shared__ float sm[];
-    float *s_w = sm;                        // [nodes][nodes]
-    float *s_hat = sm + nodes * nodes;      // [nodes][TE]
-    for (int i = threadIdx.x; i < nodes * nodes; i += TE) s_w[i] = Wmix[i];
-    const int64_t e = (int64_t)blockIdx.x * TE + threadIdx.x;
-    const bool live = e < d;
-    int s = 0;
-    if (live) {   // segment of this parameter (segments tile [0,d))
-        int a = 0, b = seg.n_seg;
-        while (b - a > 1) { int m = (a + b) >> 1; if (seg.off[m] <= e) a = m; else b = m; }
-        s = a;
-    }
-    for (int i = 0; i < nodes; ++i) {
-        float hn = 0.f;
-        if (live) {
-            const float xh = x_half[(int64_t)i * d + e], xq = x_hat[(int64_t)i * d + e];
-            const float delta = __fsub_rn(xh, xq);
-            const SelectOut so = sel[(int64_t)i * seg.n_seg + s];
-            const uint32_t key = __float_as_uint(delta) & 0x7fffffffu;
-            const bool keep = so.dense || key > so.thr || (key == so.thr && e < so.cut);
-            hn = keep ? __fadd_rn(xq, delta) : xq;
-            x_hat[(int64_t)i * d + e] = hn;
+// Row i of the mixing matrix as a compact list of its non-zero entries (j ascending), built once
+// per call by one extra CTA of the select launch.  Layout in the workspace: cnt[nodes] (int32),
+// then idx[nodes][nodes] (int32), then val[nodes][nodes] (fp32).
+__device__ void build_rows(const float *__restrict__ Wmix, int nodes, int32_t *__restrict__ tab) {
+    int32_t *cnt = tab, *idx = tab + nodes;
+    float *val = reinterpret_cast<float *>(tab + nodes + nodes * nodes);
+    for (int i = threadIdx.x; i < nodes; i += blockDim.x) {
+        int c = 0;
+        for (int j = 0; j < nodes; ++j) {
+            const float w = Wmix[i * nodes + j];
+            if (w != 0.f) { idx[i * nodes + c] = j; val[i * nodes + c] = w; ++c; }
         }
-        s_hat[i * TE + threadIdx.x] = hn;
+        cnt[i] = c;
+    }
+}
+
+__global__ void __launch_bounds__(1024)
+select_and_rows_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d,
+                       SegTable seg, SelectOut *__restrict__ out, const float *__restrict__ Wmix, int nodes,
+                       int32_t *__restrict__ tab) {
+    if ((int)blockIdx.y == nodes) { if (blockIdx.x == 0) build_rows(Wmix, nodes, tab); return; }
+    topk_select_body(x_half, x_hat, d, seg, out);
+}
+
+// Fused public-copy update + mixing.  A block owns TE*V consecutive parameters of all nodes; a thread
+// owns V consecutive ones (16-byte accesses when V = 4).  Phase 1 streams x_half and x_hat of every
+// node, writes the updated public copy and parks it in shared memory; phase 2 mixes each node with
+// its neighbours' copies from shared memory (x_half is read again: an L1/L2 hit).
+template <int V>
+__global__ void __launch_bounds__(256)
+gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float *__restrict__ x_hat,
+                  float *__restrict__ x_out, float gamma, SegTable seg, const SelectOut *__restrict__ sel,
+                  const int32_t *__restrict__ tab) {
+    extern __shared__ __align__(16) float sm[];
+    const int TE = blockDim.x;
+    int32_t *s_cnt = reinterpret_cast<int32_t *>(sm);            // [nodes]
+    int32_t *s_idx = s_cnt + nodes;                              // [nodes][nodes]
+    float *s_val = reinterpret_cast<float *>(s_idx + nodes * nodes);
+    const int tab_words = nodes + 2 * nodes * nodes;
+    float *s_hat = sm + ((tab_words + 3) & ~3);                  // [nodes][TE][V], 16-byte aligned
+    for (int i = threadIdx.x; i < tab_words; i += TE) s_cnt[i] = tab[i];
+    const int64_t e0 = ((int64_t)blockIdx.x * TE + threadIdx.x) * V;
+    const bool live = e0 < d;                                    // d % V == 0: a thread is all in or all out
+    int s0 = 0;
+    bool one_seg = true;
+    if (live) {   // segment of the first parameter (segments tile [0,d))
+        int a = 0, b = seg.n_seg;
+        while (b - a > 1) { int m = (a + b) >> 1; if (seg.off[m] <= e0) a = m; else b = m; }
+        s0 = a;
+        one_seg = seg.off[s0 + 1] >= e0 + V;
+    }
+    constexpr int kU = 4;                                        // nodes per batch of independent loads
+    for (int ib = 0; ib < nodes; ib += kU) {
+        float xh[kU][V], xq[kU][V];
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            if (live && ib + u < nodes) {
+                VecIO<V>::ld(x_half + (int64_t)(ib + u) * d + e0, xh[u]);
+                VecIO<V>::ld(x_hat + (int64_t)(ib + u) * d + e0, xq[u]);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const int i = ib + u;
+            if (i >= nodes) break;
+            float hn[V];
+#pragma unroll
+            for (int k = 0; k < V; ++k) hn[k] = 0.f;
+            if (live) {
+                SelectOut so = sel[(int64_t)i * seg.n_seg + s0];
+#pragma unroll
+                for (int k = 0; k < V; ++k) {
+                    if (!one_seg && k > 0) {
+                        int sk = s0;
+                        while (seg.off[sk + 1] <= e0 + k) ++sk;
+                        so = sel[(int64_t)i * seg.n_seg + sk];
+                    }
+                    const float delta = __fsub_rn(xh[u][k], xq[u][k]);
+                    const uint32_t key = __float_as_uint(delta) & 0x7fffffffu;
+                    const bool keep = so.dense || key > so.thr || (key == so.thr && e0 + k < so.cut);
+                    hn[k] = keep ? __fadd_rn(xq[u][k], delta) : xq[u][k];
+                }
+                VecIO<V>::st(x_hat + (int64_t)i * d + e0, hn);
+            }
+            VecIO<V>::st(s_hat + ((size_t)i * TE + threadIdx.x) * V, hn);
+        }
     }
     __syncthreads();
     if (!live) return;
-    for (int i = 0; i < nodes; ++i) {
-        const float hi_ = s_hat[i * TE + threadIdx.x];
-        float acc = 0.f;
-        for (int j = 0; j < nodes; ++j) {
-            const float w = s_w[i * nodes + j];
-            if (w != 0.f) acc = __fadd_rn(acc, __fmul_rn(w, __fsub_rn(s_hat[j * TE + threadIdx.x], hi_)));
+    for (int ib = 0; ib < nodes; ib += kU) {
+        float xh[kU][V];
+#pragma unroll
+        for (int u = 0; u < kU; ++u)
+            if (ib + u < nodes) VecIO<V>::ld(x_half + (int64_t)(ib + u) * d + e0, xh[u]);
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const int i = ib + u;
+            if (i >= nodes) break;
+            float hi_[V], acc[V], o[V];
+            VecIO<V>::ld(s_hat + ((size_t)i * TE + threadIdx.x) * V, hi_);
+#pragma unroll
+            for (int k = 0; k < V; ++k) acc[k] = 0.f;
+            const int c = s_cnt[i];
+            for (int m = 0; m < c; ++m) {                        // neighbours in ascending j
+                const int j = s_idx[i * nodes + m];
+                const float w = s_val[i * nodes + m];
+                float hj[V];
+                VecIO<V>::ld(s_hat + ((size_t)j * TE + threadIdx.x) * V, hj);
+#pragma unroll
+                for (int k = 0; k < V; ++k) acc[k] = __fadd_rn(acc[k], __fmul_rn(w, __fsub_rn(hj[k], hi_[k])));
+            }
+#pragma unroll
+            for (int k = 0; k < V; ++k) o[k] = __fadd_rn(xh[u][k], __fmul_rn(gamma, acc[k]));
+            VecIO<V>::st(x_out + (int64_t)i * d + e0, o);
         }
-        const float xh = x_half[(int64_t)i * d + e];
-        x_out[(int64_t)i * d + e] = __fadd_rn(xh, __fmul_rn(gamma, acc));
     }
 }
 
@@ -159,10 +245,14 @@ gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float 
 
 using namespace lpdt;
 
+static size_t select_bytes(int32_t nodes, int32_t n_segments) {
+    return align_up((size_t)(nodes > 0 ? nodes : 1) * (size_t)(n_segments > 0 ? n_segments : 1) * sizeof(SelectOut), 256);
+}
+
 extern "C" size_t lpdt_gossip_mix_workspace_size(int32_t nodes, int64_t d, int32_t n_segments) {
     (void)d;
-    size_t n = (size_t)(nodes > 0 ? nodes : 1) * (size_t)(n_segments > 0 ? n_segments : 1);
-    return align_up(n * sizeof(SelectOut), 256);
+    const size_t nn = (size_t)(nodes > 0 ? nodes : 1);
+    return select_bytes(nodes, n_segments) + align_up((nn + 2 * nn * nn) * sizeof(int32_t), 256);
 }
 
 extern "C" lpdt_status lpdt_gossip_mix(int32_t nodes, int64_t d, const float *x_half, float *x_hat,
@@ -188,18 +278,26 @@ extern "C" lpdt_status lpdt_gossip_mix(int32_t nodes, int64_t d, const float *x_
         return LPDT_ERR_WORKSPACE;
     cudaStream_t st = as_stream(stream);
     SelectOut *sel = (SelectOut *)ws;
-    topk_select_kernel<<<dim3(n_segments, nodes), 1024, 0, st>>>(x_half, x_hat, d, seg, sel);
+    int32_t *tab = (int32_t *)((char *)ws + select_bytes(nodes, n_segments));
+    select_and_rows_kernel<<<dim3(n_segments, nodes + 1), 1024, 0, st>>>(x_half, x_hat, d, seg, sel, Wmix, nodes, tab);
     LPDT_LAUNCH_CHECK();
-    constexpr int TE = 256;
-    size_t smem = ((size_t)nodes * nodes + (size_t)nodes * TE) * sizeof(float);
+    const bool v4 = d % 4 == 0 && aligned(x_half, 16) && aligned(x_hat, 16) && aligned(x_out, 16);
+    const int V = v4 ? 4 : 1;
+    // threads per block: as many as keep the parked public copies within 64 KB of shared memory
+    int TE = (int)((64 * 1024) / ((size_t)nodes * V * sizeof(float))) / 32 * 32;
+    if (TE > 256) TE = 256;
+    if (TE < 32) TE = 32;
+    const size_t tab_words = ((size_t)nodes + 2 * (size_t)nodes * nodes + 3) & ~(size_t)3;
+    const size_t smem = tab_words * sizeof(int32_t) + (size_t)nodes * TE * V * sizeof(float);
     static bool attr_set = false;
     if (!attr_set) {
-        LPDT_CUDA(cudaFuncSetAttribute(gossip_mix_kernel<TE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       (kMaxNodes * kMaxNodes + kMaxNodes * TE) * (int)sizeof(float)));
+        LPDT_CUDA(cudaFuncSetAttribute(gossip_mix_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
+        LPDT_CUDA(cudaFuncSetAttribute(gossip_mix_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
         attr_set = true;
     }
-    gossip_mix_kernel<TE><<<(unsigned)ceil_div(d, TE), TE, smem, st>>>(nodes, d, x_half, x_hat, x_out, Wmix,
-                                                                    gamma, seg, sel);
+    const unsigned blocks = (unsigned)ceil_div(d, (int64_t)TE * V);
+    if (v4) gossip_mix_kernel<4><<<blocks, TE, smem, st>>>(nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab);
+    else gossip_mix_kernel<1><<<blocks, TE, smem, st>>>(nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

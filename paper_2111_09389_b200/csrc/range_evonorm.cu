@@ -79,7 +79,7 @@ __device__ void reduce_groups(Ext mn, Ext mx, Ext *s_mn, Ext *s_mx, Ext *g_mn, E
     __syncthreads();
 }
 
-template <int V>
+template <int V, bool RES>
 __global__ void __launch_bounds__(512, 2)
 ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
                const float *__restrict__ x, const float *__restrict__ v,
@@ -102,7 +102,25 @@ ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
     float *ys = y + sample * (int64_t)HW * C;
 
     Ext mn, mx; mn.v = INFINITY; mn.idx = 0x7fffffff; mx.v = -INFINITY; mx.idx = 0x7fffffff;
-    for (int p = row0; p < HW; p += rstep) {
+    // kU independent 16-byte loads per thread are issued before any of them is used: the kernel
+    // is bound by the bytes in flight, not by arithmetic
+    constexpr int kU = 8;
+    int p = row0;
+    for (; p + (kU - 1) * rstep < HW; p += kU * rstep) {
+        float xv[kU][V];
+#pragma unroll
+        for (int j = 0; j < kU; ++j) VecLoad<V>::ld(xs + (int64_t)(p + j * rstep) * C + c0, xv[j]);
+#pragma unroll
+        for (int j = 0; j < kU; ++j) {
+#pragma unroll
+            for (int k = 0; k < V; ++k) {
+                int idx = (p + j * rstep) * C + c0 + k;
+                if (xv[j][k] > mx.v) { mx.v = xv[j][k]; mx.idx = idx; }
+                if (xv[j][k] < mn.v) { mn.v = xv[j][k]; mn.idx = idx; }
+            }
+        }
+    }
+    for (; p < HW; p += rstep) {
         float xv[V];
         VecLoad<V>::ld(xs + (int64_t)p * C + c0, xv);
 #pragma unroll
@@ -128,20 +146,36 @@ ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
         gc[k] = gamma[(int64_t)node * pstride + c0 + k];
         bc[k] = beta[(int64_t)node * pstride + c0 + k];
     }
-    for (int p = row0; p < HW; p += rstep) {
-        float xv[V], yv[V];
-        VecLoad<V>::ld(xs + (int64_t)p * C + c0, xv);
-        float rv[V];
-        if (res) VecLoad<V>::ld(res + sample * (int64_t)HW * C + (int64_t)p * C + c0, rv);
+    const float *rs = RES ? res + sample * (int64_t)HW * C : nullptr;
+    auto emit = [&](int pp, const float (&xv)[V], const float (&rv)[V]) {
+        float yv[V];
 #pragma unroll
         for (int k = 0; k < V; ++k) {
             float u = __fmul_rn(vc[k], xv[k]);
             float m = __fmul_rn(xv[k], hsig(u));
             yv[k] = __fadd_rn(__fmul_rn(__fmul_rn(gc[k], m), invD), bc[k]);
-            if (res) yv[k] = __fadd_rn(yv[k], rv[k]);           // fused identity shortcut: y = REN(x) + res
+            if (RES) yv[k] = __fadd_rn(yv[k], rv[k]);           // fused identity shortcut: y = REN(x) + res
             ymax = fmaxf(ymax, fabsf(yv[k]));
         }
-        VecLoad<V>::st(ys + (int64_t)p * C + c0, yv);
+        VecLoad<V>::st(ys + (int64_t)pp * C + c0, yv);
+    };
+    constexpr int kU2 = RES ? 2 : 4;
+    p = row0;
+    for (; p + (kU2 - 1) * rstep < HW; p += kU2 * rstep) {
+        float xv[kU2][V], rv[kU2][V];
+#pragma unroll
+        for (int j = 0; j < kU2; ++j) {
+            VecLoad<V>::ld(xs + (int64_t)(p + j * rstep) * C + c0, xv[j]);
+            if (RES) VecLoad<V>::ld(rs + (int64_t)(p + j * rstep) * C + c0, rv[j]);
+        }
+#pragma unroll
+        for (int j = 0; j < kU2; ++j) emit(p + j * rstep, xv[j], rv[j]);
+    }
+    for (; p < HW; p += rstep) {
+        float xv[V], rv[V];
+        VecLoad<V>::ld(xs + (int64_t)p * C + c0, xv);
+        if (RES) VecLoad<V>::ld(rs + (int64_t)p * C + c0, rv);
+        emit(p, xv, rv);
     }
     if (amax_out) block_amax_to(ymax, amax_out + node);
 }
@@ -198,30 +232,35 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
     // shuffles first, so only CV lanes per warp touch the shared fp64 accumulators.
     const bool fold = (CV <= 32) && (32 % CV == 0);
     const int iters = (HW - 1) / rstep + 1;          // same trip count for every thread (rows are predicated)
-    for (int i = 0; i < iters; ++i) {
-        const int p = row0 + i * rstep;
-        if (p < HW) {
-            float xv[V], dv_[V], o[V];
-            VecLoad<V>::ld(xs + (int64_t)p * C + c0, xv);
-            VecLoad<V>::ld(dys + (int64_t)p * C + c0, dv_);
+    auto term = [&](int p, const float (&xv)[V], const float (&dv_)[V]) {
+        float o[V];
 #pragma unroll
-            for (int k = 0; k < V; ++k) {
-                float u = __fmul_rn(vc[k], xv[k]);
-                float hs = hsig(u);
-                float hp = (u > -3.f && u < 3.f) ? sixth : 0.f;
-                float m = __fmul_rn(xv[k], hs);
-                float tt = __fmul_rn(dv_[k], gc[k]);
-                S += (double)__fmul_rn(tt, m);
-                o[k] = __fmul_rn(__fmul_rn(tt, __fadd_rn(hs, __fmul_rn(u, hp))), invD);
-                const int idx = p * C + c0 + k;
-                if (idx != g_amx && idx != g_amn) dmax = fmaxf(dmax, fabsf(o[k]));
-                fb[k] = __fadd_rn(fb[k], dv_[k]);
-                fg[k] = __fadd_rn(fg[k], __fmul_rn(dv_[k], __fmul_rn(m, invD)));
-                fv[k] = __fadd_rn(fv[k], __fmul_rn(__fmul_rn(__fmul_rn(tt, __fmul_rn(xv[k], xv[k])), hp), invD));
-            }
-            VecLoad<V>::st(dxs + (int64_t)p * C + c0, o);
+        for (int k = 0; k < V; ++k) {
+            float u = __fmul_rn(vc[k], xv[k]);
+            float hs = hsig(u);
+            float hp = (u > -3.f && u < 3.f) ? sixth : 0.f;
+            float m = __fmul_rn(xv[k], hs);
+            float tt = __fmul_rn(dv_[k], gc[k]);
+            S += (double)__fmul_rn(tt, m);
+            o[k] = __fmul_rn(__fmul_rn(tt, __fadd_rn(hs, __fmul_rn(u, hp))), invD);
+            const int idx = p * C + c0 + k;
+            if (idx != g_amx && idx != g_amn) dmax = fmaxf(dmax, fabsf(o[k]));
+            fb[k] = __fadd_rn(fb[k], dv_[k]);
+            fg[k] = __fadd_rn(fg[k], __fmul_rn(dv_[k], __fmul_rn(m, invD)));
+            fv[k] = __fadd_rn(fv[k], __fmul_rn(__fmul_rn(__fmul_rn(tt, __fmul_rn(xv[k], xv[k])), hp), invD));
         }
-        if ((i + 1) % kRunLen == 0 || i == iters - 1) {      // uniform across the block
+        VecLoad<V>::st(dxs + (int64_t)p * C + c0, o);
+    };
+    // two rows per trip: four independent 16-byte loads in flight per thread
+    for (int i = 0; i < iters; i += 2) {
+        const int p0 = row0 + i * rstep, p1 = p0 + rstep;
+        const bool ok0 = p0 < HW, ok1 = (i + 1 < iters) && (p1 < HW);
+        float xa[V], da[V], xb[V], db[V];
+        if (ok0) { VecLoad<V>::ld(xs + (int64_t)p0 * C + c0, xa); VecLoad<V>::ld(dys + (int64_t)p0 * C + c0, da); }
+        if (ok1) { VecLoad<V>::ld(xs + (int64_t)p1 * C + c0, xb); VecLoad<V>::ld(dys + (int64_t)p1 * C + c0, db); }
+        if (ok0) term(p0, xa, da);
+        if (ok1) term(p1, xb, db);
+        if ((i + 2) % kRunLen == 0 || i + 2 >= iters) {      // uniform across the block
 #pragma unroll
             for (int k = 0; k < V; ++k) {
                 double a = (double)fv[k], b = (double)fg[k], c = (double)fb[k];
@@ -337,10 +376,13 @@ extern "C" lpdt_status lpdt_range_evonorm_fwd(int32_t nodes, int32_t B, int32_t 
     if (smem > 48 * 1024) return LPDT_ERR_UNSUPPORTED;
     const float Cst = ren_const(C / groups);
     dim3 grid((unsigned)((int64_t)nodes * B));
-    if (pl.V == 4)
-        ren_fwd_kernel<4><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
-    else
-        ren_fwd_kernel<1><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
+    if (pl.V == 4) {
+        if (res) ren_fwd_kernel<4, true><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
+        else ren_fwd_kernel<4, false><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
+    } else {
+        if (res) ren_fwd_kernel<1, true><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
+        else ren_fwd_kernel<1, false><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
+    }
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

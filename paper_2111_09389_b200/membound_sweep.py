@@ -1,0 +1,122 @@
+"""Time the memory-bound kernels of the step alone, on tensors much larger than
+L2, through the C ABI, and report achieved GB/s on their algorithmic bytes.
+
+    python -m paper_2111_09389_b200.membound_sweep [--iters 20] [--peak-gbs 6549.8]
+
+Cases (activation kernels: the VGG-11-shaped workload's first layer, 8 nodes, with
+batch 128 so that each fp32 tensor is 268 MB; parameter kernels: 16 nodes with a
+32x replicated ResNet-20 parameter vector, 554 MB per array):
+
+  quantize            range pass + scale-and-round: 4 B read twice + 1 B written per element
+  quantize_stochastic the same with Philox stochastic rounding
+  quantize_with_range range supplied by the producer: 4 B read + 1 B written
+  ren_fwd             4 B read + 4 B written (the second read of a sample comes from L2)
+  ren_fwd_res         + 4 B shortcut read
+  ren_bwd             dy, x read + dx written: 12 B
+  residual_add        8 B read + 4 B written
+  sgd_update          12 B per parameter
+  gossip_dense        x_half, x_hat read; x_hat, x written: 16 B per parameter
+  gossip_top1pct      + one more pass over x_half and x_hat for the magnitude select: 24 B
+
+One JSON line per case.
+"""
+import argparse
+import json
+
+import torch
+
+from . import api, workloads
+
+
+def _time(fn, iters, warmup=3):
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(iters):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / iters
+
+
+def cases(nodes=8, B=128, H=32, W=32, Cc=64, d=32 * 270410, gossip_nodes=16):
+    """Yield (name, callable, algorithmic bytes per call)."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(7)
+    n = B * H * W * Cc
+    tot = nodes * n
+    x = torch.randn(nodes, n, generator=g, device="cuda")
+    x2 = torch.randn(nodes, n, generator=g, device="cuda")
+    y = torch.empty_like(x)
+    q = torch.empty(nodes, n, dtype=torch.int8, device="cuda")
+    scale = torch.empty(nodes, device="cuda")
+    amax = x.abs().amax(dim=1).contiguous()
+    ws = torch.empty(api.lpdt_quantize_workspace_size(nodes), dtype=torch.uint8, device="cuda")
+    yield ("quantize", lambda: api.lpdt_quantize(x, nodes, n, n, q, scale, ws), tot * 9)
+    yield ("quantize_stochastic", lambda: api.lpdt_quantize(x, nodes, n, n, q, scale, ws, rounding=1, seed=3), tot * 9)
+    yield ("quantize_with_range", lambda: api.lpdt_quantize_with_range(x, nodes, n, n, amax, q, scale), tot * 5)
+
+    groups = Cc // 8
+    v = torch.ones(nodes, Cc, device="cuda")
+    gamma = torch.ones(nodes, Cc, device="cuda")
+    beta = torch.zeros(nodes, Cc, device="cuda")
+    gmin = torch.empty(nodes, B, groups, device="cuda")
+    gmax = torch.empty_like(gmin)
+    amin_i = torch.empty(nodes, B, groups, dtype=torch.int32, device="cuda")
+    amax_i = torch.empty_like(amin_i)
+    rng = torch.zeros(nodes, device="cuda")
+
+    def ren_fwd(res=None):
+        api.lpdt_range_evonorm_fwd(nodes, B, H, W, Cc, groups, 1e-5, x, v, gamma, beta, Cc, y, gmin, gmax, amin_i,
+                                   amax_i, amax_out=rng, res=res)
+    yield ("ren_fwd", ren_fwd, tot * 8)
+    yield ("ren_fwd_res", lambda: ren_fwd(x2), tot * 12)
+
+    dx = torch.empty_like(x)
+    dv, dg, db = (torch.empty(nodes, Cc, device="cuda") for _ in range(3))
+    wsb = torch.empty(api.lpdt_range_evonorm_bwd_workspace_size(nodes, B, Cc), dtype=torch.uint8, device="cuda")
+    ren_fwd()
+    yield ("ren_bwd", lambda: api.lpdt_range_evonorm_bwd(nodes, B, H, W, Cc, groups, 1e-5, x2, x, v, gamma, Cc, gmin,
+                                                         gmax, amin_i, amax_i, dx, dv, dg, db, Cc, wsb, amax_out=rng),
+           tot * 12)
+    yield ("residual_add", lambda: api.lpdt_residual_add(nodes, B, H, W, Cc, Cc, 1, 0, x, x2, y, amax_out=rng), tot * 12)
+    del x2, dx
+
+    N = gossip_nodes
+    xh = torch.randn(N, d, generator=g, device="cuda")
+    grad = torch.randn(N, d, generator=g, device="cuda")
+    xhat = torch.zeros(N, d, device="cuda")
+    xo = torch.empty(N, d, device="cuda")
+    yield ("sgd_update", lambda: api.lpdt_sgd_update(N * d, xh, grad, 0.1, xo), N * d * 12)
+    Wm = torch.from_numpy(workloads.ring_matrix(N)).float().cuda()
+    gws = torch.empty(api.lpdt_gossip_mix_workspace_size(N, d, 1), dtype=torch.uint8, device="cuda")
+    st = torch.zeros(1, dtype=torch.int32, device="cuda")
+    yield ("gossip_dense", lambda: api.lpdt_gossip_mix(N, d, xh, xhat, xo, Wm, 1.0, [0, d], [d], gws, st), N * d * 16)
+    yield ("gossip_top1pct", lambda: api.lpdt_gossip_mix(N, d, xh, xhat, xo, Wm, 0.1, [0, d], [d // 100], gws, st),
+           N * d * 24)
+
+
+def sweep(iters=20, peak_gbs=None, out=print):
+    rows = []
+    for name, fn, nbytes in cases():
+        ms = _time(fn, iters)
+        row = {"case": name, "ms": ms, "algorithmic_bytes": nbytes, "gbs": nbytes / ms * 1e-6}
+        if peak_gbs:
+            row["frac_of_hbm_peak"] = row["gbs"] / peak_gbs
+        rows.append(row)
+        out(json.dumps(row))
+    return rows
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--iters", type=int, default=20)
+    ap.add_argument("--peak-gbs", type=float, default=None, help="HBM copy bandwidth to report fractions against")
+    a = ap.parse_args()
+    sweep(a.iters, a.peak_gbs)
+
+
+if __name__ == "__main__":
+    main()
