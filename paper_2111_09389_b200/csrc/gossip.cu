@@ -41,7 +41,47 @@ __device__ __forceinline__ uint32_t mag_bits(float xh, float xhat) {
     return __float_as_uint(__fsub_rn(xh, xhat)) & 0x7fffffffu;
 }
 
-// One CTA per (node, segment).  Four 8-bit radix passes, most significant
+// Index just past the need-th key equal to thr in [lo, hi), walking in index order (whole CTA;
+// every thread returns the same value; -1 if there are fewer than need such keys).
+__device__ long long ordered_cut(const float *__restrict__ xh, const float *__restrict__ xq, int64_t lo, int64_t hi,
+                                 uint32_t thr, long long need) {
+    __shared__ long long s_run, s_cut;
+    __shared__ int warp_cnt[32];
+    __syncthreads();
+    if (threadIdx.x == 0) { s_run = 0; s_cut = -1; }
+    __syncthreads();
+    for (int64_t base = lo; base < hi; base += blockDim.x) {
+        const int64_t e = base + threadIdx.x;
+        const int flag = (e < hi) && (mag_bits(xh[e], xq[e]) == thr);
+        const int cnt = __syncthreads_count(flag);
+        const long long run = s_run;
+        if (run + cnt >= need) {
+            // the cut lies in this stretch: rank the flags with a ballot scan
+            const unsigned bal = __ballot_sync(0xffffffffu, flag);
+            const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+            if (lane == 0) warp_cnt[warp] = __popc(bal);
+            __syncthreads();
+            int before = 0;
+            for (int w = 0; w < warp; ++w) before += warp_cnt[w];
+            const int rank = before + __popc(bal & ((1u << lane) - 1u));   // ties before me in the stretch
+            if (flag && run + rank + 1 == need) s_cut = e + 1;
+            __syncthreads();
+            break;
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) s_run = run + cnt;
+        __syncthreads();
+    }
+    __syncthreads();
+    return s_cut;
+}
+
+// A segment takes the multi-CTA path when it is long and the selection is not trivial.
+constexpr int64_t kBigMin = 32768;     // shortest segment split over several CTAs
+constexpr int kChunk = 16384;          // elements per CTA on that path
+__device__ __host__ __forceinline__ bool is_big(int64_t len, int64_t k) { return len >= kBigMin && k > 0 && k < len; }
+
+// One CTA per (node, short segment).  Four 8-bit radix passes, most significant
 // first, narrow the k-th largest key; a final ordered pass places the tie cut.
 __device__ __forceinline__ void topk_select_body(const float *__restrict__ x_half, const float *__restrict__ x_hat,
                                                  int64_t d, const SegTable &seg, SelectOut *__restrict__ out) {
@@ -49,6 +89,7 @@ __device__ __forceinline__ void topk_select_body(const float *__restrict__ x_hal
     const int64_t lo = seg.off[s], hi = seg.off[s + 1], len = hi - lo;
     const int64_t k = seg.k[s];
     SelectOut *o = out + (int64_t)node * seg.n_seg + s;
+    if (is_big(len, k)) return;          // handled by the multi-CTA kernels
     if (k >= len) {
         if (threadIdx.x == 0) { o->thr = 0; o->dense = 1; o->cut = hi; }
         return;
@@ -57,7 +98,6 @@ __device__ __forceinline__ void topk_select_body(const float *__restrict__ x_hal
     __shared__ uint32_t s_prefix, s_mask;
     __shared__ long long s_need;      // how many more keys to take inside the current prefix
     __shared__ long long s_eq;        // keys equal to the final threshold
-    __shared__ long long s_run, s_cut;
     const float *xh = x_half + (int64_t)node * d, *xq = x_hat + (int64_t)node * d;
     if (threadIdx.x == 0) { s_prefix = 0; s_mask = 0; s_need = (k > 0 ? k : 0); }
     __syncthreads();
@@ -94,33 +134,173 @@ __device__ __forceinline__ void topk_select_body(const float *__restrict__ x_hal
         if (threadIdx.x == 0) { o->thr = thr; o->dense = 0; o->cut = hi; }
         return;
     }
-    // ordered pass: find the index just past the need-th key equal to thr
-    if (threadIdx.x == 0) { s_run = 0; s_cut = -1; }
-    __syncthreads();
-    for (int64_t base = lo; base < hi; base += blockDim.x) {
-        const int64_t e = base + threadIdx.x;
-        const int flag = (e < hi) && (mag_bits(xh[e], xq[e]) == thr);
-        const int cnt = __syncthreads_count(flag);
-        const long long run = s_run;
-        if (run + cnt >= need) {
-            // the cut lies in this chunk: rank the flags with a ballot scan
-            __shared__ int warp_cnt[32];
-            const unsigned bal = __ballot_sync(0xffffffffu, flag);
-            const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-            if (lane == 0) warp_cnt[warp] = __popc(bal);
-            __syncthreads();
-            int before = 0;
-            for (int w = 0; w < warp; ++w) before += warp_cnt[w];
-            const int rank = before + __popc(bal & ((1u << lane) - 1u));   // ties before me in the chunk
-            if (flag && run + rank + 1 == need) s_cut = e + 1;
-            __syncthreads();
-            break;
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) s_run = run + cnt;
-        __syncthreads();
+    const long long cut = ordered_cut(xh, xq, lo, hi, thr, need);
+    if (threadIdx.x == 0) { o->thr = thr; o->dense = 0; o->cut = cut; }
+}
+
+// ---- long segments: the same radix select spread over many CTAs -----------------------------
+// Three histogram launches (11 + 11 + 9 key bits) accumulate per (node, segment) histograms in
+// global memory; each later launch re-derives the bucket chosen at the levels above it from those
+// histograms, so no CTA waits for another.  A fourth launch counts the keys equal to the threshold
+// per chunk (only if not all of them are taken) and a fifth places the tie cut.
+struct BigList {
+    int32_t n;
+    int32_t id[kMaxSeg];               // segment index
+    int32_t chunk_base[kMaxSeg + 1];   // prefix sums of the chunk counts
+};
+struct BigHist { uint32_t h0[2048], h1[2048], h2[512]; uint32_t tickets[4]; };   // zeroed per call
+struct BigState { uint32_t prefix, mask; long long need, eq; };   // key bits fixed so far; keys still to take; bucket population
+
+// Walk a histogram from its top bin: the bucket holding the need-th largest key, the keys still
+// needed inside it and its population.  Whole CTA (256 threads); same result in every thread.
+// The histogram was filled by other CTAs' atomics: read it from L2.
+__device__ void pick_bucket(const uint32_t *hist, int nbins, long long need, int *bucket,
+                            long long *need_out, long long *eq_out) {
+    __shared__ long long wtot[8];
+    __shared__ long long res[3];
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5, per = nbins / 256;
+    long long mine = 0;
+    for (int b = 0; b < per; ++b) mine += __ldcg(hist + t * per + b);
+    // suffix sums over the 256 slices: inside the warp by shuffles, across warps through shared memory
+    long long incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const long long v = __shfl_down_sync(0xffffffffu, incl, o);
+        if (lane + o < 32) incl += v;
     }
-    if (threadIdx.x == 0) { o->thr = thr; o->dense = 0; o->cut = s_cut; }
+    __syncthreads();
+    if (lane == 0) wtot[warp] = incl;
+    __syncthreads();
+    long long above = incl - mine;
+    for (int w = warp + 1; w < 8; ++w) above += wtot[w];
+    if (above < need && need <= above + mine) {
+        long long n = need - above;
+        int b = t * per + per - 1;
+        for (; b > t * per; --b) {
+            const long long hb = __ldcg(hist + b);
+            if (hb >= n) break;
+            n -= hb;
+        }
+        res[0] = b; res[1] = n; res[2] = __ldcg(hist + b);
+    }
+    __syncthreads();
+    *bucket = (int)res[0]; *need_out = res[1]; *eq_out = res[2];
+}
+
+// LEVEL 0..2: histogram of the next key bits (11, 11, 9) among the keys that match the prefix so
+// far; the CTA that finishes last for its (node, segment) walks the finished histogram and records
+// the new prefix.  LEVEL 3: count the keys equal to the threshold per chunk (skipped when all of
+// them are taken).
+template <int LEVEL>
+__global__ void __launch_bounds__(256)
+big_select_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d, SegTable seg,
+                  BigList big, BigHist *__restrict__ hists, BigState *__restrict__ state,
+                  uint32_t *__restrict__ tie_counts, int total_chunks, SelectOut *__restrict__ out) {
+    const int bi = blockIdx.y, node = blockIdx.z, s = big.id[bi];
+    const int64_t lo = seg.off[s], hi = seg.off[s + 1];
+    const int64_t c0 = lo + (int64_t)blockIdx.x * kChunk;
+    if (c0 >= hi) return;
+    const int64_t c1 = (c0 + kChunk < hi) ? c0 + kChunk : hi;
+    BigHist *h = hists + (int64_t)node * big.n + bi;
+    BigState *stp = state + (int64_t)node * big.n + bi;
+    BigState cur;
+    if (LEVEL == 0) { cur.prefix = 0; cur.mask = 0; cur.need = seg.k[s]; cur.eq = 0; }
+    else cur = *stp;                      // written by the previous launch
+    const float *xh = x_half + (int64_t)node * d, *xq = x_hat + (int64_t)node * d;
+    if (LEVEL == 3) {
+        if (cur.eq == cur.need) {         // every tie is taken
+            if (blockIdx.x == 0 && threadIdx.x == 0) {
+                SelectOut so; so.thr = cur.prefix; so.dense = 0; so.cut = hi;
+                out[(int64_t)node * seg.n_seg + s] = so;
+            }
+            return;
+        }
+        int cnt = 0;
+        for (int64_t e = c0 + threadIdx.x; e < c1; e += blockDim.x) cnt += mag_bits(xh[e], xq[e]) == cur.prefix;
+        __shared__ int s_cnt;
+        if (threadIdx.x == 0) s_cnt = 0;
+        __syncthreads();
+        if (cnt) atomicAdd(&s_cnt, cnt);
+        __syncthreads();
+        if (threadIdx.x == 0)
+            tie_counts[(int64_t)node * total_chunks + big.chunk_base[bi] + blockIdx.x] = (uint32_t)s_cnt;
+        return;
+    }
+    constexpr int kBins = LEVEL == 2 ? 512 : 2048;
+    constexpr int kShift = LEVEL == 0 ? 20 : LEVEL == 1 ? 9 : 0;
+    __shared__ unsigned int sh[kBins];
+    __shared__ unsigned int s_ticket;
+    for (int i = threadIdx.x; i < kBins; i += blockDim.x) sh[i] = 0;
+    __syncthreads();
+    for (int64_t e = c0 + threadIdx.x; e < c1; e += 4 * blockDim.x) {      // eight loads in flight per thread
+        float a[4], b[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int64_t eu = e + u * blockDim.x;
+            if (eu < c1) { a[u] = xh[eu]; b[u] = xq[eu]; }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            if (e + u * blockDim.x < c1) {
+                const uint32_t key = mag_bits(a[u], b[u]);
+                if ((key & cur.mask) == cur.prefix) atomicAdd(&sh[(key >> kShift) & (kBins - 1)], 1u);
+            }
+        }
+    }
+    __syncthreads();
+    uint32_t *g = LEVEL == 0 ? h->h0 : LEVEL == 1 ? h->h1 : h->h2;
+    for (int i = threadIdx.x; i < kBins; i += blockDim.x)
+        if (sh[i]) atomicAdd(&g[i], sh[i]);
+    // last CTA of this (node, segment): every chunk's counts have landed
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) s_ticket = atomicAdd(&h->tickets[LEVEL], 1u);
+    __syncthreads();
+    const unsigned nchunks = (unsigned)(big.chunk_base[bi + 1] - big.chunk_base[bi]);
+    if (s_ticket != nchunks - 1) return;
+    __threadfence();
+    int b; long long need, eq;
+    pick_bucket(g, kBins, cur.need, &b, &need, &eq);
+    if (threadIdx.x == 0) {
+        BigState nx;
+        nx.prefix = cur.prefix | ((uint32_t)b << kShift);
+        nx.mask = cur.mask | ((uint32_t)(kBins - 1) << kShift);
+        nx.need = need; nx.eq = eq;
+        *stp = nx;
+    }
+}
+
+// One CTA per (node, long segment): find the chunk that holds the need-th tie from the chunk
+// counts, then walk that chunk in index order.
+__global__ void __launch_bounds__(256)
+big_cut_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d, SegTable seg,
+               BigList big, const BigState *__restrict__ state, const uint32_t *__restrict__ tie_counts,
+               int total_chunks, SelectOut *__restrict__ out) {
+    const int bi = blockIdx.x, node = blockIdx.y, s = big.id[bi];
+    const BigState f = state[(int64_t)node * big.n + bi];
+    if (f.eq == f.need) return;
+    const int64_t lo = seg.off[s], hi = seg.off[s + 1];
+    const int nchunks = big.chunk_base[bi + 1] - big.chunk_base[bi];
+    const uint32_t *cnt = tie_counts + (int64_t)node * total_chunks + big.chunk_base[bi];
+    __shared__ int s_chunk;
+    __shared__ long long s_before;
+    if (threadIdx.x == 0) {
+        long long run = 0; int c = 0;
+        for (; c < nchunks - 1; ++c) {
+            if (run + cnt[c] >= f.need) break;
+            run += cnt[c];
+        }
+        s_chunk = c; s_before = run;
+    }
+    __syncthreads();
+    const int64_t c0 = lo + (int64_t)s_chunk * kChunk;
+    const int64_t c1 = (c0 + kChunk < hi) ? c0 + kChunk : hi;
+    const long long cut = ordered_cut(x_half + (int64_t)node * d, x_hat + (int64_t)node * d, c0, c1, f.prefix,
+                                      f.need - s_before);
+    if (threadIdx.x == 0) {
+        SelectOut so; so.thr = f.prefix; so.dense = 0; so.cut = cut;
+        out[(int64_t)node * seg.n_seg + s] = so;
+    }
 }
 
 // Row i of the mixing matrix as a compact list of its non-zero entries (j ascending), built once
@@ -248,11 +428,24 @@ using namespace lpdt;
 static size_t select_bytes(int32_t nodes, int32_t n_segments) {
     return align_up((size_t)(nodes > 0 ? nodes : 1) * (size_t)(n_segments > 0 ? n_segments : 1) * sizeof(SelectOut), 256);
 }
+static size_t rows_bytes(int32_t nodes) {
+    const size_t nn = (size_t)(nodes > 0 ? nodes : 1);
+    return align_up((nn + 2 * nn * nn) * sizeof(int32_t), 256);
+}
+// the most long segments and chunks any segmentation of d parameters into n_segments can have
+static int64_t max_big(int64_t d, int32_t n_segments) {
+    int64_t m = d / kBigMin;
+    return m < n_segments ? m : n_segments;
+}
+static int64_t max_chunks(int64_t d, int32_t n_segments) { return d / kChunk + max_big(d, n_segments); }
 
 extern "C" size_t lpdt_gossip_mix_workspace_size(int32_t nodes, int64_t d, int32_t n_segments) {
-    (void)d;
     const size_t nn = (size_t)(nodes > 0 ? nodes : 1);
-    return select_bytes(nodes, n_segments) + align_up((nn + 2 * nn * nn) * sizeof(int32_t), 256);
+    if (d < 0) d = 0;
+    if (n_segments < 1) n_segments = 1;
+    return select_bytes(nodes, n_segments) + rows_bytes(nodes) +
+           align_up(nn * (size_t)max_big(d, n_segments) * (sizeof(BigHist) + sizeof(BigState)), 256) +
+           align_up(nn * (size_t)max_chunks(d, n_segments) * sizeof(uint32_t), 256);
 }
 
 extern "C" lpdt_status lpdt_gossip_mix(int32_t nodes, int64_t d, const float *x_half, float *x_hat,
@@ -279,13 +472,43 @@ extern "C" lpdt_status lpdt_gossip_mix(int32_t nodes, int64_t d, const float *x_
     cudaStream_t st = as_stream(stream);
     SelectOut *sel = (SelectOut *)ws;
     int32_t *tab = (int32_t *)((char *)ws + select_bytes(nodes, n_segments));
+    BigList big;
+    big.n = 0; big.chunk_base[0] = 0;
+    int64_t most_chunks = 0;
+    for (int s = 0; s < n_segments; ++s) {
+        const int64_t len = seg.off[s + 1] - seg.off[s];
+        if (!is_big(len, seg.k[s])) continue;
+        const int64_t nc = ceil_div(len, (int64_t)kChunk);
+        big.id[big.n] = s;
+        big.chunk_base[big.n + 1] = big.chunk_base[big.n] + (int32_t)nc;
+        if (nc > most_chunks) most_chunks = nc;
+        ++big.n;
+    }
+    if (big.n > 0) {
+        if (most_chunks > 0x7fffffff || nodes > 65535) return LPDT_ERR_UNSUPPORTED;
+        char *p = (char *)tab + rows_bytes(nodes);
+        BigHist *hists = (BigHist *)p;
+        BigState *state = (BigState *)(hists + (size_t)nodes * big.n);
+        const size_t hist_region = align_up((size_t)nodes * (size_t)max_big(d, n_segments) * (sizeof(BigHist) + sizeof(BigState)), 256);
+        uint32_t *ties = (uint32_t *)(p + hist_region);
+        const int total_chunks = big.chunk_base[big.n];
+        LPDT_CUDA(cudaMemsetAsync(hists, 0, (size_t)nodes * big.n * sizeof(BigHist), st));
+        const dim3 g((unsigned)most_chunks, big.n, nodes);
+        big_select_kernel<0><<<g, 256, 0, st>>>(x_half, x_hat, d, seg, big, hists, state, ties, total_chunks, sel);
+        big_select_kernel<1><<<g, 256, 0, st>>>(x_half, x_hat, d, seg, big, hists, state, ties, total_chunks, sel);
+        big_select_kernel<2><<<g, 256, 0, st>>>(x_half, x_hat, d, seg, big, hists, state, ties, total_chunks, sel);
+        big_select_kernel<3><<<g, 256, 0, st>>>(x_half, x_hat, d, seg, big, hists, state, ties, total_chunks, sel);
+        LPDT_LAUNCH_CHECK();
+        big_cut_kernel<<<dim3(big.n, nodes), 256, 0, st>>>(x_half, x_hat, d, seg, big, state, ties, total_chunks, sel);
+        LPDT_LAUNCH_CHECK();
+    }
     select_and_rows_kernel<<<dim3(n_segments, nodes + 1), 1024, 0, st>>>(x_half, x_hat, d, seg, sel, Wmix, nodes, tab);
     LPDT_LAUNCH_CHECK();
     const bool v4 = d % 4 == 0 && aligned(x_half, 16) && aligned(x_hat, 16) && aligned(x_out, 16);
     const int V = v4 ? 4 : 1;
     // threads per block: as many as keep the parked public copies within 64 KB of shared memory
     int TE = (int)((64 * 1024) / ((size_t)nodes * V * sizeof(float))) / 32 * 32;
-    if (TE > 256) TE = 256;
+    if (TE > 128) TE = 128;
     if (TE < 32) TE = 32;
     const size_t tab_words = ((size_t)nodes + 2 * (size_t)nodes * nodes + 3) & ~(size_t)3;
     const size_t smem = tab_words * sizeof(int32_t) + (size_t)nodes * TE * V * sizeof(float);

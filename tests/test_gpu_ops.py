@@ -344,6 +344,9 @@ def _gossip_case(nodes, d, seed, heavy=False):
     (4, 2736, None), (16, 10007, None), (8, 50000, [(0, 50000, 500)]), (40, 27041, [(0, 27041, 270)]),
     (5, 3000, [(0, 1000, 10), (1000, 1001, 1), (1001, 3000, 1999)]), (3, 1000, [(0, 1000, 0)]),
     (1, 777, [(0, 777, 5)]), (64, 300, [(0, 300, 3)]),
+    # long segments: selection spread over several CTAs (with short and trivial ones beside them)
+    (3, 100000, [(0, 100000, 1000)]), (2, 200000, [(0, 40000, 39999), (40000, 41000, 7), (41000, 200000, 1)]),
+    (2, 70001, [(0, 33000, 0), (33000, 70001, 37001)]),
 ])
 def test_gossip_mix(nodes, d, segs):
     xh, xhat = _gossip_case(nodes, d, d, heavy=True)
@@ -380,6 +383,27 @@ def test_gossip_topk_with_massive_ties_and_alias():
     api.lpdt_gossip_mix(nodes, d, xhd, xhatd, xhd, dev(W), 0.5, [0, d], [k], ws)   # x_out aliases x_half
     assert np.array_equal(xhatd.cpu().numpy(), xhat_ref)
     close(xhd, x_ref)
+
+
+def test_gossip_topk_ties_across_chunks():
+    # a long segment whose threshold value repeats thousands of times: the tie cut falls inside
+    # one of many chunks, in the first one, or in the last one, depending on k
+    nodes, d = 3, 90001
+    rng = np.random.default_rng(11)
+    xh = rng.choice(np.array([-2, -1, 1, 2, 0.5, -0.5], np.float32), size=(nodes, d))
+    xh[0, :200] = 1.0; xh[0, 200:] = 0.25            # node 0: every tie of value 1 sits in the first chunk
+    xh[2, :-50] = 0.125; xh[2, -50:] = -3.0           # node 2: threshold ties reach into the last chunk
+    W = wlmod.ring_matrix(nodes)
+    for k in (150, 20000, 60000, 89990):
+        xhat = np.zeros((nodes, d), np.float32)
+        x_ref, xhat_ref, q_ref = oracle.gossip_mix(xh, xhat, W, 0.5, [0, d], [k])
+        assert all(np.count_nonzero(q_ref[i]) == k for i in range(nodes))
+        xhd, xhatd = dev(xh), dev(xhat)
+        xo = torch.empty_like(xhd)
+        ws = ws_bytes(api.lpdt_gossip_mix_workspace_size(nodes, d, 1))
+        api.lpdt_gossip_mix(nodes, d, xhd, xhatd, xo, dev(W), 0.5, [0, d], [k], ws)
+        assert np.array_equal(xhatd.cpu().numpy(), xhat_ref), k
+        close(xo, x_ref)
 
 
 def test_gossip_errors():
