@@ -27,7 +27,9 @@ def _rand_s8(shape, seed):
 
 
 def time_case(nodes, B, H, W, Cin, Cout, R, S, stride, pad, iters=20, warmup=3, passes=("fwd", "bwd_data", "bwd_weight"),
-              label=None):
+              label=None, graph=False):
+    """graph=True records the `iters` calls into one CUDA graph and times its replay, which
+    takes the host's launch cost out of calls that run for only a few microseconds."""
     desc = api.conv_desc(nodes, B, H, W, Cin, Cout, R, S, stride, pad)
     Ho, Wo = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - S) // stride + 1
     A = _rand_s8((nodes, B, H, W, Cin), 1)
@@ -56,9 +58,19 @@ def time_case(nodes, B, H, W, Cin, Cout, R, S, stride, pad, iters=20, warmup=3, 
             fn()
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record()
-        for _ in range(iters):
-            fn()
+        if graph:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g):
+                for _ in range(iters):
+                    fn()
+            g.replay()
+            torch.cuda.synchronize()
+            e0.record()
+            g.replay()
+        else:
+            e0.record()
+            for _ in range(iters):
+                fn()
         e1.record()
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / iters
@@ -86,12 +98,13 @@ def main(argv=None):
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--nodes", type=int, default=1)
     ap.add_argument("--passes", default="fwd,bwd_data,bwd_weight")
+    ap.add_argument("--graph", action="store_true", help="time a CUDA-graph replay of the calls")
     a = ap.parse_args(argv)
     passes = tuple(a.passes.split(","))
     if a.kind == "gemm":
-        gemm(*a.dims, iters=a.iters, warmup=a.warmup, passes=passes)
+        gemm(*a.dims, iters=a.iters, warmup=a.warmup, passes=passes, graph=a.graph)
     elif a.kind == "conv":
-        conv(*a.dims, nodes=a.nodes, iters=a.iters, warmup=a.warmup, passes=passes)
+        conv(*a.dims, nodes=a.nodes, iters=a.iters, warmup=a.warmup, passes=passes, graph=a.graph)
     else:
         sizes = (1024, 2048, 4096, 8192)
         for M in sizes:

@@ -306,11 +306,20 @@ lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, cons
     p.halo_bytes = (int)align_up((size_t)p.PH * p.PW * 16 * p.cpt, 128);
     p.wres_bytes = (int)align_up((size_t)(p.nslices + 1) * p.N * 16, 128);
     if (15 * p.PW * 16 + 128 > kZeroBytes) return LPDT_ERR_UNSUPPORTED;
-    int stages = (196 * 1024 - p.wres_bytes - kZeroBytes) / p.halo_bytes;
-    if (stages > 8) stages = 8;
+    // CTAs per SM: these tiles are short dependent chains (one TMA box, a few MMAs, a 128 x N epilogue), so
+    // several resident CTAs hide each other's latencies.  As many as leave every CTA at least four stages
+    // and fit TMEM (512 columns per SM): shared memory is sized so that no further CTA becomes resident and
+    // a TMEM allocation never has to wait.
+    p.tmem_cols = halo_pow2(2 * p.N);
+    int per_sm = 4, stages = 0;
+    for (;; --per_sm) {
+        const int budget = (224 * 1024) / per_sm - 2048;
+        stages = (budget - 1024 - p.wres_bytes - kZeroBytes) / p.halo_bytes;
+        if (stages > 8) stages = 8;
+        if (per_sm == 1 || (stages >= 4 && per_sm * p.tmem_cols <= 512)) break;
+    }
     if (stages < 2) return LPDT_ERR_UNSUPPORTED;
     p.stages = stages;
-    p.tmem_cols = halo_pow2(2 * p.N);
     p.w_rows_per_node = d.Cout;
     p.Y = Y; p.Yacc = Yacc; p.s1 = s1; p.s2 = s2; p.bias = bias; p.bias_stride = bias_stride;
     p.dev_status = dev_status;
@@ -333,7 +342,8 @@ lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, cons
         if (!make_map_u8(&mW, Wq, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE)) return LPDT_ERR_CUDA;
     }
     size_t smem = 1024 + (size_t)p.wres_bytes + (size_t)p.stages * p.halo_bytes + kZeroBytes;
-    if (smem < 120 * 1024) smem = 120 * 1024;        // one CTA per SM: TMEM allocation never waits
+    const size_t smem_floor = (size_t)(228 * 1024) / (per_sm + 1);     // keeps the (per_sm + 1)-th CTA out
+    if (smem < smem_floor) smem = smem_floor;
     static bool attr = false;
     if (!attr) {
         LPDT_CUDA(cudaFuncSetAttribute(conv_halo16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
@@ -341,7 +351,7 @@ lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, cons
     }
     const long long tiles = (long long)p.nodes * p.B * p.tilesH * p.tilesW;
     if (tiles > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
-    const int grid = (int)(tiles < kNumSMs ? tiles : kNumSMs);
+    const int grid = (int)(tiles < (long long)kNumSMs * per_sm ? tiles : (long long)kNumSMs * per_sm);
     conv_halo16_kernel<<<grid, kHaloThreads, smem, st>>>(mA, mW, p);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;

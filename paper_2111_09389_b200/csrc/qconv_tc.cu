@@ -665,17 +665,27 @@ lpdt_status tc_wgrad(const lpdt_conv_desc &d, int cin_real, const int8_t *E, con
     if (mt > mt_smem) mt = mt_smem;
     if (mt > all_tiles) mt = all_tiles;
     if (mt < 1) return LPDT_ERR_UNSUPPORTED;
+    // Few nodes with small layers: rather more CTAs with fewer M tiles each (the error tile is re-read
+    // from L2) than a deep split of the pixel loop, whose partial sums meet in atomics.
+    while (mt > 1 && (long long)d.nodes * ceil_div(all_tiles, mt) * p.ngroups < kNumSMs) --mt;
     p.mtiles = mt;
     p.mgroups = (int)ceil_div(all_tiles, mt);
     if (p.halo) { p.mtiles = d.R; p.mgroups = 1; }
-    const int stage_bytes = (p.halo ? p.halo_bytes : mt * 16384) + 128 * p.BNc;
-    p.stages = (kSmemBudget - 1024) / stage_bytes;
-    if (p.stages > 8) p.stages = 8;
-    if (p.stages < 2) return LPDT_ERR_UNSUPPORTED;
+    const int stage_bytes = (p.halo ? p.halo_bytes : p.mtiles * 16384) + 128 * p.BNc;
     p.tmem_cols = pow2_at_least(p.mtiles * p.BNc);
     if (p.tmem_cols > 512) return LPDT_ERR_UNSUPPORTED;
-    long long ctas_fixed = (long long)d.nodes * p.mgroups * p.ngroups;
-    int splits = ctas_fixed >= kNumSMs ? 1 : (int)ceil_div(2 * kNumSMs, ctas_fixed);
+    // CTAs per SM: as many (up to four) as leave each at least four stages and fit TMEM; the shared-memory
+    // request keeps any further CTA off the SM, so a TMEM allocation never waits
+    int per_sm = 4;
+    for (;; --per_sm) {
+        p.stages = ((224 * 1024) / per_sm - 2048 - 1024) / stage_bytes;
+        if (p.stages > 8) p.stages = 8;
+        if (per_sm == 1 || (p.stages >= 4 && per_sm * p.tmem_cols <= 512)) break;
+    }
+    if (p.stages < 2) return LPDT_ERR_UNSUPPORTED;
+    const long long ctas_fixed = (long long)d.nodes * p.mgroups * p.ngroups;
+    const long long slots = (long long)kNumSMs * per_sm;         // one wave of co-resident CTAs
+    int splits = ctas_fixed >= slots ? 1 : (int)(slots / ctas_fixed);
     if (splits > p.kblocks) splits = p.kblocks;
     if (splits < 1) splits = 1;
     p.kb_per_split = (int)ceil_div(p.kblocks, splits);
@@ -693,7 +703,7 @@ lpdt_status tc_wgrad(const lpdt_conv_desc &d, int cin_real, const int8_t *E, con
     else if (!act_map(&mX, A, d.nodes, d.B, d.H, d.W, d.Cin, p.RBx, p.TB, p.TH, p.TW, d.stride)) return LPDT_ERR_CUDA;
     if (!act_map(&mE, E, d.nodes, d.B, Ho, Wo, d.Cout, p.RBe, p.TB, p.TH, p.TW)) return LPDT_ERR_CUDA;
     size_t smem = 1024 + (size_t)p.stages * stage_bytes;
-    if (smem < kMinSmem) smem = kMinSmem;
+    if (smem < (size_t)(228 * 1024) / (per_sm + 1)) smem = (size_t)(228 * 1024) / (per_sm + 1);
     if (smem > 227 * 1024) return LPDT_ERR_UNSUPPORTED;
     static bool attr = false;
     if (!attr) {
