@@ -12,13 +12,19 @@ using namespace lpdt;
 
 namespace lpdt {
 
-// dst[row][0..Cp) = src[row][0..C) followed by zeros.
+// dst[row][0..Cp) = src[row][0..C) followed by zeros.  One thread per 16-byte piece of a
+// destination row (Cp is a multiple of 16), written with a single 16-byte store.
 __global__ void pad_channels_kernel(const int8_t *__restrict__ src, int8_t *__restrict__ dst, int64_t rows,
                                     int C, int Cp) {
-    const int64_t total = rows * Cp;
+    const int pieces = Cp / 16;
+    const int64_t total = rows * pieces;
     for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
-        const int c = (int)(o % Cp);
-        dst[o] = c < C ? src[(o / Cp) * C + c] : (int8_t)0;
+        const int64_t row = o / pieces;
+        const int c0 = (int)(o % pieces) * 16;
+        union { int8_t b[16]; uint4 v; } u;
+#pragma unroll
+        for (int k = 0; k < 16; ++k) u.b[k] = (c0 + k < C) ? src[row * C + c0 + k] : (int8_t)0;
+        *reinterpret_cast<uint4 *>(dst + row * Cp + c0) = u.v;
     }
 }
 
@@ -119,9 +125,9 @@ extern "C" lpdt_status lpdt_qconv_fwd(const lpdt_conv_desc *d, const int8_t *A, 
         const PadPlan pp = pad_plan(*d);
         int8_t *Ap = (int8_t *)ws, *Wp = Ap + pp.a_bytes;
         const int64_t arows = (int64_t)d->nodes * d->B * d->H * d->W, wrows = (int64_t)d->nodes * d->Cout * d->R * d->S;
-        pad_channels_kernel<<<grid_for(arows * dp.Cin), 256, 0, st>>>(A, Ap, arows, d->Cin, dp.Cin);
+        pad_channels_kernel<<<grid_for(arows * dp.Cin / 16), 256, 0, st>>>(A, Ap, arows, d->Cin, dp.Cin);
         LPDT_LAUNCH_CHECK();
-        pad_channels_kernel<<<grid_for(wrows * dp.Cin), 256, 0, st>>>(Wq, Wp, wrows, d->Cin, dp.Cin);
+        pad_channels_kernel<<<grid_for(wrows * dp.Cin / 16), 256, 0, st>>>(Wq, Wp, wrows, d->Cin, dp.Cin);
         LPDT_LAUNCH_CHECK();
         return run_pix(dp, 0, Ap, sA, Wp, sW, bias, bias_node_stride, Y, Yacc, dev_status, st);
     }
@@ -164,7 +170,7 @@ extern "C" lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8
     } else if (use_tc_padded(*d, &dp) && d->B > 0 && aligned(E, 16)) {
         int8_t *Ap = (int8_t *)((char *)ws + acc_bytes);
         const int64_t arows = (int64_t)d->nodes * d->B * d->H * d->W;
-        pad_channels_kernel<<<grid_for(arows * dp.Cin), 256, 0, st>>>(A, Ap, arows, d->Cin, dp.Cin);
+        pad_channels_kernel<<<grid_for(arows * dp.Cin / 16), 256, 0, st>>>(A, Ap, arows, d->Cin, dp.Cin);
         LPDT_LAUNCH_CHECK();
         lpdt_status r = tc::tc_wgrad(dp, d->Cin, E, sE, Ap, sA, dWacc, acc_ws, dW, dw_node_stride, dev_status, st);
         if (r != LPDT_ERR_UNSUPPORTED) return r;
