@@ -169,6 +169,48 @@ __global__ void maxpool_bwd_kernel(int64_t NB, int H, int W, int C, const float 
     }
 }
 
+// Four channels per thread (C % 4 == 0, 16-byte aligned tensors): 16-byte loads and stores, one
+// index decode per four elements.
+__global__ void maxpool_v4_kernel(int64_t NB, int H, int W, int C4, const float4 *__restrict__ x,
+                                  float4 *__restrict__ y, char4 *__restrict__ idx) {
+    const int Ho = H / 2, Wo = W / 2;
+    const int64_t total = NB * Ho * Wo * C4;
+    for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
+        const int c = (int)(o % C4);
+        int64_t pix = o / C4;
+        const int ow = (int)(pix % Wo); pix /= Wo;
+        const int oh = (int)(pix % Ho);
+        const int64_t nb = pix / Ho;
+        const int64_t base = ((nb * H + 2 * oh) * W + 2 * ow) * C4 + c;
+        const float4 v0 = x[base], v1 = x[base + C4], v2 = x[base + (int64_t)W * C4], v3 = x[base + (int64_t)W * C4 + C4];
+        float4 best = v0; char4 bi = make_char4(0, 0, 0, 0);
+#define LPDT_MP_STEP(f, v, t) if (v.f > best.f) { best.f = v.f; bi.f = t; }
+        LPDT_MP_STEP(x, v1, 1) LPDT_MP_STEP(y, v1, 1) LPDT_MP_STEP(z, v1, 1) LPDT_MP_STEP(w, v1, 1)
+        LPDT_MP_STEP(x, v2, 2) LPDT_MP_STEP(y, v2, 2) LPDT_MP_STEP(z, v2, 2) LPDT_MP_STEP(w, v2, 2)
+        LPDT_MP_STEP(x, v3, 3) LPDT_MP_STEP(y, v3, 3) LPDT_MP_STEP(z, v3, 3) LPDT_MP_STEP(w, v3, 3)
+#undef LPDT_MP_STEP
+        y[o] = best; idx[o] = bi;
+    }
+}
+
+__global__ void maxpool_bwd_v4_kernel(int64_t NB, int H, int W, int C4, const float4 *__restrict__ dy,
+                                      const char4 *__restrict__ idx, float4 *__restrict__ dx) {
+    const int Ho = H / 2, Wo = W / 2;
+    const int64_t total = NB * H * W * C4;
+    for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
+        const int c = (int)(o % C4);
+        int64_t pix = o / C4;
+        const int w = (int)(pix % W); pix /= W;
+        const int h = (int)(pix % H);
+        const int64_t nb = pix / H;
+        const int64_t po = ((nb * Ho + h / 2) * Wo + w / 2) * C4 + c;
+        const int t = (h & 1) * 2 + (w & 1);
+        const float4 g = dy[po];
+        const char4 i = idx[po];
+        dx[o] = make_float4(i.x == t ? g.x : 0.f, i.y == t ? g.y : 0.f, i.z == t ? g.z : 0.f, i.w == t ? g.w : 0.f);
+    }
+}
+
 // One block per node, one thread per sample; double arithmetic, fixed-order tree.
 __global__ void softmax_ce_kernel(int B, int K, const float *__restrict__ logits,
                                   const int32_t *__restrict__ labels, float *__restrict__ loss,
@@ -291,8 +333,13 @@ extern "C" lpdt_status lpdt_maxpool2x2(int32_t nodes, int32_t B, int32_t H, int3
     LPDT_CHECK_ARG(nodes >= 0 && B >= 0 && H > 0 && W > 0 && C > 0 && H % 2 == 0 && W % 2 == 0);
     if (nodes == 0 || B == 0) return LPDT_OK;
     LPDT_CHECK_ARG(x && y && idx);
-    maxpool_kernel<<<grid1d((int64_t)nodes * B * (H / 2) * (W / 2) * C), 256, 0, as_stream(stream)>>>(
-        (int64_t)nodes * B, H, W, C, x, y, idx);
+    if (C % 4 == 0 && aligned(x, 16) && aligned(y, 16) && aligned(idx, 4))
+        maxpool_v4_kernel<<<grid1d((int64_t)nodes * B * (H / 2) * (W / 2) * (C / 4)), 256, 0, as_stream(stream)>>>(
+            (int64_t)nodes * B, H, W, C / 4, reinterpret_cast<const float4 *>(x), reinterpret_cast<float4 *>(y),
+            reinterpret_cast<char4 *>(idx));
+    else
+        maxpool_kernel<<<grid1d((int64_t)nodes * B * (H / 2) * (W / 2) * C), 256, 0, as_stream(stream)>>>(
+            (int64_t)nodes * B, H, W, C, x, y, idx);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }
@@ -302,8 +349,13 @@ extern "C" lpdt_status lpdt_maxpool2x2_bwd(int32_t nodes, int32_t B, int32_t H, 
     LPDT_CHECK_ARG(nodes >= 0 && B >= 0 && H > 0 && W > 0 && C > 0 && H % 2 == 0 && W % 2 == 0);
     if (nodes == 0 || B == 0) return LPDT_OK;
     LPDT_CHECK_ARG(dy && idx && dx);
-    maxpool_bwd_kernel<<<grid1d((int64_t)nodes * B * H * W * C), 256, 0, as_stream(stream)>>>(
-        (int64_t)nodes * B, H, W, C, dy, idx, dx);
+    if (C % 4 == 0 && aligned(dx, 16) && aligned(dy, 16) && aligned(idx, 4))
+        maxpool_bwd_v4_kernel<<<grid1d((int64_t)nodes * B * H * W * (C / 4)), 256, 0, as_stream(stream)>>>(
+            (int64_t)nodes * B, H, W, C / 4, reinterpret_cast<const float4 *>(dy), reinterpret_cast<const char4 *>(idx),
+            reinterpret_cast<float4 *>(dx));
+    else
+        maxpool_bwd_kernel<<<grid1d((int64_t)nodes * B * H * W * C), 256, 0, as_stream(stream)>>>(
+            (int64_t)nodes * B, H, W, C, dy, idx, dx);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }
