@@ -191,8 +191,13 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
                float *__restrict__ amax_out) {
     extern __shared__ unsigned char smem_raw[];
     const int T = blockDim.x, t = threadIdx.x;
-    double *s_ch = reinterpret_cast<double *>(smem_raw);      // [3][C]
-    double *s_S = s_ch + 3 * C;                               // [T]
+    // When the column count divides the warp, lanes that share a column are folded with shuffles and
+    // every warp keeps its own partial sums (no atomics, fixed order); otherwise one shared set of
+    // fp64 accumulators takes atomic adds.
+    const bool fold = ((C / V) <= 32) && (32 % (C / V) == 0);
+    const int nsets = fold ? (T >> 5) : 1;
+    double *s_ch = reinterpret_cast<double *>(smem_raw);      // [nsets][3][C]
+    double *s_S = s_ch + nsets * 3 * C;                       // [T]
     double *g_S = s_S + T;                                    // [groups]
     const int CV = C / V, cpg = C / groups;
     const int col = t % CV, row0 = t / CV, rstep = T / CV;
@@ -202,7 +207,7 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
     const float *xs = x + sample * (int64_t)HW * C;
     const float *dys = dy + sample * (int64_t)HW * C;
     float *dxs = dx + sample * (int64_t)HW * C;
-    for (int i = t; i < 3 * C; i += T) s_ch[i] = 0.0;
+    for (int i = t; i < nsets * 3 * C; i += T) s_ch[i] = 0.0;
 
     const int64_t sg = sample * groups + grp;
     const float rng = __fsub_rn(gmax[sg], gmin[sg]);
@@ -228,9 +233,6 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
 #pragma unroll
     for (int k = 0; k < V; ++k) { fb[k] = 0.f; fg[k] = 0.f; fv[k] = 0.f; }
     __syncthreads();   // s_ch zeroed
-    // When the column count divides the warp, lanes that share a column are folded with
-    // shuffles first, so only CV lanes per warp touch the shared fp64 accumulators.
-    const bool fold = (CV <= 32) && (32 % CV == 0);
     const int iters = (HW - 1) / rstep + 1;          // same trip count for every thread (rows are predicated)
     auto term = [&](int p, const float (&xv)[V], const float (&dv_)[V]) {
         float o[V];
@@ -271,7 +273,12 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
                         c += __shfl_xor_sync(0xffffffffu, c, o);
                     }
                 }
-                if (!fold || (t & 31) < CV) {
+                if (fold) {
+                    if ((t & 31) < CV) {                 // this lane alone owns these three slots of its warp's set
+                        double *mine = s_ch + (size_t)(t >> 5) * 3 * C + c0 + k;
+                        mine[0] += a; mine[C] += b; mine[2 * C] += c;
+                    }
+                } else {
                     atomicAdd(&s_ch[0 * C + c0 + k], a);
                     atomicAdd(&s_ch[1 * C + c0 + k], b);
                     atomicAdd(&s_ch[2 * C + c0 + k], c);
@@ -292,7 +299,11 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
             if (lane == 0) g_S[g] = a;
         }
     }
-    for (int i = t; i < 3 * C; i += T) acc[sample * 3 * C + i] = s_ch[i];      // summed over the batch by the finalize kernel
+    for (int i = t; i < 3 * C; i += T) {      // warp sets in order; summed over the batch by the finalize kernel
+        double a = s_ch[i];
+        for (int w = 1; w < nsets; ++w) a += s_ch[(size_t)w * 3 * C + i];
+        acc[sample * 3 * C + i] = a;
+    }
     __syncthreads();
     // The group sum only enters dx at the two extremum positions: one thread per group
     // applies the correction to the local term already stored there (same operation order
@@ -410,7 +421,9 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t 
         return LPDT_ERR_WORKSPACE;
     RenPlan pl;
     if (!plan(C, groups, aligned(x, 16) && aligned(dy, 16) && aligned(dx, 16), &pl)) return LPDT_ERR_UNSUPPORTED;
-    size_t smem = (size_t)(3 * C + pl.threads + groups) * sizeof(double);
+    const int cv = C / pl.V;
+    const int nsets = (cv <= 32 && 32 % cv == 0) ? pl.threads / 32 : 1;      // as in the kernel
+    size_t smem = (size_t)(nsets * 3 * C + pl.threads + groups) * sizeof(double);
     if (smem > 48 * 1024) return LPDT_ERR_UNSUPPORTED;
     cudaStream_t st = as_stream(stream);
     double *acc = (double *)ws;
