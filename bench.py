@@ -52,7 +52,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(
-                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "100",
+                ["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits", "-lms", "50",
                  "-i", str(self.index)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -147,14 +147,23 @@ def run_ours(args):
     ms_total = max_over_ranks(world, e0.elapsed_time(e1))
     launches = api.KERNEL_LAUNCHES - launches0
     assert int(st.dev_status.item()) == 0
-    # the dominant entry point, bracketed by CUDA events on eager launches of the same steps
+    # the dominant entry points.  Contractions: their calls alone, on the operands the step left behind,
+    # replayed as a CUDA graph between two events (eager launches would time the host's launch gaps).
+    # Other entry points: CUDA events around each eager call of whole steps.
     names = dominant.split(",")
-    api.TIMED.update(names)
-    api.TIMINGS.clear()
-    for _ in range(args.steps):
+    kernel_ms = {}
+    passes = {"lpdt_qconv_fwd": "fwd", "lpdt_qconv_bwd_data": "bwd_data", "lpdt_qconv_bwd_weight": "bwd_weight"}
+    if all(n in passes for n in names):
         st.run()
-    torch.cuda.synchronize()
-    api.TIMED.difference_update(names)
+        for n in names:
+            kernel_ms[n] = time_contractions(st, (passes[n],), max(args.steps, 5))
+    else:
+        api.TIMED.update(names)
+        api.TIMINGS.clear()
+        for _ in range(args.steps):
+            st.run()
+        torch.cuda.synchronize()
+        api.TIMED.difference_update(names)
     clocks = sampler.stop()
     ms_step = ms_total / args.steps
     value = world * images / (ms_step * 1e-3)
@@ -181,7 +190,8 @@ def run_ours(args):
            "d2h_bytes_per_step": int(loss_host.numel() * 4)}
 
     peaks = measured_peaks()
-    roof = roofline_sum([roofline_for(n, st, wl, peaks, api) for n in names], peaks)
+    roof = roofline_sum([roofline_for(n, st, wl, peaks, api, kernel_ms.get(n)) for n in names], peaks)
+    roof = attach_traffic(roof, args.workload, dominant)
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
@@ -223,20 +233,60 @@ def roofline_sum(parts, peaks):
     tops = None
     if all(p["tops_in_kernel"] for p in parts):
         tops = sum(p["tops_in_kernel"] * p["ms_per_step_in_kernel"] for p in parts) / ms
+    launches = sum(p["launches_per_step"] for p in parts)
     return {"kernel": parts[0]["kernel"], "entry_points": [p["entry_points"][0] for p in parts], "bound": "hbm",
             "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"],
             "traffic": None, "peak_source": peaks["source"],
-            "launches_timed": sum(p["launches_timed"] for p in parts), "ms_per_step_in_kernel": ms,
-            "algorithmic_bytes_per_step": by, "tops_in_kernel": tops,
+            "launches_timed": sum(p["launches_timed"] for p in parts), "launches_per_step": launches,
+            "ms_per_step_in_kernel": ms, "algorithmic_bytes_per_step": by,
+            "algorithmic_bytes_per_launch": by / max(1, launches), "tops_in_kernel": tops,
             "timing": parts[0]["timing"]}
 
 
-def roofline_for(name, st, wl, peaks, api):
+# DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the tensor-core forward / backward-data
+# kernels over one step, from the ncu capture summarised in profiles/step_resnet20_launches.md.  Valid
+# for that workload and those entry points only, and only while those kernels are unchanged.
+MEASURED_TRAFFIC = {("resnet20", "lpdt_qconv_fwd,lpdt_qconv_bwd_data"): {"bytes_per_step": 201.0e6, "launches": 37}}
+
+
+def attach_traffic(roof, workload, entry_points):
+    m = MEASURED_TRAFFIC.get((workload, entry_points))
+    if roof is None or m is None:
+        return roof
+    roof["traffic"] = m["bytes_per_step"] / m["launches"]
+    roof["traffic_per_step"] = m["bytes_per_step"]
+    roof["traffic_note"] = ("ncu DRAM bytes per launch, mean over the step's 37 tensor-core launches; the fp32 results stay "
+                            "in L2 past the kernel's end, so this is below the algorithmic bytes")
+    return roof
+
+
+def time_contractions(st, passes, reps):
+    """Milliseconds per step spent in the contraction calls of `passes`: one CUDA graph of those
+    calls over every layer, replayed `reps` times between two events on the current stream."""
+    import torch
+    st.contractions(passes)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        st.contractions(passes)
+    for _ in range(2):
+        g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / reps
+
+
+def roofline_for(name, st, wl, peaks, api, graph_ms=None):
     """Roofline entry of the dominant kernel: algorithmic bytes (or ops) per launch,
     summed over the launches of one step, over the event-timed duration."""
     import torch
     pairs = api.TIMINGS.get(name, [])
-    if not pairs:
+    if graph_ms is None and not pairs:
         return None
     ms = sum(a.elapsed_time(b) for a, b in pairs)
     N, B = wl["nodes"], wl["batch"]
@@ -271,13 +321,19 @@ def roofline_for(name, st, wl, peaks, api):
         if name == "lpdt_quantize" and k in ("conv", "linear"):
             pass
     steps = max(1, len(pairs) // max(1, calls_per_step))
+    timing = "CUDA events around each call, eager launches of the same steps after the timed region"
+    if graph_ms is not None:
+        ms, steps = graph_ms, 1
+        timing = ("CUDA events around graph replays of these calls alone (every layer, step order, operands "
+                  "of the last step) after the timed region")
     sec = ms * 1e-3 / steps
     gbs = bytes_step / sec / 1e9
     return {"kernel": KERNEL_OF.get(name, name), "entry_points": [name],
-            "timing": "CUDA events around each call, eager launches of the same steps after the timed region",
+            "timing": timing,
             "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
             "frac": gbs / peaks["hbm_gbs"], "traffic": None, "peak_source": peaks["source"],
-            "launches_timed": len(pairs), "ms_per_step_in_kernel": ms / steps,
+            "launches_timed": len(pairs) if graph_ms is None else calls_per_step, "launches_per_step": calls_per_step,
+            "ms_per_step_in_kernel": ms / steps,
             "algorithmic_bytes_per_step": bytes_step,
             "tops_in_kernel": ops_step / sec / 1e12 if ops_step else None}
 
@@ -328,7 +384,7 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=300)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="resnet20")

@@ -268,6 +268,31 @@ class TrainStep:
         self.backward()
         self.update()
 
+    def contractions(self, passes=("fwd", "bwd_data")):
+        """Re-issue only the integer contractions of every layer, in step order, on the operands the
+        last run() left in the buffers (results are overwritten with the same values).  For timing
+        those kernels without the rest of the step; returns the number of calls made."""
+        d, n = self.d, 0
+        for li, (op, b) in enumerate(zip(self.ops, self.buf)):
+            if op["op"] in ("conv", "linear") and "fwd" in passes:
+                bias = self._p(op["b_off"]) if op["op"] == "linear" else None
+                api.lpdt_qconv_fwd(b["desc"], b["qA"], b["sA"], b["qW"], b["sW"], Y=b["out"], bias=bias,
+                                   bias_node_stride=d, ws=self.ws, dev_status=self.dev_status)
+                n += 1
+        for li in range(len(self.ops) - 1, -1, -1):
+            op, b = self.ops[li], self.buf[li]
+            if op["op"] not in ("conv", "linear"):
+                continue
+            if "bwd_weight" in passes and not self.quantize_wgrad:
+                api.lpdt_qconv_bwd_weight(b["desc"], b["E"], b["sE"], b["qA"], b["sA"], dW=self._g(op["w_off"]),
+                                          dw_node_stride=d, ws=self.ws, dev_status=self.dev_status)
+                n += 1
+            if "bwd_data" in passes and (li > 0 or self.input_grad):
+                api.lpdt_qconv_bwd_data(b["desc"], b["E"], b["sE"], b["qW"], b["sW"], dA=b["dx"], ws=self.ws,
+                                        dev_status=self.dev_status)
+                n += 1
+        return n
+
     # ---- CUDA graph: the whole step as one replayable launch -------------------------------
     def capture(self):
         """Record run() into a CUDA graph (one warm-up run first so that every
