@@ -113,6 +113,11 @@ class TrainStep:
         self.ranges = torch.zeros(2 * len(ops), N, **f32)
         self.dy = torch.zeros((N, B) + tuple(shape), **f32)      # upstream gradient / dlogits
         self.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        # The weight-gradient contractions leave the critical path of the backward pass: each is issued on a
+        # side stream (its own workspace) as soon as its quantized layer gradient exists, and joins before the
+        # parameter update.  Captured into the step's CUDA graph the fork and join become graph edges.
+        self.ws_side = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        self.side = torch.cuda.Stream(device=dev)
 
     # ---- host -> device ------------------------------------------------------------
     def load(self, wl):
@@ -218,15 +223,18 @@ class TrainStep:
                     api.lpdt_quantize(g, N, n_out, n_out, b["E"], b["sE"], self.ws, rounding=self.grad_rounding,
                                       seed=self.seed, ctr_offset=ctr)
                 ctr += 1
-                if self.quantize_wgrad:
-                    api.lpdt_qconv_bwd_weight(b["desc"], b["E"], b["sE"], b["qA"], b["sA"], dW=b["gw"],
-                                              dw_node_stride=b["wn"], ws=self.ws, dev_status=self.dev_status)
-                    api.lpdt_quantize(b["gw"], N, b["wn"], b["wn"], b["gq"], b["gs"], self.ws)
-                    api.lpdt_dequantize(b["gq"], N, b["wn"], b["gs"], self._g(op["w_off"]), d)
-                else:
-                    api.lpdt_qconv_bwd_weight(b["desc"], b["E"], b["sE"], b["qA"], b["sA"],
-                                              dW=self._g(op["w_off"]), dw_node_stride=d, ws=self.ws,
-                                              dev_status=self.dev_status)
+                main = torch.cuda.current_stream()
+                self.side.wait_stream(main)               # E (and, at the first use, everything before) is ready
+                with torch.cuda.stream(self.side):
+                    if self.quantize_wgrad:
+                        api.lpdt_qconv_bwd_weight(b["desc"], b["E"], b["sE"], b["qA"], b["sA"], dW=b["gw"],
+                                                  dw_node_stride=b["wn"], ws=self.ws_side, dev_status=self.dev_status)
+                        api.lpdt_quantize(b["gw"], N, b["wn"], b["wn"], b["gq"], b["gs"], self.ws_side)
+                        api.lpdt_dequantize(b["gq"], N, b["wn"], b["gs"], self._g(op["w_off"]), d)
+                    else:
+                        api.lpdt_qconv_bwd_weight(b["desc"], b["E"], b["sE"], b["qA"], b["sA"],
+                                                  dW=self._g(op["w_off"]), dw_node_stride=d, ws=self.ws_side,
+                                                  dev_status=self.dev_status)
                 if li > 0 or self.input_grad:
                     api.lpdt_qconv_bwd_data(b["desc"], b["E"], b["sE"], b["qW"], b["sW"], dA=b["dx"],
                                             ws=self.ws, dev_status=self.dev_status)
@@ -254,6 +262,7 @@ class TrainStep:
             elif k == "avgpool":
                 api.lpdt_avgpool_bwd(N, B, op["H"] * op["W"], op["C"], g, b["dx"])
                 g, g_range = b["dx"], None
+        torch.cuda.current_stream().wait_stream(self.side)      # weight gradients complete before the update
         self.input_grad_out = g
         return g
 
