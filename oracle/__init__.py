@@ -104,6 +104,24 @@ def qconv_fwd(A, Wq, stride=1, pad=1):
     return acc, ovf.value
 
 
+def qconv_fwd_affine(A, zA, Wq, zW, stride=1, pad=1):
+    """A uint8 [n,B,H,W,Cin], Wq uint8 [n,Cout,R,S,Cin], zero points int32 [n] ->
+    (acc int32 [n,B,Ho,Wo,Cout] of (qa - zA)(qw - zW) over the taps inside the image, overflow)."""
+    A = _c(A, np.uint8)
+    Wq = _c(Wq, np.uint8)
+    zA = _c(zA, np.int32)
+    zW = _c(zW, np.int32)
+    n, B, H, W, Cin = A.shape
+    _, Cout, R, S, _ = Wq.shape
+    assert zA.shape == (n,) and zW.shape == (n,)
+    Ho, Wo = _out_hw(H, W, R, S, stride, pad)
+    acc = np.zeros((n, B, Ho, Wo, Cout), np.int32)
+    ovf = _i64(0)
+    lib().orc_qconv_fwd_affine(n, B, H, W, Cin, Cout, R, S, stride, pad, _p(A), _p(zA), _p(Wq), _p(zW),
+                               _p(acc), C.byref(ovf))
+    return acc, ovf.value
+
+
 def qconv_bwd_data(E, Wq, H, W, stride=1, pad=1):
     """E int8 [n,B,Ho,Wo,Cout], Wq int8 [n,Cout,R,S,Cin] -> (dA int32 [n,B,H,W,Cin], overflow)."""
     E = _c(E, np.int8)

@@ -229,6 +229,41 @@ void orc_qconv_fwd(int nodes, int B, int H, int W, int Cin, int Cout, int R, int
     }
 }
 
+/* Forward contraction on affine (zero-point) 8-bit operands, the quantization scheme
+ * Section 3 names: real a = sA*(qa - zA), real w = sW*(qw - zW), qa and qw unsigned
+ * codes, one zero point per node and tensor.  The convolution pads with real zeros,
+ * so a tap outside the image contributes nothing:
+ *   acc[n,b,oh,ow,co] = sum over taps inside the image, ci of (qa - zA[n]) * (qw - zW[n]). */
+void orc_qconv_fwd_affine(int nodes, int B, int H, int W, int Cin, int Cout, int R, int S,
+                          int stride, int pad, const uint8_t *A, const int32_t *zA,
+                          const uint8_t *Wq, const int32_t *zW, int32_t *acc, i64 *overflow)
+{
+    const int Ho = (H + 2 * pad - R) / stride + 1;
+    const int Wo = (W + 2 * pad - S) / stride + 1;
+    *overflow = 0;
+    #pragma omp parallel for collapse(3) schedule(static)
+    for (int n = 0; n < nodes; ++n)
+    for (int b = 0; b < B; ++b)
+    for (int oh = 0; oh < Ho; ++oh)
+    for (int ow = 0; ow < Wo; ++ow)
+    for (int co = 0; co < Cout; ++co) {
+        i64 sum = 0;
+        for (int r = 0; r < R; ++r) {
+            int ih = oh * stride + r - pad;
+            if (ih < 0 || ih >= H) continue;
+            for (int s = 0; s < S; ++s) {
+                int iw = ow * stride + s - pad;
+                if (iw < 0 || iw >= W) continue;
+                const uint8_t *a = A + ((((i64)n * B + b) * H + ih) * W + iw) * Cin;
+                const uint8_t *w = Wq + ((((i64)n * Cout + co) * R + r) * S + s) * Cin;
+                for (int ci = 0; ci < Cin; ++ci)
+                    sum += ((int32_t)a[ci] - zA[n]) * ((int32_t)w[ci] - zW[n]);
+            }
+        }
+        acc[((((i64)n * B + b) * Ho + oh) * Wo + ow) * Cout + co] = wrap32(sum, overflow);
+    }
+}
+
 /* dA[n,b,ih,iw,ci] = sum over (oh,ow,r,s,co) with ih = oh*stride + r - pad,
  * iw = ow*stride + s - pad of E[n,b,oh,ow,co] * W[n,co,r,s,ci]. */
 void orc_qconv_bwd_data(int nodes, int B, int H, int W, int Cin, int Cout, int R, int S,

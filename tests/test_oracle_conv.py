@@ -163,3 +163,74 @@ def test_dequant_acc():
     b = np.array([[1.0, -1.0], [0.5, 0.0]], np.float32)
     yb = oracle.dequant_acc(acc, s1, s2, b)
     assert np.array_equal(yb, y + b[:, None, :])
+
+
+# ---- affine (zero-point) operands (Section 3 names the scheme; taps outside the image are real zeros) ----
+def _affine_case(seed, n=2, B=2, H=5, W=6, Cin=3, Cout=4, R=3, S=3):
+    rng = np.random.default_rng(seed)
+    A = rng.integers(0, 256, (n, B, H, W, Cin), dtype=np.uint8)
+    Wq = rng.integers(0, 256, (n, Cout, R, S, Cin), dtype=np.uint8)
+    zA = rng.integers(0, 256, n).astype(np.int32)
+    zW = rng.integers(0, 256, n).astype(np.int32)
+    return A, zA, Wq, zW
+
+
+def test_affine_zero_zero_points_is_the_plain_product():
+    # with both zero points 0 and codes below 128 the affine product is the signed one
+    rng = np.random.default_rng(1)
+    A = rng.integers(0, 128, (2, 2, 6, 5, 4), dtype=np.uint8)
+    Wq = rng.integers(0, 128, (2, 3, 3, 3, 4), dtype=np.uint8)
+    z = np.zeros(2, np.int32)
+    acc, ovf = oracle.qconv_fwd_affine(A, z, Wq, z, stride=1, pad=1)
+    ref, _ = oracle.qconv_fwd(A.astype(np.int8), Wq.astype(np.int8), stride=1, pad=1)
+    assert ovf == 0 and np.array_equal(acc, ref)
+
+
+def test_affine_constant_input_at_the_zero_point_gives_zero():
+    A, zA, Wq, zW = _affine_case(2)
+    for i in range(A.shape[0]):
+        A[i] = zA[i]                        # real 0 everywhere, borders included
+    acc, _ = oracle.qconv_fwd_affine(A, zA, Wq, zW, stride=1, pad=1)
+    assert not acc.any()
+    for i in range(Wq.shape[0]):            # and a weight tensor of real zeros
+        Wq[i] = zW[i]
+    A2 = _affine_case(3)[0]
+    acc, _ = oracle.qconv_fwd_affine(A2, zA, Wq, zW, stride=2, pad=1)
+    assert not acc.any()
+
+
+@pytest.mark.parametrize("stride,pad,R", [(1, 1, 3), (2, 1, 3), (1, 0, 1), (1, 2, 5)])
+def test_affine_equals_real_domain_correlation(stride, pad, R):
+    # dequantize, zero-pad the REAL tensor, correlate with numpy in float64: a library routine on the meaning
+    A, zA, Wq, zW = _affine_case(4, H=7, W=6, R=R, S=R)
+    sA, sW = 0.013, 0.21
+    acc, ovf = oracle.qconv_fwd_affine(A, zA, Wq, zW, stride=stride, pad=pad)
+    assert ovf == 0
+    n, B, H, W, Cin = A.shape
+    Cout = Wq.shape[1]
+    Ho, Wo = acc.shape[2], acc.shape[3]
+    for i in range(n):
+        a = sA * (A[i].astype(np.float64) - zA[i])
+        w = sW * (Wq[i].astype(np.float64) - zW[i])
+        ap = np.pad(a, ((0, 0), (pad, pad), (pad, pad), (0, 0)))
+        win = np.lib.stride_tricks.sliding_window_view(ap, (R, R), axis=(1, 2))[:, ::stride, ::stride]   # b,oh,ow,ci,r,s
+        ref = np.einsum("bhwcrs,orsc->bhwo", win[:, :Ho, :Wo], w)
+        np.testing.assert_allclose(sA * sW * acc[i].astype(np.float64), ref, rtol=1e-12, atol=1e-9)
+
+
+def test_affine_expansion_identity():
+    # sum (qa - zA)(qw - zW) = sum qa qw - zW sum qa - zA sum qw + (#terms) zA zW over the taps inside the image:
+    # each term evaluated with the zero-point-free oracle on helper tensors
+    A, zA, Wq, zW = _affine_case(5, Cin=2, Cout=3)
+    acc, _ = oracle.qconv_fwd_affine(A, zA, Wq, zW, stride=1, pad=1)
+    z0 = np.zeros(A.shape[0], np.int32)
+    raw, _ = oracle.qconv_fwd_affine(A, z0, Wq, z0, stride=1, pad=1)
+    ones_w = np.ones_like(Wq)
+    ones_a = np.ones_like(A)
+    ra, _ = oracle.qconv_fwd_affine(A, z0, ones_w, z0, stride=1, pad=1)        # sum of qa over the valid taps
+    rw, _ = oracle.qconv_fwd_affine(ones_a, z0, Wq, z0, stride=1, pad=1)       # sum of qw over the valid taps
+    cnt, _ = oracle.qconv_fwd_affine(ones_a, z0, ones_w, z0, stride=1, pad=1)  # number of terms
+    zA_, zW_ = zA[:, None, None, None, None].astype(np.int64), zW[:, None, None, None, None].astype(np.int64)
+    ref = raw.astype(np.int64) - zW_ * ra - zA_ * rw + cnt * zA_ * zW_
+    assert np.array_equal(acc.astype(np.int64), ref)
+    assert cnt[0, 0, 0, 0, 0] == 4 * 2 and cnt[0, 0, 2, 2, 0] == 9 * 2         # corner and interior term counts
