@@ -189,6 +189,33 @@ lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8_t *E, cons
                                   void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
 
 /* ---------------------------------------------------------------------------
+ * Forward contraction on affine (zero-point) operands: the quantization scheme
+ * Section 3 names maps a real tensor to unsigned 8-bit codes with a scale and a
+ * zero point, real = scale*(code - zero_point) (lpdt_quantize, LPDT_AFFINE_U8).
+ * The convolution pads with real zeros, so taps outside the image add nothing:
+ *
+ *   acc[n,b,oh,ow,co] = sum_{(r,s) inside the image, ci}
+ *                       (A[n,b,oh*st+r-p,ow*st+s-p,ci] - zA[n]) * (W[n,co,r,s,ci] - zW[n])
+ *   Y = (float)acc * (sA[n]*sW[n]) (+ bias)
+ *
+ * A, Wq   : uint8 codes in the layouts of lpdt_qconv_fwd;  zA, zW : int32 [nodes],
+ *           each in [0, 255];  sA, sW : fp32 [nodes] (needed only for Y)
+ * Y, Yacc : as in lpdt_qconv_fwd (at least one); int32 results wrap modulo 2^32
+ * ws      : lpdt_qconv_fwd_affine_workspace_size(desc) bytes, 256-byte aligned
+ * The integer contraction of the codes runs on the same kernels as
+ * lpdt_qconv_fwd (unsigned operand format); the zero-point terms are applied
+ * by a correction pass over the int32 sums.  Only the forward product is
+ * provided in this form.
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA; TIMEOUT through dev_status.
+ */
+size_t lpdt_qconv_fwd_affine_workspace_size(const lpdt_conv_desc *d);
+lpdt_status lpdt_qconv_fwd_affine(const lpdt_conv_desc *d, const uint8_t *A, const float *sA, const int32_t *zA,
+                                  const uint8_t *Wq, const float *sW, const int32_t *zW,
+                                  const float *bias, int64_t bias_node_stride,
+                                  float *Y, int32_t *Yacc,
+                                  void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
+
+/* ---------------------------------------------------------------------------
  * Range-EvoNorm (Eq. "ren"), forward and backward.
  * For node n, sample b, group G of cpg = C/groups consecutive channels:
  *   mx, mn = max/min of x over (h, w, c in G);  D = Cst*(mx-mn) + eps,

@@ -6,7 +6,9 @@ seeded random operands, through the C ABI.
     python -m paper_2111_09389_b200.contraction_sweep sweep           # the large GEMM / conv grid
 
 Operands are iid uniform int8 in [-127, 127]; every shape runs with int32
-accumulation and the fused fp32 dequantize.  Prints one JSON line per
+accumulation and the fused fp32 dequantize.  The optional pass
+`fwd_affine` times the forward product on zero-point operands (same operand
+bytes; its correction pass re-reads and re-writes the result).  Prints one JSON line per
 (shape, pass) with the CUDA-event time, int8 TOPS (2 * MACs / time) and the
 HBM bytes the pass must move at least.
 """
@@ -51,6 +53,14 @@ def time_case(nodes, B, H, W, Cin, Cout, R, S, stride, pad, iters=20, warmup=3, 
                                                          dev_status=status),
                        E.numel() + A.numel() + 4 * dW.numel()),
     }
+    if "fwd_affine" in passes:       # zero-point operands: unsigned codes, per-node zero points
+        Au, Wu = A.view(torch.uint8), Wq.view(torch.uint8)
+        zA = torch.full((nodes,), 131, dtype=torch.int32, device="cuda")
+        zW = torch.full((nodes,), 120, dtype=torch.int32, device="cuda")
+        wsa = torch.empty(api.lpdt_qconv_fwd_affine_workspace_size(desc), dtype=torch.uint8, device="cuda")
+        calls["fwd_affine"] = (lambda: api.lpdt_qconv_fwd_affine(desc, Au, sc, zA, Wu, sc, zW, Y=Y, ws=wsa,
+                                                                 dev_status=status),
+                               A.numel() + Wq.numel() + 4 * Y.numel())
     out = []
     for name in passes:
         fn, min_bytes = calls[name]

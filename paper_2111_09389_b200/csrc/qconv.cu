@@ -56,12 +56,12 @@ static bool use_halo(const lpdt_conv_desc &d, int mode) {
 }
 static lpdt_status run_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const float *s1, const int8_t *Wq,
                            const float *s2, const float *bias, int64_t bias_stride, float *Y, int32_t *Yacc,
-                           int32_t *dev_status, cudaStream_t st) {
+                           int32_t *dev_status, cudaStream_t st, bool uns = false) {
     if (use_halo(d, mode)) {
-        lpdt_status r = tc::tc_pix_halo(d, mode, A, s1, Wq, s2, bias, bias_stride, Y, Yacc, dev_status, st);
+        lpdt_status r = tc::tc_pix_halo(d, mode, A, s1, Wq, s2, bias, bias_stride, Y, Yacc, dev_status, st, uns);
         if (r != LPDT_ERR_UNSUPPORTED) return r;
     }
-    return tc::tc_pix(d, mode, A, s1, Wq, s2, bias, bias_stride, Y, Yacc, dev_status, st);
+    return tc::tc_pix(d, mode, A, s1, Wq, s2, bias, bias_stride, Y, Yacc, dev_status, st, uns);
 }
 
 static int pad16(int c) { return (c + 15) / 16 * 16; }
@@ -105,20 +105,13 @@ extern "C" size_t lpdt_qconv_workspace_size(const lpdt_conv_desc *d, int32_t whi
     return need;
 }
 
-extern "C" lpdt_status lpdt_qconv_fwd(const lpdt_conv_desc *d, const int8_t *A, const float *sA,
-                                      const int8_t *Wq, const float *sW, const float *bias,
-                                      int64_t bias_node_stride, float *Y, int32_t *Yacc, void *ws,
-                                      size_t ws_bytes, int32_t *dev_status, void *stream) {
-    lpdt_status s = check_desc(d);
-    if (s != LPDT_OK) return s;
-    if (d->nodes == 0 || d->B == 0) return LPDT_OK;
-    LPDT_CHECK_ARG(A && Wq && (Y || Yacc));
-    LPDT_CHECK_ARG(!Y || (sA && sW));
-    LPDT_CHECK_ARG(!bias || bias_node_stride >= d->Cout || d->nodes == 1);
-    cudaStream_t st = as_stream(stream);
+// Forward contraction on raw codes (signed, or unsigned when `uns`): kernel choice only.
+static lpdt_status fwd_impl(const lpdt_conv_desc *d, const int8_t *A, const float *sA, const int8_t *Wq,
+                            const float *sW, const float *bias, int64_t bias_node_stride, float *Y, int32_t *Yacc,
+                            void *ws, size_t ws_bytes, int32_t *dev_status, cudaStream_t st, bool uns) {
     const bool out_ok = (!Y || aligned(Y, 16)) && (!Yacc || aligned(Yacc, 16));
     if (use_tc(*d) && aligned(A, 16) && aligned(Wq, 16) && out_ok)
-        return run_pix(*d, 0, A, sA, Wq, sW, bias, bias_node_stride, Y, Yacc, dev_status, st);
+        return run_pix(*d, 0, A, sA, Wq, sW, bias, bias_node_stride, Y, Yacc, dev_status, st, uns);
     lpdt_conv_desc dp;
     if (use_tc_padded(*d, &dp) && out_ok && ws && aligned(ws, 256) &&
         ws_bytes >= lpdt_qconv_workspace_size(d, 0)) {
@@ -129,9 +122,224 @@ extern "C" lpdt_status lpdt_qconv_fwd(const lpdt_conv_desc *d, const int8_t *A, 
         LPDT_LAUNCH_CHECK();
         pad_channels_kernel<<<grid_for(wrows * dp.Cin / 16), 256, 0, st>>>(Wq, Wp, wrows, d->Cin, dp.Cin);
         LPDT_LAUNCH_CHECK();
-        return run_pix(dp, 0, Ap, sA, Wp, sW, bias, bias_node_stride, Y, Yacc, dev_status, st);
+        return run_pix(dp, 0, Ap, sA, Wp, sW, bias, bias_node_stride, Y, Yacc, dev_status, st, uns);
     }
-    return generic_fwd(*d, A, sA, Wq, sW, bias, bias_node_stride, Y, Yacc, st);
+    return generic_fwd(*d, A, sA, Wq, sW, bias, bias_node_stride, Y, Yacc, st, uns);
+}
+
+extern "C" lpdt_status lpdt_qconv_fwd(const lpdt_conv_desc *d, const int8_t *A, const float *sA,
+                                      const int8_t *Wq, const float *sW, const float *bias,
+                                      int64_t bias_node_stride, float *Y, int32_t *Yacc, void *ws,
+                                      size_t ws_bytes, int32_t *dev_status, void *stream) {
+    lpdt_status s = check_desc(d);
+    if (s != LPDT_OK) return s;
+    if (d->nodes == 0 || d->B == 0) return LPDT_OK;
+    LPDT_CHECK_ARG(A && Wq && (Y || Yacc));
+    LPDT_CHECK_ARG(!Y || (sA && sW));
+    LPDT_CHECK_ARG(!bias || bias_node_stride >= d->Cout || d->nodes == 1);
+    return fwd_impl(d, A, sA, Wq, sW, bias, bias_node_stride, Y, Yacc, ws, ws_bytes, dev_status, as_stream(stream),
+                    false);
+}
+
+// ---- affine (zero-point) operands -------------------------------------------------------------
+// sum (qa - zA)(qw - zW) over the taps inside the image
+//   = sum qa*qw  -  zW * sum qa  -  zA * sum qw  +  (taps inside * Cin) * zA * zW.
+// The first term is the contraction engine on the unsigned codes (taps outside the image read code 0
+// and add nothing); the other three come from per-pixel channel sums of the input and from prefix
+// sums over the filter taps of the weights' channel sums (the taps inside the image form a rectangle
+// of the filter).  All arithmetic is modulo 2^32, like the accumulators.
+namespace lpdt {
+
+// out[row] = sum of the `len` unsigned bytes of row `row`.  A group of G lanes (a power of two up to
+// 32, chosen by the launcher from the row length) shares a row: 16-byte loads when the rows allow.
+__global__ void row_sum_u8_kernel(const uint8_t *__restrict__ src, int64_t rows, int len, int G, bool vec16,
+                                  int32_t *__restrict__ out) {
+    const int lane_in_group = threadIdx.x & (G - 1);
+    const int64_t groups_total = ((int64_t)gridDim.x * blockDim.x) / G;
+    for (int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;; row += groups_total) {
+        if (row - (int)((threadIdx.x & 31) / G) >= rows) break;      // warp-uniform: the warp's first row is past the end
+        const bool valid = row < rows;                               // lanes past the end still take part in the shuffles
+        const uint8_t *a = src + (valid ? row : 0) * len;
+        unsigned sum = 0;
+        if (!valid) {
+        } else if (vec16) {
+            const uint4 *a16 = reinterpret_cast<const uint4 *>(a);
+            for (int i = lane_in_group; i < len / 16; i += G) {
+                const uint4 v = __ldg(a16 + i);
+                sum = __dp4a(v.x, 0x01010101u, sum); sum = __dp4a(v.y, 0x01010101u, sum);
+                sum = __dp4a(v.z, 0x01010101u, sum); sum = __dp4a(v.w, 0x01010101u, sum);
+            }
+        } else {
+            for (int i = lane_in_group; i < len; i += G) sum += a[i];
+        }
+        for (int o = G >> 1; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        if (valid && lane_in_group == 0) out[row] = (int32_t)sum;
+    }
+}
+
+// P[n][r][s][co] for 0 <= r <= R, 0 <= s <= S: sum of tapsum[n][co][r'][s'] over r' < r, s' < s.  The output
+// channel is the fastest index, so the correction pass reads four neighbours with one 16-byte load.
+__global__ void weight_prefix_kernel(const int32_t *__restrict__ tapsum, int nodes, int Cout, int R, int S,
+                                     int32_t *__restrict__ P) {
+    const int row = blockIdx.x * blockDim.x + threadIdx.x;        // (node, co)
+    if (row >= nodes * Cout) return;
+    const int n = row / Cout, co = row % Cout, PS = S + 1;
+    const int32_t *t = tapsum + (int64_t)row * R * S;
+    int32_t *p = P + (int64_t)n * (R + 1) * PS * Cout + co;
+    for (int s = 0; s <= S; ++s) p[(int64_t)s * Cout] = 0;
+    for (int r = 1; r <= R; ++r) {
+        p[(int64_t)(r * PS) * Cout] = 0;
+        unsigned run = 0;                                     // taps (r-1, < s)
+        for (int s = 1; s <= S; ++s) {
+            run += (unsigned)t[(r - 1) * S + (s - 1)];
+            p[(int64_t)(r * PS + s) * Cout] = (int32_t)((unsigned)p[(int64_t)((r - 1) * PS + s) * Cout] + run);
+        }
+    }
+}
+
+// One thread per (output pixel, V consecutive output channels); V = 4 with 16-byte accesses when the
+// channel count allows, else 1.
+template <int V>
+__global__ void affine_fix_kernel(lpdt_conv_desc d, int Ho, int Wo, const int32_t *__restrict__ raw,
+                                  const int32_t *__restrict__ asum, const int32_t *__restrict__ P,
+                                  const int32_t *__restrict__ zA, const int32_t *__restrict__ zW,
+                                  const float *__restrict__ sA, const float *__restrict__ sW,
+                                  const float *__restrict__ bias, int64_t bias_stride, float *__restrict__ Y,
+                                  int32_t *__restrict__ Yacc) {
+    const int chunks = d.Cout / V;
+    const int64_t total = (int64_t)d.nodes * d.B * Ho * Wo * chunks;
+    for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
+        const int co0 = (int)(o % chunks) * V;
+        const int64_t pix = o / chunks;
+        const int ow = (int)(pix % Wo);
+        const int oh = (int)((pix / Wo) % Ho);
+        const int64_t nb = pix / ((int64_t)Wo * Ho);
+        const int n = (int)(nb / d.B);
+        // filter rows / columns whose tap lies inside the image
+        int r_lo = d.pad - oh * d.stride; if (r_lo < 0) r_lo = 0;
+        int r_hi = d.H + d.pad - oh * d.stride; if (r_hi > d.R) r_hi = d.R;
+        int s_lo = d.pad - ow * d.stride; if (s_lo < 0) s_lo = 0;
+        int s_hi = d.W + d.pad - ow * d.stride; if (s_hi > d.S) s_hi = d.S;
+        if (r_hi < r_lo) r_hi = r_lo;
+        if (s_hi < s_lo) s_hi = s_lo;
+        unsigned ra = 0;
+        for (int r = r_lo; r < r_hi; ++r)
+            for (int s = s_lo; s < s_hi; ++s)
+                ra += (unsigned)__ldg(asum + (nb * d.H + oh * d.stride + r - d.pad) * d.W + ow * d.stride + s - d.pad);
+        const unsigned za = (unsigned)zA[n], zw = (unsigned)zW[n];
+        const unsigned cnt = (unsigned)((r_hi - r_lo) * (s_hi - s_lo) * d.Cin);
+        const unsigned fixed = cnt * za * zw - zw * ra;
+        const float sc = Y ? __fmul_rn(sA[n], sW[n]) : 0.f;
+        const int PS = d.S + 1;
+        const int64_t oi = pix * d.Cout + co0;
+        int rawv[V], acc[V];
+        if (V == 4) { const int4 t = *reinterpret_cast<const int4 *>(raw + oi); rawv[0] = t.x; rawv[1] = t.y; rawv[2] = t.z; rawv[3] = t.w; }
+        else rawv[0] = raw[oi];
+        // rectangle sum of the weights' channel sums over the taps inside the image: four corners of the prefix table
+        const int32_t *p = P + (int64_t)n * (d.R + 1) * PS * d.Cout + co0;
+        int c11[V], c01[V], c10[V], c00[V];
+        auto corner = [&](int r, int s2, int (&o)[V]) {
+            const int32_t *q = p + (int64_t)(r * PS + s2) * d.Cout;
+            if (V == 4) { const int4 t = __ldg(reinterpret_cast<const int4 *>(q)); o[0] = t.x; o[1] = t.y; o[2] = t.z; o[3] = t.w; }
+            else o[0] = __ldg(q);
+        };
+        corner(r_hi, s_hi, c11); corner(r_lo, s_hi, c01); corner(r_hi, s_lo, c10); corner(r_lo, s_lo, c00);
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            const unsigned rw = (unsigned)c11[k] - (unsigned)c01[k] - (unsigned)c10[k] + (unsigned)c00[k];
+            acc[k] = (int)((unsigned)rawv[k] + fixed - za * rw);
+        }
+        if (Yacc) {
+            if (V == 4) *reinterpret_cast<int4 *>(Yacc + oi) = make_int4(acc[0], acc[1], acc[2], acc[3]);
+            else Yacc[oi] = acc[0];
+        }
+        if (Y) {
+            float v[V];
+#pragma unroll
+            for (int k = 0; k < V; ++k) {
+                v[k] = __fmul_rn(__int2float_rn(acc[k]), sc);
+                if (bias) v[k] = __fadd_rn(v[k], bias[(int64_t)n * bias_stride + co0 + k]);
+            }
+            if (V == 4) *reinterpret_cast<float4 *>(Y + oi) = make_float4(v[0], v[1], v[2], v[3]);
+            else Y[oi] = v[0];
+        }
+    }
+}
+
+// rows of `len` bytes -> out[row]; lanes per row grow with the row length
+static lpdt_status row_sum_launch(const uint8_t *src, int64_t rows, int len, int32_t *out, cudaStream_t st) {
+    const bool vec16 = len % 16 == 0 && aligned(src, 16);
+    const int units = vec16 ? len / 16 : len;
+    int G = 1;
+    while (G < 32 && G * 4 <= units) G <<= 1;             // at least four loads per lane
+    int64_t blocks = ceil_div(rows * G, 256);
+    const int64_t cap = (int64_t)kNumSMs * 32;
+    if (blocks > cap) blocks = cap;
+    if (blocks < 1) blocks = 1;
+    row_sum_u8_kernel<<<(unsigned)blocks, 256, 0, st>>>(src, rows, len, G, vec16, out);
+    LPDT_LAUNCH_CHECK();
+    return LPDT_OK;
+}
+
+}  // namespace lpdt
+
+static size_t affine_raw_bytes(const lpdt_conv_desc *d) {
+    const int Ho = conv_out(d->H, d->pad, d->R, d->stride), Wo = conv_out(d->W, d->pad, d->S, d->stride);
+    return align_up((size_t)d->nodes * d->B * Ho * Wo * d->Cout * sizeof(int32_t), 256);
+}
+static size_t affine_asum_bytes(const lpdt_conv_desc *d) {
+    return align_up((size_t)d->nodes * d->B * d->H * d->W * sizeof(int32_t), 256);
+}
+static size_t affine_prefix_bytes(const lpdt_conv_desc *d) {     // prefix table + per-tap channel sums
+    return align_up((size_t)d->nodes * d->Cout * (d->R + 1) * (d->S + 1) * sizeof(int32_t), 256) +
+           align_up((size_t)d->nodes * d->Cout * d->R * d->S * sizeof(int32_t), 256);
+}
+
+extern "C" size_t lpdt_qconv_fwd_affine_workspace_size(const lpdt_conv_desc *d) {
+    if (!d || d->nodes <= 0 || check_desc(d) != LPDT_OK) return 256;
+    return affine_raw_bytes(d) + affine_asum_bytes(d) + affine_prefix_bytes(d) + lpdt_qconv_workspace_size(d, 0);
+}
+
+extern "C" lpdt_status lpdt_qconv_fwd_affine(const lpdt_conv_desc *d, const uint8_t *A, const float *sA,
+                                             const int32_t *zA, const uint8_t *Wq, const float *sW,
+                                             const int32_t *zW, const float *bias, int64_t bias_node_stride,
+                                             float *Y, int32_t *Yacc, void *ws, size_t ws_bytes,
+                                             int32_t *dev_status, void *stream) {
+    lpdt_status s = check_desc(d);
+    if (s != LPDT_OK) return s;
+    if (d->nodes == 0 || d->B == 0) return LPDT_OK;
+    LPDT_CHECK_ARG(A && Wq && zA && zW && (Y || Yacc));
+    LPDT_CHECK_ARG(!Y || (sA && sW));
+    LPDT_CHECK_ARG(!bias || bias_node_stride >= d->Cout || d->nodes == 1);
+    if (!ws || !aligned(ws, 256) || ws_bytes < lpdt_qconv_fwd_affine_workspace_size(d)) return LPDT_ERR_WORKSPACE;
+    cudaStream_t st = as_stream(stream);
+    const int Ho = conv_out(d->H, d->pad, d->R, d->stride), Wo = conv_out(d->W, d->pad, d->S, d->stride);
+    int32_t *raw = (int32_t *)ws;
+    int32_t *asum = (int32_t *)((char *)ws + affine_raw_bytes(d));
+    int32_t *P = (int32_t *)((char *)asum + affine_asum_bytes(d));
+    void *inner = (char *)P + affine_prefix_bytes(d);
+    s = fwd_impl(d, reinterpret_cast<const int8_t *>(A), nullptr, reinterpret_cast<const int8_t *>(Wq), nullptr, nullptr,
+                 0, nullptr, raw, inner, lpdt_qconv_workspace_size(d, 0), dev_status, st, true);
+    if (s != LPDT_OK) return s;
+    const int64_t pixels = (int64_t)d->nodes * d->B * d->H * d->W;
+    s = row_sum_launch(A, pixels, d->Cin, asum, st);
+    if (s != LPDT_OK) return s;
+    const int rows = d->nodes * d->Cout;
+    int32_t *tapsum = (int32_t *)((char *)P + align_up((size_t)rows * (d->R + 1) * (d->S + 1) * sizeof(int32_t), 256));
+    s = row_sum_launch(Wq, (int64_t)rows * d->R * d->S, d->Cin, tapsum, st);
+    if (s != LPDT_OK) return s;
+    weight_prefix_kernel<<<(rows + 127) / 128, 128, 0, st>>>(tapsum, d->nodes, d->Cout, d->R, d->S, P);
+    LPDT_LAUNCH_CHECK();
+    const bool v4 = d->Cout % 4 == 0 && (!Y || aligned(Y, 16)) && (!Yacc || aligned(Yacc, 16));
+    const int64_t work = (int64_t)d->nodes * d->B * Ho * Wo * (d->Cout / (v4 ? 4 : 1));
+    if (v4)
+        affine_fix_kernel<4><<<grid_for(work), 256, 0, st>>>(*d, Ho, Wo, raw, asum, P, zA, zW, sA, sW, bias,
+                                                             bias_node_stride, Y, Yacc);
+    else
+        affine_fix_kernel<1><<<grid_for(work), 256, 0, st>>>(*d, Ho, Wo, raw, asum, P, zA, zW, sA, sW, bias,
+                                                             bias_node_stride, Y, Yacc);
+    LPDT_LAUNCH_CHECK();
+    return LPDT_OK;
 }
 
 extern "C" lpdt_status lpdt_qconv_bwd_data(const lpdt_conv_desc *d, const int8_t *E, const float *sE,

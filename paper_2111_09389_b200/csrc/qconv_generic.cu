@@ -20,12 +20,25 @@ __device__ __forceinline__ int dot_s8(const int8_t *__restrict__ a, const int8_t
     return acc;
 }
 
+// the same on unsigned codes
+__device__ __forceinline__ int dot_u8(const uint8_t *__restrict__ a, const uint8_t *__restrict__ b, int n, bool vec4) {
+    unsigned acc = 0;
+    if (vec4) {
+        const unsigned *a4 = reinterpret_cast<const unsigned *>(a);
+        const unsigned *b4 = reinterpret_cast<const unsigned *>(b);
+        for (int i = 0; i < n / 4; ++i) acc = __dp4a(__ldg(a4 + i), __ldg(b4 + i), acc);
+    } else {
+        for (int i = 0; i < n; ++i) acc += (unsigned)a[i] * (unsigned)b[i];
+    }
+    return (int)acc;
+}
+
 // One thread per output element (n, b, oh, ow, co); co fastest.
 __global__ void conv_fwd_generic(lpdt_conv_desc d, int Ho, int Wo, const int8_t *__restrict__ A,
                                  const int8_t *__restrict__ Wq, int32_t *__restrict__ acc_out,
                                  float *__restrict__ Y, const float *__restrict__ s1,
                                  const float *__restrict__ s2, const float *__restrict__ bias,
-                                 int64_t bias_stride, bool vec4) {
+                                 int64_t bias_stride, bool vec4, bool uns) {
     const int64_t per_node = (int64_t)d.B * Ho * Wo * d.Cout;
     const int64_t total = per_node * d.nodes;
     for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
@@ -44,7 +57,8 @@ __global__ void conv_fwd_generic(lpdt_conv_desc d, int Ho, int Wo, const int8_t 
                 if (iw < 0 || iw >= d.W) continue;
                 const int8_t *a = A + ((((int64_t)n * d.B + b) * d.H + ih) * d.W + iw) * d.Cin;
                 const int8_t *w = Wq + ((((int64_t)n * d.Cout + co) * d.R + r) * d.S + s) * d.Cin;
-                acc += dot_s8(a, w, d.Cin, vec4);
+                acc += uns ? dot_u8(reinterpret_cast<const uint8_t *>(a), reinterpret_cast<const uint8_t *>(w), d.Cin, vec4)
+                           : dot_s8(a, w, d.Cin, vec4);
             }
         }
         if (acc_out) acc_out[o] = acc;
@@ -165,11 +179,11 @@ static unsigned grid_for(int64_t n) {
 
 lpdt_status generic_fwd(const lpdt_conv_desc &d, const int8_t *A, const float *sA, const int8_t *Wq,
                         const float *sW, const float *bias, int64_t bias_stride, float *Y, int32_t *Yacc,
-                        cudaStream_t st) {
+                        cudaStream_t st, bool uns) {
     const int Ho = conv_out(d.H, d.pad, d.R, d.stride), Wo = conv_out(d.W, d.pad, d.S, d.stride);
     const int64_t total = (int64_t)d.nodes * d.B * Ho * Wo * d.Cout;
     const bool vec4 = d.Cin % 4 == 0 && aligned(A, 4) && aligned(Wq, 4);
-    conv_fwd_generic<<<grid_for(total), 256, 0, st>>>(d, Ho, Wo, A, Wq, Yacc, Y, sA, sW, bias, bias_stride, vec4);
+    conv_fwd_generic<<<grid_for(total), 256, 0, st>>>(d, Ho, Wo, A, Wq, Yacc, Y, sA, sW, bias, bias_stride, vec4, uns);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

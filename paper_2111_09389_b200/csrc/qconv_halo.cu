@@ -29,6 +29,7 @@ constexpr int kZeroBytes = 4096;          // >= 15 halo rows of at most 256 byte
 
 struct HaloParams {
     int mode;                  // 0 forward, 1 backward-data
+    int uns;                   // operands are unsigned 8-bit codes
     int nodes, B, Hm, Wm;      // output image of this pass
     int N;                     // output channels of this pass
     int ntaps, cpt, nslices;   // taps, 16-channel chunks per tap, K slices = taps * chunks (order: tap, chunk)
@@ -152,7 +153,7 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
         }
     } else if (warp == 1) {
         {
-            const uint32_t idesc = idesc_i8(128, p.N, 0, p.mode == 0 ? 0 : 1);
+            const uint32_t idesc = idesc_i8(128, p.N, 0, p.mode == 0 ? 0 : 1, p.uns);
             const uint32_t sbo_a = p.PW * 16;                       // next 8-pixel row group = next halo row
             const uint64_t a_fixed = ((uint64_t)((sbo_a >> 4) & 0x3FFFu) << 32) | ((uint64_t)1 << 46);
             const uint64_t b_tpl = (p.mode == 0) ? smem_desc(0, p.N * 16, 128, 0)
@@ -271,10 +272,10 @@ bool halo_supported(const lpdt_conv_desc &d, int mode) {
 
 lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, const float *s1, const int8_t *Wq,
                         const float *s2, const float *bias, int64_t bias_stride, float *Y, int32_t *Yacc,
-                        int32_t *dev_status, cudaStream_t st) {
+                        int32_t *dev_status, cudaStream_t st, bool uns) {
     const int Ho = conv_out(d.H, d.pad, d.R, 1), Wo = conv_out(d.W, d.pad, d.S, 1);
     HaloParams p = {};
-    p.mode = mode; p.nodes = d.nodes; p.B = d.B;
+    p.mode = mode; p.uns = uns ? 1 : 0; p.nodes = d.nodes; p.B = d.B;
     p.N = mode == 0 ? d.Cout : d.Cin;
     p.Hm = mode == 0 ? Ho : d.H; p.Wm = mode == 0 ? Wo : d.W;
     const int Ha = mode == 0 ? d.H : Ho, Wa = mode == 0 ? d.W : Wo;     // image of operand A

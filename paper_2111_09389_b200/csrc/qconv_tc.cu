@@ -51,6 +51,7 @@ struct TapTable {
 
 struct PixParams {
     int mode;                 // 0 forward, 1 backward-data
+    int uns;                  // operands are unsigned 8-bit codes
     int nodes, B, Hm, Wm;     // M-space grid of one class
     int Hout, Wout;           // full output image; output pixel = out_mul*m + class parity
     int out_mul, cmul;        // cmul scales tile origins into operand-A coordinates (forward stride)
@@ -190,7 +191,7 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         }
     } else if (warp == 1) {
         {
-            const uint32_t idesc = idesc_i8(128, p.BN, 0, p.mode == 0 ? 0 : 1);
+            const uint32_t idesc = idesc_i8(128, p.BN, 0, p.mode == 0 ? 0 : 1, p.uns);
             // Descriptor templates (start address 0); the loop only adds address increments.
             const uint64_t a_tpl = (p.RBa == 16) ? smem_desc(0, a_unit, 128, 0)
                                                  : smem_desc(0, 16, 8 * p.RBa, layout_code(p.RBa));
@@ -537,7 +538,7 @@ static int largest_div(int C, int cap, int unit) {      // largest multiple of u
 
 lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const float *s1, const int8_t *Wq,
                    const float *s2, const float *bias, int64_t bias_stride, float *Y, int32_t *Yacc,
-                   int32_t *dev_status, cudaStream_t st) {
+                   int32_t *dev_status, cudaStream_t st, bool uns) {
     const int Ho = conv_out(d.H, d.pad, d.R, d.stride), Wo = conv_out(d.W, d.pad, d.S, d.stride);
     PixParams p = {};
     p.mode = mode; p.nodes = d.nodes; p.B = d.B;
@@ -613,7 +614,7 @@ lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const flo
     p.tmem_cols = pow2_at_least(2 * p.BN);
     p.w_rows_per_node = d.Cout;
     p.Y = Y; p.Yacc = Yacc; p.s1 = s1; p.s2 = s2; p.bias = bias; p.bias_stride = bias_stride;
-    p.dev_status = dev_status;
+    p.dev_status = dev_status; p.uns = uns ? 1 : 0;
     CUtensorMap mA, mW;
     // operand A: activations (fwd: image H x W, Cin, sampled with the conv stride) or errors
     // (bwd-data: image Ho x Wo, Cout, dense)

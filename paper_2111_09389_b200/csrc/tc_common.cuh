@@ -171,10 +171,10 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes
     d |= (uint64_t)(layout_type & 7u) << 61;
     return d;
 }
-// Instruction descriptor for kind::i8: signed 8-bit A and B, int32 accumulator,
-// M x N tile, operand majors (0 = K-major, 1 = MN-major).
-__host__ __device__ constexpr uint32_t idesc_i8(int M, int N, int a_mn_major, int b_mn_major) {
-    return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+// Instruction descriptor for kind::i8: 8-bit A and B (both signed, or both unsigned when `uns`),
+// int32 accumulator, M x N tile, operand majors (0 = K-major, 1 = MN-major).
+__host__ __device__ constexpr uint32_t idesc_i8(int M, int N, int a_mn_major, int b_mn_major, int uns = 0) {
+    return (2u << 4) | ((uns ? 0u : 1u) << 7) | ((uns ? 0u : 1u) << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
            ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
 }
 

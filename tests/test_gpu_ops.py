@@ -165,6 +165,66 @@ def _conv_inputs(case, seed=0):
 
 
 @pytest.mark.parametrize("case", CONV_CASES)
+def test_qconv_fwd_affine(case):
+    """Zero-point operands (Section 3's scheme) on every forward shape: int32 sums bit-exact, fp32 as dequant_acc."""
+    nodes, B, H, W, Cin, Cout, R, S, stride, pad = case
+    rng = np.random.default_rng(77)
+    A = rng.integers(0, 256, (nodes, B, H, W, Cin), dtype=np.uint8)
+    Wq = rng.integers(0, 256, (nodes, Cout, R, S, Cin), dtype=np.uint8)
+    zA = rng.integers(0, 256, nodes).astype(np.int32)
+    zW = rng.integers(0, 256, nodes).astype(np.int32)
+    zA[0], zW[0] = 255, 0                                   # extreme zero points on one node
+    s1 = rng.uniform(0.001, 0.1, nodes).astype(np.float32)
+    s2 = rng.uniform(0.001, 0.1, nodes).astype(np.float32)
+    acc_ref, ovf = oracle.qconv_fwd_affine(A, zA, Wq, zW, stride, pad)
+    assert ovf == 0
+    desc = api.conv_desc(*case)
+    ws = ws_bytes(api.lpdt_qconv_fwd_affine_workspace_size(desc))
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    bias = rng.standard_normal((nodes, Cout)).astype(np.float32)
+    Y = torch.empty(acc_ref.shape, dtype=torch.float32, device="cuda")
+    Yacc = torch.empty(acc_ref.shape, dtype=torch.int32, device="cuda")
+    api.lpdt_qconv_fwd_affine(desc, dev(A), dev(s1), dev(zA), dev(Wq), dev(s2), dev(zW), Y=Y, Yacc=Yacc,
+                              bias=dev(bias), bias_node_stride=Cout, ws=ws, dev_status=status)
+    assert int(status.item()) == 0
+    assert np.array_equal(Yacc.cpu().numpy(), acc_ref)
+    assert np.array_equal(Y.cpu().numpy(), oracle.dequant_acc(acc_ref, s1, s2, bias))
+
+
+def test_qconv_fwd_affine_matches_quantizer_output():
+    # end to end with lpdt_quantize's affine mode: real 0 maps to the zero point, so a zero-padded real
+    # convolution of the dequantized tensors equals scale * acc
+    nodes, B, H, W, Cin, Cout = 2, 2, 10, 9, 16, 32
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((nodes, B, H, W, Cin)).astype(np.float32) + 0.7
+    w = rng.standard_normal((nodes, Cout, 3, 3, Cin)).astype(np.float32) * 0.1
+    qx, sx, zx = oracle.quantize_affine_u8(x.reshape(nodes, -1))
+    qw, sw, zw = oracle.quantize_affine_u8(w.reshape(nodes, -1))
+    A, Wq = qx.reshape(x.shape), qw.reshape(w.shape)
+    acc_ref, _ = oracle.qconv_fwd_affine(A, zx, Wq, zw, 1, 1)
+    desc = api.conv_desc(nodes, B, H, W, Cin, Cout, 3, 3, 1, 1)
+    Yacc = torch.empty(acc_ref.shape, dtype=torch.int32, device="cuda")
+    api.lpdt_qconv_fwd_affine(desc, dev(A), dev(sx), dev(zx.astype(np.int32)), dev(Wq), dev(sw), dev(zw.astype(np.int32)),
+                              Yacc=Yacc, ws=ws_bytes(api.lpdt_qconv_fwd_affine_workspace_size(desc)))
+    assert np.array_equal(Yacc.cpu().numpy(), acc_ref)
+
+
+def test_qconv_fwd_affine_errors():
+    desc = api.conv_desc(1, 1, 4, 4, 16, 16)
+    A = torch.zeros(1, 1, 4, 4, 16, dtype=torch.uint8, device="cuda")
+    Wq = torch.zeros(1, 16, 3, 3, 16, dtype=torch.uint8, device="cuda")
+    z = torch.zeros(1, dtype=torch.int32, device="cuda")
+    Yacc = torch.zeros(1, 1, 4, 4, 16, dtype=torch.int32, device="cuda")
+    with pytest.raises(api.LpdtError) as e:
+        api.lpdt_qconv_fwd_affine(desc, A, None, z, Wq, None, z, Yacc=Yacc, ws=ws_bytes(256))
+    assert e.value.code == 3                                 # workspace too small
+    with pytest.raises(api.LpdtError) as e:
+        api.lpdt_qconv_fwd_affine(desc, A, None, None, Wq, None, z, Yacc=Yacc,
+                                  ws=ws_bytes(api.lpdt_qconv_fwd_affine_workspace_size(desc)))
+    assert e.value.code == 1                                 # zero points missing
+
+
+@pytest.mark.parametrize("case", CONV_CASES)
 def test_qconv_all_three(case):
     nodes, B, H, W, Cin, Cout, R, S, stride, pad = case
     A, Wq, E, s1, s2 = _conv_inputs(case)
@@ -476,6 +536,6 @@ def test_qconv_cases_on_every_kernel_family(env):
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     child_env = dict(os.environ, LPDT_CHILD="1", **env)
     r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_ops.py"), "-m", "gpu",
-                        "-q", "-x", "-k", "test_qconv_all_three or test_qconv_extreme"], env=child_env, cwd=root,
+                        "-q", "-x", "-k", "test_qconv_all_three or test_qconv_extreme or test_qconv_fwd_affine"], env=child_env, cwd=root,
                        capture_output=True, text=True, timeout=900)
     assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]

@@ -77,3 +77,33 @@ def test_large_conv_three_passes(C, HW, batch):
     co = [0, C - 1]
     ref, _ = oracle.qconv_bwd_weight(np.ascontiguousarray(E[..., co].cpu().numpy()), A[..., :16].cpu().numpy().copy(), 3, 3, 1, 1)
     assert np.array_equal(dW[:, co][..., :16].cpu().numpy(), ref)
+
+
+@pytest.mark.parametrize("shape", [("gemm", 4096, 4096, 4096), ("conv", 256, 32, 64)])
+def test_large_affine_forward(shape):
+    """Zero-point operands at sweep sizes: sampled rows / images recomputed by the oracle (modulo 2^32: with
+    K up to 4096 the true sums stay inside int32)."""
+    g = torch.Generator(device="cuda"); g.manual_seed(9)
+    if shape[0] == "gemm":
+        _, M, N, K = shape
+        case = (1, M, 1, 1, K, N, 1, 1, 1, 0)
+    else:
+        _, Cc, HW, batch = shape
+        case = (1, batch, HW, HW, Cc, Cc, 3, 3, 1, 1)
+    nodes, B, H, W, Cin, Cout, R, S, stride, pad = case
+    desc = api.conv_desc(*case)
+    A = torch.randint(0, 256, (nodes, B, H, W, Cin), generator=g, device="cuda", dtype=torch.uint8)
+    Wq = torch.randint(0, 256, (nodes, Cout, R, S, Cin), generator=g, device="cuda", dtype=torch.uint8)
+    zA = torch.tensor([133], dtype=torch.int32, device="cuda")
+    zW = torch.tensor([121], dtype=torch.int32, device="cuda")
+    Y = torch.empty(nodes, B, H, W, Cout, dtype=torch.int32, device="cuda")
+    ws = torch.empty(api.lpdt_qconv_fwd_affine_workspace_size(desc), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    api.lpdt_qconv_fwd_affine(desc, A, None, zA, Wq, None, zW, Yacc=Y, ws=ws, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    rows = np.unique(np.concatenate([np.arange(2), np.random.default_rng(3).integers(0, B, 4), [B - 1]]))
+    ref, ovf = oracle.qconv_fwd_affine(A.cpu().numpy()[:, rows], zA.cpu().numpy(), Wq.cpu().numpy(), zW.cpu().numpy(),
+                                       stride, pad)
+    assert ovf == 0
+    assert np.array_equal(Y.cpu().numpy()[:, rows], ref)
