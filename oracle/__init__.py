@@ -225,6 +225,26 @@ def gossip_mix(x_half, x_hat, Wmix, gamma, seg_offsets=None, seg_k=None):
     return x_out, x_hat, q
 
 
+def gossip_mix_q8(x_half, x_hat, Wmix, gamma, seg_offsets=None, seg_k=None):
+    """Gossip step with 8-bit messages.  Returns (x_out, x_hat_new, q, codes int8 [n,d], scales fp32 [n,n_seg])."""
+    x_half = _c(x_half, np.float32)
+    x_hat = np.array(x_hat, dtype=np.float32, order="C", copy=True)
+    n, d = x_half.shape
+    Wm = _c(Wmix, np.float32)
+    if seg_offsets is None:
+        seg_offsets = [0, d]
+        seg_k = [d]
+    so = _c(seg_offsets, np.int64)
+    sk = _c(seg_k, np.int64)
+    x_out = np.zeros((n, d), np.float32)
+    q = np.zeros((n, d), np.float32)
+    codes = np.zeros((n, d), np.int8)
+    scales = np.zeros((n, len(sk)), np.float32)
+    lib().orc_gossip_mix_q8(C.c_int(n), _i64(d), _p(x_half), _p(x_hat), _p(x_out), _p(Wm),
+                            C.c_float(gamma), C.c_int(len(sk)), _p(so), _p(sk), _p(q), _p(codes), _p(scales))
+    return x_out, x_hat, q, codes, scales
+
+
 def sgd_update(x, g, lr):
     x = _c(x, np.float32); g = _c(g, np.float32)
     out = np.zeros(x.shape, np.float32)

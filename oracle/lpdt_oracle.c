@@ -425,6 +425,72 @@ void orc_gossip_mix(int nodes, i64 d, const float *x_half, float *x_hat, float *
     free(q);
 }
 
+/* The same gossip step with 8-bit messages (the contributions list and the Data column of
+ * the CIFAR table: quantized exchange is a quarter of the fp32 volume, alone or on top of
+ * top-k).  The paper gives no formula for the message; the reading taken: the compressed
+ * difference q is sent as signed 8-bit codes with one range per (node, segment), by the
+ * same symmetric quantizer as every other tensor:
+ *   amax = max |q| over the segment (the kept entries are the largest, so this is max |delta|),
+ *   scale = amax / 127, inv = 127 / amax (scale = 1 when amax = 0),
+ *   code = clamp(rne(delta * inv), -127, 127) on the kept entries, q = (float)code * scale,
+ * each operation rounded to fp32 on its own.  The public copy absorbs the DEQUANTIZED message,
+ * so sender and receivers hold the same x_hat and the rounding error stays in the next
+ * difference (error feedback).  codes_out (nullable) receives the codes (0 where nothing is
+ * sent), scale_out [nodes][n_seg] the scales. */
+void orc_gossip_mix_q8(int nodes, i64 d, const float *x_half, float *x_hat, float *x_out,
+                       const float *Wmix, float gamma, int n_seg, const i64 *seg_off,
+                       const i64 *seg_k, float *q_out, int8_t *codes_out, float *scale_out)
+{
+    float *q = (float *)calloc((size_t)nodes * (size_t)d, sizeof(float));
+    unsigned char *keep = (unsigned char *)calloc((size_t)d, 1);
+    mag_idx *tmp = (mag_idx *)malloc((size_t)d * sizeof(mag_idx));
+    if (codes_out) memset(codes_out, 0, (size_t)nodes * (size_t)d);
+    for (int i = 0; i < nodes; ++i) {
+        for (int s = 0; s < n_seg; ++s) {
+            i64 lo = seg_off[s], hi = seg_off[s + 1], len = hi - lo, k = seg_k[s];
+            if (k > len) k = len;
+            for (i64 e = lo; e < hi; ++e) {
+                float delta = x_half[i * d + e] - x_hat[i * d + e];
+                tmp[e - lo].mag = fabsf(delta);
+                tmp[e - lo].idx = e;
+                keep[e] = 0;
+            }
+            if (k < len) qsort(tmp, (size_t)len, sizeof(mag_idx), cmp_mag_desc);
+            float amax = 0.f;
+            for (i64 t = 0; t < k; ++t) {
+                keep[tmp[t].idx] = 1;
+                if (tmp[t].mag > amax) amax = tmp[t].mag;
+            }
+            float scale = 1.f, inv = 1.f;
+            if (amax > 0.f) { scale = amax / 127.0f; inv = 127.0f / amax; }
+            scale_out[(i64)i * n_seg + s] = scale;
+            for (i64 e = lo; e < hi; ++e) {
+                if (!keep[e]) continue;
+                float delta = x_half[i * d + e] - x_hat[i * d + e];
+                float t = delta * inv;
+                float r = rintf(t);                /* round half to even */
+                if (r > 127.f) r = 127.f;
+                if (r < -127.f) r = -127.f;
+                q[i * d + e] = r * scale;
+                if (codes_out) codes_out[i * d + e] = (int8_t)r;
+            }
+        }
+    }
+    for (i64 t = 0; t < (i64)nodes * d; ++t) x_hat[t] = x_hat[t] + q[t];
+    for (int i = 0; i < nodes; ++i)
+        for (i64 e = 0; e < d; ++e) {
+            double acc = 0.0;
+            for (int j = 0; j < nodes; ++j)
+                acc += (double)Wmix[i * nodes + j] *
+                       ((double)x_hat[j * d + e] - (double)x_hat[i * d + e]);
+            x_out[i * d + e] = (float)((double)x_half[i * d + e] + (double)gamma * acc);
+        }
+    if (q_out) memcpy(q_out, q, (size_t)nodes * (size_t)d * sizeof(float));
+    free(tmp);
+    free(keep);
+    free(q);
+}
+
 /* ------------------------------------------------------------------------
  * Glue around the layers of the step.
  * ---------------------------------------------------------------------- */

@@ -170,3 +170,69 @@ def test_softmax_ce():
 def test_colsum():
     x = np.arange(24, dtype=np.float32).reshape(2, 3, 4)
     assert np.array_equal(oracle.colsum(x), x.sum(1))
+
+
+# ---- 8-bit messages (the quantized exchange behind the Data column's factor of four) ----
+def test_q8_messages_on_the_grid_and_error_bound():
+    rng = np.random.default_rng(3)
+    n, d = 4, 3000
+    xh = rng.standard_normal((n, d)).astype(np.float32)
+    xhat = (xh - rng.standard_normal((n, d)) * rng.choice([1.0, 0.01], (n, d))).astype(np.float32)
+    so, sk = [0, 1000, 3000], [50, 2000]                    # second segment dense
+    x, xhat2, q, codes, scales = oracle.gossip_mix_q8(xh, xhat, ring(n), 0.4, so, sk)
+    delta = xh - xhat
+    for i in range(n):
+        for s, (lo, hi) in enumerate(zip(so[:-1], so[1:])):
+            k = min(sk[s], hi - lo)
+            kept = codes[i, lo:hi] != 0
+            sent = q[i, lo:hi] != 0
+            assert sent.sum() <= k and np.array_equal(kept, sent)
+            amax = np.abs(delta[i, lo:hi]).max()
+            assert scales[i, s] == np.float32(amax) / np.float32(127.0)          # one range per (node, segment)
+            assert np.abs(codes[i, lo:hi]).max() == 127                           # the largest entry maps to +-127
+            # the message is code*scale exactly, within half a step of the difference on the entries sent
+            assert np.array_equal(q[i, lo:hi], codes[i, lo:hi].astype(np.float32) * scales[i, s])
+            err = np.abs(q[i, lo:hi][sent].astype(np.float64) - delta[i, lo:hi][sent])
+            assert err.max() <= 0.5 * float(scales[i, s]) * (1 + 1e-6)
+            # selection is the fp32-message one: same support as top-k of |delta| (up to codes that round to 0)
+            _, _, q32 = oracle.gossip_mix(xh, xhat, ring(n), 0.4, so, sk)
+            assert not (sent & (q32[i, lo:hi] == 0)).any()
+    assert np.array_equal(xhat2, xhat + q)
+
+
+def test_q8_average_is_preserved_and_error_feedback():
+    # doubly-stochastic W: sum_i x_i = sum_i x_half_i for any public copies, quantized or not
+    rng = np.random.default_rng(4)
+    n, d = 6, 500
+    xh = rng.standard_normal((n, d)).astype(np.float32)
+    xhat = np.zeros((n, d), np.float32)
+    x, xhat2, q, codes, scales = oracle.gossip_mix_q8(xh, xhat, ring(n), 0.7, [0, d], [25])
+    np.testing.assert_allclose(x.sum(0, dtype=np.float64), xh.sum(0, dtype=np.float64), atol=1e-5)
+    # what was not sent (dropped entries and rounding) stays in the next difference
+    np.testing.assert_allclose((xh - xhat2).astype(np.float64), (xh - xhat).astype(np.float64) - q, atol=1e-6)
+
+
+def test_q8_exact_when_differences_sit_on_the_grid():
+    # differences that are integer multiples of amax/127 are sent without error: same result as fp32 messages
+    n, d = 3, 254
+    codes = np.tile(np.arange(-127, 127, dtype=np.float32), (n, 1))
+    codes[:, 0] = 127                                          # the range is set by an entry equal to amax
+    xh = (codes * np.float32(0.5)).astype(np.float32)          # amax = 63.5, scale = 0.5 exactly
+    xhat = np.zeros((n, d), np.float32)
+    x8, xhat8, q8, c8, s8 = oracle.gossip_mix_q8(xh, xhat, ring(n), 1.0)
+    x32, xhat32, q32 = oracle.gossip_mix(xh, xhat, ring(n), 1.0)
+    assert np.all(s8 == np.float32(0.5))
+    assert np.array_equal(q8, q32) and np.array_equal(xhat8, xhat32) and np.array_equal(x8, x32)
+    assert np.array_equal(c8, codes.astype(np.int8))
+
+
+def test_q8_hand_case_and_zero_difference():
+    # one node pair, d = 4: delta = [1.27, -0.635, 0.004, 0] -> scale 0.01, codes [127, -64 (63.5 -> even), 0, 0]
+    xh = np.array([[1.27, -0.635, 0.004, 0.0], [0, 0, 0, 0]], np.float32)
+    W = np.array([[0.5, 0.5], [0.5, 0.5]], np.float32)
+    x, xhat, q, codes, scales = oracle.gossip_mix_q8(xh, np.zeros_like(xh), W, 1.0)
+    assert codes[0].tolist()[0] == 127 and codes[0].tolist()[2:] == [0, 0] and codes[0, 1] in (-63, -64)
+    t = np.float32(-0.635) * (np.float32(127.0) / np.float32(1.27))
+    assert codes[0, 1] == int(np.rint(t))                     # ties resolved as rint does (half to even)
+    assert scales[1, 0] == 1.0 and not codes[1].any()         # all-zero difference: scale 1, nothing sent
+    np.testing.assert_allclose(x[1], 0.5 * xhat[0], rtol=1e-6)
