@@ -275,6 +275,22 @@ lpdt_status lpdt_gossip_mix(int32_t nodes, int64_t d, const float *x_half, float
                             int32_t n_segments, const int64_t *seg_offsets, const int64_t *seg_k,
                             void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
 
+/* The same step with 8-bit messages (the quantized exchange behind the factor of four
+ * in the Data column of the CIFAR table; the paper prints no formula, this is the reading
+ * taken): the compressed difference of each (node, segment) is sent as signed 8-bit codes
+ * with one range, by the symmetric quantizer of lpdt_quantize:
+ *   amax = max |x_half - x_hat| over the segment (0 if seg_k = 0),
+ *   scale = amax/127, inv = 127/amax (both 1 if amax = 0),
+ *   message_e = (float)clamp(rne((x_half_e - x_hat_e) * inv), -127, 127) * scale on the kept entries,
+ * and x_hat absorbs the dequantized message, so the rounding error stays in the next
+ * difference.  msg_scale : fp32 [nodes][n_segments], out (the step each node transmits).
+ * A node's message is k codes (+ k indices when k < segment length) + one scale.
+ * Everything else as lpdt_gossip_mix (same workspace size). */
+lpdt_status lpdt_gossip_mix_q8(int32_t nodes, int64_t d, const float *x_half, float *x_hat, float *x_out,
+                               const float *Wmix, float gamma, int32_t n_segments,
+                               const int64_t *seg_offsets, const int64_t *seg_k, float *msg_scale,
+                               void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
+
 /* ---------------------------------------------------------------------------
  * Glue around the layers of one training step.
  */

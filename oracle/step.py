@@ -149,14 +149,18 @@ def forward_backward(ops, params, x, labels=None, dy=None, eps=1e-5, grad_roundi
     return grads, loss, dict(input_grad=g)
 
 
-def train_step(wl, grad_rounding=0, seed=0, quantize_wgrad=False, keep=None):
-    """Whole step on a workload dict (see the workloads module).
-    Returns dict(grads, loss, x_half, x_hat, x, q)."""
+def train_step(wl, grad_rounding=0, seed=0, quantize_wgrad=False, keep=None, message_bits=32):
+    """Whole step on a workload dict (see the workloads module); message_bits = 8 sends the gossip
+    messages as 8-bit codes.  Returns dict(grads, loss, x_half, x_hat, x, q)."""
     grads, loss, extra = forward_backward(
         wl["ops"], wl["params"], wl["x"], wl.get("labels"), wl.get("dy"), wl["ren_eps"],
         grad_rounding, seed, quantize_wgrad, input_grad=("dy" in wl), keep=keep)
     x_half = orc.sgd_update(wl["params"], grads, wl["lr"])
-    x, x_hat, q = orc.gossip_mix(x_half, wl["x_hat"], wl["Wmix"], wl["gamma"],
-                                 wl["seg_offsets"], wl["seg_k"])
+    if message_bits == 8:
+        x, x_hat, q, _, _ = orc.gossip_mix_q8(x_half, wl["x_hat"], wl["Wmix"], wl["gamma"],
+                                              wl["seg_offsets"], wl["seg_k"])
+    else:
+        x, x_hat, q = orc.gossip_mix(x_half, wl["x_hat"], wl["Wmix"], wl["gamma"],
+                                     wl["seg_offsets"], wl["seg_k"])
     return dict(grads=grads, loss=loss, x_half=x_half, x_hat=x_hat, x=x, q=q,
                 input_grad=extra["input_grad"])

@@ -41,6 +41,7 @@ SIGNATURES = {
     "lpdt_range_evonorm_bwd": (_i32, [_i32] * 6 + [_f32] + [_vp] * 4 + [_i64] + [_vp] * 8 + [_i64, _vp, _vp, _sz, _vp]),
     "lpdt_gossip_mix_workspace_size": (_sz, [_i32, _i64, _i32]),
     "lpdt_gossip_mix": (_i32, [_i32, _i64, _vp, _vp, _vp, _vp, _f32, _i32, _vp, _vp, _vp, _sz, _vp, _vp]),
+    "lpdt_gossip_mix_q8": (_i32, [_i32, _i64, _vp, _vp, _vp, _vp, _f32, _i32, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
     "lpdt_sgd_update": (_i32, [_i64, _vp, _vp, _f32, _vp, _vp]),
     "lpdt_residual_add": (_i32, [_i32] * 8 + [_vp] * 5),
     "lpdt_residual_add_bwd": (_i32, [_i32] * 8 + [_vp] * 4),

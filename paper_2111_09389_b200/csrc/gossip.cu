@@ -319,11 +319,59 @@ __device__ void build_rows(const float *__restrict__ Wmix, int nodes, int32_t *_
     }
 }
 
+// 8-bit messages: max |x_half - x_hat| per (node, segment), as float bits through atomicMax (zeroed by
+// the launcher).  Block = one chunk of one node's parameters; a chunk may straddle segments.
+__global__ void __launch_bounds__(256)
+delta_amax_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d, SegTable seg,
+                  unsigned int *__restrict__ amax_bits) {
+    const int node = blockIdx.y;
+    const int64_t c0 = (int64_t)blockIdx.x * kChunk, c1 = (c0 + kChunk < d) ? c0 + kChunk : d;
+    const float *xh = x_half + (int64_t)node * d, *xq = x_hat + (int64_t)node * d;
+    int a = 0, b = seg.n_seg;
+    while (b - a > 1) { const int m = (a + b) >> 1; if (seg.off[m] <= c0) a = m; else b = m; }
+    __shared__ unsigned int s_m[8];
+    for (int s = a; s < seg.n_seg && seg.off[s] < c1; ++s) {
+        const int64_t lo = seg.off[s] > c0 ? seg.off[s] : c0, hi = seg.off[s + 1] < c1 ? seg.off[s + 1] : c1;
+        unsigned int m = 0;
+        for (int64_t e = lo + threadIdx.x; e < hi; e += blockDim.x) {
+            const unsigned int key = mag_bits(xh[e], xq[e]);
+            m = key > m ? key : m;
+        }
+        for (int o = 16; o > 0; o >>= 1) { const unsigned int t = __shfl_xor_sync(0xffffffffu, m, o); m = t > m ? t : m; }
+        if ((threadIdx.x & 31) == 0) s_m[threadIdx.x >> 5] = m;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            for (int w = 1; w < 8; ++w) m = s_m[w] > m ? s_m[w] : m;
+            if (m) atomicMax(amax_bits + (int64_t)node * seg.n_seg + s, m);
+        }
+        __syncthreads();
+    }
+}
+
+// The step of the symmetric 8-bit quantizer for each (node, segment) message and its reciprocal:
+// scale = amax/127, inv = 127/amax (1 and 1 when nothing is sent or everything is zero).
+__device__ void message_scales(const unsigned int *__restrict__ amax_bits, const SegTable &seg, int nodes,
+                               float *__restrict__ scale, float *__restrict__ inv) {
+    for (int i = threadIdx.x; i < nodes * seg.n_seg; i += blockDim.x) {
+        const float amax = seg.k[i % seg.n_seg] > 0 ? __uint_as_float(amax_bits[i]) : 0.f;
+        const bool live = amax > 0.f;
+        scale[i] = live ? __fdiv_rn(amax, 127.f) : 1.f;
+        inv[i] = live ? __fdiv_rn(127.f, amax) : 1.f;
+    }
+}
+
 __global__ void __launch_bounds__(1024)
 select_and_rows_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d,
                        SegTable seg, SelectOut *__restrict__ out, const float *__restrict__ Wmix, int nodes,
-                       int32_t *__restrict__ tab) {
-    if ((int)blockIdx.y == nodes) { if (blockIdx.x == 0) build_rows(Wmix, nodes, tab); return; }
+                       int32_t *__restrict__ tab, const unsigned int *__restrict__ amax_bits,
+                       float *__restrict__ msg_scale, float *__restrict__ msg_inv) {
+    if ((int)blockIdx.y == nodes) {
+        if (blockIdx.x == 0) {
+            build_rows(Wmix, nodes, tab);
+            if (amax_bits) message_scales(amax_bits, seg, nodes, msg_scale, msg_inv);
+        }
+        return;
+    }
     topk_select_body(x_half, x_hat, d, seg, out);
 }
 
@@ -331,11 +379,12 @@ select_and_rows_kernel(const float *__restrict__ x_half, const float *__restrict
 // owns V consecutive ones (16-byte accesses when V = 4).  Phase 1 streams x_half and x_hat of every
 // node, writes the updated public copy and parks it in shared memory; phase 2 mixes each node with
 // its neighbours' copies from shared memory (x_half is read again: an L1/L2 hit).
-template <int V>
+template <int V, bool Q8>
 __global__ void __launch_bounds__(256)
 gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float *__restrict__ x_hat,
                   float *__restrict__ x_out, float gamma, SegTable seg, const SelectOut *__restrict__ sel,
-                  const int32_t *__restrict__ tab) {
+                  const int32_t *__restrict__ tab, const float *__restrict__ msg_scale,
+                  const float *__restrict__ msg_inv) {
     extern __shared__ __align__(16) float sm[];
     const int TE = blockDim.x;
     int32_t *s_cnt = reinterpret_cast<int32_t *>(sm);            // [nodes]
@@ -373,17 +422,25 @@ gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float 
             for (int k = 0; k < V; ++k) hn[k] = 0.f;
             if (live) {
                 SelectOut so = sel[(int64_t)i * seg.n_seg + s0];
+                float q_scale = 1.f, q_inv = 1.f;
+                if (Q8) { q_scale = msg_scale[(int64_t)i * seg.n_seg + s0]; q_inv = msg_inv[(int64_t)i * seg.n_seg + s0]; }
 #pragma unroll
                 for (int k = 0; k < V; ++k) {
                     if (!one_seg && k > 0) {
                         int sk = s0;
                         while (seg.off[sk + 1] <= e0 + k) ++sk;
                         so = sel[(int64_t)i * seg.n_seg + sk];
+                        if (Q8) { q_scale = msg_scale[(int64_t)i * seg.n_seg + sk]; q_inv = msg_inv[(int64_t)i * seg.n_seg + sk]; }
                     }
                     const float delta = __fsub_rn(xh[u][k], xq[u][k]);
                     const uint32_t key = __float_as_uint(delta) & 0x7fffffffu;
                     const bool keep = so.dense || key > so.thr || (key == so.thr && e0 + k < so.cut);
-                    hn[k] = keep ? __fadd_rn(xq[u][k], delta) : xq[u][k];
+                    float msg = delta;
+                    if (Q8) {      // the message is the 8-bit code times the step; the public copy absorbs exactly that
+                        const float code = fminf(fmaxf(rintf(__fmul_rn(delta, q_inv)), -127.f), 127.f);
+                        msg = __fmul_rn(code, q_scale);
+                    }
+                    hn[k] = keep ? __fadd_rn(xq[u][k], msg) : xq[u][k];
                 }
                 VecIO<V>::st(x_hat + (int64_t)i * d + e0, hn);
             }
@@ -438,6 +495,10 @@ static int64_t max_big(int64_t d, int32_t n_segments) {
     return m < n_segments ? m : n_segments;
 }
 static int64_t max_chunks(int64_t d, int32_t n_segments) { return d / kChunk + max_big(d, n_segments); }
+// range words and reciprocal steps of the 8-bit messages, one per (node, segment) each (last in the workspace)
+static size_t q8_bytes(int32_t nodes, int32_t n_segments) {
+    return align_up((size_t)(nodes > 0 ? nodes : 1) * (size_t)(n_segments > 0 ? n_segments : 1) * sizeof(float), 256);
+}
 
 extern "C" size_t lpdt_gossip_mix_workspace_size(int32_t nodes, int64_t d, int32_t n_segments) {
     const size_t nn = (size_t)(nodes > 0 ? nodes : 1);
@@ -445,17 +506,17 @@ extern "C" size_t lpdt_gossip_mix_workspace_size(int32_t nodes, int64_t d, int32
     if (n_segments < 1) n_segments = 1;
     return select_bytes(nodes, n_segments) + rows_bytes(nodes) +
            align_up(nn * (size_t)max_big(d, n_segments) * (sizeof(BigHist) + sizeof(BigState)), 256) +
-           align_up(nn * (size_t)max_chunks(d, n_segments) * sizeof(uint32_t), 256);
+           align_up(nn * (size_t)max_chunks(d, n_segments) * sizeof(uint32_t), 256) + 2 * q8_bytes(nodes, n_segments);
 }
 
-extern "C" lpdt_status lpdt_gossip_mix(int32_t nodes, int64_t d, const float *x_half, float *x_hat,
-                                       float *x_out, const float *Wmix, float gamma, int32_t n_segments,
-                                       const int64_t *seg_offsets, const int64_t *seg_k, void *ws,
-                                       size_t ws_bytes, int32_t *dev_status, void *stream) {
+static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, float *x_hat,
+                               float *x_out, const float *Wmix, float gamma, int32_t n_segments,
+                               const int64_t *seg_offsets, const int64_t *seg_k, float *msg_scale, bool q8, void *ws,
+                               size_t ws_bytes, int32_t *dev_status, void *stream) {
     (void)dev_status;
     LPDT_CHECK_ARG(nodes >= 0 && d >= 0 && n_segments >= 1);
     if (nodes == 0 || d == 0) return LPDT_OK;
-    LPDT_CHECK_ARG(x_half && x_hat && x_out && Wmix && seg_offsets && seg_k);
+    LPDT_CHECK_ARG(x_half && x_hat && x_out && Wmix && seg_offsets && seg_k && (!q8 || msg_scale));
     LPDT_CHECK_ARG(x_hat != x_half && x_hat != x_out);
     if (nodes > kMaxNodes || n_segments > kMaxSeg) return LPDT_ERR_UNSUPPORTED;
     LPDT_CHECK_ARG(seg_offsets[0] == 0 && seg_offsets[n_segments] == d);
@@ -502,7 +563,19 @@ extern "C" lpdt_status lpdt_gossip_mix(int32_t nodes, int64_t d, const float *x_
         big_cut_kernel<<<dim3(big.n, nodes), 256, 0, st>>>(x_half, x_hat, d, seg, big, state, ties, total_chunks, sel);
         LPDT_LAUNCH_CHECK();
     }
-    select_and_rows_kernel<<<dim3(n_segments, nodes + 1), 1024, 0, st>>>(x_half, x_hat, d, seg, sel, Wmix, nodes, tab);
+    // 8-bit messages: ranges of the differences first (the kept entries are the largest of their segment)
+    unsigned int *amax_bits = nullptr;
+    float *msg_inv = nullptr;
+    if (q8) {
+        amax_bits = (unsigned int *)((char *)ws + lpdt_gossip_mix_workspace_size(nodes, d, n_segments) - 2 * q8_bytes(nodes, n_segments));
+        msg_inv = (float *)((char *)amax_bits + q8_bytes(nodes, n_segments));
+        if (nodes > 65535) return LPDT_ERR_UNSUPPORTED;
+        LPDT_CUDA(cudaMemsetAsync(amax_bits, 0, (size_t)nodes * n_segments * sizeof(unsigned int), st));
+        delta_amax_kernel<<<dim3((unsigned)ceil_div(d, (int64_t)kChunk), nodes), 256, 0, st>>>(x_half, x_hat, d, seg, amax_bits);
+        LPDT_LAUNCH_CHECK();
+    }
+    select_and_rows_kernel<<<dim3(n_segments, nodes + 1), 1024, 0, st>>>(x_half, x_hat, d, seg, sel, Wmix, nodes, tab,
+                                                                         amax_bits, msg_scale, msg_inv);
     LPDT_LAUNCH_CHECK();
     const bool v4 = d % 4 == 0 && aligned(x_half, 16) && aligned(x_hat, 16) && aligned(x_out, 16);
     const int V = v4 ? 4 : 1;
@@ -514,13 +587,36 @@ extern "C" lpdt_status lpdt_gossip_mix(int32_t nodes, int64_t d, const float *x_
     const size_t smem = tab_words * sizeof(int32_t) + (size_t)nodes * TE * V * sizeof(float);
     static bool attr_set = false;
     if (!attr_set) {
-        LPDT_CUDA(cudaFuncSetAttribute(gossip_mix_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
-        LPDT_CUDA(cudaFuncSetAttribute(gossip_mix_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
+        LPDT_CUDA(cudaFuncSetAttribute(gossip_mix_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
+        LPDT_CUDA(cudaFuncSetAttribute(gossip_mix_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
+        LPDT_CUDA(cudaFuncSetAttribute(gossip_mix_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
+        LPDT_CUDA(cudaFuncSetAttribute(gossip_mix_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
         attr_set = true;
     }
     const unsigned blocks = (unsigned)ceil_div(d, (int64_t)TE * V);
-    if (v4) gossip_mix_kernel<4><<<blocks, TE, smem, st>>>(nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab);
-    else gossip_mix_kernel<1><<<blocks, TE, smem, st>>>(nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab);
+    if (q8) {
+        if (v4) gossip_mix_kernel<4, true><<<blocks, TE, smem, st>>>(nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab, msg_scale, msg_inv);
+        else gossip_mix_kernel<1, true><<<blocks, TE, smem, st>>>(nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab, msg_scale, msg_inv);
+    } else {
+        if (v4) gossip_mix_kernel<4, false><<<blocks, TE, smem, st>>>(nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab, nullptr, nullptr);
+        else gossip_mix_kernel<1, false><<<blocks, TE, smem, st>>>(nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab, nullptr, nullptr);
+    }
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
+}
+
+extern "C" lpdt_status lpdt_gossip_mix(int32_t nodes, int64_t d, const float *x_half, float *x_hat,
+                                       float *x_out, const float *Wmix, float gamma, int32_t n_segments,
+                                       const int64_t *seg_offsets, const int64_t *seg_k, void *ws,
+                                       size_t ws_bytes, int32_t *dev_status, void *stream) {
+    return gossip_impl(nodes, d, x_half, x_hat, x_out, Wmix, gamma, n_segments, seg_offsets, seg_k, nullptr, false, ws,
+                       ws_bytes, dev_status, stream);
+}
+
+extern "C" lpdt_status lpdt_gossip_mix_q8(int32_t nodes, int64_t d, const float *x_half, float *x_hat,
+                                          float *x_out, const float *Wmix, float gamma, int32_t n_segments,
+                                          const int64_t *seg_offsets, const int64_t *seg_k, float *msg_scale,
+                                          void *ws, size_t ws_bytes, int32_t *dev_status, void *stream) {
+    return gossip_impl(nodes, d, x_half, x_hat, x_out, Wmix, gamma, n_segments, seg_offsets, seg_k, msg_scale, true, ws,
+                       ws_bytes, dev_status, stream);
 }

@@ -17,6 +17,8 @@ batch 128 so that each fp32 tensor is 268 MB; parameter kernels: 16 nodes with a
   sgd_update          12 B per parameter
   gossip_dense        x_half, x_hat read; x_hat, x written: 16 B per parameter
   gossip_top1pct      + one more pass over x_half and x_hat for the magnitude select: 24 B
+  gossip_dense_q8     8-bit messages: + one range pass over x_half and x_hat: 24 B
+  gossip_top1pct_q8   range pass + select pass + mix: 32 B
 
 One JSON line per case.
 """
@@ -96,6 +98,11 @@ def cases(nodes=8, B=128, H=32, W=32, Cc=64, d=32 * 270410, gossip_nodes=16):
     yield ("gossip_dense", lambda: api.lpdt_gossip_mix(N, d, xh, xhat, xo, Wm, 1.0, [0, d], [d], gws, st), N * d * 16)
     yield ("gossip_top1pct", lambda: api.lpdt_gossip_mix(N, d, xh, xhat, xo, Wm, 0.1, [0, d], [d // 100], gws, st),
            N * d * 24)
+    ms = torch.empty(N, 1, device="cuda")
+    yield ("gossip_dense_q8", lambda: api.lpdt_gossip_mix_q8(N, d, xh, xhat, xo, Wm, 1.0, [0, d], [d], ms, gws, st),
+           N * d * 24)
+    yield ("gossip_top1pct_q8", lambda: api.lpdt_gossip_mix_q8(N, d, xh, xhat, xo, Wm, 0.1, [0, d], [d // 100], ms, gws,
+                                                              st), N * d * 32)
 
 
 def sweep(iters=20, peak_gbs=None, out=print):

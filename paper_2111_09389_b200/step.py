@@ -17,7 +17,7 @@ from . import api
 class TrainStep:
     def __init__(self, ops, d, nodes, batch, in_shape, ren_eps=1e-5, lr=0.1, gamma=1.0,
                  seg_offsets=None, seg_k=None, has_labels=True, grad_rounding=0, seed=0,
-                 quantize_wgrad=False, input_grad=False, device="cuda"):
+                 quantize_wgrad=False, input_grad=False, message_bits=32, device="cuda"):
         if not torch.cuda.is_available():
             raise RuntimeError("TrainStep needs a CUDA device; there is no CPU path")
         self.ops, self.d, self.N, self.B = ops, d, nodes, batch
@@ -26,6 +26,7 @@ class TrainStep:
         self.seg_k = [d] if seg_k is None else [int(v) for v in seg_k]
         self.grad_rounding, self.seed = grad_rounding, seed
         self.quantize_wgrad, self.input_grad = quantize_wgrad, input_grad
+        self.message_bits = message_bits          # 8: gossip messages as 8-bit codes with one range per (node, segment)
         dev = torch.device(device)
         N, B = nodes, batch
         f32 = dict(dtype=torch.float32, device=dev)
@@ -41,6 +42,7 @@ class TrainStep:
         self.labels = torch.zeros(N, B, **i32) if has_labels else None
         self.loss = torch.zeros(N, **f32)
         self.dev_status = torch.zeros(1, **i32)
+        self.msg_scale = torch.zeros(N, len(self.seg_k), **f32)
         ws_bytes = max(api.lpdt_quantize_workspace_size(N),
                        api.lpdt_gossip_mix_workspace_size(N, d, len(self.seg_k)))
         self.buf = []
@@ -269,8 +271,12 @@ class TrainStep:
     def update(self):
         N, d = self.N, self.d
         api.lpdt_sgd_update(N * d, self.params, self.grads, self.lr, self.x_half)
-        api.lpdt_gossip_mix(N, d, self.x_half, self.x_hat, self.x_out, self.Wmix, self.gamma,
-                            self.seg_offsets, self.seg_k, self.ws, self.dev_status)
+        if self.message_bits == 8:
+            api.lpdt_gossip_mix_q8(N, d, self.x_half, self.x_hat, self.x_out, self.Wmix, self.gamma,
+                                   self.seg_offsets, self.seg_k, self.msg_scale, self.ws, self.dev_status)
+        else:
+            api.lpdt_gossip_mix(N, d, self.x_half, self.x_hat, self.x_out, self.Wmix, self.gamma,
+                                self.seg_offsets, self.seg_k, self.ws, self.dev_status)
 
     def run(self):
         self.forward()

@@ -466,6 +466,33 @@ def test_gossip_topk_ties_across_chunks():
         close(xo, x_ref)
 
 
+@pytest.mark.parametrize("nodes,d,segs", [
+    (4, 2736, None), (16, 10007, None), (8, 50000, [(0, 50000, 500)]),
+    (5, 3000, [(0, 1000, 10), (1000, 1001, 1), (1001, 3000, 1999)]), (3, 1000, [(0, 1000, 0)]),
+    (3, 100000, [(0, 100000, 1000)]), (2, 200000, [(0, 40000, 39999), (40000, 41000, 7), (41000, 200000, 1)]),
+])
+def test_gossip_mix_q8(nodes, d, segs):
+    """8-bit messages: public copies (hence the codes sent) bit-exact, mixed parameters within the fp32 bar,
+    transmitted steps equal; two steps in a row so that the rounding error is fed back."""
+    xh, xhat = _gossip_case(nodes, d, d, heavy=True)
+    W = wlmod.ring_matrix(nodes) if nodes >= 3 else np.full((nodes, nodes), 1.0 / nodes, np.float32)
+    so = [0, d] if segs is None else [s[0] for s in segs] + [d]
+    sk = [d] if segs is None else [s[2] for s in segs]
+    gamma = 1.0 if segs is None else 0.3
+    xhd, xhatd = dev(xh), dev(xhat)
+    ws = ws_bytes(api.lpdt_gossip_mix_workspace_size(nodes, d, len(sk)))
+    scale = torch.empty(nodes, len(sk), device="cuda")
+    x_in, xhat_ref = xh, xhat
+    for _ in range(2):
+        x_ref, xhat_ref, q_ref, codes_ref, scale_ref = oracle.gossip_mix_q8(x_in, xhat_ref, W, gamma, so, sk)
+        xo = torch.empty_like(xhd)
+        api.lpdt_gossip_mix_q8(nodes, d, dev(x_in), xhatd, xo, dev(W), gamma, so, sk, scale, ws)
+        assert np.array_equal(scale.cpu().numpy(), scale_ref)
+        assert np.array_equal(xhatd.cpu().numpy(), xhat_ref)
+        close(xo, x_ref)
+        x_in = x_ref
+
+
 def test_gossip_errors():
     t = torch.zeros(4, 8, device="cuda"); W = torch.zeros(4, 4, device="cuda")
     with pytest.raises(api.LpdtError) as e:

@@ -158,3 +158,23 @@ def test_resnet20_topk_40_nodes():
 
 def test_vgg11_8_nodes():
     _compare(wlmod.make_workload("vgg11", batch=4))
+
+
+@pytest.mark.parametrize("name,kw", [("conv16", {}), ("resnet20_topk", dict(nodes=5, batch=2))])
+def test_step_with_8bit_messages(name, kw):
+    """Whole step with the gossip messages sent as 8-bit codes.  The op itself is bit-exact on equal inputs
+    (test_gossip_mix_q8); here its input x_half carries the step's fp32-vs-fp64 summation differences, which may
+    move a difference across a rounding boundary: such entries differ by exactly one code step and must be rare."""
+    wl = wlmod.make_workload(name, **kw)
+    ref = ostep.train_step(wl, message_bits=8)
+    st = TrainStep.from_workload(wl, message_bits=8)
+    st.run()
+    torch.cuda.synchronize()
+    assert int(st.dev_status.item()) == 0
+    close(st.x_half, ref["x_half"], what="x_half")
+    step = st.msg_scale.cpu().numpy()[:, 0]                     # one segment in these workloads
+    for got, want, what in ((st.x_hat, ref["x_hat"], "x_hat"), (st.x_out, ref["x"], "x")):
+        err = np.abs(got.cpu().numpy().astype(np.float64) - want)
+        tight = err <= 1e-6 + 1e-5 * np.abs(want)
+        assert (err <= 1.001 * step[:, None] + 1e-6).all(), what        # never more than one code step (x: a mix of steps)
+        assert (~tight).mean() < 2e-3, f"{what}: {(~tight).sum()} entries off by a code step"
