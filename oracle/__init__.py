@@ -245,6 +245,25 @@ def gossip_mix_q8(x_half, x_hat, Wmix, gamma, seg_offsets=None, seg_k=None):
     return x_out, x_hat, q, codes, scales
 
 
+def deepsqueeze_mix(x_half, delta, Wmix, eta, seg_offsets=None, seg_k=None, bits=32):
+    """Deep-Squeeze gossip step.  Returns (x_out, delta_new, c, scales fp32 [n,n_seg])."""
+    x_half = _c(x_half, np.float32)
+    delta = np.array(delta, dtype=np.float32, order="C", copy=True)
+    n, d = x_half.shape
+    Wm = _c(Wmix, np.float32)
+    if seg_offsets is None:
+        seg_offsets = [0, d]
+        seg_k = [d]
+    so = _c(seg_offsets, np.int64)
+    sk = _c(seg_k, np.int64)
+    x_out = np.zeros((n, d), np.float32)
+    c = np.zeros((n, d), np.float32)
+    scales = np.zeros((n, len(sk)), np.float32)
+    lib().orc_deepsqueeze_mix(C.c_int(n), _i64(d), _p(x_half), _p(delta), _p(x_out), _p(Wm), C.c_float(eta),
+                              C.c_int(len(sk)), _p(so), _p(sk), C.c_int(bits), _p(c), _p(scales))
+    return x_out, delta, c, scales
+
+
 def sgd_update(x, g, lr):
     x = _c(x, np.float32); g = _c(g, np.float32)
     out = np.zeros(x.shape, np.float32)

@@ -491,6 +491,72 @@ void orc_gossip_mix_q8(int nodes, i64 d, const float *x_half, float *x_hat, floa
     free(q);
 }
 
+/* Deep-Squeeze gossip step (supplementary Algorithm 2, steps 5-10), all nodes at once:
+ *   v_i = x_half_i + delta_i                       (error compensated update)
+ *   c_i = C[v_i]: per segment the k entries of largest |v| (ties: lower index), the rest 0;
+ *         with 8-bit messages the kept entries go through the symmetric quantizer
+ *         (one range per node and segment), as in orc_gossip_mix_q8
+ *   delta_i <- v_i - c_i                           (what was not sent is carried over)
+ *   x_i = x_half_i + eta * sum_j (W_ij - I_ij) c_j = x_half_i + eta * (sum_j W_ij c_j - c_i)
+ * delta is updated in place; c_out (nullable) receives the messages, scale_out (nullable
+ * unless bits = 8) the quantizer steps.  fp32 elementwise steps, double for the mix sum. */
+void orc_deepsqueeze_mix(int nodes, i64 d, const float *x_half, float *delta, float *x_out,
+                         const float *Wmix, float eta, int n_seg, const i64 *seg_off,
+                         const i64 *seg_k, int bits, float *c_out, float *scale_out)
+{
+    float *c = (float *)calloc((size_t)nodes * (size_t)d, sizeof(float));
+    unsigned char *keep = (unsigned char *)calloc((size_t)d, 1);
+    mag_idx *tmp = (mag_idx *)malloc((size_t)d * sizeof(mag_idx));
+    for (int i = 0; i < nodes; ++i) {
+        for (int s = 0; s < n_seg; ++s) {
+            i64 lo = seg_off[s], hi = seg_off[s + 1], len = hi - lo, k = seg_k[s];
+            if (k > len) k = len;
+            for (i64 e = lo; e < hi; ++e) {
+                float v = x_half[i * d + e] + delta[i * d + e];
+                tmp[e - lo].mag = fabsf(v);
+                tmp[e - lo].idx = e;
+                keep[e] = 0;
+            }
+            if (k < len) qsort(tmp, (size_t)len, sizeof(mag_idx), cmp_mag_desc);
+            float amax = 0.f;
+            for (i64 t = 0; t < k; ++t) {
+                keep[tmp[t].idx] = 1;
+                if (tmp[t].mag > amax) amax = tmp[t].mag;
+            }
+            float scale = 1.f, inv = 1.f;
+            if (amax > 0.f) { scale = amax / 127.0f; inv = 127.0f / amax; }
+            if (scale_out) scale_out[(i64)i * n_seg + s] = scale;
+            for (i64 e = lo; e < hi; ++e) {
+                float v = x_half[i * d + e] + delta[i * d + e];
+                float msg = 0.f;
+                if (keep[e]) {
+                    msg = v;
+                    if (bits == 8) {
+                        float r = rintf(v * inv);
+                        if (r > 127.f) r = 127.f;
+                        if (r < -127.f) r = -127.f;
+                        msg = r * scale;
+                    }
+                }
+                c[i * d + e] = msg;
+                delta[i * d + e] = v - msg;
+            }
+        }
+    }
+    for (int i = 0; i < nodes; ++i)
+        for (i64 e = 0; e < d; ++e) {
+            double acc = 0.0;
+            for (int j = 0; j < nodes; ++j)
+                acc += (double)Wmix[i * nodes + j] * (double)c[j * d + e];
+            acc -= (double)c[i * d + e];
+            x_out[i * d + e] = (float)((double)x_half[i * d + e] + (double)eta * acc);
+        }
+    if (c_out) memcpy(c_out, c, (size_t)nodes * (size_t)d * sizeof(float));
+    free(tmp);
+    free(keep);
+    free(c);
+}
+
 /* ------------------------------------------------------------------------
  * Glue around the layers of the step.
  * ---------------------------------------------------------------------- */

@@ -236,3 +236,53 @@ def test_q8_hand_case_and_zero_difference():
     assert codes[0, 1] == int(np.rint(t))                     # ties resolved as rint does (half to even)
     assert scales[1, 0] == 1.0 and not codes[1].any()         # all-zero difference: scale 1, nothing sent
     np.testing.assert_allclose(x[1], 0.5 * xhat[0], rtol=1e-6)
+
+
+# ---- Deep-Squeeze mixing (supplementary Algorithm 2) ----
+def test_deepsqueeze_without_compression_is_plain_mixing():
+    # k = d, zero error buffer, eta = 1: x = x_half + (W x_half - x_half) = W x_half, a matrix product
+    rng = np.random.default_rng(7)
+    n, d = 5, 64
+    xh = rng.standard_normal((n, d)).astype(np.float32)
+    x, delta, c, _ = oracle.deepsqueeze_mix(xh, np.zeros((n, d), np.float32), ring(n), 1.0)
+    np.testing.assert_allclose(x, ring(n).astype(np.float64) @ xh.astype(np.float64), rtol=1e-6, atol=1e-6)
+    assert not delta.any() and np.array_equal(c, xh)
+
+
+@pytest.mark.parametrize("bits", [32, 8])
+def test_deepsqueeze_error_feedback_and_average(bits):
+    rng = np.random.default_rng(8)
+    n, d, k = 6, 400, 20
+    xh = rng.standard_normal((n, d)).astype(np.float32)
+    delta0 = (0.1 * rng.standard_normal((n, d))).astype(np.float32)
+    x, delta, c, scales = oracle.deepsqueeze_mix(xh, delta0, ring(n), 0.5, [0, d], [k], bits)
+    v = xh + delta0
+    assert all(np.count_nonzero(c[i]) <= k for i in range(n))
+    # what is sent plus what is carried over is the compensated update (v - c is exact or within an ulp)
+    np.testing.assert_allclose((c + delta).astype(np.float64), v.astype(np.float64), rtol=2e-7, atol=1e-7)
+    # the kept entries are the largest of |v|
+    for i in range(n):
+        sent = c[i] != 0
+        if bits == 32:
+            assert sent.sum() == k and np.array_equal(c[i][sent], v[i][sent])
+        assert np.abs(v[i][sent]).min() >= np.abs(v[i][~sent]).max() - 1e-7
+        if bits == 8:
+            codes = c[i][sent] / scales[i, 0]
+            assert np.allclose(codes, np.rint(codes)) and np.abs(codes).max() <= 127
+            assert scales[i, 0] == np.float32(np.abs(v[i]).max()) / np.float32(127.0)
+    # doubly-stochastic W: the node average moves only by the local updates
+    np.testing.assert_allclose(x.sum(0, dtype=np.float64), xh.sum(0, dtype=np.float64), atol=1e-5)
+
+
+def test_deepsqueeze_hand_case():
+    # ring of 4, d = 1, W = 1/3, k = 1 (everything sent), delta = [1, 0, 0, -1], x_half = [0, 3, 6, 9], eta = 1:
+    # v = c = [1, 3, 6, 8]; x_i = x_half_i + (c_{i-1} + c_i + c_{i+1})/3 - c_i
+    xh = np.array([[0.0], [3.0], [6.0], [9.0]], np.float32)
+    d0 = np.array([[1.0], [0.0], [0.0], [-1.0]], np.float32)
+    x, delta, c, _ = oracle.deepsqueeze_mix(xh, d0, ring(4), 1.0, [0, 1], [1])
+    assert c[:, 0].tolist() == [1.0, 3.0, 6.0, 8.0] and not delta.any()
+    want = [0 + (8 + 1 + 3) / 3 - 1, 3 + (1 + 3 + 6) / 3 - 3, 6 + (3 + 6 + 8) / 3 - 6, 9 + (6 + 8 + 1) / 3 - 8]
+    np.testing.assert_allclose(x[:, 0], want, rtol=1e-6)
+    # k = 0: nothing is sent, the whole compensated update is carried over and x = x_half
+    x, delta, c, _ = oracle.deepsqueeze_mix(xh, d0, ring(4), 1.0, [0, 1], [0])
+    assert not c.any() and np.array_equal(delta, xh + d0) and np.array_equal(x, xh)
