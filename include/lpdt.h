@@ -291,6 +291,21 @@ lpdt_status lpdt_gossip_mix_q8(int32_t nodes, int64_t d, const float *x_half, fl
                                const int64_t *seg_offsets, const int64_t *seg_k, float *msg_scale,
                                void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
 
+/* Deep-Squeeze gossip step (supplementary Algorithm 2, steps 5-10) for all nodes:
+ *   v_i = x_half_i + delta_i;  c_i = C[v_i];  delta_i <- v_i - c_i;
+ *   x_i = x_half_i + eta * (sum_j W_ij c_j - c_i)
+ * C keeps, per segment, the seg_k entries of largest |v| (ties: lower index); with
+ * message_bits = 8 the kept entries are sent as 8-bit codes (one range per node and
+ * segment, as in lpdt_gossip_mix_q8) and delta keeps the rounding error too.
+ * delta     : fp32 [nodes][d], in/out (the error buffer; zeros at the start of training)
+ * message_bits : 32 or 8;  msg_scale : fp32 [nodes][n_segments], out, required for 8 bits
+ * Everything else, the workspace size included, as lpdt_gossip_mix. */
+lpdt_status lpdt_deepsqueeze_mix(int32_t nodes, int64_t d, const float *x_half, float *delta, float *x_out,
+                                 const float *Wmix, float eta, int32_t n_segments,
+                                 const int64_t *seg_offsets, const int64_t *seg_k,
+                                 int32_t message_bits, float *msg_scale,
+                                 void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
+
 /* ---------------------------------------------------------------------------
  * Glue around the layers of one training step.
  */

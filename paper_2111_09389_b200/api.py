@@ -15,7 +15,7 @@ from ._lib import ConvDesc, lib
 KERNELS_PER_CALL = {
     "lpdt_quantize": 2, "lpdt_quantize_with_range": 1, "lpdt_quantize_static": 2, "lpdt_quantize_batch": 2, "lpdt_dequantize": 1, "lpdt_qconv_fwd": 1, "lpdt_qconv_fwd_affine": 4, "lpdt_qconv_bwd_data": 2,
     "lpdt_qconv_bwd_weight": 2, "lpdt_range_evonorm_fwd": 1, "lpdt_range_evonorm_bwd": 2,
-    "lpdt_gossip_mix": 2, "lpdt_gossip_mix_q8": 3, "lpdt_sgd_update": 1, "lpdt_residual_add": 1, "lpdt_residual_add_bwd": 1,
+    "lpdt_gossip_mix": 2, "lpdt_gossip_mix_q8": 3, "lpdt_deepsqueeze_mix": 2, "lpdt_sgd_update": 1, "lpdt_residual_add": 1, "lpdt_residual_add_bwd": 1,
     "lpdt_avgpool": 1, "lpdt_avgpool_bwd": 1, "lpdt_maxpool2x2": 1, "lpdt_maxpool2x2_bwd": 1,
     "lpdt_softmax_ce": 1, "lpdt_colsum": 1,
 }
@@ -224,6 +224,19 @@ def lpdt_gossip_mix_q8(nodes, d, x_half, x_hat, x_out, Wmix, gamma, seg_offsets,
     _check("lpdt_gossip_mix_q8", lib().lpdt_gossip_mix_q8(nodes, d, _ptr(x_half), _ptr(x_hat), _ptr(x_out),
                                                           _ptr(Wmix), gamma, ns, C.addressof(so), C.addressof(sk),
                                                           _ptr(msg_scale), p, nb, _ptr(dev_status), _stream()))
+
+
+def lpdt_deepsqueeze_mix(nodes, d, x_half, delta, x_out, Wmix, eta, seg_offsets, seg_k, ws, message_bits=32,
+                         msg_scale=None, dev_status=None):
+    """Deep-Squeeze gossip step; delta [nodes][d] is the error buffer (in/out)."""
+    ns = len(seg_k)
+    so = (C.c_int64 * (ns + 1))(*[int(v) for v in seg_offsets])
+    sk = (C.c_int64 * ns)(*[int(v) for v in seg_k])
+    p, nb = _ws(ws)
+    _check("lpdt_deepsqueeze_mix", lib().lpdt_deepsqueeze_mix(nodes, d, _ptr(x_half), _ptr(delta), _ptr(x_out),
+                                                              _ptr(Wmix), eta, ns, C.addressof(so), C.addressof(sk),
+                                                              message_bits, _ptr(msg_scale), p, nb, _ptr(dev_status),
+                                                              _stream()))
 
 
 def lpdt_sgd_update(n, x, g, lr, out):

@@ -13,6 +13,7 @@ constexpr int kMaxNodes = 64;
 
 struct SegTable {
     int32_t n_seg;
+    int32_t plus;            // 0: keys are |x_half - state| (CHOCO public copy); 1: |x_half + state| (Deep-Squeeze error buffer)
     int64_t off[kMaxSeg + 1];
     int64_t k[kMaxSeg];
 };
@@ -37,14 +38,14 @@ template <> struct VecIO<1> {
     static __device__ __forceinline__ void st(float *p, const float (&o)[1]) { *p = o[0]; }
 };
 
-__device__ __forceinline__ uint32_t mag_bits(float xh, float xhat) {
-    return __float_as_uint(__fsub_rn(xh, xhat)) & 0x7fffffffu;
+__device__ __forceinline__ uint32_t mag_bits(float xh, float state, int plus) {
+    return __float_as_uint(plus ? __fadd_rn(xh, state) : __fsub_rn(xh, state)) & 0x7fffffffu;
 }
 
 // Index just past the need-th key equal to thr in [lo, hi), walking in index order (whole CTA;
 // every thread returns the same value; -1 if there are fewer than need such keys).
 __device__ long long ordered_cut(const float *__restrict__ xh, const float *__restrict__ xq, int64_t lo, int64_t hi,
-                                 uint32_t thr, long long need) {
+                                 uint32_t thr, long long need, int plus) {
     __shared__ long long s_run, s_cut;
     __shared__ int warp_cnt[32];
     __syncthreads();
@@ -52,7 +53,7 @@ __device__ long long ordered_cut(const float *__restrict__ xh, const float *__re
     __syncthreads();
     for (int64_t base = lo; base < hi; base += blockDim.x) {
         const int64_t e = base + threadIdx.x;
-        const int flag = (e < hi) && (mag_bits(xh[e], xq[e]) == thr);
+        const int flag = (e < hi) && (mag_bits(xh[e], xq[e], plus) == thr);
         const int cnt = __syncthreads_count(flag);
         const long long run = s_run;
         if (run + cnt >= need) {
@@ -85,7 +86,7 @@ __device__ __host__ __forceinline__ bool is_big(int64_t len, int64_t k) { return
 // first, narrow the k-th largest key; a final ordered pass places the tie cut.
 __device__ __forceinline__ void topk_select_body(const float *__restrict__ x_half, const float *__restrict__ x_hat,
                                                  int64_t d, const SegTable &seg, SelectOut *__restrict__ out) {
-    const int s = blockIdx.x, node = blockIdx.y;
+    const int s = blockIdx.x, node = blockIdx.y, plus = seg.plus;
     const int64_t lo = seg.off[s], hi = seg.off[s + 1], len = hi - lo;
     const int64_t k = seg.k[s];
     SelectOut *o = out + (int64_t)node * seg.n_seg + s;
@@ -110,7 +111,7 @@ __device__ __forceinline__ void topk_select_body(const float *__restrict__ x_hal
         __syncthreads();
         const uint32_t prefix = s_prefix, mask = s_mask;
         for (int64_t e = lo + threadIdx.x; e < hi; e += blockDim.x) {
-            uint32_t key = mag_bits(xh[e], xq[e]);
+            uint32_t key = mag_bits(xh[e], xq[e], plus);
             if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
         }
         __syncthreads();
@@ -134,7 +135,7 @@ __device__ __forceinline__ void topk_select_body(const float *__restrict__ x_hal
         if (threadIdx.x == 0) { o->thr = thr; o->dense = 0; o->cut = hi; }
         return;
     }
-    const long long cut = ordered_cut(xh, xq, lo, hi, thr, need);
+    const long long cut = ordered_cut(xh, xq, lo, hi, thr, need, plus);
     if (threadIdx.x == 0) { o->thr = thr; o->dense = 0; o->cut = cut; }
 }
 
@@ -196,7 +197,7 @@ __global__ void __launch_bounds__(256)
 big_select_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d, SegTable seg,
                   BigList big, BigHist *__restrict__ hists, BigState *__restrict__ state,
                   uint32_t *__restrict__ tie_counts, int total_chunks, SelectOut *__restrict__ out) {
-    const int bi = blockIdx.y, node = blockIdx.z, s = big.id[bi];
+    const int bi = blockIdx.y, node = blockIdx.z, s = big.id[bi], plus = seg.plus;
     const int64_t lo = seg.off[s], hi = seg.off[s + 1];
     const int64_t c0 = lo + (int64_t)blockIdx.x * kChunk;
     if (c0 >= hi) return;
@@ -216,7 +217,7 @@ big_select_kernel(const float *__restrict__ x_half, const float *__restrict__ x_
             return;
         }
         int cnt = 0;
-        for (int64_t e = c0 + threadIdx.x; e < c1; e += blockDim.x) cnt += mag_bits(xh[e], xq[e]) == cur.prefix;
+        for (int64_t e = c0 + threadIdx.x; e < c1; e += blockDim.x) cnt += mag_bits(xh[e], xq[e], plus) == cur.prefix;
         __shared__ int s_cnt;
         if (threadIdx.x == 0) s_cnt = 0;
         __syncthreads();
@@ -242,7 +243,7 @@ big_select_kernel(const float *__restrict__ x_half, const float *__restrict__ x_
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
             if (e + u * blockDim.x < c1) {
-                const uint32_t key = mag_bits(a[u], b[u]);
+                const uint32_t key = mag_bits(a[u], b[u], plus);
                 if ((key & cur.mask) == cur.prefix) atomicAdd(&sh[(key >> kShift) & (kBins - 1)], 1u);
             }
         }
@@ -296,7 +297,7 @@ big_cut_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat
     const int64_t c0 = lo + (int64_t)s_chunk * kChunk;
     const int64_t c1 = (c0 + kChunk < hi) ? c0 + kChunk : hi;
     const long long cut = ordered_cut(x_half + (int64_t)node * d, x_hat + (int64_t)node * d, c0, c1, f.prefix,
-                                      f.need - s_before);
+                                      f.need - s_before, seg.plus);
     if (threadIdx.x == 0) {
         SelectOut so; so.thr = f.prefix; so.dense = 0; so.cut = cut;
         out[(int64_t)node * seg.n_seg + s] = so;
@@ -324,7 +325,7 @@ __device__ void build_rows(const float *__restrict__ Wmix, int nodes, int32_t *_
 __global__ void __launch_bounds__(256)
 delta_amax_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d, SegTable seg,
                   unsigned int *__restrict__ amax_bits) {
-    const int node = blockIdx.y;
+    const int node = blockIdx.y, plus = seg.plus;
     const int64_t c0 = (int64_t)blockIdx.x * kChunk, c1 = (c0 + kChunk < d) ? c0 + kChunk : d;
     const float *xh = x_half + (int64_t)node * d, *xq = x_hat + (int64_t)node * d;
     int a = 0, b = seg.n_seg;
@@ -334,7 +335,7 @@ delta_amax_kernel(const float *__restrict__ x_half, const float *__restrict__ x_
         const int64_t lo = seg.off[s] > c0 ? seg.off[s] : c0, hi = seg.off[s + 1] < c1 ? seg.off[s + 1] : c1;
         unsigned int m = 0;
         for (int64_t e = lo + threadIdx.x; e < hi; e += blockDim.x) {
-            const unsigned int key = mag_bits(xh[e], xq[e]);
+            const unsigned int key = mag_bits(xh[e], xq[e], plus);
             m = key > m ? key : m;
         }
         for (int o = 16; o > 0; o >>= 1) { const unsigned int t = __shfl_xor_sync(0xffffffffu, m, o); m = t > m ? t : m; }
@@ -379,7 +380,9 @@ select_and_rows_kernel(const float *__restrict__ x_half, const float *__restrict
 // owns V consecutive ones (16-byte accesses when V = 4).  Phase 1 streams x_half and x_hat of every
 // node, writes the updated public copy and parks it in shared memory; phase 2 mixes each node with
 // its neighbours' copies from shared memory (x_half is read again: an L1/L2 hit).
-template <int V, bool Q8>
+// DS: Deep-Squeeze form (supplementary Algorithm 2): the state array is the error buffer, the message is the
+// compressed x_half + state, the buffer keeps what was not sent and the mix runs over the messages themselves.
+template <int V, bool Q8, bool DS>
 __global__ void __launch_bounds__(256)
 gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float *__restrict__ x_hat,
                   float *__restrict__ x_out, float gamma, SegTable seg, const SelectOut *__restrict__ sel,
@@ -417,7 +420,7 @@ gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float 
         for (int u = 0; u < kU; ++u) {
             const int i = ib + u;
             if (i >= nodes) break;
-            float hn[V];
+            float hn[V], st_new[V];
 #pragma unroll
             for (int k = 0; k < V; ++k) hn[k] = 0.f;
             if (live) {
@@ -432,17 +435,23 @@ gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float 
                         so = sel[(int64_t)i * seg.n_seg + sk];
                         if (Q8) { q_scale = msg_scale[(int64_t)i * seg.n_seg + sk]; q_inv = msg_inv[(int64_t)i * seg.n_seg + sk]; }
                     }
-                    const float delta = __fsub_rn(xh[u][k], xq[u][k]);
+                    const float delta = DS ? __fadd_rn(xh[u][k], xq[u][k]) : __fsub_rn(xh[u][k], xq[u][k]);
                     const uint32_t key = __float_as_uint(delta) & 0x7fffffffu;
                     const bool keep = so.dense || key > so.thr || (key == so.thr && e0 + k < so.cut);
                     float msg = delta;
-                    if (Q8) {      // the message is the 8-bit code times the step; the public copy absorbs exactly that
+                    if (Q8) {      // the message is the 8-bit code times the step; the state absorbs exactly that
                         const float code = fminf(fmaxf(rintf(__fmul_rn(delta, q_inv)), -127.f), 127.f);
                         msg = __fmul_rn(code, q_scale);
                     }
-                    hn[k] = keep ? __fadd_rn(xq[u][k], msg) : xq[u][k];
+                    if (DS) {      // park the message, keep the remainder in the error buffer
+                        hn[k] = keep ? msg : 0.f;
+                        st_new[k] = __fsub_rn(delta, hn[k]);
+                    } else {       // public copy + message; that sum is also what the neighbours mix
+                        hn[k] = keep ? __fadd_rn(xq[u][k], msg) : xq[u][k];
+                        st_new[k] = hn[k];
+                    }
                 }
-                VecIO<V>::st(x_hat + (int64_t)i * d + e0, hn);
+                VecIO<V>::st(x_hat + (int64_t)i * d + e0, st_new);
             }
             VecIO<V>::st(s_hat + ((size_t)i * TE + threadIdx.x) * V, hn);
         }
@@ -469,7 +478,13 @@ gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float 
                 float hj[V];
                 VecIO<V>::ld(s_hat + ((size_t)j * TE + threadIdx.x) * V, hj);
 #pragma unroll
-                for (int k = 0; k < V; ++k) acc[k] = __fadd_rn(acc[k], __fmul_rn(w, __fsub_rn(hj[k], hi_[k])));
+                for (int k = 0; k < V; ++k)
+                    acc[k] = DS ? __fadd_rn(acc[k], __fmul_rn(w, hj[k]))                         // sum_j W_ij c_j
+                                : __fadd_rn(acc[k], __fmul_rn(w, __fsub_rn(hj[k], hi_[k])));      // sum_j W_ij (xhat_j - xhat_i)
+            }
+            if (DS) {
+#pragma unroll
+                for (int k = 0; k < V; ++k) acc[k] = __fsub_rn(acc[k], hi_[k]);                   // - I_ij c_j
             }
 #pragma unroll
             for (int k = 0; k < V; ++k) o[k] = __fadd_rn(xh[u][k], __fmul_rn(gamma, acc[k]));
@@ -511,8 +526,8 @@ extern "C" size_t lpdt_gossip_mix_workspace_size(int32_t nodes, int64_t d, int32
 
 static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, float *x_hat,
                                float *x_out, const float *Wmix, float gamma, int32_t n_segments,
-                               const int64_t *seg_offsets, const int64_t *seg_k, float *msg_scale, bool q8, void *ws,
-                               size_t ws_bytes, int32_t *dev_status, void *stream) {
+                               const int64_t *seg_offsets, const int64_t *seg_k, float *msg_scale, bool q8, bool ds,
+                               void *ws, size_t ws_bytes, int32_t *dev_status, void *stream) {
     (void)dev_status;
     LPDT_CHECK_ARG(nodes >= 0 && d >= 0 && n_segments >= 1);
     if (nodes == 0 || d == 0) return LPDT_OK;
@@ -522,6 +537,7 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
     LPDT_CHECK_ARG(seg_offsets[0] == 0 && seg_offsets[n_segments] == d);
     SegTable seg;
     seg.n_seg = n_segments;
+    seg.plus = ds ? 1 : 0;
     for (int s = 0; s < n_segments; ++s) {
         LPDT_CHECK_ARG(seg_offsets[s + 1] > seg_offsets[s] && seg_k[s] >= 0);
         seg.off[s] = seg_offsets[s];
@@ -585,22 +601,21 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
     if (TE < 32) TE = 32;
     const size_t tab_words = ((size_t)nodes + 2 * (size_t)nodes * nodes + 3) & ~(size_t)3;
     const size_t smem = tab_words * sizeof(int32_t) + (size_t)nodes * TE * V * sizeof(float);
+    using MixFn = void (*)(int, int64_t, const float *, float *, float *, float, SegTable, const SelectOut *,
+                           const int32_t *, const float *, const float *);
+    static const MixFn fns[8] = {
+        gossip_mix_kernel<1, false, false>, gossip_mix_kernel<4, false, false>, gossip_mix_kernel<1, true, false>,
+        gossip_mix_kernel<4, true, false>,  gossip_mix_kernel<1, false, true>,  gossip_mix_kernel<4, false, true>,
+        gossip_mix_kernel<1, true, true>,   gossip_mix_kernel<4, true, true>};
     static bool attr_set = false;
     if (!attr_set) {
-        LPDT_CUDA(cudaFuncSetAttribute(gossip_mix_kernel<4, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
-        LPDT_CUDA(cudaFuncSetAttribute(gossip_mix_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
-        LPDT_CUDA(cudaFuncSetAttribute(gossip_mix_kernel<4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
-        LPDT_CUDA(cudaFuncSetAttribute(gossip_mix_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
+        for (int i = 0; i < 8; ++i)
+            LPDT_CUDA(cudaFuncSetAttribute(fns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
         attr_set = true;
     }
     const unsigned blocks = (unsigned)ceil_div(d, (int64_t)TE * V);
-    if (q8) {
-        if (v4) gossip_mix_kernel<4, true><<<blocks, TE, smem, st>>>(nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab, msg_scale, msg_inv);
-        else gossip_mix_kernel<1, true><<<blocks, TE, smem, st>>>(nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab, msg_scale, msg_inv);
-    } else {
-        if (v4) gossip_mix_kernel<4, false><<<blocks, TE, smem, st>>>(nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab, nullptr, nullptr);
-        else gossip_mix_kernel<1, false><<<blocks, TE, smem, st>>>(nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab, nullptr, nullptr);
-    }
+    fns[(ds ? 4 : 0) + (q8 ? 2 : 0) + (v4 ? 1 : 0)]<<<blocks, TE, smem, st>>>(nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab,
+                                                                            q8 ? msg_scale : nullptr, msg_inv);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }
@@ -609,14 +624,24 @@ extern "C" lpdt_status lpdt_gossip_mix(int32_t nodes, int64_t d, const float *x_
                                        float *x_out, const float *Wmix, float gamma, int32_t n_segments,
                                        const int64_t *seg_offsets, const int64_t *seg_k, void *ws,
                                        size_t ws_bytes, int32_t *dev_status, void *stream) {
-    return gossip_impl(nodes, d, x_half, x_hat, x_out, Wmix, gamma, n_segments, seg_offsets, seg_k, nullptr, false, ws,
-                       ws_bytes, dev_status, stream);
+    return gossip_impl(nodes, d, x_half, x_hat, x_out, Wmix, gamma, n_segments, seg_offsets, seg_k, nullptr, false, false,
+                       ws, ws_bytes, dev_status, stream);
 }
 
 extern "C" lpdt_status lpdt_gossip_mix_q8(int32_t nodes, int64_t d, const float *x_half, float *x_hat,
                                           float *x_out, const float *Wmix, float gamma, int32_t n_segments,
                                           const int64_t *seg_offsets, const int64_t *seg_k, float *msg_scale,
                                           void *ws, size_t ws_bytes, int32_t *dev_status, void *stream) {
-    return gossip_impl(nodes, d, x_half, x_hat, x_out, Wmix, gamma, n_segments, seg_offsets, seg_k, msg_scale, true, ws,
-                       ws_bytes, dev_status, stream);
+    return gossip_impl(nodes, d, x_half, x_hat, x_out, Wmix, gamma, n_segments, seg_offsets, seg_k, msg_scale, true, false,
+                       ws, ws_bytes, dev_status, stream);
+}
+
+extern "C" lpdt_status lpdt_deepsqueeze_mix(int32_t nodes, int64_t d, const float *x_half, float *delta,
+                                            float *x_out, const float *Wmix, float eta, int32_t n_segments,
+                                            const int64_t *seg_offsets, const int64_t *seg_k, int32_t message_bits,
+                                            float *msg_scale, void *ws, size_t ws_bytes, int32_t *dev_status,
+                                            void *stream) {
+    LPDT_CHECK_ARG(message_bits == 32 || message_bits == 8);
+    return gossip_impl(nodes, d, x_half, delta, x_out, Wmix, eta, n_segments, seg_offsets, seg_k, msg_scale,
+                       message_bits == 8, true, ws, ws_bytes, dev_status, stream);
 }

@@ -493,6 +493,38 @@ def test_gossip_mix_q8(nodes, d, segs):
         x_in = x_ref
 
 
+@pytest.mark.parametrize("bits", [32, 8])
+@pytest.mark.parametrize("nodes,d,segs", [
+    (4, 2736, None), (16, 10007, [(0, 10007, 100)]), (8, 50000, [(0, 50000, 500)]),
+    (5, 3000, [(0, 1000, 10), (1000, 1001, 1), (1001, 3000, 1999)]), (3, 1000, [(0, 1000, 0)]),
+    (3, 100000, [(0, 100000, 1000)]),
+])
+def test_deepsqueeze_mix(nodes, d, segs, bits):
+    """Deep-Squeeze step: error buffer (hence the messages) bit-exact, mixed parameters within the fp32 bar;
+    three steps in a row so that the buffer is carried over."""
+    rng = np.random.default_rng(nodes * 1000 + d)
+    xh = rng.standard_normal((nodes, d)).astype(np.float32)
+    delta_ref = np.zeros((nodes, d), np.float32)
+    W = wlmod.ring_matrix(nodes) if nodes >= 3 else np.full((nodes, nodes), 1.0 / nodes, np.float32)
+    so = [0, d] if segs is None else [s[0] for s in segs] + [d]
+    sk = [d] if segs is None else [s[2] for s in segs]
+    eta = 1.0 if segs is None else 0.3
+    deltad = dev(delta_ref)
+    ws = ws_bytes(api.lpdt_gossip_mix_workspace_size(nodes, d, len(sk)))
+    scale = torch.empty(nodes, len(sk), device="cuda")
+    x_in = xh
+    for step in range(3):
+        x_ref, delta_ref, c_ref, scale_ref = oracle.deepsqueeze_mix(x_in, delta_ref, W, eta, so, sk, bits)
+        xo = torch.empty(nodes, d, device="cuda")
+        api.lpdt_deepsqueeze_mix(nodes, d, dev(x_in), deltad, xo, dev(W), eta, so, sk, ws, message_bits=bits,
+                                 msg_scale=scale if bits == 8 else None)
+        if bits == 8:
+            assert np.array_equal(scale.cpu().numpy(), scale_ref)
+        assert np.array_equal(deltad.cpu().numpy(), delta_ref), step
+        close(xo, x_ref)
+        x_in = (x_ref - 0.05 * rng.standard_normal((nodes, d))).astype(np.float32)      # a stand-in local update
+
+
 def test_gossip_errors():
     t = torch.zeros(4, 8, device="cuda"); W = torch.zeros(4, 4, device="cuda")
     with pytest.raises(api.LpdtError) as e:
