@@ -264,6 +264,16 @@ def deepsqueeze_mix(x_half, delta, Wmix, eta, seg_offsets=None, seg_k=None, bits
     return x_out, delta, c, scales
 
 
+def pushsum_debias(x, u, Wmix, eta):
+    """x fp32 [n,d], u fp32 [n].  Returns (u_new [n], z [n,d])."""
+    x = _c(x, np.float32); u = _c(u, np.float32); Wm = _c(Wmix, np.float32)
+    n, d = x.shape
+    u_new = np.zeros(n, np.float32)
+    z = np.zeros((n, d), np.float32)
+    lib().orc_pushsum_debias(C.c_int(n), _i64(d), _p(x), _p(u), _p(Wm), C.c_float(eta), _p(u_new), _p(z))
+    return u_new, z
+
+
 def sgd_update(x, g, lr):
     x = _c(x, np.float32); g = _c(g, np.float32)
     out = np.zeros(x.shape, np.float32)

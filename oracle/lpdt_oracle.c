@@ -557,6 +557,28 @@ void orc_deepsqueeze_mix(int nodes, i64 d, const float *x_half, float *delta, fl
     free(c);
 }
 
+/* Push-sum bias weights and de-biasing (supplementary Algorithms 4 and 5, the second line of
+ * step 9 and step 10), for column-stochastic mixing matrices on directed graphs:
+ *   u_new_i = u_i + eta * (sum_j W_ij u_j - u_i)        j ascending, fp32 steps
+ *   z_i = x_i / u_new_i                                  the model the next gradient is taken at
+ * x is the mixed model of the same step (from the Deep-Squeeze or CHOCO mix with the same W). */
+void orc_pushsum_debias(int nodes, i64 d, const float *x, const float *u, const float *Wmix,
+                        float eta, float *u_new, float *z)
+{
+    for (int i = 0; i < nodes; ++i) {
+        float acc = 0.f;
+        for (int j = 0; j < nodes; ++j) {
+            float t = Wmix[i * nodes + j] * u[j];
+            acc = acc + t;
+        }
+        acc = acc - u[i];
+        float step = eta * acc;
+        u_new[i] = u[i] + step;
+    }
+    for (int i = 0; i < nodes; ++i)
+        for (i64 e = 0; e < d; ++e) z[i * d + e] = x[i * d + e] / u_new[i];
+}
+
 /* ------------------------------------------------------------------------
  * Glue around the layers of the step.
  * ---------------------------------------------------------------------- */

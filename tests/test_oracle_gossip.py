@@ -286,3 +286,49 @@ def test_deepsqueeze_hand_case():
     # k = 0: nothing is sent, the whole compensated update is carried over and x = x_half
     x, delta, c, _ = oracle.deepsqueeze_mix(xh, d0, ring(4), 1.0, [0, 1], [0])
     assert not c.any() and np.array_equal(delta, xh + d0) and np.array_equal(x, xh)
+
+
+# ---- push-sum bias weights (supplementary Algorithms 4-5) ----
+def _column_stochastic(n, seed):
+    rng = np.random.default_rng(seed)
+    W = rng.random((n, n)) * (rng.random((n, n)) < 0.5)
+    W[np.arange(n), np.arange(n)] += 0.5                      # every node keeps part of its own mass
+    return (W / W.sum(0, keepdims=True)).astype(np.float32)   # columns sum to one: mass is conserved
+
+
+def test_pushsum_mass_conservation_and_debias():
+    n, d = 7, 33
+    W = _column_stochastic(n, 1)
+    rng = np.random.default_rng(2)
+    u = np.ones(n, np.float32)
+    x = rng.standard_normal((n, d)).astype(np.float32)
+    for _ in range(5):
+        u2, z = oracle.pushsum_debias(x, u, W, 1.0)
+        # eta = 1: u_new = W u, a matrix-vector product; column-stochastic W keeps sum(u) = n
+        np.testing.assert_allclose(u2, W.astype(np.float64) @ u.astype(np.float64), rtol=1e-6)
+        np.testing.assert_allclose(u2.sum(dtype=np.float64), n, rtol=1e-6)
+        np.testing.assert_allclose(z * u2[:, None], x, rtol=3e-7, atol=1e-30)     # z = x / u_new
+        u = u2
+    assert np.abs(u - 1).max() > 1e-3                         # a directed graph does move the weights
+
+
+def test_pushsum_trivial_on_doubly_stochastic_ring():
+    n, d = 6, 10
+    x = np.random.default_rng(3).standard_normal((n, d)).astype(np.float32)
+    u2, z = oracle.pushsum_debias(x, np.ones(n, np.float32), ring(n), 0.7)
+    np.testing.assert_allclose(u2, 1.0, rtol=1e-6)            # rows also sum to one: weights stay at 1
+    np.testing.assert_allclose(z, x, rtol=1e-6)
+
+
+def test_pushsum_average_consensus_through_debiasing():
+    # uncompressed push-sum gossip with zero gradients converges to the average of the initial models
+    # although W is only column-stochastic: x <- W x, u <- W u, z = x / u
+    n, d = 5, 4
+    W = _column_stochastic(n, 4)
+    x = np.random.default_rng(5).standard_normal((n, d)).astype(np.float32)
+    mean = x.mean(0, dtype=np.float64)
+    u = np.ones(n, np.float32)
+    for _ in range(200):
+        x, _, _, _ = oracle.deepsqueeze_mix(x, np.zeros_like(x), W, 1.0)        # k = d: x <- W x
+        u, z = oracle.pushsum_debias(x, u, W, 1.0)
+    np.testing.assert_allclose(z, np.tile(mean, (n, 1)), atol=1e-4)
