@@ -306,6 +306,20 @@ lpdt_status lpdt_deepsqueeze_mix(int32_t nodes, int64_t d, const float *x_half, 
                                  int32_t message_bits, float *msg_scale,
                                  void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
 
+/* Push-sum bias weights and de-biasing (supplementary Algorithms 4 and 5, Sparse-Push and
+ * Quant-SGP: second line of the gossip update, then the de-biasing step), for column-stochastic
+ * mixing matrices on directed graphs:
+ *   u_new_i = u_i + eta * (sum_j Wmix[i][j]*u_j - u_i)     (j ascending, each step rounded to fp32)
+ *   z_i     = x_i / u_new_i                                 (the model the next gradient is taken at)
+ * x is the mixed model of the same step: x_out of lpdt_deepsqueeze_mix (Sparse-Push) or of
+ * lpdt_gossip_mix / lpdt_gossip_mix_q8 (Quant-SGP) called with the same Wmix and eta.
+ * x, z : fp32 [nodes][d] (z may alias x);  u, u_new : fp32 [nodes], distinct arrays (u starts at 1);
+ * Wmix : fp32 [nodes][nodes] row-major, row i = the weights node i applies to what it receives.
+ * d = 0 updates the bias weights alone.  Errors: INVALID_ARG, UNSUPPORTED (nodes > 64), CUDA.
+ */
+lpdt_status lpdt_pushsum_debias(int32_t nodes, int64_t d, const float *x, const float *u, const float *Wmix,
+                                float eta, float *u_new, float *z, void *stream);
+
 /* ---------------------------------------------------------------------------
  * Glue around the layers of one training step.
  */

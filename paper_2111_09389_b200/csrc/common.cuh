@@ -2,6 +2,7 @@
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include "../../include/lpdt.h"
 
 #define LPDT_CHECK_ARG(cond)                       \
@@ -30,6 +31,36 @@ static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 constexpr int kNumSMs = 148;  // B200
+
+// Programmatic dependent launch.  Every kernel of the library waits for the grids before it
+// in the stream (griddepcontrol.wait returns once they have completed and their writes are
+// visible) before it touches global memory, and then allows the grid after it to be scheduled.
+// Launched through launch_k, a kernel's launch latency and its prologue (barrier set-up,
+// tensor-memory allocation, descriptor prefetch) overlap the tail of its predecessor; stream
+// order of every global access is unchanged.  LPDT_NO_PDL=1 launches without the attribute
+// (the instructions are then no-ops).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_enter() { pdl_wait(); pdl_trigger(); }
+
+static inline bool pdl_enabled() {
+    static int on = -1;
+    if (on < 0) { const char *e = getenv("LPDT_NO_PDL"); on = (e && e[0] == '1') ? 0 : 1; }
+    return on == 1;
+}
+
+template <typename... KArgs, typename... Args>
+static inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                   Args &&...args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<Args &&>(args)...);
+}
 
 // double atomicAdd is native on sm_60+
 __device__ __forceinline__ float warp_max(float v) {

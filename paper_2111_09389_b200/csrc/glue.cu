@@ -14,6 +14,7 @@ static inline unsigned grid1d(int64_t n, int threads = 256) {
 
 __global__ void sgd_kernel(int64_t n, const float *__restrict__ x, const float *__restrict__ g,
                            float lr, float *__restrict__ out) {
+    pdl_enter();
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
         out[i] = __fsub_rn(x[i], __fmul_rn(lr, g[i]));
 }
@@ -22,6 +23,7 @@ __global__ void sgd_kernel(int64_t n, const float *__restrict__ x, const float *
 __global__ void residual_add_kernel(int B, int H, int W, int Ca, int C, int stride, int ch_off,
                                     const float *__restrict__ r, const float *__restrict__ a,
                                     float *__restrict__ y, float *__restrict__ amax_out) {
+    pdl_enter();
     const int Ho = (H + stride - 1) / stride, Wo = (W + stride - 1) / stride;
     const int64_t per_node = (int64_t)B * Ho * Wo * C;
     const int64_t base = (int64_t)blockIdx.y * per_node;
@@ -47,6 +49,7 @@ __global__ void residual_add_kernel(int B, int H, int W, int Ca, int C, int stri
 __global__ void residual_add_v4_kernel(int B, int H, int W, int Ca4, int C4, int stride, int ch_off4,
                                        const float4 *__restrict__ r, const float4 *__restrict__ a,
                                        float4 *__restrict__ y, float *__restrict__ amax_out) {
+    pdl_enter();
     const int Ho = (H + stride - 1) / stride, Wo = (W + stride - 1) / stride;
     const long long per_node = (long long)B * Ho * Wo * C4;
     const long long base = (long long)blockIdx.y * per_node;
@@ -73,6 +76,7 @@ __global__ void residual_add_v4_kernel(int B, int H, int W, int Ca4, int C4, int
 __global__ void residual_add_bwd_v4_kernel(int NB, int H, int W, int Ca4, int C4, int stride, int ch_off4,
                                            const float4 *__restrict__ dy, const float4 *__restrict__ gm,
                                            float4 *__restrict__ da) {
+    pdl_enter();
     const int Ho = (H + stride - 1) / stride, Wo = (W + stride - 1) / stride;
     const long long total = (long long)NB * H * W * Ca4;
     for (long long o = (long long)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (long long)gridDim.x * blockDim.x) {
@@ -99,6 +103,7 @@ __global__ void residual_add_bwd_v4_kernel(int NB, int H, int W, int Ca4, int C4
 __global__ void residual_add_bwd_kernel(int64_t NB, int H, int W, int Ca, int C, int stride, int ch_off,
                                         const float *__restrict__ dy, const float *__restrict__ gm,
                                         float *__restrict__ da) {
+    pdl_enter();
     const int Ho = (H + stride - 1) / stride, Wo = (W + stride - 1) / stride;
     const int64_t total = NB * H * W * Ca;
     for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
@@ -115,6 +120,7 @@ __global__ void residual_add_bwd_kernel(int64_t NB, int H, int W, int Ca, int C,
 }
 
 __global__ void avgpool_kernel(int64_t NB, int HW, int C, const float *__restrict__ x, float *__restrict__ y) {
+    pdl_enter();
     int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= NB * C) return;
     int64_t nb = i / C; int c = (int)(i % C);
@@ -124,6 +130,7 @@ __global__ void avgpool_kernel(int64_t NB, int HW, int C, const float *__restric
 }
 
 __global__ void avgpool_bwd_kernel(int64_t NB, int HW, int C, const float *__restrict__ dy, float *__restrict__ dx) {
+    pdl_enter();
     const int64_t total = NB * HW * C;
     const float fhw = (float)HW;
     for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
@@ -135,6 +142,7 @@ __global__ void avgpool_bwd_kernel(int64_t NB, int HW, int C, const float *__res
 
 __global__ void maxpool_kernel(int64_t NB, int H, int W, int C, const float *__restrict__ x,
                                float *__restrict__ y, int8_t *__restrict__ idx) {
+    pdl_enter();
     const int Ho = H / 2, Wo = W / 2;
     const int64_t total = NB * Ho * Wo * C;
     for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
@@ -155,6 +163,7 @@ __global__ void maxpool_kernel(int64_t NB, int H, int W, int C, const float *__r
 
 __global__ void maxpool_bwd_kernel(int64_t NB, int H, int W, int C, const float *__restrict__ dy,
                                    const int8_t *__restrict__ idx, float *__restrict__ dx) {
+    pdl_enter();
     const int Ho = H / 2, Wo = W / 2;
     const int64_t total = NB * H * W * C;
     for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
@@ -173,6 +182,7 @@ __global__ void maxpool_bwd_kernel(int64_t NB, int H, int W, int C, const float 
 // index decode per four elements.
 __global__ void maxpool_v4_kernel(int64_t NB, int H, int W, int C4, const float4 *__restrict__ x,
                                   float4 *__restrict__ y, char4 *__restrict__ idx) {
+    pdl_enter();
     const int Ho = H / 2, Wo = W / 2;
     const int64_t total = NB * Ho * Wo * C4;
     for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
@@ -195,6 +205,7 @@ __global__ void maxpool_v4_kernel(int64_t NB, int H, int W, int C4, const float4
 
 __global__ void maxpool_bwd_v4_kernel(int64_t NB, int H, int W, int C4, const float4 *__restrict__ dy,
                                       const char4 *__restrict__ idx, float4 *__restrict__ dx) {
+    pdl_enter();
     const int Ho = H / 2, Wo = W / 2;
     const int64_t total = NB * H * W * C4;
     for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
@@ -215,6 +226,7 @@ __global__ void maxpool_bwd_v4_kernel(int64_t NB, int H, int W, int C4, const fl
 __global__ void softmax_ce_kernel(int B, int K, const float *__restrict__ logits,
                                   const int32_t *__restrict__ labels, float *__restrict__ loss,
                                   float *__restrict__ dlogits) {
+    pdl_enter();
     extern __shared__ double s_part[];
     const int n = blockIdx.x;
     double mine = 0.0;
@@ -243,6 +255,7 @@ __global__ void softmax_ce_kernel(int B, int K, const float *__restrict__ logits
 
 __global__ void colsum_kernel(int nodes, int B, int C, const float *__restrict__ x,
                               float *__restrict__ out, int64_t ostride) {
+    pdl_enter();
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= nodes * C) return;
     int n = i / C, c = i % C;
@@ -260,7 +273,7 @@ extern "C" lpdt_status lpdt_sgd_update(int64_t n, const float *x, const float *g
     LPDT_CHECK_ARG(n >= 0);
     if (n == 0) return LPDT_OK;
     LPDT_CHECK_ARG(x && g && out);
-    sgd_kernel<<<grid1d(n), 256, 0, as_stream(stream)>>>(n, x, g, lr, out);
+    launch_k(sgd_kernel, grid1d(n), 256, 0, as_stream(stream), n, x, g, lr, out);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }
@@ -279,10 +292,10 @@ extern "C" lpdt_status lpdt_residual_add(int32_t nodes, int32_t B, int32_t H, in
         return (unsigned)(b < 1 ? 1 : (b > cap ? cap : b));
     };
     if (C % 4 == 0 && Ca % 4 == 0 && ch_off % 4 == 0 && aligned(r, 16) && aligned(a, 16) && aligned(y, 16))
-        residual_add_v4_kernel<<<dim3(gx(per_node / 4), nodes), 256, 0, as_stream(stream)>>>(
+        launch_k(residual_add_v4_kernel, dim3(gx(per_node / 4), nodes), 256, 0, as_stream(stream), 
             B, H, W, Ca / 4, C / 4, stride, ch_off / 4, (const float4 *)r, (const float4 *)a, (float4 *)y, amax_out);
     else
-        residual_add_kernel<<<dim3(gx(per_node), nodes), 256, 0, as_stream(stream)>>>(
+        launch_k(residual_add_kernel, dim3(gx(per_node), nodes), 256, 0, as_stream(stream), 
             B, H, W, Ca, C, stride, ch_off, r, a, y, amax_out);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
@@ -297,10 +310,10 @@ extern "C" lpdt_status lpdt_residual_add_bwd(int32_t nodes, int32_t B, int32_t H
     LPDT_CHECK_ARG(dy && g_main && da);
     if (C % 4 == 0 && Ca % 4 == 0 && ch_off % 4 == 0 && aligned(dy, 16) && aligned(g_main, 16) && aligned(da, 16) &&
         (int64_t)nodes * B < 0x7fffffff)
-        residual_add_bwd_v4_kernel<<<grid1d((int64_t)nodes * B * H * W * Ca / 4), 256, 0, as_stream(stream)>>>(
+        launch_k(residual_add_bwd_v4_kernel, grid1d((int64_t)nodes * B * H * W * Ca / 4), 256, 0, as_stream(stream), 
             nodes * B, H, W, Ca / 4, C / 4, stride, ch_off / 4, (const float4 *)dy, (const float4 *)g_main, (float4 *)da);
     else
-    residual_add_bwd_kernel<<<grid1d((int64_t)nodes * B * H * W * Ca), 256, 0, as_stream(stream)>>>(
+    launch_k(residual_add_bwd_kernel, grid1d((int64_t)nodes * B * H * W * Ca), 256, 0, as_stream(stream), 
         (int64_t)nodes * B, H, W, Ca, C, stride, ch_off, dy, g_main, da);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
@@ -312,7 +325,7 @@ extern "C" lpdt_status lpdt_avgpool(int32_t nodes, int32_t B, int32_t HW, int32_
     if (nodes == 0 || B == 0) return LPDT_OK;
     LPDT_CHECK_ARG(x && y);
     int64_t n = (int64_t)nodes * B * C;
-    avgpool_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, as_stream(stream)>>>((int64_t)nodes * B, HW, C, x, y);
+    launch_k(avgpool_kernel, (unsigned)ceil_div(n, 256), 256, 0, as_stream(stream), (int64_t)nodes * B, HW, C, x, y);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }
@@ -322,7 +335,7 @@ extern "C" lpdt_status lpdt_avgpool_bwd(int32_t nodes, int32_t B, int32_t HW, in
     LPDT_CHECK_ARG(nodes >= 0 && B >= 0 && HW > 0 && C > 0);
     if (nodes == 0 || B == 0) return LPDT_OK;
     LPDT_CHECK_ARG(dy && dx);
-    avgpool_bwd_kernel<<<grid1d((int64_t)nodes * B * HW * C), 256, 0, as_stream(stream)>>>(
+    launch_k(avgpool_bwd_kernel, grid1d((int64_t)nodes * B * HW * C), 256, 0, as_stream(stream), 
         (int64_t)nodes * B, HW, C, dy, dx);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
@@ -334,11 +347,11 @@ extern "C" lpdt_status lpdt_maxpool2x2(int32_t nodes, int32_t B, int32_t H, int3
     if (nodes == 0 || B == 0) return LPDT_OK;
     LPDT_CHECK_ARG(x && y && idx);
     if (C % 4 == 0 && aligned(x, 16) && aligned(y, 16) && aligned(idx, 4))
-        maxpool_v4_kernel<<<grid1d((int64_t)nodes * B * (H / 2) * (W / 2) * (C / 4)), 256, 0, as_stream(stream)>>>(
+        launch_k(maxpool_v4_kernel, grid1d((int64_t)nodes * B * (H / 2) * (W / 2) * (C / 4)), 256, 0, as_stream(stream), 
             (int64_t)nodes * B, H, W, C / 4, reinterpret_cast<const float4 *>(x), reinterpret_cast<float4 *>(y),
             reinterpret_cast<char4 *>(idx));
     else
-        maxpool_kernel<<<grid1d((int64_t)nodes * B * (H / 2) * (W / 2) * C), 256, 0, as_stream(stream)>>>(
+        launch_k(maxpool_kernel, grid1d((int64_t)nodes * B * (H / 2) * (W / 2) * C), 256, 0, as_stream(stream), 
             (int64_t)nodes * B, H, W, C, x, y, idx);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
@@ -350,11 +363,11 @@ extern "C" lpdt_status lpdt_maxpool2x2_bwd(int32_t nodes, int32_t B, int32_t H, 
     if (nodes == 0 || B == 0) return LPDT_OK;
     LPDT_CHECK_ARG(dy && idx && dx);
     if (C % 4 == 0 && aligned(dx, 16) && aligned(dy, 16) && aligned(idx, 4))
-        maxpool_bwd_v4_kernel<<<grid1d((int64_t)nodes * B * H * W * (C / 4)), 256, 0, as_stream(stream)>>>(
+        launch_k(maxpool_bwd_v4_kernel, grid1d((int64_t)nodes * B * H * W * (C / 4)), 256, 0, as_stream(stream), 
             (int64_t)nodes * B, H, W, C / 4, reinterpret_cast<const float4 *>(dy), reinterpret_cast<const char4 *>(idx),
             reinterpret_cast<float4 *>(dx));
     else
-        maxpool_bwd_kernel<<<grid1d((int64_t)nodes * B * H * W * C), 256, 0, as_stream(stream)>>>(
+        launch_k(maxpool_bwd_kernel, grid1d((int64_t)nodes * B * H * W * C), 256, 0, as_stream(stream), 
             (int64_t)nodes * B, H, W, C, dy, idx, dx);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
@@ -367,7 +380,7 @@ extern "C" lpdt_status lpdt_softmax_ce(int32_t nodes, int32_t B, int32_t K, cons
     LPDT_CHECK_ARG(logits && labels && loss && dlogits);
     int threads = 32;
     while (threads < B && threads < 256) threads <<= 1;
-    softmax_ce_kernel<<<nodes, threads, threads * sizeof(double), as_stream(stream)>>>(B, K, logits, labels,
+    launch_k(softmax_ce_kernel, nodes, threads, threads * sizeof(double), as_stream(stream), B, K, logits, labels,
                                                                                      loss, dlogits);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
@@ -378,7 +391,7 @@ extern "C" lpdt_status lpdt_colsum(int32_t nodes, int32_t B, int32_t C, const fl
     LPDT_CHECK_ARG(nodes >= 0 && B >= 0 && C > 0);
     if (nodes == 0) return LPDT_OK;
     LPDT_CHECK_ARG(x && out && (out_node_stride >= C || nodes == 1));
-    colsum_kernel<<<(nodes * C + 255) / 256, 256, 0, as_stream(stream)>>>(nodes, B, C, x, out, out_node_stride);
+    launch_k(colsum_kernel, (nodes * C + 255) / 256, 256, 0, as_stream(stream), nodes, B, C, x, out, out_node_stride);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

@@ -197,6 +197,7 @@ __global__ void __launch_bounds__(256)
 big_select_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d, SegTable seg,
                   BigList big, BigHist *__restrict__ hists, BigState *__restrict__ state,
                   uint32_t *__restrict__ tie_counts, int total_chunks, SelectOut *__restrict__ out) {
+    pdl_enter();
     const int bi = blockIdx.y, node = blockIdx.z, s = big.id[bi], plus = seg.plus;
     const int64_t lo = seg.off[s], hi = seg.off[s + 1];
     const int64_t c0 = lo + (int64_t)blockIdx.x * kChunk;
@@ -277,6 +278,7 @@ __global__ void __launch_bounds__(256)
 big_cut_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d, SegTable seg,
                BigList big, const BigState *__restrict__ state, const uint32_t *__restrict__ tie_counts,
                int total_chunks, SelectOut *__restrict__ out) {
+    pdl_enter();
     const int bi = blockIdx.x, node = blockIdx.y, s = big.id[bi];
     const BigState f = state[(int64_t)node * big.n + bi];
     if (f.eq == f.need) return;
@@ -325,6 +327,7 @@ __device__ void build_rows(const float *__restrict__ Wmix, int nodes, int32_t *_
 __global__ void __launch_bounds__(256)
 delta_amax_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d, SegTable seg,
                   unsigned int *__restrict__ amax_bits) {
+    pdl_enter();
     const int node = blockIdx.y, plus = seg.plus;
     const int64_t c0 = (int64_t)blockIdx.x * kChunk, c1 = (c0 + kChunk < d) ? c0 + kChunk : d;
     const float *xh = x_half + (int64_t)node * d, *xq = x_hat + (int64_t)node * d;
@@ -366,6 +369,7 @@ select_and_rows_kernel(const float *__restrict__ x_half, const float *__restrict
                        SegTable seg, SelectOut *__restrict__ out, const float *__restrict__ Wmix, int nodes,
                        int32_t *__restrict__ tab, const unsigned int *__restrict__ amax_bits,
                        float *__restrict__ msg_scale, float *__restrict__ msg_inv) {
+    pdl_enter();
     if ((int)blockIdx.y == nodes) {
         if (blockIdx.x == 0) {
             build_rows(Wmix, nodes, tab);
@@ -388,6 +392,7 @@ gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float 
                   float *__restrict__ x_out, float gamma, SegTable seg, const SelectOut *__restrict__ sel,
                   const int32_t *__restrict__ tab, const float *__restrict__ msg_scale,
                   const float *__restrict__ msg_inv) {
+    pdl_enter();
     extern __shared__ __align__(16) float sm[];
     const int TE = blockDim.x;
     int32_t *s_cnt = reinterpret_cast<int32_t *>(sm);            // [nodes]
@@ -493,6 +498,49 @@ gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float 
     }
 }
 
+// Push-sum bias weights and de-biased model (supplementary Algorithms 4 and 5: second half of the gossip
+// update, then the de-biasing step).  Grid (chunks, nodes); every CTA recomputes its node's new bias
+// weight (one row of W times u: at most 64 multiply-adds, j ascending, by one thread) and then streams
+// z = x / u_new over its chunk (4 B read + 4 B write per parameter).
+template <int V>
+__global__ void __launch_bounds__(256)
+pushsum_debias_kernel(int nodes, int64_t d, const float *__restrict__ x, const float *__restrict__ u,
+                      const float *__restrict__ Wmix, float eta, float *__restrict__ u_new, float *__restrict__ z) {
+    pdl_enter();
+    const int node = blockIdx.y;
+    __shared__ float s_u;
+    if (threadIdx.x == 0) {
+        float acc = 0.f;
+        for (int j = 0; j < nodes; ++j) acc = __fadd_rn(acc, __fmul_rn(Wmix[node * nodes + j], u[j]));
+        acc = __fsub_rn(acc, u[node]);
+        const float un = __fadd_rn(u[node], __fmul_rn(eta, acc));
+        s_u = un;
+        if (blockIdx.x == 0) u_new[node] = un;
+    }
+    __syncthreads();
+    const float un = s_u;
+    const float *xr = x + (int64_t)node * d;
+    float *zr = z + (int64_t)node * d;
+    constexpr int kU = 4;                                        // independent loads per thread
+    const int64_t per_block = (int64_t)blockDim.x * V * kU;
+    const int64_t b0 = (int64_t)blockIdx.x * per_block;
+    float v[kU][V];
+#pragma unroll
+    for (int q = 0; q < kU; ++q) {
+        const int64_t e = b0 + ((int64_t)q * blockDim.x + threadIdx.x) * V;
+        if (e < d) VecIO<V>::ld(xr + e, v[q]);
+    }
+#pragma unroll
+    for (int q = 0; q < kU; ++q) {
+        const int64_t e = b0 + ((int64_t)q * blockDim.x + threadIdx.x) * V;
+        if (e < d) {
+#pragma unroll
+            for (int k = 0; k < V; ++k) v[q][k] = __fdiv_rn(v[q][k], un);
+            VecIO<V>::st(zr + e, v[q]);
+        }
+    }
+}
+
 }  // namespace lpdt
 
 using namespace lpdt;
@@ -571,12 +619,12 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
         const int total_chunks = big.chunk_base[big.n];
         LPDT_CUDA(cudaMemsetAsync(hists, 0, (size_t)nodes * big.n * sizeof(BigHist), st));
         const dim3 g((unsigned)most_chunks, big.n, nodes);
-        big_select_kernel<0><<<g, 256, 0, st>>>(x_half, x_hat, d, seg, big, hists, state, ties, total_chunks, sel);
-        big_select_kernel<1><<<g, 256, 0, st>>>(x_half, x_hat, d, seg, big, hists, state, ties, total_chunks, sel);
-        big_select_kernel<2><<<g, 256, 0, st>>>(x_half, x_hat, d, seg, big, hists, state, ties, total_chunks, sel);
-        big_select_kernel<3><<<g, 256, 0, st>>>(x_half, x_hat, d, seg, big, hists, state, ties, total_chunks, sel);
+        launch_k(big_select_kernel<0>, g, 256, 0, st, x_half, x_hat, d, seg, big, hists, state, ties, total_chunks, sel);
+        launch_k(big_select_kernel<1>, g, 256, 0, st, x_half, x_hat, d, seg, big, hists, state, ties, total_chunks, sel);
+        launch_k(big_select_kernel<2>, g, 256, 0, st, x_half, x_hat, d, seg, big, hists, state, ties, total_chunks, sel);
+        launch_k(big_select_kernel<3>, g, 256, 0, st, x_half, x_hat, d, seg, big, hists, state, ties, total_chunks, sel);
         LPDT_LAUNCH_CHECK();
-        big_cut_kernel<<<dim3(big.n, nodes), 256, 0, st>>>(x_half, x_hat, d, seg, big, state, ties, total_chunks, sel);
+        launch_k(big_cut_kernel, dim3(big.n, nodes), 256, 0, st, x_half, x_hat, d, seg, big, state, ties, total_chunks, sel);
         LPDT_LAUNCH_CHECK();
     }
     // 8-bit messages: ranges of the differences first (the kept entries are the largest of their segment)
@@ -587,10 +635,10 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
         msg_inv = (float *)((char *)amax_bits + q8_bytes(nodes, n_segments));
         if (nodes > 65535) return LPDT_ERR_UNSUPPORTED;
         LPDT_CUDA(cudaMemsetAsync(amax_bits, 0, (size_t)nodes * n_segments * sizeof(unsigned int), st));
-        delta_amax_kernel<<<dim3((unsigned)ceil_div(d, (int64_t)kChunk), nodes), 256, 0, st>>>(x_half, x_hat, d, seg, amax_bits);
+        launch_k(delta_amax_kernel, dim3((unsigned)ceil_div(d, (int64_t)kChunk), nodes), 256, 0, st, x_half, x_hat, d, seg, amax_bits);
         LPDT_LAUNCH_CHECK();
     }
-    select_and_rows_kernel<<<dim3(n_segments, nodes + 1), 1024, 0, st>>>(x_half, x_hat, d, seg, sel, Wmix, nodes, tab,
+    launch_k(select_and_rows_kernel, dim3(n_segments, nodes + 1), 1024, 0, st, x_half, x_hat, d, seg, sel, Wmix, nodes, tab,
                                                                          amax_bits, msg_scale, msg_inv);
     LPDT_LAUNCH_CHECK();
     const bool v4 = d % 4 == 0 && aligned(x_half, 16) && aligned(x_hat, 16) && aligned(x_out, 16);
@@ -614,7 +662,7 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
         attr_set = true;
     }
     const unsigned blocks = (unsigned)ceil_div(d, (int64_t)TE * V);
-    fns[(ds ? 4 : 0) + (q8 ? 2 : 0) + (v4 ? 1 : 0)]<<<blocks, TE, smem, st>>>(nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab,
+    launch_k(fns[(ds ? 4 : 0) + (q8 ? 2 : 0) + (v4 ? 1 : 0)], blocks, TE, smem, st, nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab,
                                                                             q8 ? msg_scale : nullptr, msg_inv);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
@@ -644,4 +692,23 @@ extern "C" lpdt_status lpdt_deepsqueeze_mix(int32_t nodes, int64_t d, const floa
     LPDT_CHECK_ARG(message_bits == 32 || message_bits == 8);
     return gossip_impl(nodes, d, x_half, delta, x_out, Wmix, eta, n_segments, seg_offsets, seg_k, msg_scale,
                        message_bits == 8, true, ws, ws_bytes, dev_status, stream);
+}
+
+extern "C" lpdt_status lpdt_pushsum_debias(int32_t nodes, int64_t d, const float *x, const float *u, const float *Wmix,
+                                           float eta, float *u_new, float *z, void *stream) {
+    LPDT_CHECK_ARG(nodes >= 0 && d >= 0);
+    if (nodes == 0) return LPDT_OK;
+    LPDT_CHECK_ARG(u && Wmix && u_new && u_new != u && (d == 0 || (x && z)));
+    if (nodes > kMaxNodes) return LPDT_ERR_UNSUPPORTED;
+    cudaStream_t st = as_stream(stream);
+    const bool v4 = d % 4 == 0 && aligned(x, 16) && aligned(z, 16);
+    const int64_t per_block = 256 * 4 * (v4 ? 4 : 1);
+    int64_t chunks = ceil_div(d, per_block);
+    if (chunks < 1) chunks = 1;                                  // d = 0: the bias weights alone
+    if (chunks > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
+    const dim3 g((unsigned)chunks, nodes);
+    if (v4) launch_k(pushsum_debias_kernel<4>, g, 256, 0, st, nodes, d, x, u, Wmix, eta, u_new, z);
+    else launch_k(pushsum_debias_kernel<1>, g, 256, 0, st, nodes, d, x, u, Wmix, eta, u_new, z);
+    LPDT_LAUNCH_CHECK();
+    return LPDT_OK;
 }

@@ -16,6 +16,7 @@ namespace lpdt {
 // destination row (Cp is a multiple of 16), written with a single 16-byte store.
 __global__ void pad_channels_kernel(const int8_t *__restrict__ src, int8_t *__restrict__ dst, int64_t rows,
                                     int C, int Cp) {
+    pdl_enter();
     const int pieces = Cp / 16;
     const int64_t total = rows * pieces;
     for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
@@ -118,9 +119,9 @@ static lpdt_status fwd_impl(const lpdt_conv_desc *d, const int8_t *A, const floa
         const PadPlan pp = pad_plan(*d);
         int8_t *Ap = (int8_t *)ws, *Wp = Ap + pp.a_bytes;
         const int64_t arows = (int64_t)d->nodes * d->B * d->H * d->W, wrows = (int64_t)d->nodes * d->Cout * d->R * d->S;
-        pad_channels_kernel<<<grid_for(arows * dp.Cin / 16), 256, 0, st>>>(A, Ap, arows, d->Cin, dp.Cin);
+        launch_k(pad_channels_kernel, grid_for(arows * dp.Cin / 16), 256, 0, st, A, Ap, arows, d->Cin, dp.Cin);
         LPDT_LAUNCH_CHECK();
-        pad_channels_kernel<<<grid_for(wrows * dp.Cin / 16), 256, 0, st>>>(Wq, Wp, wrows, d->Cin, dp.Cin);
+        launch_k(pad_channels_kernel, grid_for(wrows * dp.Cin / 16), 256, 0, st, Wq, Wp, wrows, d->Cin, dp.Cin);
         LPDT_LAUNCH_CHECK();
         return run_pix(dp, 0, Ap, sA, Wp, sW, bias, bias_node_stride, Y, Yacc, dev_status, st, uns);
     }
@@ -154,6 +155,7 @@ namespace lpdt {
 // 32, chosen by the launcher from the row length) shares a row: 16-byte loads when the rows allow.
 __global__ void row_sum_u8_kernel(const uint8_t *__restrict__ src, int64_t rows, int len, int G, bool vec16,
                                   int32_t *__restrict__ out) {
+    pdl_enter();
     const int lane_in_group = threadIdx.x & (G - 1);
     const int64_t groups_total = ((int64_t)gridDim.x * blockDim.x) / G;
     for (int64_t row = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / G;; row += groups_total) {
@@ -181,6 +183,7 @@ __global__ void row_sum_u8_kernel(const uint8_t *__restrict__ src, int64_t rows,
 // channel is the fastest index, so the correction pass reads four neighbours with one 16-byte load.
 __global__ void weight_prefix_kernel(const int32_t *__restrict__ tapsum, int nodes, int Cout, int R, int S,
                                      int32_t *__restrict__ P) {
+    pdl_enter();
     const int row = blockIdx.x * blockDim.x + threadIdx.x;        // (node, co)
     if (row >= nodes * Cout) return;
     const int n = row / Cout, co = row % Cout, PS = S + 1;
@@ -206,6 +209,7 @@ __global__ void affine_fix_kernel(lpdt_conv_desc d, int Ho, int Wo, const int32_
                                   const float *__restrict__ sA, const float *__restrict__ sW,
                                   const float *__restrict__ bias, int64_t bias_stride, float *__restrict__ Y,
                                   int32_t *__restrict__ Yacc) {
+    pdl_enter();
     const int chunks = d.Cout / V;
     const int64_t total = (int64_t)d.nodes * d.B * Ho * Wo * chunks;
     for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
@@ -276,7 +280,7 @@ static lpdt_status row_sum_launch(const uint8_t *src, int64_t rows, int len, int
     const int64_t cap = (int64_t)kNumSMs * 32;
     if (blocks > cap) blocks = cap;
     if (blocks < 1) blocks = 1;
-    row_sum_u8_kernel<<<(unsigned)blocks, 256, 0, st>>>(src, rows, len, G, vec16, out);
+    launch_k(row_sum_u8_kernel, (unsigned)blocks, 256, 0, st, src, rows, len, G, vec16, out);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }
@@ -328,15 +332,15 @@ extern "C" lpdt_status lpdt_qconv_fwd_affine(const lpdt_conv_desc *d, const uint
     int32_t *tapsum = (int32_t *)((char *)P + align_up((size_t)rows * (d->R + 1) * (d->S + 1) * sizeof(int32_t), 256));
     s = row_sum_launch(Wq, (int64_t)rows * d->R * d->S, d->Cin, tapsum, st);
     if (s != LPDT_OK) return s;
-    weight_prefix_kernel<<<(rows + 127) / 128, 128, 0, st>>>(tapsum, d->nodes, d->Cout, d->R, d->S, P);
+    launch_k(weight_prefix_kernel, (rows + 127) / 128, 128, 0, st, tapsum, d->nodes, d->Cout, d->R, d->S, P);
     LPDT_LAUNCH_CHECK();
     const bool v4 = d->Cout % 4 == 0 && (!Y || aligned(Y, 16)) && (!Yacc || aligned(Yacc, 16));
     const int64_t work = (int64_t)d->nodes * d->B * Ho * Wo * (d->Cout / (v4 ? 4 : 1));
     if (v4)
-        affine_fix_kernel<4><<<grid_for(work), 256, 0, st>>>(*d, Ho, Wo, raw, asum, P, zA, zW, sA, sW, bias,
+        launch_k(affine_fix_kernel<4>, grid_for(work), 256, 0, st, *d, Ho, Wo, raw, asum, P, zA, zW, sA, sW, bias,
                                                              bias_node_stride, Y, Yacc);
     else
-        affine_fix_kernel<1><<<grid_for(work), 256, 0, st>>>(*d, Ho, Wo, raw, asum, P, zA, zW, sA, sW, bias,
+        launch_k(affine_fix_kernel<1>, grid_for(work), 256, 0, st, *d, Ho, Wo, raw, asum, P, zA, zW, sA, sW, bias,
                                                              bias_node_stride, Y, Yacc);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
@@ -378,7 +382,7 @@ extern "C" lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8
     } else if (use_tc_padded(*d, &dp) && d->B > 0 && aligned(E, 16)) {
         int8_t *Ap = (int8_t *)((char *)ws + acc_bytes);
         const int64_t arows = (int64_t)d->nodes * d->B * d->H * d->W;
-        pad_channels_kernel<<<grid_for(arows * dp.Cin / 16), 256, 0, st>>>(A, Ap, arows, d->Cin, dp.Cin);
+        launch_k(pad_channels_kernel, grid_for(arows * dp.Cin / 16), 256, 0, st, A, Ap, arows, d->Cin, dp.Cin);
         LPDT_LAUNCH_CHECK();
         lpdt_status r = tc::tc_wgrad(dp, d->Cin, E, sE, Ap, sA, dWacc, acc_ws, dW, dw_node_stride, dev_status, st);
         if (r != LPDT_ERR_UNSUPPORTED) return r;

@@ -39,6 +39,7 @@ __global__ void conv_fwd_generic(lpdt_conv_desc d, int Ho, int Wo, const int8_t 
                                  float *__restrict__ Y, const float *__restrict__ s1,
                                  const float *__restrict__ s2, const float *__restrict__ bias,
                                  int64_t bias_stride, bool vec4, bool uns) {
+    pdl_enter();
     const int64_t per_node = (int64_t)d.B * Ho * Wo * d.Cout;
     const int64_t total = per_node * d.nodes;
     for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
@@ -73,6 +74,7 @@ __global__ void conv_fwd_generic(lpdt_conv_desc d, int Ho, int Wo, const int8_t 
 // Wt[n][ci][r][s][co] = W[n][co][r][s][ci]
 __global__ void transpose_weights_kernel(lpdt_conv_desc d, const int8_t *__restrict__ Wq,
                                          int8_t *__restrict__ Wt) {
+    pdl_enter();
     const int64_t per_node = (int64_t)d.Cout * d.R * d.S * d.Cin;
     const int64_t total = per_node * d.nodes;
     for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
@@ -91,6 +93,7 @@ __global__ void conv_bwd_data_generic(lpdt_conv_desc d, int Ho, int Wo, const in
                                       const int8_t *__restrict__ Wt, int32_t *__restrict__ acc_out,
                                       float *__restrict__ dA, const float *__restrict__ s1,
                                       const float *__restrict__ s2, bool vec4) {
+    pdl_enter();
     const int64_t per_node = (int64_t)d.B * d.H * d.W * d.Cin;
     const int64_t total = per_node * d.nodes;
     for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
@@ -126,6 +129,7 @@ __global__ void conv_bwd_data_generic(lpdt_conv_desc d, int Ho, int Wo, const in
 __global__ void conv_bwd_weight_generic(lpdt_conv_desc d, int Ho, int Wo, int chunk,
                                         const int8_t *__restrict__ E, const int8_t *__restrict__ A,
                                         int32_t *__restrict__ acc_out) {
+    pdl_enter();
     const int n = blockIdx.y;
     const int64_t npix = (int64_t)d.B * Ho * Wo;
     const int64_t p0 = (int64_t)blockIdx.x * chunk;
@@ -155,6 +159,7 @@ __global__ void conv_bwd_weight_generic(lpdt_conv_desc d, int Ho, int Wo, int ch
 __global__ void dequant_acc_kernel(const int32_t *__restrict__ acc, int nodes, int64_t per_node,
                                    const float *__restrict__ s1, const float *__restrict__ s2,
                                    float *__restrict__ out, int64_t out_stride) {
+    pdl_enter();
     const int64_t total = per_node * nodes;
     for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
         int n = (int)(o / per_node);
@@ -167,7 +172,7 @@ static unsigned grid_for(int64_t n);
 
 lpdt_status dequant_acc_launch(const int32_t *acc, int nodes, int64_t per_node, const float *s1,
                                const float *s2, float *out, int64_t out_stride, cudaStream_t st) {
-    dequant_acc_kernel<<<grid_for(per_node * nodes), 256, 0, st>>>(acc, nodes, per_node, s1, s2, out, out_stride);
+    launch_k(dequant_acc_kernel, grid_for(per_node * nodes), 256, 0, st, acc, nodes, per_node, s1, s2, out, out_stride);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }
@@ -183,7 +188,7 @@ lpdt_status generic_fwd(const lpdt_conv_desc &d, const int8_t *A, const float *s
     const int Ho = conv_out(d.H, d.pad, d.R, d.stride), Wo = conv_out(d.W, d.pad, d.S, d.stride);
     const int64_t total = (int64_t)d.nodes * d.B * Ho * Wo * d.Cout;
     const bool vec4 = d.Cin % 4 == 0 && aligned(A, 4) && aligned(Wq, 4);
-    conv_fwd_generic<<<grid_for(total), 256, 0, st>>>(d, Ho, Wo, A, Wq, Yacc, Y, sA, sW, bias, bias_stride, vec4, uns);
+    launch_k(conv_fwd_generic, grid_for(total), 256, 0, st, d, Ho, Wo, A, Wq, Yacc, Y, sA, sW, bias, bias_stride, vec4, uns);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }
@@ -193,11 +198,11 @@ lpdt_status generic_bwd_data(const lpdt_conv_desc &d, const int8_t *E, const flo
     const int Ho = conv_out(d.H, d.pad, d.R, d.stride), Wo = conv_out(d.W, d.pad, d.S, d.stride);
     int8_t *Wt = (int8_t *)ws;
     const int64_t wn = (int64_t)d.nodes * d.Cout * d.R * d.S * d.Cin;
-    transpose_weights_kernel<<<grid_for(wn), 256, 0, st>>>(d, Wq, Wt);
+    launch_k(transpose_weights_kernel, grid_for(wn), 256, 0, st, d, Wq, Wt);
     LPDT_LAUNCH_CHECK();
     const int64_t total = (int64_t)d.nodes * d.B * d.H * d.W * d.Cin;
     const bool vec4 = d.Cout % 4 == 0 && aligned(E, 4) && aligned(Wt, 4);
-    conv_bwd_data_generic<<<grid_for(total), 256, 0, st>>>(d, Ho, Wo, E, Wt, dAacc, dA, sE, sW, vec4);
+    launch_k(conv_bwd_data_generic, grid_for(total), 256, 0, st, d, Ho, Wo, E, Wt, dAacc, dA, sE, sW, vec4);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }
@@ -212,10 +217,10 @@ lpdt_status generic_bwd_weight(const lpdt_conv_desc &d, const int8_t *E, const f
     const int64_t npix = (int64_t)d.B * Ho * Wo;
     int chunk = 4;
     while (ceil_div(npix, chunk) * d.nodes > (int64_t)kNumSMs * 16) chunk *= 2;
-    conv_bwd_weight_generic<<<dim3((unsigned)ceil_div(npix, chunk), d.nodes), 256, 0, st>>>(d, Ho, Wo, chunk, E, A, acc);
+    launch_k(conv_bwd_weight_generic, dim3((unsigned)ceil_div(npix, chunk), d.nodes), 256, 0, st, d, Ho, Wo, chunk, E, A, acc);
     LPDT_LAUNCH_CHECK();
     if (dW) {
-        dequant_acc_kernel<<<grid_for(per_node * d.nodes), 256, 0, st>>>(acc, d.nodes, per_node, sE, sA, dW, dw_stride);
+        launch_k(dequant_acc_kernel, grid_for(per_node * d.nodes), 256, 0, st, acc, d.nodes, per_node, sE, sA, dW, dw_stride);
         LPDT_LAUNCH_CHECK();
     }
     return LPDT_OK;

@@ -98,6 +98,7 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_enter();          // nothing above touches global memory
     const uint32_t tmem_base = __shfl_sync(0xffffffffu, ctl->tmem_base, 0);
     const int slot_bytes = p.mode == 0 ? p.N * 16 : 256;      // one K slice of weights (backward: per 16-column chunk)
     const int nchunk = p.N / 16;
@@ -353,7 +354,7 @@ lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, cons
     const long long tiles = (long long)p.nodes * p.B * p.tilesH * p.tilesW;
     if (tiles > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
     const int grid = (int)(tiles < (long long)kNumSMs * per_sm ? tiles : (long long)kNumSMs * per_sm);
-    conv_halo16_kernel<<<grid, kHaloThreads, smem, st>>>(mA, mW, p);
+    launch_k(conv_halo16_kernel, grid, kHaloThreads, smem, st, mA, mW, p);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

@@ -142,6 +142,7 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_enter();          // nothing above touches global memory
     const uint32_t tmem_base = __shfl_sync(0xffffffffu, ctl->tmem_base, 0);
     const int cpt = p.Kc / p.RBa;          // A boxes per tap
 
@@ -348,6 +349,7 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
+    pdl_enter();          // nothing above touches global memory
     const uint32_t tmem_base = __shfl_sync(0xffffffffu, ctl->tmem_base, 0);
 
     if (warp == 0) {
@@ -633,7 +635,7 @@ lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const flo
     const long long tiles = (long long)p.nodes * p.tilesB * p.tilesH * p.tilesW * p.tilesN * p.ncls;
     if (tiles > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
     const int grid = (int)(tiles < kNumSMs ? tiles : kNumSMs);
-    conv_pix_kernel<<<grid, kThreads, smem, st>>>(mA, mW, p);
+    launch_k(conv_pix_kernel, grid, kThreads, smem, st, mA, mW, p);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }
@@ -717,7 +719,7 @@ lpdt_status tc_wgrad(const lpdt_conv_desc &d, int cin_real, const int8_t *E, con
         if (!p.acc_out) return LPDT_ERR_WORKSPACE;
         LPDT_CUDA(cudaMemsetAsync(p.acc_out, 0, (size_t)d.nodes * per_node * sizeof(int32_t), st));
     }
-    conv_wgrad_kernel<<<dim3(p.splits, p.mgroups * p.ngroups, d.nodes), kThreads, smem, st>>>(mX, mE, p);
+    launch_k(conv_wgrad_kernel, dim3(p.splits, p.mgroups * p.ngroups, d.nodes), kThreads, smem, st, mX, mE, p);
     LPDT_LAUNCH_CHECK();
     if (p.splits > 1 && dW) return dequant_acc_launch(p.acc_out, d.nodes, per_node, sE, sA, dW, dw_stride, st);
     return LPDT_OK;

@@ -25,6 +25,7 @@ __device__ __forceinline__ float u24(uint32_t r) { return __uint2float_rn(r >> 8
 template <bool AFFINE, bool VEC>
 __global__ void range_kernel(const float *__restrict__ x, int64_t n, int64_t stride,
                              uint32_t *__restrict__ ws) {
+    pdl_enter();
     const int node = blockIdx.y;
     const float *xn = x + (int64_t)node * stride;
     float hi = 0.f, nlo = 0.f;
@@ -93,6 +94,7 @@ __global__ void quantize_kernel(const float *__restrict__ x, int64_t n, int64_t 
                                 const uint32_t *__restrict__ ws, int8_t *__restrict__ q,
                                 float *__restrict__ scale, int32_t *__restrict__ zero_point,
                                 uint2 key, uint32_t ctr_offset, int wstride) {
+    pdl_enter();
     const int node = blockIdx.y;
     const float *xn = x + (int64_t)node * stride;
     int8_t *qn = q + (int64_t)node * n;
@@ -155,6 +157,7 @@ __global__ void dequantize_kernel(const int8_t *__restrict__ q, int64_t n,
                                   const float *__restrict__ scale,
                                   const int32_t *__restrict__ zp, float *__restrict__ y,
                                   int64_t ystride) {
+    pdl_enter();
     const int node = blockIdx.y;
     const float s = scale[node];
     const int z = AFFINE ? zp[node] : 0;
@@ -206,21 +209,21 @@ extern "C" lpdt_status lpdt_quantize(const float *x, int32_t nodes, int64_t n, i
     dim3 grid(blocks_for(vec ? n / 4 : n, nodes), nodes), block(256);
     const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
     if (mode == LPDT_AFFINE_U8) {
-        if (vec) range_kernel<true, true><<<grid, block, 0, st>>>(x, n, x_node_stride, w);
-        else range_kernel<true, false><<<grid, block, 0, st>>>(x, n, x_node_stride, w);
+        if (vec) launch_k(range_kernel<true, true>, grid, block, 0, st, x, n, x_node_stride, w);
+        else launch_k(range_kernel<true, false>, grid, block, 0, st, x, n, x_node_stride, w);
         LPDT_LAUNCH_CHECK();
-        if (vec) quantize_kernel<2, true><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
-        else quantize_kernel<2, false><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
+        if (vec) launch_k(quantize_kernel<2, true>, grid, block, 0, st, x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
+        else launch_k(quantize_kernel<2, false>, grid, block, 0, st, x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
     } else {
-        if (vec) range_kernel<false, true><<<grid, block, 0, st>>>(x, n, x_node_stride, w);
-        else range_kernel<false, false><<<grid, block, 0, st>>>(x, n, x_node_stride, w);
+        if (vec) launch_k(range_kernel<false, true>, grid, block, 0, st, x, n, x_node_stride, w);
+        else launch_k(range_kernel<false, false>, grid, block, 0, st, x, n, x_node_stride, w);
         LPDT_LAUNCH_CHECK();
         if (rounding == LPDT_ROUND_NEAREST_EVEN) {
-            if (vec) quantize_kernel<0, true><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
-            else quantize_kernel<0, false><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
+            if (vec) launch_k(quantize_kernel<0, true>, grid, block, 0, st, x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
+            else launch_k(quantize_kernel<0, false>, grid, block, 0, st, x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
         } else {
-            if (vec) quantize_kernel<1, true><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
-            else quantize_kernel<1, false><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
+            if (vec) launch_k(quantize_kernel<1, true>, grid, block, 0, st, x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
+            else launch_k(quantize_kernel<1, false>, grid, block, 0, st, x, n, x_node_stride, w, q, scale, zero_point, key, ctr_offset, 2);
         }
     }
     LPDT_LAUNCH_CHECK();
@@ -234,8 +237,8 @@ extern "C" lpdt_status lpdt_dequantize(const int8_t *q, int32_t nodes, int64_t n
     if (nodes == 0 || n == 0) return LPDT_OK;
     LPDT_CHECK_ARG(q && scale && y && nodes <= 65535 && (y_node_stride >= n || nodes == 1));
     dim3 grid(blocks_for(n, nodes), nodes), block(256);
-    if (zero_point) dequantize_kernel<true><<<grid, block, 0, as_stream(stream)>>>(q, n, scale, zero_point, y, y_node_stride);
-    else dequantize_kernel<false><<<grid, block, 0, as_stream(stream)>>>(q, n, scale, zero_point, y, y_node_stride);
+    if (zero_point) launch_k(dequantize_kernel<true>, grid, block, 0, as_stream(stream), q, n, scale, zero_point, y, y_node_stride);
+    else launch_k(dequantize_kernel<false>, grid, block, 0, as_stream(stream), q, n, scale, zero_point, y, y_node_stride);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }
@@ -256,11 +259,11 @@ extern "C" lpdt_status lpdt_quantize_with_range(const float *x, int32_t nodes, i
     dim3 grid(blocks_for(vec ? n / 4 : n, nodes), nodes), block(256);
     const uint2 key = make_uint2((uint32_t)seed, (uint32_t)(seed >> 32));
     if (rounding == LPDT_ROUND_NEAREST_EVEN) {
-        if (vec) quantize_kernel<0, true><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, nullptr, key, ctr_offset, 1);
-        else quantize_kernel<0, false><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, nullptr, key, ctr_offset, 1);
+        if (vec) launch_k(quantize_kernel<0, true>, grid, block, 0, st, x, n, x_node_stride, w, q, scale, nullptr, key, ctr_offset, 1);
+        else launch_k(quantize_kernel<0, false>, grid, block, 0, st, x, n, x_node_stride, w, q, scale, nullptr, key, ctr_offset, 1);
     } else {
-        if (vec) quantize_kernel<1, true><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, nullptr, key, ctr_offset, 1);
-        else quantize_kernel<1, false><<<grid, block, 0, st>>>(x, n, x_node_stride, w, q, scale, nullptr, key, ctr_offset, 1);
+        if (vec) launch_k(quantize_kernel<1, true>, grid, block, 0, st, x, n, x_node_stride, w, q, scale, nullptr, key, ctr_offset, 1);
+        else launch_k(quantize_kernel<1, false>, grid, block, 0, st, x, n, x_node_stride, w, q, scale, nullptr, key, ctr_offset, 1);
     }
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
@@ -336,6 +339,7 @@ struct QuantBatch {
 // grid = (blocks, nodes, tensors); blocks beyond a tensor's length fall through
 __global__ void batch_range_kernel(const float *__restrict__ params, long long row_stride, QuantBatch qb,
                                    uint32_t *__restrict__ ws) {
+    pdl_enter();
     const int t = blockIdx.z, node = blockIdx.y;
     const long long n = qb.size[t];
     const float *x = params + (long long)node * row_stride + qb.src_off[t];
@@ -349,6 +353,7 @@ __global__ void batch_range_kernel(const float *__restrict__ params, long long r
 __global__ void batch_quantize_kernel(const float *__restrict__ params, long long row_stride, QuantBatch qb,
                                       const uint32_t *__restrict__ ws, int8_t *__restrict__ q,
                                       float *__restrict__ scales) {
+    pdl_enter();
     const int t = blockIdx.z, node = blockIdx.y, nodes = gridDim.y;
     const long long n = qb.size[t];
     const float *x = params + (long long)node * row_stride + qb.src_off[t];
@@ -392,9 +397,9 @@ extern "C" lpdt_status lpdt_quantize_batch(const float *params, int32_t nodes, i
     if (bx > 64) bx = 64;
     if (bx < 1) bx = 1;
     dim3 grid(bx, nodes, n_tensors);
-    batch_range_kernel<<<grid, 256, 0, st>>>(params, row_stride, qb, w);
+    launch_k(batch_range_kernel, grid, 256, 0, st, params, row_stride, qb, w);
     LPDT_LAUNCH_CHECK();
-    batch_quantize_kernel<<<grid, 256, 0, st>>>(params, row_stride, qb, w, q, scales);
+    launch_k(batch_quantize_kernel, grid, 256, 0, st, params, row_stride, qb, w, q, scales);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

@@ -87,6 +87,7 @@ ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
                int B, float *__restrict__ y, float *__restrict__ gmin, float *__restrict__ gmax,
                int32_t *__restrict__ argmin, int32_t *__restrict__ argmax, float *__restrict__ amax_out,
                const float *__restrict__ res) {
+    pdl_enter();
     extern __shared__ unsigned char smem_raw[];
     const int T = blockDim.x, t = threadIdx.x;
     Ext *s_mn = reinterpret_cast<Ext *>(smem_raw);
@@ -189,6 +190,7 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
                const int32_t *__restrict__ argmin, const int32_t *__restrict__ argmax,
                float *__restrict__ dx, double *__restrict__ acc /*[nodes][B][3][C] per-sample partial sums*/,
                float *__restrict__ amax_out) {
+    pdl_enter();
     extern __shared__ unsigned char smem_raw[];
     const int T = blockDim.x, t = threadIdx.x;
     // When the column count divides the warp, lanes that share a column are folded with shuffles and
@@ -332,6 +334,7 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
 __global__ void ren_bwd_finalize(const double *__restrict__ acc, int nodes, int B, int C,
                                  float *__restrict__ dv, float *__restrict__ dgamma,
                                  float *__restrict__ dbeta, int64_t gstride) {
+    pdl_enter();
     const int i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
     if (i >= nodes * 3 * C) return;
     const int node = i / (3 * C), j = i % (3 * C), which = j / C, c = j % C;
@@ -388,11 +391,11 @@ extern "C" lpdt_status lpdt_range_evonorm_fwd(int32_t nodes, int32_t B, int32_t 
     const float Cst = ren_const(C / groups);
     dim3 grid((unsigned)((int64_t)nodes * B));
     if (pl.V == 4) {
-        if (res) ren_fwd_kernel<4, true><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
-        else ren_fwd_kernel<4, false><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
+        if (res) launch_k(ren_fwd_kernel<4, true>, grid, pl.threads, smem, as_stream(stream), H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
+        else launch_k(ren_fwd_kernel<4, false>, grid, pl.threads, smem, as_stream(stream), H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
     } else {
-        if (res) ren_fwd_kernel<1, true><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
-        else ren_fwd_kernel<1, false><<<grid, pl.threads, smem, as_stream(stream)>>>(H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
+        if (res) launch_k(ren_fwd_kernel<1, true>, grid, pl.threads, smem, as_stream(stream), H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
+        else launch_k(ren_fwd_kernel<1, false>, grid, pl.threads, smem, as_stream(stream), H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
     }
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
@@ -430,11 +433,11 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t 
     const float Cst = ren_const(C / groups);
     dim3 grid((unsigned)((int64_t)nodes * B));
     if (pl.V == 4)
-        ren_bwd_kernel<4><<<grid, pl.threads, smem, st>>>(H * W, C, groups, eps, Cst, dy, x, v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc, amax_out);
+        launch_k(ren_bwd_kernel<4>, grid, pl.threads, smem, st, H * W, C, groups, eps, Cst, dy, x, v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc, amax_out);
     else
-        ren_bwd_kernel<1><<<grid, pl.threads, smem, st>>>(H * W, C, groups, eps, Cst, dy, x, v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc, amax_out);
+        launch_k(ren_bwd_kernel<1>, grid, pl.threads, smem, st, H * W, C, groups, eps, Cst, dy, x, v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc, amax_out);
     LPDT_LAUNCH_CHECK();
-    ren_bwd_finalize<<<(nodes * 3 * C + 7) / 8, 256, 0, st>>>(acc, nodes, B, C, dv, dgamma, dbeta, gstride);
+    launch_k(ren_bwd_finalize, (nodes * 3 * C + 7) / 8, 256, 0, st, acc, nodes, B, C, dv, dgamma, dbeta, gstride);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

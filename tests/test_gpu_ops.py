@@ -525,6 +525,64 @@ def test_deepsqueeze_mix(nodes, d, segs, bits):
         x_in = (x_ref - 0.05 * rng.standard_normal((nodes, d))).astype(np.float32)      # a stand-in local update
 
 
+def directed_ring_matrix(n, rng):
+    """Column-stochastic, not row-stochastic: node j keeps a share and pushes the rest to j+1 and j+2."""
+    W = np.zeros((n, n), np.float32)
+    for j in range(n):
+        w = rng.dirichlet(np.ones(3)).astype(np.float32)
+        W[j, j] += w[0]; W[(j + 1) % n, j] += w[1]; W[(j + 2) % n, j] += w[2]
+    return W
+
+
+@pytest.mark.parametrize("nodes,d", [(4, 1), (5, 1001), (16, 40000), (64, 4096), (3, 270410)])
+def test_pushsum_debias(nodes, d):
+    """Sparse-Push over three steps: Deep-Squeeze mix with a column-stochastic matrix, then the bias
+    weights and the de-biased model; bias weights and z bit-exact given the same mixed model."""
+    rng = np.random.default_rng(nodes * 7 + d)
+    W = directed_ring_matrix(nodes, rng)
+    x = rng.standard_normal((nodes, d)).astype(np.float32)
+    u_ref = np.ones(nodes, np.float32)
+    ud = dev(u_ref)
+    for step in range(3):
+        u_new_ref, z_ref = oracle.pushsum_debias(x, u_ref, W, 0.8)
+        un = torch.empty(nodes, device="cuda"); z = torch.empty(nodes, d, device="cuda")
+        api.lpdt_pushsum_debias(nodes, d, dev(x), ud, dev(W), 0.8, un, z)
+        assert np.array_equal(un.cpu().numpy(), u_new_ref), step
+        assert np.array_equal(z.cpu().numpy(), z_ref), step
+        u_ref, ud = u_new_ref, un
+        x = (x + 0.1 * rng.standard_normal((nodes, d))).astype(np.float32)
+    # in place, and the bias weights alone
+    xd = dev(x)
+    api.lpdt_pushsum_debias(nodes, d, xd, ud, dev(W), 0.8, un2 := torch.empty(nodes, device="cuda"), xd)
+    u3, z3 = oracle.pushsum_debias(x, u_ref, W, 0.8)
+    assert np.array_equal(xd.cpu().numpy(), z3) and np.array_equal(un2.cpu().numpy(), u3)
+    api.lpdt_pushsum_debias(nodes, 0, None, ud, dev(W), 0.8, un3 := torch.empty(nodes, device="cuda"), None)
+    assert np.array_equal(un3.cpu().numpy(), u3)
+
+
+def test_sparse_push_chain():
+    """Supplementary Algorithm 4 end to end on a directed graph: Deep-Squeeze mix (top-10 %) then push-sum
+    de-biasing, against the same two oracle calls; total mass sum_i x_i / sum_i u_i is what z tracks."""
+    rng = np.random.default_rng(44)
+    nodes, d = 8, 5000
+    W = directed_ring_matrix(nodes, rng)
+    x = rng.standard_normal((nodes, d)).astype(np.float32)
+    delta_ref = np.zeros((nodes, d), np.float32); u_ref = np.ones(nodes, np.float32)
+    deltad, ud = dev(delta_ref), dev(u_ref)
+    ws = ws_bytes(api.lpdt_gossip_mix_workspace_size(nodes, d, 1))
+    for step in range(3):
+        x_ref, delta_ref, _, _ = oracle.deepsqueeze_mix(x, delta_ref, W, 0.5, [0, d], [d // 10], 32)
+        u_ref, z_ref = oracle.pushsum_debias(x_ref, u_ref, W, 0.5)
+        xo = torch.empty(nodes, d, device="cuda"); un = torch.empty(nodes, device="cuda"); z = torch.empty_like(xo)
+        api.lpdt_deepsqueeze_mix(nodes, d, dev(x), deltad, xo, dev(W), 0.5, [0, d], [d // 10], ws)
+        api.lpdt_pushsum_debias(nodes, d, xo, ud, dev(W), 0.5, un, z)
+        assert np.array_equal(deltad.cpu().numpy(), delta_ref)
+        assert np.array_equal(un.cpu().numpy(), u_ref)
+        close(z, z_ref)
+        ud = un
+        x = (z_ref - 0.05 * rng.standard_normal((nodes, d))).astype(np.float32)
+
+
 def test_gossip_errors():
     t = torch.zeros(4, 8, device="cuda"); W = torch.zeros(4, 4, device="cuda")
     with pytest.raises(api.LpdtError) as e:
