@@ -1,16 +1,21 @@
 // Range-EvoNorm (Eq. "ren") forward and backward.
 //
-// One CTA per (node, sample).  Every thread owns a fixed vector-column of V
-// channels and walks the pixels, so global accesses are fully coalesced 16-byte
-// loads and the thread's channel parameters and group live in registers.
+// One CTA per (node, sample); the forward kernel can split a sample over a cluster
+// of up to 8 CTAs.  Every thread owns a fixed vector-column of V channels and walks
+// the pixels, so global accesses are fully coalesced 16-byte loads and the thread's
+// channel parameters and group live in registers.
 // Forward: pass 1 finds the per-group extrema; a warp-shuffle reduction with a
-// (value, lowest index) comparator merges the threads of a group; pass 2 re-reads
-// the sample (an L2 hit: a sample is at most a few hundred KB) and writes the
-// output.  Backward is a single pass: the local term of dx is written while the
+// (value, lowest index) comparator merges the threads of a group, the CTAs of a
+// cluster exchange their group extrema through distributed shared memory; pass 2
+// re-reads the sample and writes the output.  The second read is an L2 hit as long
+// as the samples in flight fit the L2: with large samples the cluster split keeps
+// that footprint small (fewer samples in flight, each finished sooner).  Backward is a single pass: the local term of dx is written while the
 // group sum S and the per-channel gradient sums accumulate, and S is applied
 // afterwards at the two extremum positions of each group.  Both kernels are
 // HBM-bound: forward moves 4 B in + 4 B out per element, backward 8 B in + 4 B out.
 #include <math.h>
+#include <stdlib.h>
+#include <cooperative_groups.h>
 #include "common.cuh"
 
 namespace lpdt {
@@ -86,18 +91,24 @@ ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
                const float *__restrict__ gamma, const float *__restrict__ beta, int64_t pstride,
                int B, float *__restrict__ y, float *__restrict__ gmin, float *__restrict__ gmax,
                int32_t *__restrict__ argmin, int32_t *__restrict__ argmax, float *__restrict__ amax_out,
-               const float *__restrict__ res) {
+               const float *__restrict__ res, int R /*CTAs per sample (cluster size)*/, int ppc /*pixels per CTA*/) {
+    namespace cg = cooperative_groups;
     pdl_enter();
     extern __shared__ unsigned char smem_raw[];
     const int T = blockDim.x, t = threadIdx.x;
     Ext *s_mn = reinterpret_cast<Ext *>(smem_raw);
     Ext *s_mx = s_mn + T;
-    Ext *g_mn = s_mx + T;
+    Ext *g_mn = s_mx + T;                 // the sample's group extrema
     Ext *g_mx = g_mn + groups;
+    Ext *part_mn = g_mx + groups;         // this CTA's group extrema, read by the whole cluster (R > 1)
+    Ext *part_mx = part_mn + groups;
     const int CV = C / V, cpg = C / groups;
     const int col = t % CV, row0 = t / CV, rstep = T / CV;
     const int c0 = col * V, grp = c0 / cpg;
-    const int64_t sample = blockIdx.x;         // node*B + b
+    const int rank = (int)(blockIdx.x % R);
+    const int64_t sample = blockIdx.x / R;     // node*B + b
+    const int p_lo = rank * ppc;
+    const int p_end = (p_lo + ppc < HW) ? p_lo + ppc : HW;     // this CTA's pixels: [p_lo, p_end)
     const int node = (int)(sample / B);
     const float *xs = x + sample * (int64_t)HW * C;
     float *ys = y + sample * (int64_t)HW * C;
@@ -106,8 +117,8 @@ ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
     // kU independent 16-byte loads per thread are issued before any of them is used: the kernel
     // is bound by the bytes in flight, not by arithmetic
     constexpr int kU = 8;
-    int p = row0;
-    for (; p + (kU - 1) * rstep < HW; p += kU * rstep) {
+    int p = p_lo + row0;
+    for (; p + (kU - 1) * rstep < p_end; p += kU * rstep) {
         float xv[kU][V];
 #pragma unroll
         for (int j = 0; j < kU; ++j) VecLoad<V>::ld(xs + (int64_t)(p + j * rstep) * C + c0, xv[j]);
@@ -121,7 +132,7 @@ ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
             }
         }
     }
-    for (; p < HW; p += rstep) {
+    for (; p < p_end; p += rstep) {
         float xv[V];
         VecLoad<V>::ld(xs + (int64_t)p * C + c0, xv);
 #pragma unroll
@@ -131,8 +142,25 @@ ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
             if (xv[k] < mn.v) { mn.v = xv[k]; mn.idx = idx; }
         }
     }
-    reduce_groups<V>(mn, mx, s_mn, s_mx, g_mn, g_mx, CV, cpg, groups);
-    if (t < groups) {
+    if (R == 1) {
+        reduce_groups<V>(mn, mx, s_mn, s_mx, g_mn, g_mx, CV, cpg, groups);
+    } else {
+        reduce_groups<V>(mn, mx, s_mn, s_mx, part_mn, part_mx, CV, cpg, groups);
+        cg::cluster_group cluster = cg::this_cluster();
+        cluster.sync();                        // every CTA's part_* is complete and visible
+        if (t < groups) {
+            Ext a = part_mn[t], b = part_mx[t];
+            for (int r = 1; r < R; ++r) {      // equal values: the lowest index wins, in any order
+                const int other = (rank + r) % R;
+                a = ext_min(a, *cluster.map_shared_rank(part_mn + t, other));
+                b = ext_max(b, *cluster.map_shared_rank(part_mx + t, other));
+            }
+            g_mn[t] = a; g_mx[t] = b;
+        }
+        __syncthreads();
+        cluster.barrier_arrive();              // done reading the others' shared memory; waited for before exit
+    }
+    if (t < groups && rank == 0) {
         int64_t sg = sample * groups + t;
         gmin[sg] = g_mn[t].v; gmax[sg] = g_mx[t].v; argmin[sg] = g_mn[t].idx; argmax[sg] = g_mx[t].idx;
     }
@@ -161,8 +189,8 @@ ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
         VecLoad<V>::st(ys + (int64_t)pp * C + c0, yv);
     };
     constexpr int kU2 = RES ? 2 : 4;
-    p = row0;
-    for (; p + (kU2 - 1) * rstep < HW; p += kU2 * rstep) {
+    p = p_lo + row0;
+    for (; p + (kU2 - 1) * rstep < p_end; p += kU2 * rstep) {
         float xv[kU2][V], rv[kU2][V];
 #pragma unroll
         for (int j = 0; j < kU2; ++j) {
@@ -172,13 +200,14 @@ ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
 #pragma unroll
         for (int j = 0; j < kU2; ++j) emit(p + j * rstep, xv[j], rv[j]);
     }
-    for (; p < HW; p += rstep) {
+    for (; p < p_end; p += rstep) {
         float xv[V], rv[V];
         VecLoad<V>::ld(xs + (int64_t)p * C + c0, xv);
         if (RES) VecLoad<V>::ld(rs + (int64_t)p * C + c0, rv);
         emit(p, xv, rv);
     }
     if (amax_out) block_amax_to(ymax, amax_out + node);
+    if (R > 1) cg::this_cluster().barrier_wait();      // nobody still reads this CTA's shared memory
 }
 
 template <int V>
@@ -367,6 +396,30 @@ static bool plan(int C, int groups, bool aligned16, RenPlan *pl) {
     return true;
 }
 
+// CTAs per sample of the forward kernel (cluster size: 1, 2, 4 or 8).  Two reasons to split a sample:
+// the samples in flight (one per resident CTA or cluster, 4 CTAs of 256 threads per SM) should fit
+// well inside the 126 MB L2 together with the output being written, so that pass 2 reads from L2; and a
+// small batch should still give every SM a few CTAs.  LPDT_REN_CLUSTER=1|2|4|8 overrides (parity tests).
+static int ren_cluster_size(int64_t samples, int HW, int C, int rstep) {
+    static int forced = -1;
+    if (forced < 0) { const char *e = getenv("LPDT_REN_CLUSTER"); forced = e ? atoi(e) : 0; }
+    const int rows = (int)ceil_div(HW, rstep);               // thread rows of a sample
+    int cap = 1;
+    while (cap < 8 && cap * 2 <= rows) cap *= 2;             // every CTA keeps at least one thread row
+    if (forced == 1 || forced == 2 || forced == 4 || forced == 8) return forced < cap ? forced : cap;
+    const double sample_bytes = (double)HW * C * 4.0;
+    const int64_t slots = (int64_t)kNumSMs * 4;
+    int R = 1;
+    while (R < cap) {
+        const int64_t in_flight = samples < slots / R ? samples : slots / R;
+        const bool l2_ok = (double)in_flight * sample_bytes <= 40.0 * 1024 * 1024;
+        const bool fills = samples * R >= 2 * (int64_t)kNumSMs;
+        if (l2_ok && fills) break;
+        R *= 2;
+    }
+    return R;
+}
+
 static float ren_const(int cpg) { return (float)(1.0 / sqrt(2.0 * log((double)cpg))); }
 
 }  // namespace lpdt
@@ -386,17 +439,20 @@ extern "C" lpdt_status lpdt_range_evonorm_fwd(int32_t nodes, int32_t B, int32_t 
     if ((int64_t)H * W * C > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
     RenPlan pl;
     if (!plan(C, groups, aligned(x, 16) && aligned(y, 16) && (!res || aligned(res, 16)), &pl)) return LPDT_ERR_UNSUPPORTED;
-    size_t smem = (size_t)(2 * pl.threads + 2 * groups) * sizeof(Ext);
+    size_t smem = (size_t)(2 * pl.threads + 4 * groups) * sizeof(Ext);
     if (smem > 48 * 1024) return LPDT_ERR_UNSUPPORTED;
     const float Cst = ren_const(C / groups);
-    dim3 grid((unsigned)((int64_t)nodes * B));
-    if (pl.V == 4) {
-        if (res) launch_k(ren_fwd_kernel<4, true>, grid, pl.threads, smem, as_stream(stream), H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
-        else launch_k(ren_fwd_kernel<4, false>, grid, pl.threads, smem, as_stream(stream), H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
-    } else {
-        if (res) launch_k(ren_fwd_kernel<1, true>, grid, pl.threads, smem, as_stream(stream), H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
-        else launch_k(ren_fwd_kernel<1, false>, grid, pl.threads, smem, as_stream(stream), H * W, C, groups, eps, Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res);
-    }
+    const int R = ren_cluster_size((int64_t)nodes * B, H * W, C, pl.threads / (C / pl.V));
+    const int rstep = pl.threads / (C / pl.V);
+    const int ppc = (int)ceil_div(ceil_div(H * W, R), rstep) * rstep;       // whole thread rows per CTA
+    if ((int64_t)nodes * B * R > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
+    dim3 grid((unsigned)((int64_t)nodes * B * R));
+    using Fn = void (*)(int, int, int, float, float, const float *, const float *, const float *, const float *, int64_t,
+                        int, float *, float *, float *, int32_t *, int32_t *, float *, const float *, int, int);
+    static const Fn fns[2][2] = {{ren_fwd_kernel<1, false>, ren_fwd_kernel<1, true>},
+                                 {ren_fwd_kernel<4, false>, ren_fwd_kernel<4, true>}};
+    launch_k_cluster(fns[pl.V == 4 ? 1 : 0][res ? 1 : 0], grid, pl.threads, smem, as_stream(stream), R, H * W, C, groups, eps,
+                     Cst, x, v, gamma, beta, pstride, B, y, gmin, gmax, argmin, argmax, amax_out, res, R, ppc);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

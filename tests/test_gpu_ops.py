@@ -289,7 +289,10 @@ def test_qconv_extreme_values_and_errors():
 
 # ------------------------------------------------------------------ Range-EvoNorm
 REN_CASES = [(4, 8, 16, 16, 16, 4), (2, 3, 32, 32, 16, 2), (2, 2, 8, 8, 64, 8), (1, 3, 5, 7, 6, 3),
-             (1, 2, 4, 4, 12, 1), (2, 2, 32, 32, 64, 8), (1, 2, 2, 2, 512, 64), (1, 1, 1, 1, 8, 2)]
+             (1, 2, 4, 4, 12, 1), (2, 2, 32, 32, 64, 8), (1, 2, 2, 2, 512, 64), (1, 1, 1, 1, 8, 2),
+             # samples split over a cluster: ragged pixel counts, odd column counts, large samples
+             (1, 3, 7, 9, 24, 3), (1, 2, 15, 15, 32, 4), (2, 1, 9, 9, 16, 2), (1, 2, 31, 33, 64, 16), (1, 1, 40, 40, 64, 8),
+             (2, 40, 16, 16, 32, 4)]
 
 
 def _ren_inputs(case, seed=0, ties=False):
@@ -342,6 +345,29 @@ def test_range_evonorm_fwd_bwd(case, ties):
     close(Gh[:, C:2 * C], dg64, RTOL, scale(dg64))
     close(Gh[:, 2 * C:3 * C], db64, RTOL, scale(db64))
     assert not Gh[:, 3 * C:].any()
+
+
+@pytest.mark.parametrize("case", REN_CASES)
+def test_range_evonorm_fwd_fused_shortcut(case):
+    """y = RangeEvoNorm(x) + res in one launch: one more fp32 addition on the bit-equal norm output; the
+    per-node max|y| it reports is that of the sum."""
+    nodes, B, H, W, C, groups = case
+    x, P, _ = _ren_inputs(case, seed=3)
+    v, g, b = P[:, :C], P[:, C:2 * C], P[:, 2 * C:3 * C]
+    res = np.random.default_rng(11).standard_normal(x.shape).astype(np.float32)
+    y32, mn, mx, amn, amx = oracle.range_evonorm_fwd(x, v, g, b, groups, 1e-5, "f32")
+    want = oracle.residual_add(res, y32)
+    f = lambda *s: torch.empty(*s, dtype=torch.float32, device="cuda")
+    i = lambda *s: torch.empty(*s, dtype=torch.int32, device="cuda")
+    Pd = dev(P)
+    y, gmin, gmax, amin_, amax_ = f(*x.shape), f(nodes, B, groups), f(nodes, B, groups), i(nodes, B, groups), i(nodes, B, groups)
+    rng_out = torch.zeros(nodes, device="cuda")
+    api.lpdt_range_evonorm_fwd(nodes, B, H, W, C, groups, 1e-5, dev(x), Pd, Pd[:, C:], Pd[:, 2 * C:], P.shape[1], y, gmin,
+                               gmax, amin_, amax_, amax_out=rng_out, res=dev(res))
+    assert np.array_equal(y.cpu().numpy(), want)
+    assert np.array_equal(amin_.cpu().numpy(), amn) and np.array_equal(amax_.cpu().numpy(), amx)
+    assert np.array_equal(gmin.cpu().numpy(), mn) and np.array_equal(gmax.cpu().numpy(), mx)
+    assert np.array_equal(rng_out.cpu().numpy(), np.abs(want).reshape(nodes, -1).max(1))
 
 
 def test_fused_ranges_feed_the_quantizer_exactly():
@@ -640,6 +666,21 @@ def test_glue_ops():
     cs = torch.zeros(3, 14, device="cuda")
     api.lpdt_colsum(3, 32, 10, dev(z), cs[:, 4:], 14)
     close(cs[:, 4:], oracle.colsum(z), 1e-6, 1e-7)
+
+
+@pytest.mark.parametrize("cluster", ["1", "2", "8"])
+def test_range_evonorm_cases_on_every_cluster_size(cluster):
+    """The forward kernel splits a sample over 1-8 CTAs by a size rule; the cases are re-run in child
+    processes with the cluster size forced (capped so that every CTA keeps a thread row)."""
+    import os, subprocess, sys
+    if os.environ.get("LPDT_CHILD") == "1":
+        pytest.skip("already inside a child run")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    child_env = dict(os.environ, LPDT_CHILD="1", LPDT_REN_CLUSTER=cluster)
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_ops.py"), "-m", "gpu",
+                        "-q", "-x", "-k", "test_range_evonorm_fwd or test_fused_ranges"], env=child_env, cwd=root,
+                       capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]
 
 
 @pytest.mark.parametrize("env", [{"LPDT_FORCE_HALO": "1"}, {"LPDT_DISABLE_HALO": "1"}, {"LPDT_DISABLE_TC": "1"}])
