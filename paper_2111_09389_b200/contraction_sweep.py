@@ -6,7 +6,12 @@ seeded random operands, through the C ABI.
     python -m paper_2111_09389_b200.contraction_sweep sweep           # the large GEMM / conv grid
 
 Operands are iid uniform int8 in [-127, 127]; every shape runs with int32
-accumulation and the fused fp32 dequantize.  The optional pass
+accumulation and the fused fp32 dequantize.  With --graph (the sweep's default)
+the calls are recorded into one CUDA graph and its replay is timed, so that the
+host's per-call cost (two tensor-map encodes and the ctypes call, 15-20 us) does
+not hide kernels of a few microseconds; consecutive calls then rotate through
+enough operand/result sets that the bytes touched between two uses of the same
+set exceed the 126 MB L2 (shapes whose own operands exceed it use one set).  The optional pass
 `fwd_affine` times the forward product on zero-point operands (same operand
 bytes; its correction pass re-reads and re-writes the result).  Prints one JSON line per
 (shape, pass) with the CUDA-event time, int8 TOPS (2 * MACs / time) and the
@@ -28,65 +33,74 @@ def _rand_s8(shape, seed):
     return torch.randint(-127, 128, shape, generator=g, device="cuda", dtype=torch.int8)
 
 
+L2_BYTES = 126 * 1024 * 1024
+
+
 def time_case(nodes, B, H, W, Cin, Cout, R, S, stride, pad, iters=20, warmup=3, passes=("fwd", "bwd_data", "bwd_weight"),
               label=None, graph=False):
     """graph=True records the `iters` calls into one CUDA graph and times its replay, which
-    takes the host's launch cost out of calls that run for only a few microseconds."""
+    takes the host's launch cost out of calls that run for only a few microseconds; the calls
+    rotate through `nsets` operand sets so that no call finds its operands in L2."""
     desc = api.conv_desc(nodes, B, H, W, Cin, Cout, R, S, stride, pad)
     Ho, Wo = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - S) // stride + 1
-    A = _rand_s8((nodes, B, H, W, Cin), 1)
-    Wq = _rand_s8((nodes, Cout, R, S, Cin), 2)
-    E = _rand_s8((nodes, B, Ho, Wo, Cout), 3)
+    set_bytes = nodes * (B * H * W * Cin + Cout * R * S * Cin + B * Ho * Wo * Cout) + \
+        4 * nodes * min(B * Ho * Wo * Cout, B * H * W * Cin, Cout * R * S * Cin)
+    nsets = 1 if not graph else max(1, min(iters, -(-int(1.25 * L2_BYTES) // set_bytes)))
+    sets = []
+    for i in range(nsets):
+        sets.append(dict(A=_rand_s8((nodes, B, H, W, Cin), 1 + 3 * i), Wq=_rand_s8((nodes, Cout, R, S, Cin), 2 + 3 * i),
+                         E=_rand_s8((nodes, B, Ho, Wo, Cout), 3 + 3 * i),
+                         Y=torch.empty(nodes, B, Ho, Wo, Cout, device="cuda"), dA=torch.empty(nodes, B, H, W, Cin, device="cuda"),
+                         dW=torch.empty(nodes, Cout * R * S * Cin, device="cuda")))
     sc = torch.full((nodes,), 1.0 / 127, device="cuda")
-    Y = torch.empty(nodes, B, Ho, Wo, Cout, device="cuda")
-    dA = torch.empty(nodes, B, H, W, Cin, device="cuda")
-    dW = torch.empty(nodes, Cout * R * S * Cin, device="cuda")
     ws = torch.empty(max(api.lpdt_qconv_workspace_size(desc, w) for w in (0, 1, 2)), dtype=torch.uint8, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     macs = nodes * B * Ho * Wo * Cout * Cin * R * S
+    t0 = sets[0]
     calls = {
-        "fwd": (lambda: api.lpdt_qconv_fwd(desc, A, sc, Wq, sc, Y=Y, ws=ws, dev_status=status),
-                A.numel() + Wq.numel() + 4 * Y.numel()),
-        "bwd_data": (lambda: api.lpdt_qconv_bwd_data(desc, E, sc, Wq, sc, dA=dA, ws=ws, dev_status=status),
-                     E.numel() + Wq.numel() + 4 * dA.numel()),
-        "bwd_weight": (lambda: api.lpdt_qconv_bwd_weight(desc, E, sc, A, sc, dW=dW, dw_node_stride=dW.shape[1], ws=ws,
-                                                         dev_status=status),
-                       E.numel() + A.numel() + 4 * dW.numel()),
+        "fwd": (lambda t: api.lpdt_qconv_fwd(desc, t["A"], sc, t["Wq"], sc, Y=t["Y"], ws=ws, dev_status=status),
+                t0["A"].numel() + t0["Wq"].numel() + 4 * t0["Y"].numel()),
+        "bwd_data": (lambda t: api.lpdt_qconv_bwd_data(desc, t["E"], sc, t["Wq"], sc, dA=t["dA"], ws=ws, dev_status=status),
+                     t0["E"].numel() + t0["Wq"].numel() + 4 * t0["dA"].numel()),
+        "bwd_weight": (lambda t: api.lpdt_qconv_bwd_weight(desc, t["E"], sc, t["A"], sc, dW=t["dW"],
+                                                           dw_node_stride=t["dW"].shape[1], ws=ws, dev_status=status),
+                       t0["E"].numel() + t0["A"].numel() + 4 * t0["dW"].numel()),
     }
     if "fwd_affine" in passes:       # zero-point operands: unsigned codes, per-node zero points
-        Au, Wu = A.view(torch.uint8), Wq.view(torch.uint8)
         zA = torch.full((nodes,), 131, dtype=torch.int32, device="cuda")
         zW = torch.full((nodes,), 120, dtype=torch.int32, device="cuda")
         wsa = torch.empty(api.lpdt_qconv_fwd_affine_workspace_size(desc), dtype=torch.uint8, device="cuda")
-        calls["fwd_affine"] = (lambda: api.lpdt_qconv_fwd_affine(desc, Au, sc, zA, Wu, sc, zW, Y=Y, ws=wsa,
-                                                                 dev_status=status),
-                               A.numel() + Wq.numel() + 4 * Y.numel())
+        calls["fwd_affine"] = (lambda t: api.lpdt_qconv_fwd_affine(desc, t["A"].view(torch.uint8), sc, zA,
+                                                                   t["Wq"].view(torch.uint8), sc, zW, Y=t["Y"], ws=wsa,
+                                                                   dev_status=status),
+                               t0["A"].numel() + t0["Wq"].numel() + 4 * t0["Y"].numel())
     out = []
     for name in passes:
         fn, min_bytes = calls[name]
-        for _ in range(warmup):
-            fn()
+        for i in range(warmup):
+            fn(sets[i % nsets])
         torch.cuda.synchronize()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         if graph:
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g):
-                for _ in range(iters):
-                    fn()
+                for i in range(iters):
+                    fn(sets[i % nsets])
             g.replay()
             torch.cuda.synchronize()
             e0.record()
             g.replay()
         else:
             e0.record()
-            for _ in range(iters):
-                fn()
+            for i in range(iters):
+                fn(sets[i % nsets])
         e1.record()
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / iters
         rec = {"shape": label or f"conv n{nodes} b{B} {H}x{W} {Cin}->{Cout} {R}x{S} s{stride}", "pass": name,
                "ms": ms, "tops": 2 * macs / (ms * 1e-3) / 1e12, "macs": macs, "min_hbm_bytes": int(min_bytes),
-               "gbs_at_min_bytes": min_bytes / (ms * 1e-3) / 1e9, "dev_status": int(status.item())}
+               "gbs_at_min_bytes": min_bytes / (ms * 1e-3) / 1e9, "dev_status": int(status.item()),
+               "timing": f"graph replay of {iters} calls over {nsets} operand sets" if graph else f"{iters} eager calls"}
         print(json.dumps(rec), flush=True)
         out.append(rec)
     return out
@@ -109,6 +123,7 @@ def main(argv=None):
     ap.add_argument("--nodes", type=int, default=1)
     ap.add_argument("--passes", default="fwd,bwd_data,bwd_weight")
     ap.add_argument("--graph", action="store_true", help="time a CUDA-graph replay of the calls")
+    ap.add_argument("--eager", action="store_true", help="sweep: time eager calls instead of a graph replay")
     a = ap.parse_args(argv)
     passes = tuple(a.passes.split(","))
     if a.kind == "gemm":
@@ -120,10 +135,10 @@ def main(argv=None):
         for M in sizes:
             for N in sizes:
                 for K in sizes:
-                    gemm(M, N, K, iters=max(3, a.iters // 4), warmup=2, passes=passes)
+                    gemm(M, N, K, iters=a.iters, warmup=2, passes=passes, graph=not a.eager)
         for C in (64, 256, 512):
             for HW in (32, 56):
-                conv(C, HW, 256, iters=max(3, a.iters // 4), warmup=2, passes=passes)
+                conv(C, HW, 256, iters=a.iters, warmup=2, passes=passes, graph=not a.eager)
 
 
 if __name__ == "__main__":
