@@ -82,55 +82,98 @@ constexpr int64_t kBigMin = 32768;     // shortest segment split over several CT
 constexpr int kChunk = 16384;          // elements per CTA on that path
 __device__ __host__ __forceinline__ bool is_big(int64_t len, int64_t k) { return len >= kBigMin && k > 0 && k < len; }
 
-// One CTA per (node, short segment).  Four 8-bit radix passes, most significant
-// first, narrow the k-th largest key; a final ordered pass places the tie cut.
-__device__ __forceinline__ void topk_select_body(const float *__restrict__ x_half, const float *__restrict__ x_hat,
-                                                 int64_t d, const SegTable &seg, SelectOut *__restrict__ out) {
-    const int s = blockIdx.x, node = blockIdx.y, plus = seg.plus;
-    const int64_t lo = seg.off[s], hi = seg.off[s + 1], len = hi - lo;
-    const int64_t k = seg.k[s];
-    SelectOut *o = out + (int64_t)node * seg.n_seg + s;
-    if (is_big(len, k)) return;          // handled by the multi-CTA kernels
-    if (k >= len) {
-        if (threadIdx.x == 0) { o->thr = 0; o->dense = 1; o->cut = hi; }
-        return;
-    }
+// Block-wide radix select over n 32-bit keys given by key(e), e in [0, n), 8 bits per pass, most
+// significant first.  The keys agree on their bits above `free_bits` (prefix0 holds them), so only the
+// low free_bits are scanned; with SKIP_ZERO, keys equal to 0 are left out.  Returns in every thread the
+// need-th largest key (need at least 1 and at most the number of keys scanned), how many keys equal to
+// it are among the need largest (*need_out) and how many keys equal it in all (*eq_out).
+template <bool SKIP_ZERO, typename KeyFn>
+__device__ uint32_t radix_select(int64_t n, KeyFn key, long long need, int free_bits, uint32_t prefix0,
+                                 long long *need_out, long long *eq_out) {
     __shared__ unsigned int hist[256];
     __shared__ uint32_t s_prefix, s_mask;
     __shared__ long long s_need;      // how many more keys to take inside the current prefix
-    __shared__ long long s_eq;        // keys equal to the final threshold
-    const float *xh = x_half + (int64_t)node * d, *xq = x_hat + (int64_t)node * d;
-    if (threadIdx.x == 0) { s_prefix = 0; s_mask = 0; s_need = (k > 0 ? k : 0); }
+    __shared__ long long s_eq;        // population of the chosen bucket
     __syncthreads();
-    if (k <= 0) {   // keep nothing: threshold above every finite key, no ties
-        if (threadIdx.x == 0) { o->thr = 0xffffffffu; o->dense = 0; o->cut = lo; }
-        return;
+    if (threadIdx.x == 0) {
+        s_mask = free_bits >= 32 ? 0u : ~((1u << free_bits) - 1u);
+        s_prefix = prefix0 & s_mask;
+        s_need = need;
     }
-    for (int shift = 24; shift >= 0; shift -= 8) {
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    for (int top = free_bits; top > 0;) {
+        const int w = top >= 8 ? 8 : top, shift = top - w;
+        const uint32_t dmask = (1u << w) - 1u;
         for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
         __syncthreads();
         const uint32_t prefix = s_prefix, mask = s_mask;
-        for (int64_t e = lo + threadIdx.x; e < hi; e += blockDim.x) {
-            uint32_t key = mag_bits(xh[e], xq[e], plus);
-            if ((key & mask) == prefix) atomicAdd(&hist[(key >> shift) & 255u], 1u);
-        }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            long long need = s_need;
-            int b = 255;
-            for (; b > 0; --b) {
-                if ((long long)hist[b] >= need) break;
-                need -= hist[b];
+        // uniform trip count (the warp votes below need every lane); eight independent loads per thread
+        for (int64_t base = 0; base < n; base += 8 * (int64_t)blockDim.x) {
+            uint32_t k[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int64_t eu = base + u * (int64_t)blockDim.x + threadIdx.x;
+                k[u] = eu < n ? key(eu) : 0u;
             }
-            s_need = need;                       // 1 <= need <= hist[b]
-            s_eq = hist[b];
-            s_prefix = prefix | ((uint32_t)b << shift);
-            s_mask = mask | (255u << shift);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int64_t eu = base + u * (int64_t)blockDim.x + threadIdx.x;
+                const bool hit = eu < n && !(SKIP_ZERO && k[u] == 0u) && (k[u] & mask) == prefix;
+                const uint32_t bin = (k[u] >> shift) & dmask;
+                // a warp whose hits all fall into one bin (constant data, shared leading bits) adds once
+                const unsigned hits = __ballot_sync(0xffffffffu, hit);
+                if (hits == 0u) continue;
+                const int leader = __ffs(hits) - 1;
+                const uint32_t lbin = __shfl_sync(0xffffffffu, bin, leader);
+                if (__all_sync(0xffffffffu, !hit || bin == lbin)) {
+                    if (lane == leader) atomicAdd(&hist[lbin], (unsigned)__popc(hits));
+                } else if (hit) {
+                    atomicAdd(&hist[bin], 1u);
+                }
+            }
         }
         __syncthreads();
+        if (threadIdx.x < 32) {
+            // bucket of the need-th largest key: lane l owns bins [8l, 8l+8); suffix sums across lanes by shuffles
+            long long mine = 0;
+#pragma unroll
+            for (int j = 0; j < 8; ++j) mine += hist[lane * 8 + j];
+            long long incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const long long v = __shfl_down_sync(0xffffffffu, incl, o);
+                if (lane + o < 32) incl += v;
+            }
+            const long long above = incl - mine, nd0 = s_need;
+            if (above < nd0 && nd0 <= above + mine) {
+                long long nd = nd0 - above;
+                int bsel = lane * 8 + 7;
+                for (; bsel > lane * 8; --bsel) {
+                    if ((long long)hist[bsel] >= nd) break;
+                    nd -= hist[bsel];
+                }
+                s_need = nd;                     // 1 <= nd <= hist[bsel]
+                s_eq = hist[bsel];
+                s_prefix = prefix | ((uint32_t)bsel << shift);
+                s_mask = mask | (dmask << shift);
+            }
+        }
+        __syncthreads();
+        top = shift;
     }
-    const uint32_t thr = s_prefix;
-    const long long need = s_need, eq = s_eq;
+    *need_out = s_need; *eq_out = s_eq;
+    return s_prefix;
+}
+
+// One CTA selects over a whole segment: the k-th largest magnitude by radix select, then an ordered
+// pass that places the tie cut.  The path of short segments, and of long ones whose candidates did
+// not fit (below).
+__device__ void select_whole_segment(const float *__restrict__ xh, const float *__restrict__ xq, int64_t lo, int64_t hi,
+                                     int64_t k, int plus, SelectOut *o) {
+    long long need, eq;
+    const uint32_t thr = radix_select<false>(hi - lo, [&](int64_t e) { return mag_bits(xh[lo + e], xq[lo + e], plus); },
+                                             (long long)k, 32, 0u, &need, &eq);
     if (eq == need) {        // every tie is taken
         if (threadIdx.x == 0) { o->thr = thr; o->dense = 0; o->cut = hi; }
         return;
@@ -139,18 +182,26 @@ __device__ __forceinline__ void topk_select_body(const float *__restrict__ x_hal
     if (threadIdx.x == 0) { o->thr = thr; o->dense = 0; o->cut = cut; }
 }
 
-// ---- long segments: the same radix select spread over many CTAs -----------------------------
-// Three histogram launches (11 + 11 + 9 key bits) accumulate per (node, segment) histograms in
-// global memory; each later launch re-derives the bucket chosen at the levels above it from those
-// histograms, so no CTA waits for another.  A fourth launch counts the keys equal to the threshold
-// per chunk (only if not all of them are taken) and a fifth places the tie cut.
+// ---- long segments: two streaming passes spread over many CTAs ------------------------------
+// Pass 1 (big_hist_kernel) builds, per (node, segment), a histogram of the top 12 magnitude bits
+// (exponent and four mantissa bits: buckets 1/16 of an octave wide); the CTA that finishes last walks it and records the bucket
+// that holds the k-th largest key.  Pass 2 (big_collect_kernel) copies the keys of that bucket with
+// their positions into a candidate list.  The select launch then finds the threshold and the tie
+// cut among the candidates alone (one CTA per segment, a few per cent of the data at most).  A
+// bucket that outgrows the list (1/8 of the segment; a Gaussian's fullest bucket holds 3 %, a uniform
+// distribution's 6 %: only near-constant magnitudes get there) falls back to the whole-segment path.
 struct BigList {
     int32_t n;
     int32_t id[kMaxSeg];               // segment index
     int32_t chunk_base[kMaxSeg + 1];   // prefix sums of the chunk counts
+    int64_t cand_base[kMaxSeg + 1];    // prefix sums of the candidate capacities
 };
-struct BigHist { uint32_t h0[2048], h1[2048], h2[512]; uint32_t tickets[4]; };   // zeroed per call
-struct BigState { uint32_t prefix, mask; long long need, eq; };   // key bits fixed so far; keys still to take; bucket population
+constexpr int kTopBins = 4096;
+struct BigCtl { uint32_t h0[kTopBins]; uint32_t ticket, cand_count; };   // zeroed per call
+struct BigState { uint32_t prefix; uint32_t overflow; long long need, eq; };   // chosen bucket; keys still to take in it; its population
+struct __align__(8) Cand { uint32_t key, pos; };    // magnitude bits, position inside the segment
+
+__device__ __host__ __forceinline__ int64_t cand_capacity(int64_t len) { return len / 8 + 4096; }
 
 // Walk a histogram from its top bin: the bucket holding the need-th largest key, the keys still
 // needed inside it and its population.  Whole CTA (256 threads); same result in every thread.
@@ -188,51 +239,22 @@ __device__ void pick_bucket(const uint32_t *hist, int nbins, long long need, int
     *bucket = (int)res[0]; *need_out = res[1]; *eq_out = res[2];
 }
 
-// LEVEL 0..2: histogram of the next key bits (11, 11, 9) among the keys that match the prefix so
-// far; the CTA that finishes last for its (node, segment) walks the finished histogram and records
-// the new prefix.  LEVEL 3: count the keys equal to the threshold per chunk (skipped when all of
-// them are taken).
-template <int LEVEL>
+constexpr int kTopShift = 19;          // the histogram keys on magnitude bits 30..19
+
 __global__ void __launch_bounds__(256)
-big_select_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d, SegTable seg,
-                  BigList big, BigHist *__restrict__ hists, BigState *__restrict__ state,
-                  uint32_t *__restrict__ tie_counts, int total_chunks, SelectOut *__restrict__ out) {
+big_hist_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d, SegTable seg,
+                BigList big, BigCtl *__restrict__ ctl, BigState *__restrict__ state) {
     pdl_enter();
     const int bi = blockIdx.y, node = blockIdx.z, s = big.id[bi], plus = seg.plus;
     const int64_t lo = seg.off[s], hi = seg.off[s + 1];
     const int64_t c0 = lo + (int64_t)blockIdx.x * kChunk;
     if (c0 >= hi) return;
     const int64_t c1 = (c0 + kChunk < hi) ? c0 + kChunk : hi;
-    BigHist *h = hists + (int64_t)node * big.n + bi;
-    BigState *stp = state + (int64_t)node * big.n + bi;
-    BigState cur;
-    if (LEVEL == 0) { cur.prefix = 0; cur.mask = 0; cur.need = seg.k[s]; cur.eq = 0; }
-    else cur = *stp;                      // written by the previous launch
+    BigCtl *h = ctl + (int64_t)node * big.n + bi;
     const float *xh = x_half + (int64_t)node * d, *xq = x_hat + (int64_t)node * d;
-    if (LEVEL == 3) {
-        if (cur.eq == cur.need) {         // every tie is taken
-            if (blockIdx.x == 0 && threadIdx.x == 0) {
-                SelectOut so; so.thr = cur.prefix; so.dense = 0; so.cut = hi;
-                out[(int64_t)node * seg.n_seg + s] = so;
-            }
-            return;
-        }
-        int cnt = 0;
-        for (int64_t e = c0 + threadIdx.x; e < c1; e += blockDim.x) cnt += mag_bits(xh[e], xq[e], plus) == cur.prefix;
-        __shared__ int s_cnt;
-        if (threadIdx.x == 0) s_cnt = 0;
-        __syncthreads();
-        if (cnt) atomicAdd(&s_cnt, cnt);
-        __syncthreads();
-        if (threadIdx.x == 0)
-            tie_counts[(int64_t)node * total_chunks + big.chunk_base[bi] + blockIdx.x] = (uint32_t)s_cnt;
-        return;
-    }
-    constexpr int kBins = LEVEL == 2 ? 512 : 2048;
-    constexpr int kShift = LEVEL == 0 ? 20 : LEVEL == 1 ? 9 : 0;
-    __shared__ unsigned int sh[kBins];
+    __shared__ unsigned int sh[kTopBins];
     __shared__ unsigned int s_ticket;
-    for (int i = threadIdx.x; i < kBins; i += blockDim.x) sh[i] = 0;
+    for (int i = threadIdx.x; i < kTopBins; i += blockDim.x) sh[i] = 0;
     __syncthreads();
     for (int64_t e = c0 + threadIdx.x; e < c1; e += 4 * blockDim.x) {      // eight loads in flight per thread
         float a[4], b[4];
@@ -242,68 +264,102 @@ big_select_kernel(const float *__restrict__ x_half, const float *__restrict__ x_
             if (eu < c1) { a[u] = xh[eu]; b[u] = xq[eu]; }
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            if (e + u * blockDim.x < c1) {
-                const uint32_t key = mag_bits(a[u], b[u], plus);
-                if ((key & cur.mask) == cur.prefix) atomicAdd(&sh[(key >> kShift) & (kBins - 1)], 1u);
-            }
-        }
+        for (int u = 0; u < 4; ++u)
+            if (e + u * blockDim.x < c1) atomicAdd(&sh[mag_bits(a[u], b[u], plus) >> kTopShift], 1u);
     }
     __syncthreads();
-    uint32_t *g = LEVEL == 0 ? h->h0 : LEVEL == 1 ? h->h1 : h->h2;
-    for (int i = threadIdx.x; i < kBins; i += blockDim.x)
-        if (sh[i]) atomicAdd(&g[i], sh[i]);
+    for (int i = threadIdx.x; i < kTopBins; i += blockDim.x)
+        if (sh[i]) atomicAdd(&h->h0[i], sh[i]);
     // last CTA of this (node, segment): every chunk's counts have landed
     __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) s_ticket = atomicAdd(&h->tickets[LEVEL], 1u);
+    if (threadIdx.x == 0) s_ticket = atomicAdd(&h->ticket, 1u);
     __syncthreads();
     const unsigned nchunks = (unsigned)(big.chunk_base[bi + 1] - big.chunk_base[bi]);
     if (s_ticket != nchunks - 1) return;
     __threadfence();
     int b; long long need, eq;
-    pick_bucket(g, kBins, cur.need, &b, &need, &eq);
+    pick_bucket(h->h0, kTopBins, seg.k[s], &b, &need, &eq);
     if (threadIdx.x == 0) {
         BigState nx;
-        nx.prefix = cur.prefix | ((uint32_t)b << kShift);
-        nx.mask = cur.mask | ((uint32_t)(kBins - 1) << kShift);
+        nx.prefix = (uint32_t)b << kTopShift;
+        nx.overflow = eq > cand_capacity(hi - lo) ? 1u : 0u;
         nx.need = need; nx.eq = eq;
-        *stp = nx;
+        state[(int64_t)node * big.n + bi] = nx;
     }
 }
 
-// One CTA per (node, long segment): find the chunk that holds the need-th tie from the chunk
-// counts, then walk that chunk in index order.
+// Copy the keys of the chosen bucket, with their positions, into the (node, segment)'s candidate
+// list.  Matches are staged in shared memory and flushed with one reservation per CTA; the order
+// inside the list is arbitrary (the selection over it does not depend on it).
+constexpr int kStage = 2048;
 __global__ void __launch_bounds__(256)
-big_cut_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d, SegTable seg,
-               BigList big, const BigState *__restrict__ state, const uint32_t *__restrict__ tie_counts,
-               int total_chunks, SelectOut *__restrict__ out) {
+big_collect_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d, SegTable seg,
+                   BigList big, BigCtl *__restrict__ ctl, const BigState *__restrict__ state,
+                   Cand *__restrict__ cands, int64_t cand_per_node) {
     pdl_enter();
-    const int bi = blockIdx.x, node = blockIdx.y, s = big.id[bi];
-    const BigState f = state[(int64_t)node * big.n + bi];
-    if (f.eq == f.need) return;
+    const int bi = blockIdx.y, node = blockIdx.z, s = big.id[bi], plus = seg.plus;
     const int64_t lo = seg.off[s], hi = seg.off[s + 1];
-    const int nchunks = big.chunk_base[bi + 1] - big.chunk_base[bi];
-    const uint32_t *cnt = tie_counts + (int64_t)node * total_chunks + big.chunk_base[bi];
-    __shared__ int s_chunk;
-    __shared__ long long s_before;
-    if (threadIdx.x == 0) {
-        long long run = 0; int c = 0;
-        for (; c < nchunks - 1; ++c) {
-            if (run + cnt[c] >= f.need) break;
-            run += cnt[c];
+    const int64_t c0 = lo + (int64_t)blockIdx.x * kChunk;
+    if (c0 >= hi) return;
+    const int64_t c1 = (c0 + kChunk < hi) ? c0 + kChunk : hi;
+    const BigState stt = state[(int64_t)node * big.n + bi];
+    if (stt.overflow) return;                   // the whole-segment path takes this one
+    BigCtl *h = ctl + (int64_t)node * big.n + bi;
+    Cand *list = cands + (int64_t)node * cand_per_node + big.cand_base[bi];
+    const float *xh = x_half + (int64_t)node * d, *xq = x_hat + (int64_t)node * d;
+    const uint32_t bucket = stt.prefix >> kTopShift;
+    __shared__ Cand stage[kStage];
+    __shared__ unsigned int s_cnt, s_base;
+    if (threadIdx.x == 0) s_cnt = 0;
+    __syncthreads();
+    for (int64_t e = c0 + threadIdx.x; e < c1; e += 4 * blockDim.x) {
+        float a[4], b[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int64_t eu = e + u * blockDim.x;
+            if (eu < c1) { a[u] = xh[eu]; b[u] = xq[eu]; }
         }
-        s_chunk = c; s_before = run;
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int64_t eu = e + u * blockDim.x;
+            if (eu < c1) {
+                const uint32_t key = mag_bits(a[u], b[u], plus);
+                if ((key >> kTopShift) == bucket) {
+                    Cand c; c.key = key; c.pos = (uint32_t)(eu - lo);
+                    const unsigned slot = atomicAdd(&s_cnt, 1u);
+                    if (slot < kStage) stage[slot] = c;
+                    else list[atomicAdd(&h->cand_count, 1u)] = c;      // a dense stretch: straight to the list
+                }
+            }
+        }
     }
     __syncthreads();
-    const int64_t c0 = lo + (int64_t)s_chunk * kChunk;
-    const int64_t c1 = (c0 + kChunk < hi) ? c0 + kChunk : hi;
-    const long long cut = ordered_cut(x_half + (int64_t)node * d, x_hat + (int64_t)node * d, c0, c1, f.prefix,
-                                      f.need - s_before, seg.plus);
-    if (threadIdx.x == 0) {
-        SelectOut so; so.thr = f.prefix; so.dense = 0; so.cut = cut;
-        out[(int64_t)node * seg.n_seg + s] = so;
+    const unsigned n = s_cnt < kStage ? s_cnt : kStage;
+    if (n == 0) return;
+    if (threadIdx.x == 0) s_base = atomicAdd(&h->cand_count, n);
+    __syncthreads();
+    for (unsigned i = threadIdx.x; i < n; i += blockDim.x) list[s_base + i] = stage[i];
+}
+
+// Threshold and tie cut of a long segment from its candidate list (one CTA).  All keys of the chosen
+// bucket are in the list, so the need-th largest of the list is the segment's k-th largest; if only
+// some of the keys equal to it are taken, those at the lowest positions are: the cut follows the
+// need-th smallest position among them.
+__device__ void select_from_candidates(const Cand *__restrict__ list, const BigState &stt, int64_t lo, int64_t hi,
+                                       SelectOut *o) {
+    long long need, eq;
+    const uint32_t thr = radix_select<false>((int64_t)stt.eq, [&](int64_t e) { return list[e].key; }, stt.need, kTopShift,
+                                             stt.prefix, &need, &eq);
+    if (eq == need) {
+        if (threadIdx.x == 0) { o->thr = thr; o->dense = 0; o->cut = hi; }
+        return;
     }
+    long long n2, e2;      // ties keyed by descending position (never 0); the other candidates are skipped
+    const uint32_t inv = radix_select<true>((int64_t)stt.eq,
+                                            [&](int64_t e) { return list[e].key == thr ? 0xFFFFFFFFu - list[e].pos : 0u; },
+                                            need, 32, 0u, &n2, &e2);
+    if (threadIdx.x == 0) { o->thr = thr; o->dense = 0; o->cut = lo + (int64_t)(0xFFFFFFFFu - inv) + 1; }
 }
 
 // Row i of the mixing matrix as a compact list of its non-zero entries (j ascending), built once
@@ -368,7 +424,8 @@ __global__ void __launch_bounds__(1024)
 select_and_rows_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d,
                        SegTable seg, SelectOut *__restrict__ out, const float *__restrict__ Wmix, int nodes,
                        int32_t *__restrict__ tab, const unsigned int *__restrict__ amax_bits,
-                       float *__restrict__ msg_scale, float *__restrict__ msg_inv) {
+                       float *__restrict__ msg_scale, float *__restrict__ msg_inv, BigList big,
+                       const BigState *__restrict__ state, const Cand *__restrict__ cands, int64_t cand_per_node) {
     pdl_enter();
     if ((int)blockIdx.y == nodes) {
         if (blockIdx.x == 0) {
@@ -377,7 +434,28 @@ select_and_rows_kernel(const float *__restrict__ x_half, const float *__restrict
         }
         return;
     }
-    topk_select_body(x_half, x_hat, d, seg, out);
+    const int s = blockIdx.x, node = blockIdx.y;
+    const int64_t lo = seg.off[s], hi = seg.off[s + 1], len = hi - lo, k = seg.k[s];
+    SelectOut *o = out + (int64_t)node * seg.n_seg + s;
+    if (k >= len) {          // keep everything
+        if (threadIdx.x == 0) { o->thr = 0; o->dense = 1; o->cut = hi; }
+        return;
+    }
+    if (k <= 0) {            // keep nothing: threshold above every finite key, no ties
+        if (threadIdx.x == 0) { o->thr = 0xffffffffu; o->dense = 0; o->cut = lo; }
+        return;
+    }
+    const float *xh = x_half + (int64_t)node * d, *xq = x_hat + (int64_t)node * d;
+    if (is_big(len, k)) {
+        int bi = 0;
+        while (big.id[bi] != s) ++bi;            // every long segment is in the list
+        const BigState stt = state[(int64_t)node * big.n + bi];
+        if (!stt.overflow) {
+            select_from_candidates(cands + (int64_t)node * cand_per_node + big.cand_base[bi], stt, lo, hi, o);
+            return;
+        }
+    }
+    select_whole_segment(xh, xq, lo, hi, k, seg.plus, o);
 }
 
 // Fused public-copy update + mixing.  A block owns TE*V consecutive parameters of all nodes; a thread
@@ -552,24 +630,29 @@ static size_t rows_bytes(int32_t nodes) {
     const size_t nn = (size_t)(nodes > 0 ? nodes : 1);
     return align_up((nn + 2 * nn * nn) * sizeof(int32_t), 256);
 }
-// the most long segments and chunks any segmentation of d parameters into n_segments can have
+// the most long segments any segmentation of d parameters into n_segments can have
 static int64_t max_big(int64_t d, int32_t n_segments) {
     int64_t m = d / kBigMin;
     return m < n_segments ? m : n_segments;
 }
-static int64_t max_chunks(int64_t d, int32_t n_segments) { return d / kChunk + max_big(d, n_segments); }
+// candidate entries per node that any segmentation can need: sum over long segments of cand_capacity(len)
+static int64_t max_cands(int64_t d, int32_t n_segments) { return d / 8 + 4096 * max_big(d, n_segments); }
+static size_t big_ctl_bytes(int32_t nodes, int64_t d, int32_t n_segments) {
+    return align_up((size_t)(nodes > 0 ? nodes : 1) * (size_t)max_big(d, n_segments) * (sizeof(BigCtl) + sizeof(BigState)), 256);
+}
+static size_t cand_bytes(int32_t nodes, int64_t d, int32_t n_segments) {
+    return align_up((size_t)(nodes > 0 ? nodes : 1) * (size_t)max_cands(d, n_segments) * sizeof(Cand), 256);
+}
 // range words and reciprocal steps of the 8-bit messages, one per (node, segment) each (last in the workspace)
 static size_t q8_bytes(int32_t nodes, int32_t n_segments) {
     return align_up((size_t)(nodes > 0 ? nodes : 1) * (size_t)(n_segments > 0 ? n_segments : 1) * sizeof(float), 256);
 }
 
 extern "C" size_t lpdt_gossip_mix_workspace_size(int32_t nodes, int64_t d, int32_t n_segments) {
-    const size_t nn = (size_t)(nodes > 0 ? nodes : 1);
     if (d < 0) d = 0;
     if (n_segments < 1) n_segments = 1;
-    return select_bytes(nodes, n_segments) + rows_bytes(nodes) +
-           align_up(nn * (size_t)max_big(d, n_segments) * (sizeof(BigHist) + sizeof(BigState)), 256) +
-           align_up(nn * (size_t)max_chunks(d, n_segments) * sizeof(uint32_t), 256) + 2 * q8_bytes(nodes, n_segments);
+    return select_bytes(nodes, n_segments) + rows_bytes(nodes) + big_ctl_bytes(nodes, d, n_segments) +
+           cand_bytes(nodes, d, n_segments) + 2 * q8_bytes(nodes, n_segments);
 }
 
 static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, float *x_hat,
@@ -598,33 +681,31 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
     SelectOut *sel = (SelectOut *)ws;
     int32_t *tab = (int32_t *)((char *)ws + select_bytes(nodes, n_segments));
     BigList big;
-    big.n = 0; big.chunk_base[0] = 0;
+    big.n = 0; big.chunk_base[0] = 0; big.cand_base[0] = 0;
     int64_t most_chunks = 0;
     for (int s = 0; s < n_segments; ++s) {
         const int64_t len = seg.off[s + 1] - seg.off[s];
         if (!is_big(len, seg.k[s])) continue;
+        if (len > 0xFFFFFFFFll) return LPDT_ERR_UNSUPPORTED;      // candidate positions are 32-bit
         const int64_t nc = ceil_div(len, (int64_t)kChunk);
         big.id[big.n] = s;
         big.chunk_base[big.n + 1] = big.chunk_base[big.n] + (int32_t)nc;
+        big.cand_base[big.n + 1] = big.cand_base[big.n] + cand_capacity(len);
         if (nc > most_chunks) most_chunks = nc;
         ++big.n;
     }
+    char *big_region = (char *)tab + rows_bytes(nodes);
+    BigCtl *ctl = (BigCtl *)big_region;
+    BigState *state = (BigState *)(ctl + (size_t)nodes * big.n);
+    Cand *cands = (Cand *)(big_region + big_ctl_bytes(nodes, d, n_segments));
+    const int64_t cand_per_node = big.cand_base[big.n];
     if (big.n > 0) {
         if (most_chunks > 0x7fffffff || nodes > 65535) return LPDT_ERR_UNSUPPORTED;
-        char *p = (char *)tab + rows_bytes(nodes);
-        BigHist *hists = (BigHist *)p;
-        BigState *state = (BigState *)(hists + (size_t)nodes * big.n);
-        const size_t hist_region = align_up((size_t)nodes * (size_t)max_big(d, n_segments) * (sizeof(BigHist) + sizeof(BigState)), 256);
-        uint32_t *ties = (uint32_t *)(p + hist_region);
-        const int total_chunks = big.chunk_base[big.n];
-        LPDT_CUDA(cudaMemsetAsync(hists, 0, (size_t)nodes * big.n * sizeof(BigHist), st));
+        LPDT_CUDA(cudaMemsetAsync(ctl, 0, (size_t)nodes * big.n * sizeof(BigCtl), st));
         const dim3 g((unsigned)most_chunks, big.n, nodes);
-        launch_k(big_select_kernel<0>, g, 256, 0, st, x_half, x_hat, d, seg, big, hists, state, ties, total_chunks, sel);
-        launch_k(big_select_kernel<1>, g, 256, 0, st, x_half, x_hat, d, seg, big, hists, state, ties, total_chunks, sel);
-        launch_k(big_select_kernel<2>, g, 256, 0, st, x_half, x_hat, d, seg, big, hists, state, ties, total_chunks, sel);
-        launch_k(big_select_kernel<3>, g, 256, 0, st, x_half, x_hat, d, seg, big, hists, state, ties, total_chunks, sel);
+        launch_k(big_hist_kernel, g, 256, 0, st, x_half, x_hat, d, seg, big, ctl, state);
         LPDT_LAUNCH_CHECK();
-        launch_k(big_cut_kernel, dim3(big.n, nodes), 256, 0, st, x_half, x_hat, d, seg, big, state, ties, total_chunks, sel);
+        launch_k(big_collect_kernel, g, 256, 0, st, x_half, x_hat, d, seg, big, ctl, state, cands, cand_per_node);
         LPDT_LAUNCH_CHECK();
     }
     // 8-bit messages: ranges of the differences first (the kept entries are the largest of their segment)
@@ -639,7 +720,7 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
         LPDT_LAUNCH_CHECK();
     }
     launch_k(select_and_rows_kernel, dim3(n_segments, nodes + 1), 1024, 0, st, x_half, x_hat, d, seg, sel, Wmix, nodes, tab,
-                                                                         amax_bits, msg_scale, msg_inv);
+             amax_bits, msg_scale, msg_inv, big, state, cands, cand_per_node);
     LPDT_LAUNCH_CHECK();
     const bool v4 = d % 4 == 0 && aligned(x_half, 16) && aligned(x_hat, 16) && aligned(x_out, 16);
     const int V = v4 ? 4 : 1;

@@ -171,6 +171,15 @@ def init_params(ops, d, nodes, rng, node_jitter=0.01):
     return np.ascontiguousarray(params, dtype=np.float32)
 
 
+def layer_segments(ops, d):
+    """Offsets of the per-layer segments of the flat parameter vector: a segment starts at the weights
+    of every conv/linear layer and runs to the next layer's weights (so it also holds the norm
+    parameters or bias that follow), n_layers + 1 entries."""
+    starts = sorted(op["w_off"] for op in ops if op["op"] in ("conv", "linear"))
+    assert starts and starts[0] == 0
+    return np.array(starts + [d], np.int64)
+
+
 def make_labels(nodes, batch, classes, rng, dirichlet_alpha=None):
     if dirichlet_alpha is None:
         return rng.integers(0, classes, (nodes, batch)).astype(np.int32)
@@ -189,10 +198,13 @@ def make_workload(name, nodes=None, batch=None, seed=None, dirichlet_alpha=None)
     names: "conv16"       one 3x3 conv 16->16 on 16x16, 4 nodes x batch 8, 4 norm groups
            "resnet20"     16 nodes x batch 32, dense gossip, gamma 1
            "resnet20_topk" 40 nodes x batch 32, top-1% of the flattened update, gamma 0.1
+           "resnet20_topk_layerwise" the same with the paper's layer-wise top-K: one segment per
+                          conv/linear layer (its weights plus the norm parameters or bias that
+                          follow them), the top 1% of each kept
            "vgg11"        8 nodes x batch 32, dense gossip
     """
     defaults = dict(conv16=(4, 8, 0), resnet20=(16, 32, 1001), resnet20_topk=(40, 32, 1003),
-                    vgg11=(8, 32, 1002))
+                    resnet20_topk_layerwise=(40, 32, 1004), vgg11=(8, 32, 1002))
     dn, db, ds = defaults[name]
     nodes = dn if nodes is None else nodes
     batch = db if batch is None else batch
@@ -210,14 +222,17 @@ def make_workload(name, nodes=None, batch=None, seed=None, dirichlet_alpha=None)
     wl["ops"], wl["d"] = ops, d
     wl["params"] = init_params(ops, d, nodes, rng)
     wl["Wmix"] = ring_matrix(nodes)
-    if name == "resnet20_topk":
+    if name in ("resnet20_topk", "resnet20_topk_layerwise"):
         # public copies lag the models by a heavy-tailed residual, so that the
         # top 1% by magnitude is a non-trivial selection
         resid = rng.standard_normal((nodes, d)) * np.where(rng.random((nodes, d)) < 0.05, 1e-2, 1e-4)
         wl["x_hat"] = (wl["params"] - resid).astype(np.float32)
         wl["gamma"] = 0.1
-        wl["seg_offsets"] = np.array([0, d], np.int64)
-        wl["seg_k"] = np.array([max(1, d // 100)], np.int64)
+        if name == "resnet20_topk_layerwise":
+            wl["seg_offsets"] = layer_segments(ops, d)
+        else:
+            wl["seg_offsets"] = np.array([0, d], np.int64)
+        wl["seg_k"] = np.maximum(1, np.diff(wl["seg_offsets"]) // 100).astype(np.int64)
     else:
         wl["x_hat"] = np.zeros((nodes, d), np.float32)
         wl["seg_offsets"] = np.array([0, d], np.int64)

@@ -492,6 +492,34 @@ def test_gossip_topk_ties_across_chunks():
         close(xo, x_ref)
 
 
+def test_gossip_topk_candidate_list_with_planted_ties():
+    """Long segments of distinct magnitudes (the candidate-list path) with the threshold value planted a few
+    hundred times at scattered positions, so that only the ties at the lowest positions are kept; a second
+    segment of constant magnitude overflows its list and takes the whole-segment path in the same call."""
+    nodes, d1, d2, k1 = 3, 300000, 40000, 3000
+    d = d1 + d2
+    rng = np.random.default_rng(21)
+    xh = rng.standard_normal((nodes, d)).astype(np.float32)
+    for i in range(nodes):
+        mags = np.sort(np.abs(xh[i, :d1]))[::-1]
+        v = mags[k1 - 100]                                    # inside the top k1
+        pos = rng.choice(d1, size=400, replace=False)
+        xh[i, pos] = v * rng.choice(np.array([-1.0, 1.0], np.float32), size=400)
+    xh[:, d1:] = 0.75
+    xh[1, d1:] = 0.0                                          # all-zero differences
+    xhat = np.zeros((nodes, d), np.float32)
+    W = wlmod.ring_matrix(nodes)
+    so, sk = [0, d1, d], [k1, 12345]
+    x_ref, xhat_ref, q_ref = oracle.gossip_mix(xh, xhat, W, 0.4, so, sk)
+    assert all(np.count_nonzero(q_ref[i][:d1]) == k1 for i in range(nodes))
+    xhd, xhatd = dev(xh), dev(xhat)
+    xo = torch.empty_like(xhd)
+    ws = ws_bytes(api.lpdt_gossip_mix_workspace_size(nodes, d, 2))
+    api.lpdt_gossip_mix(nodes, d, xhd, xhatd, xo, dev(W), 0.4, so, sk, ws)
+    assert np.array_equal(xhatd.cpu().numpy(), xhat_ref)
+    close(xo, x_ref)
+
+
 @pytest.mark.parametrize("nodes,d,segs", [
     (4, 2736, None), (16, 10007, None), (8, 50000, [(0, 50000, 500)]),
     (5, 3000, [(0, 1000, 10), (1000, 1001, 1), (1001, 3000, 1999)]), (3, 1000, [(0, 1000, 0)]),

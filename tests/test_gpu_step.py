@@ -62,6 +62,16 @@ def test_resnet20_topk_step_small():
     assert all(np.count_nonzero(ref["q"][i]) == k for i in range(5))
 
 
+def test_resnet20_layerwise_topk_step_small():
+    """The paper's layer-wise top-K: one segment per layer (20 for this network), the top 1 % of each kept."""
+    wl = wlmod.make_workload("resnet20_topk_layerwise", nodes=5, batch=2)
+    assert len(wl["seg_k"]) == 20 and wl["seg_offsets"][-1] == wl["d"]
+    st, ref = _compare(wl)
+    for s in range(20):
+        lo, hi = int(wl["seg_offsets"][s]), int(wl["seg_offsets"][s + 1])
+        assert all(np.count_nonzero(ref["q"][i][lo:hi]) == int(wl["seg_k"][s]) for i in range(5))
+
+
 def test_vgg11_step_small():
     _compare(wlmod.make_workload("vgg11", nodes=2, batch=2))
 
@@ -122,17 +132,18 @@ def _compare_sampled_nodes(wl, sel):
     # mix, from the GPU's own x_half (properties only)
     xh = st.x_half.cpu().numpy(); xhat0 = wl["x_hat"]; xhat1 = st.x_hat.cpu().numpy()
     q = xhat1 - xhat0
-    k = int(wl["seg_k"][0])
-    if k < wl["d"]:
-        delta = xh - xhat0
+    delta = xh - xhat0
+    for s, k in enumerate(int(v) for v in wl["seg_k"]):
+        lo, hi = int(wl["seg_offsets"][s]), int(wl["seg_offsets"][s + 1])
+        if k >= hi - lo:
+            assert np.array_equal(xhat1[:, lo:hi], xh[:, lo:hi])
+            continue
         for i in range(wl["nodes"]):
-            nz = np.flatnonzero(q[i])
+            nz = np.flatnonzero(q[i, lo:hi])
             assert len(nz) <= k and len(nz) >= k - 8           # exact zeros among the kept deltas are possible
-            keptmin = np.abs(delta[i, nz]).min()
-            dropped = np.setdiff1d(np.arange(wl["d"]), nz)
-            assert keptmin >= np.abs(delta[i, dropped]).max()
-    else:
-        assert np.array_equal(xhat1, xh)
+            keptmin = np.abs(delta[i, lo:hi][nz]).min()
+            dropped = np.setdiff1d(np.arange(hi - lo), nz)
+            assert keptmin >= np.abs(delta[i, lo:hi][dropped]).max()
     assert np.allclose(st.x_out.double().sum(0).cpu().numpy(), xh.astype(np.float64).sum(0),
                        atol=1e-5 * wl["nodes"] * max(1.0, float(np.abs(xh).max())))
 
@@ -143,6 +154,10 @@ def test_vgg11_full_size_sampled_nodes():
 
 def test_resnet20_topk_full_size_sampled_nodes():
     _compare_sampled_nodes(wlmod.make_workload("resnet20_topk"), [0, 17, 39])
+
+
+def test_resnet20_layerwise_topk_full_size_sampled_nodes():
+    _compare_sampled_nodes(wlmod.make_workload("resnet20_topk_layerwise"), [3, 22])
 
 
 def test_resnet20_topk_40_nodes():

@@ -126,3 +126,18 @@ def test_network_step_tracks_float_model(name):
         sl = slice(0, first["cout"] * 9 * first["cin"])
         assert _cos(out["grads"][n, sl], gref[sl]) > 0.8
         assert _cos(out["grads"][n], gref) > 0.9
+
+
+def test_layerwise_topk_segments_tile_the_parameters():
+    """Layer-wise top-K: one segment per conv/linear layer, tiling the flat parameter vector; the oracle
+    step keeps exactly seg_k entries of every (node, segment)."""
+    wl = wlmod.make_workload("resnet20_topk_layerwise", nodes=3, batch=2)
+    off, k = wl["seg_offsets"], wl["seg_k"]
+    assert off[0] == 0 and off[-1] == wl["d"] and (np.diff(off) > 0).all() and len(k) == 20
+    starts = [op["w_off"] for op in wl["ops"] if op["op"] in ("conv", "linear")]
+    assert list(off[:-1]) == starts
+    ref = ostep.train_step(wl)
+    for s in range(len(k)):
+        for i in range(3):
+            assert np.count_nonzero(ref["q"][i][off[s]:off[s + 1]]) == k[s]
+    assert np.array_equal(ref["x_hat"], (wl["x_hat"] + ref["q"]).astype(np.float32))
