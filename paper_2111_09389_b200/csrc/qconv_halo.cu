@@ -41,6 +41,9 @@ struct HaloParams {
     int PH, PW;                // halo rows / pixels per row
     int tilesH, tilesW;
     int stages, halo_bytes, wres_bytes, tmem_cols;
+    int nacc_log2;             // log2 of the number of TMEM accumulators (2, 4 or 8 tiles in flight)
+    int tma_out;               // fp32 result leaves through shared memory and bulk tensor stores
+    int out_inner;             // channels per store box: 32 (128-byte swizzled rows) or 16 (64-byte)
     int w_rows_per_node;
     float *Y; int32_t *Yacc;
     const float *s1, *s2, *bias; long long bias_stride;
@@ -48,7 +51,8 @@ struct HaloParams {
 };
 
 struct HaloCtl {
-    unsigned long long full[8], empty[8], tmem_full[2], tmem_empty[2], wfull;
+    unsigned long long full[8], empty[8], tmem_full[8], tmem_empty[8], wfull;
+    unsigned long long out_full[2], out_free[2];      // result tiles in shared memory: written by the 4 epilogue warps / read by the store
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -70,12 +74,14 @@ __device__ __forceinline__ void halo_next(const HaloParams &p, HaloTile &c) {
 
 __global__ void __launch_bounds__(kHaloThreads, 1)
 conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapW,
-                   const HaloParams p) {
+                   const __grid_constant__ CUtensorMap mapY, const HaloParams p) {
     extern __shared__ __align__(1024) unsigned char smem[];
     HaloCtl *ctl = reinterpret_cast<HaloCtl *>(smem);
     unsigned char *wres = smem + 1024;
     unsigned char *stage0 = wres + p.wres_bytes;
     unsigned char *zeros = stage0 + (size_t)p.stages * p.halo_bytes;     // above every tile: offsets to it are positive
+    // two result tiles of 128 x N fp32 (tma_out), on a swizzle-atom boundary
+    unsigned char *out_tiles = smem + (((size_t)(zeros - smem) + kZeroBytes + 1023) & ~(size_t)1023);
     // warp index and TMEM base are broadcast through a shuffle so that the compiler knows they are
     // warp-uniform and keeps the role loops on the uniform datapath
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
@@ -87,8 +93,9 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
     for (int i = threadIdx.x; i < p.wres_bytes / 4; i += blockDim.x) reinterpret_cast<uint32_t *>(wres)[i] = 0u;
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.stages; ++i) { mbar_init(smem_u32(&ctl->full[i]), 1); mbar_init(smem_u32(&ctl->empty[i]), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&ctl->tmem_full[i]), 1); mbar_init(smem_u32(&ctl->tmem_empty[i]), 4); }
+        for (int i = 0; i < 8; ++i) { mbar_init(smem_u32(&ctl->tmem_full[i]), 1); mbar_init(smem_u32(&ctl->tmem_empty[i]), 4); }
         mbar_init(smem_u32(&ctl->wfull), 1);
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&ctl->out_full[i]), 4); mbar_init(smem_u32(&ctl->out_free[i]), 1); }
         ctl->abort_flag = 0;
         mbar_fence_init();
     }
@@ -170,8 +177,8 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
                     if (!mbar_wait(smem_u32(&ctl->wfull), wph, &ctl->abort_flag, p.dev_status)) break;
                     wph ^= 1; cur_node = c.node;
                 }
-                const int acc = tcount & 1;
-                const uint32_t aph = (tcount >> 1) & 1;
+                const int acc = tcount & ((1u << p.nacc_log2) - 1u);
+                const uint32_t aph = (tcount >> p.nacc_log2) & 1;
                 if (!mbar_wait(smem_u32(&ctl->tmem_empty[acc]), aph ^ 1, &ctl->abort_flag, p.dev_status)) break;
                 if (!mbar_wait(smem_u32(&ctl->full[st]), ph, &ctl->abort_flag, p.dev_status)) break;
                 tc_fence_after();
@@ -197,19 +204,69 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
         const int q = warp & 3;
         const int row = q * 32 + lane;
         const int pw = row % kTileW, phh = row / kTileW;
+        const bool issuer = (warp == 2 && lane == 0);        // issues and tracks the bulk stores
         uint32_t tcount = 0;
         HaloTile c = halo_decode(p, tile_lo);
         int sc_node = -1; float sc = 0.f;
+        if (p.tma_out && issuer) tma_prefetch_desc(&mapY);
         for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; ++tile, ++tcount, halo_next(p, c)) {
             const int w = c.tw * kTileW + pw, h = c.th * kTileH + phh;
             const bool valid = (w < p.Wm) && (h < p.Hm);
             if (p.Y && c.node != sc_node) { sc_node = c.node; sc = __fmul_rn(p.s1[c.node], p.s2[c.node]); }
-            const int acc = tcount & 1;
-            const uint32_t aph = (tcount >> 1) & 1;
+            const int acc = tcount & ((1u << p.nacc_log2) - 1u);
+            const uint32_t aph = (tcount >> p.nacc_log2) & 1;
             if (!mbar_wait(smem_u32(&ctl->tmem_full[acc]), aph, &ctl->abort_flag, p.dev_status)) break;
             tc_fence_after();
             const long long pix = (((long long)c.node * p.B + c.b) * p.Hm + h) * p.Wm + w;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * p.N;
+            if (p.tma_out) {
+                // Result tile -> shared memory (pixel-major, the layout of the store's box) -> one bulk tensor
+                // store per tile; parts of the box outside the image are not written.  Two tile buffers: the
+                // store of the tile before last must have finished reading this one.
+                const int ob = tcount & 1u;
+                const uint32_t use = tcount >> 1;
+                unsigned char *ot = out_tiles + (size_t)ob * 128 * p.N * 4;
+                if (use > 0 && !mbar_wait(smem_u32(&ctl->out_free[ob]), (use - 1) & 1, &ctl->abort_flag, p.dev_status)) break;
+                const int inner = p.out_inner;
+                const uint32_t sw = inner == 32 ? (uint32_t)(row & 7) : (uint32_t)((row >> 1) & 3);   // the box's swizzle
+                for (int cc = 0; cc < p.N; cc += 16) {
+                    uint32_t v[16];
+                    tmem_ld_32x16(t_row + cc, v);
+                    tmem_ld_wait();
+                    float f[16];
+#pragma unroll
+                    for (int k = 0; k < 16; ++k) {
+                        f[k] = __fmul_rn(__int2float_rn((int)v[k]), sc);
+                        if (p.bias) f[k] = __fadd_rn(f[k], p.bias[(long long)c.node * p.bias_stride + cc + k]);
+                    }
+                    const int g = cc / inner, k0 = (cc % inner) >> 2;
+                    float4 *grow = reinterpret_cast<float4 *>(ot + ((size_t)g * 128 + row) * inner * 4);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        grow[(uint32_t)(k0 + k) ^ sw] = make_float4(f[4 * k], f[4 * k + 1], f[4 * k + 2], f[4 * k + 3]);
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+                fence_proxy_async_smem();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->out_full[ob]));
+                int ok = 1;
+                if (issuer) {
+                    ok = mbar_wait(smem_u32(&ctl->out_full[ob]), use & 1, &ctl->abort_flag, p.dev_status) ? 1 : 0;
+                    if (ok) {
+                        for (int g = 0; g * p.out_inner < p.N; ++g)
+                            tma_store_5d(&mapY, smem_u32(ot + (size_t)g * 128 * p.out_inner * 4), g * p.out_inner,
+                                         c.tw * kTileW, c.th * kTileH, c.b, c.node);
+                        tma_store_commit();
+                        // every store but this one has finished reading: the other buffer may be written again
+                        tma_store_wait_read<1>();
+                        if (tcount > 0) mbar_arrive(smem_u32(&ctl->out_free[ob ^ 1]));
+                    }
+                }
+                if (warp == 2 && !__shfl_sync(0xffffffffu, ok, 0)) break;     // the whole warp leaves together
+                continue;
+            }
             for (int cc = 0; cc < p.N; cc += 16) {
                 uint32_t v[16];
                 tmem_ld_32x16(t_row + cc, v);
@@ -239,6 +296,7 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
         }
+        if (p.tma_out && issuer) tma_store_wait_all();       // the tiles in shared memory have been read and written out
     }
     tc_fence_before();
     __syncthreads();
@@ -312,11 +370,19 @@ lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, cons
     // several resident CTAs hide each other's latencies.  As many as leave every CTA at least four stages
     // and fit TMEM (512 columns per SM): shared memory is sized so that no further CTA becomes resident and
     // a TMEM allocation never has to wait.
-    p.tmem_cols = halo_pow2(2 * p.N);
+    // TMEM accumulators: as many tiles in flight between the MMA warp and the epilogue warps as 128 columns
+    // hold (8 at N = 16, 4 at N = 32, 2 from N = 64 on), so that the MMA warp does not wait for the epilogue's
+    // round trip on these short tiles
+    p.nacc_log2 = p.N <= 16 ? 3 : p.N <= 32 ? 2 : 1;
+    p.tmem_cols = halo_pow2((1 << p.nacc_log2) * p.N);
+    // fp32 result through shared memory and bulk tensor stores (not when the raw accumulators are asked for)
+    p.tma_out = (Y && !Yacc && aligned(Y, 16)) ? 1 : 0;
+    p.out_inner = p.N % 32 == 0 ? 32 : 16;
+    const int out_bytes = p.tma_out ? 2 * 128 * p.N * 4 + 1024 : 0;          // + slack to reach a 1024-byte boundary
     int per_sm = 4, stages = 0;
     for (;; --per_sm) {
         const int budget = (224 * 1024) / per_sm - 2048;
-        stages = (budget - 1024 - p.wres_bytes - kZeroBytes) / p.halo_bytes;
+        stages = (budget - 1024 - p.wres_bytes - kZeroBytes - out_bytes) / p.halo_bytes;
         if (stages > 8) stages = 8;
         if (per_sm == 1 || (stages >= 4 && per_sm * p.tmem_cols <= 512)) break;
     }
@@ -325,7 +391,12 @@ lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, cons
     p.w_rows_per_node = d.Cout;
     p.Y = Y; p.Yacc = Yacc; p.s1 = s1; p.s2 = s2; p.bias = bias; p.bias_stride = bias_stride;
     p.dev_status = dev_status;
-    CUtensorMap mA, mW;
+    CUtensorMap mA, mW, mY;
+    if (p.tma_out) {
+        if (!make_map_out_f32(&mY, Y, d.nodes, d.B, p.Hm, p.Wm, p.N, p.out_inner, kTileH, kTileW)) return LPDT_ERR_CUDA;
+    } else {
+        mY = CUtensorMap{};
+    }
     if (p.cpt > 1) {   // 16-byte chunk rows; the chunk index is the outermost box dimension
         uint64_t dims[5] = {16, (uint64_t)Wa, (uint64_t)Ha, (uint64_t)d.nodes * d.B, (uint64_t)p.cpt};
         uint64_t strides[4] = {(uint64_t)Kc, (uint64_t)Wa * Kc, (uint64_t)Ha * Wa * Kc, 16};
@@ -343,7 +414,7 @@ lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, cons
         uint32_t box[3] = {16, 1, (uint32_t)(mode == 0 ? p.N : 16)};
         if (!make_map_u8(&mW, Wq, 3, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_NONE)) return LPDT_ERR_CUDA;
     }
-    size_t smem = 1024 + (size_t)p.wres_bytes + (size_t)p.stages * p.halo_bytes + kZeroBytes;
+    size_t smem = 1024 + (size_t)p.wres_bytes + (size_t)p.stages * p.halo_bytes + kZeroBytes + out_bytes;
     const size_t smem_floor = (size_t)(228 * 1024) / (per_sm + 1);     // keeps the (per_sm + 1)-th CTA out
     if (smem < smem_floor) smem = smem_floor;
     static bool attr = false;
@@ -354,7 +425,7 @@ lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, cons
     const long long tiles = (long long)p.nodes * p.B * p.tilesH * p.tilesW;
     if (tiles > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
     const int grid = (int)(tiles < (long long)kNumSMs * per_sm ? tiles : (long long)kNumSMs * per_sm);
-    launch_k(conv_halo16_kernel, grid, kHaloThreads, smem, st, mA, mW, p);
+    launch_k(conv_halo16_kernel, grid, kHaloThreads, smem, st, mA, mW, mY, p);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

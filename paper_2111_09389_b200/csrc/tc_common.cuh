@@ -98,6 +98,25 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap *map
         " [%0], [%1, {%3, %4, %5, %6, %7}], [%2];"
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
 }
+// Bulk tensor store shared -> global (bulk-group completion), and the group waits.  Box parts outside the
+// tensor are not written.
+__device__ __forceinline__ void tma_store_5d(const CUtensorMap *map, uint32_t src, int c0, int c1, int c2, int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];"
+        ::"l"(map), "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4) : "memory");
+}
+__device__ __forceinline__ void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// at most N of this thread's store groups still read their shared-memory source
+template <int N> __device__ __forceinline__ void tma_store_wait_read() {
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// generic-proxy writes to shared memory become visible to the async proxy (TMA, tensor core)
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// named barrier among `count` threads of the CTA (id 0 is __syncthreads)
+__device__ __forceinline__ void named_bar_sync(int id, int count) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(count) : "memory");
+}
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap *map) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
 }
@@ -196,21 +215,38 @@ static inline EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// Byte tensor, rank <= 5.  dims[0] is the contiguous dimension; strides[i] is the
-// byte stride of dims[i+1] (multiples of 16).  Out-of-range box elements read zero.
-static inline bool make_map_u8(CUtensorMap *map, const void *base, int rank, const uint64_t *dims,
-                               const uint64_t *strides, const uint32_t *box, CUtensorMapSwizzle swz,
-                               const uint32_t *elem_strides = nullptr) {
+// Tensor of bytes (or of 32-bit words), rank <= 5.  dims[0] is the contiguous dimension, in elements;
+// strides[i] is the byte stride of dims[i+1] (multiples of 16).  Out-of-range box elements read zero
+// and are not written by stores.
+static inline bool make_map(CUtensorMap *map, CUtensorMapDataType dtype, const void *base, int rank, const uint64_t *dims,
+                            const uint64_t *strides, const uint32_t *box, CUtensorMapSwizzle swz,
+                            const uint32_t *elem_strides = nullptr) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
     cuuint64_t d[5], s[4];
     cuuint32_t b[5], e[5];
     for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; e[i] = elem_strides ? elem_strides[i] : 1; }
     for (int i = 0; i + 1 < rank; ++i) s[i] = strides[i];
-    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void *>(base), d, s, b, e,
+    CUresult r = fn(map, dtype, (cuuint32_t)rank, const_cast<void *>(base), d, s, b, e,
                     CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
+}
+static inline bool make_map_u8(CUtensorMap *map, const void *base, int rank, const uint64_t *dims,
+                               const uint64_t *strides, const uint32_t *box, CUtensorMapSwizzle swz,
+                               const uint32_t *elem_strides = nullptr) {
+    return make_map(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, base, rank, dims, strides, box, swz, elem_strides);
+}
+// fp32 NHWC result [nodes][B][H][W][C] with a box of TW x TH pixels x `inner` channels (16 or 32): the
+// shared-memory image of the box has rows of 64 or 128 bytes and the matching swizzle, so that a warp writing
+// one row per lane spreads over all banks.
+static inline bool make_map_out_f32(CUtensorMap *map, float *base, int nodes, int B, int H, int W, int C, int inner,
+                                    int TH, int TW) {
+    uint64_t dims[5] = {(uint64_t)C, (uint64_t)W, (uint64_t)H, (uint64_t)B, (uint64_t)nodes};
+    uint64_t strides[4] = {(uint64_t)C * 4, (uint64_t)W * C * 4, (uint64_t)H * W * C * 4, (uint64_t)B * H * W * C * 4};
+    uint32_t box[5] = {(uint32_t)inner, (uint32_t)TW, (uint32_t)TH, 1, 1};
+    return make_map(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, base, 5, dims, strides, box,
+                    inner == 32 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B);
 }
 
 }  // namespace tc

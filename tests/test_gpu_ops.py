@@ -242,6 +242,16 @@ def test_qconv_all_three(case):
                        ws=ws, dev_status=status)
     assert np.array_equal(Yacc.cpu().numpy(), acc_ref)
     assert np.array_equal(Y.cpu().numpy(), oracle.dequant_acc(acc_ref, s1, s2, bias[:, 3:]))
+    # fp32-only output (the path the training step takes; results may leave through bulk tensor stores):
+    # same values, every element written, nothing written outside the tensor
+    def guarded(shape):
+        n = int(np.prod(shape))
+        buf = torch.full((n + 2048,), float("nan"), dtype=torch.float32, device="cuda")
+        return buf, buf[1024:1024 + n].view(*shape)
+    buf, Y2 = guarded(acc_ref.shape)
+    api.lpdt_qconv_fwd(desc, Ad, s1d, Wd, s2d, Y=Y2, bias=dev(bias)[:, 3:], bias_node_stride=Cout + 3, ws=ws,
+                       dev_status=status)
+    assert torch.equal(Y2, Y) and bool(buf[:1024].isnan().all()) and bool(buf[-1024:].isnan().all())
     # backward data
     dA_ref, _ = oracle.qconv_bwd_data(E, Wq, H, W, stride, pad)
     dA = torch.empty(dA_ref.shape, dtype=torch.float32, device="cuda")
@@ -249,6 +259,9 @@ def test_qconv_all_three(case):
     api.lpdt_qconv_bwd_data(desc, Ed, s1d, Wd, s2d, dA=dA, dAacc=dAacc, ws=ws, dev_status=status)
     assert np.array_equal(dAacc.cpu().numpy(), dA_ref)
     assert np.array_equal(dA.cpu().numpy(), oracle.dequant_acc(dA_ref, s1, s2))
+    buf, dA2 = guarded(dA_ref.shape)
+    api.lpdt_qconv_bwd_data(desc, Ed, s1d, Wd, s2d, dA=dA2, ws=ws, dev_status=status)
+    assert torch.equal(dA2, dA) and bool(buf[:1024].isnan().all()) and bool(buf[-1024:].isnan().all())
     # backward weight, into a strided gradient vector
     dW_ref, _ = oracle.qconv_bwd_weight(E, A, R, S, stride, pad)
     wn = Cout * R * S * Cin
