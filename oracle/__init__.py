@@ -207,6 +207,59 @@ def range_evonorm_bwd(dy, x, v, gamma, gmin, gmax, argmin, argmax, groups, eps, 
     return dx, dv, dg, db
 
 
+def evonorm_s0_fwd(x, v, gamma, beta, groups, eps):
+    """EvoNorm-S0 in double.  Returns (y, gmean, gvar); statistics are [n,B,groups]."""
+    x = _c(x, np.float32)
+    n, B, H, W, Cc = x.shape
+    v = _c(v, np.float32); gamma = _c(gamma, np.float32); beta = _c(beta, np.float32)
+    y = np.zeros(x.shape, np.float64)
+    gmean = np.zeros((n, B, groups), np.float64); gvar = np.zeros((n, B, groups), np.float64)
+    lib().orc_evonorm_s0_fwd(n, B, H, W, Cc, groups, C.c_double(eps), _p(x), _p(v), _p(gamma), _p(beta), _p(y),
+                             _p(gmean), _p(gvar))
+    return y, gmean, gvar
+
+
+def evonorm_s0_bwd(dy, x, v, gamma, gmean, gvar, groups, eps):
+    """gmean, gvar: the stored fp32 statistics.  Returns (dx, dv, dgamma, dbeta) in double."""
+    x = _c(x, np.float32); dy = _c(dy, np.float32)
+    n, B, H, W, Cc = x.shape
+    v = _c(v, np.float32); gamma = _c(gamma, np.float32)
+    gmean = _c(gmean, np.float32); gvar = _c(gvar, np.float32)
+    dx = np.zeros(x.shape, np.float64)
+    dv = np.zeros((n, Cc), np.float64); dg = np.zeros((n, Cc), np.float64); db = np.zeros((n, Cc), np.float64)
+    lib().orc_evonorm_s0_bwd(n, B, H, W, Cc, groups, C.c_double(eps), _p(dy), _p(x), _p(v), _p(gamma), _p(gmean),
+                             _p(gvar), _p(dx), _p(dv), _p(dg), _p(db))
+    return dx, dv, dg, db
+
+
+def range_bn_fwd(x, gamma, beta, eps):
+    """Range batch-norm in double.  Returns (y, cmean, cmin, cmax, argmin, argmax); statistics are [n,C]."""
+    x = _c(x, np.float32)
+    n, B, H, W, Cc = x.shape
+    gamma = _c(gamma, np.float32); beta = _c(beta, np.float32)
+    y = np.zeros(x.shape, np.float64)
+    cmean = np.zeros((n, Cc), np.float64)
+    cmin = np.zeros((n, Cc), np.float32); cmax = np.zeros((n, Cc), np.float32)
+    amin = np.zeros((n, Cc), np.int32); amax = np.zeros((n, Cc), np.int32)
+    lib().orc_range_bn_fwd(n, B, H, W, Cc, C.c_double(eps), _p(x), _p(gamma), _p(beta), _p(y), _p(cmean), _p(cmin),
+                           _p(cmax), _p(amin), _p(amax))
+    return y, cmean, cmin, cmax, amin, amax
+
+
+def range_bn_bwd(dy, x, gamma, cmean, cmin, cmax, argmin, argmax, eps):
+    """cmean: the stored fp32 mean.  Returns (dx, dgamma, dbeta) in double."""
+    x = _c(x, np.float32); dy = _c(dy, np.float32)
+    n, B, H, W, Cc = x.shape
+    gamma = _c(gamma, np.float32); cmean = _c(cmean, np.float32)
+    cmin = _c(cmin, np.float32); cmax = _c(cmax, np.float32)
+    argmin = _c(argmin, np.int32); argmax = _c(argmax, np.int32)
+    dx = np.zeros(x.shape, np.float64)
+    dg = np.zeros((n, Cc), np.float64); db = np.zeros((n, Cc), np.float64)
+    lib().orc_range_bn_bwd(n, B, H, W, Cc, C.c_double(eps), _p(dy), _p(x), _p(gamma), _p(cmean), _p(cmin), _p(cmax),
+                           _p(argmin), _p(argmax), _p(dx), _p(dg), _p(db))
+    return dx, dg, db
+
+
 def gossip_mix(x_half, x_hat, Wmix, gamma, seg_offsets=None, seg_k=None):
     """x_half, x_hat fp32 [n,d]; Wmix [n,n].  Returns (x_out, x_hat_new, q)."""
     x_half = _c(x_half, np.float32)

@@ -365,6 +365,163 @@ void orc_dequant_acc(const int32_t *acc, int nodes, i64 n_per_node, int C,
 #undef SUFFIX
 
 /* ------------------------------------------------------------------------
+ * The comparison layers of Section 3 (Eq. "en" and Eq. "rbn"), in double.
+ * ---------------------------------------------------------------------- */
+
+/* EvoNorm-S0 (Eq. "en"), per node n, sample b, group G of cpg = C/groups consecutive channels:
+ *     mu, var = mean and (biased) variance of x over the group's (h, w, c)
+ *     D       = sqrt(var + eps)
+ *     y       = gamma_c * (x * sigmoid(v_c * x)) / D + beta_c
+ * The equation has no eps (eps = 0 reproduces it) and does not say which variance; the divide-by-count
+ * form is the reading taken.  gmean / gvar [nodes][B][groups] receive the statistics. */
+void orc_evonorm_s0_fwd(int nodes, int B, int H, int W, int C, int groups, double eps,
+                        const float *x, const float *v, const float *gamma, const float *beta,
+                        double *y, double *gmean, double *gvar)
+{
+    const int cpg = C / groups;
+    const double cnt = (double)H * W * cpg;
+    for (int n = 0; n < nodes; ++n)
+    for (int b = 0; b < B; ++b)
+    for (int g = 0; g < groups; ++g) {
+        const float *xs = x + ((i64)n * B + b) * H * W * C;
+        double *ys = y + ((i64)n * B + b) * H * W * C;
+        double sum = 0.0;
+        for (int p = 0; p < H * W; ++p)
+            for (int c = g * cpg; c < (g + 1) * cpg; ++c) sum += (double)xs[p * C + c];
+        const double mu = sum / cnt;
+        double sq = 0.0;
+        for (int p = 0; p < H * W; ++p)
+            for (int c = g * cpg; c < (g + 1) * cpg; ++c) {
+                double dlt = (double)xs[p * C + c] - mu;
+                sq += dlt * dlt;
+            }
+        const double var = sq / cnt;
+        const i64 sg = ((i64)n * B + b) * groups + g;
+        gmean[sg] = mu; gvar[sg] = var;
+        const double D = sqrt(var + eps);
+        for (int p = 0; p < H * W; ++p)
+            for (int c = g * cpg; c < (g + 1) * cpg; ++c) {
+                double xv = (double)xs[p * C + c];
+                double sig = 1.0 / (1.0 + exp(-(double)v[(i64)n * C + c] * xv));
+                ys[p * C + c] = (double)gamma[(i64)n * C + c] * (xv * sig) / D + (double)beta[(i64)n * C + c];
+            }
+    }
+}
+
+/* Backward of EvoNorm-S0 (derived from the forward; the paper prints none).  With t = dy*gamma_c,
+ * sig = sigmoid(v_c x), m = x*sig, cnt = H*W*cpg and S = sum over the group of t*m:
+ *     dx      = t * (sig + v_c*x*sig*(1 - sig)) / D  -  S * (x - mu) / (cnt * D^3)
+ *     dbeta_c = sum dy;  dgamma_c = sum dy * m / D;  dv_c = sum t * x*x*sig*(1 - sig) / D
+ * (sums over the node's b, h, w).  gmean / gvar are the forward's statistics as the caller stored them. */
+void orc_evonorm_s0_bwd(int nodes, int B, int H, int W, int C, int groups, double eps,
+                        const float *dy, const float *x, const float *v, const float *gamma,
+                        const float *gmean, const float *gvar,
+                        double *dx, double *dv, double *dgamma, double *dbeta)
+{
+    const int cpg = C / groups;
+    const double cnt = (double)H * W * cpg;
+    for (i64 i = 0; i < (i64)nodes * C; ++i) { dv[i] = 0.0; dgamma[i] = 0.0; dbeta[i] = 0.0; }
+    for (int n = 0; n < nodes; ++n)
+    for (int b = 0; b < B; ++b)
+    for (int g = 0; g < groups; ++g) {
+        const float *xs = x + ((i64)n * B + b) * H * W * C;
+        const float *dys = dy + ((i64)n * B + b) * H * W * C;
+        double *dxs = dx + ((i64)n * B + b) * H * W * C;
+        const i64 sg = ((i64)n * B + b) * groups + g;
+        const double mu = (double)gmean[sg], D = sqrt((double)gvar[sg] + eps);
+        double S = 0.0;
+        for (int p = 0; p < H * W; ++p)
+            for (int c = g * cpg; c < (g + 1) * cpg; ++c) {
+                double xv = (double)xs[p * C + c], vc = (double)v[(i64)n * C + c];
+                double sig = 1.0 / (1.0 + exp(-vc * xv));
+                S += (double)dys[p * C + c] * (double)gamma[(i64)n * C + c] * (xv * sig);
+            }
+        for (int p = 0; p < H * W; ++p)
+            for (int c = g * cpg; c < (g + 1) * cpg; ++c) {
+                double xv = (double)xs[p * C + c], vc = (double)v[(i64)n * C + c];
+                double gc = (double)gamma[(i64)n * C + c], dyv = (double)dys[p * C + c];
+                double sig = 1.0 / (1.0 + exp(-vc * xv));
+                double m = xv * sig, t = dyv * gc, sp = sig * (1.0 - sig);
+                dxs[p * C + c] = t * (sig + vc * xv * sp) / D - S * (xv - mu) / (cnt * D * D * D);
+                dbeta[(i64)n * C + c] += dyv;
+                dgamma[(i64)n * C + c] += dyv * m / D;
+                dv[(i64)n * C + c] += t * xv * xv * sp / D;
+            }
+    }
+}
+
+/* Range batch-norm (Eq. "rbn"), per node n and channel c over the node's batch (b, h, w):
+ *     mu    = mean of x;  range = max(x - mu) - min(x - mu) = max x - min x
+ *     D     = Cb * range + eps,  Cb = 1/sqrt(2 ln B)  (the equation's C(b), b = batch size; B >= 2)
+ *     y     = gamma_c * (x - mu) / D + beta_c
+ * cmean / cmin / cmax [nodes][C] receive the statistics, argmin / argmax the lowest (b*H*W + p)
+ * position attaining the extremum (for the backward's sub-gradient, as in Range-EvoNorm). */
+void orc_range_bn_fwd(int nodes, int B, int H, int W, int C, double eps,
+                      const float *x, const float *gamma, const float *beta,
+                      double *y, double *cmean, float *cmin, float *cmax, int32_t *argmin, int32_t *argmax)
+{
+    const double Cb = 1.0 / sqrt(2.0 * log((double)B));
+    const i64 P = (i64)B * H * W;
+    for (int n = 0; n < nodes; ++n)
+    for (int c = 0; c < C; ++c) {
+        const float *xs = x + (i64)n * P * C;
+        double *ys = y + (i64)n * P * C;
+        double sum = 0.0;
+        float mx = 0, mn = 0; int32_t amx = -1, amn = -1;
+        for (i64 p = 0; p < P; ++p) {
+            float val = xs[p * C + c];
+            sum += (double)val;
+            if (amx < 0 || val > mx) { mx = val; amx = (int32_t)p; }
+            if (amn < 0 || val < mn) { mn = val; amn = (int32_t)p; }
+        }
+        const double mu = sum / (double)P;
+        cmean[(i64)n * C + c] = mu; cmin[(i64)n * C + c] = mn; cmax[(i64)n * C + c] = mx;
+        argmin[(i64)n * C + c] = amn; argmax[(i64)n * C + c] = amx;
+        const double D = Cb * ((double)mx - (double)mn) + eps;
+        for (i64 p = 0; p < P; ++p)
+            ys[p * C + c] = (double)gamma[(i64)n * C + c] * ((double)xs[p * C + c] - mu) / D + (double)beta[(i64)n * C + c];
+    }
+}
+
+/* Backward of range batch-norm (derived).  With t = dy*gamma_c, P = B*H*W, xc = x - mu:
+ *     dx      = t / D - (sum t) / (P * D) - Cb * (sum t*xc) / D^2 * ([p = argmax] - [p = argmin])
+ *     dbeta_c = sum dy;  dgamma_c = sum dy * xc / D
+ * (the last dx term is skipped when argmax = argmin). */
+void orc_range_bn_bwd(int nodes, int B, int H, int W, int C, double eps,
+                      const float *dy, const float *x, const float *gamma,
+                      const float *cmean, const float *cmin, const float *cmax,
+                      const int32_t *argmin, const int32_t *argmax,
+                      double *dx, double *dgamma, double *dbeta)
+{
+    const double Cb = 1.0 / sqrt(2.0 * log((double)B));
+    const i64 P = (i64)B * H * W;
+    for (int n = 0; n < nodes; ++n)
+    for (int c = 0; c < C; ++c) {
+        const float *xs = x + (i64)n * P * C;
+        const float *dys = dy + (i64)n * P * C;
+        double *dxs = dx + (i64)n * P * C;
+        const i64 nc = (i64)n * C + c;
+        const double mu = (double)cmean[nc], gc = (double)gamma[nc];
+        const double D = Cb * ((double)cmax[nc] - (double)cmin[nc]) + eps;
+        double sdy = 0.0, sdx = 0.0;          /* sum dy, sum dy*xc */
+        for (i64 p = 0; p < P; ++p) {
+            double dyv = (double)dys[p * C + c], xc = (double)xs[p * C + c] - mu;
+            sdy += dyv; sdx += dyv * xc;
+        }
+        const double st = gc * sdy, stx = gc * sdx;
+        for (i64 p = 0; p < P; ++p)
+            dxs[p * C + c] = (double)dys[p * C + c] * gc / D - st / ((double)P * D);
+        if (argmax[nc] != argmin[nc]) {
+            const double coef = Cb * stx / (D * D);
+            dxs[(i64)argmax[nc] * C + c] -= coef;
+            dxs[(i64)argmin[nc] * C + c] += coef;
+        }
+        dbeta[nc] = sdy;
+        dgamma[nc] = sdx / D;
+    }
+}
+
+/* ------------------------------------------------------------------------
  * Gossip with compressed model updates (Algorithm 3, CHOCO-SGD, the steps
  * "compute and compress", "update the public copies", "gossip update").
  *   delta_i = xhalf_i - xhat_i                      (fp32: it decides the top-k)
