@@ -254,6 +254,56 @@ lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t H, int32_t 
                                    void *ws, size_t ws_bytes, void *stream);
 
 /* ---------------------------------------------------------------------------
+ * Comparison layers of Section 3 (the normalization study; not on the 8-bit path).
+ *
+ * lpdt_evonorm_s0_fwd / _bwd — EvoNorm-S0 (Eq. "en"), the layer the paper trains with at full
+ * precision.  Per node, sample and group of cpg = C/groups consecutive channels:
+ *   mu, var = mean and divide-by-count variance of x over the group's (h, w, c)
+ *   D = sqrt(var + eps);   y = gamma_c * (x * sigmoid(v_c*x)) / D + beta_c
+ * (the equation has no eps: eps = 0 reproduces it).  Backward, derived, with t = dy*gamma_c,
+ * sig = sigmoid(v_c*x), m = x*sig, cnt = H*W*cpg and S = sum over the group of t*m:
+ *   dx = t*(sig + v_c*x*sig*(1 - sig))/D - S*(x - mu)/(cnt*D^3)
+ *   dbeta_c = sum dy;  dgamma_c = sum dy*m/D;  dv_c = sum t*x*x*sig*(1 - sig)/D   (over b, h, w)
+ * Layouts as lpdt_range_evonorm_*: x, y, dy, dx fp32 NHWC; parameters per node at p + n*param_node_stride;
+ * gmean, gvar : fp32 [nodes][B][groups], written by the forward, read by the backward.
+ * Statistics and parameter-gradient sums are accumulated in double; elementwise work is fp32.
+ * Errors: INVALID_ARG, UNSUPPORTED (more than 256 channel vectors), WORKSPACE, CUDA.
+ */
+lpdt_status lpdt_evonorm_s0_fwd(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C, int32_t groups,
+                                float eps, const float *x, const float *v, const float *gamma, const float *beta,
+                                int64_t param_node_stride, float *y, float *gmean, float *gvar, void *stream);
+size_t lpdt_evonorm_s0_bwd_workspace_size(int32_t nodes, int32_t B, int32_t C);
+lpdt_status lpdt_evonorm_s0_bwd(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C, int32_t groups,
+                                float eps, const float *dy, const float *x, const float *v, const float *gamma,
+                                int64_t param_node_stride, const float *gmean, const float *gvar,
+                                float *dx, float *dv, float *dgamma, float *dbeta, int64_t grad_node_stride,
+                                void *ws, size_t ws_bytes, void *stream);
+
+/* lpdt_range_bn_fwd / _bwd — range batch-norm (Eq. "rbn").  Per node and channel over the node's
+ * batch (b, h, w), P = B*H*W positions:
+ *   mu = mean of x;  D = Cb*(max x - min x) + eps,  Cb = 1/sqrt(2 ln B)   (the equation's C(b), b = the
+ *   batch size; B >= 2);   y = gamma_c*(x - mu)/D + beta_c
+ * Backward, derived, with t = dy*gamma_c and xc = x - mu:
+ *   dx = t/D - (sum t)/(P*D) - Cb*(sum t*xc)/D^2 * ([p = argmax] - [p = argmin])   (no last term if they coincide)
+ *   dbeta_c = sum dy;  dgamma_c = sum dy*xc/D
+ * cmean, cmin, cmax : fp32 [nodes][C];  argmin, argmax : int32 [nodes][C], the lowest position b*H*W + h*W + w
+ * attaining the extremum; all five written by the forward and read by the backward.
+ * ws : lpdt_range_bn_workspace_size(nodes, C) bytes (cross-CTA sums and extrema; cleared by the call).
+ * Errors: INVALID_ARG (B < 2 included), UNSUPPORTED, WORKSPACE, CUDA.
+ */
+size_t lpdt_range_bn_workspace_size(int32_t nodes, int32_t C);
+lpdt_status lpdt_range_bn_fwd(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C, float eps,
+                              const float *x, const float *gamma, const float *beta, int64_t param_node_stride,
+                              float *y, float *cmean, float *cmin, float *cmax, int32_t *argmin, int32_t *argmax,
+                              void *ws, size_t ws_bytes, void *stream);
+lpdt_status lpdt_range_bn_bwd(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C, float eps,
+                              const float *dy, const float *x, const float *gamma, int64_t param_node_stride,
+                              const float *cmean, const float *cmin, const float *cmax,
+                              const int32_t *argmin, const int32_t *argmax,
+                              float *dx, float *dgamma, float *dbeta, int64_t grad_node_stride,
+                              void *ws, size_t ws_bytes, void *stream);
+
+/* ---------------------------------------------------------------------------
  * lpdt_gossip_mix — compression, public-copy update and gossip averaging of
  * CHOCO-SGD (Algorithm 3: "compute and compress", the x_hat update, and the
  * gossip update), for all nodes at once:

@@ -15,7 +15,7 @@ from ._lib import ConvDesc, lib
 KERNELS_PER_CALL = {
     "lpdt_quantize": 2, "lpdt_quantize_with_range": 1, "lpdt_quantize_static": 2, "lpdt_quantize_batch": 2, "lpdt_dequantize": 1, "lpdt_qconv_fwd": 1, "lpdt_qconv_fwd_affine": 4, "lpdt_qconv_bwd_data": 2,
     "lpdt_qconv_bwd_weight": 2, "lpdt_range_evonorm_fwd": 1, "lpdt_range_evonorm_bwd": 2,
-    "lpdt_gossip_mix": 2, "lpdt_gossip_mix_q8": 3, "lpdt_deepsqueeze_mix": 2, "lpdt_pushsum_debias": 1, "lpdt_sgd_update": 1, "lpdt_residual_add": 1, "lpdt_residual_add_bwd": 1,
+    "lpdt_gossip_mix": 2, "lpdt_gossip_mix_q8": 3, "lpdt_deepsqueeze_mix": 2, "lpdt_pushsum_debias": 1, "lpdt_evonorm_s0_fwd": 1, "lpdt_evonorm_s0_bwd": 2, "lpdt_range_bn_fwd": 2, "lpdt_range_bn_bwd": 2, "lpdt_sgd_update": 1, "lpdt_residual_add": 1, "lpdt_residual_add_bwd": 1,
     "lpdt_avgpool": 1, "lpdt_avgpool_bwd": 1, "lpdt_maxpool2x2": 1, "lpdt_maxpool2x2_bwd": 1,
     "lpdt_softmax_ce": 1, "lpdt_colsum": 1,
 }
@@ -197,6 +197,44 @@ def lpdt_range_evonorm_bwd(nodes, B, H, W, Cc, groups, eps, dy, x, v, gamma, par
         nodes, B, H, W, Cc, groups, eps, _ptr(dy), _ptr(x), _ptr(v), _ptr(gamma), param_node_stride,
         _ptr(gmin), _ptr(gmax), _ptr(argmin), _ptr(argmax), _ptr(dx), _ptr(dv), _ptr(dgamma), _ptr(dbeta),
         grad_node_stride, _ptr(amax_out), p, nb, _stream()))
+
+
+def lpdt_evonorm_s0_fwd(nodes, B, H, W, Cc, groups, eps, x, v, gamma, beta, param_node_stride, y, gmean, gvar):
+    _check("lpdt_evonorm_s0_fwd", lib().lpdt_evonorm_s0_fwd(
+        nodes, B, H, W, Cc, groups, eps, _ptr(x), _ptr(v), _ptr(gamma), _ptr(beta), param_node_stride, _ptr(y),
+        _ptr(gmean), _ptr(gvar), _stream()))
+
+
+def lpdt_evonorm_s0_bwd_workspace_size(nodes, B, Cc):
+    return lib().lpdt_evonorm_s0_bwd_workspace_size(nodes, B, Cc)
+
+
+def lpdt_evonorm_s0_bwd(nodes, B, H, W, Cc, groups, eps, dy, x, v, gamma, param_node_stride, gmean, gvar, dx, dv,
+                        dgamma, dbeta, grad_node_stride, ws):
+    p, nb = _ws(ws)
+    _check("lpdt_evonorm_s0_bwd", lib().lpdt_evonorm_s0_bwd(
+        nodes, B, H, W, Cc, groups, eps, _ptr(dy), _ptr(x), _ptr(v), _ptr(gamma), param_node_stride, _ptr(gmean),
+        _ptr(gvar), _ptr(dx), _ptr(dv), _ptr(dgamma), _ptr(dbeta), grad_node_stride, p, nb, _stream()))
+
+
+def lpdt_range_bn_workspace_size(nodes, Cc):
+    return lib().lpdt_range_bn_workspace_size(nodes, Cc)
+
+
+def lpdt_range_bn_fwd(nodes, B, H, W, Cc, eps, x, gamma, beta, param_node_stride, y, cmean, cmin, cmax, argmin, argmax,
+                      ws):
+    p, nb = _ws(ws)
+    _check("lpdt_range_bn_fwd", lib().lpdt_range_bn_fwd(
+        nodes, B, H, W, Cc, eps, _ptr(x), _ptr(gamma), _ptr(beta), param_node_stride, _ptr(y), _ptr(cmean), _ptr(cmin),
+        _ptr(cmax), _ptr(argmin), _ptr(argmax), p, nb, _stream()))
+
+
+def lpdt_range_bn_bwd(nodes, B, H, W, Cc, eps, dy, x, gamma, param_node_stride, cmean, cmin, cmax, argmin, argmax, dx,
+                      dgamma, dbeta, grad_node_stride, ws):
+    p, nb = _ws(ws)
+    _check("lpdt_range_bn_bwd", lib().lpdt_range_bn_bwd(
+        nodes, B, H, W, Cc, eps, _ptr(dy), _ptr(x), _ptr(gamma), param_node_stride, _ptr(cmean), _ptr(cmin), _ptr(cmax),
+        _ptr(argmin), _ptr(argmax), _ptr(dx), _ptr(dgamma), _ptr(dbeta), grad_node_stride, p, nb, _stream()))
 
 
 def lpdt_gossip_mix_workspace_size(nodes, d, n_segments):

@@ -13,6 +13,10 @@ batch 128 so that each fp32 tensor is 268 MB; parameter kernels: 16 nodes with a
   ren_fwd             4 B read + 4 B written (the second read of a sample comes from L2)
   ren_fwd_res         + 4 B shortcut read
   ren_bwd             dy, x read + dx written: 12 B
+  evonorm_s0_fwd      comparison layer: 4 B read + 4 B written (second read of a sample from L2)
+  evonorm_s0_bwd      dy, x read (twice, the second time from L2) + dx written: 12 B
+  range_bn_fwd        statistics pass 4 B + apply pass 4 B read + 4 B written: 12 B (batch statistics: two launches)
+  range_bn_bwd        sums pass 8 B + apply pass 4 B read + 4 B written: 16 B
   residual_add        8 B read + 4 B written
   sgd_update          12 B per parameter
   gossip_dense        x_half, x_hat read; x_hat, x written: 16 B per parameter
@@ -83,6 +87,19 @@ def cases(nodes=8, B=128, H=32, W=32, Cc=64, d=32 * 270410, gossip_nodes=16):
     yield ("ren_bwd", lambda: api.lpdt_range_evonorm_bwd(nodes, B, H, W, Cc, groups, 1e-5, x2, x, v, gamma, Cc, gmin,
                                                          gmax, amin_i, amax_i, dx, dv, dg, db, Cc, wsb, amax_out=rng),
            tot * 12)
+    gm, gv = torch.empty(nodes, B, groups, device="cuda"), torch.empty(nodes, B, groups, device="cuda")
+    yield ("evonorm_s0_fwd", lambda: api.lpdt_evonorm_s0_fwd(nodes, B, H, W, Cc, groups, 1e-5, x, v, gamma, beta, Cc, y,
+                                                             gm, gv), tot * 8)
+    wse = torch.empty(api.lpdt_evonorm_s0_bwd_workspace_size(nodes, B, Cc), dtype=torch.uint8, device="cuda")
+    yield ("evonorm_s0_bwd", lambda: api.lpdt_evonorm_s0_bwd(nodes, B, H, W, Cc, groups, 1e-5, x2, x, v, gamma, Cc, gm,
+                                                             gv, dx, dv, dg, db, Cc, wse), tot * 12)
+    cm, cn, cx = (torch.empty(nodes, Cc, device="cuda") for _ in range(3))
+    an, ax = (torch.empty(nodes, Cc, dtype=torch.int32, device="cuda") for _ in range(2))
+    wsr = torch.empty(api.lpdt_range_bn_workspace_size(nodes, Cc), dtype=torch.uint8, device="cuda")
+    yield ("range_bn_fwd", lambda: api.lpdt_range_bn_fwd(nodes, B, H, W, Cc, 1e-5, x, gamma, beta, Cc, y, cm, cn, cx, an,
+                                                         ax, wsr), tot * 12)
+    yield ("range_bn_bwd", lambda: api.lpdt_range_bn_bwd(nodes, B, H, W, Cc, 1e-5, x2, x, gamma, Cc, cm, cn, cx, an, ax,
+                                                         dx, dg, db, Cc, wsr), tot * 16)
     yield ("residual_add", lambda: api.lpdt_residual_add(nodes, B, H, W, Cc, Cc, 1, 0, x, x2, y, amax_out=rng), tot * 12)
     del x2, dx
 

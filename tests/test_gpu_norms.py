@@ -1,0 +1,127 @@
+"""GPU parity of the comparison layers (EvoNorm-S0, range batch-norm) against the double-precision oracle,
+through the C ABI.  fp32 elementwise work with double sums: 1e-5 relative + 1e-6 absolute, the absolute term
+scaled by the tensor's largest magnitude for sums of signed terms."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2111_09389_b200 import api
+
+pytestmark = pytest.mark.gpu
+
+RTOL, ATOL = 1e-5, 1e-6
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def close(got, want, scale=1.0):
+    got = got.cpu().numpy().astype(np.float64) if isinstance(got, torch.Tensor) else got
+    want = np.asarray(want, np.float64)
+    err = np.abs(got - want)
+    ok = err <= ATOL * max(1.0, scale) + RTOL * np.abs(want)
+    assert ok.all(), f"{(~ok).sum()} of {ok.size} outside tolerance, worst {err.max():.3e}"
+
+
+def ws_bytes(n):
+    return torch.empty(max(int(n), 256), dtype=torch.uint8, device="cuda")
+
+
+def _inputs(case, seed):
+    nodes, B, H, W, C = case
+    rng = np.random.default_rng(seed)
+    x = (1.5 * rng.standard_normal((nodes, B, H, W, C)) + 0.3).astype(np.float32)
+    pad = 5
+    P = rng.uniform(0.5, 1.5, (nodes, 3 * C + pad)).astype(np.float32)
+    P[:, 2 * C:3 * C] -= 1.0
+    dy = rng.standard_normal(x.shape).astype(np.float32)
+    return x, P, dy
+
+
+EVO_CASES = [((4, 8, 16, 16, 16), 4), ((2, 3, 32, 32, 16), 2), ((2, 2, 8, 8, 64), 8), ((1, 3, 5, 7, 6), 3),
+             ((1, 2, 4, 4, 12), 1), ((2, 2, 32, 32, 64), 8), ((1, 2, 2, 2, 512), 64), ((1, 1, 1, 1, 8), 2),
+             ((1, 2, 9, 9, 24), 3)]
+
+
+@pytest.mark.parametrize("case,groups", EVO_CASES)
+def test_evonorm_s0_fwd_bwd(case, groups):
+    nodes, B, H, W, C = case
+    x, P, dy = _inputs(case, seed=C + groups)
+    eps = 1e-5
+    v, g, b = P[:, :C], P[:, C:2 * C], P[:, 2 * C:3 * C]
+    y_ref, mu_ref, var_ref = oracle.evonorm_s0_fwd(x, v, g, b, groups, eps)
+    xd, Pd = dev(x), dev(P)
+    stride = P.shape[1]
+    f = lambda *s: torch.empty(*s, dtype=torch.float32, device="cuda")
+    y, gmean, gvar = f(*x.shape), f(nodes, B, groups), f(nodes, B, groups)
+    api.lpdt_evonorm_s0_fwd(nodes, B, H, W, C, groups, eps, xd, Pd, Pd[:, C:], Pd[:, 2 * C:], stride, y, gmean, gvar)
+    close(gmean, mu_ref); close(gvar, var_ref)
+    close(y, y_ref, scale=float(np.abs(y_ref).max()))
+    # backward from the statistics the forward stored (both sides read the same fp32 values)
+    mu32, var32 = gmean.cpu().numpy(), gvar.cpu().numpy()
+    dx_ref, dv_ref, dg_ref, db_ref = oracle.evonorm_s0_bwd(dy, x, v, g, mu32, var32, groups, eps)
+    G = torch.zeros(nodes, stride, dtype=torch.float32, device="cuda")
+    dx = f(*x.shape)
+    ws = ws_bytes(api.lpdt_evonorm_s0_bwd_workspace_size(nodes, B, C))
+    api.lpdt_evonorm_s0_bwd(nodes, B, H, W, C, groups, eps, dev(dy), xd, Pd, Pd[:, C:], stride, gmean, gvar, dx, G,
+                            G[:, C:], G[:, 2 * C:], stride, ws)
+    close(dx, dx_ref, scale=float(np.abs(dx_ref).max()))
+    Gh = G.cpu().numpy()
+    close(Gh[:, :C], dv_ref, scale=float(np.abs(dv_ref).max()))
+    close(Gh[:, C:2 * C], dg_ref, scale=float(np.abs(dg_ref).max()))
+    close(Gh[:, 2 * C:3 * C], db_ref, scale=float(np.abs(db_ref).max()))
+    assert not Gh[:, 3 * C:].any()
+
+
+RBN_CASES = [(4, 8, 16, 16, 16), (2, 3, 32, 32, 16), (2, 2, 8, 8, 64), (1, 3, 5, 7, 6), (1, 2, 1, 1, 12),
+             (2, 32, 8, 8, 64), (1, 2, 2, 2, 512), (3, 40, 9, 7, 24)]
+
+
+@pytest.mark.parametrize("case", RBN_CASES)
+@pytest.mark.parametrize("ties", [False, True])
+def test_range_bn_fwd_bwd(case, ties):
+    nodes, B, H, W, C = case
+    x, P, dy = _inputs(case, seed=C + B)
+    if ties:
+        x = (np.round(x * 2) / 2).astype(np.float32)      # coarse grid: the extrema repeat, zeros of both signs occur
+        x[x == 0] *= -1.0
+    eps = 1e-5
+    g, b = P[:, :C], P[:, C:2 * C]
+    y_ref, mu_ref, mn_ref, mx_ref, amn_ref, amx_ref = oracle.range_bn_fwd(x, g, b, eps)
+    xd, Pd = dev(x), dev(P)
+    stride = P.shape[1]
+    f = lambda *s: torch.empty(*s, dtype=torch.float32, device="cuda")
+    i = lambda *s: torch.empty(*s, dtype=torch.int32, device="cuda")
+    y, cmean, cmin, cmax, amin_, amax_ = f(*x.shape), f(nodes, C), f(nodes, C), f(nodes, C), i(nodes, C), i(nodes, C)
+    ws = ws_bytes(api.lpdt_range_bn_workspace_size(nodes, C))
+    api.lpdt_range_bn_fwd(nodes, B, H, W, C, eps, xd, Pd, Pd[:, C:], stride, y, cmean, cmin, cmax, amin_, amax_, ws)
+    assert np.array_equal(cmin.cpu().numpy(), mn_ref) and np.array_equal(cmax.cpu().numpy(), mx_ref)
+    assert np.array_equal(amin_.cpu().numpy(), amn_ref) and np.array_equal(amax_.cpu().numpy(), amx_ref)
+    close(cmean, mu_ref)
+    close(y, y_ref, scale=float(np.abs(y_ref).max()))
+    mu32 = cmean.cpu().numpy()
+    dx_ref, dg_ref, db_ref = oracle.range_bn_bwd(dy, x, g, mu32, mn_ref, mx_ref, amn_ref, amx_ref, eps)
+    G = torch.zeros(nodes, stride, dtype=torch.float32, device="cuda")
+    dx = f(*x.shape)
+    api.lpdt_range_bn_bwd(nodes, B, H, W, C, eps, dev(dy), xd, Pd, stride, cmean, cmin, cmax, amin_, amax_, dx, G,
+                          G[:, C:], stride, ws)
+    close(dx, dx_ref, scale=float(np.abs(dx_ref).max()))
+    Gh = G.cpu().numpy()
+    close(Gh[:, :C], dg_ref, scale=float(np.abs(dg_ref).max()))
+    close(Gh[:, C:2 * C], db_ref, scale=float(np.abs(db_ref).max()))
+    assert not Gh[:, 2 * C:].any()
+
+
+def test_norm_layer_errors():
+    t = torch.zeros(64, device="cuda"); ti = torch.zeros(64, dtype=torch.int32, device="cuda")
+    with pytest.raises(api.LpdtError) as e:      # batch of one: the constant C(b) is infinite
+        api.lpdt_range_bn_fwd(1, 1, 2, 2, 4, 1e-5, t, t, t, 4, t, t, t, t, ti, ti, ws_bytes(4096))
+    assert e.value.code == 1
+    with pytest.raises(api.LpdtError) as e:      # workspace too small
+        api.lpdt_range_bn_fwd(1, 2, 2, 2, 4, 1e-5, t, t, t, 4, t, t, t, t, ti, ti, None)
+    assert e.value.code == 3
+    with pytest.raises(api.LpdtError) as e:      # groups must divide C
+        api.lpdt_evonorm_s0_fwd(1, 1, 2, 2, 6, 4, 1e-5, t, t, t, t, 6, t, t, t)
+    assert e.value.code == 1
