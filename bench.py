@@ -94,22 +94,35 @@ def dist_setup(n_gpus):
     return world, rank, local
 
 
-def barrier(world):
+def barrier(world, device="cuda"):
     import torch
     if world > 1:
         import torch.distributed as dist
         dist.barrier()
-    torch.cuda.synchronize()
+    if device == "cuda":
+        torch.cuda.synchronize()
 
 
-def max_over_ranks(world, value):
+def max_over_ranks(world, value, device="cuda"):
+    """The slowest rank's time: every rank gets the maximum of `value` over the job."""
     import torch
     if world == 1:
         return value
     import torch.distributed as dist
-    t = torch.tensor([value], dtype=torch.float64, device="cuda")
+    t = torch.tensor([value], dtype=torch.float64, device=device)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return float(t.item())
+
+
+def job_value(world, images_per_rank, ms_total, steps):
+    """Whole-job images/s of `world` replicas that each ran `steps` steps of `images_per_rank` images in
+    `ms_total` milliseconds (the maximum over ranks): weak scaling, no rank shares work with another."""
+    return world * images_per_rank / (ms_total / steps * 1e-3)
+
+
+def rank_seed(rank):
+    """Workload seed of a replica: the default recipe on rank 0, a different draw on every other rank."""
+    return None if rank == 0 else 1001 + rank
 
 
 def run_ours(args):
@@ -119,7 +132,7 @@ def run_ours(args):
     from paper_2111_09389_b200.step import TrainStep
 
     world, rank, local = dist_setup(args.gpus)
-    wl = workloads.make_workload(args.workload, seed=None if rank == 0 else 1001 + rank)
+    wl = workloads.make_workload(args.workload, seed=rank_seed(rank))
     st = TrainStep.from_workload(wl)
     images = wl["nodes"] * wl["batch"]
     macs_step = 3 * workloads.conv_macs(wl["ops"], images)
@@ -166,7 +179,7 @@ def run_ours(args):
         api.TIMED.difference_update(names)
     clocks = sampler.stop()
     ms_step = ms_total / args.steps
-    value = world * images / (ms_step * 1e-3)
+    value = job_value(world, images, ms_total, args.steps)
 
     # end to end: inputs start in pinned host memory, the loss is read back every step
     x_host = torch.from_numpy(wl["x"]).pin_memory()

@@ -479,6 +479,7 @@ gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float 
     const int tab_words = nodes + 2 * nodes * nodes;
     float *s_hat = sm + ((tab_words + 3) & ~3);                  // [nodes][TE][V], 16-byte aligned
     for (int i = threadIdx.x; i < tab_words; i += TE) s_cnt[i] = tab[i];
+    __syncthreads();       // the only block-wide wait: the parked copies below are read back by the thread that wrote them
     const int64_t e0 = ((int64_t)blockIdx.x * TE + threadIdx.x) * V;
     const bool live = e0 < d;                                    // d % V == 0: a thread is all in or all out
     int s0 = 0;
@@ -489,7 +490,7 @@ gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float 
         s0 = a;
         one_seg = seg.off[s0 + 1] >= e0 + V;
     }
-    constexpr int kU = 4;                                        // nodes per batch of independent loads
+    constexpr int kU = 8;                                        // nodes per batch of independent loads
     for (int ib = 0; ib < nodes; ib += kU) {
         float xh[kU][V], xq[kU][V];
 #pragma unroll
@@ -539,7 +540,6 @@ gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float 
             VecIO<V>::st(s_hat + ((size_t)i * TE + threadIdx.x) * V, hn);
         }
     }
-    __syncthreads();
     if (!live) return;
     for (int ib = 0; ib < nodes; ib += kU) {
         float xh[kU][V];
