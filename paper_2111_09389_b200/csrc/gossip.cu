@@ -33,6 +33,14 @@ template <> struct VecIO<4> {
         *reinterpret_cast<float4 *>(p) = make_float4(o[0], o[1], o[2], o[3]);
     }
 };
+template <> struct VecIO<2> {
+    static __device__ __forceinline__ void ld(const float *p, float (&o)[2]) {
+        float2 t = *reinterpret_cast<const float2 *>(p); o[0] = t.x; o[1] = t.y;
+    }
+    static __device__ __forceinline__ void st(float *p, const float (&o)[2]) {
+        *reinterpret_cast<float2 *>(p) = make_float2(o[0], o[1]);
+    }
+};
 template <> struct VecIO<1> {
     static __device__ __forceinline__ void ld(const float *p, float (&o)[1]) { o[0] = *p; }
     static __device__ __forceinline__ void st(float *p, const float (&o)[1]) { *p = o[0]; }
@@ -490,7 +498,7 @@ gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float 
         s0 = a;
         one_seg = seg.off[s0 + 1] >= e0 + V;
     }
-    constexpr int kU = 8;                                        // nodes per batch of independent loads
+    constexpr int kU = V == 4 ? 8 : 4;                           // nodes per batch of independent loads (as measured)
     for (int ib = 0; ib < nodes; ib += kU) {
         float xh[kU][V], xq[kU][V];
 #pragma unroll
@@ -722,8 +730,12 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
     launch_k(select_and_rows_kernel, dim3(n_segments, nodes + 1), 1024, 0, st, x_half, x_hat, d, seg, sel, Wmix, nodes, tab,
              amax_bits, msg_scale, msg_inv, big, state, cands, cand_per_node);
     LPDT_LAUNCH_CHECK();
+    // parameters per thread: 16-byte accesses need every node's row on a 16-byte boundary (d a multiple of 4);
+    // the networks' parameter counts are even but not multiples of 4, which still allows 8-byte accesses
     const bool v4 = d % 4 == 0 && aligned(x_half, 16) && aligned(x_hat, 16) && aligned(x_out, 16);
-    const int V = v4 ? 4 : 1;
+    const bool v2 = !v4 && d % 2 == 0 && aligned(x_half, 8) && aligned(x_hat, 8) && aligned(x_out, 8);
+    const int V = v4 ? 4 : v2 ? 2 : 1;
+    const int vi = v4 ? 2 : v2 ? 1 : 0;
     // threads per block: as many as keep the parked public copies within 64 KB of shared memory
     int TE = (int)((64 * 1024) / ((size_t)nodes * V * sizeof(float))) / 32 * 32;
     if (TE > 128) TE = 128;
@@ -732,18 +744,19 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
     const size_t smem = tab_words * sizeof(int32_t) + (size_t)nodes * TE * V * sizeof(float);
     using MixFn = void (*)(int, int64_t, const float *, float *, float *, float, SegTable, const SelectOut *,
                            const int32_t *, const float *, const float *);
-    static const MixFn fns[8] = {
-        gossip_mix_kernel<1, false, false>, gossip_mix_kernel<4, false, false>, gossip_mix_kernel<1, true, false>,
-        gossip_mix_kernel<4, true, false>,  gossip_mix_kernel<1, false, true>,  gossip_mix_kernel<4, false, true>,
-        gossip_mix_kernel<1, true, true>,   gossip_mix_kernel<4, true, true>};
+    static const MixFn fns[12] = {
+        gossip_mix_kernel<1, false, false>, gossip_mix_kernel<2, false, false>, gossip_mix_kernel<4, false, false>,
+        gossip_mix_kernel<1, true, false>,  gossip_mix_kernel<2, true, false>,  gossip_mix_kernel<4, true, false>,
+        gossip_mix_kernel<1, false, true>,  gossip_mix_kernel<2, false, true>,  gossip_mix_kernel<4, false, true>,
+        gossip_mix_kernel<1, true, true>,   gossip_mix_kernel<2, true, true>,   gossip_mix_kernel<4, true, true>};
     static bool attr_set = false;
     if (!attr_set) {
-        for (int i = 0; i < 8; ++i)
+        for (int i = 0; i < 12; ++i)
             LPDT_CUDA(cudaFuncSetAttribute(fns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
         attr_set = true;
     }
     const unsigned blocks = (unsigned)ceil_div(d, (int64_t)TE * V);
-    launch_k(fns[(ds ? 4 : 0) + (q8 ? 2 : 0) + (v4 ? 1 : 0)], blocks, TE, smem, st, nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab,
+    launch_k(fns[(ds ? 6 : 0) + (q8 ? 3 : 0) + vi], blocks, TE, smem, st, nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab,
                                                                             q8 ? msg_scale : nullptr, msg_inv);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;

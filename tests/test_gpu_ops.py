@@ -446,6 +446,8 @@ def _gossip_case(nodes, d, seed, heavy=False):
     # long segments: selection spread over several CTAs (with short and trivial ones beside them)
     (3, 100000, [(0, 100000, 1000)]), (2, 200000, [(0, 40000, 39999), (40000, 41000, 7), (41000, 200000, 1)]),
     (2, 70001, [(0, 33000, 0), (33000, 70001, 37001)]),
+    # parameter counts that are even but not multiples of 4 (8-byte accesses), segments starting at odd offsets
+    (4, 2738, None), (8, 270410, None), (6, 100002, [(0, 33333, 300), (33333, 100002, 700)]),
 ])
 def test_gossip_mix(nodes, d, segs):
     xh, xhat = _gossip_case(nodes, d, d, heavy=True)
