@@ -132,6 +132,36 @@ class TrainStep:
         if "dy" in wl:
             self.dy.copy_(torch.from_numpy(wl["dy"]))
 
+    # ---- host inputs, one batch ahead -------------------------------------------------
+    def upload(self, x_host, labels_host=None):
+        """Start copying a batch (pinned host tensors) into staging buffers on a copy stream; returns at once.
+        The copy overlaps whatever step is running: the step's own input buffers are untouched until
+        step_from_upload() takes the staged batch."""
+        if not hasattr(self, "_copy"):
+            self._copy = torch.cuda.Stream(device=self.x.device)
+            self._x_stage = torch.empty_like(self.x)
+            self._lab_stage = torch.empty_like(self.labels) if self.labels is not None else None
+            self._staged = torch.cuda.Event()
+            self._taken = torch.cuda.Event()
+            self._taken.record()
+        self._copy.wait_event(self._taken)                 # the previous batch has left the staging buffers
+        with torch.cuda.stream(self._copy):
+            self._x_stage.copy_(x_host, non_blocking=True)
+            if labels_host is not None and self._lab_stage is not None:
+                self._lab_stage.copy_(labels_host, non_blocking=True)
+            self._staged.record()
+
+    def step_from_upload(self, step=None):
+        """Take the staged batch (device-to-device copy into the step's inputs, ordered after the upload) and
+        run one step: `step` is run() by default, or replay() once the step has been captured."""
+        cur = torch.cuda.current_stream()
+        cur.wait_event(self._staged)
+        self.x.copy_(self._x_stage, non_blocking=True)
+        if self._lab_stage is not None:
+            self.labels.copy_(self._lab_stage, non_blocking=True)
+        self._taken.record()
+        (step or self.run)()
+
     @classmethod
     def from_workload(cls, wl, **kw):
         st = cls(wl["ops"], wl["d"], wl["nodes"], wl["batch"], wl["x"].shape[2:], wl["ren_eps"], wl["lr"],

@@ -93,6 +93,28 @@ def test_graph_replay_matches_eager():
     assert b.graph_launches > 100
 
 
+def test_step_from_upload_matches_loaded_inputs():
+    """The host-input pipeline (upload on a copy stream, one batch ahead) feeds the step the same bytes as load():
+    two batches in a row, the second uploaded while the first step runs."""
+    wl = wlmod.make_workload("resnet20", nodes=2, batch=4)
+    wl2 = wlmod.make_workload("resnet20", nodes=2, batch=4, seed=77)
+    ref = TrainStep.from_workload(wl)
+    ref.run()
+    ref.x.copy_(torch.from_numpy(wl2["x"])); ref.labels.copy_(torch.from_numpy(wl2["labels"]))
+    ref.params.copy_(ref.x_out)
+    ref.run()
+    st = TrainStep.from_workload(wl)
+    st.x.zero_(); st.labels.zero_()
+    pin = lambda a: torch.from_numpy(a).pin_memory()
+    st.upload(pin(wl["x"]), pin(wl["labels"]))
+    st.step_from_upload()
+    st.upload(pin(wl2["x"]), pin(wl2["labels"]))          # overlaps the first step
+    st.params.copy_(st.x_out)
+    st.step_from_upload()
+    torch.cuda.synchronize()
+    assert torch.equal(st.x_out, ref.x_out) and torch.equal(st.grads, ref.grads) and torch.equal(st.loss, ref.loss)
+
+
 def test_resnet20_full_size_step():
     # the benchmark workload at its full size (16 nodes x batch 32): every node's codes, outputs,
     # gradients and the gossip result against the oracle's whole step
