@@ -309,7 +309,7 @@ def roofline_for(name, st, wl, peaks, api, graph_ms=None):
     calls_per_step = 0
     bytes_step = 0
     ops_step = 0
-    for op in wl["ops"]:
+    for li, op in enumerate(wl["ops"]):
         k = op["op"]
         if name in ("lpdt_range_evonorm_fwd", "lpdt_range_evonorm_bwd") and k == "ren":
             n = N * B * op["H"] * op["W"] * op["C"]
@@ -331,6 +331,8 @@ def roofline_for(name, st, wl, peaks, api, graph_ms=None):
                 bytes_step += n_in + n_w + 4 * n_out
             elif name == "lpdt_qconv_bwd_data":
                 bytes_step += n_out + n_w + 4 * n_in
+                if st.buf[li].get("addend") is not None:      # fused shortcut gradient: one more fp32 read
+                    bytes_step += 4 * n_in
             else:
                 bytes_step += n_out + n_in + 4 * n_w
             calls_per_step += 1

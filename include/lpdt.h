@@ -168,6 +168,10 @@ lpdt_status lpdt_quantize_static(const float *x, int32_t nodes, int64_t n_per_no
  * bias     : fp32, node n at bias + n*bias_node_stride, Cout entries (nullable)
  * dW       : node n at dW + n*dw_node_stride (weight gradients stay fp32:
  *            "gradient bifurcation"); dWacc is contiguous.
+ * addend   : (bwd_data, nullable) fp32, shape of dA, 16-byte aligned, not dA itself: dA = dequantized
+ *            sums + addend, one more fp32 addition.  This is the adjoint of a residual block's identity
+ *            shortcut (the block-output gradient joins the gradient of the block's first convolution),
+ *            fused into the contraction's epilogue; dAacc is not affected.
  * ws       : lpdt_qconv_workspace_size(desc, which) bytes, which = 0 fwd,
  *            1 bwd_data, 2 bwd_weight.
  * Errors: INVALID_ARG, UNSUPPORTED (shape outside every kernel's range),
@@ -181,7 +185,7 @@ lpdt_status lpdt_qconv_fwd(const lpdt_conv_desc *d, const int8_t *A, const float
                            void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
 lpdt_status lpdt_qconv_bwd_data(const lpdt_conv_desc *d, const int8_t *E, const float *sE,
                                 const int8_t *Wq, const float *sW,
-                                float *dA, int32_t *dAacc,
+                                float *dA, int32_t *dAacc, const float *addend,
                                 void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
 lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8_t *E, const float *sE,
                                   const int8_t *A, const float *sA,

@@ -163,10 +163,10 @@ def lpdt_qconv_fwd_affine(desc, A, sA, zA, Wq, sW, zW, Y=None, Yacc=None, bias=N
         _ptr(Y), _ptr(Yacc), p, nb, _ptr(dev_status), _stream()))
 
 
-def lpdt_qconv_bwd_data(desc, E, sE, Wq, sW, dA=None, dAacc=None, ws=None, dev_status=None):
+def lpdt_qconv_bwd_data(desc, E, sE, Wq, sW, dA=None, dAacc=None, ws=None, dev_status=None, addend=None):
     p, nb = _ws(ws)
     _check("lpdt_qconv_bwd_data", lib().lpdt_qconv_bwd_data(C.byref(desc), _ptr(E), _ptr(sE), _ptr(Wq),
-                                                            _ptr(sW), _ptr(dA), _ptr(dAacc), p, nb,
+                                                            _ptr(sW), _ptr(dA), _ptr(dAacc), _ptr(addend), p, nb,
                                                             _ptr(dev_status), _stream()))
 
 

@@ -57,12 +57,12 @@ static bool use_halo(const lpdt_conv_desc &d, int mode) {
 }
 static lpdt_status run_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const float *s1, const int8_t *Wq,
                            const float *s2, const float *bias, int64_t bias_stride, float *Y, int32_t *Yacc,
-                           int32_t *dev_status, cudaStream_t st, bool uns = false) {
+                           int32_t *dev_status, cudaStream_t st, bool uns = false, const float *addend = nullptr) {
     if (use_halo(d, mode)) {
-        lpdt_status r = tc::tc_pix_halo(d, mode, A, s1, Wq, s2, bias, bias_stride, Y, Yacc, dev_status, st, uns);
+        lpdt_status r = tc::tc_pix_halo(d, mode, A, s1, Wq, s2, bias, bias_stride, Y, Yacc, dev_status, st, uns, addend);
         if (r != LPDT_ERR_UNSUPPORTED) return r;
     }
-    return tc::tc_pix(d, mode, A, s1, Wq, s2, bias, bias_stride, Y, Yacc, dev_status, st, uns);
+    return tc::tc_pix(d, mode, A, s1, Wq, s2, bias, bias_stride, Y, Yacc, dev_status, st, uns, addend);
 }
 
 static int pad16(int c) { return (c + 15) / 16 * 16; }
@@ -348,16 +348,18 @@ extern "C" lpdt_status lpdt_qconv_fwd_affine(const lpdt_conv_desc *d, const uint
 
 extern "C" lpdt_status lpdt_qconv_bwd_data(const lpdt_conv_desc *d, const int8_t *E, const float *sE,
                                            const int8_t *Wq, const float *sW, float *dA, int32_t *dAacc,
-                                           void *ws, size_t ws_bytes, int32_t *dev_status, void *stream) {
+                                           const float *addend, void *ws, size_t ws_bytes, int32_t *dev_status,
+                                           void *stream) {
     lpdt_status s = check_desc(d);
     if (s != LPDT_OK) return s;
     if (d->nodes == 0 || d->B == 0) return LPDT_OK;
     LPDT_CHECK_ARG(E && Wq && (dA || dAacc));
     LPDT_CHECK_ARG(!dA || (sE && sW));
+    LPDT_CHECK_ARG(!addend || (dA && addend != dA && aligned(addend, 16)));
     if (!ws || ws_bytes < lpdt_qconv_workspace_size(d, 1)) return LPDT_ERR_WORKSPACE;
     if (use_tc(*d) && aligned(E, 16) && aligned(Wq, 16) && (!dA || aligned(dA, 16)) && (!dAacc || aligned(dAacc, 16)))
-        return run_pix(*d, 1, E, sE, Wq, sW, nullptr, 0, dA, dAacc, dev_status, as_stream(stream));
-    return generic_bwd_data(*d, E, sE, Wq, sW, dA, dAacc, ws, as_stream(stream));
+        return run_pix(*d, 1, E, sE, Wq, sW, nullptr, 0, dA, dAacc, dev_status, as_stream(stream), false, addend);
+    return generic_bwd_data(*d, E, sE, Wq, sW, dA, dAacc, addend, ws, as_stream(stream));
 }
 
 extern "C" lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8_t *E, const float *sE,

@@ -92,7 +92,7 @@ __global__ void transpose_weights_kernel(lpdt_conv_desc d, const int8_t *__restr
 __global__ void conv_bwd_data_generic(lpdt_conv_desc d, int Ho, int Wo, const int8_t *__restrict__ E,
                                       const int8_t *__restrict__ Wt, int32_t *__restrict__ acc_out,
                                       float *__restrict__ dA, const float *__restrict__ s1,
-                                      const float *__restrict__ s2, bool vec4) {
+                                      const float *__restrict__ s2, bool vec4, const float *__restrict__ addend) {
     pdl_enter();
     const int64_t per_node = (int64_t)d.B * d.H * d.W * d.Cin;
     const int64_t total = per_node * d.nodes;
@@ -120,7 +120,11 @@ __global__ void conv_bwd_data_generic(lpdt_conv_desc d, int Ho, int Wo, const in
             }
         }
         if (acc_out) acc_out[o] = acc;
-        if (dA) dA[o] = __fmul_rn(__int2float_rn(acc), __fmul_rn(s1[n], s2[n]));
+        if (dA) {
+            float v = __fmul_rn(__int2float_rn(acc), __fmul_rn(s1[n], s2[n]));
+            if (addend) v = __fadd_rn(v, addend[o]);
+            dA[o] = v;
+        }
     }
 }
 
@@ -194,7 +198,7 @@ lpdt_status generic_fwd(const lpdt_conv_desc &d, const int8_t *A, const float *s
 }
 
 lpdt_status generic_bwd_data(const lpdt_conv_desc &d, const int8_t *E, const float *sE, const int8_t *Wq,
-                             const float *sW, float *dA, int32_t *dAacc, void *ws, cudaStream_t st) {
+                             const float *sW, float *dA, int32_t *dAacc, const float *addend, void *ws, cudaStream_t st) {
     const int Ho = conv_out(d.H, d.pad, d.R, d.stride), Wo = conv_out(d.W, d.pad, d.S, d.stride);
     int8_t *Wt = (int8_t *)ws;
     const int64_t wn = (int64_t)d.nodes * d.Cout * d.R * d.S * d.Cin;
@@ -202,7 +206,7 @@ lpdt_status generic_bwd_data(const lpdt_conv_desc &d, const int8_t *E, const flo
     LPDT_LAUNCH_CHECK();
     const int64_t total = (int64_t)d.nodes * d.B * d.H * d.W * d.Cin;
     const bool vec4 = d.Cout % 4 == 0 && aligned(E, 4) && aligned(Wt, 4);
-    launch_k(conv_bwd_data_generic, grid_for(total), 256, 0, st, d, Ho, Wo, E, Wt, dAacc, dA, sE, sW, vec4);
+    launch_k(conv_bwd_data_generic, grid_for(total), 256, 0, st, d, Ho, Wo, E, Wt, dAacc, dA, sE, sW, vec4, addend);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

@@ -47,6 +47,7 @@ struct HaloParams {
     int w_rows_per_node;
     float *Y; int32_t *Yacc;
     const float *s1, *s2, *bias; long long bias_stride;
+    const float *addend;       // nullable: fp32 tensor of the result's shape, added to the dequantized result
     int32_t *dev_status;
 };
 
@@ -239,6 +240,15 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
                         f[k] = __fmul_rn(__int2float_rn((int)v[k]), sc);
                         if (p.bias) f[k] = __fadd_rn(f[k], p.bias[(long long)c.node * p.bias_stride + cc + k]);
                     }
+                    if (p.addend && valid) {
+                        const float4 *ad = reinterpret_cast<const float4 *>(p.addend + pix * p.N + cc);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            const float4 a4 = ad[k];
+                            f[4 * k] = __fadd_rn(f[4 * k], a4.x); f[4 * k + 1] = __fadd_rn(f[4 * k + 1], a4.y);
+                            f[4 * k + 2] = __fadd_rn(f[4 * k + 2], a4.z); f[4 * k + 3] = __fadd_rn(f[4 * k + 3], a4.w);
+                        }
+                    }
                     const int g = cc / inner, k0 = (cc % inner) >> 2;
                     float4 *grow = reinterpret_cast<float4 *>(ot + ((size_t)g * 128 + row) * inner * 4);
 #pragma unroll
@@ -285,6 +295,7 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
                         for (int k = 0; k < 16; ++k) {
                             f[k] = __fmul_rn(__int2float_rn((int)v[k]), sc);
                             if (p.bias) f[k] = __fadd_rn(f[k], p.bias[(long long)c.node * p.bias_stride + cc + k]);
+                            if (p.addend) f[k] = __fadd_rn(f[k], p.addend[o + k]);
                         }
                         float4 *dst = reinterpret_cast<float4 *>(p.Y + o);
 #pragma unroll
@@ -331,9 +342,10 @@ bool halo_supported(const lpdt_conv_desc &d, int mode) {
 
 lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, const float *s1, const int8_t *Wq,
                         const float *s2, const float *bias, int64_t bias_stride, float *Y, int32_t *Yacc,
-                        int32_t *dev_status, cudaStream_t st, bool uns) {
+                        int32_t *dev_status, cudaStream_t st, bool uns, const float *addend) {
     const int Ho = conv_out(d.H, d.pad, d.R, 1), Wo = conv_out(d.W, d.pad, d.S, 1);
     HaloParams p = {};
+    p.addend = addend;
     p.mode = mode; p.uns = uns ? 1 : 0; p.nodes = d.nodes; p.B = d.B;
     p.N = mode == 0 ? d.Cout : d.Cin;
     p.Hm = mode == 0 ? Ho : d.H; p.Wm = mode == 0 ? Wo : d.W;

@@ -66,6 +66,7 @@ struct PixParams {
     int w_rows_per_node;      // Cout: rows of the weight map per node
     float *Y; int32_t *Yacc;
     const float *s1, *s2, *bias; long long bias_stride;
+    const float *addend;      // nullable: fp32 tensor of the result's shape, added to the dequantized result
     int32_t *dev_status;
 };
 
@@ -284,6 +285,15 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                         for (int k = 0; k < 16; ++k) {
                             f[k] = __fmul_rn(__int2float_rn((int)v[k]), sc);
                             if (p.bias) f[k] = __fadd_rn(f[k], p.bias[(long long)c.node * p.bias_stride + n0 + cc + k]);
+                        }
+                        if (p.addend) {
+                            const float4 *ad = reinterpret_cast<const float4 *>(p.addend + o);
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const float4 a4 = ad[k];
+                                f[4 * k] = __fadd_rn(f[4 * k], a4.x); f[4 * k + 1] = __fadd_rn(f[4 * k + 1], a4.y);
+                                f[4 * k + 2] = __fadd_rn(f[4 * k + 2], a4.z); f[4 * k + 3] = __fadd_rn(f[4 * k + 3], a4.w);
+                            }
                         }
                         float4 *dst = reinterpret_cast<float4 *>(p.Y + o);
 #pragma unroll
@@ -540,9 +550,10 @@ static int largest_div(int C, int cap, int unit) {      // largest multiple of u
 
 lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const float *s1, const int8_t *Wq,
                    const float *s2, const float *bias, int64_t bias_stride, float *Y, int32_t *Yacc,
-                   int32_t *dev_status, cudaStream_t st, bool uns) {
+                   int32_t *dev_status, cudaStream_t st, bool uns, const float *addend) {
     const int Ho = conv_out(d.H, d.pad, d.R, d.stride), Wo = conv_out(d.W, d.pad, d.S, d.stride);
     PixParams p = {};
+    p.addend = addend;
     p.mode = mode; p.nodes = d.nodes; p.B = d.B;
     p.Nc = mode == 0 ? d.Cout : d.Cin; p.Kc = mode == 0 ? d.Cin : d.Cout;
     p.out_mul = 1; p.cmul = 1; p.ncls = 1;

@@ -240,6 +240,7 @@ class TrainStep:
         g_range = None
         L = len(self.ops)
         sc = []
+        fused_shortcut = False
         ctr = 0
         for li in range(len(self.ops) - 1, -1, -1):
             op, b = self.ops[li], self.buf[li]
@@ -268,8 +269,17 @@ class TrainStep:
                                                   dW=self._g(op["w_off"]), dw_node_stride=d, ws=self.ws_side,
                                                   dev_status=self.dev_status)
                 if li > 0 or self.input_grad:
+                    # first convolution of a residual block with an identity shortcut: the block-output gradient
+                    # joins this gradient in the contraction's epilogue (no separate residual_add_bwd pass)
+                    addend = None
+                    if li > 0 and self.ops[li - 1]["op"] == "save" and sc:
+                        aop = sc[-1][1]
+                        if aop["stride"] == 1 and aop["Ca"] == aop["C"]:
+                            addend = sc[-1][0]
+                            fused_shortcut = True
+                    b["addend"] = addend
                     api.lpdt_qconv_bwd_data(b["desc"], b["E"], b["sE"], b["qW"], b["sW"], dA=b["dx"],
-                                            ws=self.ws, dev_status=self.dev_status)
+                                            ws=self.ws, dev_status=self.dev_status, addend=addend)
                     g, g_range = b["dx"], None
                 else:
                     g = None
@@ -285,9 +295,12 @@ class TrainStep:
                 sc.append((g, op))
             elif k == "save":
                 dy_sc, aop = sc.pop()
-                api.lpdt_residual_add_bwd(N, B, aop["H"], aop["W"], aop["Ca"], aop["C"], aop["stride"],
-                                          aop["ch_off"], dy_sc, g, b["dx"])
-                g, g_range = b["dx"], None
+                if fused_shortcut:                  # already added by the convolution above
+                    fused_shortcut = False
+                else:
+                    api.lpdt_residual_add_bwd(N, B, aop["H"], aop["W"], aop["Ca"], aop["C"], aop["stride"],
+                                              aop["ch_off"], dy_sc, g, b["dx"])
+                    g, g_range = b["dx"], None
             elif k == "maxpool":
                 api.lpdt_maxpool2x2_bwd(N, B, op["H"], op["W"], op["C"], g, b["idx"], b["dx"])
                 g, g_range = b["dx"], None
@@ -334,7 +347,7 @@ class TrainStep:
                 n += 1
             if "bwd_data" in passes and (li > 0 or self.input_grad):
                 api.lpdt_qconv_bwd_data(b["desc"], b["E"], b["sE"], b["qW"], b["sW"], dA=b["dx"], ws=self.ws,
-                                        dev_status=self.dev_status)
+                                        dev_status=self.dev_status, addend=b.get("addend"))
                 n += 1
         return n
 

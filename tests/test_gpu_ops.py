@@ -262,6 +262,15 @@ def test_qconv_all_three(case):
     buf, dA2 = guarded(dA_ref.shape)
     api.lpdt_qconv_bwd_data(desc, Ed, s1d, Wd, s2d, dA=dA2, ws=ws, dev_status=status)
     assert torch.equal(dA2, dA) and bool(buf[:1024].isnan().all()) and bool(buf[-1024:].isnan().all())
+    # fused shortcut gradient: dA = dequantized sums + addend, one more fp32 addition (= the oracle's residual adjoint)
+    addend = np.random.default_rng(2).standard_normal(dA_ref.shape).astype(np.float32)
+    buf, dA3 = guarded(dA_ref.shape)
+    api.lpdt_qconv_bwd_data(desc, Ed, s1d, Wd, s2d, dA=dA3, ws=ws, dev_status=status, addend=dev(addend))
+    want = oracle.residual_add_bwd(addend, oracle.dequant_acc(dA_ref, s1, s2))
+    assert np.array_equal(dA3.cpu().numpy(), want) and bool(buf[:1024].isnan().all()) and bool(buf[-1024:].isnan().all())
+    dA4 = torch.empty_like(dA); dAacc4 = torch.empty_like(dAacc)
+    api.lpdt_qconv_bwd_data(desc, Ed, s1d, Wd, s2d, dA=dA4, dAacc=dAacc4, ws=ws, dev_status=status, addend=dev(addend))
+    assert torch.equal(dA4, dA3) and torch.equal(dAacc4, dAacc)
     # backward weight, into a strided gradient vector
     dW_ref, _ = oracle.qconv_bwd_weight(E, A, R, S, stride, pad)
     wn = Cout * R * S * Cin
