@@ -239,6 +239,11 @@ lpdt_status lpdt_qconv_fwd_affine(const lpdt_conv_desc *d, const uint8_t *A, con
  * amax_out (nullable) : fp32 [nodes], caller-zeroed; receives max|y| (forward) or max|dx|
  *            (backward) per node by atomic maximum, for lpdt_quantize_with_range
  * Requires C % groups == 0 and cpg >= 2 (Cst is infinite for cpg = 1).
+ * Backward with dv = dgamma = dbeta = NULL writes dx only and leaves the parameter-gradient sums as
+ * per-sample partial sums in ws; lpdt_range_evonorm_bwd_params(nodes, B, C, ws, ...) then adds them over
+ * the batch (fixed order, same result as the one-call form).  The second call may run on another
+ * stream once the first has finished, which takes the small reduction off the backward pass's critical
+ * path; ws must not be reused in between.
  * Errors: INVALID_ARG, UNSUPPORTED (C beyond the kernels' range), WORKSPACE, CUDA.
  */
 lpdt_status lpdt_range_evonorm_fwd(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C,
@@ -256,6 +261,9 @@ lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t H, int32_t 
                                    float *dx, float *dv, float *dgamma, float *dbeta,
                                    int64_t grad_node_stride, float *amax_out,
                                    void *ws, size_t ws_bytes, void *stream);
+lpdt_status lpdt_range_evonorm_bwd_params(int32_t nodes, int32_t B, int32_t C, const void *ws, size_t ws_bytes,
+                                          float *dv, float *dgamma, float *dbeta, int64_t grad_node_stride,
+                                          void *stream);
 
 /* ---------------------------------------------------------------------------
  * Comparison layers of Section 3 (the normalization study; not on the 8-bit path).

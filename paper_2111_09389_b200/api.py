@@ -14,7 +14,7 @@ from ._lib import ConvDesc, lib
 # Kernels each entry point enqueues (memsets not counted); KERNEL_LAUNCHES accumulates them.
 KERNELS_PER_CALL = {
     "lpdt_quantize": 2, "lpdt_quantize_with_range": 1, "lpdt_quantize_static": 2, "lpdt_quantize_batch": 2, "lpdt_dequantize": 1, "lpdt_qconv_fwd": 1, "lpdt_qconv_fwd_affine": 4, "lpdt_qconv_bwd_data": 2,
-    "lpdt_qconv_bwd_weight": 2, "lpdt_range_evonorm_fwd": 1, "lpdt_range_evonorm_bwd": 2,
+    "lpdt_qconv_bwd_weight": 2, "lpdt_range_evonorm_fwd": 1, "lpdt_range_evonorm_bwd": 2, "lpdt_range_evonorm_bwd_params": 1,
     "lpdt_gossip_mix": 2, "lpdt_gossip_mix_q8": 3, "lpdt_deepsqueeze_mix": 2, "lpdt_pushsum_debias": 1, "lpdt_evonorm_s0_fwd": 1, "lpdt_evonorm_s0_bwd": 2, "lpdt_range_bn_fwd": 2, "lpdt_range_bn_bwd": 2, "lpdt_sgd_update": 1, "lpdt_residual_add": 1, "lpdt_residual_add_bwd": 1,
     "lpdt_avgpool": 1, "lpdt_avgpool_bwd": 1, "lpdt_maxpool2x2": 1, "lpdt_maxpool2x2_bwd": 1,
     "lpdt_softmax_ce": 1, "lpdt_colsum": 1,
@@ -235,6 +235,13 @@ def lpdt_range_bn_bwd(nodes, B, H, W, Cc, eps, dy, x, gamma, param_node_stride, 
     _check("lpdt_range_bn_bwd", lib().lpdt_range_bn_bwd(
         nodes, B, H, W, Cc, eps, _ptr(dy), _ptr(x), _ptr(gamma), param_node_stride, _ptr(cmean), _ptr(cmin), _ptr(cmax),
         _ptr(argmin), _ptr(argmax), _ptr(dx), _ptr(dgamma), _ptr(dbeta), grad_node_stride, p, nb, _stream()))
+
+
+def lpdt_range_evonorm_bwd_params(nodes, B, Cc, ws, dv, dgamma, dbeta, grad_node_stride):
+    """Second half of a backward call made with dv = dgamma = dbeta = None: adds the partial sums in ws."""
+    p, nb = _ws(ws)
+    _check("lpdt_range_evonorm_bwd_params", lib().lpdt_range_evonorm_bwd_params(
+        nodes, B, Cc, p, nb, _ptr(dv), _ptr(dgamma), _ptr(dbeta), grad_node_stride, _stream()))
 
 
 def lpdt_gossip_mix_workspace_size(nodes, d, n_segments):

@@ -473,8 +473,10 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t 
     LPDT_CHECK_ARG(nodes >= 0 && B >= 0 && H > 0 && W > 0 && C > 0 && groups > 0);
     LPDT_CHECK_ARG(C % groups == 0 && C / groups >= 2);
     if (nodes == 0 || B == 0) return LPDT_OK;
-    LPDT_CHECK_ARG(dy && x && v && gamma && gmin && gmax && argmin && argmax && dx && dv && dgamma && dbeta);
-    LPDT_CHECK_ARG((pstride >= C && gstride >= C) || nodes == 1);
+    LPDT_CHECK_ARG(dy && x && v && gamma && gmin && gmax && argmin && argmax && dx);
+    const bool deferred = !dv && !dgamma && !dbeta;       // parameter gradients left as partial sums in ws
+    LPDT_CHECK_ARG(deferred || (dv && dgamma && dbeta));
+    LPDT_CHECK_ARG((pstride >= C && (deferred || gstride >= C)) || nodes == 1);
     if ((int64_t)H * W * C > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
     if (!ws || ws_bytes < lpdt_range_evonorm_bwd_workspace_size(nodes, B, C) || !aligned(ws, 8))
         return LPDT_ERR_WORKSPACE;
@@ -493,7 +495,22 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t 
     else
         launch_k(ren_bwd_kernel<1>, grid, pl.threads, smem, st, H * W, C, groups, eps, Cst, dy, x, v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc, amax_out);
     LPDT_LAUNCH_CHECK();
+    if (deferred) return LPDT_OK;
     launch_k(ren_bwd_finalize, (nodes * 3 * C + 7) / 8, 256, 0, st, acc, nodes, B, C, dv, dgamma, dbeta, gstride);
+    LPDT_LAUNCH_CHECK();
+    return LPDT_OK;
+}
+
+extern "C" lpdt_status lpdt_range_evonorm_bwd_params(int32_t nodes, int32_t B, int32_t C, const void *ws,
+                                                     size_t ws_bytes, float *dv, float *dgamma, float *dbeta,
+                                                     int64_t gstride, void *stream) {
+    LPDT_CHECK_ARG(nodes >= 0 && B >= 0 && C > 0);
+    if (nodes == 0 || B == 0) return LPDT_OK;
+    LPDT_CHECK_ARG(dv && dgamma && dbeta && (gstride >= C || nodes == 1));
+    if (!ws || ws_bytes < lpdt_range_evonorm_bwd_workspace_size(nodes, B, C) || !aligned(ws, 8))
+        return LPDT_ERR_WORKSPACE;
+    launch_k(ren_bwd_finalize, (nodes * 3 * C + 7) / 8, 256, 0, as_stream(stream), (const double *)ws, nodes, B, C, dv,
+             dgamma, dbeta, gstride);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

@@ -90,7 +90,10 @@ class TrainStep:
                 b.update(out=torch.empty(N, B, H, W, Cc, **f32), dx=torch.empty(N, B, H, W, Cc, **f32),
                          gmin=torch.empty(N, B, G, **f32), gmax=torch.empty(N, B, G, **f32),
                          amin=torch.empty(N, B, G, **i32), amax=torch.empty(N, B, G, **i32))
-                ws_bytes = max(ws_bytes, api.lpdt_range_evonorm_bwd_workspace_size(N, B, Cc))
+                # per-sample partial sums of the parameter gradients: a buffer per layer, because their reduction
+                # runs later, on the side stream
+                b["ws_ren"] = torch.empty(api.lpdt_range_evonorm_bwd_workspace_size(N, B, Cc), dtype=torch.uint8,
+                                          device=dev)
             elif k == "add":
                 Ho, Wo = (op["H"] + op["stride"] - 1) // op["stride"], (op["W"] + op["stride"] - 1) // op["stride"]
                 b.update(out=torch.empty(N, B, Ho, Wo, op["C"], **f32))
@@ -240,6 +243,7 @@ class TrainStep:
         g_range = None
         L = len(self.ops)
         sc = []
+        pending_ren = []
         fused_shortcut = False
         ctr = 0
         for li in range(len(self.ops) - 1, -1, -1):
@@ -259,6 +263,7 @@ class TrainStep:
                 main = torch.cuda.current_stream()
                 self.side.wait_stream(main)               # E (and, at the first use, everything before) is ready
                 with torch.cuda.stream(self.side):
+                    self._ren_param_sums(pending_ren)
                     if self.quantize_wgrad:
                         api.lpdt_qconv_bwd_weight(b["desc"], b["E"], b["sE"], b["qA"], b["sA"], dW=b["gw"],
                                                   dw_node_stride=b["wn"], ws=self.ws_side, dev_status=self.dev_status)
@@ -285,11 +290,12 @@ class TrainStep:
                     g = None
             elif k == "ren":
                 Cc = op["C"]
+                # dx only; the parameter-gradient sums stay as partial sums and are reduced on the side stream
                 api.lpdt_range_evonorm_bwd(N, B, op["H"], op["W"], Cc, op["groups"], self.eps, g, b["x"],
                                            self._p(op["p_off"]), self._p(op["p_off"] + Cc), d, b["gmin"],
-                                           b["gmax"], b["amin"], b["amax"], b["dx"], self._g(op["p_off"]),
-                                           self._g(op["p_off"] + Cc), self._g(op["p_off"] + 2 * Cc), d, self.ws,
+                                           b["gmax"], b["amin"], b["amax"], b["dx"], None, None, None, d, b["ws_ren"],
                                            amax_out=self.ranges[L + li])
+                pending_ren.append((op, b))
                 g, g_range = b["dx"], self.ranges[L + li]
             elif k == "add":
                 sc.append((g, op))
@@ -307,9 +313,21 @@ class TrainStep:
             elif k == "avgpool":
                 api.lpdt_avgpool_bwd(N, B, op["H"] * op["W"], op["C"], g, b["dx"])
                 g, g_range = b["dx"], None
+        if pending_ren:                                         # a norm layer with no convolution below it
+            self.side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(self.side):
+                self._ren_param_sums(pending_ren)
         torch.cuda.current_stream().wait_stream(self.side)      # weight gradients complete before the update
         self.input_grad_out = g
         return g
+
+    def _ren_param_sums(self, pending):
+        """Reduce the Range-EvoNorm parameter-gradient partial sums of the layers in `pending` (current stream)."""
+        for op, b in pending:
+            Cc = op["C"]
+            api.lpdt_range_evonorm_bwd_params(self.N, self.B, Cc, b["ws_ren"], self._g(op["p_off"]),
+                                              self._g(op["p_off"] + Cc), self._g(op["p_off"] + 2 * Cc), self.d)
+        pending.clear()
 
     def update(self):
         N, d = self.N, self.d

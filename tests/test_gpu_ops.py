@@ -361,6 +361,12 @@ def test_range_evonorm_fwd_bwd(case, ties):
                                dx, G, G[:, C:], G[:, 2 * C:], stride, ws)
     close(dx, dx32, 1e-6, 1e-7)
     close(dx, dx64)
+    # two-call form: dx first, the parameter-gradient sums later from the partial sums in the workspace
+    G2 = torch.zeros_like(G); dx2 = f(*x.shape)
+    api.lpdt_range_evonorm_bwd(nodes, B, H, W, C, groups, eps, dev(dy), xd, Pd, Pd[:, C:], stride, gmin, gmax, amin_, amax_,
+                               dx2, None, None, None, stride, ws)
+    api.lpdt_range_evonorm_bwd_params(nodes, B, C, ws, G2, G2[:, C:], G2[:, 2 * C:], stride)
+    assert torch.equal(dx2, dx) and torch.equal(G2, G)
     Gh = G.cpu().numpy()
     scale = lambda r: 1e-6 * max(1.0, float(np.abs(r).max()))
     close(Gh[:, :C], dv64, RTOL, scale(dv64))
