@@ -262,7 +262,7 @@ def roofline_sum(parts, peaks):
 # DRAM bytes (dram__bytes_read.sum + dram__bytes_write.sum) of the tensor-core forward / backward-data
 # kernels over one step, from the ncu capture summarised in profiles/step_resnet20_launches.md.  Valid
 # for that workload and those entry points only, and only while those kernels are unchanged.
-MEASURED_TRAFFIC = {("resnet20", "lpdt_qconv_fwd,lpdt_qconv_bwd_data"): {"bytes_per_step": 201.0e6, "launches": 37}}
+MEASURED_TRAFFIC = {("resnet20", "lpdt_qconv_fwd,lpdt_qconv_bwd_data"): {"bytes_per_step": 353.6e6, "launches": 37}}
 
 
 def attach_traffic(roof, workload, entry_points):

@@ -197,6 +197,9 @@ def lpdt_range_evonorm_bwd(nodes, B, H, W, Cc, groups, eps, dy, x, v, gamma, par
         nodes, B, H, W, Cc, groups, eps, _ptr(dy), _ptr(x), _ptr(v), _ptr(gamma), param_node_stride,
         _ptr(gmin), _ptr(gmax), _ptr(argmin), _ptr(argmax), _ptr(dx), _ptr(dv), _ptr(dgamma), _ptr(dbeta),
         grad_node_stride, _ptr(amax_out), p, nb, _stream()))
+    if dv is None:                      # dx only: the reduction launch belongs to lpdt_range_evonorm_bwd_params
+        global KERNEL_LAUNCHES
+        KERNEL_LAUNCHES -= 1
 
 
 def lpdt_evonorm_s0_fwd(nodes, B, H, W, Cc, groups, eps, x, v, gamma, beta, param_node_stride, y, gmean, gvar):
