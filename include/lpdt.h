@@ -368,6 +368,19 @@ lpdt_status lpdt_deepsqueeze_mix(int32_t nodes, int64_t d, const float *x_half, 
                                  int32_t message_bits, float *msg_scale,
                                  void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
 
+/* The SGD half-step and the UNCOMPRESSED gossip step in one launch (Algorithm 1 "update the model", then
+ * Algorithm 3 with every entry of the difference kept):
+ *   x_half_i = x_i - lr*g_i;  x_hat_i <- x_hat_i + (x_half_i - x_hat_i);
+ *   x_out_i  = x_half_i + gamma * sum_j Wmix[i][j] * (x_hat_j - x_hat_i)
+ * the same fp32 operations in the same order as lpdt_sgd_update followed by lpdt_gossip_mix with
+ * seg_k >= segment length, without the separate update pass over the parameters.
+ * x, g : fp32 [nodes][d] (parameters, gradients);  x_half (out), x_hat (in/out), x_out (out) : fp32 [nodes][d];
+ * the five arrays are distinct.  No workspace.  Errors: INVALID_ARG, UNSUPPORTED (nodes > 64), CUDA.
+ */
+lpdt_status lpdt_sgd_gossip_mix(int32_t nodes, int64_t d, const float *x, const float *g, float lr,
+                                float *x_half, float *x_hat, float *x_out, const float *Wmix, float gamma,
+                                void *stream);
+
 /* Push-sum bias weights and de-biasing (supplementary Algorithms 4 and 5, Sparse-Push and
  * Quant-SGP: second line of the gossip update, then the de-biasing step), for column-stochastic
  * mixing matrices on directed graphs:

@@ -51,6 +51,7 @@ SIGNATURES = {
     "lpdt_gossip_mix_q8": (_i32, [_i32, _i64, _vp, _vp, _vp, _vp, _f32, _i32, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
     "lpdt_deepsqueeze_mix": (_i32, [_i32, _i64, _vp, _vp, _vp, _vp, _f32, _i32, _vp, _vp, _i32, _vp, _vp, _sz, _vp,
                                     _vp]),
+    "lpdt_sgd_gossip_mix": (_i32, [_i32, _i64, _vp, _vp, _f32, _vp, _vp, _vp, _vp, _f32, _vp]),
     "lpdt_pushsum_debias": (_i32, [_i32, _i64, _vp, _vp, _vp, _f32, _vp, _vp, _vp]),
     "lpdt_sgd_update": (_i32, [_i64, _vp, _vp, _f32, _vp, _vp]),
     "lpdt_residual_add": (_i32, [_i32] * 8 + [_vp] * 5),

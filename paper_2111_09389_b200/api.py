@@ -15,7 +15,7 @@ from ._lib import ConvDesc, lib
 KERNELS_PER_CALL = {
     "lpdt_quantize": 2, "lpdt_quantize_with_range": 1, "lpdt_quantize_static": 2, "lpdt_quantize_batch": 2, "lpdt_dequantize": 1, "lpdt_qconv_fwd": 1, "lpdt_qconv_fwd_affine": 4, "lpdt_qconv_bwd_data": 2,
     "lpdt_qconv_bwd_weight": 2, "lpdt_range_evonorm_fwd": 1, "lpdt_range_evonorm_bwd": 2, "lpdt_range_evonorm_bwd_params": 1,
-    "lpdt_gossip_mix": 2, "lpdt_gossip_mix_q8": 3, "lpdt_deepsqueeze_mix": 2, "lpdt_pushsum_debias": 1, "lpdt_evonorm_s0_fwd": 1, "lpdt_evonorm_s0_bwd": 2, "lpdt_range_bn_fwd": 2, "lpdt_range_bn_bwd": 2, "lpdt_sgd_update": 1, "lpdt_residual_add": 1, "lpdt_residual_add_bwd": 1,
+    "lpdt_gossip_mix": 2, "lpdt_gossip_mix_q8": 3, "lpdt_deepsqueeze_mix": 2, "lpdt_pushsum_debias": 1, "lpdt_sgd_gossip_mix": 1, "lpdt_evonorm_s0_fwd": 1, "lpdt_evonorm_s0_bwd": 2, "lpdt_range_bn_fwd": 2, "lpdt_range_bn_bwd": 2, "lpdt_sgd_update": 1, "lpdt_residual_add": 1, "lpdt_residual_add_bwd": 1,
     "lpdt_avgpool": 1, "lpdt_avgpool_bwd": 1, "lpdt_maxpool2x2": 1, "lpdt_maxpool2x2_bwd": 1,
     "lpdt_softmax_ce": 1, "lpdt_colsum": 1,
 }
@@ -285,6 +285,12 @@ def lpdt_deepsqueeze_mix(nodes, d, x_half, delta, x_out, Wmix, eta, seg_offsets,
                                                               _ptr(Wmix), eta, ns, C.addressof(so), C.addressof(sk),
                                                               message_bits, _ptr(msg_scale), p, nb, _ptr(dev_status),
                                                               _stream()))
+
+
+def lpdt_sgd_gossip_mix(nodes, d, x, g, lr, x_half, x_hat, x_out, Wmix, gamma):
+    """SGD half-step + uncompressed gossip step in one launch."""
+    _check("lpdt_sgd_gossip_mix", lib().lpdt_sgd_gossip_mix(nodes, d, _ptr(x), _ptr(g), lr, _ptr(x_half), _ptr(x_hat),
+                                                            _ptr(x_out), _ptr(Wmix), gamma, _stream()))
 
 
 def lpdt_pushsum_debias(nodes, d, x, u, Wmix, eta, u_new, z):

@@ -627,6 +627,91 @@ pushsum_debias_kernel(int nodes, int64_t d, const float *__restrict__ x, const f
     }
 }
 
+
+// SGD half-step fused into the uncompressed gossip step (Algorithm 1 "update the model" followed by Algorithm 3
+// with every entry kept): x_half = x - lr*g is computed where the mix needs it, so the parameters and gradients
+// are read once and the separate update pass (12 B per parameter) disappears.  Same operation order as
+// lpdt_sgd_update followed by lpdt_gossip_mix with dense segments: x_hat <- x_hat + (x_half - x_hat), then the mix
+// over the updated copies.  Every CTA builds the compact rows of W itself (nodes^2 values).
+template <int V>
+__global__ void __launch_bounds__(256)
+sgd_dense_mix_kernel(int nodes, int64_t d, const float *__restrict__ x, const float *__restrict__ g, float lr,
+                     float *x_half, float *__restrict__ x_hat, float *__restrict__ x_out,
+                     const float *__restrict__ Wmix, float gamma) {
+    pdl_enter();
+    extern __shared__ __align__(16) float sm[];
+    const int TE = blockDim.x;
+    int32_t *s_cnt = reinterpret_cast<int32_t *>(sm);            // [nodes]
+    int32_t *s_idx = s_cnt + nodes;                              // [nodes][nodes]
+    float *s_val = reinterpret_cast<float *>(s_idx + nodes * nodes);
+    const int tab_words = nodes + 2 * nodes * nodes;
+    float *s_hat = sm + ((tab_words + 3) & ~3);                  // [nodes][TE][V]
+    for (int i = threadIdx.x; i < nodes; i += TE) {
+        int c = 0;
+        for (int j = 0; j < nodes; ++j) {
+            const float w = Wmix[i * nodes + j];
+            if (w != 0.f) { s_idx[i * nodes + c] = j; s_val[i * nodes + c] = w; ++c; }
+        }
+        s_cnt[i] = c;
+    }
+    __syncthreads();
+    const int64_t e0 = ((int64_t)blockIdx.x * TE + threadIdx.x) * V;
+    if (e0 >= d) return;                                         // d % V == 0: a thread is all in or all out
+    constexpr int kU = 4;
+    for (int ib = 0; ib < nodes; ib += kU) {
+        float xv[kU][V], gv[kU][V], xq[kU][V];
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            if (ib + u < nodes) {
+                VecIO<V>::ld(x + (int64_t)(ib + u) * d + e0, xv[u]);
+                VecIO<V>::ld(g + (int64_t)(ib + u) * d + e0, gv[u]);
+                VecIO<V>::ld(x_hat + (int64_t)(ib + u) * d + e0, xq[u]);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const int i = ib + u;
+            if (i >= nodes) break;
+            float xh[V], hn[V];
+#pragma unroll
+            for (int k = 0; k < V; ++k) {
+                xh[k] = __fsub_rn(xv[u][k], __fmul_rn(lr, gv[u][k]));
+                hn[k] = __fadd_rn(xq[u][k], __fsub_rn(xh[k], xq[u][k]));
+            }
+            VecIO<V>::st(x_half + (int64_t)i * d + e0, xh);
+            VecIO<V>::st(x_hat + (int64_t)i * d + e0, hn);
+            VecIO<V>::st(s_hat + ((size_t)i * TE + threadIdx.x) * V, hn);
+        }
+    }
+    for (int ib = 0; ib < nodes; ib += kU) {
+        float xh[kU][V];
+#pragma unroll
+        for (int u = 0; u < kU; ++u)           // written above by this thread (plain pointer: no read-only path)
+            if (ib + u < nodes) VecIO<V>::ld(x_half + (int64_t)(ib + u) * d + e0, xh[u]);
+#pragma unroll
+        for (int u = 0; u < kU; ++u) {
+            const int i = ib + u;
+            if (i >= nodes) break;
+            float hi_[V], acc[V], o[V];
+            VecIO<V>::ld(s_hat + ((size_t)i * TE + threadIdx.x) * V, hi_);
+#pragma unroll
+            for (int k = 0; k < V; ++k) acc[k] = 0.f;
+            const int c = s_cnt[i];
+            for (int m = 0; m < c; ++m) {                        // neighbours in ascending j
+                const int j = s_idx[i * nodes + m];
+                const float w = s_val[i * nodes + m];
+                float hj[V];
+                VecIO<V>::ld(s_hat + ((size_t)j * TE + threadIdx.x) * V, hj);
+#pragma unroll
+                for (int k = 0; k < V; ++k) acc[k] = __fadd_rn(acc[k], __fmul_rn(w, __fsub_rn(hj[k], hi_[k])));
+            }
+#pragma unroll
+            for (int k = 0; k < V; ++k) o[k] = __fadd_rn(xh[u][k], __fmul_rn(gamma, acc[k]));
+            VecIO<V>::st(x_out + (int64_t)i * d + e0, o);
+        }
+    }
+}
+
 }  // namespace lpdt
 
 using namespace lpdt;
@@ -803,6 +888,42 @@ extern "C" lpdt_status lpdt_pushsum_debias(int32_t nodes, int64_t d, const float
     const dim3 g((unsigned)chunks, nodes);
     if (v4) launch_k(pushsum_debias_kernel<4>, g, 256, 0, st, nodes, d, x, u, Wmix, eta, u_new, z);
     else launch_k(pushsum_debias_kernel<1>, g, 256, 0, st, nodes, d, x, u, Wmix, eta, u_new, z);
+    LPDT_LAUNCH_CHECK();
+    return LPDT_OK;
+}
+
+extern "C" lpdt_status lpdt_sgd_gossip_mix(int32_t nodes, int64_t d, const float *x, const float *g, float lr,
+                                           float *x_half, float *x_hat, float *x_out, const float *Wmix, float gamma,
+                                           void *stream) {
+    LPDT_CHECK_ARG(nodes >= 0 && d >= 0);
+    if (nodes == 0 || d == 0) return LPDT_OK;
+    LPDT_CHECK_ARG(x && g && x_half && x_hat && x_out && Wmix);
+    LPDT_CHECK_ARG(x_half != x && x_half != g && x_hat != x_half && x_out != x_half && x_out != x_hat && x_out != x &&
+                   x_out != g && x_hat != x && x_hat != g);
+    if (nodes > kMaxNodes) return LPDT_ERR_UNSUPPORTED;
+    const float *in[2] = {x, g};
+    float *io[3] = {x_half, x_hat, x_out};
+    bool a16 = d % 4 == 0, a8 = d % 2 == 0;
+    for (int i = 0; i < 2; ++i) { a16 = a16 && aligned(in[i], 16); a8 = a8 && aligned(in[i], 8); }
+    for (int i = 0; i < 3; ++i) { a16 = a16 && aligned(io[i], 16); a8 = a8 && aligned(io[i], 8); }
+    const int V = a16 ? 4 : a8 ? 2 : 1;
+    int TE = (int)((64 * 1024) / ((size_t)nodes * V * sizeof(float))) / 32 * 32;
+    if (TE > 128) TE = 128;
+    if (TE < 32) TE = 32;
+    const size_t tab_words = ((size_t)nodes + 2 * (size_t)nodes * nodes + 3) & ~(size_t)3;
+    const size_t smem = tab_words * sizeof(int32_t) + (size_t)nodes * TE * V * sizeof(float);
+    using Fn = void (*)(int, int64_t, const float *, const float *, float, float *, float *, float *, const float *, float);
+    static const Fn fns[3] = {sgd_dense_mix_kernel<1>, sgd_dense_mix_kernel<2>, sgd_dense_mix_kernel<4>};
+    static bool attr_set = false;
+    if (!attr_set) {
+        for (int i = 0; i < 3; ++i)
+            LPDT_CUDA(cudaFuncSetAttribute(fns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
+        attr_set = true;
+    }
+    const int64_t blocks = ceil_div(d, (int64_t)TE * V);
+    if (blocks > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
+    launch_k(fns[V == 4 ? 2 : V == 2 ? 1 : 0], (unsigned)blocks, TE, smem, as_stream(stream), nodes, d, x, g, lr, x_half,
+             x_hat, x_out, Wmix, gamma);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

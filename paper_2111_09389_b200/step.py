@@ -331,6 +331,12 @@ class TrainStep:
 
     def update(self):
         N, d = self.N, self.d
+        dense = all(k >= hi - lo for k, lo, hi in zip(self.seg_k, self.seg_offsets[:-1], self.seg_offsets[1:]))
+        if dense and self.message_bits != 8:
+            # no compression: the half-step is computed inside the mix kernel (one pass over parameters and gradients)
+            api.lpdt_sgd_gossip_mix(N, d, self.params, self.grads, self.lr, self.x_half, self.x_hat, self.x_out,
+                                    self.Wmix, self.gamma)
+            return
         api.lpdt_sgd_update(N * d, self.params, self.grads, self.lr, self.x_half)
         if self.message_bits == 8:
             api.lpdt_gossip_mix_q8(N, d, self.x_half, self.x_hat, self.x_out, self.Wmix, self.gamma,

@@ -609,6 +609,28 @@ def test_deepsqueeze_mix(nodes, d, segs, bits):
         x_in = (x_ref - 0.05 * rng.standard_normal((nodes, d))).astype(np.float32)      # a stand-in local update
 
 
+@pytest.mark.parametrize("nodes,d", [(4, 2736), (16, 10007), (8, 270410), (64, 300), (1, 777), (3, 100002)])
+def test_sgd_gossip_mix(nodes, d):
+    """Fused half-step + dense mix: x_half and x_hat bit-equal to lpdt_sgd_update / the oracle, x within the fp32 bar;
+    also bit-equal to the two separate launches."""
+    rng = np.random.default_rng(nodes + d)
+    x = rng.standard_normal((nodes, d)).astype(np.float32)
+    g = rng.standard_normal((nodes, d)).astype(np.float32)
+    xhat = (x - 0.1 * rng.standard_normal((nodes, d))).astype(np.float32)
+    W = wlmod.ring_matrix(nodes) if nodes >= 3 else np.full((nodes, nodes), 1.0 / nodes, np.float32)
+    xh_ref = oracle.sgd_update(x, g, 0.1)
+    x_ref, xhat_ref, _ = oracle.gossip_mix(xh_ref, xhat, W, 0.9, [0, d], [d])
+    xhd, xhatd, xo = torch.empty(nodes, d, device="cuda"), dev(xhat), torch.empty(nodes, d, device="cuda")
+    api.lpdt_sgd_gossip_mix(nodes, d, dev(x), dev(g), 0.1, xhd, xhatd, xo, dev(W), 0.9)
+    assert np.array_equal(xhd.cpu().numpy(), xh_ref) and np.array_equal(xhatd.cpu().numpy(), xhat_ref)
+    close(xo, x_ref)
+    xh2, xhat2, xo2 = torch.empty(nodes, d, device="cuda"), dev(xhat), torch.empty(nodes, d, device="cuda")
+    api.lpdt_sgd_update(nodes * d, dev(x), dev(g), 0.1, xh2)
+    api.lpdt_gossip_mix(nodes, d, xh2, xhat2, xo2, dev(W), 0.9, [0, d], [d],
+                        ws_bytes(api.lpdt_gossip_mix_workspace_size(nodes, d, 1)))
+    assert torch.equal(xo, xo2) and torch.equal(xhatd, xhat2)
+
+
 def directed_ring_matrix(n, rng):
     """Column-stochastic, not row-stochastic: node j keeps a share and pushes the rest to j+1 and j+2."""
     W = np.zeros((n, n), np.float32)
