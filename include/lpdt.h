@@ -64,6 +64,18 @@ const char *lpdt_version(void);
 const char *lpdt_status_string(lpdt_status s);
 /* Enqueue a zero fill of `bytes` bytes at device pointer p (range accumulators, status words). */
 lpdt_status lpdt_fill_zero(void *p, size_t bytes, void *stream);
+/* Read a status word back: waits until everything enqueued on `stream` so far has finished (the one
+ * call of this library that synchronises), then returns the value of *dev_status: LPDT_OK, or the
+ * code a kernel recorded there (LPDT_ERR_TIMEOUT from a bounded wait that ran out,
+ * LPDT_ERR_INVALID_ARG from an out-of-range label).  LPDT_ERR_CUDA if the copy or the wait fails.
+ * The word is not cleared. */
+lpdt_status lpdt_check_status(const int32_t *dev_status, void *stream);
+/* Diagnostics (no counterpart in the paper): runs the bounded barrier wait of the tensor-core
+ * kernels on a barrier that nothing arrives at, with a limit of limit_ns nanoseconds (1 us to
+ * 50 ms; INVALID_ARG outside).  The one-CTA kernel returns once the limit has passed, writes
+ * LPDT_ERR_TIMEOUT to *dev_status and 2 to *returned (nullable; 1 would mean the wait succeeded).
+ * The production kernels use the same routine with a limit of two seconds. */
+lpdt_status lpdt_selftest_bounded_wait(uint64_t limit_ns, int32_t *dev_status, int32_t *returned, void *stream);
 
 /* ---------------------------------------------------------------------------
  * lpdt_quantize — per-tensor, per-node 8-bit quantization.
@@ -138,8 +150,12 @@ lpdt_status lpdt_dequantize(const int8_t *q, int32_t nodes, int64_t n_per_node,
  * gone.  Limits and rules:
  *   - nodes <= LPDT_QUANTIZE_STATIC_MAX_NODES, otherwise LPDT_ERR_WORKSPACE
  *     (the built-in scratch is too small) and nothing is enqueued.
- *   - The first call on each device looks up the array's device address (with
- *     that device current); make that first call before any stream capture.
+ *   - The first call on each device that has work to do (nodes > 0 and
+ *     n_per_node > 0) looks up the array's device address; make that first call
+ *     before any stream capture.  The device that owns `stream` must be the
+ *     current device, as for every call of this library.  The looked-up address
+ *     is cached per device ordinal and does not survive a cudaDeviceReset in
+ *     the same process.
  *   - All calls share the one array, so two calls whose kernels may overlap on
  *     the GPU (different streams, no ordering between them) race; calls on one
  *     stream, or otherwise ordered, are safe.  The words a call uses are cleared
@@ -353,6 +369,18 @@ lpdt_status lpdt_gossip_mix_q8(int32_t nodes, int64_t d, const float *x_half, fl
                                const int64_t *seg_offsets, const int64_t *seg_k, float *msg_scale,
                                void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
 
+/* Bytes one node hands to EACH neighbour in one gossip step (host arithmetic, no device work), the
+ * quantity behind the Data column of the paper's CIFAR table (data sent per node over a run =
+ * this x iterations; the table's full-precision rows are 32-bit values, its low-precision rows
+ * exactly a quarter of them):
+ *   sum over segments of  k_s*value_bits + (k_s < len_s ? k_s*index_bits : 0) + (value_bits == 8 && k_s > 0 ? 32 : 0)
+ * bits, rounded up to bytes, with k_s = min(seg_k[s], len_s): kept values, their positions inside
+ * the segment when the segment is compressed, and the fp32 step of a segment sent as 8-bit codes.
+ * seg_offsets / seg_k : HOST arrays as in lpdt_gossip_mix;  value_bits 32, 16 or 8;  index_bits 0..64
+ * (0 = count values only).  Returns -1 for invalid arguments. */
+int64_t lpdt_message_bytes(int64_t d, int32_t n_segments, const int64_t *seg_offsets, const int64_t *seg_k,
+                           int32_t value_bits, int32_t index_bits);
+
 /* Deep-Squeeze gossip step (supplementary Algorithm 2, steps 5-10) for all nodes:
  *   v_i = x_half_i + delta_i;  c_i = C[v_i];  delta_i <- v_i - c_i;
  *   x_i = x_half_i + eta * (sum_j W_ij c_j - c_i)
@@ -430,9 +458,14 @@ lpdt_status lpdt_maxpool2x2_bwd(int32_t nodes, int32_t B, int32_t H, int32_t W, 
                                 const float *dy, const int8_t *idx, float *dx, void *stream);
 
 /* Softmax cross-entropy per node (mean over the node's batch):
- * loss[n], dlogits = (softmax - onehot)/B.  logits fp32 [nodes][B][K], labels int32. */
+ * loss[n], dlogits = (softmax - onehot)/B.  logits fp32 [nodes][B][K], labels int32 [nodes][B].
+ * Labels must lie in [0, K).  The kernel checks each one before using it: a sample whose label
+ * is out of range adds nothing to its node's loss, gets dlogits = softmax/B (no one-hot term), and
+ * LPDT_ERR_INVALID_ARG is written to dev_status (one int32, caller-zeroed, nullable); no memory
+ * outside the logits row is touched. */
 lpdt_status lpdt_softmax_ce(int32_t nodes, int32_t B, int32_t K, const float *logits,
-                            const int32_t *labels, float *loss, float *dlogits, void *stream);
+                            const int32_t *labels, float *loss, float *dlogits, int32_t *dev_status,
+                            void *stream);
 
 /* out[n][c] = sum_b x[n][b][c] (bias gradient); node n of out at out + n*out_node_stride. */
 lpdt_status lpdt_colsum(int32_t nodes, int32_t B, int32_t C, const float *x,

@@ -22,6 +22,9 @@ SIGNATURES = {
     "lpdt_version": (C.c_char_p, []),
     "lpdt_status_string": (C.c_char_p, [_i32]),
     "lpdt_fill_zero": (_i32, [_vp, _sz, _vp]),
+    "lpdt_check_status": (_i32, [_vp, _vp]),
+    "lpdt_selftest_bounded_wait": (_i32, [_u64, _vp, _vp, _vp]),
+    "lpdt_message_bytes": (_i64, [_i64, _i32, _vp, _vp, _i32, _i32]),
     "lpdt_quantize_workspace_size": (_sz, [_i32]),
     "lpdt_quantize": (_i32, [_vp, _i32, _i64, _i64, _i32, _i32, _u64, _u32, _vp, _vp, _vp, _vp, _sz, _vp]),
     "lpdt_quantize_static": (_i32, [_vp, _i32, _i64, _i64, _i32, _i32, _u64, _u32, _vp, _vp, _vp, _vp]),
@@ -60,7 +63,7 @@ SIGNATURES = {
     "lpdt_avgpool_bwd": (_i32, [_i32] * 4 + [_vp] * 3),
     "lpdt_maxpool2x2": (_i32, [_i32] * 5 + [_vp] * 4),
     "lpdt_maxpool2x2_bwd": (_i32, [_i32] * 5 + [_vp] * 4),
-    "lpdt_softmax_ce": (_i32, [_i32] * 3 + [_vp] * 5),
+    "lpdt_softmax_ce": (_i32, [_i32] * 3 + [_vp] * 6),
     "lpdt_colsum": (_i32, [_i32] * 3 + [_vp, _vp, _i64, _vp]),
 }
 

@@ -17,7 +17,7 @@ KERNELS_PER_CALL = {
     "lpdt_qconv_bwd_weight": 2, "lpdt_range_evonorm_fwd": 1, "lpdt_range_evonorm_bwd": 2, "lpdt_range_evonorm_bwd_params": 1,
     "lpdt_gossip_mix": 2, "lpdt_gossip_mix_q8": 3, "lpdt_deepsqueeze_mix": 2, "lpdt_pushsum_debias": 1, "lpdt_sgd_gossip_mix": 1, "lpdt_evonorm_s0_fwd": 1, "lpdt_evonorm_s0_bwd": 2, "lpdt_range_bn_fwd": 2, "lpdt_range_bn_bwd": 2, "lpdt_sgd_update": 1, "lpdt_residual_add": 1, "lpdt_residual_add_bwd": 1,
     "lpdt_avgpool": 1, "lpdt_avgpool_bwd": 1, "lpdt_maxpool2x2": 1, "lpdt_maxpool2x2_bwd": 1,
-    "lpdt_softmax_ce": 1, "lpdt_colsum": 1,
+    "lpdt_softmax_ce": 1, "lpdt_colsum": 1, "lpdt_selftest_bounded_wait": 1,
 }
 KERNEL_LAUNCHES = 0
 # Optional per-entry-point timing: {name: [(start_event, end_event), ...]} when TIMED holds names.
@@ -105,6 +105,24 @@ def lpdt_quantize_with_range(x, nodes, n_per_node, x_node_stride, amax, q, scale
 
 def lpdt_fill_zero(t):
     _check("lpdt_fill_zero", lib().lpdt_fill_zero(_ptr(t), t.numel() * t.element_size(), _stream()))
+
+
+def lpdt_check_status(dev_status):
+    """Waits for the current stream and returns the status word (0 = ok); raises nothing."""
+    return int(lib().lpdt_check_status(_ptr(dev_status), _stream()))
+
+
+def lpdt_selftest_bounded_wait(limit_ns, dev_status, returned=None):
+    _check("lpdt_selftest_bounded_wait", lib().lpdt_selftest_bounded_wait(int(limit_ns), _ptr(dev_status),
+                                                                          _ptr(returned), _stream()))
+
+
+def lpdt_message_bytes(d, seg_offsets, seg_k, value_bits=32, index_bits=32):
+    """Bytes one node sends to each neighbour per gossip step (host arithmetic in the library)."""
+    ns = len(seg_k)
+    so = (C.c_int64 * (ns + 1))(*[int(v) for v in seg_offsets])
+    sk = (C.c_int64 * ns)(*[int(v) for v in seg_k])
+    return int(lib().lpdt_message_bytes(int(d), ns, C.addressof(so), C.addressof(sk), value_bits, index_bits))
 
 
 def lpdt_quantize_batch_workspace_size(nodes, n_tensors):
@@ -330,9 +348,9 @@ def lpdt_maxpool2x2_bwd(nodes, B, H, W, Cc, dy, idx, dx):
                                                             _stream()))
 
 
-def lpdt_softmax_ce(nodes, B, K, logits, labels, loss, dlogits):
+def lpdt_softmax_ce(nodes, B, K, logits, labels, loss, dlogits, dev_status=None):
     _check("lpdt_softmax_ce", lib().lpdt_softmax_ce(nodes, B, K, _ptr(logits), _ptr(labels), _ptr(loss),
-                                                    _ptr(dlogits), _stream()))
+                                                    _ptr(dlogits), _ptr(dev_status), _stream()))
 
 
 def lpdt_colsum(nodes, B, Cc, x, out, out_node_stride):

@@ -1,6 +1,7 @@
 // Shared host/device helpers of the lpdt CUDA library (not part of the ABI).
 #pragma once
 #include <cuda_runtime.h>
+#include <atomic>
 #include <stdint.h>
 #include <stdlib.h>
 #include "../../include/lpdt.h"
@@ -31,6 +32,21 @@ static inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 constexpr int kNumSMs = 148;  // B200
+
+// A kernel attribute (the opt-in dynamic shared memory limit) belongs to the device it was set on, so
+// "already set" is remembered per device ordinal: one bit per device, devices beyond 63 set it every call.
+struct PerDeviceOnce {
+    std::atomic<unsigned long long> done{0};
+    // true when the attribute still has to be set on the current device; *dev receives its ordinal
+    bool pending(int *dev) {
+        *dev = -1;
+        if (cudaGetDevice(dev) != cudaSuccess || *dev < 0 || *dev >= 64) return true;
+        return !((done.load(std::memory_order_acquire) >> *dev) & 1ull);
+    }
+    void mark(int dev) {
+        if (dev >= 0 && dev < 64) done.fetch_or(1ull << dev, std::memory_order_release);
+    }
+};
 
 // Programmatic dependent launch.  Every kernel of the library waits for the grids before it
 // in the stream (griddepcontrol.wait returns once they have completed and their writes are

@@ -223,9 +223,11 @@ __global__ void maxpool_bwd_v4_kernel(int64_t NB, int H, int W, int C4, const fl
 }
 
 // One block per node, one thread per sample; double arithmetic, fixed-order tree.
+// A label outside [0, K) is never used as an index: that sample adds nothing to the loss, its gradient is the
+// plain softmax/B, and LPDT_ERR_INVALID_ARG is written to the status word.
 __global__ void softmax_ce_kernel(int B, int K, const float *__restrict__ logits,
                                   const int32_t *__restrict__ labels, float *__restrict__ loss,
-                                  float *__restrict__ dlogits) {
+                                  float *__restrict__ dlogits, int32_t *__restrict__ dev_status) {
     pdl_enter();
     extern __shared__ double s_part[];
     const int n = blockIdx.x;
@@ -238,7 +240,9 @@ __global__ void softmax_ce_kernel(int B, int K, const float *__restrict__ logits
         double den = 0.0;
         for (int k = 0; k < K; ++k) den += exp((double)z[k] - zmax);
         const int lab = labels[(int64_t)n * B + b];
-        mine += log(den) + zmax - (double)z[lab];
+        const bool lab_ok = lab >= 0 && lab < K;
+        if (lab_ok) mine += log(den) + zmax - (double)z[lab];
+        else if (dev_status) atomicCAS(dev_status, 0, (int32_t)LPDT_ERR_INVALID_ARG);
         for (int k = 0; k < K; ++k) {
             double p = exp((double)z[k] - zmax) / den;
             dz[k] = (float)((p - (k == lab ? 1.0 : 0.0)) / (double)B);
@@ -374,14 +378,15 @@ extern "C" lpdt_status lpdt_maxpool2x2_bwd(int32_t nodes, int32_t B, int32_t H, 
 }
 
 extern "C" lpdt_status lpdt_softmax_ce(int32_t nodes, int32_t B, int32_t K, const float *logits,
-                                       const int32_t *labels, float *loss, float *dlogits, void *stream) {
+                                       const int32_t *labels, float *loss, float *dlogits, int32_t *dev_status,
+                                       void *stream) {
     LPDT_CHECK_ARG(nodes >= 0 && B > 0 && K > 0);
     if (nodes == 0) return LPDT_OK;
     LPDT_CHECK_ARG(logits && labels && loss && dlogits);
     int threads = 32;
     while (threads < B && threads < 256) threads <<= 1;
     launch_k(softmax_ce_kernel, nodes, threads, threads * sizeof(double), as_stream(stream), B, K, logits, labels,
-                                                                                     loss, dlogits);
+             loss, dlogits, dev_status);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

@@ -834,11 +834,12 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
         gossip_mix_kernel<1, true, false>,  gossip_mix_kernel<2, true, false>,  gossip_mix_kernel<4, true, false>,
         gossip_mix_kernel<1, false, true>,  gossip_mix_kernel<2, false, true>,  gossip_mix_kernel<4, false, true>,
         gossip_mix_kernel<1, true, true>,   gossip_mix_kernel<2, true, true>,   gossip_mix_kernel<4, true, true>};
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce attr_set;
+    int dev;
+    if (attr_set.pending(&dev)) {
         for (int i = 0; i < 12; ++i)
             LPDT_CUDA(cudaFuncSetAttribute(fns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
-        attr_set = true;
+        attr_set.mark(dev);
     }
     const unsigned blocks = (unsigned)ceil_div(d, (int64_t)TE * V);
     launch_k(fns[(ds ? 6 : 0) + (q8 ? 3 : 0) + vi], blocks, TE, smem, st, nodes, d, x_half, x_hat, x_out, gamma, seg, sel, tab,
@@ -914,11 +915,12 @@ extern "C" lpdt_status lpdt_sgd_gossip_mix(int32_t nodes, int64_t d, const float
     const size_t smem = tab_words * sizeof(int32_t) + (size_t)nodes * TE * V * sizeof(float);
     using Fn = void (*)(int, int64_t, const float *, const float *, float, float *, float *, float *, const float *, float);
     static const Fn fns[3] = {sgd_dense_mix_kernel<1>, sgd_dense_mix_kernel<2>, sgd_dense_mix_kernel<4>};
-    static bool attr_set = false;
-    if (!attr_set) {
+    static PerDeviceOnce attr_set;
+    int dev;
+    if (attr_set.pending(&dev)) {
         for (int i = 0; i < 3; ++i)
             LPDT_CUDA(cudaFuncSetAttribute(fns[i], cudaFuncAttributeMaxDynamicSharedMemorySize, 128 * 1024));
-        attr_set = true;
+        attr_set.mark(dev);
     }
     const int64_t blocks = ceil_div(d, (int64_t)TE * V);
     if (blocks > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;

@@ -216,13 +216,16 @@ lpdt_status generic_bwd_weight(const lpdt_conv_desc &d, const int8_t *E, const f
                                cudaStream_t st) {
     const int Ho = conv_out(d.H, d.pad, d.R, d.stride), Wo = conv_out(d.W, d.pad, d.S, d.stride);
     const int64_t per_node = (int64_t)d.Cout * d.R * d.S * d.Cin;
+    if (d.nodes > 65535) return LPDT_ERR_UNSUPPORTED;        // nodes ride in grid.y
     int32_t *acc = dWacc ? dWacc : (int32_t *)ws;
     LPDT_CUDA(cudaMemsetAsync(acc, 0, (size_t)d.nodes * per_node * sizeof(int32_t), st));
     const int64_t npix = (int64_t)d.B * Ho * Wo;
-    int chunk = 4;
-    while (ceil_div(npix, chunk) * d.nodes > (int64_t)kNumSMs * 16) chunk *= 2;
-    launch_k(conv_bwd_weight_generic, dim3((unsigned)ceil_div(npix, chunk), d.nodes), 256, 0, st, d, Ho, Wo, chunk, E, A, acc);
-    LPDT_LAUNCH_CHECK();
+    if (npix > 0) {                      // an empty batch leaves the zeroed sums: the gradient of no samples
+        int chunk = 4;
+        while (ceil_div(npix, chunk) * d.nodes > (int64_t)kNumSMs * 16) chunk *= 2;
+        launch_k(conv_bwd_weight_generic, dim3((unsigned)ceil_div(npix, chunk), d.nodes), 256, 0, st, d, Ho, Wo, chunk, E, A, acc);
+        LPDT_LAUNCH_CHECK();
+    }
     if (dW) {
         launch_k(dequant_acc_kernel, grid_for(per_node * d.nodes), 256, 0, st, acc, d.nodes, per_node, sE, sA, dW, dw_stride);
         LPDT_LAUNCH_CHECK();

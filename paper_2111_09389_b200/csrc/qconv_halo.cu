@@ -429,10 +429,11 @@ lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, cons
     size_t smem = 1024 + (size_t)p.wres_bytes + (size_t)p.stages * p.halo_bytes + kZeroBytes + out_bytes;
     const size_t smem_floor = (size_t)(228 * 1024) / (per_sm + 1);     // keeps the (per_sm + 1)-th CTA out
     if (smem < smem_floor) smem = smem_floor;
-    static bool attr = false;
-    if (!attr) {
+    static PerDeviceOnce attr;
+    int dev;
+    if (attr.pending(&dev)) {
         LPDT_CUDA(cudaFuncSetAttribute(conv_halo16_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        attr = true;
+        attr.mark(dev);
     }
     const long long tiles = (long long)p.nodes * p.B * p.tilesH * p.tilesW;
     if (tiles > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;

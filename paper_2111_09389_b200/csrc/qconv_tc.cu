@@ -646,10 +646,11 @@ lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const flo
     else if (!weight_map(&mW, Wq, d.nodes, d.Cout, d.R * d.S, d.Cin, p.RBn, p.RBa)) return LPDT_ERR_CUDA;
     size_t smem = 1024 + (size_t)p.stages * stage_bytes;
     if (smem < kMinSmem) smem = kMinSmem;
-    static bool attr = false;
-    if (!attr) {
+    static PerDeviceOnce attr;
+    int dev;
+    if (attr.pending(&dev)) {
         LPDT_CUDA(cudaFuncSetAttribute(conv_pix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        attr = true;
+        attr.mark(dev);
     }
     const long long tiles = (long long)p.nodes * p.tilesB * p.tilesH * p.tilesW * p.tilesN * p.ncls;
     if (tiles > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
@@ -735,10 +736,11 @@ lpdt_status tc_wgrad(const lpdt_conv_desc &d, int cin_real, const int8_t *E, con
     size_t smem = 1024 + (size_t)p.stages * stage_bytes;
     if (smem < (size_t)(228 * 1024) / (per_sm + 1)) smem = (size_t)(228 * 1024) / (per_sm + 1);
     if (smem > 227 * 1024) return LPDT_ERR_UNSUPPORTED;
-    static bool attr = false;
-    if (!attr) {
+    static PerDeviceOnce attr;
+    int dev;
+    if (attr.pending(&dev)) {
         LPDT_CUDA(cudaFuncSetAttribute(conv_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        attr = true;
+        attr.mark(dev);
     }
     if (d.nodes > 65535 || p.mgroups * p.ngroups > 65535) return LPDT_ERR_UNSUPPORTED;
     const int64_t per_node = (int64_t)d.Cout * p.taps * cin_real;

@@ -2,6 +2,7 @@
 // scale-and-round pass (Section 3, "Low Precision Training").  Both passes are
 // HBM-bound streaming kernels: 16-byte loads, warp-shuffle reduction of the
 // range, one atomic per block; the second pass stores 4 codes per thread.
+#include <atomic>
 #include "common.cuh"
 
 namespace lpdt {
@@ -288,22 +289,25 @@ extern "C" lpdt_status lpdt_quantize_with_range(const float *x, int32_t nodes, i
 constexpr int kStaticMaxNodes = LPDT_QUANTIZE_STATIC_MAX_NODES;
 static __device__ __align__(256) uint32_t g_static_range_words[2 * kStaticMaxNodes];
 
+// One cached address per device ordinal.  Two host threads that both make the first call on a device
+// look the same address up and store the same value (an atomic pointer store), so the race is benign.
+// The cache does not outlive a cudaDeviceReset: after one, the library must be reloaded.
 constexpr int kMaxDevices = 64;
-static uint32_t *g_static_range_ptr[kMaxDevices] = {};
+static std::atomic<uint32_t *> g_static_range_ptr[kMaxDevices];
 
 static lpdt_status static_range_words(uint32_t **out) {
     int dev = -1;
     LPDT_CUDA(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices) return LPDT_ERR_UNSUPPORTED;
-    if (!g_static_range_ptr[dev]) {
-        uint32_t *p = nullptr;
+    uint32_t *p = g_static_range_ptr[dev].load(std::memory_order_acquire);
+    if (!p) {
         if (cudaGetSymbolAddress((void **)&p, g_static_range_words) != cudaSuccess || !p) {
             (void)cudaGetLastError();
             return LPDT_ERR_CUDA;
         }
-        g_static_range_ptr[dev] = p;
+        g_static_range_ptr[dev].store(p, std::memory_order_release);
     }
-    *out = g_static_range_ptr[dev];
+    *out = p;
     return LPDT_OK;
 }
 
@@ -311,8 +315,9 @@ extern "C" lpdt_status lpdt_quantize_static(const float *x, int32_t nodes, int64
                                             int64_t x_node_stride, lpdt_qmode mode, lpdt_round rounding,
                                             uint64_t seed, uint32_t ctr_offset, int8_t *q, float *scale,
                                             int32_t *zero_point, void *stream) {
-    LPDT_CHECK_ARG(nodes >= 0);
+    LPDT_CHECK_ARG(nodes >= 0 && n_per_node >= 0);
     if (nodes > kStaticMaxNodes) return LPDT_ERR_WORKSPACE;     // the built-in scratch holds 1024 nodes
+    if (nodes == 0 || n_per_node == 0) return LPDT_OK;          // nothing to do: no address lookup either
     uint32_t *words = nullptr;
     lpdt_status s = static_range_words(&words);
     if (s != LPDT_OK) return s;

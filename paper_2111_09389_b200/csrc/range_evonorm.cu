@@ -251,18 +251,17 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
         vc[k] = v[(int64_t)node * pstride + c0 + k];
         gc[k] = gamma[(int64_t)node * pstride + c0 + k];
     }
-    // S feeds dx (and through it the next quantizer): accumulated in double term by term.
-    // The per-channel parameter-gradient sums take a short fp32 run per thread (at most
-    // kRunLen terms) before they join the double accumulators.
-    constexpr int kRunLen = 16;
+    // Every sum is accumulated in double term by term: S feeds dx (and through it the next
+    // quantizer), and the per-channel parameter-gradient sums then differ from a serial double
+    // sum of the same fp32 terms only by double rounding noise.
     // max|dx| for the consumer's quantizer: the two extremum positions are left out here and
     // added after their correction
     const int g_amx = argmax[sg], g_amn = argmin[sg];
     float dmax = 0.f;
     double S = 0.0;
-    float fb[V], fg[V], fv[V];
+    double fb[V], fg[V], fv[V];
 #pragma unroll
-    for (int k = 0; k < V; ++k) { fb[k] = 0.f; fg[k] = 0.f; fv[k] = 0.f; }
+    for (int k = 0; k < V; ++k) { fb[k] = 0.0; fg[k] = 0.0; fv[k] = 0.0; }
     __syncthreads();   // s_ch zeroed
     const int iters = (HW - 1) / rstep + 1;          // same trip count for every thread (rows are predicated)
     auto term = [&](int p, const float (&xv)[V], const float (&dv_)[V]) {
@@ -278,9 +277,9 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
             o[k] = __fmul_rn(__fmul_rn(tt, __fadd_rn(hs, __fmul_rn(u, hp))), invD);
             const int idx = p * C + c0 + k;
             if (idx != g_amx && idx != g_amn) dmax = fmaxf(dmax, fabsf(o[k]));
-            fb[k] = __fadd_rn(fb[k], dv_[k]);
-            fg[k] = __fadd_rn(fg[k], __fmul_rn(dv_[k], __fmul_rn(m, invD)));
-            fv[k] = __fadd_rn(fv[k], __fmul_rn(__fmul_rn(__fmul_rn(tt, __fmul_rn(xv[k], xv[k])), hp), invD));
+            fb[k] += (double)dv_[k];
+            fg[k] += (double)__fmul_rn(dv_[k], __fmul_rn(m, invD));
+            fv[k] += (double)__fmul_rn(__fmul_rn(__fmul_rn(tt, __fmul_rn(xv[k], xv[k])), hp), invD);
         }
         VecLoad<V>::st(dxs + (int64_t)p * C + c0, o);
     };
@@ -293,29 +292,24 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
         if (ok1) { VecLoad<V>::ld(xs + (int64_t)p1 * C + c0, xb); VecLoad<V>::ld(dys + (int64_t)p1 * C + c0, db); }
         if (ok0) term(p0, xa, da);
         if (ok1) term(p1, xb, db);
-        if ((i + 2) % kRunLen == 0 || i + 2 >= iters) {      // uniform across the block
+    }
 #pragma unroll
-            for (int k = 0; k < V; ++k) {
-                double a = (double)fv[k], b = (double)fg[k], c = (double)fb[k];
-                if (fold) {
-                    for (int o = 16; o >= CV; o >>= 1) {
-                        a += __shfl_xor_sync(0xffffffffu, a, o);
-                        b += __shfl_xor_sync(0xffffffffu, b, o);
-                        c += __shfl_xor_sync(0xffffffffu, c, o);
-                    }
-                }
-                if (fold) {
-                    if ((t & 31) < CV) {                 // this lane alone owns these three slots of its warp's set
-                        double *mine = s_ch + (size_t)(t >> 5) * 3 * C + c0 + k;
-                        mine[0] += a; mine[C] += b; mine[2 * C] += c;
-                    }
-                } else {
-                    atomicAdd(&s_ch[0 * C + c0 + k], a);
-                    atomicAdd(&s_ch[1 * C + c0 + k], b);
-                    atomicAdd(&s_ch[2 * C + c0 + k], c);
-                }
-                fb[k] = 0.f; fg[k] = 0.f; fv[k] = 0.f;
+    for (int k = 0; k < V; ++k) {
+        double a = fv[k], b = fg[k], c = fb[k];
+        if (fold) {
+            for (int o = 16; o >= CV; o >>= 1) {
+                a += __shfl_xor_sync(0xffffffffu, a, o);
+                b += __shfl_xor_sync(0xffffffffu, b, o);
+                c += __shfl_xor_sync(0xffffffffu, c, o);
             }
+            if ((t & 31) < CV) {                 // this lane alone owns these three slots of its warp's set
+                double *mine = s_ch + (size_t)(t >> 5) * 3 * C + c0 + k;
+                mine[0] = a; mine[C] = b; mine[2 * C] = c;
+            }
+        } else {
+            atomicAdd(&s_ch[0 * C + c0 + k], a);
+            atomicAdd(&s_ch[1 * C + c0 + k], b);
+            atomicAdd(&s_ch[2 * C + c0 + k], c);
         }
     }
     s_S[t] = S;

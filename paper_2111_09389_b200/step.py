@@ -238,7 +238,7 @@ class TrainStep:
         N, B, d = self.N, self.B, self.d
         if self.labels is not None:
             K = self.out.numel() // (N * B)
-            api.lpdt_softmax_ce(N, B, K, self.out, self.labels, self.loss, self.dy)
+            api.lpdt_softmax_ce(N, B, K, self.out, self.labels, self.loss, self.dy, self.dev_status)
         g = self.dy
         g_range = None
         L = len(self.ops)

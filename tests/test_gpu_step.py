@@ -32,8 +32,7 @@ def _compare(wl, nodes_to_check=None, **kw):
             assert np.array_equal(b["out"].cpu().numpy().reshape(keep[f"out{li}"].shape), keep[f"out{li}"]), f"out{li}"
     if ref["loss"] is not None:
         close(st.loss, ref["loss"], what="loss")
-    gscale = float(np.abs(ref["grads"]).max())
-    close(st.grads, ref["grads"], 1e-5, 1e-6 * max(1.0, gscale), "grads")
+    close(st.grads, ref["grads"], what="grads")
     close(st.x_half, ref["x_half"], what="x_half")
     close(st.x_hat, ref["x_hat"], what="x_hat")
     close(st.x_out, ref["x"], what="x")
@@ -147,8 +146,7 @@ def _compare_sampled_nodes(wl, sel):
             got = b["E"][sel].cpu().numpy()
             assert np.array_equal(got.reshape(keep[f"E{li}"].shape), keep[f"E{li}"]), f"E{li}"
     close(st.loss[sel], loss, what="loss")
-    gscale = float(np.abs(grads).max())
-    close(st.grads[sel], grads, 1e-5, 1e-6 * max(1.0, gscale), "grads")
+    close(st.grads[sel], grads, what="grads")
     import oracle
     close(st.x_half[sel], oracle.sgd_update(sub["params"], grads, wl["lr"]), what="x_half")
     # mix, from the GPU's own x_half (properties only)

@@ -17,10 +17,49 @@ def _rand(shape, seed):
     return torch.randint(-127, 128, shape, generator=g, device="cuda", dtype=torch.int8)
 
 
-@pytest.mark.parametrize("M,N,K", [(4096, 8192, 2048), (8192, 8192, 8192), (1024, 1024, 8192)])
-def test_large_gemm_three_passes(M, N, K):
+SIZES = (1024, 2048, 4096, 8192)
+GEMMS = [(M, N, K) for M in SIZES for N in SIZES for K in SIZES]      # all 64 shapes of the sweep
+N_SAMPLED = 64
+
+
+def _sampled(n, seed):
+    """64 distinct indices in [0, n): the first three, the last one, and random ones (first, middle
+    and last tiles are all hit)."""
+    r = np.random.default_rng(seed).permutation(n)[:N_SAMPLED]
+    r[:4] = [0, 1, 2, n - 1]
+    return np.unique(r)
+
+
+def _check_fp32_paths(desc, A, Wq, E, Y, dA, dW, ws, status):
+    """The calls as the benchmark makes them (fp32 results only, scales 1/127): each must equal the
+    dequantized int32 result of the raw-accumulator call element for element; the oracle's dequantize
+    is the reference on a sample of rows."""
+    sc = torch.full((1,), 1.0 / 127, device="cuda")
+    Yf = torch.empty(Y.shape, device="cuda"); dAf = torch.empty(dA.shape, device="cuda")
+    dWf = torch.empty(1, dW.numel(), device="cuda")
+    api.lpdt_qconv_fwd(desc, A, sc, Wq, sc, Y=Yf, ws=ws, dev_status=status)
+    api.lpdt_qconv_bwd_data(desc, E, sc, Wq, sc, dA=dAf, ws=ws, dev_status=status)
+    api.lpdt_qconv_bwd_weight(desc, E, sc, A, sc, dW=dWf, dw_node_stride=dWf.shape[1], ws=ws, dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    s_h = sc.cpu().numpy()
+    for f, i in ((Yf, Y), (dAf, dA), (dWf, dW)):
+        f2, i2 = f.reshape(-1, f.shape[-1]), i.reshape(-1, f.shape[-1])
+        rows = torch.from_numpy(_sampled(f2.shape[0], 5)).cuda()
+        want = oracle.dequant_acc(i2[rows].cpu().numpy()[None], s_h, s_h)[0]
+        assert np.array_equal(f2[rows].cpu().numpy(), want)
+        step = max(1, (1 << 26) // f2.shape[1])
+        for r in range(0, f2.shape[0], step):                     # whole tensor, in slabs
+            assert torch.equal(f2[r:r + step], i2[r:r + step].to(torch.float32) * (sc * sc))
+
+
+@pytest.mark.parametrize("M,N,K", GEMMS, ids=[f"M{m}N{n}K{k}" for m, n, k in GEMMS])
+def test_sweep_gemm_three_passes(M, N, K):
+    """Every GEMM shape of the sweep, forward / backward-data / backward-weight: the exact int64 checksum of
+    the whole result and 64 full-length rows (columns of the weight gradient) recomputed by the oracle."""
     desc = api.conv_desc(1, M, 1, 1, K, N, 1, 1, 1, 0)
-    A, Wq, E = _rand((1, M, 1, 1, K), 1), _rand((1, N, 1, 1, K), 2), _rand((1, M, 1, 1, N), 3)
+    seed = (M * 31 + N) * 31 + K
+    A, Wq, E = _rand((1, M, 1, 1, K), seed), _rand((1, N, 1, 1, K), seed + 1), _rand((1, M, 1, 1, N), seed + 2)
     ws = torch.empty(max(api.lpdt_qconv_workspace_size(desc, w) for w in (0, 1, 2)), dtype=torch.uint8, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     Y = torch.empty(1, M, 1, 1, N, dtype=torch.int32, device="cuda")
@@ -36,22 +75,29 @@ def test_large_gemm_three_passes(M, N, K):
     assert int(Y.sum(dtype=torch.int64)) == int((a64(A, 0) * a64(Wq, 0)).sum())
     assert int(dA.sum(dtype=torch.int64)) == int((a64(E, 0) * a64(Wq, 1)).sum())
     assert int(dW.sum(dtype=torch.int64)) == int((a64(E, 1) * a64(A, 1)).sum())
-    # sampled rows (spanning the first, a middle and the ragged last tile), recomputed by the oracle
-    rows = np.unique(np.concatenate([np.arange(3), np.random.default_rng(0).integers(0, M, 10), [M - 1]]))
-    Ah, Wh, Eh = A.cpu().numpy(), Wq.cpu().numpy(), E.cpu().numpy()
-    ref, _ = oracle.qconv_fwd(Ah[:, rows], Wh, 1, 0)
-    assert np.array_equal(Y.cpu().numpy()[:, rows], ref)
-    ref, _ = oracle.qconv_bwd_data(Eh[:, rows], Wh, 1, 1, 1, 0)
-    assert np.array_equal(dA.cpu().numpy()[:, rows], ref)
-    cols = np.unique(np.concatenate([np.arange(2), np.random.default_rng(1).integers(0, N, 6), [N - 1]]))
-    ref, _ = oracle.qconv_bwd_weight(np.ascontiguousarray(Eh[..., cols]), Ah, 1, 1, 1, 0)   # dW rows = output channels
-    assert np.array_equal(dW.cpu().numpy()[:, cols], ref)
+    rows = _sampled(M, seed)
+    rows_d = torch.from_numpy(rows).cuda()
+    Wh = Wq.cpu().numpy()
+    ref, ovf = oracle.qconv_fwd(A[:, rows_d].cpu().numpy(), Wh, 1, 0)
+    assert ovf == 0 and np.array_equal(Y[:, rows_d].cpu().numpy(), ref)
+    ref, ovf = oracle.qconv_bwd_data(E[:, rows_d].cpu().numpy(), Wh, 1, 1, 1, 0)
+    assert ovf == 0 and np.array_equal(dA[:, rows_d].cpu().numpy(), ref)
+    cols = _sampled(N, seed + 7)
+    cols_d = torch.from_numpy(cols).cuda()
+    ref, ovf = oracle.qconv_bwd_weight(E[..., cols_d].contiguous().cpu().numpy(), A.cpu().numpy(), 1, 1, 1, 0)
+    assert ovf == 0 and np.array_equal(dW[:, cols_d].cpu().numpy(), ref)     # dW rows = output channels
+    _check_fp32_paths(desc, A, Wq, E, Y, dA, dW, ws, status)
 
 
-@pytest.mark.parametrize("C,HW,batch", [(64, 56, 256), (256, 32, 256), (512, 32, 64)])
-def test_large_conv_three_passes(C, HW, batch):
+@pytest.mark.parametrize("C", [64, 256, 512])
+@pytest.mark.parametrize("HW", [32, 56])
+def test_sweep_conv_three_passes(C, HW):
+    """Every 3x3 convolution of the sweep at batch 256, three passes: three whole images recomputed by the
+    oracle (forward and backward-data), the exact adjoint identities over the whole batch, and a block of
+    weight-gradient entries recomputed over all 256 images."""
+    batch = 256
     desc = api.conv_desc(1, batch, HW, HW, C, C, 3, 3, 1, 1)
-    A, Wq, E = _rand((1, batch, HW, HW, C), 4), _rand((1, C, 3, 3, C), 5), _rand((1, batch, HW, HW, C), 6)
+    A, Wq, E = _rand((1, batch, HW, HW, C), 4 + C), _rand((1, C, 3, 3, C), 5 + C), _rand((1, batch, HW, HW, C), 6 + C)
     ws = torch.empty(max(api.lpdt_qconv_workspace_size(desc, w) for w in (0, 1, 2)), dtype=torch.uint8, device="cuda")
     status = torch.zeros(1, dtype=torch.int32, device="cuda")
     Y = torch.empty(1, batch, HW, HW, C, dtype=torch.int32, device="cuda")
@@ -65,18 +111,25 @@ def test_large_conv_three_passes(C, HW, batch):
     # sampled images, every pixel and channel of them
     imgs = [0, batch // 2 + 1, batch - 1]
     Ah, Wh, Eh = A[:, imgs].cpu().numpy(), Wq.cpu().numpy(), E[:, imgs].cpu().numpy()
-    ref, _ = oracle.qconv_fwd(Ah, Wh, 1, 1)
-    assert np.array_equal(Y[:, imgs].cpu().numpy(), ref)
-    ref, _ = oracle.qconv_bwd_data(Eh, Wh, HW, HW, 1, 1)
-    assert np.array_equal(dA[:, imgs].cpu().numpy(), ref)
+    ref, ovf = oracle.qconv_fwd(Ah, Wh, 1, 1)
+    assert ovf == 0 and np.array_equal(Y[:, imgs].cpu().numpy(), ref)
+    ref, ovf = oracle.qconv_bwd_data(Eh, Wh, HW, HW, 1, 1)
+    assert ovf == 0 and np.array_equal(dA[:, imgs].cpu().numpy(), ref)
     # adjoint identity over the whole batch: <fwd(A,W), E> = <W, bwd_weight(E,A)> = <A, bwd_data(E,W)> (int64)
-    lhs = int((Y.to(torch.int64) * E.to(torch.int64)).sum())
+    dot = lambda a, b: sum(int((a[:, i:i + 32].to(torch.int64) * b[:, i:i + 32].to(torch.int64)).sum())
+                           for i in range(0, a.shape[1], 32))
+    lhs = dot(Y, E)
     assert lhs == int((dW.to(torch.int64) * Wq.to(torch.int64)).sum())
-    assert lhs == int((dA.to(torch.int64) * A.to(torch.int64)).sum())
-    # a few weight-gradient entries recomputed over the full batch by the oracle (one output channel at a time)
-    co = [0, C - 1]
-    ref, _ = oracle.qconv_bwd_weight(np.ascontiguousarray(E[..., co].cpu().numpy()), A[..., :16].cpu().numpy().copy(), 3, 3, 1, 1)
-    assert np.array_equal(dW[:, co][..., :16].cpu().numpy(), ref)
+    assert lhs == dot(dA, A)
+    # weight-gradient entries recomputed over the full batch by the oracle: 8 output channels (first, last,
+    # one per 64-channel tile) x the first and the last 16 input channels x all 9 taps
+    co = sorted({0, C - 1, C // 2, C // 2 + 1, 17 % C, C - 18, (C // 4) * 3, 5})
+    for c0 in (0, C - 16):
+        ref, ovf = oracle.qconv_bwd_weight(np.ascontiguousarray(E[..., co].cpu().numpy()),
+                                           A[..., c0:c0 + 16].contiguous().cpu().numpy(), 3, 3, 1, 1)
+        assert ovf == 0 and np.array_equal(dW[:, co][..., c0:c0 + 16].cpu().numpy(), ref)
+    del Ah, Eh
+    _check_fp32_paths(desc, A, Wq, E, Y, dA, dW, ws, status)
 
 
 @pytest.mark.parametrize("shape", [("gemm", 4096, 4096, 4096), ("conv", 256, 32, 64)])
