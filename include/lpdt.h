@@ -62,6 +62,11 @@ typedef struct {
 
 const char *lpdt_version(void);
 const char *lpdt_status_string(lpdt_status s);
+/* Name of the contraction kernel that the most recent lpdt_qconv_* call of the calling host thread
+ * launched ("" before the first one): the tensor-core pixel-tile, halo-tile or weight-gradient kernel, or
+ * a CUDA-core kernel.  For labelling timings; the choice depends on the shape, the alignment and on which
+ * outputs were asked for. */
+const char *lpdt_last_kernel(void);
 /* Enqueue a zero fill of `bytes` bytes at device pointer p (range accumulators, status words). */
 lpdt_status lpdt_fill_zero(void *p, size_t bytes, void *stream);
 /* Read a status word back: waits until everything enqueued on `stream` so far has finished (the one

@@ -81,6 +81,10 @@ def lpdt_version():
     return lib().lpdt_version().decode()
 
 
+def lpdt_last_kernel():
+    return lib().lpdt_last_kernel().decode()
+
+
 def conv_desc(nodes, B, H, W, Cin, Cout, R=3, S=3, stride=1, pad=1):
     return ConvDesc(nodes, B, H, W, Cin, Cout, R, S, stride, pad)
 
@@ -357,10 +361,20 @@ def lpdt_colsum(nodes, B, Cc, x, out, out_node_stride):
     _check("lpdt_colsum", lib().lpdt_colsum(nodes, B, Cc, _ptr(x), _ptr(out), out_node_stride, _stream()))
 
 
+# Optional call log: while RECORD is a list, every entry-point call appends (name, function, args, kwargs,
+# contraction kernel launched or "").  The logged calls can be re-issued later on the same buffers, which is
+# how the benchmark times one kind of call of a whole step in isolation.
+RECORD = None
+
+
 def _with_timing(fn):
     name = fn.__name__
 
     def call(*a, **kw):
+        if RECORD is not None:
+            r = fn(*a, **kw)
+            RECORD.append((name, fn, a, kw, lpdt_last_kernel() if name.startswith("lpdt_qconv") else ""))
+            return r
         if name in TIMED:
             with timed(name):
                 return fn(*a, **kw)
@@ -371,6 +385,6 @@ def _with_timing(fn):
     return call
 
 
-for _n in [n for n in list(globals()) if n.startswith("lpdt_") and n in KERNELS_PER_CALL]:
+for _n in [n for n in list(globals()) if n.startswith("lpdt_") and (n in KERNELS_PER_CALL or n == "lpdt_fill_zero")]:
     globals()[_n] = _with_timing(globals()[_n])
 del _n

@@ -37,7 +37,7 @@ L2_BYTES = 126 * 1024 * 1024
 
 
 def time_case(nodes, B, H, W, Cin, Cout, R, S, stride, pad, iters=20, warmup=3, passes=("fwd", "bwd_data", "bwd_weight"),
-              label=None, graph=False):
+              label=None, graph=False, quiet=False):
     """graph=True records the `iters` calls into one CUDA graph and times its replay, which
     takes the host's launch cost out of calls that run for only a few microseconds; the calls
     rotate through `nsets` operand sets so that no call finds its operands in L2."""
@@ -101,7 +101,8 @@ def time_case(nodes, B, H, W, Cin, Cout, R, S, stride, pad, iters=20, warmup=3, 
                "ms": ms, "tops": 2 * macs / (ms * 1e-3) / 1e12, "macs": macs, "min_hbm_bytes": int(min_bytes),
                "gbs_at_min_bytes": min_bytes / (ms * 1e-3) / 1e9, "dev_status": int(status.item()),
                "timing": f"graph replay of {iters} calls over {nsets} operand sets" if graph else f"{iters} eager calls"}
-        print(json.dumps(rec), flush=True)
+        if not quiet:
+            print(json.dumps(rec), flush=True)
         out.append(rec)
     return out
 

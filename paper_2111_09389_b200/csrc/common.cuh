@@ -33,6 +33,10 @@ static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; 
 
 constexpr int kNumSMs = 148;  // B200
 
+// Name of the contraction kernel the calling host thread launched last (lpdt_last_kernel): lets a
+// caller that times a call label the number with the kernel that actually ran.
+inline thread_local const char *g_last_kernel = "";
+
 // A kernel attribute (the opt-in dynamic shared memory limit) belongs to the device it was set on, so
 // "already set" is remembered per device ordinal: one bit per device, devices beyond 63 set it every call.
 struct PerDeviceOnce {

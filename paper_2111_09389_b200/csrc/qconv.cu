@@ -369,7 +369,7 @@ extern "C" lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8
     lpdt_status s = check_desc(d);
     if (s != LPDT_OK) return s;
     if (d->nodes == 0) return LPDT_OK;
-    LPDT_CHECK_ARG(E && A && (dW || dWacc));
+    LPDT_CHECK_ARG((d->B == 0 || (E && A)) && (dW || dWacc));      // an empty batch has no operands to point at
     LPDT_CHECK_ARG(!dW || (sE && sA));
     LPDT_CHECK_ARG(!dW || dw_node_stride >= (int64_t)d->Cout * d->R * d->S * d->Cin || d->nodes == 1);
     if (!ws || ws_bytes < lpdt_qconv_workspace_size(d, 2) || !aligned(ws, 256)) return LPDT_ERR_WORKSPACE;

@@ -192,6 +192,7 @@ lpdt_status generic_fwd(const lpdt_conv_desc &d, const int8_t *A, const float *s
     const int Ho = conv_out(d.H, d.pad, d.R, d.stride), Wo = conv_out(d.W, d.pad, d.S, d.stride);
     const int64_t total = (int64_t)d.nodes * d.B * Ho * Wo * d.Cout;
     const bool vec4 = d.Cin % 4 == 0 && aligned(A, 4) && aligned(Wq, 4);
+    g_last_kernel = "lpdt::conv_fwd_generic";
     launch_k(conv_fwd_generic, grid_for(total), 256, 0, st, d, Ho, Wo, A, Wq, Yacc, Y, sA, sW, bias, bias_stride, vec4, uns);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
@@ -206,6 +207,7 @@ lpdt_status generic_bwd_data(const lpdt_conv_desc &d, const int8_t *E, const flo
     LPDT_LAUNCH_CHECK();
     const int64_t total = (int64_t)d.nodes * d.B * d.H * d.W * d.Cin;
     const bool vec4 = d.Cout % 4 == 0 && aligned(E, 4) && aligned(Wt, 4);
+    g_last_kernel = "lpdt::conv_bwd_data_generic";
     launch_k(conv_bwd_data_generic, grid_for(total), 256, 0, st, d, Ho, Wo, E, Wt, dAacc, dA, sE, sW, vec4, addend);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
@@ -223,6 +225,7 @@ lpdt_status generic_bwd_weight(const lpdt_conv_desc &d, const int8_t *E, const f
     if (npix > 0) {                      // an empty batch leaves the zeroed sums: the gradient of no samples
         int chunk = 4;
         while (ceil_div(npix, chunk) * d.nodes > (int64_t)kNumSMs * 16) chunk *= 2;
+        g_last_kernel = "lpdt::conv_bwd_weight_generic";
         launch_k(conv_bwd_weight_generic, dim3((unsigned)ceil_div(npix, chunk), d.nodes), 256, 0, st, d, Ho, Wo, chunk, E, A, acc);
         LPDT_LAUNCH_CHECK();
     }

@@ -438,6 +438,7 @@ lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, cons
     const long long tiles = (long long)p.nodes * p.B * p.tilesH * p.tilesW;
     if (tiles > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
     const int grid = (int)(tiles < (long long)kNumSMs * per_sm ? tiles : (long long)kNumSMs * per_sm);
+    g_last_kernel = "lpdt::tc::conv_halo16_kernel";
     launch_k(conv_halo16_kernel, grid, kHaloThreads, smem, st, mA, mW, mY, p);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;

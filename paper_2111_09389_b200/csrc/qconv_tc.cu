@@ -20,8 +20,11 @@
 // TMEM accumulator, so the epilogue of tile i overlaps the MMAs of tile i+1.
 // conv_wgrad_kernel: M = (tap, input channel), N = output channels, K = pixels,
 // split over CTAs with exact int32 atomics.  Warp roles: warp 0 issues TMA,
-// warp 1 owns TMEM and issues the MMAs, warps 2-5 run the epilogue (one TMEM
-// lane quarter each).  Every wait is bounded (tc_common.cuh).
+// warp 1 owns TMEM and issues the MMAs, the remaining warps run the epilogue
+// (conv_wgrad_kernel: warps 2-5, one TMEM lane quarter each; conv_pix_kernel:
+// warps 2-9, two per lane quarter taking alternate column chunks).  The pixel
+// kernel's fp32 result leaves through shared memory and bulk tensor stores where
+// its layout allows.  Every wait is bounded (tc_common.cuh).
 #include <stdlib.h>
 #include "qconv_internal.cuh"
 #include "tc_common.cuh"
@@ -30,6 +33,7 @@ namespace lpdt {
 namespace tc {
 
 constexpr int kThreads = 192;
+constexpr int kPixThreads = 320;      // pixel kernel: TMA warp, MMA warp, eight epilogue warps (two per TMEM lane quarter)
 constexpr int kMaxTaps = 64;
 
 // Row format of an operand tile: RB bytes per row and the UMMA layout code.
@@ -69,6 +73,10 @@ struct PixParams {
     const float *s1, *s2, *bias; long long bias_stride;
     const float *addend;      // nullable: fp32 tensor of the result's shape, added to the dequantized result
     int32_t *dev_status;
+    // fp32 result through shared memory and bulk tensor stores: every epilogue warp stages its 32 pixels x 32
+    // channels (128-byte rows, 128-byte swizzle) and stores them as one box {32 channels, bw, bh, bb pixels}
+    int tma_out, out_off;     // out_off: byte offset of the staging area in shared memory (1024-byte aligned)
+    int bw, bh;               // the warp's sub-box of the pixel tile: bw x bh x 32/(bw*bh) pixels
 };
 
 struct SharedCtl {
@@ -116,9 +124,9 @@ __device__ __forceinline__ TileCoord decode_raster(const PixParams &p, int tile)
     return c;
 }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kPixThreads, 1)
 conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapW,
-                const PixParams p) {
+                const __grid_constant__ CUtensorMap mapY, const PixParams p) {
     extern __shared__ __align__(1024) unsigned char smem[];
     SharedCtl *ctl = reinterpret_cast<SharedCtl *>(smem);
     unsigned char *data = smem + 1024;
@@ -136,7 +144,7 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.stages; ++i) { mbar_init(smem_u32(&ctl->full[i]), 1); mbar_init(smem_u32(&ctl->empty[i]), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&ctl->tmem_full[i]), 1); mbar_init(smem_u32(&ctl->tmem_empty[i]), 4); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&ctl->tmem_full[i]), 1); mbar_init(smem_u32(&ctl->tmem_empty[i]), 8); }
         ctl->abort_flag = 0;
         mbar_fence_init();
     }
@@ -254,6 +262,13 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
         uint32_t tcount = 0;
         TileCoord c = decode_tile(p, p.raster ? 0 : tile_lo);
         int sc_node = -1; float sc = 0.f;
+        // Two warps share a TMEM lane quarter and take alternate column chunks of its 32 pixels.
+        const int half = (warp - 2) >> 2;
+        // bulk-store path: this warp's 4 KB staging buffer and the origin of its 32 pixels inside the tile
+        unsigned char *buf = smem + p.out_off + (warp - 2) * 4096;
+        const int r0 = q * 32;
+        const int box_w0 = r0 % p.TW, box_h0 = (r0 / p.TW) % p.TH, box_b0 = r0 / (p.TW * p.TH);
+        if (p.tma_out && lane == 0) tma_prefetch_desc(&mapY);
         for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; tile += tile_step, ++tcount) {
             if (p.raster) c = decode_raster(p, tile); else if (tile != tile_lo) next_tile(p, c);
             const int n0 = c.nt * p.BN;
@@ -268,7 +283,60 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             tc_fence_after();
             const long long pix = (((long long)c.node * p.B + b) * p.Hout + h) * p.Wout + w;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * p.BN;
-            for (int cc = 0; cc < p.BN; cc += 16) {
+            if (p.tma_out) {
+                // 32 channels at a time: accumulators -> fp32 -> this warp's staging buffer (one 128-byte row per
+                // lane, 16-byte pieces XOR-swizzled by the row so that the lanes spread over all banks, which is
+                // also the layout the store's box expects) -> one bulk tensor store.  Box parts outside the
+                // image are not written.  The next chunk's accumulators are fetched while this one is converted,
+                // and the buffer is rewritten only after the previous store has read it.
+                const uint32_t sw = (uint32_t)(lane & 7);
+                uint32_t v[32];
+                int cc = half * 32;
+                bool have = cc < p.BN;
+                if (have) tmem_ld_32x32(t_row + cc, v);
+                while (have) {
+                    tmem_ld_wait();
+                    float f[32];
+#pragma unroll
+                    for (int k = 0; k < 32; ++k) f[k] = __fmul_rn(__int2float_rn((int)v[k]), sc);
+                    const int ncc = cc + 64;
+                    const bool more = ncc < p.BN;
+                    if (more) tmem_ld_32x32(t_row + ncc, v);
+                    if (p.bias) {
+#pragma unroll
+                        for (int k = 0; k < 32; ++k)
+                            f[k] = __fadd_rn(f[k], p.bias[(long long)c.node * p.bias_stride + n0 + cc + k]);
+                    }
+                    if (p.addend && valid) {
+                        const float4 *ad = reinterpret_cast<const float4 *>(p.addend + pix * p.Nc + n0 + cc);
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) {
+                            const float4 a4 = ad[k];
+                            f[4 * k] = __fadd_rn(f[4 * k], a4.x); f[4 * k + 1] = __fadd_rn(f[4 * k + 1], a4.y);
+                            f[4 * k + 2] = __fadd_rn(f[4 * k + 2], a4.z); f[4 * k + 3] = __fadd_rn(f[4 * k + 3], a4.w);
+                        }
+                    }
+                    if (lane == 0) tma_store_wait_read<0>();
+                    __syncwarp();
+                    float4 *grow = reinterpret_cast<float4 *>(buf + lane * 128);
+#pragma unroll
+                    for (int k = 0; k < 8; ++k)
+                        grow[(uint32_t)k ^ sw] = make_float4(f[4 * k], f[4 * k + 1], f[4 * k + 2], f[4 * k + 3]);
+                    fence_proxy_async_smem();
+                    __syncwarp();
+                    if (lane == 0) {
+                        tma_store_5d(&mapY, smem_u32(buf), n0 + cc, c.tw * p.TW + box_w0, c.th * p.TH + box_h0,
+                                     c.tb * p.TB + box_b0, c.node);
+                        tma_store_commit();
+                    }
+                    cc = ncc; have = more;
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
+                continue;
+            }
+            for (int cc = half * 16; cc < p.BN; cc += 32) {
                 uint32_t v[16];
                 tmem_ld_32x16(t_row + cc, v);
                 tmem_ld_wait();
@@ -306,6 +374,7 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
         }
+        if (p.tma_out && lane == 0) tma_store_wait_all();     // staged tiles read and written out before the CTA ends
     }
     tc_fence_before();
     __syncthreads();
@@ -544,6 +613,13 @@ bool tc_supported(const lpdt_conv_desc &d) {
     return true;
 }
 
+// LPDT_PIX_DIRECT_STORE=1 keeps the pixel kernel's per-lane global stores (A/B timing and parity tests).
+static bool pix_tma_out_enabled() {
+    static int off = -1;
+    if (off < 0) { const char *e = getenv("LPDT_PIX_DIRECT_STORE"); off = (e && e[0] == '1') ? 1 : 0; }
+    return off == 0;
+}
+
 static int largest_div(int C, int cap, int unit) {      // largest multiple of unit dividing C, <= cap
     for (int v = cap - cap % unit; v >= unit; v -= unit) if (C % v == 0) return v;
     return unit;
@@ -629,7 +705,14 @@ lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const flo
     // long K loops (GEMM-like): blocked round-robin tile order; short ones: contiguous ranges
     p.raster = (p.ncls == 1 && p.cls_iters[0] >= 8) ? 1 : 0;
     const int stage_bytes = U * unit_bytes;
-    p.stages = (kSmemBudget - 1024) / stage_bytes;
+    // fp32 result through shared memory and bulk tensor stores (not with raw accumulators, not for the strided
+    // pixel classes of a stride-2 backward-data pass): 8 warps x 4 KB of staging after the ring
+    p.tma_out = (Y && !Yacc && aligned(Y, 16) && p.ncls == 1 && p.out_mul == 1 && p.BN % 32 == 0 &&
+                 pix_tma_out_enabled()) ? 1 : 0;
+    p.bw = p.TW < 32 ? p.TW : 32;
+    p.bh = p.TH < 32 / p.bw ? p.TH : 32 / p.bw;
+    const int out_bytes = p.tma_out ? 32 * 1024 + 1024 : 0;        // 8 warps x 4 KB + slack to reach a 1024-byte boundary
+    p.stages = ((p.tma_out ? 227 * 1024 - out_bytes : kSmemBudget) - 1024) / stage_bytes;
     if (p.stages > 8) p.stages = 8;
     if (p.stages < 2) return LPDT_ERR_UNSUPPORTED;
     p.tmem_cols = pow2_at_least(2 * p.BN);
@@ -645,7 +728,19 @@ lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const flo
     if (mode == 0) { if (!weight_map(&mW, Wq, d.nodes, d.Cout, d.R * d.S, d.Cin, p.RBa, p.BN)) return LPDT_ERR_CUDA; }
     else if (!weight_map(&mW, Wq, d.nodes, d.Cout, d.R * d.S, d.Cin, p.RBn, p.RBa)) return LPDT_ERR_CUDA;
     size_t smem = 1024 + (size_t)p.stages * stage_bytes;
+    CUtensorMap mY = CUtensorMap{};
+    if (p.tma_out) {
+        p.out_off = (int)align_up(smem, 1024);
+        smem = (size_t)p.out_off + 32 * 1024;
+        uint64_t dims[5] = {(uint64_t)p.Nc, (uint64_t)p.Wout, (uint64_t)p.Hout, (uint64_t)d.B, (uint64_t)d.nodes};
+        uint64_t strides[4] = {(uint64_t)p.Nc * 4, (uint64_t)p.Wout * p.Nc * 4, (uint64_t)p.Hout * p.Wout * p.Nc * 4,
+                               (uint64_t)d.B * p.Hout * p.Wout * p.Nc * 4};
+        uint32_t box[5] = {32, (uint32_t)p.bw, (uint32_t)p.bh, (uint32_t)(32 / (p.bw * p.bh)), 1};
+        if (!make_map(&mY, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, Y, 5, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
+            return LPDT_ERR_CUDA;
+    }
     if (smem < kMinSmem) smem = kMinSmem;
+    if (smem > 227 * 1024) return LPDT_ERR_UNSUPPORTED;
     static PerDeviceOnce attr;
     int dev;
     if (attr.pending(&dev)) {
@@ -655,7 +750,8 @@ lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const flo
     const long long tiles = (long long)p.nodes * p.tilesB * p.tilesH * p.tilesW * p.tilesN * p.ncls;
     if (tiles > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
     const int grid = (int)(tiles < kNumSMs ? tiles : kNumSMs);
-    launch_k(conv_pix_kernel, grid, kThreads, smem, st, mA, mW, p);
+    g_last_kernel = "lpdt::tc::conv_pix_kernel";
+    launch_k(conv_pix_kernel, grid, kPixThreads, smem, st, mA, mW, mY, p);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }
@@ -748,6 +844,7 @@ lpdt_status tc_wgrad(const lpdt_conv_desc &d, int cin_real, const int8_t *E, con
         if (!p.acc_out) return LPDT_ERR_WORKSPACE;
         LPDT_CUDA(cudaMemsetAsync(p.acc_out, 0, (size_t)d.nodes * per_node * sizeof(int32_t), st));
     }
+    g_last_kernel = "lpdt::tc::conv_wgrad_kernel";
     launch_k(conv_wgrad_kernel, dim3(p.splits, p.mgroups * p.ngroups, d.nodes), kThreads, smem, st, mX, mE, p);
     LPDT_LAUNCH_CHECK();
     if (p.splits > 1 && dW) return dequant_acc_launch(p.acc_out, d.nodes, per_node, sE, sA, dW, dw_stride, st);

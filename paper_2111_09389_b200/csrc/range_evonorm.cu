@@ -210,8 +210,10 @@ ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
     if (R > 1) cg::this_cluster().barrier_wait();      // nobody still reads this CTA's shared memory
 }
 
-template <int V>
-__global__ void __launch_bounds__(512, 2)
+// MAXT = 256: three CTAs per SM at 80 registers (the thirteen double accumulators of a thread stay in
+// registers); MAXT = 512 serves the rare plans with more than 256 threads.
+template <int V, int MAXT>
+__global__ void __launch_bounds__(MAXT, MAXT == 256 ? 3 : 1)
 ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
                const float *__restrict__ dy, const float *__restrict__ x,
                const float *__restrict__ v, const float *__restrict__ gamma, int64_t pstride, int B,
@@ -484,10 +486,11 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t 
     double *acc = (double *)ws;
     const float Cst = ren_const(C / groups);
     dim3 grid((unsigned)((int64_t)nodes * B));
-    if (pl.V == 4)
-        launch_k(ren_bwd_kernel<4>, grid, pl.threads, smem, st, H * W, C, groups, eps, Cst, dy, x, v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc, amax_out);
-    else
-        launch_k(ren_bwd_kernel<1>, grid, pl.threads, smem, st, H * W, C, groups, eps, Cst, dy, x, v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc, amax_out);
+    using Fn = void (*)(int, int, int, float, float, const float *, const float *, const float *, const float *, int64_t, int,
+                        const float *, const float *, const int32_t *, const int32_t *, float *, double *, float *);
+    static const Fn fns[2][2] = {{ren_bwd_kernel<1, 256>, ren_bwd_kernel<1, 512>}, {ren_bwd_kernel<4, 256>, ren_bwd_kernel<4, 512>}};
+    launch_k(fns[pl.V == 4 ? 1 : 0][pl.threads > 256 ? 1 : 0], grid, pl.threads, smem, st, H * W, C, groups, eps, Cst, dy, x,
+             v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc, amax_out);
     LPDT_LAUNCH_CHECK();
     if (deferred) return LPDT_OK;
     launch_k(ren_bwd_finalize, (nodes * 3 * C + 7) / 8, 256, 0, st, acc, nodes, B, C, dv, dgamma, dbeta, gstride);

@@ -350,6 +350,17 @@ class TrainStep:
         self.backward()
         self.update()
 
+    def record(self):
+        """Run one step eagerly and return the log of its entry-point calls, in issue order:
+        [(name, function, args, kwargs, contraction kernel or "")].  The calls of a log can be issued
+        again on the buffers the step left behind (every call reads and writes the same tensors)."""
+        api.RECORD = log = []
+        try:
+            self.run()
+        finally:
+            api.RECORD = None
+        return log
+
     def contractions(self, passes=("fwd", "bwd_data")):
         """Re-issue only the integer contractions of every layer, in step order, on the operands the
         last run() left in the buffers (results are overwritten with the same values).  For timing

@@ -26,8 +26,7 @@ def _sampled(n, seed):
     """64 distinct indices in [0, n): the first three, the last one, and random ones (first, middle
     and last tiles are all hit)."""
     r = np.random.default_rng(seed).permutation(n)[:N_SAMPLED]
-    r[:4] = [0, 1, 2, n - 1]
-    return np.unique(r)
+    return np.unique(np.concatenate([r, np.array([0, 1, 2, n - 1]) % n]))
 
 
 def _check_fp32_paths(desc, A, Wq, E, Y, dA, dW, ws, status):
@@ -44,7 +43,7 @@ def _check_fp32_paths(desc, A, Wq, E, Y, dA, dW, ws, status):
     assert int(status.item()) == 0
     s_h = sc.cpu().numpy()
     for f, i in ((Yf, Y), (dAf, dA), (dWf, dW)):
-        f2, i2 = f.reshape(-1, f.shape[-1]), i.reshape(-1, f.shape[-1])
+        f2, i2 = f.reshape(-1, i.shape[-1]), i.reshape(-1, i.shape[-1])
         rows = torch.from_numpy(_sampled(f2.shape[0], 5)).cuda()
         want = oracle.dequant_acc(i2[rows].cpu().numpy()[None], s_h, s_h)[0]
         assert np.array_equal(f2[rows].cpu().numpy(), want)
