@@ -210,9 +210,23 @@ ren_fwd_kernel(int HW, int C, int groups, float eps, float Cst,
     if (R > 1) cg::this_cluster().barrier_wait();      // nobody still reads this CTA's shared memory
 }
 
+// Asynchronous 16-byte copy global -> shared (bypasses registers) and its group bookkeeping.
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gsrc) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() {
+    asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
+}
+
 // MAXT = 256: three CTAs per SM at 80 registers (the thirteen double accumulators of a thread stay in
 // registers); MAXT = 512 serves the rare plans with more than 256 threads.
-template <int V, int MAXT>
+// DEPTH > 0 (V = 4 only): every thread keeps its next DEPTH rows of x and dy in flight as asynchronous copies into
+// a private shared-memory ring, so the bytes in flight per SM (what a streaming kernel of 13-60 us lives
+// on) no longer depend on the register budget; the first DEPTH rows are requested before the group
+// statistics and parameters are read.  DEPTH = 0: rows are loaded into registers, two per trip.
+template <int V, int MAXT, int DEPTH>
 __global__ void __launch_bounds__(MAXT, MAXT == 256 ? 3 : 1)
 ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
                const float *__restrict__ dy, const float *__restrict__ x,
@@ -232,6 +246,8 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
     double *s_ch = reinterpret_cast<double *>(smem_raw);      // [nsets][3][C]
     double *s_S = s_ch + nsets * 3 * C;                       // [T]
     double *g_S = s_S + T;                                    // [groups]
+    // ring of DEPTH slots: slot s holds, for every thread, 16 bytes of x and 16 bytes of dy
+    float4 *ring = reinterpret_cast<float4 *>(smem_raw + (((size_t)(nsets * 3 * C + T + groups) * sizeof(double) + 15) & ~(size_t)15));
     const int CV = C / V, cpg = C / groups;
     const int col = t % CV, row0 = t / CV, rstep = T / CV;
     const int c0 = col * V, grp = c0 / cpg;
@@ -240,6 +256,22 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
     const float *xs = x + sample * (int64_t)HW * C;
     const float *dys = dy + sample * (int64_t)HW * C;
     float *dxs = dx + sample * (int64_t)HW * C;
+    const int iters = (HW - 1) / rstep + 1;          // same trip count for every thread (rows are predicated)
+    auto request = [&](int j) {                      // row j of this thread -> slot j % DEPTH; one group per row, even when empty
+        if (DEPTH > 0) {
+            const int p = row0 + j * rstep;
+            if (j < iters && p < HW) {
+                float4 *slot = ring + (size_t)(j % (DEPTH > 0 ? DEPTH : 1)) * 2 * T + t;
+                cp_async16(slot, xs + (int64_t)p * C + c0);
+                cp_async16(slot + T, dys + (int64_t)p * C + c0);
+            }
+            cp_async_commit();
+        }
+    };
+    if (DEPTH > 0) {
+#pragma unroll
+        for (int j = 0; j < (DEPTH > 0 ? DEPTH : 1); ++j) request(j);
+    }
     for (int i = t; i < nsets * 3 * C; i += T) s_ch[i] = 0.0;
 
     const int64_t sg = sample * groups + grp;
@@ -265,7 +297,6 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
 #pragma unroll
     for (int k = 0; k < V; ++k) { fb[k] = 0.0; fg[k] = 0.0; fv[k] = 0.0; }
     __syncthreads();   // s_ch zeroed
-    const int iters = (HW - 1) / rstep + 1;          // same trip count for every thread (rows are predicated)
     auto term = [&](int p, const float (&xv)[V], const float (&dv_)[V]) {
         float o[V];
 #pragma unroll
@@ -285,8 +316,22 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
         }
         VecLoad<V>::st(dxs + (int64_t)p * C + c0, o);
     };
-    // two rows per trip: four independent 16-byte loads in flight per thread
-    for (int i = 0; i < iters; i += 2) {
+    if (DEPTH > 0) {
+        for (int j = 0; j < iters; ++j) {
+            cp_async_wait<(DEPTH > 0 ? DEPTH - 1 : 0)>();                // the oldest pending group, row j, has landed
+            const int p = row0 + j * rstep;
+            if (p < HW) {
+                const float4 *slot = ring + (size_t)(j % (DEPTH > 0 ? DEPTH : 1)) * 2 * T + t;
+                const float4 a = slot[0], b = slot[T];
+                const float xa[4] = {a.x, a.y, a.z, a.w}, da[4] = {b.x, b.y, b.z, b.w};
+                term(p, reinterpret_cast<const float (&)[V]>(xa), reinterpret_cast<const float (&)[V]>(da));
+            }
+            request(j + DEPTH);                                  // the slot just read takes row j + DEPTH
+        }
+        cp_async_wait<0>();
+    }
+    // DEPTH = 0, two rows per trip: four independent 16-byte loads in flight per thread
+    for (int i = 0; DEPTH == 0 && i < iters; i += 2) {
         const int p0 = row0 + i * rstep, p1 = p0 + rstep;
         const bool ok0 = p0 < HW, ok1 = (i + 1 < iters) && (p1 < HW);
         float xa[V], da[V], xb[V], db[V];
@@ -376,13 +421,13 @@ __global__ void ren_bwd_finalize(const double *__restrict__ acc, int nodes, int 
 
 struct RenPlan { int V, threads; };
 
-static bool plan(int C, int groups, bool aligned16, RenPlan *pl) {
+static bool plan(int C, int groups, bool aligned16, RenPlan *pl, int cap = 256) {
     const int cpg = C / groups;
     int V = (aligned16 && C % 4 == 0 && cpg % 4 == 0) ? 4 : 1;
     int CV = C / V;
     if (CV > 512) return false;
     pl->V = V;
-    pl->threads = CV <= 256 ? CV * (256 / CV) : CV;
+    pl->threads = CV <= cap ? CV * (cap / CV) : (CV <= 256 ? CV * (256 / CV) : CV);
     if (pl->threads % 32) {                      // keep whole warps: pad down to a multiple of lcm
         int th = pl->threads;
         while (th > 0 && (th % 32 || th % CV)) th -= CV;
@@ -434,7 +479,10 @@ extern "C" lpdt_status lpdt_range_evonorm_fwd(int32_t nodes, int32_t B, int32_t 
     LPDT_CHECK_ARG(pstride >= C || nodes == 1);
     if ((int64_t)H * W * C > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
     RenPlan pl;
-    if (!plan(C, groups, aligned(x, 16) && aligned(y, 16) && (!res || aligned(res, 16)), &pl)) return LPDT_ERR_UNSUPPORTED;
+    static int tforce = -1;
+    if (tforce < 0) { const char *e = getenv("LPDT_REN_FWD_THREADS"); tforce = e ? atoi(e) : 0; }
+    if (!plan(C, groups, aligned(x, 16) && aligned(y, 16) && (!res || aligned(res, 16)), &pl, tforce == 128 ? 128 : 256))
+        return LPDT_ERR_UNSUPPORTED;
     size_t smem = (size_t)(2 * pl.threads + 4 * groups) * sizeof(Ext);
     if (smem > 48 * 1024) return LPDT_ERR_UNSUPPORTED;
     const float Cst = ren_const(C / groups);
@@ -477,18 +525,38 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t 
     if (!ws || ws_bytes < lpdt_range_evonorm_bwd_workspace_size(nodes, B, C) || !aligned(ws, 8))
         return LPDT_ERR_WORKSPACE;
     RenPlan pl;
-    if (!plan(C, groups, aligned(x, 16) && aligned(dy, 16) && aligned(dx, 16), &pl)) return LPDT_ERR_UNSUPPORTED;
+    // Samples of up to 64 KB with few channel columns run as 128-thread CTAs, six per SM instead of three: the
+    // serial head and tail of such a short CTA (statistics, reductions, the patch at the extrema) then overlap
+    // with the streaming phase of more neighbours (measured: 16x16x32 samples 0.041 -> 0.033 ms, 32x32x16
+    // 0.058 -> 0.053 ms; 256 KB samples lose 5 %).  LPDT_REN_BWD_THREADS=128|256 overrides (A/B timing).
+    static int tforce = -1;
+    if (tforce < 0) { const char *e = getenv("LPDT_REN_BWD_THREADS"); tforce = e ? atoi(e) : 0; }
+    const bool v4 = aligned(x, 16) && aligned(dy, 16) && aligned(dx, 16) && C % 4 == 0 && (C / groups) % 4 == 0;
+    int cap = ((int64_t)H * W * C * 4 <= 64 * 1024 && C / (v4 ? 4 : 1) <= 32) ? 128 : 256;
+    if (tforce == 128 || tforce == 256) cap = tforce;
+    if (!plan(C, groups, aligned(x, 16) && aligned(dy, 16) && aligned(dx, 16), &pl, cap)) return LPDT_ERR_UNSUPPORTED;
     const int cv = C / pl.V;
     const int nsets = (cv <= 32 && 32 % cv == 0) ? pl.threads / 32 : 1;      // as in the kernel
     size_t smem = (size_t)(nsets * 3 * C + pl.threads + groups) * sizeof(double);
     if (smem > 48 * 1024) return LPDT_ERR_UNSUPPORTED;
+    // rows in flight per thread (V = 4): 8 with up to 256 threads (64 KB of ring, three CTAs per SM), 4 beyond
+    const int depth = pl.V == 4 ? (pl.threads <= 256 ? 8 : 4) : 0;
+    smem = align_up(smem, 16) + (size_t)depth * 2 * pl.threads * 16;
     cudaStream_t st = as_stream(stream);
     double *acc = (double *)ws;
     const float Cst = ren_const(C / groups);
     dim3 grid((unsigned)((int64_t)nodes * B));
     using Fn = void (*)(int, int, int, float, float, const float *, const float *, const float *, const float *, int64_t, int,
                         const float *, const float *, const int32_t *, const int32_t *, float *, double *, float *);
-    static const Fn fns[2][2] = {{ren_bwd_kernel<1, 256>, ren_bwd_kernel<1, 512>}, {ren_bwd_kernel<4, 256>, ren_bwd_kernel<4, 512>}};
+    static const Fn fns[2][2] = {{ren_bwd_kernel<1, 256, 0>, ren_bwd_kernel<1, 512, 0>},
+                                 {ren_bwd_kernel<4, 256, 8>, ren_bwd_kernel<4, 512, 4>}};
+    static PerDeviceOnce attr;
+    int dev;
+    if (attr.pending(&dev)) {
+        for (int i = 0; i < 2; ++i)
+            LPDT_CUDA(cudaFuncSetAttribute(fns[1][i], cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
+        attr.mark(dev);
+    }
     launch_k(fns[pl.V == 4 ? 1 : 0][pl.threads > 256 ? 1 : 0], grid, pl.threads, smem, st, H * W, C, groups, eps, Cst, dy, x,
              v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc, amax_out);
     LPDT_LAUNCH_CHECK();
