@@ -150,6 +150,40 @@ def qconv_bwd_weight(E, A, R, S, stride=1, pad=1):
     return dW, ovf.value
 
 
+def qconv_bwd_data_affine(E, zE, Wq, zW, H, W, stride=1, pad=1):
+    """E uint8 [n,B,Ho,Wo,Cout], Wq uint8 [n,Cout,R,S,Cin], zero points int32 [n] ->
+    (dA int32 [n,B,H,W,Cin] of (qe - zE)(qw - zW) over the taps that exist, overflow)."""
+    E = _c(E, np.uint8)
+    Wq = _c(Wq, np.uint8)
+    zE = _c(zE, np.int32)
+    zW = _c(zW, np.int32)
+    n, B, Ho, Wo, Cout = E.shape
+    _, _, R, S, Cin = Wq.shape
+    assert (Ho, Wo) == _out_hw(H, W, R, S, stride, pad) and zE.shape == (n,) and zW.shape == (n,)
+    dA = np.zeros((n, B, H, W, Cin), np.int32)
+    ovf = _i64(0)
+    lib().orc_qconv_bwd_data_affine(n, B, H, W, Cin, Cout, R, S, stride, pad, _p(E), _p(zE), _p(Wq), _p(zW),
+                                    _p(dA), C.byref(ovf))
+    return dA, ovf.value
+
+
+def qconv_bwd_weight_affine(E, zE, A, zA, R, S, stride=1, pad=1):
+    """E uint8 [n,B,Ho,Wo,Cout], A uint8 [n,B,H,W,Cin], zero points int32 [n] ->
+    (dW int32 [n,Cout,R,S,Cin] of (qe - zE)(qa - zA) over the taps inside the image, overflow)."""
+    E = _c(E, np.uint8)
+    A = _c(A, np.uint8)
+    zE = _c(zE, np.int32)
+    zA = _c(zA, np.int32)
+    n, B, Ho, Wo, Cout = E.shape
+    _, _, H, W, Cin = A.shape
+    assert (Ho, Wo) == _out_hw(H, W, R, S, stride, pad) and zE.shape == (n,) and zA.shape == (n,)
+    dW = np.zeros((n, Cout, R, S, Cin), np.int32)
+    ovf = _i64(0)
+    lib().orc_qconv_bwd_weight_affine(n, B, H, W, Cin, Cout, R, S, stride, pad, _p(E), _p(zE), _p(A), _p(zA),
+                                      _p(dW), C.byref(ovf))
+    return dW, ovf.value
+
+
 def dequant_acc(acc, s1, s2, bias=None):
     """y = float(acc) * (s1*s2) (+ bias over the last axis); per-node scales."""
     acc = _c(acc, np.int32)

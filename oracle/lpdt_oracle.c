@@ -331,6 +331,77 @@ void orc_qconv_bwd_weight(int nodes, int B, int H, int W, int Cin, int Cout, int
     }
 }
 
+/* Backward products on affine (zero-point) 8-bit operands (Section 3 names the scheme; the layer
+ * gradient, the weights and the saved activations are unsigned codes with one zero point per node and
+ * tensor: real = scale*(code - zero point)).  They are the adjoints of orc_qconv_fwd_affine: a tap that
+ * lies outside the image pairs nothing with nothing, so it is simply absent from the sums.
+ *   dA[n,b,ih,iw,ci] = sum over (oh,ow,r,s,co) with ih = oh*stride + r - pad, iw = ow*stride + s - pad
+ *                      of (E[n,b,oh,ow,co] - zE[n]) * (W[n,co,r,s,ci] - zW[n]) */
+void orc_qconv_bwd_data_affine(int nodes, int B, int H, int W, int Cin, int Cout, int R, int S,
+                               int stride, int pad, const uint8_t *E, const int32_t *zE,
+                               const uint8_t *Wq, const int32_t *zW, int32_t *dA, i64 *overflow)
+{
+    const int Ho = (H + 2 * pad - R) / stride + 1;
+    const int Wo = (W + 2 * pad - S) / stride + 1;
+    *overflow = 0;
+    #pragma omp parallel for collapse(3) schedule(static)
+    for (int n = 0; n < nodes; ++n)
+    for (int b = 0; b < B; ++b)
+    for (int ih = 0; ih < H; ++ih)
+    for (int iw = 0; iw < W; ++iw)
+    for (int ci = 0; ci < Cin; ++ci) {
+        i64 sum = 0;
+        for (int r = 0; r < R; ++r) {
+            int th = ih + pad - r;
+            if (th < 0 || th % stride != 0) continue;
+            int oh = th / stride;
+            if (oh >= Ho) continue;
+            for (int s = 0; s < S; ++s) {
+                int tw = iw + pad - s;
+                if (tw < 0 || tw % stride != 0) continue;
+                int ow = tw / stride;
+                if (ow >= Wo) continue;
+                const uint8_t *e = E + ((((i64)n * B + b) * Ho + oh) * Wo + ow) * Cout;
+                for (int co = 0; co < Cout; ++co)
+                    sum += ((int32_t)e[co] - zE[n]) *
+                           ((int32_t)Wq[((((i64)n * Cout + co) * R + r) * S + s) * Cin + ci] - zW[n]);
+            }
+        }
+        dA[((((i64)n * B + b) * H + ih) * W + iw) * Cin + ci] = wrap32(sum, overflow);
+    }
+}
+
+/*   dW[n,co,r,s,ci] = sum over (b,oh,ow) whose tap (r,s) lies inside the image of
+ *                     (E[n,b,oh,ow,co] - zE[n]) * (A[n,b,oh*stride+r-pad,ow*stride+s-pad,ci] - zA[n]) */
+void orc_qconv_bwd_weight_affine(int nodes, int B, int H, int W, int Cin, int Cout, int R, int S,
+                                 int stride, int pad, const uint8_t *E, const int32_t *zE,
+                                 const uint8_t *A, const int32_t *zA, int32_t *dW, i64 *overflow)
+{
+    const int Ho = (H + 2 * pad - R) / stride + 1;
+    const int Wo = (W + 2 * pad - S) / stride + 1;
+    *overflow = 0;
+    #pragma omp parallel for collapse(2) schedule(static)
+    for (int n = 0; n < nodes; ++n)
+    for (int co = 0; co < Cout; ++co)
+    for (int r = 0; r < R; ++r)
+    for (int s = 0; s < S; ++s)
+    for (int ci = 0; ci < Cin; ++ci) {
+        i64 sum = 0;
+        for (int b = 0; b < B; ++b)
+        for (int oh = 0; oh < Ho; ++oh) {
+            int ih = oh * stride + r - pad;
+            if (ih < 0 || ih >= H) continue;
+            for (int ow = 0; ow < Wo; ++ow) {
+                int iw = ow * stride + s - pad;
+                if (iw < 0 || iw >= W) continue;
+                sum += ((int32_t)E[((((i64)n * B + b) * Ho + oh) * Wo + ow) * Cout + co] - zE[n]) *
+                       ((int32_t)A[((((i64)n * B + b) * H + ih) * W + iw) * Cin + ci] - zA[n]);
+            }
+        }
+        dW[((((i64)n * Cout + co) * R + r) * S + s) * Cin + ci] = wrap32(sum, overflow);
+    }
+}
+
 /* Dequantize accumulators: sc = s1[n]*s2[n] (one fp32 multiply),
  * y = (float)acc * sc, then + bias[n][i mod C] when bias != NULL. */
 void orc_dequant_acc(const int32_t *acc, int nodes, i64 n_per_node, int C,

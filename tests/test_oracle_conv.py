@@ -234,3 +234,84 @@ def test_affine_expansion_identity():
     ref = raw.astype(np.int64) - zW_ * ra - zA_ * rw + cnt * zA_ * zW_
     assert np.array_equal(acc.astype(np.int64), ref)
     assert cnt[0, 0, 0, 0, 0] == 4 * 2 and cnt[0, 0, 2, 2, 0] == 9 * 2         # corner and interior term counts
+
+
+# ---- affine backward products: pinned to the (already pinned) affine forward product and to its meaning ----
+@pytest.mark.parametrize("stride,pad,R", [(1, 1, 3), (2, 1, 3), (1, 0, 1), (1, 2, 5), (2, 0, 2)])
+def test_affine_backward_products_are_the_adjoints_of_the_forward_product(stride, pad, R):
+    # <fwd(A, W), E'> = <A', bwd_data(E, W)> = <W', bwd_weight(E, A)> exactly in int64, primes = code - zero point:
+    # a dropped tap, a wrong border rule or a transposed index in either backward product breaks one of the two
+    A, zA, Wq, zW = _affine_case(11 + R, H=7, W=6, R=R, S=R)
+    n, B, H, W, Cin = A.shape
+    fwd, ovf = oracle.qconv_fwd_affine(A, zA, Wq, zW, stride=stride, pad=pad)
+    assert ovf == 0
+    rng = np.random.default_rng(stride * 10 + R)
+    E = rng.integers(0, 256, fwd.shape, dtype=np.uint8)
+    zE = rng.integers(0, 256, n).astype(np.int32)
+    dA, o1 = oracle.qconv_bwd_data_affine(E, zE, Wq, zW, H, W, stride=stride, pad=pad)
+    dW, o2 = oracle.qconv_bwd_weight_affine(E, zE, A, zA, R, R, stride=stride, pad=pad)
+    assert o1 == 0 and o2 == 0
+    c = lambda q, z: q.astype(np.int64) - z.reshape((-1,) + (1,) * (q.ndim - 1))
+    for i in range(n):
+        lhs = int((fwd[i].astype(np.int64) * c(E, zE)[i]).sum())
+        assert lhs == int((c(A, zA)[i] * dA[i]).sum())
+        assert lhs == int((c(Wq, zW)[i] * dW[i]).sum())
+
+
+@pytest.mark.parametrize("stride,pad", [(1, 1), (2, 1)])
+def test_affine_backward_products_equal_real_domain_gradients(stride, pad):
+    # the real-valued layer y = conv(a, w) with zero padding: dL/da and dL/dw for upstream gradient e, computed
+    # in float64 by probing the bilinear form with numpy (a library routine on the meaning of the codes)
+    A, zA, Wq, zW = _affine_case(21, n=1, B=2, H=5, W=4, Cin=2, Cout=3)
+    n, B, H, W, Cin = A.shape
+    Cout, R = Wq.shape[1], Wq.shape[2]
+    rng = np.random.default_rng(5)
+    Ho, Wo = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - R) // stride + 1
+    E = rng.integers(0, 256, (n, B, Ho, Wo, Cout), dtype=np.uint8)
+    zE = np.array([97], np.int32)
+    a = A[0].astype(np.float64) - zA[0]
+    w = Wq[0].astype(np.float64) - zW[0]
+    e = E[0].astype(np.float64) - zE[0]
+
+    def fwd_real(a_, w_):
+        ap = np.pad(a_, ((0, 0), (pad, pad), (pad, pad), (0, 0)))
+        win = np.lib.stride_tricks.sliding_window_view(ap, (R, R), axis=(1, 2))[:, ::stride, ::stride]
+        return np.einsum("bhwcrs,orsc->bhwo", win[:, :Ho, :Wo], w_)
+    # gradients of <fwd_real(a, w), e> by unit probes (the form is linear in a and in w)
+    da = np.zeros_like(a); dw = np.zeros_like(w)
+    for idx in np.ndindex(a.shape):
+        u = np.zeros_like(a); u[idx] = 1.0
+        da[idx] = (fwd_real(u, w) * e).sum()
+    for idx in np.ndindex(w.shape):
+        u = np.zeros_like(w); u[idx] = 1.0
+        dw[idx] = (fwd_real(a, u) * e).sum()
+    dA, _ = oracle.qconv_bwd_data_affine(E, zE, Wq, zW, H, W, stride=stride, pad=pad)
+    dW, _ = oracle.qconv_bwd_weight_affine(E, zE, A, zA, R, R, stride=stride, pad=pad)
+    assert np.array_equal(dA[0].astype(np.float64), da)
+    assert np.array_equal(dW[0].astype(np.float64), dw)
+
+
+def test_affine_backward_with_zero_zero_points_is_the_plain_product():
+    rng = np.random.default_rng(31)
+    E = rng.integers(0, 128, (2, 2, 6, 5, 3), dtype=np.uint8)
+    Wq = rng.integers(0, 128, (2, 3, 3, 3, 4), dtype=np.uint8)
+    A = rng.integers(0, 128, (2, 2, 6, 5, 4), dtype=np.uint8)
+    z = np.zeros(2, np.int32)
+    dA, _ = oracle.qconv_bwd_data_affine(E, z, Wq, z, 6, 5, stride=1, pad=1)
+    ref, _ = oracle.qconv_bwd_data(E.astype(np.int8), Wq.astype(np.int8), 6, 5, stride=1, pad=1)
+    assert np.array_equal(dA, ref)
+    dW, _ = oracle.qconv_bwd_weight_affine(E, z, A, z, 3, 3, stride=1, pad=1)
+    ref, _ = oracle.qconv_bwd_weight(E.astype(np.int8), A.astype(np.int8), 3, 3, stride=1, pad=1)
+    assert np.array_equal(dW, ref)
+
+
+def test_affine_backward_of_a_real_zero_gradient_is_zero():
+    A, zA, Wq, zW = _affine_case(41)
+    n = A.shape[0]
+    zE = np.array([200, 3], np.int32)
+    E = np.empty((n, 2, 5, 6, 4), np.uint8)
+    for i in range(n):
+        E[i] = zE[i]
+    dA, _ = oracle.qconv_bwd_data_affine(E, zE, Wq, zW, 5, 6, stride=1, pad=1)
+    dW, _ = oracle.qconv_bwd_weight_affine(E, zE, A, zA, 3, 3, stride=1, pad=1)
+    assert not dA.any() and not dW.any()
