@@ -229,9 +229,19 @@ lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8_t *E, cons
  * ws      : lpdt_qconv_fwd_affine_workspace_size(desc) bytes, 256-byte aligned
  * The integer contraction of the codes runs on the same kernels as
  * lpdt_qconv_fwd (unsigned operand format); the zero-point terms are applied
- * by a correction pass over the int32 sums.  Only the forward product is
- * provided in this form.
+ * by a correction pass over the int32 sums.
  * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA; TIMEOUT through dev_status.
+ *
+ * The two backward products in the same form (the adjoints of the forward product: a tap
+ * outside the image is absent from the sums), with E the layer gradient as unsigned codes
+ * with zero point zE and scale sE:
+ *   dA[n,b,ih,iw,ci] = sum_{(oh,ow,r,s) with ih = oh*st+r-p, iw = ow*st+s-p; co}
+ *                      (E[n,b,oh,ow,co] - zE[n]) * (W[n,co,r,s,ci] - zW[n])
+ *   dW[n,co,r,s,ci]  = sum_{(b,oh,ow) with the tap (r,s) inside the image}
+ *                      (E[n,b,oh,ow,co] - zE[n]) * (A[n,b,oh*st+r-p,ow*st+s-p,ci] - zA[n])
+ *   fp32 results: (float)sum * (sE[n]*sW[n]) and (float)sum * (sE[n]*sA[n]).
+ * Layouts, nullable outputs and dw_node_stride as in lpdt_qconv_bwd_data / _bwd_weight;
+ * ws: the matching *_affine_workspace_size(desc) bytes, 256-byte aligned.
  */
 size_t lpdt_qconv_fwd_affine_workspace_size(const lpdt_conv_desc *d);
 lpdt_status lpdt_qconv_fwd_affine(const lpdt_conv_desc *d, const uint8_t *A, const float *sA, const int32_t *zA,
@@ -239,6 +249,16 @@ lpdt_status lpdt_qconv_fwd_affine(const lpdt_conv_desc *d, const uint8_t *A, con
                                   const float *bias, int64_t bias_node_stride,
                                   float *Y, int32_t *Yacc,
                                   void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
+size_t lpdt_qconv_bwd_data_affine_workspace_size(const lpdt_conv_desc *d);
+lpdt_status lpdt_qconv_bwd_data_affine(const lpdt_conv_desc *d, const uint8_t *E, const float *sE, const int32_t *zE,
+                                       const uint8_t *Wq, const float *sW, const int32_t *zW,
+                                       float *dA, int32_t *dAacc,
+                                       void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
+size_t lpdt_qconv_bwd_weight_affine_workspace_size(const lpdt_conv_desc *d);
+lpdt_status lpdt_qconv_bwd_weight_affine(const lpdt_conv_desc *d, const uint8_t *E, const float *sE, const int32_t *zE,
+                                         const uint8_t *A, const float *sA, const int32_t *zA,
+                                         float *dW, int64_t dw_node_stride, int32_t *dWacc,
+                                         void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
 
 /* ---------------------------------------------------------------------------
  * Range-EvoNorm (Eq. "ren"), forward and backward.

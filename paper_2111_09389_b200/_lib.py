@@ -38,6 +38,11 @@ SIGNATURES = {
     "lpdt_qconv_fwd_affine_workspace_size": (_sz, [C.POINTER(ConvDesc)]),
     "lpdt_qconv_fwd_affine": (_i32, [C.POINTER(ConvDesc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _vp, _vp, _sz,
                                      _vp, _vp]),
+    "lpdt_qconv_bwd_data_affine_workspace_size": (_sz, [C.POINTER(ConvDesc)]),
+    "lpdt_qconv_bwd_data_affine": (_i32, [C.POINTER(ConvDesc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
+    "lpdt_qconv_bwd_weight_affine_workspace_size": (_sz, [C.POINTER(ConvDesc)]),
+    "lpdt_qconv_bwd_weight_affine": (_i32, [C.POINTER(ConvDesc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp, _vp, _sz,
+                                            _vp, _vp]),
     "lpdt_qconv_bwd_data": (_i32, [C.POINTER(ConvDesc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
     "lpdt_qconv_bwd_weight": (_i32, [C.POINTER(ConvDesc), _vp, _vp, _vp, _vp, _vp, _i64, _vp, _vp, _sz, _vp, _vp]),
     "lpdt_range_evonorm_fwd": (_i32, [_i32] * 6 + [_f32] + [_vp] * 4 + [_i64] + [_vp] * 7 + [_vp]),

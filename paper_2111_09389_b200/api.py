@@ -13,7 +13,7 @@ from ._lib import ConvDesc, lib
 
 # Kernels each entry point enqueues (memsets not counted); KERNEL_LAUNCHES accumulates them.
 KERNELS_PER_CALL = {
-    "lpdt_quantize": 2, "lpdt_quantize_with_range": 1, "lpdt_quantize_static": 2, "lpdt_quantize_batch": 2, "lpdt_dequantize": 1, "lpdt_qconv_fwd": 1, "lpdt_qconv_fwd_affine": 4, "lpdt_qconv_bwd_data": 2,
+    "lpdt_quantize": 2, "lpdt_quantize_with_range": 1, "lpdt_quantize_static": 2, "lpdt_quantize_batch": 2, "lpdt_dequantize": 1, "lpdt_qconv_fwd": 1, "lpdt_qconv_fwd_affine": 4, "lpdt_qconv_bwd_data_affine": 4, "lpdt_qconv_bwd_weight_affine": 7, "lpdt_qconv_bwd_data": 2,
     "lpdt_qconv_bwd_weight": 2, "lpdt_range_evonorm_fwd": 1, "lpdt_range_evonorm_bwd": 2, "lpdt_range_evonorm_bwd_params": 1,
     "lpdt_gossip_mix": 2, "lpdt_gossip_mix_q8": 3, "lpdt_deepsqueeze_mix": 2, "lpdt_pushsum_debias": 1, "lpdt_sgd_gossip_mix": 1, "lpdt_evonorm_s0_fwd": 1, "lpdt_evonorm_s0_bwd": 2, "lpdt_range_bn_fwd": 2, "lpdt_range_bn_bwd": 2, "lpdt_sgd_update": 1, "lpdt_residual_add": 1, "lpdt_residual_add_bwd": 1,
     "lpdt_avgpool": 1, "lpdt_avgpool_bwd": 1, "lpdt_maxpool2x2": 1, "lpdt_maxpool2x2_bwd": 1,
@@ -183,6 +183,31 @@ def lpdt_qconv_fwd_affine(desc, A, sA, zA, Wq, sW, zW, Y=None, Yacc=None, bias=N
     _check("lpdt_qconv_fwd_affine", lib().lpdt_qconv_fwd_affine(
         C.byref(desc), _ptr(A), _ptr(sA), _ptr(zA), _ptr(Wq), _ptr(sW), _ptr(zW), _ptr(bias), bias_node_stride,
         _ptr(Y), _ptr(Yacc), p, nb, _ptr(dev_status), _stream()))
+
+
+def lpdt_qconv_bwd_data_affine_workspace_size(desc):
+    return lib().lpdt_qconv_bwd_data_affine_workspace_size(C.byref(desc))
+
+
+def lpdt_qconv_bwd_data_affine(desc, E, sE, zE, Wq, sW, zW, dA=None, dAacc=None, ws=None, dev_status=None):
+    """Backward-data contraction on unsigned codes with per-node zero points (E, Wq uint8; zE, zW int32)."""
+    p, nb = _ws(ws)
+    _check("lpdt_qconv_bwd_data_affine", lib().lpdt_qconv_bwd_data_affine(
+        C.byref(desc), _ptr(E), _ptr(sE), _ptr(zE), _ptr(Wq), _ptr(sW), _ptr(zW), _ptr(dA), _ptr(dAacc), p, nb,
+        _ptr(dev_status), _stream()))
+
+
+def lpdt_qconv_bwd_weight_affine_workspace_size(desc):
+    return lib().lpdt_qconv_bwd_weight_affine_workspace_size(C.byref(desc))
+
+
+def lpdt_qconv_bwd_weight_affine(desc, E, sE, zE, A, sA, zA, dW=None, dw_node_stride=0, dWacc=None, ws=None,
+                                 dev_status=None):
+    """Backward-weight contraction on unsigned codes with per-node zero points (E, A uint8; zE, zA int32)."""
+    p, nb = _ws(ws)
+    _check("lpdt_qconv_bwd_weight_affine", lib().lpdt_qconv_bwd_weight_affine(
+        C.byref(desc), _ptr(E), _ptr(sE), _ptr(zE), _ptr(A), _ptr(sA), _ptr(zA), _ptr(dW), dw_node_stride,
+        _ptr(dWacc), p, nb, _ptr(dev_status), _stream()))
 
 
 def lpdt_qconv_bwd_data(desc, E, sE, Wq, sW, dA=None, dAacc=None, ws=None, dev_status=None, addend=None):

@@ -346,6 +346,15 @@ extern "C" lpdt_status lpdt_qconv_fwd_affine(const lpdt_conv_desc *d, const uint
     return LPDT_OK;
 }
 
+// Backward-data contraction on raw codes (signed, or unsigned when `uns`): kernel choice only.
+static lpdt_status bwd_data_impl(const lpdt_conv_desc *d, const int8_t *E, const float *sE, const int8_t *Wq,
+                                 const float *sW, float *dA, int32_t *dAacc, const float *addend, void *ws,
+                                 int32_t *dev_status, cudaStream_t st, bool uns) {
+    if (use_tc(*d) && aligned(E, 16) && aligned(Wq, 16) && (!dA || aligned(dA, 16)) && (!dAacc || aligned(dAacc, 16)))
+        return run_pix(*d, 1, E, sE, Wq, sW, nullptr, 0, dA, dAacc, dev_status, st, uns, addend);
+    return generic_bwd_data(*d, E, sE, Wq, sW, dA, dAacc, addend, ws, st, uns);
+}
+
 extern "C" lpdt_status lpdt_qconv_bwd_data(const lpdt_conv_desc *d, const int8_t *E, const float *sE,
                                            const int8_t *Wq, const float *sW, float *dA, int32_t *dAacc,
                                            const float *addend, void *ws, size_t ws_bytes, int32_t *dev_status,
@@ -357,9 +366,29 @@ extern "C" lpdt_status lpdt_qconv_bwd_data(const lpdt_conv_desc *d, const int8_t
     LPDT_CHECK_ARG(!dA || (sE && sW));
     LPDT_CHECK_ARG(!addend || (dA && addend != dA && aligned(addend, 16)));
     if (!ws || ws_bytes < lpdt_qconv_workspace_size(d, 1)) return LPDT_ERR_WORKSPACE;
-    if (use_tc(*d) && aligned(E, 16) && aligned(Wq, 16) && (!dA || aligned(dA, 16)) && (!dAacc || aligned(dAacc, 16)))
-        return run_pix(*d, 1, E, sE, Wq, sW, nullptr, 0, dA, dAacc, dev_status, as_stream(stream), false, addend);
-    return generic_bwd_data(*d, E, sE, Wq, sW, dA, dAacc, addend, ws, as_stream(stream));
+    return bwd_data_impl(d, E, sE, Wq, sW, dA, dAacc, addend, ws, dev_status, as_stream(stream), false);
+}
+
+// Backward-weight contraction on raw codes.  Workspace: [int32 sums (used unless the caller gave dWacc) |
+// zero-padded input copy].
+static lpdt_status bwd_weight_impl(const lpdt_conv_desc *d, const int8_t *E, const float *sE, const int8_t *A,
+                                   const float *sA, float *dW, int64_t dw_node_stride, int32_t *dWacc, void *ws,
+                                   int32_t *dev_status, cudaStream_t st, bool uns) {
+    const size_t acc_bytes = align_up((size_t)d->nodes * d->Cout * d->R * d->S * d->Cin * sizeof(int32_t), 256);
+    int32_t *acc_ws = (int32_t *)ws;
+    lpdt_conv_desc dp;
+    if (use_tc(*d) && d->B > 0 && aligned(E, 16) && aligned(A, 16)) {
+        lpdt_status r = tc::tc_wgrad(*d, d->Cin, E, sE, A, sA, dWacc, acc_ws, dW, dw_node_stride, dev_status, st, uns);
+        if (r != LPDT_ERR_UNSUPPORTED) return r;
+    } else if (use_tc_padded(*d, &dp) && d->B > 0 && aligned(E, 16)) {
+        int8_t *Ap = (int8_t *)((char *)ws + acc_bytes);
+        const int64_t arows = (int64_t)d->nodes * d->B * d->H * d->W;
+        launch_k(pad_channels_kernel, grid_for(arows * dp.Cin / 16), 256, 0, st, A, Ap, arows, d->Cin, dp.Cin);
+        LPDT_LAUNCH_CHECK();
+        lpdt_status r = tc::tc_wgrad(dp, d->Cin, E, sE, Ap, sA, dWacc, acc_ws, dW, dw_node_stride, dev_status, st, uns);
+        if (r != LPDT_ERR_UNSUPPORTED) return r;
+    }
+    return generic_bwd_weight(*d, E, sE, A, sA, dW, dw_node_stride, dWacc, acc_ws, st, uns);
 }
 
 extern "C" lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8_t *E, const float *sE,
@@ -373,21 +402,259 @@ extern "C" lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8
     LPDT_CHECK_ARG(!dW || (sE && sA));
     LPDT_CHECK_ARG(!dW || dw_node_stride >= (int64_t)d->Cout * d->R * d->S * d->Cin || d->nodes == 1);
     if (!ws || ws_bytes < lpdt_qconv_workspace_size(d, 2) || !aligned(ws, 256)) return LPDT_ERR_WORKSPACE;
-    cudaStream_t st = as_stream(stream);
-    // workspace: [int32 sums (used unless the caller gave dWacc) | zero-padded input copy]
-    const size_t acc_bytes = align_up((size_t)d->nodes * d->Cout * d->R * d->S * d->Cin * sizeof(int32_t), 256);
-    int32_t *acc_ws = (int32_t *)ws;
-    lpdt_conv_desc dp;
-    if (use_tc(*d) && d->B > 0 && aligned(E, 16) && aligned(A, 16)) {
-        lpdt_status r = tc::tc_wgrad(*d, d->Cin, E, sE, A, sA, dWacc, acc_ws, dW, dw_node_stride, dev_status, st);
-        if (r != LPDT_ERR_UNSUPPORTED) return r;
-    } else if (use_tc_padded(*d, &dp) && d->B > 0 && aligned(E, 16)) {
-        int8_t *Ap = (int8_t *)((char *)ws + acc_bytes);
-        const int64_t arows = (int64_t)d->nodes * d->B * d->H * d->W;
-        launch_k(pad_channels_kernel, grid_for(arows * dp.Cin / 16), 256, 0, st, A, Ap, arows, d->Cin, dp.Cin);
-        LPDT_LAUNCH_CHECK();
-        lpdt_status r = tc::tc_wgrad(dp, d->Cin, E, sE, Ap, sA, dWacc, acc_ws, dW, dw_node_stride, dev_status, st);
-        if (r != LPDT_ERR_UNSUPPORTED) return r;
+    return bwd_weight_impl(d, E, sE, A, sA, dW, dw_node_stride, dWacc, ws, dev_status, as_stream(stream), false);
+}
+
+// ---- backward products on affine (zero-point) operands -----------------------------------------
+// With e' = qe - zE, w' = qw - zW, a' = qa - zA and the sums running over the taps that exist,
+//   sum e'w' = sum qe*qw - zW * sum qe - zE * sum qw + (terms) * zE*zW          (backward-data)
+//   sum e'a' = sum qe*qa - zA * sum qe - zE * sum qa + (terms) * zE*zA          (backward-weight)
+// the first term is the contraction engine on the unsigned codes; the others come from channel sums
+// of the operands, gathered over the same taps.  All arithmetic is modulo 2^32.
+namespace lpdt {
+
+// wsum[n][r][s][ci] = sum over co of W[n][co][r][s][ci]; one thread per output, ci fastest.
+__global__ void weight_cout_sum_kernel(lpdt_conv_desc d, const uint8_t *__restrict__ Wq, int32_t *__restrict__ wsum) {
+    pdl_enter();
+    const int per = d.R * d.S * d.Cin;
+    const int64_t total = (int64_t)d.nodes * per;
+    for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
+        const int n = (int)(o / per), i = (int)(o % per);
+        const uint8_t *w = Wq + (int64_t)n * d.Cout * per + i;
+        unsigned sum = 0;
+        for (int co = 0; co < d.Cout; ++co) sum += w[(int64_t)co * per];
+        wsum[o] = (int32_t)sum;
     }
-    return generic_bwd_weight(*d, E, sE, A, sA, dW, dw_node_stride, dWacc, acc_ws, st);
+}
+
+// One thread per (input pixel, V consecutive input channels).
+template <int V>
+__global__ void affine_fix_bwd_data_kernel(lpdt_conv_desc d, int Ho, int Wo, const int32_t *__restrict__ raw,
+                                           const int32_t *__restrict__ esum, const int32_t *__restrict__ wsum,
+                                           const int32_t *__restrict__ zE, const int32_t *__restrict__ zW,
+                                           const float *__restrict__ sE, const float *__restrict__ sW,
+                                           float *__restrict__ dA, int32_t *__restrict__ dAacc) {
+    pdl_enter();
+    const int chunks = d.Cin / V;
+    const int64_t total = (int64_t)d.nodes * d.B * d.H * d.W * chunks;
+    for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
+        const int ci0 = (int)(o % chunks) * V;
+        const int64_t pix = o / chunks;
+        const int iw = (int)(pix % d.W);
+        const int ih = (int)((pix / d.W) % d.H);
+        const int64_t nb = pix / ((int64_t)d.W * d.H);
+        const int n = (int)(nb / d.B);
+        unsigned es = 0, cnt = 0, ws_[V];
+#pragma unroll
+        for (int k = 0; k < V; ++k) ws_[k] = 0;
+        for (int r = 0; r < d.R; ++r) {
+            const int th = ih + d.pad - r;
+            if (th < 0 || th % d.stride) continue;
+            const int oh = th / d.stride;
+            if (oh >= Ho) continue;
+            for (int s = 0; s < d.S; ++s) {
+                const int tw = iw + d.pad - s;
+                if (tw < 0 || tw % d.stride) continue;
+                const int ow = tw / d.stride;
+                if (ow >= Wo) continue;
+                es += (unsigned)__ldg(esum + (nb * Ho + oh) * Wo + ow);
+                cnt += (unsigned)d.Cout;
+                const int32_t *wp = wsum + (((int64_t)n * d.R + r) * d.S + s) * d.Cin + ci0;
+#pragma unroll
+                for (int k = 0; k < V; ++k) ws_[k] += (unsigned)__ldg(wp + k);
+            }
+        }
+        const unsigned ze = (unsigned)zE[n], zw = (unsigned)zW[n];
+        const unsigned fixed = cnt * ze * zw - zw * es;
+        const float sc = dA ? __fmul_rn(sE[n], sW[n]) : 0.f;
+        const int64_t oi = pix * d.Cin + ci0;
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            const int acc = (int)((unsigned)raw[oi + k] + fixed - ze * ws_[k]);
+            if (dAacc) dAacc[oi + k] = acc;
+            if (dA) dA[oi + k] = __fmul_rn(__int2float_rn(acc), sc);
+        }
+    }
+}
+
+// col[n][pos][c] = sum over the batch of src[n][b][pos][c] (unsigned codes); one thread per output, c fastest.
+__global__ void batch_sum_u8_kernel(const uint8_t *__restrict__ src, int nodes, int B, int64_t per_image,
+                                    int32_t *__restrict__ col) {
+    pdl_enter();
+    const int64_t total = (int64_t)nodes * per_image;
+    for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t n = o / per_image, i = o % per_image;
+        const uint8_t *p = src + n * B * per_image + i;
+        unsigned sum = 0;
+        for (int b = 0; b < B; ++b) sum += p[(int64_t)b * per_image];
+        col[o] = (int32_t)sum;
+    }
+}
+
+// Sums of a batch-summed image over the output positions whose tap (r, s) lies inside the input image:
+//   of_input = 0: tab[n][r][s][c] = sum col[n][oh][ow][c]                        (col over the OUTPUT image, C = Cout)
+//   of_input = 1: tab[n][r][s][c] = sum col[n][oh*st+r-pad][ow*st+s-pad][c]      (col over the INPUT image, C = Cin)
+// block (tap, node), threads over channels.
+__global__ void tap_table_kernel(lpdt_conv_desc d, int Ho, int Wo, int of_input, int C,
+                                 const int32_t *__restrict__ col, int32_t *__restrict__ tab) {
+    pdl_enter();
+    const int tap = blockIdx.x, n = blockIdx.y, r = tap / d.S, s = tap % d.S;
+    const int Hc = of_input ? d.H : Ho, Wc = of_input ? d.W : Wo;
+    for (int c = threadIdx.x; c < C; c += blockDim.x) {
+        unsigned sum = 0;
+        for (int oh = 0; oh < Ho; ++oh) {
+            const int ih = oh * d.stride + r - d.pad;
+            if (ih < 0 || ih >= d.H) continue;
+            for (int ow = 0; ow < Wo; ++ow) {
+                const int iw = ow * d.stride + s - d.pad;
+                if (iw < 0 || iw >= d.W) continue;
+                const int ph = of_input ? ih : oh, pw = of_input ? iw : ow;
+                sum += (unsigned)col[(((int64_t)n * Hc + ph) * Wc + pw) * C + c];
+            }
+        }
+        tab[((int64_t)n * d.R * d.S + tap) * C + c] = (int32_t)sum;
+    }
+}
+
+// One thread per weight-gradient entry (n, co, r, s, ci); ci fastest.
+__global__ void affine_fix_bwd_weight_kernel(lpdt_conv_desc d, int Ho, int Wo, const int32_t *__restrict__ raw,
+                                             const int32_t *__restrict__ tabE, const int32_t *__restrict__ tabA,
+                                             const int32_t *__restrict__ zE, const int32_t *__restrict__ zA,
+                                             const float *__restrict__ sE, const float *__restrict__ sA,
+                                             float *__restrict__ dW, int64_t dw_stride, int32_t *__restrict__ dWacc) {
+    pdl_enter();
+    const int taps = d.R * d.S;
+    const int64_t per_node = (int64_t)d.Cout * taps * d.Cin;
+    const int64_t total = per_node * d.nodes;
+    for (int64_t o = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; o < total; o += (int64_t)gridDim.x * blockDim.x) {
+        const int n = (int)(o / per_node);
+        const int64_t i = o % per_node;
+        const int ci = (int)(i % d.Cin);
+        const int tap = (int)((i / d.Cin) % taps);
+        const int co = (int)(i / ((int64_t)d.Cin * taps));
+        const int r = tap / d.S, s = tap % d.S;
+        // output rows / columns whose tap lies inside the input image
+        int nh = 0, nw = 0;
+        for (int oh = 0; oh < Ho; ++oh) { const int ih = oh * d.stride + r - d.pad; nh += (ih >= 0 && ih < d.H); }
+        for (int ow = 0; ow < Wo; ++ow) { const int iw = ow * d.stride + s - d.pad; nw += (iw >= 0 && iw < d.W); }
+        const unsigned cnt = (unsigned)d.B * (unsigned)nh * (unsigned)nw;
+        const unsigned ze = (unsigned)zE[n], za = (unsigned)zA[n];
+        const unsigned te = (unsigned)tabE[((int64_t)n * taps + tap) * d.Cout + co];
+        const unsigned ta = (unsigned)tabA[((int64_t)n * taps + tap) * d.Cin + ci];
+        const int acc = (int)((unsigned)raw[o] - za * te - ze * ta + cnt * ze * za);
+        if (dWacc) dWacc[o] = acc;
+        if (dW) dW[(int64_t)n * dw_stride + i] = __fmul_rn(__int2float_rn(acc), __fmul_rn(sE[n], sA[n]));
+    }
+}
+
+}  // namespace lpdt
+
+static size_t affine_bwd_data_raw_bytes(const lpdt_conv_desc *d) {
+    return align_up((size_t)d->nodes * d->B * d->H * d->W * d->Cin * sizeof(int32_t), 256);
+}
+static size_t affine_esum_bytes(const lpdt_conv_desc *d) {
+    const int Ho = conv_out(d->H, d->pad, d->R, d->stride), Wo = conv_out(d->W, d->pad, d->S, d->stride);
+    return align_up((size_t)d->nodes * d->B * Ho * Wo * sizeof(int32_t), 256);
+}
+static size_t affine_wsum_bytes(const lpdt_conv_desc *d) {
+    return align_up((size_t)d->nodes * d->R * d->S * d->Cin * sizeof(int32_t), 256);
+}
+
+extern "C" size_t lpdt_qconv_bwd_data_affine_workspace_size(const lpdt_conv_desc *d) {
+    if (!d || d->nodes <= 0 || check_desc(d) != LPDT_OK) return 256;
+    return affine_bwd_data_raw_bytes(d) + affine_esum_bytes(d) + affine_wsum_bytes(d) + lpdt_qconv_workspace_size(d, 1);
+}
+
+extern "C" lpdt_status lpdt_qconv_bwd_data_affine(const lpdt_conv_desc *d, const uint8_t *E, const float *sE,
+                                                  const int32_t *zE, const uint8_t *Wq, const float *sW,
+                                                  const int32_t *zW, float *dA, int32_t *dAacc, void *ws,
+                                                  size_t ws_bytes, int32_t *dev_status, void *stream) {
+    lpdt_status s = check_desc(d);
+    if (s != LPDT_OK) return s;
+    if (d->nodes == 0 || d->B == 0) return LPDT_OK;
+    LPDT_CHECK_ARG(E && Wq && zE && zW && (dA || dAacc));
+    LPDT_CHECK_ARG(!dA || (sE && sW));
+    if (!ws || !aligned(ws, 256) || ws_bytes < lpdt_qconv_bwd_data_affine_workspace_size(d)) return LPDT_ERR_WORKSPACE;
+    cudaStream_t st = as_stream(stream);
+    const int Ho = conv_out(d->H, d->pad, d->R, d->stride), Wo = conv_out(d->W, d->pad, d->S, d->stride);
+    int32_t *raw = (int32_t *)ws;
+    int32_t *esum = (int32_t *)((char *)ws + affine_bwd_data_raw_bytes(d));
+    int32_t *wsum = (int32_t *)((char *)esum + affine_esum_bytes(d));
+    void *inner = (char *)wsum + affine_wsum_bytes(d);
+    s = bwd_data_impl(d, reinterpret_cast<const int8_t *>(E), nullptr, reinterpret_cast<const int8_t *>(Wq), nullptr,
+                      nullptr, raw, nullptr, inner, dev_status, st, true);
+    if (s != LPDT_OK) return s;
+    s = row_sum_launch(E, (int64_t)d->nodes * d->B * Ho * Wo, d->Cout, esum, st);
+    if (s != LPDT_OK) return s;
+    launch_k(weight_cout_sum_kernel, grid_for((int64_t)d->nodes * d->R * d->S * d->Cin), 256, 0, st, *d, Wq, wsum);
+    LPDT_LAUNCH_CHECK();
+    const bool v4 = d->Cin % 4 == 0;
+    const int64_t work = (int64_t)d->nodes * d->B * d->H * d->W * (d->Cin / (v4 ? 4 : 1));
+    if (v4)
+        launch_k(affine_fix_bwd_data_kernel<4>, grid_for(work), 256, 0, st, *d, Ho, Wo, raw, esum, wsum, zE, zW, sE, sW, dA, dAacc);
+    else
+        launch_k(affine_fix_bwd_data_kernel<1>, grid_for(work), 256, 0, st, *d, Ho, Wo, raw, esum, wsum, zE, zW, sE, sW, dA, dAacc);
+    LPDT_LAUNCH_CHECK();
+    return LPDT_OK;
+}
+
+static size_t affine_wg_raw_bytes(const lpdt_conv_desc *d) {
+    return align_up((size_t)d->nodes * d->Cout * d->R * d->S * d->Cin * sizeof(int32_t), 256);
+}
+static size_t affine_colE_bytes(const lpdt_conv_desc *d) {
+    const int Ho = conv_out(d->H, d->pad, d->R, d->stride), Wo = conv_out(d->W, d->pad, d->S, d->stride);
+    return align_up((size_t)d->nodes * Ho * Wo * d->Cout * sizeof(int32_t), 256);
+}
+static size_t affine_colA_bytes(const lpdt_conv_desc *d) {
+    return align_up((size_t)d->nodes * d->H * d->W * d->Cin * sizeof(int32_t), 256);
+}
+static size_t affine_tab_bytes(const lpdt_conv_desc *d, int C) {
+    return align_up((size_t)d->nodes * d->R * d->S * C * sizeof(int32_t), 256);
+}
+
+extern "C" size_t lpdt_qconv_bwd_weight_affine_workspace_size(const lpdt_conv_desc *d) {
+    if (!d || d->nodes <= 0 || check_desc(d) != LPDT_OK) return 256;
+    return affine_wg_raw_bytes(d) + affine_colE_bytes(d) + affine_colA_bytes(d) + affine_tab_bytes(d, d->Cout) +
+           affine_tab_bytes(d, d->Cin) + lpdt_qconv_workspace_size(d, 2);
+}
+
+extern "C" lpdt_status lpdt_qconv_bwd_weight_affine(const lpdt_conv_desc *d, const uint8_t *E, const float *sE,
+                                                    const int32_t *zE, const uint8_t *A, const float *sA,
+                                                    const int32_t *zA, float *dW, int64_t dw_node_stride,
+                                                    int32_t *dWacc, void *ws, size_t ws_bytes, int32_t *dev_status,
+                                                    void *stream) {
+    lpdt_status s = check_desc(d);
+    if (s != LPDT_OK) return s;
+    if (d->nodes == 0) return LPDT_OK;
+    LPDT_CHECK_ARG((d->B == 0 || (E && A)) && zE && zA && (dW || dWacc));
+    LPDT_CHECK_ARG(!dW || (sE && sA));
+    LPDT_CHECK_ARG(!dW || dw_node_stride >= (int64_t)d->Cout * d->R * d->S * d->Cin || d->nodes == 1);
+    if (d->nodes > 65535) return LPDT_ERR_UNSUPPORTED;
+    if (!ws || !aligned(ws, 256) || ws_bytes < lpdt_qconv_bwd_weight_affine_workspace_size(d)) return LPDT_ERR_WORKSPACE;
+    cudaStream_t st = as_stream(stream);
+    const int Ho = conv_out(d->H, d->pad, d->R, d->stride), Wo = conv_out(d->W, d->pad, d->S, d->stride);
+    int32_t *raw = (int32_t *)ws;
+    int32_t *colE = (int32_t *)((char *)ws + affine_wg_raw_bytes(d));
+    int32_t *colA = (int32_t *)((char *)colE + affine_colE_bytes(d));
+    int32_t *tabE = (int32_t *)((char *)colA + affine_colA_bytes(d));
+    int32_t *tabA = (int32_t *)((char *)tabE + affine_tab_bytes(d, d->Cout));
+    void *inner = (char *)tabA + affine_tab_bytes(d, d->Cin);
+    s = bwd_weight_impl(d, reinterpret_cast<const int8_t *>(E), nullptr, reinterpret_cast<const int8_t *>(A), nullptr,
+                        nullptr, 0, raw, inner, dev_status, st, true);
+    if (s != LPDT_OK) return s;
+    launch_k(batch_sum_u8_kernel, grid_for((int64_t)d->nodes * Ho * Wo * d->Cout), 256, 0, st, E, d->nodes, d->B,
+             (int64_t)Ho * Wo * d->Cout, colE);
+    LPDT_LAUNCH_CHECK();
+    launch_k(batch_sum_u8_kernel, grid_for((int64_t)d->nodes * d->H * d->W * d->Cin), 256, 0, st, A, d->nodes, d->B,
+             (int64_t)d->H * d->W * d->Cin, colA);
+    LPDT_LAUNCH_CHECK();
+    const dim3 tgrid(d->R * d->S, d->nodes);
+    launch_k(tap_table_kernel, tgrid, 128, 0, st, *d, Ho, Wo, 0, d->Cout, colE, tabE);
+    LPDT_LAUNCH_CHECK();
+    launch_k(tap_table_kernel, tgrid, 128, 0, st, *d, Ho, Wo, 1, d->Cin, colA, tabA);
+    LPDT_LAUNCH_CHECK();
+    launch_k(affine_fix_bwd_weight_kernel, grid_for((int64_t)d->nodes * d->Cout * d->R * d->S * d->Cin), 256, 0, st, *d, Ho,
+             Wo, raw, tabE, tabA, zE, zA, sE, sA, dW, dw_node_stride, dWacc);
+    LPDT_LAUNCH_CHECK();
+    return LPDT_OK;
 }

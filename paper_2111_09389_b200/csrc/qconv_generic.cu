@@ -92,7 +92,8 @@ __global__ void transpose_weights_kernel(lpdt_conv_desc d, const int8_t *__restr
 __global__ void conv_bwd_data_generic(lpdt_conv_desc d, int Ho, int Wo, const int8_t *__restrict__ E,
                                       const int8_t *__restrict__ Wt, int32_t *__restrict__ acc_out,
                                       float *__restrict__ dA, const float *__restrict__ s1,
-                                      const float *__restrict__ s2, bool vec4, const float *__restrict__ addend) {
+                                      const float *__restrict__ s2, bool vec4, const float *__restrict__ addend,
+                                      bool uns) {
     pdl_enter();
     const int64_t per_node = (int64_t)d.B * d.H * d.W * d.Cin;
     const int64_t total = per_node * d.nodes;
@@ -116,7 +117,8 @@ __global__ void conv_bwd_data_generic(lpdt_conv_desc d, int Ho, int Wo, const in
                 if (ow >= Wo) continue;
                 const int8_t *e = E + ((((int64_t)n * d.B + b) * Ho + oh) * Wo + ow) * d.Cout;
                 const int8_t *w = Wt + ((((int64_t)n * d.Cin + ci) * d.R + r) * d.S + s) * d.Cout;
-                acc += dot_s8(e, w, d.Cout, vec4);
+                acc += uns ? dot_u8(reinterpret_cast<const uint8_t *>(e), reinterpret_cast<const uint8_t *>(w), d.Cout, vec4)
+                           : dot_s8(e, w, d.Cout, vec4);
             }
         }
         if (acc_out) acc_out[o] = acc;
@@ -132,7 +134,7 @@ __global__ void conv_bwd_data_generic(lpdt_conv_desc d, int Ho, int Wo, const in
 // pixel chunk and adds the partial sums with integer atomics (exact).
 __global__ void conv_bwd_weight_generic(lpdt_conv_desc d, int Ho, int Wo, int chunk,
                                         const int8_t *__restrict__ E, const int8_t *__restrict__ A,
-                                        int32_t *__restrict__ acc_out) {
+                                        int32_t *__restrict__ acc_out, bool uns) {
     pdl_enter();
     const int n = blockIdx.y;
     const int64_t npix = (int64_t)d.B * Ho * Wo;
@@ -153,8 +155,9 @@ __global__ void conv_bwd_weight_generic(lpdt_conv_desc d, int Ho, int Wo, int ch
             int b = (int)(q / Ho);
             int ih = oh * d.stride + r - d.pad, iw = ow * d.stride + s - d.pad;
             if (ih < 0 || ih >= d.H || iw < 0 || iw >= d.W) continue;
-            acc += (int)E[((int64_t)n * npix + p) * d.Cout + co] *
-                   (int)A[((((int64_t)n * d.B + b) * d.H + ih) * d.W + iw) * d.Cin + ci];
+            const int8_t e = E[((int64_t)n * npix + p) * d.Cout + co];
+            const int8_t a = A[((((int64_t)n * d.B + b) * d.H + ih) * d.W + iw) * d.Cin + ci];
+            acc += uns ? (int)((unsigned)(uint8_t)e * (unsigned)(uint8_t)a) : (int)e * (int)a;
         }
         if (acc) atomicAdd(acc_out + (int64_t)n * nout + o, acc);
     }
@@ -199,7 +202,8 @@ lpdt_status generic_fwd(const lpdt_conv_desc &d, const int8_t *A, const float *s
 }
 
 lpdt_status generic_bwd_data(const lpdt_conv_desc &d, const int8_t *E, const float *sE, const int8_t *Wq,
-                             const float *sW, float *dA, int32_t *dAacc, const float *addend, void *ws, cudaStream_t st) {
+                             const float *sW, float *dA, int32_t *dAacc, const float *addend, void *ws, cudaStream_t st,
+                             bool uns) {
     const int Ho = conv_out(d.H, d.pad, d.R, d.stride), Wo = conv_out(d.W, d.pad, d.S, d.stride);
     int8_t *Wt = (int8_t *)ws;
     const int64_t wn = (int64_t)d.nodes * d.Cout * d.R * d.S * d.Cin;
@@ -208,14 +212,14 @@ lpdt_status generic_bwd_data(const lpdt_conv_desc &d, const int8_t *E, const flo
     const int64_t total = (int64_t)d.nodes * d.B * d.H * d.W * d.Cin;
     const bool vec4 = d.Cout % 4 == 0 && aligned(E, 4) && aligned(Wt, 4);
     g_last_kernel = "lpdt::conv_bwd_data_generic";
-    launch_k(conv_bwd_data_generic, grid_for(total), 256, 0, st, d, Ho, Wo, E, Wt, dAacc, dA, sE, sW, vec4, addend);
+    launch_k(conv_bwd_data_generic, grid_for(total), 256, 0, st, d, Ho, Wo, E, Wt, dAacc, dA, sE, sW, vec4, addend, uns);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }
 
 lpdt_status generic_bwd_weight(const lpdt_conv_desc &d, const int8_t *E, const float *sE, const int8_t *A,
                                const float *sA, float *dW, int64_t dw_stride, int32_t *dWacc, void *ws,
-                               cudaStream_t st) {
+                               cudaStream_t st, bool uns) {
     const int Ho = conv_out(d.H, d.pad, d.R, d.stride), Wo = conv_out(d.W, d.pad, d.S, d.stride);
     const int64_t per_node = (int64_t)d.Cout * d.R * d.S * d.Cin;
     if (d.nodes > 65535) return LPDT_ERR_UNSUPPORTED;        // nodes ride in grid.y
@@ -226,7 +230,7 @@ lpdt_status generic_bwd_weight(const lpdt_conv_desc &d, const int8_t *E, const f
         int chunk = 4;
         while (ceil_div(npix, chunk) * d.nodes > (int64_t)kNumSMs * 16) chunk *= 2;
         g_last_kernel = "lpdt::conv_bwd_weight_generic";
-        launch_k(conv_bwd_weight_generic, dim3((unsigned)ceil_div(npix, chunk), d.nodes), 256, 0, st, d, Ho, Wo, chunk, E, A, acc);
+        launch_k(conv_bwd_weight_generic, dim3((unsigned)ceil_div(npix, chunk), d.nodes), 256, 0, st, d, Ho, Wo, chunk, E, A, acc, uns);
         LPDT_LAUNCH_CHECK();
     }
     if (dW) {

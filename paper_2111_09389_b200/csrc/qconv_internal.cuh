@@ -11,10 +11,11 @@ lpdt_status generic_fwd(const lpdt_conv_desc &d, const int8_t *A, const float *s
                         const float *sW, const float *bias, int64_t bias_stride, float *Y, int32_t *Yacc,
                         cudaStream_t st, bool uns = false);
 lpdt_status generic_bwd_data(const lpdt_conv_desc &d, const int8_t *E, const float *sE, const int8_t *Wq,
-                             const float *sW, float *dA, int32_t *dAacc, const float *addend, void *ws, cudaStream_t st);
+                             const float *sW, float *dA, int32_t *dAacc, const float *addend, void *ws, cudaStream_t st,
+                             bool uns = false);
 lpdt_status generic_bwd_weight(const lpdt_conv_desc &d, const int8_t *E, const float *sE, const int8_t *A,
                                const float *sA, float *dW, int64_t dw_stride, int32_t *dWacc, void *ws,
-                               cudaStream_t st);
+                               cudaStream_t st, bool uns = false);
 
 lpdt_status dequant_acc_launch(const int32_t *acc, int nodes, int64_t per_node, const float *s1,
                                const float *s2, float *out, int64_t out_stride, cudaStream_t st);
@@ -33,7 +34,7 @@ lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, cons
                         int32_t *dev_status, cudaStream_t st, bool uns = false, const float *addend = nullptr);
 lpdt_status tc_wgrad(const lpdt_conv_desc &d, int cin_real, const int8_t *E, const float *sE, const int8_t *A,
                      const float *sA, int32_t *acc_user, int32_t *acc_ws, float *dW, int64_t dw_stride,
-                     int32_t *dev_status, cudaStream_t st);
+                     int32_t *dev_status, cudaStream_t st, bool uns = false);
 }  // namespace tc
 
 }  // namespace lpdt

@@ -395,6 +395,7 @@ struct WgParams {
     float *dW; long long dw_stride;               // fp32 result, written here only if 1 split (nullable)
     const float *s1, *s2;                         // per-node scales of the two operands
     int32_t *dev_status;
+    int uns;                                      // operands are unsigned 8-bit codes
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -466,7 +467,7 @@ conv_wgrad_kernel(const __grid_constant__ CUtensorMap mapX, const __grid_constan
         }
     } else if (warp == 1) {
         {
-            const uint32_t idesc = idesc_i8(128, p.BNc, 1, 1);
+            const uint32_t idesc = idesc_i8(128, p.BNc, 1, 1, p.uns);
             // halo mode: M tile r stacks the S taps of filter row r, one pixel (16 bytes) apart; 8-pixel
             // K groups are one halo row apart
             const uint64_t a_tpl = p.halo ? smem_desc(0, p.PW * 16, 16, 0)
@@ -761,7 +762,7 @@ lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const flo
 // itself; with several it accumulates into zeroed int32 storage and a conversion launch follows.
 lpdt_status tc_wgrad(const lpdt_conv_desc &d, int cin_real, const int8_t *E, const float *sE, const int8_t *A,
                      const float *sA, int32_t *acc_user, int32_t *acc_ws, float *dW, int64_t dw_stride,
-                     int32_t *dev_status, cudaStream_t st) {
+                     int32_t *dev_status, cudaStream_t st, bool uns) {
     const int Ho = conv_out(d.H, d.pad, d.R, d.stride), Wo = conv_out(d.W, d.pad, d.S, d.stride);
     WgParams p = {};
     p.nodes = d.nodes; p.B = d.B; p.Ho = Ho; p.Wo = Wo; p.Cin = d.Cin; p.Cout = d.Cout;
@@ -819,7 +820,7 @@ lpdt_status tc_wgrad(const lpdt_conv_desc &d, int cin_real, const int8_t *E, con
     p.splits = (int)ceil_div(p.kblocks, p.kb_per_split);
     p.cin_real = cin_real; p.dW = dW; p.dw_stride = dw_stride; p.s1 = sE; p.s2 = sA;
     p.acc_out = p.splits == 1 ? acc_user : (acc_user ? acc_user : acc_ws);
-    p.dev_status = dev_status;
+    p.dev_status = dev_status; p.uns = uns ? 1 : 0;
     CUtensorMap mX, mE;
     if (p.halo) {
         uint64_t dims[4] = {(uint64_t)d.W * 16, (uint64_t)d.H, (uint64_t)d.B, (uint64_t)d.nodes};

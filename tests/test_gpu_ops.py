@@ -191,6 +191,44 @@ def test_qconv_fwd_affine(case):
     assert np.array_equal(Y.cpu().numpy(), oracle.dequant_acc(acc_ref, s1, s2, bias))
 
 
+@pytest.mark.parametrize("case", CONV_CASES)
+def test_qconv_bwd_affine(case):
+    """Both backward products on zero-point operands, every shape: int32 sums bit-exact, fp32 as dequant_acc;
+    the weight gradient also into a strided destination."""
+    nodes, B, H, W, Cin, Cout, R, S, stride, pad = case
+    rng = np.random.default_rng(78)
+    Ho, Wo = (H + 2 * pad - R) // stride + 1, (W + 2 * pad - S) // stride + 1
+    A = rng.integers(0, 256, (nodes, B, H, W, Cin), dtype=np.uint8)
+    Wq = rng.integers(0, 256, (nodes, Cout, R, S, Cin), dtype=np.uint8)
+    E = rng.integers(0, 256, (nodes, B, Ho, Wo, Cout), dtype=np.uint8)
+    zA, zW, zE = (rng.integers(0, 256, nodes).astype(np.int32) for _ in range(3))
+    zE[0], zW[0], zA[0] = 255, 0, 255                       # extreme zero points on one node
+    sA, sW, sE = (rng.uniform(0.001, 0.1, nodes).astype(np.float32) for _ in range(3))
+    dA_ref, o1 = oracle.qconv_bwd_data_affine(E, zE, Wq, zW, H, W, stride, pad)
+    dW_ref, o2 = oracle.qconv_bwd_weight_affine(E, zE, A, zA, R, S, stride, pad)
+    assert o1 == 0 and o2 == 0
+    desc = api.conv_desc(*case)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    Ed, Wd, Ad = dev(E), dev(Wq), dev(A)
+    dA = torch.empty(dA_ref.shape, dtype=torch.float32, device="cuda")
+    dAacc = torch.empty(dA_ref.shape, dtype=torch.int32, device="cuda")
+    api.lpdt_qconv_bwd_data_affine(desc, Ed, dev(sE), dev(zE), Wd, dev(sW), dev(zW), dA=dA, dAacc=dAacc,
+                                   ws=ws_bytes(api.lpdt_qconv_bwd_data_affine_workspace_size(desc)), dev_status=status)
+    assert np.array_equal(dAacc.cpu().numpy(), dA_ref)
+    assert np.array_equal(dA.cpu().numpy(), oracle.dequant_acc(dA_ref, sE, sW))
+    wn = Cout * R * S * Cin
+    stride_w = wn + 12
+    dW = torch.zeros(nodes, stride_w, dtype=torch.float32, device="cuda")
+    dWacc = torch.empty(dW_ref.shape, dtype=torch.int32, device="cuda")
+    api.lpdt_qconv_bwd_weight_affine(desc, Ed, dev(sE), dev(zE), Ad, dev(sA), dev(zA), dW=dW, dw_node_stride=stride_w,
+                                     dWacc=dWacc, ws=ws_bytes(api.lpdt_qconv_bwd_weight_affine_workspace_size(desc)),
+                                     dev_status=status)
+    assert int(status.item()) == 0
+    assert np.array_equal(dWacc.cpu().numpy(), dW_ref)
+    assert np.array_equal(dW[:, :wn].cpu().numpy(), oracle.dequant_acc(dW_ref, sE, sA).reshape(nodes, wn))
+    assert not dW[:, wn:].any()
+
+
 def test_qconv_fwd_affine_matches_quantizer_output():
     # end to end with lpdt_quantize's affine mode: real 0 maps to the zero point, so a zero-padded real
     # convolution of the dequantized tensors equals scale * acc
@@ -844,6 +882,6 @@ def test_qconv_cases_on_every_kernel_family(env):
     root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
     child_env = dict(os.environ, LPDT_CHILD="1", **env)
     r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_ops.py"), "-m", "gpu",
-                        "-q", "-x", "-k", "test_qconv_all_three or test_qconv_extreme or test_qconv_fwd_affine"], env=child_env, cwd=root,
+                        "-q", "-x", "-k", "test_qconv_all_three or test_qconv_extreme or test_qconv_fwd_affine or test_qconv_bwd_affine"], env=child_env, cwd=root,
                        capture_output=True, text=True, timeout=900)
     assert r.returncode == 0, r.stdout[-3000:] + r.stderr[-2000:]

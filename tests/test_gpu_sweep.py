@@ -159,3 +159,38 @@ def test_large_affine_forward(shape):
                                        stride, pad)
     assert ovf == 0
     assert np.array_equal(Y.cpu().numpy()[:, rows], ref)
+
+
+@pytest.mark.parametrize("shape", [("gemm", 2048, 4096, 4096), ("conv", 256, 32, 32)])
+def test_large_affine_backward(shape):
+    """Zero-point operands at sweep sizes, both backward products: sampled rows / images and a block of
+    weight-gradient entries recomputed by the oracle."""
+    g = torch.Generator(device="cuda"); g.manual_seed(19)
+    if shape[0] == "gemm":
+        _, M, N, K = shape
+        case = (1, M, 1, 1, K, N, 1, 1, 1, 0)
+    else:
+        _, Cc, HW, batch = shape
+        case = (1, batch, HW, HW, Cc, Cc, 3, 3, 1, 1)
+    nodes, B, H, W, Cin, Cout, R, S, stride, pad = case
+    desc = api.conv_desc(*case)
+    u8 = lambda *sh: torch.randint(0, 256, sh, generator=g, device="cuda", dtype=torch.uint8)
+    A, Wq, E = u8(nodes, B, H, W, Cin), u8(nodes, Cout, R, S, Cin), u8(nodes, B, H, W, Cout)
+    zA, zW, zE = (torch.tensor([v], dtype=torch.int32, device="cuda") for v in (133, 121, 90))
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    dA = torch.empty(nodes, B, H, W, Cin, dtype=torch.int32, device="cuda")
+    dW = torch.empty(nodes, Cout, R, S, Cin, dtype=torch.int32, device="cuda")
+    api.lpdt_qconv_bwd_data_affine(desc, E, None, zE, Wq, None, zW, dAacc=dA, dev_status=status,
+                                   ws=torch.empty(api.lpdt_qconv_bwd_data_affine_workspace_size(desc), dtype=torch.uint8, device="cuda"))
+    api.lpdt_qconv_bwd_weight_affine(desc, E, None, zE, A, None, zA, dWacc=dW, dev_status=status,
+                                     ws=torch.empty(api.lpdt_qconv_bwd_weight_affine_workspace_size(desc), dtype=torch.uint8, device="cuda"))
+    torch.cuda.synchronize()
+    assert int(status.item()) == 0
+    rows = np.unique(np.concatenate([np.arange(2), np.random.default_rng(3).integers(0, B, 4), [B - 1]]))
+    ref, _ = oracle.qconv_bwd_data_affine(E.cpu().numpy()[:, rows], zE.cpu().numpy(), Wq.cpu().numpy(), zW.cpu().numpy(),
+                                          H, W, stride, pad)
+    assert np.array_equal(dA.cpu().numpy()[:, rows], ref)             # the wrapped int32 sums
+    co = [0, Cout // 2 + 1, Cout - 1]
+    ref, _ = oracle.qconv_bwd_weight_affine(np.ascontiguousarray(E[..., co].cpu().numpy()), zE.cpu().numpy(),
+                                            A[..., :16].contiguous().cpu().numpy(), zA.cpu().numpy(), R, S, stride, pad)
+    assert np.array_equal(dW[:, co][..., :16].cpu().numpy(), ref)
