@@ -213,6 +213,17 @@ lpdt_status lpdt_qconv_bwd_weight(const lpdt_conv_desc *d, const int8_t *E, cons
                                   float *dW, int64_t dw_node_stride, int32_t *dWacc,
                                   void *ws, size_t ws_bytes, int32_t *dev_status, void *stream);
 
+/* Dequantize the raw int32 sums of up to 64 tensors in one launch (all weight gradients of a network, each
+ * left by lpdt_qconv_bwd_weight through dWacc as a contiguous [nodes][sizes[t]] block at acc + acc_offsets[t]):
+ *   out[n*out_node_stride + out_offsets[t] + i] = (float)acc[acc_offsets[t] + n*sizes[t] + i] * (s1[t][n]*s2[t][n])
+ * for i < sizes[t]: the fp32 result of lpdt_qconv_bwd_weight, bit for bit.  acc_offsets, sizes and out_offsets
+ * are HOST arrays (elements); s1 and s2 are HOST arrays of device pointers to the per-node scales of each
+ * tensor's two operands.  Errors: INVALID_ARG, UNSUPPORTED (more than 64 tensors), CUDA. */
+lpdt_status lpdt_dequantize_acc_batch(const int32_t *acc, int32_t nodes, int32_t n_tensors,
+                                      const int64_t *acc_offsets, const int64_t *sizes, const int64_t *out_offsets,
+                                      const float *const *s1, const float *const *s2,
+                                      float *out, int64_t out_node_stride, void *stream);
+
 /* ---------------------------------------------------------------------------
  * Forward contraction on affine (zero-point) operands: the quantization scheme
  * Section 3 names maps a real tensor to unsigned 8-bit codes with a scale and a
@@ -305,6 +316,15 @@ lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t H, int32_t 
 lpdt_status lpdt_range_evonorm_bwd_params(int32_t nodes, int32_t B, int32_t C, const void *ws, size_t ws_bytes,
                                           float *dv, float *dgamma, float *dbeta, int64_t grad_node_stride,
                                           void *stream);
+/* The second call for up to 64 layers in one launch (a network's norm layers at the end of its backward
+ * pass).  Layer l has C[l] channels, its partial sums in ws[l] (as left by lpdt_range_evonorm_bwd with null
+ * gradient pointers; same nodes and B for all layers), and its three gradient vectors back to back - dv,
+ * dgamma, dbeta, C[l] entries each - at grads + n*grad_node_stride + grad_offsets[l].  C, ws and
+ * grad_offsets are HOST arrays (ws holds device pointers).  Same sums, same order, same results as
+ * n_layers single calls.  Errors: INVALID_ARG, UNSUPPORTED (more than 64 layers), CUDA. */
+lpdt_status lpdt_range_evonorm_bwd_params_batch(int32_t nodes, int32_t B, int32_t n_layers, const int32_t *C,
+                                                const void *const *ws, const int64_t *grad_offsets,
+                                                float *grads, int64_t grad_node_stride, void *stream);
 
 /* ---------------------------------------------------------------------------
  * Comparison layers of Section 3 (the normalization study; not on the 8-bit path).

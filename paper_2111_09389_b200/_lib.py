@@ -54,6 +54,8 @@ SIGNATURES = {
     "lpdt_range_bn_workspace_size": (_sz, [_i32, _i32]),
     "lpdt_range_bn_fwd": (_i32, [_i32] * 5 + [_f32] + [_vp] * 3 + [_i64] + [_vp] * 6 + [_vp, _sz, _vp]),
     "lpdt_range_bn_bwd": (_i32, [_i32] * 5 + [_f32] + [_vp] * 3 + [_i64] + [_vp] * 8 + [_i64, _vp, _sz, _vp]),
+    "lpdt_range_evonorm_bwd_params_batch": (_i32, [_i32, _i32, _i32, _vp, _vp, _vp, _vp, _i64, _vp]),
+    "lpdt_dequantize_acc_batch": (_i32, [_vp, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp, _i64, _vp]),
     "lpdt_range_evonorm_bwd_params": (_i32, [_i32, _i32, _i32, _vp, _sz, _vp, _vp, _vp, _i64, _vp]),
     "lpdt_gossip_mix_workspace_size": (_sz, [_i32, _i64, _i32]),
     "lpdt_gossip_mix": (_i32, [_i32, _i64, _vp, _vp, _vp, _vp, _f32, _i32, _vp, _vp, _vp, _sz, _vp, _vp]),

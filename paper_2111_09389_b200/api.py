@@ -14,7 +14,7 @@ from ._lib import ConvDesc, lib
 # Kernels each entry point enqueues (memsets not counted); KERNEL_LAUNCHES accumulates them.
 KERNELS_PER_CALL = {
     "lpdt_quantize": 2, "lpdt_quantize_with_range": 1, "lpdt_quantize_static": 2, "lpdt_quantize_batch": 2, "lpdt_dequantize": 1, "lpdt_qconv_fwd": 1, "lpdt_qconv_fwd_affine": 4, "lpdt_qconv_bwd_data_affine": 4, "lpdt_qconv_bwd_weight_affine": 7, "lpdt_qconv_bwd_data": 2,
-    "lpdt_qconv_bwd_weight": 2, "lpdt_range_evonorm_fwd": 1, "lpdt_range_evonorm_bwd": 2, "lpdt_range_evonorm_bwd_params": 1,
+    "lpdt_qconv_bwd_weight": 2, "lpdt_range_evonorm_fwd": 1, "lpdt_range_evonorm_bwd": 2, "lpdt_range_evonorm_bwd_params": 1, "lpdt_range_evonorm_bwd_params_batch": 1, "lpdt_dequantize_acc_batch": 1,
     "lpdt_gossip_mix": 2, "lpdt_gossip_mix_q8": 3, "lpdt_deepsqueeze_mix": 2, "lpdt_pushsum_debias": 1, "lpdt_sgd_gossip_mix": 1, "lpdt_evonorm_s0_fwd": 1, "lpdt_evonorm_s0_bwd": 2, "lpdt_range_bn_fwd": 2, "lpdt_range_bn_bwd": 2, "lpdt_sgd_update": 1, "lpdt_residual_add": 1, "lpdt_residual_add_bwd": 1,
     "lpdt_avgpool": 1, "lpdt_avgpool_bwd": 1, "lpdt_maxpool2x2": 1, "lpdt_maxpool2x2_bwd": 1,
     "lpdt_softmax_ce": 1, "lpdt_colsum": 1, "lpdt_selftest_bounded_wait": 1,
@@ -224,6 +224,9 @@ def lpdt_qconv_bwd_weight(desc, E, sE, A, sA, dW=None, dw_node_stride=0, dWacc=N
                                                                 _ptr(sA), _ptr(dW), dw_node_stride,
                                                                 _ptr(dWacc), p, nb, _ptr(dev_status),
                                                                 _stream()))
+    if dW is None:                      # raw sums only: no conversion launch
+        global KERNEL_LAUNCHES
+        KERNEL_LAUNCHES -= 1
 
 
 def lpdt_range_evonorm_fwd(nodes, B, H, W, Cc, groups, eps, x, v, gamma, beta, param_node_stride, y,
@@ -292,6 +295,30 @@ def lpdt_range_evonorm_bwd_params(nodes, B, Cc, ws, dv, dgamma, dbeta, grad_node
     p, nb = _ws(ws)
     _check("lpdt_range_evonorm_bwd_params", lib().lpdt_range_evonorm_bwd_params(
         nodes, B, Cc, p, nb, _ptr(dv), _ptr(dgamma), _ptr(dbeta), grad_node_stride, _stream()))
+
+
+def lpdt_range_evonorm_bwd_params_batch(nodes, B, channels, workspaces, grad_offsets, grads, grad_node_stride):
+    """channels / grad_offsets: host sequences of ints; workspaces: the layers' partial-sum tensors."""
+    n = len(channels)
+    cc = (C.c_int32 * n)(*[int(v) for v in channels])
+    wp = (C.c_void_p * n)(*[_ptr(w) for w in workspaces])
+    go = (C.c_int64 * n)(*[int(v) for v in grad_offsets])
+    _check("lpdt_range_evonorm_bwd_params_batch", lib().lpdt_range_evonorm_bwd_params_batch(
+        nodes, B, n, C.addressof(cc), C.addressof(wp), C.addressof(go), _ptr(grads), grad_node_stride, _stream()))
+
+
+def lpdt_dequantize_acc_batch(acc, nodes, acc_offsets, sizes, out_offsets, s1, s2, out, out_node_stride):
+    """acc_offsets / sizes / out_offsets: host sequences of ints; s1 / s2: sequences of per-node scale tensors,
+    one pair per tensor."""
+    n = len(sizes)
+    af = (C.c_int64 * n)(*[int(v) for v in acc_offsets])
+    sz = (C.c_int64 * n)(*[int(v) for v in sizes])
+    of = (C.c_int64 * n)(*[int(v) for v in out_offsets])
+    p1 = (C.c_void_p * n)(*[_ptr(t) for t in s1])
+    p2 = (C.c_void_p * n)(*[_ptr(t) for t in s2])
+    _check("lpdt_dequantize_acc_batch", lib().lpdt_dequantize_acc_batch(
+        _ptr(acc), nodes, n, C.addressof(af), C.addressof(sz), C.addressof(of), C.addressof(p1), C.addressof(p2),
+        _ptr(out), out_node_stride, _stream()))
 
 
 def lpdt_gossip_mix_workspace_size(nodes, d, n_segments):

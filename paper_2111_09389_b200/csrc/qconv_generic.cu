@@ -175,6 +175,28 @@ __global__ void dequant_acc_kernel(const int32_t *__restrict__ acc, int nodes, i
     }
 }
 
+// The same conversion for many tensors in one launch (all weight gradients of a network): the sums of
+// tensor t are a contiguous [nodes][size[t]] block at acc + acc_off[t]; its fp32 values go to offset
+// out_off[t] of every node's output row; each tensor has its own pair of per-node scales.
+// grid = (blocks, nodes, tensors).
+constexpr int kMaxDequantBatch = 64;
+struct DequantBatch {
+    int count;
+    long long acc_off[kMaxDequantBatch], size[kMaxDequantBatch], out_off[kMaxDequantBatch];
+    const float *s1[kMaxDequantBatch], *s2[kMaxDequantBatch];
+};
+__global__ void dequant_acc_batch_kernel(const int32_t *__restrict__ acc, DequantBatch db,
+                                         float *__restrict__ out, long long out_stride) {
+    pdl_enter();
+    const int t = blockIdx.z, n = blockIdx.y;
+    const long long size = db.size[t];
+    const float sc = __fmul_rn(db.s1[t][n], db.s2[t][n]);
+    const int32_t *a = acc + db.acc_off[t] + (long long)n * size;
+    float *o = out + (long long)n * out_stride + db.out_off[t];
+    for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < size; i += (long long)gridDim.x * blockDim.x)
+        o[i] = __fmul_rn(__int2float_rn(a[i]), sc);
+}
+
 static unsigned grid_for(int64_t n);
 
 lpdt_status dequant_acc_launch(const int32_t *acc, int nodes, int64_t per_node, const float *s1,
@@ -241,3 +263,33 @@ lpdt_status generic_bwd_weight(const lpdt_conv_desc &d, const int8_t *E, const f
 }
 
 }  // namespace lpdt
+
+extern "C" lpdt_status lpdt_dequantize_acc_batch(const int32_t *acc, int32_t nodes, int32_t n_tensors,
+                                                 const int64_t *acc_offsets, const int64_t *sizes,
+                                                 const int64_t *out_offsets, const float *const *s1,
+                                                 const float *const *s2, float *out, int64_t out_node_stride,
+                                                 void *stream) {
+    using namespace lpdt;
+    LPDT_CHECK_ARG(nodes >= 0 && n_tensors >= 0);
+    if (nodes == 0 || n_tensors == 0) return LPDT_OK;
+    LPDT_CHECK_ARG(acc && acc_offsets && sizes && out_offsets && s1 && s2 && out);
+    if (n_tensors > kMaxDequantBatch || nodes > 65535) return LPDT_ERR_UNSUPPORTED;
+    DequantBatch db;
+    db.count = n_tensors;
+    long long longest = 0;
+    for (int t = 0; t < n_tensors; ++t) {
+        LPDT_CHECK_ARG(acc_offsets[t] >= 0 && out_offsets[t] >= 0 && sizes[t] >= 0 && s1[t] && s2[t]);
+        LPDT_CHECK_ARG(out_offsets[t] + sizes[t] <= out_node_stride || nodes == 1);
+        db.acc_off[t] = acc_offsets[t]; db.size[t] = sizes[t]; db.out_off[t] = out_offsets[t];
+        db.s1[t] = s1[t]; db.s2[t] = s2[t];
+        if (sizes[t] > longest) longest = sizes[t];
+    }
+    if (longest == 0) return LPDT_OK;
+    int bx = (int)ceil_div(longest, 256 * 4);
+    if (bx > 64) bx = 64;
+    if (bx < 1) bx = 1;
+    launch_k(dequant_acc_batch_kernel, dim3(bx, nodes, n_tensors), 256, 0, as_stream(stream), acc, db, out,
+             out_node_stride);
+    LPDT_LAUNCH_CHECK();
+    return LPDT_OK;
+}

@@ -419,6 +419,32 @@ __global__ void ren_bwd_finalize(const double *__restrict__ acc, int nodes, int 
     }
 }
 
+// The same reduction for many layers in one launch: layer l owns warps [start[l], start[l+1]).
+constexpr int kMaxRenBatch = 64;
+struct RenBatch {
+    int count;
+    const double *acc[kMaxRenBatch];      // per-sample partial sums of the layer [nodes][B][3][C]
+    int C[kMaxRenBatch];
+    long long off[kMaxRenBatch];          // element offset of the layer's v gradient inside a node's gradient row
+    int start[kMaxRenBatch + 1];          // first warp of each layer
+};
+__global__ void ren_bwd_finalize_batch(RenBatch rb, int nodes, int B, float *__restrict__ grads, int64_t gstride) {
+    pdl_enter();
+    const int w = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+    if (w >= rb.start[rb.count]) return;
+    int l = 0;
+    while (w >= rb.start[l + 1]) ++l;                       // at most 64 layers: a short scan, uniform per warp
+    const int C = rb.C[l], i = w - rb.start[l];
+    const int node = i / (3 * C), j = i % (3 * C), which = j / C, c = j % C;
+    const double *a = rb.acc[l] + (int64_t)node * B * 3 * C + j;
+    double s = 0.0;
+    for (int b = lane; b < B; b += 32) s += a[(int64_t)b * 3 * C];
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_down_sync(0xffffffffu, s, o);
+    // the layer's three parameter vectors sit back to back in the gradient row: v, gamma, beta
+    if (lane == 0) grads[(int64_t)node * gstride + rb.off[l] + (int64_t)which * C + c] = (float)s;
+}
+
 struct RenPlan { int V, threads; };
 
 static bool plan(int C, int groups, bool aligned16, RenPlan *pl, int cap = 256) {
@@ -576,6 +602,31 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd_params(int32_t nodes, int32_t B, i
         return LPDT_ERR_WORKSPACE;
     launch_k(ren_bwd_finalize, (nodes * 3 * C + 7) / 8, 256, 0, as_stream(stream), (const double *)ws, nodes, B, C, dv,
              dgamma, dbeta, gstride);
+    LPDT_LAUNCH_CHECK();
+    return LPDT_OK;
+}
+
+extern "C" lpdt_status lpdt_range_evonorm_bwd_params_batch(int32_t nodes, int32_t B, int32_t n_layers, const int32_t *C,
+                                                           const void *const *ws, const int64_t *grad_offsets,
+                                                           float *grads, int64_t grad_node_stride, void *stream) {
+    LPDT_CHECK_ARG(nodes >= 0 && B >= 0 && n_layers >= 0);
+    if (nodes == 0 || B == 0 || n_layers == 0) return LPDT_OK;
+    LPDT_CHECK_ARG(C && ws && grad_offsets && grads);
+    if (n_layers > kMaxRenBatch) return LPDT_ERR_UNSUPPORTED;
+    RenBatch rb;
+    rb.count = n_layers;
+    int64_t warps = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        LPDT_CHECK_ARG(C[l] > 0 && ws[l] && aligned(ws[l], 8) && grad_offsets[l] >= 0);
+        LPDT_CHECK_ARG(grad_offsets[l] + 3 * (int64_t)C[l] <= grad_node_stride || nodes == 1);
+        rb.acc[l] = (const double *)ws[l]; rb.C[l] = C[l]; rb.off[l] = grad_offsets[l];
+        rb.start[l] = (int)warps;
+        warps += (int64_t)nodes * 3 * C[l];
+        if (warps > 0x3fffffff) return LPDT_ERR_UNSUPPORTED;
+    }
+    rb.start[n_layers] = (int)warps;
+    launch_k(ren_bwd_finalize_batch, (unsigned)ceil_div(warps, 8), 256, 0, as_stream(stream), rb, nodes, B, grads,
+             grad_node_stride);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

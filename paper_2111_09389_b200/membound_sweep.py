@@ -1,7 +1,7 @@
 """Time the memory-bound kernels of the step alone, on tensors much larger than
 L2, through the C ABI, and report achieved GB/s on their algorithmic bytes.
 
-    python -m paper_2111_09389_b200.membound_sweep [--iters 20] [--peak-gbs 6549.8]
+    python -m paper_2111_09389_b200.membound_sweep [--iters 20] [--peak-gbs 6547.2] [--only ren_bwd,quantize]
 
 Cases (activation kernels: the VGG-11-shaped workload's first layer, 8 nodes, with
 batch 128 so that each fp32 tensor is 268 MB; parameter kernels: 16 nodes with a
@@ -126,9 +126,11 @@ def cases(nodes=8, B=128, H=32, W=32, Cc=64, d=32 * 270410, gossip_nodes=16):
                                                               st), N * d * 32)
 
 
-def sweep(iters=20, peak_gbs=None, out=print):
+def sweep(iters=20, peak_gbs=None, out=print, only=None):
     rows = []
     for name, fn, nbytes in cases():
+        if only and name not in only:
+            continue
         ms = _time(fn, iters)
         row = {"case": name, "ms": ms, "algorithmic_bytes": nbytes, "gbs": nbytes / ms * 1e-6}
         if peak_gbs:
@@ -142,8 +144,9 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--peak-gbs", type=float, default=None, help="HBM copy bandwidth to report fractions against")
+    ap.add_argument("--only", default=None, help="comma-separated case names to run")
     a = ap.parse_args()
-    sweep(a.iters, a.peak_gbs)
+    sweep(a.iters, a.peak_gbs, only=a.only.split(",") if a.only else None)
 
 
 if __name__ == "__main__":

@@ -17,7 +17,8 @@ from . import api
 class TrainStep:
     def __init__(self, ops, d, nodes, batch, in_shape, ren_eps=1e-5, lr=0.1, gamma=1.0,
                  seg_offsets=None, seg_k=None, has_labels=True, grad_rounding=0, seed=0,
-                 quantize_wgrad=False, input_grad=False, message_bits=32, device="cuda"):
+                 quantize_wgrad=False, input_grad=False, message_bits=32, recompute_norm_input=False,
+                 device="cuda"):
         if not torch.cuda.is_available():
             raise RuntimeError("TrainStep needs a CUDA device; there is no CPU path")
         self.ops, self.d, self.N, self.B = ops, d, nodes, batch
@@ -27,6 +28,12 @@ class TrainStep:
         self.grad_rounding, self.seed = grad_rounding, seed
         self.quantize_wgrad, self.input_grad = quantize_wgrad, input_grad
         self.message_bits = message_bits          # 8: gossip messages as 8-bit codes with one range per (node, segment)
+        # True: nothing but 8-bit tensors (and the small norm statistics) is kept from the forward to the
+        # backward pass.  The fp32 input of every Range-EvoNorm layer, i.e. the output of the convolution
+        # before it, is not stored per layer; the backward pass recomputes it from the saved 8-bit operands
+        # into one shared buffer (same integer sums, same dequantization: bit-identical values).
+        self.recompute_norm_input = recompute_norm_input
+        self._shared_out = {}
         dev = torch.device(device)
         N, B = nodes, batch
         f32 = dict(dtype=torch.float32, device=dev)
@@ -56,6 +63,13 @@ class TrainStep:
             self.w_src.append(op["w_off"]); self.w_size.append(wn); self.w_dst.append(qbytes)
             qbytes += (N * wn + 255) // 256 * 256
         self.qW_all = torch.empty(max(qbytes, 256), **i8)
+        # raw int32 weight-gradient sums of every layer, each a contiguous [nodes][size] block (256-byte aligned
+        # starts): converted to fp32 by one batched launch at the end of the backward pass
+        self.g_acc_off, n_acc = [], 0
+        for wn in self.w_size:
+            self.g_acc_off.append(n_acc)
+            n_acc += (N * wn + 63) // 64 * 64
+        self.g_acc = torch.empty(max(n_acc, 64), **i32)
         self.sW_all = torch.empty(max(len(wlist), 1), N, **f32)
         ws_bytes = max(ws_bytes, api.lpdt_quantize_batch_workspace_size(N, min(len(wlist), 64)))
         wi = 0
@@ -74,10 +88,10 @@ class TrainStep:
                          qA=torch.empty(N, B, H, W, op["cin"], **i8), sA=torch.empty(N, **f32),
                          qW=self.qW_all[self.w_dst[wi]:self.w_dst[wi] + N * self.w_size[wi]].view(N, op["cout"], R, S, op["cin"]),
                          sW=self.sW_all[wi],
-                         out=torch.empty(N, B, Ho, Wo, op["cout"], **f32),
+                         out=self._conv_out((N, B, Ho, Wo, op["cout"]), f32),
                          E=torch.empty(N, B, Ho, Wo, op["cout"], **i8), sE=torch.empty(N, **f32),
                          dx=torch.empty(N, B, H, W, op["cin"], **f32),
-                         wn=op["cout"] * R * S * op["cin"])
+                         wn=op["cout"] * R * S * op["cin"], wi=wi)
                 if quantize_wgrad:
                     b.update(gq=torch.empty(N, b["wn"], **i8), gs=torch.empty(N, **f32),
                              gw=torch.empty(N, b["wn"], **f32))
@@ -123,6 +137,33 @@ class TrainStep:
         # parameter update.  Captured into the step's CUDA graph the fork and join become graph edges.
         self.ws_side = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
         self.side = torch.cuda.Stream(device=dev)
+
+    def _conv_out(self, shape, f32):
+        """fp32 output buffer of a convolution: one per layer, or (recompute_norm_input) one per distinct
+        shape shared by all layers of that shape, since no layer's output has to outlive its consumers."""
+        if not self.recompute_norm_input:
+            return torch.empty(*shape, **f32)
+        if shape not in self._shared_out:
+            self._shared_out[shape] = torch.empty(*shape, **f32)
+        return self._shared_out[shape]
+
+    def saved_bytes_per_node(self):
+        """Bytes one node keeps from its forward pass for its backward pass, by kind."""
+        N = self.N
+        rep = {"int8_activations": 0, "int8_weights": 0, "fp32_norm_inputs": 0, "norm_statistics": 0, "pool_indices": 0}
+        for op, b in zip(self.ops, self.buf):
+            k = op["op"]
+            if k in ("conv", "linear"):
+                rep["int8_activations"] += b["qA"].numel() // N
+                rep["int8_weights"] += b["qW"].numel() // N
+            elif k == "ren":
+                if not self.recompute_norm_input:
+                    rep["fp32_norm_inputs"] += 4 * self.B * op["H"] * op["W"] * op["C"]
+                rep["norm_statistics"] += 4 * 4 * self.B * op["groups"]
+            elif k == "maxpool":
+                rep["pool_indices"] += b["idx"].numel() // N
+        rep["total"] = sum(rep.values())
+        return rep
 
     # ---- host -> device ------------------------------------------------------------
     def load(self, wl):
@@ -205,6 +246,7 @@ class TrainStep:
             elif k == "ren":
                 Cc = op["C"]
                 b["x"] = cur
+                b["x_from"] = li - 1 if (li > 0 and self.ops[li - 1]["op"] in ("conv", "linear")) else None
                 # an identity shortcut right after this layer is added inside the kernel
                 nxt = self.ops[li + 1] if li + 1 < len(self.ops) else None
                 fuse = nxt is not None and nxt["op"] == "add" and nxt["stride"] == 1 and nxt["Ca"] == nxt["C"]
@@ -263,15 +305,16 @@ class TrainStep:
                 main = torch.cuda.current_stream()
                 self.side.wait_stream(main)               # E (and, at the first use, everything before) is ready
                 with torch.cuda.stream(self.side):
-                    self._ren_param_sums(pending_ren)
                     if self.quantize_wgrad:
                         api.lpdt_qconv_bwd_weight(b["desc"], b["E"], b["sE"], b["qA"], b["sA"], dW=b["gw"],
                                                   dw_node_stride=b["wn"], ws=self.ws_side, dev_status=self.dev_status)
                         api.lpdt_quantize(b["gw"], N, b["wn"], b["wn"], b["gq"], b["gs"], self.ws_side)
                         api.lpdt_dequantize(b["gq"], N, b["wn"], b["gs"], self._g(op["w_off"]), d)
                     else:
+                        # raw sums now, one conversion launch for all layers after the last of them
+                        lo = self.g_acc_off[b["wi"]]
                         api.lpdt_qconv_bwd_weight(b["desc"], b["E"], b["sE"], b["qA"], b["sA"],
-                                                  dW=self._g(op["w_off"]), dw_node_stride=d, ws=self.ws_side,
+                                                  dWacc=self.g_acc[lo:lo + N * b["wn"]], ws=self.ws_side,
                                                   dev_status=self.dev_status)
                 if li > 0 or self.input_grad:
                     # first convolution of a residual block with an identity shortcut: the block-output gradient
@@ -290,6 +333,12 @@ class TrainStep:
                     g = None
             elif k == "ren":
                 Cc = op["C"]
+                if self.recompute_norm_input and b["x_from"] is not None:
+                    # the layer's input again, from the convolution's saved 8-bit operands into the shared buffer
+                    cb, cop = self.buf[b["x_from"]], self.ops[b["x_from"]]
+                    api.lpdt_qconv_fwd(cb["desc"], cb["qA"], cb["sA"], cb["qW"], cb["sW"], Y=cb["out"],
+                                       bias=self._p(cop["b_off"]) if cop["op"] == "linear" else None,
+                                       bias_node_stride=d, ws=self.ws, dev_status=self.dev_status)
                 # dx only; the parameter-gradient sums stay as partial sums and are reduced on the side stream
                 api.lpdt_range_evonorm_bwd(N, B, op["H"], op["W"], Cc, op["groups"], self.eps, g, b["x"],
                                            self._p(op["p_off"]), self._p(op["p_off"] + Cc), d, b["gmin"],
@@ -313,20 +362,31 @@ class TrainStep:
             elif k == "avgpool":
                 api.lpdt_avgpool_bwd(N, B, op["H"] * op["W"], op["C"], g, b["dx"])
                 g, g_range = b["dx"], None
-        if pending_ren:                                         # a norm layer with no convolution below it
-            self.side.wait_stream(torch.cuda.current_stream())
-            with torch.cuda.stream(self.side):
-                self._ren_param_sums(pending_ren)
+        # side stream, after the last weight-gradient contraction: all norm layers' parameter-gradient sums in one
+        # launch, all layers' int32 weight-gradient sums to fp32 in another
+        self.side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.stream(self.side):
+            self._ren_param_sums(pending_ren)
+            if not self.quantize_wgrad:
+                convs = [(op, b) for op, b in zip(self.ops, self.buf) if op["op"] in ("conv", "linear")]
+                for lo in range(0, len(convs), 64):
+                    part = convs[lo:lo + 64]
+                    api.lpdt_dequantize_acc_batch(self.g_acc, N, [self.g_acc_off[b["wi"]] for _, b in part],
+                                                  [b["wn"] for _, b in part], [op["w_off"] for op, _ in part],
+                                                  [b["sE"] for _, b in part], [b["sA"] for _, b in part],
+                                                  self.grads, d)
         torch.cuda.current_stream().wait_stream(self.side)      # weight gradients complete before the update
         self.input_grad_out = g
         return g
 
     def _ren_param_sums(self, pending):
-        """Reduce the Range-EvoNorm parameter-gradient partial sums of the layers in `pending` (current stream)."""
-        for op, b in pending:
-            Cc = op["C"]
-            api.lpdt_range_evonorm_bwd_params(self.N, self.B, Cc, b["ws_ren"], self._g(op["p_off"]),
-                                              self._g(op["p_off"] + Cc), self._g(op["p_off"] + 2 * Cc), self.d)
+        """Reduce the Range-EvoNorm parameter-gradient partial sums of the layers in `pending` (current stream):
+        one launch per 64 layers."""
+        for lo in range(0, len(pending), 64):
+            part = pending[lo:lo + 64]
+            api.lpdt_range_evonorm_bwd_params_batch(self.N, self.B, [op["C"] for op, _ in part],
+                                                    [b["ws_ren"] for _, b in part], [op["p_off"] for op, _ in part],
+                                                    self.grads, self.d)
         pending.clear()
 
     def update(self):

@@ -856,6 +856,45 @@ def test_bounded_wait_runs_out_and_reports():
     assert np.array_equal(q.cpu().numpy(), q_ref) and np.array_equal(s.cpu().numpy(), s_ref)
 
 
+def test_batched_reductions_equal_the_single_calls():
+    """lpdt_range_evonorm_bwd_params_batch and lpdt_dequantize_acc_batch: many layers in one launch, bit-identical
+    to the per-layer calls (which the tests above compare with the oracle)."""
+    rng = np.random.default_rng(12)
+    nodes, B = 3, 5
+    layers = [(8, 8, 16, 4), (4, 4, 64, 8), (6, 5, 12, 3)]                   # H, W, C, groups
+    stride = sum(3 * c for _, _, c, _ in layers) + 11
+    G1 = torch.zeros(nodes, stride, device="cuda"); G2 = torch.zeros_like(G1)
+    wss, offs, off = [], [], 3
+    for H, W, C, groups in layers:
+        x, P, dy = _ren_inputs((nodes, B, H, W, C, groups), seed=C)
+        Pd, xd = dev(P), dev(x)
+        f = lambda *sh: torch.empty(*sh, dtype=torch.float32, device="cuda")
+        i = lambda *sh: torch.empty(*sh, dtype=torch.int32, device="cuda")
+        y, gmin, gmax, amn, amx = f(*x.shape), f(nodes, B, groups), f(nodes, B, groups), i(nodes, B, groups), i(nodes, B, groups)
+        api.lpdt_range_evonorm_fwd(nodes, B, H, W, C, groups, 1e-5, xd, Pd, Pd[:, C:], Pd[:, 2 * C:], P.shape[1], y, gmin,
+                                   gmax, amn, amx)
+        ws = ws_bytes(api.lpdt_range_evonorm_bwd_workspace_size(nodes, B, C))
+        api.lpdt_range_evonorm_bwd(nodes, B, H, W, C, groups, 1e-5, dev(dy), xd, Pd, Pd[:, C:], P.shape[1], gmin, gmax, amn,
+                                   amx, f(*x.shape), None, None, None, stride, ws)
+        api.lpdt_range_evonorm_bwd_params(nodes, B, C, ws, G1[:, off:], G1[:, off + C:], G1[:, off + 2 * C:], stride)
+        wss.append(ws); offs.append(off)
+        off += 3 * C
+    api.lpdt_range_evonorm_bwd_params_batch(nodes, B, [c for _, _, c, _ in layers], wss, offs, G2, stride)
+    assert torch.equal(G1, G2) and G1.abs().sum() > 0
+    # int32 sums of three tensors, each a contiguous [nodes][size] block, into one strided fp32 row per node
+    sizes, acc_off, out_off = [432, 1000, 7], [0, 64 * 21, 64 * 21 + 64 * 47], [5, 600, 1700]
+    acc = torch.from_numpy(rng.integers(-2 ** 31, 2 ** 31 - 1, 64 * 21 + 64 * 47 + 64, dtype=np.int64).astype(np.int32)).cuda()
+    s1 = [dev(rng.uniform(0.001, 0.1, nodes).astype(np.float32)) for _ in sizes]
+    s2 = [dev(rng.uniform(0.001, 0.1, nodes).astype(np.float32)) for _ in sizes]
+    out = torch.zeros(nodes, 1800, device="cuda")
+    api.lpdt_dequantize_acc_batch(acc, nodes, acc_off, sizes, out_off, s1, s2, out, 1800)
+    want = np.zeros((nodes, 1800), np.float32)
+    for t, n in enumerate(sizes):
+        a = acc[acc_off[t]:acc_off[t] + nodes * n].cpu().numpy().reshape(nodes, 1, n)
+        want[:, out_off[t]:out_off[t] + n] = oracle.dequant_acc(a, s1[t].cpu().numpy(), s2[t].cpu().numpy()).reshape(nodes, n)
+    assert np.array_equal(out.cpu().numpy(), want)
+
+
 @pytest.mark.parametrize("cluster", ["1", "2", "8"])
 def test_range_evonorm_cases_on_every_cluster_size(cluster):
     """The forward kernel splits a sample over 1-8 CTAs by a size rule; the cases are re-run in child

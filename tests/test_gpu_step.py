@@ -213,3 +213,25 @@ def test_step_with_8bit_messages(name, kw):
         tight = err <= 1e-6 + 1e-5 * np.abs(want)
         assert (err <= 1.001 * step[:, None] + 1e-6).all(), what        # never more than one code step (x: a mix of steps)
         assert (~tight).mean() < 2e-3, f"{what}: {(~tight).sum()} entries off by a code step"
+
+
+@pytest.mark.parametrize("name,nodes,batch", [("resnet20", 3, 4), ("vgg11", 2, 2), ("resnet20_topk", 5, 2)])
+def test_step_keeping_only_8bit_tensors_for_backward(name, nodes, batch):
+    """recompute_norm_input: the fp32 inputs of the norm layers are not kept per layer but recomputed in the
+    backward pass from the saved 8-bit operands.  Same integer sums and the same dequantization, so every
+    result of the step is bit-identical to the default mode (which is compared with the oracle above), and
+    what a node keeps between the passes shrinks to its 8-bit tensors and the norm statistics."""
+    wl = wlmod.make_workload(name, nodes=nodes, batch=batch)
+    a = TrainStep.from_workload(wl)
+    b = TrainStep.from_workload(wl, recompute_norm_input=True)
+    a.run(); b.run()
+    torch.cuda.synchronize()
+    assert int(b.dev_status.item()) == 0
+    for t in ("grads", "x_half", "x_hat", "x_out", "loss"):
+        assert torch.equal(getattr(a, t), getattr(b, t)), t
+    for li, op in enumerate(wl["ops"]):
+        if op["op"] in ("conv", "linear"):
+            assert torch.equal(a.buf[li]["E"], b.buf[li]["E"]), f"E{li}"
+    ma, mb = a.saved_bytes_per_node(), b.saved_bytes_per_node()
+    assert mb["fp32_norm_inputs"] == 0 and ma["fp32_norm_inputs"] > 0
+    assert mb["int8_activations"] == ma["int8_activations"] and mb["total"] < ma["total"]
