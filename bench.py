@@ -239,10 +239,10 @@ def time_group(calls, reps):
     recorded into one CUDA graph and replayed `reps` times between two events on the current stream."""
     import torch
     from paper_2111_09389_b200 import api
-    before = api.KERNEL_LAUNCHES
+    before = api.lpdt_launch_count()
     for _, fn, a, kw, _ in calls:
         fn(*a, **kw)
-    time_group.launches = api.KERNEL_LAUNCHES - before       # kernels one issue of `calls` enqueues
+    time_group.launches = api.lpdt_launch_count() - before       # kernels one issue of `calls` enqueues
     torch.cuda.synchronize()
     g = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g):
@@ -377,7 +377,7 @@ def run_step_workload(name, rank, world, steps, warmup, graph=True, **step_optio
     for _ in range(warmup):
         step()
     barrier(world)
-    launches0 = api.KERNEL_LAUNCHES
+    launches0 = api.lpdt_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier(world)
     e0.record()
@@ -387,7 +387,7 @@ def run_step_workload(name, rank, world, steps, warmup, graph=True, **step_optio
     torch.cuda.synchronize()
     barrier(world)
     ms_total = max_over_ranks(world, e0.elapsed_time(e1))
-    launches = api.KERNEL_LAUNCHES - launches0
+    launches = api.lpdt_launch_count() - launches0
     assert int(st.dev_status.item()) == 0
 
     # end to end: inputs start in pinned host memory, the loss is read back every step; the upload of the

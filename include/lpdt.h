@@ -67,6 +67,9 @@ const char *lpdt_status_string(lpdt_status s);
  * a CUDA-core kernel.  For labelling timings; the choice depends on the shape, the alignment and on which
  * outputs were asked for. */
 const char *lpdt_last_kernel(void);
+/* Number of kernels the calling host thread has enqueued through this library so far (memsets and
+ * copies not counted; a launch recorded during stream capture counts once, its replays do not). */
+uint64_t lpdt_launch_count(void);
 /* Enqueue a zero fill of `bytes` bytes at device pointer p (range accumulators, status words). */
 lpdt_status lpdt_fill_zero(void *p, size_t bytes, void *stream);
 /* Read a status word back: waits until everything enqueued on `stream` so far has finished (the one

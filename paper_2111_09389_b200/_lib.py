@@ -22,6 +22,7 @@ SIGNATURES = {
     "lpdt_version": (C.c_char_p, []),
     "lpdt_status_string": (C.c_char_p, [_i32]),
     "lpdt_last_kernel": (C.c_char_p, []),
+    "lpdt_launch_count": (_u64, []),
     "lpdt_fill_zero": (_i32, [_vp, _sz, _vp]),
     "lpdt_check_status": (_i32, [_vp, _vp]),
     "lpdt_selftest_bounded_wait": (_i32, [_u64, _vp, _vp, _vp]),

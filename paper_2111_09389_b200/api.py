@@ -11,15 +11,22 @@ import torch
 from ._lib import ConvDesc, lib
 
 
-# Kernels each entry point enqueues (memsets not counted); KERNEL_LAUNCHES accumulates them.
-KERNELS_PER_CALL = {
-    "lpdt_quantize": 2, "lpdt_quantize_with_range": 1, "lpdt_quantize_static": 2, "lpdt_quantize_batch": 2, "lpdt_dequantize": 1, "lpdt_qconv_fwd": 1, "lpdt_qconv_fwd_affine": 4, "lpdt_qconv_bwd_data_affine": 4, "lpdt_qconv_bwd_weight_affine": 7, "lpdt_qconv_bwd_data": 2,
-    "lpdt_qconv_bwd_weight": 2, "lpdt_range_evonorm_fwd": 1, "lpdt_range_evonorm_bwd": 2, "lpdt_range_evonorm_bwd_params": 1, "lpdt_range_evonorm_bwd_params_batch": 1, "lpdt_dequantize_acc_batch": 1,
-    "lpdt_gossip_mix": 2, "lpdt_gossip_mix_q8": 3, "lpdt_deepsqueeze_mix": 2, "lpdt_pushsum_debias": 1, "lpdt_sgd_gossip_mix": 1, "lpdt_evonorm_s0_fwd": 1, "lpdt_evonorm_s0_bwd": 2, "lpdt_range_bn_fwd": 2, "lpdt_range_bn_bwd": 2, "lpdt_sgd_update": 1, "lpdt_residual_add": 1, "lpdt_residual_add_bwd": 1,
-    "lpdt_avgpool": 1, "lpdt_avgpool_bwd": 1, "lpdt_maxpool2x2": 1, "lpdt_maxpool2x2_bwd": 1,
-    "lpdt_softmax_ce": 1, "lpdt_colsum": 1, "lpdt_selftest_bounded_wait": 1,
-}
-KERNEL_LAUNCHES = 0
+# Entry points that enqueue kernels (wrapped for the optional call log and per-call timing).
+LAUNCHING = {"lpdt_quantize", "lpdt_quantize_with_range", "lpdt_quantize_static", "lpdt_quantize_batch", "lpdt_dequantize", "lpdt_qconv_fwd", "lpdt_qconv_fwd_affine", "lpdt_qconv_bwd_data_affine", "lpdt_qconv_bwd_weight_affine", "lpdt_qconv_bwd_data", "lpdt_qconv_bwd_weight", "lpdt_range_evonorm_fwd", "lpdt_range_evonorm_bwd", "lpdt_range_evonorm_bwd_params", "lpdt_range_evonorm_bwd_params_batch", "lpdt_dequantize_acc_batch", "lpdt_gossip_mix", "lpdt_gossip_mix_q8", "lpdt_deepsqueeze_mix", "lpdt_pushsum_debias", "lpdt_sgd_gossip_mix", "lpdt_evonorm_s0_fwd", "lpdt_evonorm_s0_bwd", "lpdt_range_bn_fwd", "lpdt_range_bn_bwd", "lpdt_sgd_update", "lpdt_residual_add", "lpdt_residual_add_bwd", "lpdt_avgpool", "lpdt_avgpool_bwd", "lpdt_maxpool2x2", "lpdt_maxpool2x2_bwd", "lpdt_softmax_ce", "lpdt_colsum", "lpdt_selftest_bounded_wait"}
+# Kernel launches are counted inside the library (lpdt_launch_count); replays of a captured CUDA graph launch
+# the recorded kernels again without passing through the library, so TrainStep.replay adds them here.
+_REPLAYED = 0
+
+
+def lpdt_launch_count():
+    """Kernels enqueued by this thread through the library, plus those of graph replays."""
+    return int(lib().lpdt_launch_count()) + _REPLAYED
+
+
+def add_replayed_launches(n):
+    global _REPLAYED
+    _REPLAYED += int(n)
+
 # Optional per-entry-point timing: {name: [(start_event, end_event), ...]} when TIMED holds names.
 TIMED = set()
 TIMINGS = {}
@@ -32,10 +39,8 @@ class LpdtError(RuntimeError):
 
 
 def _check(fn, code):
-    global KERNEL_LAUNCHES
     if code != 0:
         raise LpdtError(fn, code)
-    KERNEL_LAUNCHES += KERNELS_PER_CALL.get(fn, 0)
 
 
 def timed(name):
@@ -224,9 +229,6 @@ def lpdt_qconv_bwd_weight(desc, E, sE, A, sA, dW=None, dw_node_stride=0, dWacc=N
                                                                 _ptr(sA), _ptr(dW), dw_node_stride,
                                                                 _ptr(dWacc), p, nb, _ptr(dev_status),
                                                                 _stream()))
-    if dW is None:                      # raw sums only: no conversion launch
-        global KERNEL_LAUNCHES
-        KERNEL_LAUNCHES -= 1
 
 
 def lpdt_range_evonorm_fwd(nodes, B, H, W, Cc, groups, eps, x, v, gamma, beta, param_node_stride, y,
@@ -247,9 +249,6 @@ def lpdt_range_evonorm_bwd(nodes, B, H, W, Cc, groups, eps, dy, x, v, gamma, par
         nodes, B, H, W, Cc, groups, eps, _ptr(dy), _ptr(x), _ptr(v), _ptr(gamma), param_node_stride,
         _ptr(gmin), _ptr(gmax), _ptr(argmin), _ptr(argmax), _ptr(dx), _ptr(dv), _ptr(dgamma), _ptr(dbeta),
         grad_node_stride, _ptr(amax_out), p, nb, _stream()))
-    if dv is None:                      # dx only: the reduction launch belongs to lpdt_range_evonorm_bwd_params
-        global KERNEL_LAUNCHES
-        KERNEL_LAUNCHES -= 1
 
 
 def lpdt_evonorm_s0_fwd(nodes, B, H, W, Cc, groups, eps, x, v, gamma, beta, param_node_stride, y, gmean, gvar):
@@ -437,6 +436,6 @@ def _with_timing(fn):
     return call
 
 
-for _n in [n for n in list(globals()) if n.startswith("lpdt_") and (n in KERNELS_PER_CALL or n == "lpdt_fill_zero")]:
+for _n in [n for n in list(globals()) if n in LAUNCHING or n == "lpdt_fill_zero"]:
     globals()[_n] = _with_timing(globals()[_n])
 del _n

@@ -4,6 +4,7 @@
 extern "C" const char *lpdt_version(void) { return "lpdt 0.1 (sm_100a)"; }
 
 extern "C" const char *lpdt_last_kernel(void) { return lpdt::g_last_kernel; }
+extern "C" uint64_t lpdt_launch_count(void) { return lpdt::g_launch_count; }
 
 extern "C" lpdt_status lpdt_fill_zero(void *p, size_t bytes, void *stream) {
     if (bytes == 0) return LPDT_OK;

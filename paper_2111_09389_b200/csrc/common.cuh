@@ -36,6 +36,8 @@ constexpr int kNumSMs = 148;  // B200
 // Name of the contraction kernel the calling host thread launched last (lpdt_last_kernel): lets a
 // caller that times a call label the number with the kernel that actually ran.
 inline thread_local const char *g_last_kernel = "";
+// Kernels the calling host thread has enqueued through this library so far (lpdt_launch_count).
+inline thread_local unsigned long long g_launch_count = 0;
 
 // A kernel attribute (the opt-in dynamic shared memory limit) belongs to the device it was set on, so
 // "already set" is remembered per device ordinal: one bit per device, devices beyond 63 set it every call.
@@ -79,6 +81,7 @@ static inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 blo
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    ++g_launch_count;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<Args &&>(args)...);
 }
 
@@ -102,6 +105,7 @@ static inline cudaError_t launch_k_cluster(void (*kernel)(KArgs...), dim3 grid, 
     }
     cfg.attrs = attr;
     cfg.numAttrs = n;
+    ++g_launch_count;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<Args &&>(args)...);
 }
 

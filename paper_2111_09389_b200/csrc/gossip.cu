@@ -116,7 +116,10 @@ __device__ uint32_t radix_select(int64_t n, KeyFn key, long long need, int free_
         for (int i = threadIdx.x; i < 256; i += blockDim.x) hist[i] = 0;
         __syncthreads();
         const uint32_t prefix = s_prefix, mask = s_mask;
-        // uniform trip count (the warp votes below need every lane); eight independent loads per thread
+        // eight independent loads per thread.  Consecutive hits of a thread that fall into the same bin are
+        // counted in a register and added once: in the first passes one or two bins (the common exponents)
+        // take nearly every key, and per-key atomics would queue up on those few shared-memory words.
+        uint32_t run_bin = 0; unsigned run_cnt = 0;
         for (int64_t base = 0; base < n; base += 8 * (int64_t)blockDim.x) {
             uint32_t k[8];
 #pragma unroll
@@ -128,19 +131,14 @@ __device__ uint32_t radix_select(int64_t n, KeyFn key, long long need, int free_
             for (int u = 0; u < 8; ++u) {
                 const int64_t eu = base + u * (int64_t)blockDim.x + threadIdx.x;
                 const bool hit = eu < n && !(SKIP_ZERO && k[u] == 0u) && (k[u] & mask) == prefix;
+                if (!hit) continue;
                 const uint32_t bin = (k[u] >> shift) & dmask;
-                // a warp whose hits all fall into one bin (constant data, shared leading bits) adds once
-                const unsigned hits = __ballot_sync(0xffffffffu, hit);
-                if (hits == 0u) continue;
-                const int leader = __ffs(hits) - 1;
-                const uint32_t lbin = __shfl_sync(0xffffffffu, bin, leader);
-                if (__all_sync(0xffffffffu, !hit || bin == lbin)) {
-                    if (lane == leader) atomicAdd(&hist[lbin], (unsigned)__popc(hits));
-                } else if (hit) {
-                    atomicAdd(&hist[bin], 1u);
-                }
+                if (run_cnt && bin == run_bin) { ++run_cnt; continue; }
+                if (run_cnt) atomicAdd(&hist[run_bin], run_cnt);
+                run_bin = bin; run_cnt = 1;
             }
         }
+        if (run_cnt) atomicAdd(&hist[run_bin], run_cnt);
         __syncthreads();
         if (threadIdx.x < 32) {
             // bucket of the need-th largest key: lane l owns bins [8l, 8l+8); suffix sums across lanes by shuffles
@@ -190,14 +188,16 @@ __device__ void select_whole_segment(const float *__restrict__ xh, const float *
     if (threadIdx.x == 0) { o->thr = thr; o->dense = 0; o->cut = cut; }
 }
 
-// ---- long segments: two streaming passes spread over many CTAs ------------------------------
-// Pass 1 (big_hist_kernel) builds, per (node, segment), a histogram of the top 12 magnitude bits
-// (exponent and four mantissa bits: buckets 1/16 of an octave wide); the CTA that finishes last walks it and records the bucket
-// that holds the k-th largest key.  Pass 2 (big_collect_kernel) copies the keys of that bucket with
-// their positions into a candidate list.  The select launch then finds the threshold and the tie
-// cut among the candidates alone (one CTA per segment, a few per cent of the data at most).  A
-// bucket that outgrows the list (1/8 of the segment; a Gaussian's fullest bucket holds 3 %, a uniform
-// distribution's 6 %: only near-constant magnitudes get there) falls back to the whole-segment path.
+// ---- long segments: a sampled threshold, one streaming pass, a selection over the candidates ----
+// Sample (big_sample_kernel): 1/64 of the segment, read as runs of eight consecutive parameters, goes into
+// a histogram of the top 12 magnitude bits (exponent and four mantissa bits: buckets 1/16 of an octave
+// wide); the CTA that finishes last walks it from the top and picks a bucket that, by the sample, has
+// comfortably more than k keys at or above it.  Collect (big_collect_kernel): the one pass over the
+// segment copies every key at or above that bucket, with its position, into a candidate list and counts
+// them exactly.  Select (one CTA per segment): if the exact count reached k, the k largest keys are all
+// in the list, and the threshold and the tie cut are found there (1-2 % of the data).  The sample only
+// steers: when the count falls short of k, or the candidates outgrow the list (1/8 of the segment: near-
+// constant magnitudes), the exact whole-segment path takes over, so the result never depends on the sample.
 struct BigList {
     int32_t n;
     int32_t id[kMaxSeg];               // segment index
@@ -205,8 +205,8 @@ struct BigList {
     int64_t cand_base[kMaxSeg + 1];    // prefix sums of the candidate capacities
 };
 constexpr int kTopBins = 4096;
-struct BigCtl { uint32_t h0[kTopBins]; uint32_t ticket, cand_count; };   // zeroed per call
-struct BigState { uint32_t prefix; uint32_t overflow; long long need, eq; };   // chosen bucket; keys still to take in it; its population
+struct BigCtl { uint32_t h0[kTopBins]; uint32_t ticket, cand_count, sampled, pad; };   // zeroed per call; cand_count: keys at or above the bucket
+struct BigState { uint32_t prefix; uint32_t sampled; };    // lowest magnitude bits of the chosen bucket; keys sampled
 struct __align__(8) Cand { uint32_t key, pos; };    // magnitude bits, position inside the segment
 
 __device__ __host__ __forceinline__ int64_t cand_capacity(int64_t len) { return len / 8 + 4096; }
@@ -248,58 +248,74 @@ __device__ void pick_bucket(const uint32_t *hist, int nbins, long long need, int
 }
 
 constexpr int kTopShift = 19;          // the histogram keys on magnitude bits 30..19
+__device__ __forceinline__ int64_t ceil_div_dev(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+constexpr int kSampleRun = 8;                 // consecutive parameters per sampled run
+constexpr int kSampleEvery = 64;              // one run per kSampleRun * kSampleEvery parameters
+constexpr int64_t kSampleChunk = 1 << 17;     // parameters per CTA of the sample launch: eight runs per group of eight threads
 
 __global__ void __launch_bounds__(256)
-big_hist_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d, SegTable seg,
-                BigList big, BigCtl *__restrict__ ctl, BigState *__restrict__ state) {
+big_sample_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d, SegTable seg,
+                  BigList big, BigCtl *__restrict__ ctl, BigState *__restrict__ state) {
     pdl_enter();
     const int bi = blockIdx.y, node = blockIdx.z, s = big.id[bi], plus = seg.plus;
     const int64_t lo = seg.off[s], hi = seg.off[s + 1];
-    const int64_t c0 = lo + (int64_t)blockIdx.x * kChunk;
+    const int64_t c0 = lo + (int64_t)blockIdx.x * kSampleChunk;
     if (c0 >= hi) return;
-    const int64_t c1 = (c0 + kChunk < hi) ? c0 + kChunk : hi;
+    const int64_t c1 = (c0 + kSampleChunk < hi) ? c0 + kSampleChunk : hi;
     BigCtl *h = ctl + (int64_t)node * big.n + bi;
     const float *xh = x_half + (int64_t)node * d, *xq = x_hat + (int64_t)node * d;
     __shared__ unsigned int sh[kTopBins];
-    __shared__ unsigned int s_ticket;
+    __shared__ unsigned int s_ticket, s_taken;
     for (int i = threadIdx.x; i < kTopBins; i += blockDim.x) sh[i] = 0;
+    if (threadIdx.x == 0) s_taken = 0;
     __syncthreads();
-    for (int64_t e = c0 + threadIdx.x; e < c1; e += 4 * blockDim.x) {      // eight loads in flight per thread
-        float a[4], b[4];
+    // thread t of a group of eight reads parameter t of a run: 32 contiguous bytes per run and array
+    const int64_t span = (int64_t)kSampleRun * kSampleEvery;
+    unsigned taken = 0;
+    const int64_t r0 = c0 + (int64_t)(threadIdx.x / kSampleRun) * span + (threadIdx.x % kSampleRun);
+    const int64_t rstep = (int64_t)(blockDim.x / kSampleRun) * span;
+    constexpr int kU = (int)(kSampleChunk / ((256 / kSampleRun) * kSampleRun * kSampleEvery));     // runs per thread group
+    float va[kU], vb[kU];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int64_t eu = e + u * blockDim.x;
-            if (eu < c1) { a[u] = xh[eu]; b[u] = xq[eu]; }
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u)
-            if (e + u * blockDim.x < c1) atomicAdd(&sh[mag_bits(a[u], b[u], plus) >> kTopShift], 1u);
+    for (int u = 0; u < kU; ++u) {                   // every load of the thread in flight at once
+        const int64_t e = r0 + u * rstep;
+        if (e < c1) { va[u] = xh[e]; vb[u] = xq[e]; }
     }
+#pragma unroll
+    for (int u = 0; u < kU; ++u)
+        if (r0 + u * rstep < c1) { atomicAdd(&sh[mag_bits(va[u], vb[u], plus) >> kTopShift], 1u); ++taken; }
+    atomicAdd(&s_taken, taken);
     __syncthreads();
     for (int i = threadIdx.x; i < kTopBins; i += blockDim.x)
         if (sh[i]) atomicAdd(&h->h0[i], sh[i]);
+    if (threadIdx.x == 0) atomicAdd(&h->sampled, s_taken);
     // last CTA of this (node, segment): every chunk's counts have landed
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) s_ticket = atomicAdd(&h->ticket, 1u);
     __syncthreads();
-    const unsigned nchunks = (unsigned)(big.chunk_base[bi + 1] - big.chunk_base[bi]);
+    const unsigned nchunks = (unsigned)ceil_div_dev(hi - lo, kSampleChunk);
     if (s_ticket != nchunks - 1) return;
     __threadfence();
-    int b; long long need, eq;
-    pick_bucket(h->h0, kTopBins, seg.k[s], &b, &need, &eq);
+    // keys the sample must show at or above the bucket: the sampled share of k, a quarter more, and four
+    // standard deviations of the sampled count
+    const double m = (double)__ldcg(&h->sampled), f = m / (double)(hi - lo), fk = f * (double)seg.k[s];
+    long long target = (long long)(1.25 * fk + 4.0 * sqrt(fk) + 8.0);
+    int b = 0; long long need, eq;
+    if (target <= (long long)m) pick_bucket(h->h0, kTopBins, target, &b, &need, &eq);
     if (threadIdx.x == 0) {
         BigState nx;
         nx.prefix = (uint32_t)b << kTopShift;
-        nx.overflow = eq > cand_capacity(hi - lo) ? 1u : 0u;
-        nx.need = need; nx.eq = eq;
+        nx.sampled = (uint32_t)m;
         state[(int64_t)node * big.n + bi] = nx;
     }
 }
 
-// Copy the keys of the chosen bucket, with their positions, into the (node, segment)'s candidate
-// list.  Matches are staged in shared memory and flushed with one reservation per CTA; the order
-// inside the list is arbitrary (the selection over it does not depend on it).
+// Copy every key at or above the chosen bucket, with its position, into the (node, segment)'s candidate
+// list, and count them all (the count keeps running past the list's capacity; writes stop there).
+// Matches are staged in shared memory and flushed with one reservation per CTA; the order inside the
+// list is arbitrary (the selection over it does not depend on it).
 constexpr int kStage = 2048;
 __global__ void __launch_bounds__(256)
 big_collect_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d, SegTable seg,
@@ -312,7 +328,7 @@ big_collect_kernel(const float *__restrict__ x_half, const float *__restrict__ x
     if (c0 >= hi) return;
     const int64_t c1 = (c0 + kChunk < hi) ? c0 + kChunk : hi;
     const BigState stt = state[(int64_t)node * big.n + bi];
-    if (stt.overflow) return;                   // the whole-segment path takes this one
+    const unsigned cap = (unsigned)cand_capacity(hi - lo);
     BigCtl *h = ctl + (int64_t)node * big.n + bi;
     Cand *list = cands + (int64_t)node * cand_per_node + big.cand_base[bi];
     const float *xh = x_half + (int64_t)node * d, *xq = x_hat + (int64_t)node * d;
@@ -333,11 +349,14 @@ big_collect_kernel(const float *__restrict__ x_half, const float *__restrict__ x
             const int64_t eu = e + u * blockDim.x;
             if (eu < c1) {
                 const uint32_t key = mag_bits(a[u], b[u], plus);
-                if ((key >> kTopShift) == bucket) {
+                if ((key >> kTopShift) >= bucket) {
                     Cand c; c.key = key; c.pos = (uint32_t)(eu - lo);
                     const unsigned slot = atomicAdd(&s_cnt, 1u);
                     if (slot < kStage) stage[slot] = c;
-                    else list[atomicAdd(&h->cand_count, 1u)] = c;      // a dense stretch: straight to the list
+                    else {                                             // a dense stretch: straight to the list
+                        const unsigned at = atomicAdd(&h->cand_count, 1u);
+                        if (at < cap) list[at] = c;
+                    }
                 }
             }
         }
@@ -347,24 +366,25 @@ big_collect_kernel(const float *__restrict__ x_half, const float *__restrict__ x
     if (n == 0) return;
     if (threadIdx.x == 0) s_base = atomicAdd(&h->cand_count, n);
     __syncthreads();
-    for (unsigned i = threadIdx.x; i < n; i += blockDim.x) list[s_base + i] = stage[i];
+    for (unsigned i = threadIdx.x; i < n; i += blockDim.x)
+        if (s_base + i < cap) list[s_base + i] = stage[i];
 }
 
-// Threshold and tie cut of a long segment from its candidate list (one CTA).  All keys of the chosen
-// bucket are in the list, so the need-th largest of the list is the segment's k-th largest; if only
+// Threshold and tie cut of a long segment from its candidate list (one CTA).  The list holds every key
+// at or above a bucket and at least k of them, so its k-th largest is the segment's k-th largest; if only
 // some of the keys equal to it are taken, those at the lowest positions are: the cut follows the
 // need-th smallest position among them.
-__device__ void select_from_candidates(const Cand *__restrict__ list, const BigState &stt, int64_t lo, int64_t hi,
+__device__ void select_from_candidates(const Cand *__restrict__ list, int64_t n_cand, int64_t k, int64_t lo, int64_t hi,
                                        SelectOut *o) {
     long long need, eq;
-    const uint32_t thr = radix_select<false>((int64_t)stt.eq, [&](int64_t e) { return list[e].key; }, stt.need, kTopShift,
-                                             stt.prefix, &need, &eq);
+    const uint32_t thr = radix_select<false>(n_cand, [&](int64_t e) { return list[e].key; }, (long long)k, 32, 0u,
+                                             &need, &eq);
     if (eq == need) {
         if (threadIdx.x == 0) { o->thr = thr; o->dense = 0; o->cut = hi; }
         return;
     }
     long long n2, e2;      // ties keyed by descending position (never 0); the other candidates are skipped
-    const uint32_t inv = radix_select<true>((int64_t)stt.eq,
+    const uint32_t inv = radix_select<true>(n_cand,
                                             [&](int64_t e) { return list[e].key == thr ? 0xFFFFFFFFu - list[e].pos : 0u; },
                                             need, 32, 0u, &n2, &e2);
     if (threadIdx.x == 0) { o->thr = thr; o->dense = 0; o->cut = lo + (int64_t)(0xFFFFFFFFu - inv) + 1; }
@@ -433,7 +453,7 @@ select_and_rows_kernel(const float *__restrict__ x_half, const float *__restrict
                        SegTable seg, SelectOut *__restrict__ out, const float *__restrict__ Wmix, int nodes,
                        int32_t *__restrict__ tab, const unsigned int *__restrict__ amax_bits,
                        float *__restrict__ msg_scale, float *__restrict__ msg_inv, BigList big,
-                       const BigState *__restrict__ state, const Cand *__restrict__ cands, int64_t cand_per_node) {
+                       const BigCtl *__restrict__ ctl, const Cand *__restrict__ cands, int64_t cand_per_node) {
     pdl_enter();
     if ((int)blockIdx.y == nodes) {
         if (blockIdx.x == 0) {
@@ -457,9 +477,11 @@ select_and_rows_kernel(const float *__restrict__ x_half, const float *__restrict
     if (is_big(len, k)) {
         int bi = 0;
         while (big.id[bi] != s) ++bi;            // every long segment is in the list
-        const BigState stt = state[(int64_t)node * big.n + bi];
-        if (!stt.overflow) {
-            select_from_candidates(cands + (int64_t)node * cand_per_node + big.cand_base[bi], stt, lo, hi, o);
+        // exact count of the keys at or above the sampled bucket: with at least k of them, all in the list,
+        // the k largest are among the candidates; otherwise the whole-segment path below decides
+        const int64_t n_cand = (int64_t)ctl[(int64_t)node * big.n + bi].cand_count;
+        if (n_cand >= k && n_cand <= cand_capacity(len)) {
+            select_from_candidates(cands + (int64_t)node * cand_per_node + big.cand_base[bi], n_cand, k, lo, hi, o);
             return;
         }
     }
@@ -775,7 +797,7 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
     int32_t *tab = (int32_t *)((char *)ws + select_bytes(nodes, n_segments));
     BigList big;
     big.n = 0; big.chunk_base[0] = 0; big.cand_base[0] = 0;
-    int64_t most_chunks = 0;
+    int64_t most_chunks = 0, longest = 0;
     for (int s = 0; s < n_segments; ++s) {
         const int64_t len = seg.off[s + 1] - seg.off[s];
         if (!is_big(len, seg.k[s])) continue;
@@ -785,6 +807,7 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
         big.chunk_base[big.n + 1] = big.chunk_base[big.n] + (int32_t)nc;
         big.cand_base[big.n + 1] = big.cand_base[big.n] + cand_capacity(len);
         if (nc > most_chunks) most_chunks = nc;
+        if (len > longest) longest = len;
         ++big.n;
     }
     char *big_region = (char *)tab + rows_bytes(nodes);
@@ -796,7 +819,9 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
         if (most_chunks > 0x7fffffff || nodes > 65535) return LPDT_ERR_UNSUPPORTED;
         LPDT_CUDA(cudaMemsetAsync(ctl, 0, (size_t)nodes * big.n * sizeof(BigCtl), st));
         const dim3 g((unsigned)most_chunks, big.n, nodes);
-        launch_k(big_hist_kernel, g, 256, 0, st, x_half, x_hat, d, seg, big, ctl, state);
+        const int64_t sample_ctas = ceil_div(longest, kSampleChunk);
+        if (sample_ctas > 65535) return LPDT_ERR_UNSUPPORTED;
+        launch_k(big_sample_kernel, dim3((unsigned)sample_ctas, big.n, nodes), 256, 0, st, x_half, x_hat, d, seg, big, ctl, state);
         LPDT_LAUNCH_CHECK();
         launch_k(big_collect_kernel, g, 256, 0, st, x_half, x_hat, d, seg, big, ctl, state, cands, cand_per_node);
         LPDT_LAUNCH_CHECK();
@@ -813,7 +838,7 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
         LPDT_LAUNCH_CHECK();
     }
     launch_k(select_and_rows_kernel, dim3(n_segments, nodes + 1), 1024, 0, st, x_half, x_hat, d, seg, sel, Wmix, nodes, tab,
-             amax_bits, msg_scale, msg_inv, big, state, cands, cand_per_node);
+             amax_bits, msg_scale, msg_inv, big, ctl, cands, cand_per_node);
     LPDT_LAUNCH_CHECK();
     // parameters per thread: 16-byte accesses need every node's row on a 16-byte boundary (d a multiple of 4);
     // the networks' parameter counts are even but not multiples of 4, which still allows 8-byte accesses

@@ -579,8 +579,12 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t 
     static PerDeviceOnce attr;
     int dev;
     if (attr.pending(&dev)) {
-        for (int i = 0; i < 2; ++i)
+        for (int i = 0; i < 2; ++i) {
             LPDT_CUDA(cudaFuncSetAttribute(fns[1][i], cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
+            // the rings of three (six) resident CTAs need nearly all of the SM's shared memory
+            LPDT_CUDA(cudaFuncSetAttribute(fns[1][i], cudaFuncAttributePreferredSharedMemoryCarveout,
+                                           (int)cudaSharedmemCarveoutMaxShared));
+        }
         attr.mark(dev);
     }
     launch_k(fns[pl.V == 4 ? 1 : 0][pl.threads > 256 ? 1 : 0], grid, pl.threads, smem, st, H * W, C, groups, eps, Cst, dy, x,

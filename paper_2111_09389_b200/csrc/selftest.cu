@@ -31,6 +31,7 @@ extern "C" lpdt_status lpdt_selftest_bounded_wait(uint64_t limit_ns, int32_t *de
                                                   void *stream) {
     LPDT_CHECK_ARG(dev_status != nullptr);
     LPDT_CHECK_ARG(limit_ns >= 1000 && limit_ns <= 50ull * 1000 * 1000);      // 1 us .. 50 ms
+    ++lpdt::g_launch_count;
     lpdt::bounded_wait_probe_kernel<<<1, 64, 0, lpdt::as_stream(stream)>>>((unsigned long long)limit_ns, dev_status,
                                                                           returned);
     LPDT_LAUNCH_CHECK();

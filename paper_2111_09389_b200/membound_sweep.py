@@ -10,6 +10,7 @@ batch 128 so that each fp32 tensor is 268 MB; parameter kernels: 16 nodes with a
   quantize            range pass + scale-and-round: 4 B read twice + 1 B written per element
   quantize_stochastic the same with Philox stochastic rounding
   quantize_with_range range supplied by the producer: 4 B read + 1 B written
+  dequantize          1 B read + 4 B written: a write-dominated stream (80 % of its bytes are stores)
   ren_fwd             4 B read + 4 B written (the second read of a sample comes from L2)
   ren_fwd_res         + 4 B shortcut read
   ren_bwd             dy, x read + dx written: 12 B
@@ -63,6 +64,8 @@ def cases(nodes=8, B=128, H=32, W=32, Cc=64, d=32 * 270410, gossip_nodes=16):
     yield ("quantize", lambda: api.lpdt_quantize(x, nodes, n, n, q, scale, ws), tot * 9)
     yield ("quantize_stochastic", lambda: api.lpdt_quantize(x, nodes, n, n, q, scale, ws, rounding=1, seed=3), tot * 9)
     yield ("quantize_with_range", lambda: api.lpdt_quantize_with_range(x, nodes, n, n, amax, q, scale), tot * 5)
+    api.lpdt_quantize_with_range(x, nodes, n, n, amax, q, scale)
+    yield ("dequantize", lambda: api.lpdt_dequantize(q, nodes, n, scale, y), tot * 5)
 
     groups = Cc // 8
     v = torch.ones(nodes, Cc, device="cuda")

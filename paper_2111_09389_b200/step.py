@@ -452,33 +452,14 @@ class TrainStep:
         one-time kernel attribute is set before capture)."""
         self.run()
         torch.cuda.synchronize()
-        before = api.KERNEL_LAUNCHES
+        before = api.lpdt_launch_count()
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
             self.run()
-        self.graph_launches = api.KERNEL_LAUNCHES - before
+        self.graph_launches = api.lpdt_launch_count() - before
         self.graph = g
         return g
 
     def replay(self):
         self.graph.replay()
-        api.KERNEL_LAUNCHES += self.graph_launches
-
-    def launches_per_step(self):
-        """Kernel launches of one run(): counted from the op list (memsets excluded)."""
-        n = 0
-        for op in self.ops:
-            k = op["op"]
-            if k in ("conv", "linear"):
-                first = op is self.ops[0] and not self.input_grad
-                n += 2 * 2 + 1            # two quantizes (2 kernels each) + fwd
-                n += 2                    # quantize E
-                n += 2                    # bwd-weight + dequant (generic path upper bound)
-                n += 0 if first else 2    # transpose + bwd-data
-                n += 1 if k == "linear" else 0
-            elif k == "ren":
-                n += 1 + 2
-            elif k in ("add", "maxpool", "avgpool"):
-                n += 2
-        n += 1 if self.labels is not None else 0
-        return n + 1 + 2                  # sgd + select + mix
+        api.add_replayed_launches(self.graph_launches)
