@@ -243,7 +243,9 @@ lpdt_status lpdt_dequantize_acc_batch(const int32_t *acc, int32_t nodes, int32_t
  * ws      : lpdt_qconv_fwd_affine_workspace_size(desc) bytes, 256-byte aligned
  * The integer contraction of the codes runs on the same kernels as
  * lpdt_qconv_fwd (unsigned operand format); the zero-point terms are applied
- * by a correction pass over the int32 sums.
+ * in the tensor-core kernel's epilogue (forward product) or by a correction
+ * pass over the int32 sums (shapes outside the tensor-core path, and both
+ * backward products).
  * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE, CUDA; TIMEOUT through dev_status.
  *
  * The two backward products in the same form (the adjoints of the forward product: a tap

@@ -205,20 +205,22 @@ struct BigList {
     int64_t cand_base[kMaxSeg + 1];    // prefix sums of the candidate capacities
 };
 constexpr int kTopBins = 4096;
-struct BigCtl { uint32_t h0[kTopBins]; uint32_t ticket, cand_count, sampled, pad; };   // zeroed per call; cand_count: keys at or above the bucket
+// zeroed per call.  h0: histogram of the sample; h1: exact histogram of the collected keys (same 12 bits);
+// cand_count: keys at or above the chosen bucket
+struct BigCtl { uint32_t h0[kTopBins], h1[kTopBins]; uint32_t ticket, cand_count, sampled, pad; };
 struct BigState { uint32_t prefix; uint32_t sampled; };    // lowest magnitude bits of the chosen bucket; keys sampled
 struct __align__(8) Cand { uint32_t key, pos; };    // magnitude bits, position inside the segment
 
 __device__ __host__ __forceinline__ int64_t cand_capacity(int64_t len) { return len / 8 + 4096; }
 
 // Walk a histogram from its top bin: the bucket holding the need-th largest key, the keys still
-// needed inside it and its population.  Whole CTA (256 threads); same result in every thread.
+// needed inside it and its population.  Whole CTA (its thread count divides nbins); same result in every thread.
 // The histogram was filled by other CTAs' atomics: read it from L2.
 __device__ void pick_bucket(const uint32_t *hist, int nbins, long long need, int *bucket,
                             long long *need_out, long long *eq_out) {
-    __shared__ long long wtot[8];
+    __shared__ long long wtot[32];
     __shared__ long long res[3];
-    const int t = threadIdx.x, lane = t & 31, warp = t >> 5, per = nbins / 256;
+    const int t = threadIdx.x, lane = t & 31, warp = t >> 5, nwarps = blockDim.x >> 5, per = nbins / blockDim.x;
     long long mine = 0;
     for (int b = 0; b < per; ++b) mine += __ldcg(hist + t * per + b);
     // suffix sums over the 256 slices: inside the warp by shuffles, across warps through shared memory
@@ -232,7 +234,7 @@ __device__ void pick_bucket(const uint32_t *hist, int nbins, long long need, int
     if (lane == 0) wtot[warp] = incl;
     __syncthreads();
     long long above = incl - mine;
-    for (int w = warp + 1; w < 8; ++w) above += wtot[w];
+    for (int w = warp + 1; w < nwarps; ++w) above += wtot[w];
     if (above < need && need <= above + mine) {
         long long n = need - above;
         int b = t * per + per - 1;
@@ -298,10 +300,10 @@ big_sample_kernel(const float *__restrict__ x_half, const float *__restrict__ x_
     const unsigned nchunks = (unsigned)ceil_div_dev(hi - lo, kSampleChunk);
     if (s_ticket != nchunks - 1) return;
     __threadfence();
-    // keys the sample must show at or above the bucket: the sampled share of k, a quarter more, and four
+    // keys the sample must show at or above the bucket: the sampled share of k, a tenth more, and four
     // standard deviations of the sampled count
     const double m = (double)__ldcg(&h->sampled), f = m / (double)(hi - lo), fk = f * (double)seg.k[s];
-    long long target = (long long)(1.25 * fk + 4.0 * sqrt(fk) + 8.0);
+    long long target = (long long)(1.10 * fk + 4.0 * sqrt(fk) + 8.0);
     int b = 0; long long need, eq;
     if (target <= (long long)m) pick_bucket(h->h0, kTopBins, target, &b, &need, &eq);
     if (threadIdx.x == 0) {
@@ -334,7 +336,9 @@ big_collect_kernel(const float *__restrict__ x_half, const float *__restrict__ x
     const float *xh = x_half + (int64_t)node * d, *xq = x_hat + (int64_t)node * d;
     const uint32_t bucket = stt.prefix >> kTopShift;
     __shared__ Cand stage[kStage];
+    __shared__ unsigned int sh1[kTopBins];       // this CTA's share of the exact histogram of the collected keys
     __shared__ unsigned int s_cnt, s_base;
+    for (int i = threadIdx.x; i < kTopBins; i += blockDim.x) sh1[i] = 0;
     if (threadIdx.x == 0) s_cnt = 0;
     __syncthreads();
     for (int64_t e = c0 + threadIdx.x; e < c1; e += 4 * blockDim.x) {
@@ -350,6 +354,7 @@ big_collect_kernel(const float *__restrict__ x_half, const float *__restrict__ x
             if (eu < c1) {
                 const uint32_t key = mag_bits(a[u], b[u], plus);
                 if ((key >> kTopShift) >= bucket) {
+                    atomicAdd(&sh1[key >> kTopShift], 1u);
                     Cand c; c.key = key; c.pos = (uint32_t)(eu - lo);
                     const unsigned slot = atomicAdd(&s_cnt, 1u);
                     if (slot < kStage) stage[slot] = c;
@@ -362,6 +367,8 @@ big_collect_kernel(const float *__restrict__ x_half, const float *__restrict__ x
         }
     }
     __syncthreads();
+    for (int i = bucket + threadIdx.x; i < kTopBins; i += blockDim.x)
+        if (sh1[i]) atomicAdd(&h->h1[i], sh1[i]);
     const unsigned n = s_cnt < kStage ? s_cnt : kStage;
     if (n == 0) return;
     if (threadIdx.x == 0) s_base = atomicAdd(&h->cand_count, n);
@@ -374,11 +381,15 @@ big_collect_kernel(const float *__restrict__ x_half, const float *__restrict__ x
 // at or above a bucket and at least k of them, so its k-th largest is the segment's k-th largest; if only
 // some of the keys equal to it are taken, those at the lowest positions are: the cut follows the
 // need-th smallest position among them.
-__device__ void select_from_candidates(const Cand *__restrict__ list, int64_t n_cand, int64_t k, int64_t lo, int64_t hi,
-                                       SelectOut *o) {
+__device__ void select_from_candidates(const Cand *__restrict__ list, int64_t n_cand, int64_t k, const uint32_t *h1,
+                                       int64_t lo, int64_t hi, SelectOut *o) {
+    // the collect pass left the exact histogram of the candidates' top 12 bits: the bucket of the k-th largest
+    // key comes from it without a scan, and only the 19 bits below are searched in the list
+    int b1; long long need1, eq1;
+    pick_bucket(h1, kTopBins, (long long)k, &b1, &need1, &eq1);
     long long need, eq;
-    const uint32_t thr = radix_select<false>(n_cand, [&](int64_t e) { return list[e].key; }, (long long)k, 32, 0u,
-                                             &need, &eq);
+    const uint32_t thr = radix_select<false>(n_cand, [&](int64_t e) { return list[e].key; }, need1, kTopShift,
+                                             (uint32_t)b1 << kTopShift, &need, &eq);
     if (eq == need) {
         if (threadIdx.x == 0) { o->thr = thr; o->dense = 0; o->cut = hi; }
         return;
@@ -481,7 +492,8 @@ select_and_rows_kernel(const float *__restrict__ x_half, const float *__restrict
         // the k largest are among the candidates; otherwise the whole-segment path below decides
         const int64_t n_cand = (int64_t)ctl[(int64_t)node * big.n + bi].cand_count;
         if (n_cand >= k && n_cand <= cand_capacity(len)) {
-            select_from_candidates(cands + (int64_t)node * cand_per_node + big.cand_base[bi], n_cand, k, lo, hi, o);
+            select_from_candidates(cands + (int64_t)node * cand_per_node + big.cand_base[bi], n_cand, k,
+                                   ctl[(int64_t)node * big.n + bi].h1, lo, hi, o);
             return;
         }
     }

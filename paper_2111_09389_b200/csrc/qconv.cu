@@ -322,9 +322,6 @@ extern "C" lpdt_status lpdt_qconv_fwd_affine(const lpdt_conv_desc *d, const uint
     int32_t *asum = (int32_t *)((char *)ws + affine_raw_bytes(d));
     int32_t *P = (int32_t *)((char *)asum + affine_asum_bytes(d));
     void *inner = (char *)P + affine_prefix_bytes(d);
-    s = fwd_impl(d, reinterpret_cast<const int8_t *>(A), nullptr, reinterpret_cast<const int8_t *>(Wq), nullptr, nullptr,
-                 0, nullptr, raw, inner, lpdt_qconv_workspace_size(d, 0), dev_status, st, true);
-    if (s != LPDT_OK) return s;
     const int64_t pixels = (int64_t)d->nodes * d->B * d->H * d->W;
     s = row_sum_launch(A, pixels, d->Cin, asum, st);
     if (s != LPDT_OK) return s;
@@ -334,6 +331,20 @@ extern "C" lpdt_status lpdt_qconv_fwd_affine(const lpdt_conv_desc *d, const uint
     if (s != LPDT_OK) return s;
     launch_k(weight_prefix_kernel, (rows + 127) / 128, 128, 0, st, tapsum, d->nodes, d->Cout, d->R, d->S, P);
     LPDT_LAUNCH_CHECK();
+    // Tensor-core path: the zero-point terms are applied in the contraction's own epilogue (no raw sums in
+    // memory, no second pass over the result).  LPDT_AFFINE_SEPARATE=1 keeps the separate correction pass.
+    static int separate = -1;
+    if (separate < 0) { const char *e = getenv("LPDT_AFFINE_SEPARATE"); separate = (e && e[0] == '1') ? 1 : 0; }
+    if (!separate && use_tc(*d) && d->Cout % 4 == 0 && aligned(A, 16) && aligned(Wq, 16) && (!Y || aligned(Y, 16)) &&
+        (!Yacc || aligned(Yacc, 16))) {
+        const tc::AffineArgs aff = {asum, P, zA, zW};
+        lpdt_status r = tc::tc_pix(*d, 0, reinterpret_cast<const int8_t *>(A), sA, reinterpret_cast<const int8_t *>(Wq), sW,
+                                   bias, bias_node_stride, Y, Yacc, dev_status, st, true, nullptr, &aff);
+        if (r != LPDT_ERR_UNSUPPORTED) return r;
+    }
+    s = fwd_impl(d, reinterpret_cast<const int8_t *>(A), nullptr, reinterpret_cast<const int8_t *>(Wq), nullptr, nullptr,
+                 0, nullptr, raw, inner, lpdt_qconv_workspace_size(d, 0), dev_status, st, true);
+    if (s != LPDT_OK) return s;
     const bool v4 = d->Cout % 4 == 0 && (!Y || aligned(Y, 16)) && (!Yacc || aligned(Yacc, 16));
     const int64_t work = (int64_t)d->nodes * d->B * Ho * Wo * (d->Cout / (v4 ? 4 : 1));
     if (v4)

@@ -24,9 +24,14 @@ namespace tc {
 // Tensor-core engine (tcgen05 kind::i8): stride-1 convolutions and GEMMs whose
 // channel counts are multiples of 16.  mode 0 = forward, 1 = backward-data.
 bool tc_supported(const lpdt_conv_desc &d);
+// Zero-point correction applied in the forward epilogue (unsigned operands): per-pixel channel sums of the
+// input [nodes][B][H][W], prefix table of the weights' channel sums over the filter taps
+// [nodes][R+1][S+1][Cout], and the per-node zero points.
+struct AffineArgs { const int32_t *asum, *wpre, *zA, *zW; };
 lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const float *s1, const int8_t *Wq,
                    const float *s2, const float *bias, int64_t bias_stride, float *Y, int32_t *Yacc,
-                   int32_t *dev_status, cudaStream_t st, bool uns = false, const float *addend = nullptr);
+                   int32_t *dev_status, cudaStream_t st, bool uns = false, const float *addend = nullptr,
+                   const AffineArgs *aff = nullptr);
 // Halo-tile kernel for 16-channel operands at stride 1 (one TMA request per tile).
 bool halo_supported(const lpdt_conv_desc &d, int mode);
 lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, const float *s1, const int8_t *Wq,

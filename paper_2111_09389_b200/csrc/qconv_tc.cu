@@ -77,7 +77,59 @@ struct PixParams {
     // channels (128-byte rows, 128-byte swizzle) and stores them as one box {32 channels, bw, bh, bb pixels}
     int tma_out, out_off;     // out_off: byte offset of the staging area in shared memory (1024-byte aligned)
     int bw, bh;               // the warp's sub-box of the pixel tile: bw x bh x 32/(bw*bh) pixels
+    // Forward product on affine (zero-point) operands, corrected in the epilogue (null asum: plain product):
+    //   sum (qa - zA)(qw - zW) = acc - zW * ra - zA * rw + cnt * zA * zW   over the taps inside the image,
+    // ra = the per-pixel channel sums of the input (asum [nodes][B][H][W]) over those taps, rw = the weights'
+    // channel sums over them, from a prefix table over the filter taps (wpre [nodes][R+1][S+1][Cout]; the taps
+    // inside the image form a rectangle of the filter), cnt = taps inside x Cin.  All modulo 2^32.
+    const int32_t *asum, *wpre, *zA, *zW;
+    int aH, aW, aR, aS, apad, astride, aCin;
 };
+
+// Zero-point terms of one output pixel: what does not depend on the output channel (fixed) and the corners of
+// the pixel's tap rectangle in the prefix table.
+struct AffinePixel { unsigned fixed, za; int c11, c01, c10, c00; bool interior; };
+__device__ __forceinline__ AffinePixel affine_pixel(const PixParams &p, int node, int b, int oh, int ow) {
+    int r_lo = p.apad - oh * p.astride; if (r_lo < 0) r_lo = 0;
+    int r_hi = p.aH + p.apad - oh * p.astride; if (r_hi > p.aR) r_hi = p.aR;
+    int s_lo = p.apad - ow * p.astride; if (s_lo < 0) s_lo = 0;
+    int s_hi = p.aW + p.apad - ow * p.astride; if (s_hi > p.aS) s_hi = p.aS;
+    if (r_hi < r_lo) r_hi = r_lo;
+    if (s_hi < s_lo) s_hi = s_lo;
+    const long long nb = (long long)node * p.B + b;
+    unsigned ra = 0;
+    for (int r = r_lo; r < r_hi; ++r)
+        for (int s = s_lo; s < s_hi; ++s)
+            ra += (unsigned)__ldg(p.asum + (nb * p.aH + oh * p.astride + r - p.apad) * p.aW + ow * p.astride + s - p.apad);
+    AffinePixel a;
+    const unsigned za = (unsigned)p.zA[node], zw = (unsigned)p.zW[node];
+    a.za = za;
+    a.fixed = (unsigned)((r_hi - r_lo) * (s_hi - s_lo) * p.aCin) * za * zw - zw * ra;
+    const int PS = p.aS + 1;
+    a.c11 = (r_hi * PS + s_hi) * p.Nc; a.c01 = (r_lo * PS + s_hi) * p.Nc;
+    a.c10 = (r_hi * PS + s_lo) * p.Nc; a.c00 = (r_lo * PS + s_lo) * p.Nc;
+    a.interior = r_lo == 0 && s_lo == 0;          // the three other corners are zero
+    return a;
+}
+// acc[k] += fixed - za * rw[channel c0 + k], k < NV (NV a multiple of 4, c0 a multiple of 4)
+template <int NV>
+__device__ __forceinline__ void affine_apply(const PixParams &p, const AffinePixel &a, int node, int c0, uint32_t (&v)[NV]) {
+    const int32_t *t = p.wpre + (long long)node * (p.aR + 1) * (p.aS + 1) * p.Nc + c0;
+#pragma unroll
+    for (int k = 0; k < NV; k += 4) {
+        const int4 q11 = __ldg(reinterpret_cast<const int4 *>(t + a.c11 + k));
+        unsigned rw[4] = {(unsigned)q11.x, (unsigned)q11.y, (unsigned)q11.z, (unsigned)q11.w};
+        if (!a.interior) {
+            const int4 q01 = __ldg(reinterpret_cast<const int4 *>(t + a.c01 + k));
+            const int4 q10 = __ldg(reinterpret_cast<const int4 *>(t + a.c10 + k));
+            const int4 q00 = __ldg(reinterpret_cast<const int4 *>(t + a.c00 + k));
+            rw[0] += (unsigned)q00.x - (unsigned)q01.x - (unsigned)q10.x; rw[1] += (unsigned)q00.y - (unsigned)q01.y - (unsigned)q10.y;
+            rw[2] += (unsigned)q00.z - (unsigned)q01.z - (unsigned)q10.z; rw[3] += (unsigned)q00.w - (unsigned)q01.w - (unsigned)q10.w;
+        }
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[k + j] = v[k + j] + a.fixed - a.za * rw[j];
+    }
+}
 
 struct SharedCtl {
     unsigned long long full[8], empty[8], tmem_full[2], tmem_empty[2];
@@ -283,6 +335,8 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
             tc_fence_after();
             const long long pix = (((long long)c.node * p.B + b) * p.Hout + h) * p.Wout + w;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * p.BN;
+            AffinePixel aff = {};
+            if (p.asum && valid) aff = affine_pixel(p, c.node, b, h, w);
             if (p.tma_out) {
                 // 32 channels at a time: accumulators -> fp32 -> this warp's staging buffer (one 128-byte row per
                 // lane, 16-byte pieces XOR-swizzled by the row so that the lanes spread over all banks, which is
@@ -296,6 +350,7 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 if (have) tmem_ld_32x32(t_row + cc, v);
                 while (have) {
                     tmem_ld_wait();
+                    if (p.asum && valid) affine_apply<32>(p, aff, c.node, n0 + cc, v);
                     float f[32];
 #pragma unroll
                     for (int k = 0; k < 32; ++k) f[k] = __fmul_rn(__int2float_rn((int)v[k]), sc);
@@ -342,6 +397,7 @@ conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant_
                 tmem_ld_wait();
                 if (valid) {
                     const long long o = pix * p.Nc + n0 + cc;
+                    if (p.asum) affine_apply<16>(p, aff, c.node, n0 + cc, v);
                     if (p.Yacc) {
                         int4 *dst = reinterpret_cast<int4 *>(p.Yacc + o);
 #pragma unroll
@@ -628,10 +684,15 @@ static int largest_div(int C, int cap, int unit) {      // largest multiple of u
 
 lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const float *s1, const int8_t *Wq,
                    const float *s2, const float *bias, int64_t bias_stride, float *Y, int32_t *Yacc,
-                   int32_t *dev_status, cudaStream_t st, bool uns, const float *addend) {
+                   int32_t *dev_status, cudaStream_t st, bool uns, const float *addend, const AffineArgs *aff) {
     const int Ho = conv_out(d.H, d.pad, d.R, d.stride), Wo = conv_out(d.W, d.pad, d.S, d.stride);
     PixParams p = {};
     p.addend = addend;
+    if (aff) {
+        if (mode != 0 || d.Cout % 4) return LPDT_ERR_UNSUPPORTED;
+        p.asum = aff->asum; p.wpre = aff->wpre; p.zA = aff->zA; p.zW = aff->zW;
+        p.aH = d.H; p.aW = d.W; p.aR = d.R; p.aS = d.S; p.apad = d.pad; p.astride = d.stride; p.aCin = d.Cin;
+    }
     p.mode = mode; p.nodes = d.nodes; p.B = d.B;
     p.Nc = mode == 0 ? d.Cout : d.Cin; p.Kc = mode == 0 ? d.Cin : d.Cout;
     p.out_mul = 1; p.cmul = 1; p.ncls = 1;
