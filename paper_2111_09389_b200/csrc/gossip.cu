@@ -322,7 +322,7 @@ constexpr int kStage = 2048;
 __global__ void __launch_bounds__(256)
 big_collect_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d, SegTable seg,
                    BigList big, BigCtl *__restrict__ ctl, const BigState *__restrict__ state,
-                   Cand *__restrict__ cands, int64_t cand_per_node) {
+                   Cand *__restrict__ cands, int64_t cand_per_node, unsigned int *__restrict__ amax_bits) {
     pdl_enter();
     const int bi = blockIdx.y, node = blockIdx.z, s = big.id[bi], plus = seg.plus;
     const int64_t lo = seg.off[s], hi = seg.off[s + 1];
@@ -341,6 +341,7 @@ big_collect_kernel(const float *__restrict__ x_half, const float *__restrict__ x
     for (int i = threadIdx.x; i < kTopBins; i += blockDim.x) sh1[i] = 0;
     if (threadIdx.x == 0) s_cnt = 0;
     __syncthreads();
+    uint32_t kmax = 0;          // largest magnitude of the chunk: the range of the segment's 8-bit message
     for (int64_t e = c0 + threadIdx.x; e < c1; e += 4 * blockDim.x) {
         float a[4], b[4];
 #pragma unroll
@@ -353,6 +354,7 @@ big_collect_kernel(const float *__restrict__ x_half, const float *__restrict__ x
             const int64_t eu = e + u * blockDim.x;
             if (eu < c1) {
                 const uint32_t key = mag_bits(a[u], b[u], plus);
+                kmax = key > kmax ? key : kmax;
                 if ((key >> kTopShift) >= bucket) {
                     atomicAdd(&sh1[key >> kTopShift], 1u);
                     Cand c; c.key = key; c.pos = (uint32_t)(eu - lo);
@@ -367,6 +369,10 @@ big_collect_kernel(const float *__restrict__ x_half, const float *__restrict__ x
         }
     }
     __syncthreads();
+    if (amax_bits) {            // the same value the range pass of the 8-bit messages would find
+        for (int o = 16; o > 0; o >>= 1) { const uint32_t t = __shfl_xor_sync(0xffffffffu, kmax, o); kmax = t > kmax ? t : kmax; }
+        if ((threadIdx.x & 31) == 0 && kmax) atomicMax(amax_bits + (int64_t)node * seg.n_seg + s, kmax);
+    }
     for (int i = bucket + threadIdx.x; i < kTopBins; i += blockDim.x)
         if (sh1[i]) atomicAdd(&h->h1[i], sh1[i]);
     const unsigned n = s_cnt < kStage ? s_cnt : kStage;
@@ -827,6 +833,17 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
     BigState *state = (BigState *)(ctl + (size_t)nodes * big.n);
     Cand *cands = (Cand *)(big_region + big_ctl_bytes(nodes, d, n_segments));
     const int64_t cand_per_node = big.cand_base[big.n];
+    // 8-bit messages: ranges of the differences (the kept entries are the largest of their segment).  The collect
+    // pass of a long compressed segment sees every difference anyway and records the range itself; the separate
+    // range pass runs only when some segment does not go through it.
+    unsigned int *amax_bits = nullptr;
+    float *msg_inv = nullptr;
+    if (q8) {
+        amax_bits = (unsigned int *)((char *)ws + lpdt_gossip_mix_workspace_size(nodes, d, n_segments) - 2 * q8_bytes(nodes, n_segments));
+        msg_inv = (float *)((char *)amax_bits + q8_bytes(nodes, n_segments));
+        if (nodes > 65535) return LPDT_ERR_UNSUPPORTED;
+        LPDT_CUDA(cudaMemsetAsync(amax_bits, 0, (size_t)nodes * n_segments * sizeof(unsigned int), st));
+    }
     if (big.n > 0) {
         if (most_chunks > 0x7fffffff || nodes > 65535) return LPDT_ERR_UNSUPPORTED;
         LPDT_CUDA(cudaMemsetAsync(ctl, 0, (size_t)nodes * big.n * sizeof(BigCtl), st));
@@ -835,17 +852,10 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
         if (sample_ctas > 65535) return LPDT_ERR_UNSUPPORTED;
         launch_k(big_sample_kernel, dim3((unsigned)sample_ctas, big.n, nodes), 256, 0, st, x_half, x_hat, d, seg, big, ctl, state);
         LPDT_LAUNCH_CHECK();
-        launch_k(big_collect_kernel, g, 256, 0, st, x_half, x_hat, d, seg, big, ctl, state, cands, cand_per_node);
+        launch_k(big_collect_kernel, g, 256, 0, st, x_half, x_hat, d, seg, big, ctl, state, cands, cand_per_node, amax_bits);
         LPDT_LAUNCH_CHECK();
     }
-    // 8-bit messages: ranges of the differences first (the kept entries are the largest of their segment)
-    unsigned int *amax_bits = nullptr;
-    float *msg_inv = nullptr;
-    if (q8) {
-        amax_bits = (unsigned int *)((char *)ws + lpdt_gossip_mix_workspace_size(nodes, d, n_segments) - 2 * q8_bytes(nodes, n_segments));
-        msg_inv = (float *)((char *)amax_bits + q8_bytes(nodes, n_segments));
-        if (nodes > 65535) return LPDT_ERR_UNSUPPORTED;
-        LPDT_CUDA(cudaMemsetAsync(amax_bits, 0, (size_t)nodes * n_segments * sizeof(unsigned int), st));
+    if (q8 && big.n < n_segments) {
         launch_k(delta_amax_kernel, dim3((unsigned)ceil_div(d, (int64_t)kChunk), nodes), 256, 0, st, x_half, x_hat, d, seg, amax_bits);
         LPDT_LAUNCH_CHECK();
     }

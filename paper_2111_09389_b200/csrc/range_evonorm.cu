@@ -565,8 +565,13 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t 
     const int nsets = (cv <= 32 && 32 % cv == 0) ? pl.threads / 32 : 1;      // as in the kernel
     size_t smem = (size_t)(nsets * 3 * C + pl.threads + groups) * sizeof(double);
     if (smem > 48 * 1024) return LPDT_ERR_UNSUPPORTED;
-    // rows in flight per thread (V = 4): 8 with up to 256 threads (64 KB of ring, three CTAs per SM), 4 beyond
-    const int depth = pl.V == 4 ? (pl.threads <= 256 ? 8 : 4) : 0;
+    // rows in flight per thread (V = 4): 8 with up to 256 threads, or 6 when the sums' shared memory would push a
+    // CTA past its share of the SM's shared memory (three CTAs per SM, six of 128 threads) and a thread has more
+    // than 8 rows anyway (with 8 or fewer, all of a thread's rows are requested at once); 4 beyond 256 threads
+    int depth = pl.V == 4 ? (pl.threads <= 256 ? 8 : 4) : 0;
+    const size_t third = (size_t)(227 * 1024) / (pl.threads <= 128 ? 6 : 3) - 1024;
+    const int rows_per_thread = (int)ceil_div((int64_t)H * W, pl.threads / cv);
+    if (depth == 8 && rows_per_thread > 8 && align_up(smem, 16) + (size_t)8 * 2 * pl.threads * 16 > third) depth = 6;
     smem = align_up(smem, 16) + (size_t)depth * 2 * pl.threads * 16;
     cudaStream_t st = as_stream(stream);
     double *acc = (double *)ws;
@@ -574,12 +579,12 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t 
     dim3 grid((unsigned)((int64_t)nodes * B));
     using Fn = void (*)(int, int, int, float, float, const float *, const float *, const float *, const float *, int64_t, int,
                         const float *, const float *, const int32_t *, const int32_t *, float *, double *, float *);
-    static const Fn fns[2][2] = {{ren_bwd_kernel<1, 256, 0>, ren_bwd_kernel<1, 512, 0>},
-                                 {ren_bwd_kernel<4, 256, 8>, ren_bwd_kernel<4, 512, 4>}};
+    static const Fn fns[2][3] = {{ren_bwd_kernel<1, 256, 0>, ren_bwd_kernel<1, 512, 0>, ren_bwd_kernel<1, 256, 0>},
+                                 {ren_bwd_kernel<4, 256, 8>, ren_bwd_kernel<4, 512, 4>, ren_bwd_kernel<4, 256, 6>}};
     static PerDeviceOnce attr;
     int dev;
     if (attr.pending(&dev)) {
-        for (int i = 0; i < 2; ++i) {
+        for (int i = 0; i < 3; ++i) {
             LPDT_CUDA(cudaFuncSetAttribute(fns[1][i], cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
             // the rings of three (six) resident CTAs need nearly all of the SM's shared memory
             LPDT_CUDA(cudaFuncSetAttribute(fns[1][i], cudaFuncAttributePreferredSharedMemoryCarveout,
@@ -587,7 +592,7 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t 
         }
         attr.mark(dev);
     }
-    launch_k(fns[pl.V == 4 ? 1 : 0][pl.threads > 256 ? 1 : 0], grid, pl.threads, smem, st, H * W, C, groups, eps, Cst, dy, x,
+    launch_k(fns[pl.V == 4 ? 1 : 0][pl.threads > 256 ? 1 : depth == 6 ? 2 : 0], grid, pl.threads, smem, st, H * W, C, groups, eps, Cst, dy, x,
              v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc, amax_out);
     LPDT_LAUNCH_CHECK();
     if (deferred) return LPDT_OK;
