@@ -229,24 +229,47 @@ def call_bytes(name, a, kw):
 
 
 def group_key(rec):
-    name, _, _, _, kernel = rec
+    name, kernel = rec[0], rec[4]
     return f"{name} [{kernel}]" if kernel else name
 
 
+_REPLAY_STREAMS = {}
+
+
+def issue(calls):
+    """Issue logged calls as the step does: the calls of each node group on a stream of that group, side by
+    side between a fork and a join (one group: plainly on the current stream)."""
+    import torch
+    tags = sorted({c[5] for c in calls})
+    if len(tags) <= 1:
+        for c in calls:
+            c[1](*c[2], **c[3])
+        return
+    main = torch.cuda.current_stream()
+    for t in tags:
+        st = _REPLAY_STREAMS.setdefault(t, torch.cuda.Stream())
+        st.wait_stream(main)
+        with torch.cuda.stream(st):
+            for c in calls:
+                if c[5] == t:
+                    c[1](*c[2], **c[3])
+    for t in tags:
+        main.wait_stream(_REPLAY_STREAMS[t])
+
+
 def time_group(calls, reps):
-    """Milliseconds per issue of `calls` (logged entry-point calls of one step, in step order):
-    recorded into one CUDA graph and replayed `reps` times between two events on the current stream."""
+    """Milliseconds per issue of `calls` (logged entry-point calls of one step, in step order; node groups side
+    by side as in the step): recorded into one CUDA graph and replayed `reps` times between two events on the
+    current stream."""
     import torch
     from paper_2111_09389_b200 import api
     before = api.lpdt_launch_count()
-    for _, fn, a, kw, _ in calls:
-        fn(*a, **kw)
+    issue(calls)
     time_group.launches = api.lpdt_launch_count() - before       # kernels one issue of `calls` enqueues
     torch.cuda.synchronize()
     g = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g):
-        for _, fn, a, kw, _ in calls:
-            fn(*a, **kw)
+        issue(calls)
     for _ in range(2):
         g.replay()
     torch.cuda.synchronize()
@@ -366,6 +389,8 @@ def run_step_workload(name, rank, world, steps, warmup, graph=True, **step_optio
     from paper_2111_09389_b200 import api, workloads
     from paper_2111_09389_b200.step import TrainStep
     wl = workloads.make_workload(name, seed=rank_seed(rank))
+    if not step_options.get("node_groups"):
+        step_options["node_groups"] = 2 if wl["nodes"] >= 32 else 1
     st = TrainStep.from_workload(wl, **step_options)
     images = wl["nodes"] * wl["batch"]
     if graph:
@@ -416,7 +441,7 @@ def run_step_workload(name, rank, world, steps, warmup, graph=True, **step_optio
            "int8_tops": 2 * macs * world / (ms_total / steps * 1e-3) / 1e12, "macs_per_step": macs,
            "launches": int(launches), "launches_per_step": int(launches) // max(1, steps),
            "nodes": wl["nodes"], "batch_per_node": wl["batch"], "params_per_node": wl["d"],
-           "saved_bytes_per_node": st.saved_bytes_per_node()}
+           "node_groups": st.node_groups, "saved_bytes_per_node": st.saved_bytes_per_node()}
     return res, st, wl
 
 
@@ -463,7 +488,8 @@ def run_ours(args):
     sampler = ClockSampler(local)
     sampler.start()
     sampler.wait_for_samples(2)
-    head, st, wl = run_step_workload(args.workload, rank, world, args.steps, args.warmup, graph=args.graph)
+    head, st, wl = run_step_workload(args.workload, rank, world, args.steps, args.warmup, graph=args.graph,
+                                     node_groups=args.node_groups)
     reps = max(args.steps, 5)
     rows, log = breakdown(st, reps, peaks)
     roof = roofline_record(rows, log, args.roofline_kernel, peaks, args.workload, reps)
@@ -477,7 +503,9 @@ def run_ours(args):
         "config": {"workload": args.workload, "description": WORKLOAD_DESC.get(args.workload, args.workload),
                    "nodes": wl["nodes"], "batch_per_node": wl["batch"], "params_per_node": wl["d"],
                    "parallelism": "replicas only" if world > 1 else "1 GPU, nodes batched",
-                   "launch": "CUDA graph replay of the whole step" if args.graph else "eager launches",
+                   "launch": ("CUDA graph replay of the whole step" if args.graph else "eager launches") +
+                             (f", forward/backward of {head['node_groups']} node groups on parallel streams"
+                              if head["node_groups"] > 1 else ""),
                    "l2": "activations touched per step exceed L2 (working set of several GB vs 126 MB)"},
         "int8_tops": head["int8_tops"], "macs_per_step": head["macs_per_step"],
         "clocks": clocks, "e2e": head["e2e"], "gpu_launches": head["launches"],
@@ -495,7 +523,8 @@ def run_ours(args):
             if name == args.workload:
                 r = dict(head)
             else:
-                r, st2, _ = run_step_workload(name, rank, world, args.steps, args.warmup, graph=args.graph)
+                r, st2, _ = run_step_workload(name, rank, world, args.steps, args.warmup, graph=args.graph,
+                                              node_groups=args.node_groups)
                 del st2
                 torch.cuda.empty_cache()
             r["images_per_s"] = r.pop("value")
@@ -581,6 +610,9 @@ def main():
     ap.add_argument("--workload", default=HEADLINE)
     ap.add_argument("--roofline-kernel", default="auto",
                     help="kernel the roofline record is taken on (auto = the one with the most time in the step)")
+    ap.add_argument("--node-groups", type=int, default=0,
+                    help="split the nodes' forward/backward passes into this many groups on parallel streams "
+                         "(0 = two groups from 32 nodes on, else one: measured best per workload)")
     ap.add_argument("--cpu-nodes", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", dest="extra", action="store_false",

@@ -413,9 +413,10 @@ def lpdt_colsum(nodes, B, Cc, x, out, out_node_stride):
 
 
 # Optional call log: while RECORD is a list, every entry-point call appends (name, function, args, kwargs,
-# contraction kernel launched or "").  The logged calls can be re-issued later on the same buffers, which is
+# contraction kernel launched or "", node group).  The logged calls can be re-issued later on the same buffers, which is
 # how the benchmark times one kind of call of a whole step in isolation.
 RECORD = None
+GROUP = 0          # node group whose calls are being issued (set by TrainStep; logged with every call)
 
 
 def _with_timing(fn):
@@ -424,7 +425,7 @@ def _with_timing(fn):
     def call(*a, **kw):
         if RECORD is not None:
             r = fn(*a, **kw)
-            RECORD.append((name, fn, a, kw, lpdt_last_kernel() if name.startswith("lpdt_qconv") else ""))
+            RECORD.append((name, fn, a, kw, lpdt_last_kernel() if name.startswith("lpdt_qconv") else "", GROUP))
             return r
         if name in TIMED:
             with timed(name):

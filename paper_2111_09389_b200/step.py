@@ -18,7 +18,7 @@ class TrainStep:
     def __init__(self, ops, d, nodes, batch, in_shape, ren_eps=1e-5, lr=0.1, gamma=1.0,
                  seg_offsets=None, seg_k=None, has_labels=True, grad_rounding=0, seed=0,
                  quantize_wgrad=False, input_grad=False, message_bits=32, recompute_norm_input=False,
-                 device="cuda"):
+                 node_groups=1, device="cuda"):
         if not torch.cuda.is_available():
             raise RuntimeError("TrainStep needs a CUDA device; there is no CPU path")
         self.ops, self.d, self.N, self.B = ops, d, nodes, batch
@@ -34,6 +34,11 @@ class TrainStep:
         # into one shared buffer (same integer sums, same dequantization: bit-identical values).
         self.recompute_norm_input = recompute_norm_input
         self._shared_out = {}
+        # node_groups > 1: the nodes are split into that many contiguous groups whose forward and backward passes
+        # run side by side on streams of their own (the nodes are independent until the gossip mix).  Every call
+        # then covers fewer nodes, and the launches of one group fill the gaps of the others; results do not
+        # change.  Not with stochastic rounding, whose random numbers are keyed by the node's index inside a call.
+        self.node_groups = max(1, min(int(node_groups), nodes)) if not grad_rounding else 1
         dev = torch.device(device)
         N, B = nodes, batch
         f32 = dict(dtype=torch.float32, device=dev)
@@ -92,6 +97,7 @@ class TrainStep:
                          E=torch.empty(N, B, Ho, Wo, op["cout"], **i8), sE=torch.empty(N, **f32),
                          dx=torch.empty(N, B, H, W, op["cin"], **f32),
                          wn=op["cout"] * R * S * op["cin"], wi=wi)
+                b["gacc"] = self.g_acc[self.g_acc_off[wi]:self.g_acc_off[wi] + N * b["wn"]].view(N, b["wn"])
                 if quantize_wgrad:
                     b.update(gq=torch.empty(N, b["wn"], **i8), gs=torch.empty(N, **f32),
                              gw=torch.empty(N, b["wn"], **f32))
@@ -137,6 +143,57 @@ class TrainStep:
         # parameter update.  Captured into the step's CUDA graph the fork and join become graph edges.
         self.ws_side = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
         self.side = torch.cuda.Stream(device=dev)
+        self.groups = []
+        if self.node_groups > 1:
+            bounds = [N * g // self.node_groups for g in range(self.node_groups + 1)]
+            self.groups = [self._node_view(bounds[g], bounds[g + 1], ws_bytes, dev) for g in range(self.node_groups)]
+
+    def _node_view(self, n0, n1, ws_bytes, dev):
+        """A TrainStep over nodes [n0, n1) that shares this one's storage: every per-node tensor is a slice,
+        every convolution descriptor carries the group's node count; it has its own streams and workspaces."""
+        N = self.N
+        c = TrainStep.__new__(TrainStep)
+        c.__dict__.update({k: v for k, v in self.__dict__.items() if not isinstance(v, (torch.Tensor, list, dict))})
+        c.ops, c.w_src, c.w_size, c.w_dst, c.seg_offsets, c.seg_k = (self.ops, self.w_src, self.w_size, self.w_dst,
+                                                                     self.seg_offsets, self.seg_k)
+        c.N, c.node_groups, c.groups, c._shared_out = n1 - n0, 1, [], {}
+        cut = lambda t: t[n0:n1] if isinstance(t, torch.Tensor) and t.dim() > 0 and t.shape[0] == N else t
+        for name in ("params", "grads", "x", "labels", "loss", "dy"):
+            setattr(c, name, cut(getattr(self, name)))
+        c.dev_status = self.dev_status
+        c.ranges = self.ranges[:, n0:n1]
+        c.buf = []
+        for op, b in zip(self.ops, self.buf):
+            cb = {}
+            for k, v in b.items():
+                if k == "desc":
+                    cb[k] = api.conv_desc(n1 - n0, v.B, v.H, v.W, v.Cin, v.Cout, v.R, v.S, v.stride, v.pad)
+                elif k == "ws_ren":
+                    per = v.numel() // N
+                    cb[k] = v[n0 * per:n1 * per]
+                else:
+                    cb[k] = cut(v)
+            c.buf.append(cb)
+        c.ws = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        c.ws_side = torch.empty(ws_bytes, dtype=torch.uint8, device=dev)
+        c.stream = torch.cuda.Stream(device=dev)
+        c.side = torch.cuda.Stream(device=dev)
+        return c
+
+    def _each_group(self, fn):
+        """fn(step) for this step, or for every node group on its own stream between a fork and a join."""
+        if not self.groups:
+            fn(self)
+            return
+        main = torch.cuda.current_stream()
+        for i, g in enumerate(self.groups):
+            g.stream.wait_stream(main)
+            api.GROUP = i + 1
+            with torch.cuda.stream(g.stream):
+                fn(g)
+        api.GROUP = 0
+        for g in self.groups:
+            main.wait_stream(g.stream)
 
     def _conv_out(self, shape, f32):
         """fp32 output buffer of a convolution: one per layer, or (recompute_norm_input) one per distinct
@@ -221,16 +278,26 @@ class TrainStep:
     def _g(self, off):
         return self.grads[:, off:]
 
-    def forward(self):
-        N, B, d = self.N, self.B, self.d
-        cur = self.x
-        cur_range = None          # per-node max|cur| when the producer of cur emitted it
-        saved = []
+    def _prepare(self):
+        """Once per step, all nodes: clear the range accumulators, quantize every layer's weights."""
+        N, d = self.N, self.d
         api.lpdt_fill_zero(self.ranges)
         for lo in range(0, len(self.w_size), 64):        # every layer's weights, 64 tensors per call
             hi = min(lo + 64, len(self.w_size))
             api.lpdt_quantize_batch(self.params, N, d, self.w_src[lo:hi], self.w_size[lo:hi], self.w_dst[lo:hi],
                                     self.qW_all, self.sW_all[lo:hi], self.ws)
+
+    def forward(self):
+        self._prepare()
+        self._each_group(lambda g: g._forward_layers())
+        self.out = self.buf[-1]["out"]
+        return self.out
+
+    def _forward_layers(self):
+        N, B, d = self.N, self.B, self.d
+        cur = self.x
+        cur_range = None          # per-node max|cur| when the producer of cur emitted it
+        saved = []
         for li, (op, b) in enumerate(zip(self.ops, self.buf)):
             k = op["op"]
             if k in ("conv", "linear"):
@@ -277,6 +344,13 @@ class TrainStep:
         return cur
 
     def backward(self):
+        self._each_group(lambda g: g._backward_layers())
+        self._finish_gradients()
+        if self.groups:
+            self.input_grad_out = self.buf[0]["dx"] if self.input_grad else None
+        return self.input_grad_out
+
+    def _backward_layers(self):
         N, B, d = self.N, self.B, self.d
         if self.labels is not None:
             K = self.out.numel() // (N * B)
@@ -285,7 +359,6 @@ class TrainStep:
         g_range = None
         L = len(self.ops)
         sc = []
-        pending_ren = []
         fused_shortcut = False
         ctr = 0
         for li in range(len(self.ops) - 1, -1, -1):
@@ -312,10 +385,8 @@ class TrainStep:
                         api.lpdt_dequantize(b["gq"], N, b["wn"], b["gs"], self._g(op["w_off"]), d)
                     else:
                         # raw sums now, one conversion launch for all layers after the last of them
-                        lo = self.g_acc_off[b["wi"]]
-                        api.lpdt_qconv_bwd_weight(b["desc"], b["E"], b["sE"], b["qA"], b["sA"],
-                                                  dWacc=self.g_acc[lo:lo + N * b["wn"]], ws=self.ws_side,
-                                                  dev_status=self.dev_status)
+                        api.lpdt_qconv_bwd_weight(b["desc"], b["E"], b["sE"], b["qA"], b["sA"], dWacc=b["gacc"],
+                                                  ws=self.ws_side, dev_status=self.dev_status)
                 if li > 0 or self.input_grad:
                     # first convolution of a residual block with an identity shortcut: the block-output gradient
                     # joins this gradient in the contraction's epilogue (no separate residual_add_bwd pass)
@@ -344,7 +415,6 @@ class TrainStep:
                                            self._p(op["p_off"]), self._p(op["p_off"] + Cc), d, b["gmin"],
                                            b["gmax"], b["amin"], b["amax"], b["dx"], None, None, None, d, b["ws_ren"],
                                            amax_out=self.ranges[L + li])
-                pending_ren.append((op, b))
                 g, g_range = b["dx"], self.ranges[L + li]
             elif k == "add":
                 sc.append((g, op))
@@ -362,8 +432,15 @@ class TrainStep:
             elif k == "avgpool":
                 api.lpdt_avgpool_bwd(N, B, op["H"] * op["W"], op["C"], g, b["dx"])
                 g, g_range = b["dx"], None
-        # side stream, after the last weight-gradient contraction: all norm layers' parameter-gradient sums in one
-        # launch, all layers' int32 weight-gradient sums to fp32 in another
+        torch.cuda.current_stream().wait_stream(self.side)      # this group's weight-gradient contractions are done
+        self.input_grad_out = g
+        return g
+
+    def _finish_gradients(self):
+        """After every group's backward pass, all nodes at once on the side stream: all norm layers'
+        parameter-gradient sums in one launch, all layers' int32 weight-gradient sums to fp32 in another."""
+        N, d = self.N, self.d
+        pending_ren = [(op, b) for op, b in zip(self.ops, self.buf) if op["op"] == "ren"]
         self.side.wait_stream(torch.cuda.current_stream())
         with torch.cuda.stream(self.side):
             self._ren_param_sums(pending_ren)
@@ -376,8 +453,6 @@ class TrainStep:
                                                   [b["sE"] for _, b in part], [b["sA"] for _, b in part],
                                                   self.grads, d)
         torch.cuda.current_stream().wait_stream(self.side)      # weight gradients complete before the update
-        self.input_grad_out = g
-        return g
 
     def _ren_param_sums(self, pending):
         """Reduce the Range-EvoNorm parameter-gradient partial sums of the layers in `pending` (current stream):
@@ -406,13 +481,20 @@ class TrainStep:
                                 self.seg_offsets, self.seg_k, self.ws, self.dev_status)
 
     def run(self):
-        self.forward()
-        self.backward()
+        if self.groups:      # one fork for both passes: a group's backward pass follows its own forward pass
+            self._prepare()
+            self._each_group(lambda g: (g._forward_layers(), g._backward_layers()))
+            self.out = self.buf[-1]["out"]
+            self._finish_gradients()
+            self.input_grad_out = self.buf[0]["dx"] if self.input_grad else None
+        else:
+            self.forward()
+            self.backward()
         self.update()
 
     def record(self):
         """Run one step eagerly and return the log of its entry-point calls, in issue order:
-        [(name, function, args, kwargs, contraction kernel or "")].  The calls of a log can be issued
+        [(name, function, args, kwargs, contraction kernel or "", node group)].  The calls of a log can be issued
         again on the buffers the step left behind (every call reads and writes the same tensors)."""
         api.RECORD = log = []
         try:

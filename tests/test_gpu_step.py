@@ -130,10 +130,10 @@ def _subset(wl, sel):
     return sub
 
 
-def _compare_sampled_nodes(wl, sel):
+def _compare_sampled_nodes(wl, sel, **step_options):
     """Full-size GPU step; the oracle recomputes the sampled nodes' gradients and half-steps, and the mix
     is checked through what holds at any size (top-k count, x_hat update, average preservation)."""
-    st = TrainStep.from_workload(wl)
+    st = TrainStep.from_workload(wl, **step_options)
     st.run()
     torch.cuda.synchronize()
     assert int(st.dev_status.item()) == 0
@@ -174,6 +174,11 @@ def test_vgg11_full_size_sampled_nodes():
 
 def test_resnet20_topk_full_size_sampled_nodes():
     _compare_sampled_nodes(wlmod.make_workload("resnet20_topk"), [0, 17, 39])
+
+
+def test_resnet20_topk_full_size_in_the_benchmark_configuration():
+    # two node groups on parallel streams, as bench.py runs this workload: nodes of both groups sampled
+    _compare_sampled_nodes(wlmod.make_workload("resnet20_topk"), [1, 19, 20, 38], node_groups=2)
 
 
 def test_resnet20_layerwise_topk_full_size_sampled_nodes():
@@ -235,3 +240,34 @@ def test_step_keeping_only_8bit_tensors_for_backward(name, nodes, batch):
     ma, mb = a.saved_bytes_per_node(), b.saved_bytes_per_node()
     assert mb["fp32_norm_inputs"] == 0 and ma["fp32_norm_inputs"] > 0
     assert mb["int8_activations"] == ma["int8_activations"] and mb["total"] < ma["total"]
+
+
+@pytest.mark.parametrize("name,nodes,batch,groups", [("resnet20", 5, 4, 2), ("vgg11", 4, 2, 4), ("resnet20_topk", 6, 2, 3),
+                                                     ("conv16", 4, 8, 2)])
+def test_step_with_node_groups_on_separate_streams(name, nodes, batch, groups):
+    """node_groups: the nodes' forward and backward passes split into groups that run side by side on their own
+    streams (uneven group sizes included).  The nodes are independent until the mix, so every result is
+    bit-identical to the one-group step; also as a captured CUDA graph."""
+    wl = wlmod.make_workload(name, nodes=nodes, batch=batch)
+    a = TrainStep.from_workload(wl)
+    b = TrainStep.from_workload(wl, node_groups=groups)
+    assert len(b.groups) == groups
+    a.run(); b.run()
+    torch.cuda.synchronize()
+    assert int(b.dev_status.item()) == 0
+    names = ["grads", "x_half", "x_hat", "x_out"] + (["loss"] if "labels" in wl else [])
+    for t in names:
+        assert torch.equal(getattr(a, t), getattr(b, t)), t
+    for li, op in enumerate(wl["ops"]):
+        if op["op"] in ("conv", "linear"):
+            assert torch.equal(a.buf[li]["E"], b.buf[li]["E"]), f"E{li}"
+    if "dy" in wl:
+        assert torch.equal(a.input_grad_out, b.input_grad_out)
+    # a second step from the same state, eager against graph replay (capture() runs the step once to warm up)
+    b.capture()
+    a.params.copy_(a.x_out)
+    b.params.copy_(a.params); b.x_hat.copy_(a.x_hat)
+    a.run(); b.replay()
+    torch.cuda.synchronize()
+    for t in names:
+        assert torch.equal(getattr(a, t), getattr(b, t)), t
