@@ -331,6 +331,45 @@ lpdt_status lpdt_range_evonorm_bwd_params_batch(int32_t nodes, int32_t B, int32_
                                                 const void *const *ws, const int64_t *grad_offsets,
                                                 float *grads, int64_t grad_node_stride, void *stream);
 
+/* Range-EvoNorm with the requantize step inside (Section 3, "Low Precision Training": activations and layer
+ * gradients travel between layers as 8-bit tensors).  lpdt_range_evonorm_fwd_q8 computes y as
+ * lpdt_range_evonorm_fwd does and ALSO writes y's symmetric 8-bit codes q (int8, shape of y) and per-node scale
+ * (fp32 [nodes]): exactly what lpdt_quantize_with_range(y, max|y|, LPDT_ROUND_NEAREST_EVEN) would write.  y may
+ * be NULL when only the codes are wanted.  lpdt_range_evonorm_bwd_q8 computes dx as lpdt_range_evonorm_bwd does
+ * but writes only its codes q and scale; the parameter gradients (or, with the three pointers NULL, the partial
+ * sums in ws) are those of lpdt_range_evonorm_bwd.  amax_out (nullable, fp32 [nodes]) is overwritten with
+ * max|y| / max|dx| (no caller zeroing here).
+ * One CTA per sample keeps the sample's fp32 result in shared memory until the node-wide range is known; the
+ * CTAs of a node meet through the control block ctl (device memory, lpdt_range_evonorm_q8_ctl_size(nodes)
+ * bytes, 4-byte aligned): ZERO it once before the first call; every call that completes leaves it zero again,
+ * so consecutive calls may share it, concurrent calls may not.  The meeting is a bounded wait: if it ever ran
+ * out, dev_status (nullable device int32) would receive LPDT_ERR_TIMEOUT, the codes of the affected nodes
+ * would be left unwritten and ctl would have to be zeroed again.
+ * lpdt_range_evonorm_fwd_q8_fits / _bwd_q8_fits return 1 when the shape is served: a sample (H*W*C fp32) fits
+ * one CTA's shared memory beside the kernel's scratch, C/groups is a multiple of 4, and the device has room for
+ * 2*B resident CTAs; otherwise the call returns UNSUPPORTED and the two-call form (lpdt_range_evonorm_*
+ * followed by lpdt_quantize_with_range) serves.  x, dy, res, y 16-byte aligned, q 4-byte aligned.
+ * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE (ws or ctl missing or too small), CUDA. */
+size_t lpdt_range_evonorm_q8_ctl_size(int32_t nodes);
+int32_t lpdt_range_evonorm_fwd_q8_fits(int32_t B, int32_t H, int32_t W, int32_t C, int32_t groups);
+lpdt_status lpdt_range_evonorm_fwd_q8(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C,
+                                      int32_t groups, float eps, const float *x,
+                                      const float *v, const float *gamma, const float *beta,
+                                      int64_t param_node_stride, float *y,
+                                      float *gmin, float *gmax, int32_t *argmin, int32_t *argmax,
+                                      float *amax_out, const float *res, int8_t *q, float *scale,
+                                      void *ctl, size_t ctl_bytes, int32_t *dev_status, void *stream);
+int32_t lpdt_range_evonorm_bwd_q8_fits(int32_t B, int32_t H, int32_t W, int32_t C, int32_t groups);
+lpdt_status lpdt_range_evonorm_bwd_q8(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C,
+                                      int32_t groups, float eps, const float *dy, const float *x,
+                                      const float *v, const float *gamma, int64_t param_node_stride,
+                                      const float *gmin, const float *gmax,
+                                      const int32_t *argmin, const int32_t *argmax,
+                                      int8_t *q, float *scale, float *dv, float *dgamma, float *dbeta,
+                                      int64_t grad_node_stride, float *amax_out,
+                                      void *ws, size_t ws_bytes, void *ctl, size_t ctl_bytes,
+                                      int32_t *dev_status, void *stream);
+
 /* ---------------------------------------------------------------------------
  * Comparison layers of Section 3 (the normalization study; not on the 8-bit path).
  *

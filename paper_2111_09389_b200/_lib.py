@@ -47,6 +47,12 @@ SIGNATURES = {
     "lpdt_qconv_bwd_data": (_i32, [C.POINTER(ConvDesc), _vp, _vp, _vp, _vp, _vp, _vp, _vp, _vp, _sz, _vp, _vp]),
     "lpdt_qconv_bwd_weight": (_i32, [C.POINTER(ConvDesc), _vp, _vp, _vp, _vp, _vp, _i64, _vp, _vp, _sz, _vp, _vp]),
     "lpdt_range_evonorm_fwd": (_i32, [_i32] * 6 + [_f32] + [_vp] * 4 + [_i64] + [_vp] * 7 + [_vp]),
+    "lpdt_range_evonorm_q8_ctl_size": (_sz, [_i32]),
+    "lpdt_range_evonorm_fwd_q8_fits": (_i32, [_i32] * 5),
+    "lpdt_range_evonorm_fwd_q8": (_i32, [_i32] * 6 + [_f32] + [_vp] * 4 + [_i64] + [_vp] * 9 + [_vp, _sz, _vp, _vp]),
+    "lpdt_range_evonorm_bwd_q8_fits": (_i32, [_i32] * 5),
+    "lpdt_range_evonorm_bwd_q8": (_i32, [_i32] * 6 + [_f32] + [_vp] * 4 + [_i64] + [_vp] * 9 +
+                                  [_i64, _vp, _vp, _sz, _vp, _sz, _vp, _vp]),
     "lpdt_range_evonorm_bwd_workspace_size": (_sz, [_i32, _i32, _i32]),
     "lpdt_range_evonorm_bwd": (_i32, [_i32] * 6 + [_f32] + [_vp] * 4 + [_i64] + [_vp] * 8 + [_i64, _vp, _vp, _sz, _vp]),
     "lpdt_evonorm_s0_fwd": (_i32, [_i32] * 6 + [_f32] + [_vp] * 4 + [_i64] + [_vp] * 4),

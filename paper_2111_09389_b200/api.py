@@ -12,7 +12,7 @@ from ._lib import ConvDesc, lib
 
 
 # Entry points that enqueue kernels (wrapped for the optional call log and per-call timing).
-LAUNCHING = {"lpdt_quantize", "lpdt_quantize_with_range", "lpdt_quantize_static", "lpdt_quantize_batch", "lpdt_dequantize", "lpdt_qconv_fwd", "lpdt_qconv_fwd_affine", "lpdt_qconv_bwd_data_affine", "lpdt_qconv_bwd_weight_affine", "lpdt_qconv_bwd_data", "lpdt_qconv_bwd_weight", "lpdt_range_evonorm_fwd", "lpdt_range_evonorm_bwd", "lpdt_range_evonorm_bwd_params", "lpdt_range_evonorm_bwd_params_batch", "lpdt_dequantize_acc_batch", "lpdt_gossip_mix", "lpdt_gossip_mix_q8", "lpdt_deepsqueeze_mix", "lpdt_pushsum_debias", "lpdt_sgd_gossip_mix", "lpdt_evonorm_s0_fwd", "lpdt_evonorm_s0_bwd", "lpdt_range_bn_fwd", "lpdt_range_bn_bwd", "lpdt_sgd_update", "lpdt_residual_add", "lpdt_residual_add_bwd", "lpdt_avgpool", "lpdt_avgpool_bwd", "lpdt_maxpool2x2", "lpdt_maxpool2x2_bwd", "lpdt_softmax_ce", "lpdt_colsum", "lpdt_selftest_bounded_wait"}
+LAUNCHING = {"lpdt_quantize", "lpdt_quantize_with_range", "lpdt_quantize_static", "lpdt_quantize_batch", "lpdt_dequantize", "lpdt_qconv_fwd", "lpdt_qconv_fwd_affine", "lpdt_qconv_bwd_data_affine", "lpdt_qconv_bwd_weight_affine", "lpdt_qconv_bwd_data", "lpdt_qconv_bwd_weight", "lpdt_range_evonorm_fwd", "lpdt_range_evonorm_bwd", "lpdt_range_evonorm_fwd_q8", "lpdt_range_evonorm_bwd_q8", "lpdt_range_evonorm_bwd_params", "lpdt_range_evonorm_bwd_params_batch", "lpdt_dequantize_acc_batch", "lpdt_gossip_mix", "lpdt_gossip_mix_q8", "lpdt_deepsqueeze_mix", "lpdt_pushsum_debias", "lpdt_sgd_gossip_mix", "lpdt_evonorm_s0_fwd", "lpdt_evonorm_s0_bwd", "lpdt_range_bn_fwd", "lpdt_range_bn_bwd", "lpdt_sgd_update", "lpdt_residual_add", "lpdt_residual_add_bwd", "lpdt_avgpool", "lpdt_avgpool_bwd", "lpdt_maxpool2x2", "lpdt_maxpool2x2_bwd", "lpdt_softmax_ce", "lpdt_colsum", "lpdt_selftest_bounded_wait"}
 # Kernel launches are counted inside the library (lpdt_launch_count); replays of a captured CUDA graph launch
 # the recorded kernels again without passing through the library, so TrainStep.replay adds them here.
 _REPLAYED = 0
@@ -236,6 +236,38 @@ def lpdt_range_evonorm_fwd(nodes, B, H, W, Cc, groups, eps, x, v, gamma, beta, p
     _check("lpdt_range_evonorm_fwd", lib().lpdt_range_evonorm_fwd(
         nodes, B, H, W, Cc, groups, eps, _ptr(x), _ptr(v), _ptr(gamma), _ptr(beta), param_node_stride,
         _ptr(y), _ptr(gmin), _ptr(gmax), _ptr(argmin), _ptr(argmax), _ptr(amax_out), _ptr(res), _stream()))
+
+
+def lpdt_range_evonorm_q8_ctl_size(nodes):
+    return lib().lpdt_range_evonorm_q8_ctl_size(nodes)
+
+
+def lpdt_range_evonorm_fwd_q8_fits(B, H, W, Cc, groups):
+    return lib().lpdt_range_evonorm_fwd_q8_fits(B, H, W, Cc, groups)
+
+
+def lpdt_range_evonorm_fwd_q8(nodes, B, H, W, Cc, groups, eps, x, v, gamma, beta, param_node_stride, y,
+                              gmin, gmax, argmin, argmax, q, scale, ctl, amax_out=None, res=None, dev_status=None):
+    c, cb = _ws(ctl)
+    _check("lpdt_range_evonorm_fwd_q8", lib().lpdt_range_evonorm_fwd_q8(
+        nodes, B, H, W, Cc, groups, eps, _ptr(x), _ptr(v), _ptr(gamma), _ptr(beta), param_node_stride,
+        _ptr(y), _ptr(gmin), _ptr(gmax), _ptr(argmin), _ptr(argmax), _ptr(amax_out), _ptr(res), _ptr(q), _ptr(scale),
+        c, cb, _ptr(dev_status), _stream()))
+
+
+def lpdt_range_evonorm_bwd_q8_fits(B, H, W, Cc, groups):
+    return lib().lpdt_range_evonorm_bwd_q8_fits(B, H, W, Cc, groups)
+
+
+def lpdt_range_evonorm_bwd_q8(nodes, B, H, W, Cc, groups, eps, dy, x, v, gamma, param_node_stride, gmin,
+                              gmax, argmin, argmax, q, scale, dv, dgamma, dbeta, grad_node_stride, ws, ctl,
+                              amax_out=None, dev_status=None):
+    p, nb = _ws(ws)
+    c, cb = _ws(ctl)
+    _check("lpdt_range_evonorm_bwd_q8", lib().lpdt_range_evonorm_bwd_q8(
+        nodes, B, H, W, Cc, groups, eps, _ptr(dy), _ptr(x), _ptr(v), _ptr(gamma), param_node_stride,
+        _ptr(gmin), _ptr(gmax), _ptr(argmin), _ptr(argmax), _ptr(q), _ptr(scale), _ptr(dv), _ptr(dgamma), _ptr(dbeta),
+        grad_node_stride, _ptr(amax_out), p, nb, c, cb, _ptr(dev_status), _stream()))
 
 
 def lpdt_range_evonorm_bwd_workspace_size(nodes, B, Cc):

@@ -15,6 +15,9 @@
 // HBM-bound: forward moves 4 B in + 4 B out per element, backward 8 B in + 4 B out.
 #include <math.h>
 #include <stdlib.h>
+#include <map>
+#include <mutex>
+#include <tuple>
 #include <cooperative_groups.h>
 #include "common.cuh"
 
@@ -220,23 +223,238 @@ template <int N> __device__ __forceinline__ void cp_async_wait() {
     asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
 }
 
-// MAXT = 256: three CTAs per SM at 80 registers (the thirteen double accumulators of a thread stay in
-// registers); MAXT = 512 serves the rare plans with more than 256 threads.
+// Symmetric 8-bit code of x for a tensor whose max|x| gave inv = 127 / max|x| (round to nearest even, clamped):
+// the arithmetic of the library's quantizer, so that a producer writing codes itself gives the same codes.
+__device__ __forceinline__ int ren_q_sym_rne(float x, float inv) {
+    float r = rintf(__fmul_rn(x, inv));
+    r = fminf(fmaxf(r, -127.f), 127.f);
+    return (int)r;
+}
+
+// ---- Kernels that write 8-bit codes themselves (requantize inside the producer) ------------------------
+// The node-wide range must be known before the first code is written, so the CTAs of a node meet once:
+// one CTA per sample keeps its fp32 result in shared memory, adds its max|.| to the node's word and
+// arrives at the node's counter; when all B samples of the node have arrived every CTA reads the node's
+// maximum and rounds what it holds.  Samples are handed out by a ticket counter in the order in which CTAs
+// start, so whenever a CTA waits for its node, every sample of every earlier node and every lower sample of
+// its own node is held by a CTA that has started; the missing samples are the next tickets and go to the
+// next CTAs that start.  At most B - 1 CTAs can wait for an incomplete node, so with room for at least
+// 2 B resident CTAs (checked by the host) some CTA always makes progress.  The wait is bounded all the
+// same: after kNodeWaitLimitNs it records LPDT_ERR_TIMEOUT and the CTA returns without writing codes.
+//
+// Control block (int32 words, zero before the first launch; the kernels leave it zero again):
+//   [0, nodes) arrivals   [nodes, 2 nodes) departures   [2 nodes, 3 nodes) bits of max|.|
+//   [3 nodes] ticket      [3 nodes + 1] CTAs finished
+constexpr unsigned long long kNodeWaitLimitNs = 2000000000ull;
+
+__device__ __forceinline__ unsigned long long ren_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ int ld_acquire_gpu(const int *p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Sample index for this CTA: the next ticket, or -1 (with LPDT_ERR_INVALID_ARG recorded) when the control
+// block was not zero at launch and the ticket is no sample of this call.  Every thread of the CTA must call.
+__device__ __forceinline__ int take_ticket(int *ctl, int nodes, int B, int32_t *dev_status) {
+    __shared__ int s_ticket;
+    if (threadIdx.x == 0) {
+        int tk = atomicAdd(ctl + 3 * nodes, 1);
+        if (tk < 0 || tk >= nodes * B) {
+            if (dev_status) atomicExch(dev_status, (int32_t)LPDT_ERR_INVALID_ARG);
+            tk = -1;
+        }
+        s_ticket = tk;
+    }
+    __syncthreads();
+    return s_ticket;
+}
+
+// Meet the other samples of the node, then round the held sample (n_el fp32 values at `hold`, maximum
+// magnitude `cta_max` as found by this thread) to codes at q.  Every thread of the CTA must call.
+__device__ __forceinline__ void node_meet_and_quantize(float cta_max, const float *hold, int n_el, int nodes, int B,
+                                                       int node, int64_t sample, int *ctl, int8_t *__restrict__ q,
+                                                       float *__restrict__ scale, float *__restrict__ amax_out,
+                                                       int32_t *dev_status) {
+    __shared__ float s_warp[32];
+    __shared__ float s_node_amax;
+    __shared__ int s_abort;
+    const int T = blockDim.x, t = threadIdx.x;
+    cta_max = warp_max(cta_max);
+    if ((t & 31) == 0) s_warp[t >> 5] = cta_max;
+    __syncthreads();                                     // also: the held sample is complete
+    if (t < 32) {
+        float m = t < ((T + 31) >> 5) ? s_warp[t] : 0.f;
+        m = warp_max(m);
+        if (t == 0) {
+            int *arrive = ctl + node;
+            unsigned *bits = reinterpret_cast<unsigned *>(ctl + 2 * nodes + node);
+            atomicMax(bits, __float_as_uint(m));         // non-negative floats order like their bit patterns
+            __threadfence();
+            atomicAdd(arrive, 1);
+            int ok = 1;
+            if (ld_acquire_gpu(arrive) < B) {
+                const unsigned long long t0 = ren_timer_ns();
+                unsigned spins = 0;
+                while (ld_acquire_gpu(arrive) < B) {
+                    __nanosleep(64);
+                    if ((++spins & 63u) == 0 && ren_timer_ns() - t0 > kNodeWaitLimitNs) {
+                        if (dev_status) atomicExch(dev_status, (int32_t)LPDT_ERR_TIMEOUT);
+                        ok = 0;
+                        break;
+                    }
+                }
+            }
+            s_abort = !ok;
+            s_node_amax = __uint_as_float(*reinterpret_cast<volatile unsigned *>(bits));
+        }
+    }
+    __syncthreads();
+    if (s_abort) return;
+    const float amax = s_node_amax;
+    float s, inv;
+    if (amax == 0.f) { s = 1.f; inv = 0.f; }
+    else { s = __fdiv_rn(amax, 127.f); inv = __fdiv_rn(127.f, amax); }
+    const float4 *h4 = reinterpret_cast<const float4 *>(hold);
+    char4 *q4 = reinterpret_cast<char4 *>(q + sample * (int64_t)n_el);
+    for (int i = t; i < n_el / 4; i += T) {
+        const float4 a = h4[i];
+        q4[i] = make_char4((signed char)ren_q_sym_rne(a.x, inv), (signed char)ren_q_sym_rne(a.y, inv),
+                           (signed char)ren_q_sym_rne(a.z, inv), (signed char)ren_q_sym_rne(a.w, inv));
+    }
+    if (t == 0) {
+        // the last sample of the node to get here clears the node's words (everybody has read the maximum
+        // by then) and writes the scale; the last CTA of the grid clears the ticket
+        if (atomicAdd(ctl + nodes + node, 1) == B - 1) {
+            scale[node] = s;
+            if (amax_out) amax_out[node] = amax;
+            ctl[node] = 0; ctl[nodes + node] = 0; ctl[2 * nodes + node] = 0;
+        }
+        __threadfence();
+        if (atomicAdd(ctl + 3 * nodes + 1, 1) == nodes * B - 1) { ctl[3 * nodes] = 0; ctl[3 * nodes + 1] = 0; }
+    }
+}
+
+// Forward that also hands y on as 8-bit codes: one CTA per sample.  The sample arrives in shared memory by
+// asynchronous copies (all of it in flight at once), its group extrema are found there, y replaces x in
+// place (and goes to global memory as fp32 only when `y` is given), then the node's CTAs meet and every CTA
+// rounds its sample.  x is read from global memory once: 4 B in and 1 B out per element when only the codes
+// are wanted.  Vector columns of 4 channels only.
+template <bool RES>
+__global__ void __launch_bounds__(256, 3)
+ren_fwd_q8_kernel(int HW, int C, int groups, float eps, float Cst,
+                  const float *__restrict__ x, const float *__restrict__ v,
+                  const float *__restrict__ gamma, const float *__restrict__ beta, int64_t pstride,
+                  int nodes, int B, float *__restrict__ y, float *__restrict__ gmin, float *__restrict__ gmax,
+                  int32_t *__restrict__ argmin, int32_t *__restrict__ argmax, float *__restrict__ amax_out,
+                  const float *__restrict__ res, int8_t *__restrict__ q, float *__restrict__ scale,
+                  int *ctl, int32_t *dev_status, unsigned hold_off) {
+    constexpr int V = 4;
+    pdl_enter();
+    extern __shared__ unsigned char smem_raw[];
+    const int T = blockDim.x, t = threadIdx.x;
+    Ext *s_mn = reinterpret_cast<Ext *>(smem_raw);
+    Ext *s_mx = s_mn + T;
+    Ext *g_mn = s_mx + T;
+    Ext *g_mx = g_mn + groups;
+    float *hold = reinterpret_cast<float *>(smem_raw + hold_off);
+    const int CV = C / V, cpg = C / groups;
+    const int col = t % CV, row0 = t / CV, rstep = T / CV;
+    const int c0 = col * V, grp = c0 / cpg;
+    const int n_el = HW * C;
+    const int64_t sample = take_ticket(ctl, nodes, B, dev_status);
+    if (sample < 0) return;
+    const int node = (int)(sample / B);
+    {
+        const float *xs = x + sample * (int64_t)n_el;
+        for (int p = row0; p < HW; p += rstep) cp_async16(hold + p * C + c0, xs + (int64_t)p * C + c0);
+        cp_async_commit();
+    }
+    float vc[V], gc[V], bc[V];
+#pragma unroll
+    for (int k = 0; k < V; ++k) {
+        vc[k] = v[(int64_t)node * pstride + c0 + k];
+        gc[k] = gamma[(int64_t)node * pstride + c0 + k];
+        bc[k] = beta[(int64_t)node * pstride + c0 + k];
+    }
+    const float *rs = RES ? res + sample * (int64_t)n_el : nullptr;
+    float *ys = y ? y + sample * (int64_t)n_el : nullptr;
+    cp_async_wait<0>();
+    // every thread reads only what its own copies brought: no barrier needed here
+    Ext mn, mx; mn.v = INFINITY; mn.idx = 0x7fffffff; mx.v = -INFINITY; mx.idx = 0x7fffffff;
+    for (int p = row0; p < HW; p += rstep) {
+        const float4 a = *reinterpret_cast<const float4 *>(hold + p * C + c0);
+        const float xv[V] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+            const int idx = p * C + c0 + j;
+            if (xv[j] > mx.v) { mx.v = xv[j]; mx.idx = idx; }
+            if (xv[j] < mn.v) { mn.v = xv[j]; mn.idx = idx; }
+        }
+    }
+    reduce_groups<V>(mn, mx, s_mn, s_mx, g_mn, g_mx, CV, cpg, groups);
+    if (t < groups) {
+        const int64_t sg = sample * groups + t;
+        gmin[sg] = g_mn[t].v; gmax[sg] = g_mx[t].v; argmin[sg] = g_mn[t].idx; argmax[sg] = g_mx[t].idx;
+    }
+    const float rng = __fsub_rn(g_mx[grp].v, g_mn[grp].v);
+    const float D = __fadd_rn(__fmul_rn(Cst, rng), eps);
+    const float invD = __fdiv_rn(1.f, D);
+    float ymax = 0.f;
+    auto emit = [&](int pp, const float (&rv)[V]) {
+        const float4 a = *reinterpret_cast<const float4 *>(hold + pp * C + c0);
+        const float xv[V] = {a.x, a.y, a.z, a.w};
+        float yv[V];
+#pragma unroll
+        for (int j = 0; j < V; ++j) {
+            float u = __fmul_rn(vc[j], xv[j]);
+            float m = __fmul_rn(xv[j], hsig(u));
+            yv[j] = __fadd_rn(__fmul_rn(__fmul_rn(gc[j], m), invD), bc[j]);
+            if (RES) yv[j] = __fadd_rn(yv[j], rv[j]);
+            ymax = fmaxf(ymax, fabsf(yv[j]));
+        }
+        *reinterpret_cast<float4 *>(hold + pp * C + c0) = make_float4(yv[0], yv[1], yv[2], yv[3]);
+        if (ys) VecLoad<V>::st(ys + (int64_t)pp * C + c0, yv);
+    };
+    constexpr int kU = RES ? 4 : 1;
+    int p = row0;
+    for (; p + (kU - 1) * rstep < HW; p += kU * rstep) {
+        float rv[kU][V];
+#pragma unroll
+        for (int j = 0; j < kU; ++j)
+            if (RES) VecLoad<V>::ld(rs + (int64_t)(p + j * rstep) * C + c0, rv[j]);
+#pragma unroll
+        for (int j = 0; j < kU; ++j) emit(p + j * rstep, rv[j]);
+    }
+    for (; p < HW; p += rstep) {
+        float rv[V];
+        if (RES) VecLoad<V>::ld(rs + (int64_t)p * C + c0, rv);
+        emit(p, rv);
+    }
+    node_meet_and_quantize(ymax, hold, n_el, nodes, B, node, sample, ctl, q, scale, amax_out, dev_status);
+}
+
+// Backward of one sample by the whole CTA: the local term of dx and the correction at the group extrema go to
+// `dxs` (the sample's place in global memory, or a copy of it held in shared memory), the per-sample partial
+// sums of the parameter gradients to `acc`; `dmax` takes max|dx|.  Leaves no asynchronous copy pending.
 // DEPTH > 0 (V = 4 only): every thread keeps its next DEPTH rows of x and dy in flight as asynchronous copies into
 // a private shared-memory ring, so the bytes in flight per SM (what a streaming kernel of 13-60 us lives
 // on) no longer depend on the register budget; the first DEPTH rows are requested before the group
 // statistics and parameters are read.  DEPTH = 0: rows are loaded into registers, two per trip.
-template <int V, int MAXT, int DEPTH>
-__global__ void __launch_bounds__(MAXT, MAXT == 256 ? 3 : 1)
-ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
-               const float *__restrict__ dy, const float *__restrict__ x,
-               const float *__restrict__ v, const float *__restrict__ gamma, int64_t pstride, int B,
-               const float *__restrict__ gmin, const float *__restrict__ gmax,
-               const int32_t *__restrict__ argmin, const int32_t *__restrict__ argmax,
-               float *__restrict__ dx, double *__restrict__ acc /*[nodes][B][3][C] per-sample partial sums*/,
-               float *__restrict__ amax_out) {
-    pdl_enter();
-    extern __shared__ unsigned char smem_raw[];
+// XHOLD (with DEPTH > 0): the sample's x has been requested into `dxs` (shared memory) as the oldest pending
+// copy group; only dy goes through the ring, and dx overwrites x in place.
+template <int V, int DEPTH, bool XHOLD = false>
+__device__ __forceinline__ void ren_bwd_sample(unsigned char *smem_raw, int HW, int C, int groups, float eps, float Cst,
+                                               const float *__restrict__ dy, const float *__restrict__ x,
+                                               const float *__restrict__ v, const float *__restrict__ gamma,
+                                               int64_t pstride, const float *__restrict__ gmin,
+                                               const float *__restrict__ gmax, const int32_t *__restrict__ argmin,
+                                               const int32_t *__restrict__ argmax, double *__restrict__ acc,
+                                               int64_t sample, int node, float *dxs, float &dmax) {
     const int T = blockDim.x, t = threadIdx.x;
     // When the column count divides the warp, lanes that share a column are folded with shuffles and
     // every warp keeps its own partial sums (no atomics, fixed order); otherwise one shared set of
@@ -246,24 +464,22 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
     double *s_ch = reinterpret_cast<double *>(smem_raw);      // [nsets][3][C]
     double *s_S = s_ch + nsets * 3 * C;                       // [T]
     double *g_S = s_S + T;                                    // [groups]
-    // ring of DEPTH slots: slot s holds, for every thread, 16 bytes of x and 16 bytes of dy
+    // ring of DEPTH slots: slot s holds, for every thread, 16 bytes of x and 16 bytes of dy (XHOLD: of dy)
+    constexpr int kPerSlot = XHOLD ? 1 : 2;
     float4 *ring = reinterpret_cast<float4 *>(smem_raw + (((size_t)(nsets * 3 * C + T + groups) * sizeof(double) + 15) & ~(size_t)15));
     const int CV = C / V, cpg = C / groups;
     const int col = t % CV, row0 = t / CV, rstep = T / CV;
     const int c0 = col * V, grp = c0 / cpg;
-    const int64_t sample = blockIdx.x;
-    const int node = (int)(sample / B);
     const float *xs = x + sample * (int64_t)HW * C;
     const float *dys = dy + sample * (int64_t)HW * C;
-    float *dxs = dx + sample * (int64_t)HW * C;
     const int iters = (HW - 1) / rstep + 1;          // same trip count for every thread (rows are predicated)
     auto request = [&](int j) {                      // row j of this thread -> slot j % DEPTH; one group per row, even when empty
         if (DEPTH > 0) {
             const int p = row0 + j * rstep;
             if (j < iters && p < HW) {
-                float4 *slot = ring + (size_t)(j % (DEPTH > 0 ? DEPTH : 1)) * 2 * T + t;
-                cp_async16(slot, xs + (int64_t)p * C + c0);
-                cp_async16(slot + T, dys + (int64_t)p * C + c0);
+                float4 *slot = ring + (size_t)(j % (DEPTH > 0 ? DEPTH : 1)) * kPerSlot * T + t;
+                if (!XHOLD) cp_async16(slot, xs + (int64_t)p * C + c0);
+                cp_async16(slot + (kPerSlot - 1) * T, dys + (int64_t)p * C + c0);
             }
             cp_async_commit();
         }
@@ -291,7 +507,6 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
     // max|dx| for the consumer's quantizer: the two extremum positions are left out here and
     // added after their correction
     const int g_amx = argmax[sg], g_amn = argmin[sg];
-    float dmax = 0.f;
     double S = 0.0;
     double fb[V], fg[V], fv[V];
 #pragma unroll
@@ -321,8 +536,9 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
             cp_async_wait<(DEPTH > 0 ? DEPTH - 1 : 0)>();                // the oldest pending group, row j, has landed
             const int p = row0 + j * rstep;
             if (p < HW) {
-                const float4 *slot = ring + (size_t)(j % (DEPTH > 0 ? DEPTH : 1)) * 2 * T + t;
-                const float4 a = slot[0], b = slot[T];
+                const float4 *slot = ring + (size_t)(j % (DEPTH > 0 ? DEPTH : 1)) * kPerSlot * T + t;
+                const float4 a = XHOLD ? *reinterpret_cast<const float4 *>(dxs + (size_t)p * C + c0) : slot[0];
+                const float4 b = slot[(kPerSlot - 1) * T];
                 const float xa[4] = {a.x, a.y, a.z, a.w}, da[4] = {b.x, b.y, b.z, b.w};
                 term(p, reinterpret_cast<const float (&)[V]>(xa), reinterpret_cast<const float (&)[V]>(da));
             }
@@ -396,7 +612,63 @@ ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
             dmax = fmaxf(dmax, fabsf(dxs[amx]));
         }
     }
+}
+
+// One CTA per (node, sample).  MAXT = 256: three CTAs per SM at 80 registers (the thirteen double accumulators
+// of a thread stay in registers); MAXT = 512 serves the rare plans with more than 256 threads.
+template <int V, int MAXT, int DEPTH>
+__global__ void __launch_bounds__(MAXT, MAXT == 256 ? 3 : 1)
+ren_bwd_kernel(int HW, int C, int groups, float eps, float Cst,
+               const float *__restrict__ dy, const float *__restrict__ x,
+               const float *__restrict__ v, const float *__restrict__ gamma, int64_t pstride, int B,
+               const float *__restrict__ gmin, const float *__restrict__ gmax,
+               const int32_t *__restrict__ argmin, const int32_t *__restrict__ argmax,
+               float *__restrict__ dx, double *__restrict__ acc /*[nodes][B][3][C] per-sample partial sums*/,
+               float *__restrict__ amax_out) {
+    pdl_enter();
+    extern __shared__ unsigned char smem_raw[];
+    const int64_t sample = blockIdx.x;
+    const int node = (int)(sample / B);
+    float dmax = 0.f;
+    ren_bwd_sample<V, DEPTH>(smem_raw, HW, C, groups, eps, Cst, dy, x, v, gamma, pstride, gmin, gmax, argmin, argmax, acc,
+                             sample, node, dx + sample * (int64_t)HW * C, dmax);
     if (amax_out) block_amax_to(dmax, amax_out + node);
+}
+
+// Backward that hands the layer gradient on as 8-bit codes: one CTA per sample.  x arrives in shared memory
+// by asynchronous copies (all of it in flight at once), dy through the ring; dx replaces x in place and never
+// reaches global memory as fp32 - the node's CTAs meet and every CTA rounds its sample: 8 B read and 1 B
+// written per element instead of 8 + 4 and another 4 + 1 in a separate quantizer launch.  The codes equal
+// those of the two-kernel form bit for bit (same dx, same maximum, same rounding).
+template <int MAXT, int MINB, int DEPTH>
+__global__ void __launch_bounds__(MAXT, MINB)
+ren_bwd_q8_kernel(int HW, int C, int groups, float eps, float Cst,
+                  const float *__restrict__ dy, const float *__restrict__ x,
+                  const float *__restrict__ v, const float *__restrict__ gamma, int64_t pstride, int nodes, int B,
+                  const float *__restrict__ gmin, const float *__restrict__ gmax,
+                  const int32_t *__restrict__ argmin, const int32_t *__restrict__ argmax,
+                  double *__restrict__ acc, int8_t *__restrict__ q, float *__restrict__ scale,
+                  float *__restrict__ amax_out, int *ctl, int32_t *dev_status,
+                  unsigned hold_off /*byte offset of the held sample*/) {
+    constexpr int V = 4;
+    pdl_enter();
+    extern __shared__ unsigned char smem_raw[];
+    const int T = blockDim.x, t = threadIdx.x;
+    const int64_t sample = take_ticket(ctl, nodes, B, dev_status);
+    if (sample < 0) return;
+    const int node = (int)(sample / B);
+    float *hold = reinterpret_cast<float *>(smem_raw + hold_off);
+    const int n_el = HW * C;
+    {
+        const int CV = C / V, col = t % CV, row0 = t / CV, rstep = T / CV, c0 = col * V;
+        const float *xs = x + sample * (int64_t)n_el;
+        for (int p = row0; p < HW; p += rstep) cp_async16(hold + p * C + c0, xs + (int64_t)p * C + c0);
+        cp_async_commit();
+    }
+    float dmax = 0.f;
+    ren_bwd_sample<V, DEPTH, true>(smem_raw, HW, C, groups, eps, Cst, dy, x, v, gamma, pstride, gmin, gmax, argmin, argmax,
+                                   acc, sample, node, hold, dmax);
+    node_meet_and_quantize(dmax, hold, n_el, nodes, B, node, sample, ctl, q, scale, amax_out, dev_status);
 }
 
 // Sum the per-sample partials of a node and round once.  One warp per output: lane l adds samples
@@ -594,6 +866,193 @@ extern "C" lpdt_status lpdt_range_evonorm_bwd(int32_t nodes, int32_t B, int32_t 
     }
     launch_k(fns[pl.V == 4 ? 1 : 0][pl.threads > 256 ? 1 : depth == 6 ? 2 : 0], grid, pl.threads, smem, st, H * W, C, groups, eps, Cst, dy, x,
              v, gamma, pstride, B, gmin, gmax, argmin, argmax, dx, acc, amax_out);
+    LPDT_LAUNCH_CHECK();
+    if (deferred) return LPDT_OK;
+    launch_k(ren_bwd_finalize, (nodes * 3 * C + 7) / 8, 256, 0, st, acc, nodes, B, C, dv, dgamma, dbeta, gstride);
+    LPDT_LAUNCH_CHECK();
+    return LPDT_OK;
+}
+
+namespace lpdt {
+
+using RenFwdQ8Fn = void (*)(int, int, int, float, float, const float *, const float *, const float *, const float *, int64_t,
+                            int, int, float *, float *, float *, int32_t *, int32_t *, float *, const float *, int8_t *,
+                            float *, int *, int32_t *, unsigned);
+using RenBwdQ8Fn = void (*)(int, int, int, float, float, const float *, const float *, const float *, const float *, int64_t,
+                            int, int, const float *, const float *, const int32_t *, const int32_t *, double *, int8_t *,
+                            float *, float *, int *, int32_t *, unsigned);
+
+struct RenQ8Plan { int threads, depth; unsigned hold_off; size_t smem; RenBwdQ8Fn bwd; };
+
+static int q8_threads_forced() {
+    static int tforce = -1;
+    if (tforce < 0) { const char *e = getenv("LPDT_REN_Q8_THREADS"); tforce = e ? atoi(e) : 0; }
+    return tforce;
+}
+
+// CTAs of this kernel, CTA size and shared memory that can be resident on the device at once (asked of the
+// driver once per shape and device).  The kernels that meet per node need room for 2 B of them.
+static int q8_resident_ctas(const void *fn, int threads, size_t smem) {
+    static std::mutex mu;
+    static std::map<std::tuple<int, const void *, int, size_t>, int> seen;
+    std::lock_guard<std::mutex> lock(mu);
+    int d = 0;
+    (void)cudaGetDevice(&d);
+    const auto key = std::make_tuple(d, fn, threads, smem);
+    auto it = seen.find(key);
+    if (it == seen.end()) {
+        int per_sm = 0, sms = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, fn, threads, smem) != cudaSuccess ||
+            cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, d) != cudaSuccess) {
+            (void)cudaGetLastError();
+            per_sm = 0;
+        }
+        it = seen.emplace(key, per_sm * sms).first;
+    }
+    return it->second;
+}
+
+static bool q8_kernel_attrs(const void *fn) {
+    return cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, 226 * 1024) == cudaSuccess &&
+           cudaFuncSetAttribute(fn, cudaFuncAttributePreferredSharedMemoryCarveout, (int)cudaSharedmemCarveoutMaxShared) ==
+               cudaSuccess;
+}
+
+// Launch shape of the forward that writes 8-bit codes: shared memory [extrema scratch | the sample].
+static bool ren_fwd_q8_plan(int B, int HW, int C, int groups, bool res, RenQ8Plan *out) {
+    if (C % 4 || (C / groups) % 4 || (int64_t)HW * C > (1 << 24)) return false;
+    static PerDeviceOnce attr;
+    int dev;
+    if (attr.pending(&dev)) {
+        if (!q8_kernel_attrs((const void *)ren_fwd_q8_kernel<false>) || !q8_kernel_attrs((const void *)ren_fwd_q8_kernel<true>)) {
+            (void)cudaGetLastError();
+            return false;
+        }
+        attr.mark(dev);
+    }
+    const void *fn = res ? (const void *)ren_fwd_q8_kernel<true> : (const void *)ren_fwd_q8_kernel<false>;
+    const size_t hold = (size_t)HW * C * 4;
+    int cap = hold <= 16 * 1024 ? 128 : 256;
+    const int tf = q8_threads_forced();
+    if (tf == 128 || tf == 256) cap = tf;
+    RenPlan pl;
+    if (!plan(C, groups, true, &pl, cap) || pl.V != 4 || pl.threads > 256) return false;
+    const size_t scratch = align_up((size_t)(2 * pl.threads + 2 * groups) * sizeof(Ext), 16);
+    const size_t smem = scratch + hold;
+    if (scratch > 48 * 1024 || smem > 226 * 1024) return false;
+    if (q8_resident_ctas(fn, pl.threads, smem) < 2 * B) return false;
+    out->threads = pl.threads; out->depth = 0; out->hold_off = (unsigned)scratch; out->smem = smem; out->bwd = nullptr;
+    return true;
+}
+
+// Launch shape of the backward that writes 8-bit codes: shared memory [sums | dy ring | the sample].
+static bool ren_bwd_q8_plan(int B, int HW, int C, int groups, RenQ8Plan *out) {
+    if (C % 4 || (C / groups) % 4 || (int64_t)HW * C > (1 << 24)) return false;
+    // <threads, CTAs per SM the register budget is compiled for, ring depth>
+    static const RenBwdQ8Fn fns[3] = {ren_bwd_q8_kernel<256, 3, 8>, ren_bwd_q8_kernel<256, 3, 4>, ren_bwd_q8_kernel<384, 2, 4>};
+    static PerDeviceOnce attr;
+    int dev;
+    if (attr.pending(&dev)) {
+        for (int i = 0; i < 3; ++i)
+            if (!q8_kernel_attrs((const void *)fns[i])) { (void)cudaGetLastError(); return false; }
+        attr.mark(dev);
+    }
+    const size_t hold = (size_t)HW * C * 4;
+    int cap = hold <= 32 * 1024 && C / 4 <= 32 ? 128 : 256;
+    const int tf = q8_threads_forced();
+    if (tf == 128 || tf == 256 || tf == 384) cap = tf;
+    RenPlan pl;
+    if (!plan(C, groups, true, &pl, cap) || pl.V != 4 || pl.threads > 384) return false;
+    const int cv = C / 4;
+    const int nsets = (cv <= 32 && 32 % cv == 0) ? pl.threads / 32 : 1;
+    const size_t sums = align_up((size_t)(nsets * 3 * C + pl.threads + groups) * sizeof(double), 16);
+    if (sums > 48 * 1024) return false;
+    static int dforce = -1;
+    if (dforce < 0) { const char *e = getenv("LPDT_REN_Q8_DEPTH"); dforce = e ? atoi(e) : 0; }
+    int depth = pl.threads > 256 ? 4 : 8;
+    if (dforce == 4 || (dforce == 8 && pl.threads <= 256)) depth = dforce;
+    const size_t smem = sums + (size_t)depth * pl.threads * 16 + hold;
+    if (smem > 226 * 1024) return false;
+    RenBwdQ8Fn fn = pl.threads > 256 ? fns[2] : depth == 8 ? fns[0] : fns[1];
+    if (q8_resident_ctas((const void *)fn, pl.threads, smem) < 2 * B) return false;
+    out->threads = pl.threads; out->depth = depth; out->hold_off = (unsigned)(sums + (size_t)depth * pl.threads * 16);
+    out->smem = smem; out->bwd = fn;
+    return true;
+}
+
+}  // namespace lpdt
+
+extern "C" size_t lpdt_range_evonorm_q8_ctl_size(int32_t nodes) {
+    return align_up((size_t)(3 * (size_t)(nodes > 0 ? nodes : 1) + 2) * sizeof(int32_t), 256);
+}
+
+extern "C" int32_t lpdt_range_evonorm_fwd_q8_fits(int32_t B, int32_t H, int32_t W, int32_t C, int32_t groups) {
+    if (B <= 0 || H <= 0 || W <= 0 || C <= 0 || groups <= 0 || C % groups || C / groups < 2) return 0;
+    if ((int64_t)H * W * C > 0x7fffffff) return 0;
+    RenQ8Plan qp;
+    return ren_fwd_q8_plan(B, H * W, C, groups, false, &qp) && ren_fwd_q8_plan(B, H * W, C, groups, true, &qp) ? 1 : 0;
+}
+
+extern "C" lpdt_status lpdt_range_evonorm_fwd_q8(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C,
+                                                 int32_t groups, float eps, const float *x, const float *v,
+                                                 const float *gamma, const float *beta, int64_t pstride,
+                                                 float *y, float *gmin, float *gmax, int32_t *argmin,
+                                                 int32_t *argmax, float *amax_out, const float *res, int8_t *q,
+                                                 float *scale, void *ctl, size_t ctl_bytes, int32_t *dev_status,
+                                                 void *stream) {
+    LPDT_CHECK_ARG(nodes >= 0 && B >= 0 && H > 0 && W > 0 && C > 0 && groups > 0);
+    LPDT_CHECK_ARG(C % groups == 0 && C / groups >= 2);
+    if (nodes == 0 || B == 0) return LPDT_OK;
+    LPDT_CHECK_ARG(x && v && gamma && beta && gmin && gmax && argmin && argmax && q && scale);
+    LPDT_CHECK_ARG(pstride >= C || nodes == 1);
+    if ((int64_t)H * W * C > 0x7fffffff || (int64_t)nodes * B > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
+    if (!ctl || ctl_bytes < lpdt_range_evonorm_q8_ctl_size(nodes) || !aligned(ctl, 4)) return LPDT_ERR_WORKSPACE;
+    if (!aligned(x, 16) || (y && !aligned(y, 16)) || (res && !aligned(res, 16)) || !aligned(q, 4)) return LPDT_ERR_UNSUPPORTED;
+    RenQ8Plan qp;
+    if (!ren_fwd_q8_plan(B, H * W, C, groups, res != nullptr, &qp)) return LPDT_ERR_UNSUPPORTED;
+    const float Cst = ren_const(C / groups);
+    RenFwdQ8Fn fn = res ? ren_fwd_q8_kernel<true> : ren_fwd_q8_kernel<false>;
+    launch_k(fn, dim3((unsigned)((int64_t)nodes * B)), qp.threads, qp.smem, as_stream(stream), H * W, C, groups, eps, Cst, x, v,
+             gamma, beta, pstride, nodes, B, y, gmin, gmax, argmin, argmax, amax_out, res, q, scale, (int *)ctl, dev_status,
+             qp.hold_off);
+    LPDT_LAUNCH_CHECK();
+    return LPDT_OK;
+}
+
+extern "C" int32_t lpdt_range_evonorm_bwd_q8_fits(int32_t B, int32_t H, int32_t W, int32_t C, int32_t groups) {
+    if (B <= 0 || H <= 0 || W <= 0 || C <= 0 || groups <= 0 || C % groups || C / groups < 2) return 0;
+    if ((int64_t)H * W * C > 0x7fffffff) return 0;
+    RenQ8Plan qp;
+    return ren_bwd_q8_plan(B, H * W, C, groups, &qp) ? 1 : 0;
+}
+
+extern "C" lpdt_status lpdt_range_evonorm_bwd_q8(int32_t nodes, int32_t B, int32_t H, int32_t W, int32_t C,
+                                                 int32_t groups, float eps, const float *dy, const float *x,
+                                                 const float *v, const float *gamma, int64_t pstride,
+                                                 const float *gmin, const float *gmax,
+                                                 const int32_t *argmin, const int32_t *argmax,
+                                                 int8_t *q, float *scale, float *dv, float *dgamma, float *dbeta,
+                                                 int64_t gstride, float *amax_out, void *ws, size_t ws_bytes,
+                                                 void *ctl, size_t ctl_bytes, int32_t *dev_status, void *stream) {
+    LPDT_CHECK_ARG(nodes >= 0 && B >= 0 && H > 0 && W > 0 && C > 0 && groups > 0);
+    LPDT_CHECK_ARG(C % groups == 0 && C / groups >= 2);
+    if (nodes == 0 || B == 0) return LPDT_OK;
+    LPDT_CHECK_ARG(dy && x && v && gamma && gmin && gmax && argmin && argmax && q && scale);
+    const bool deferred = !dv && !dgamma && !dbeta;
+    LPDT_CHECK_ARG(deferred || (dv && dgamma && dbeta));
+    LPDT_CHECK_ARG((pstride >= C && (deferred || gstride >= C)) || nodes == 1);
+    if ((int64_t)H * W * C > 0x7fffffff || (int64_t)nodes * B > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
+    if (!ws || ws_bytes < lpdt_range_evonorm_bwd_workspace_size(nodes, B, C) || !aligned(ws, 8))
+        return LPDT_ERR_WORKSPACE;
+    if (!ctl || ctl_bytes < lpdt_range_evonorm_q8_ctl_size(nodes) || !aligned(ctl, 4)) return LPDT_ERR_WORKSPACE;
+    if (!aligned(x, 16) || !aligned(dy, 16) || !aligned(q, 4)) return LPDT_ERR_UNSUPPORTED;
+    RenQ8Plan qp;
+    if (!ren_bwd_q8_plan(B, H * W, C, groups, &qp)) return LPDT_ERR_UNSUPPORTED;
+    cudaStream_t st = as_stream(stream);
+    double *acc = (double *)ws;
+    const float Cst = ren_const(C / groups);
+    launch_k(qp.bwd, dim3((unsigned)((int64_t)nodes * B)), qp.threads, qp.smem, st, H * W, C, groups, eps, Cst, dy, x, v, gamma,
+             pstride, nodes, B, gmin, gmax, argmin, argmax, acc, q, scale, amax_out, (int *)ctl, dev_status, qp.hold_off);
     LPDT_LAUNCH_CHECK();
     if (deferred) return LPDT_OK;
     launch_k(ren_bwd_finalize, (nodes * 3 * C + 7) / 8, 256, 0, st, acc, nodes, B, C, dv, dgamma, dbeta, gstride);

@@ -25,6 +25,11 @@ batch 128 so that each fp32 tensor is 268 MB; parameter kernels: 16 nodes with a
   gossip_dense_q8     8-bit messages: + one range pass over x_half and x_hat: 24 B
   gossip_top1pct_q8   range pass + select pass + mix: 32 B
 
+  ren_*_q8_<shape>    Range-EvoNorm with the requantize step inside, on ResNet-20-shaped layers (32 samples per
+                      node; enough nodes for 134 MB per fp32 tensor): forward 4 B read + 1 B written, backward
+                      8 B read + 1 B written; ren_*_then_quantize_<shape> is the two-call form doing the same
+                      job (charged the same bytes, so the two lines compare directly)
+
 One JSON line per case.
 """
 import argparse
@@ -129,10 +134,67 @@ def cases(nodes=8, B=128, H=32, W=32, Cc=64, d=32 * 270410, gossip_nodes=16):
                                                               st), N * d * 32)
 
 
+def q8_cases(B=32):
+    """Range-EvoNorm handing 8-bit codes on, fused and as two calls, on the three ResNet-20 layer shapes."""
+    g = torch.Generator(device="cuda")
+    g.manual_seed(11)
+    for tag, nodes, HW, Cc in (("32x32x16", 64, 32, 16), ("16x16x32", 128, 16, 32), ("8x8x64", 256, 8, 64)):
+        n = B * HW * HW * Cc
+        tot = nodes * n
+        groups = Cc // 8
+        x = torch.randn(nodes, n, generator=g, device="cuda")
+        dy = torch.randn(nodes, n, generator=g, device="cuda")
+        y = torch.empty_like(x)
+        q = torch.empty(nodes, n, dtype=torch.int8, device="cuda")
+        scale = torch.empty(nodes, device="cuda")
+        v = torch.ones(nodes, Cc, device="cuda")
+        gamma = torch.ones(nodes, Cc, device="cuda")
+        beta = torch.zeros(nodes, Cc, device="cuda")
+        gmin = torch.empty(nodes, B, groups, device="cuda")
+        gmax = torch.empty_like(gmin)
+        amin_i = torch.empty(nodes, B, groups, dtype=torch.int32, device="cuda")
+        amax_i = torch.empty_like(amin_i)
+        rng = torch.zeros(nodes, device="cuda")
+        wsb = torch.empty(api.lpdt_range_evonorm_bwd_workspace_size(nodes, B, Cc), dtype=torch.uint8, device="cuda")
+        ctl = torch.zeros(api.lpdt_range_evonorm_q8_ctl_size(nodes), dtype=torch.uint8, device="cuda")
+        status = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+        def fwd2():
+            api.lpdt_range_evonorm_fwd(nodes, B, HW, HW, Cc, groups, 1e-5, x, v, gamma, beta, Cc, y, gmin, gmax, amin_i,
+                                       amax_i, amax_out=rng)
+            api.lpdt_quantize_with_range(y, nodes, n, n, rng, q, scale)
+
+        def fwd1():
+            api.lpdt_range_evonorm_fwd_q8(nodes, B, HW, HW, Cc, groups, 1e-5, x, v, gamma, beta, Cc, None, gmin, gmax,
+                                          amin_i, amax_i, q, scale, ctl, dev_status=status)
+
+        def bwd2():
+            api.lpdt_range_evonorm_bwd(nodes, B, HW, HW, Cc, groups, 1e-5, dy, x, v, gamma, Cc, gmin, gmax, amin_i, amax_i,
+                                       y, None, None, None, Cc, wsb, amax_out=rng)
+            api.lpdt_quantize_with_range(y, nodes, n, n, rng, q, scale)
+
+        def bwd1():
+            api.lpdt_range_evonorm_bwd_q8(nodes, B, HW, HW, Cc, groups, 1e-5, dy, x, v, gamma, Cc, gmin, gmax, amin_i,
+                                          amax_i, q, scale, None, None, None, Cc, wsb, ctl, dev_status=status)
+
+        yield (f"ren_fwd_then_quantize_{tag}", fwd2, tot * 5)
+        if api.lpdt_range_evonorm_fwd_q8_fits(B, HW, HW, Cc, groups):
+            yield (f"ren_fwd_q8_{tag}", fwd1, tot * 5)
+        yield (f"ren_bwd_then_quantize_{tag}", bwd2, tot * 9)
+        if api.lpdt_range_evonorm_bwd_q8_fits(B, HW, HW, Cc, groups):
+            yield (f"ren_bwd_q8_{tag}", bwd1, tot * 9)
+        del x, dy, y, q
+
+
+def all_cases():
+    yield from cases()
+    yield from q8_cases()
+
+
 def sweep(iters=20, peak_gbs=None, out=print, only=None):
     rows = []
-    for name, fn, nbytes in cases():
-        if only and name not in only:
+    for name, fn, nbytes in all_cases():
+        if only and not any(name == o or (o.endswith("*") and name.startswith(o[:-1])) for o in only):
             continue
         ms = _time(fn, iters)
         row = {"case": name, "ms": ms, "algorithmic_bytes": nbytes, "gbs": nbytes / ms * 1e-6}
@@ -147,7 +209,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--iters", type=int, default=20)
     ap.add_argument("--peak-gbs", type=float, default=None, help="HBM copy bandwidth to report fractions against")
-    ap.add_argument("--only", default=None, help="comma-separated case names to run")
+    ap.add_argument("--only", default=None, help="comma-separated case names to run (a trailing * matches a prefix)")
     a = ap.parse_args()
     sweep(a.iters, a.peak_gbs, only=a.only.split(",") if a.only else None)
 

@@ -18,7 +18,7 @@ class TrainStep:
     def __init__(self, ops, d, nodes, batch, in_shape, ren_eps=1e-5, lr=0.1, gamma=1.0,
                  seg_offsets=None, seg_k=None, has_labels=True, grad_rounding=0, seed=0,
                  quantize_wgrad=False, input_grad=False, message_bits=32, recompute_norm_input=False,
-                 node_groups=1, device="cuda"):
+                 node_groups=1, fuse_requantize=False, device="cuda"):
         if not torch.cuda.is_available():
             raise RuntimeError("TrainStep needs a CUDA device; there is no CPU path")
         self.ops, self.d, self.N, self.B = ops, d, nodes, batch
@@ -34,6 +34,12 @@ class TrainStep:
         # into one shared buffer (same integer sums, same dequantization: bit-identical values).
         self.recompute_norm_input = recompute_norm_input
         self._shared_out = {}
+        # True: a Range-EvoNorm layer whose result goes straight into a convolution's quantizer writes the 8-bit
+        # codes itself where the shape allows (lpdt_range_evonorm_fwd_q8 / _bwd_q8: no fp32 round trip, no separate
+        # quantizer launch; identical codes; a quarter fewer launches per ResNet-20 step).  Off by default: on the
+        # benchmark workloads the step measured 2-8 % slower with it (the CTAs of a node have to meet before the
+        # first code can be written).  Not with stochastic rounding of the layer gradients.
+        self.fuse_requantize = bool(fuse_requantize)
         # node_groups > 1: the nodes are split into that many contiguous groups whose forward and backward passes
         # run side by side on streams of their own (the nodes are independent until the gossip mix).  Every call
         # then covers fewer nodes, and the launches of one group fill the gaps of the others; results do not
@@ -114,6 +120,10 @@ class TrainStep:
                 # runs later, on the side stream
                 b["ws_ren"] = torch.empty(api.lpdt_range_evonorm_bwd_workspace_size(N, B, Cc), dtype=torch.uint8,
                                           device=dev)
+                b["q8_fwd"] = self.fuse_requantize and bool(api.lpdt_range_evonorm_fwd_q8_fits(B, H, W, Cc, G))
+                b["q8_bwd"] = (self.fuse_requantize and not grad_rounding and
+                               bool(api.lpdt_range_evonorm_bwd_q8_fits(B, H, W, Cc, G)))
+                b["ctl"] = torch.zeros(api.lpdt_range_evonorm_q8_ctl_size(N), dtype=torch.uint8, device=dev)
             elif k == "add":
                 Ho, Wo = (op["H"] + op["stride"] - 1) // op["stride"], (op["W"] + op["stride"] - 1) // op["stride"]
                 b.update(out=torch.empty(N, B, Ho, Wo, op["C"], **f32))
@@ -171,6 +181,8 @@ class TrainStep:
                 elif k == "ws_ren":
                     per = v.numel() // N
                     cb[k] = v[n0 * per:n1 * per]
+                elif k == "ctl":          # the meeting point of a group's own launches
+                    cb[k] = torch.zeros(api.lpdt_range_evonorm_q8_ctl_size(n1 - n0), dtype=torch.uint8, device=dev)
                 else:
                     cb[k] = cut(v)
             c.buf.append(cb)
@@ -302,7 +314,9 @@ class TrainStep:
             k = op["op"]
             if k in ("conv", "linear"):
                 n_in = cur.numel() // N
-                if cur_range is not None:
+                if b.pop("pre_quantized", False):
+                    pass                            # the norm layer before it wrote qA and sA
+                elif cur_range is not None:
                     api.lpdt_quantize_with_range(cur, N, n_in, n_in, cur_range, b["qA"], b["sA"])
                 else:
                     api.lpdt_quantize(cur, N, n_in, n_in, b["qA"], b["sA"], self.ws)
@@ -318,11 +332,31 @@ class TrainStep:
                 nxt = self.ops[li + 1] if li + 1 < len(self.ops) else None
                 fuse = nxt is not None and nxt["op"] == "add" and nxt["stride"] == 1 and nxt["Ca"] == nxt["C"]
                 res = saved[-1] if fuse else None
-                api.lpdt_range_evonorm_fwd(N, B, op["H"], op["W"], Cc, op["groups"], self.eps, cur,
-                                           self._p(op["p_off"]), self._p(op["p_off"] + Cc),
-                                           self._p(op["p_off"] + 2 * Cc), d, b["out"], b["gmin"], b["gmax"],
-                                           b["amin"], b["amax"], amax_out=self.ranges[li], res=res)
-                cur, cur_range = b["out"], self.ranges[li]
+                # the next operation that computes: a convolution right behind this layer (or behind the fused
+                # shortcut and the block boundary) takes the 8-bit codes from this kernel
+                lj = li + 1
+                if fuse:
+                    lj += 1
+                while lj < len(self.ops) and self.ops[lj]["op"] == "save":
+                    lj += 1
+                to_conv = lj < len(self.ops) and self.ops[lj]["op"] in ("conv", "linear")
+                if b["q8_fwd"] and to_conv:
+                    cb = self.buf[lj]
+                    # y itself is still needed when something else reads it: the shortcut of the next block
+                    keep_y = lj != li + 1
+                    api.lpdt_range_evonorm_fwd_q8(N, B, op["H"], op["W"], Cc, op["groups"], self.eps, cur,
+                                                  self._p(op["p_off"]), self._p(op["p_off"] + Cc),
+                                                  self._p(op["p_off"] + 2 * Cc), d, b["out"] if keep_y else None,
+                                                  b["gmin"], b["gmax"], b["amin"], b["amax"], cb["qA"], cb["sA"],
+                                                  b["ctl"], res=res, dev_status=self.dev_status)
+                    cb["pre_quantized"] = True
+                    cur, cur_range = b["out"], None
+                else:
+                    api.lpdt_range_evonorm_fwd(N, B, op["H"], op["W"], Cc, op["groups"], self.eps, cur,
+                                               self._p(op["p_off"]), self._p(op["p_off"] + Cc),
+                                               self._p(op["p_off"] + 2 * Cc), d, b["out"], b["gmin"], b["gmax"],
+                                               b["amin"], b["amax"], amax_out=self.ranges[li], res=res)
+                    cur, cur_range = b["out"], self.ranges[li]
                 b["fused_add"] = fuse
             elif k == "save":
                 saved.append(cur)
@@ -367,8 +401,10 @@ class TrainStep:
             if k in ("conv", "linear"):
                 if k == "linear":
                     api.lpdt_colsum(N, B, op["cout"], g, self._g(op["b_off"]), d)
-                n_out = g.numel() // N
-                if g_range is not None:
+                n_out = b["E"].numel() // N
+                if b.pop("E_ready", False):
+                    pass                            # the norm layer behind it wrote E and sE
+                elif g_range is not None:
                     api.lpdt_quantize_with_range(g, N, n_out, n_out, g_range, b["E"], b["sE"],
                                                  rounding=self.grad_rounding, seed=self.seed, ctr_offset=ctr)
                 else:
@@ -411,11 +447,21 @@ class TrainStep:
                                        bias=self._p(cop["b_off"]) if cop["op"] == "linear" else None,
                                        bias_node_stride=d, ws=self.ws, dev_status=self.dev_status)
                 # dx only; the parameter-gradient sums stay as partial sums and are reduced on the side stream
-                api.lpdt_range_evonorm_bwd(N, B, op["H"], op["W"], Cc, op["groups"], self.eps, g, b["x"],
-                                           self._p(op["p_off"]), self._p(op["p_off"] + Cc), d, b["gmin"],
-                                           b["gmax"], b["amin"], b["amax"], b["dx"], None, None, None, d, b["ws_ren"],
-                                           amax_out=self.ranges[L + li])
-                g, g_range = b["dx"], self.ranges[L + li]
+                if b["q8_bwd"] and li > 0 and self.ops[li - 1]["op"] == "conv":
+                    # dx goes nowhere but into that convolution's quantizer: its codes are written here
+                    cb = self.buf[li - 1]
+                    api.lpdt_range_evonorm_bwd_q8(N, B, op["H"], op["W"], Cc, op["groups"], self.eps, g, b["x"],
+                                                  self._p(op["p_off"]), self._p(op["p_off"] + Cc), d, b["gmin"],
+                                                  b["gmax"], b["amin"], b["amax"], cb["E"], cb["sE"], None, None, None,
+                                                  d, b["ws_ren"], b["ctl"], dev_status=self.dev_status)
+                    cb["E_ready"] = True
+                    g, g_range = None, None
+                else:
+                    api.lpdt_range_evonorm_bwd(N, B, op["H"], op["W"], Cc, op["groups"], self.eps, g, b["x"],
+                                               self._p(op["p_off"]), self._p(op["p_off"] + Cc), d, b["gmin"],
+                                               b["gmax"], b["amin"], b["amax"], b["dx"], None, None, None, d, b["ws_ren"],
+                                               amax_out=self.ranges[L + li])
+                    g, g_range = b["dx"], self.ranges[L + li]
             elif k == "add":
                 sc.append((g, op))
             elif k == "save":

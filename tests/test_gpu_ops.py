@@ -475,6 +475,124 @@ def test_fused_ranges_feed_the_quantizer_exactly():
         assert torch.equal(q1, q2) and torch.equal(s1, s2)
 
 
+# cases whose sample fits one CTA's shared memory: one to 40 samples per node, ragged pixel counts, 2 to 128
+# vector columns
+REN_Q8_CASES = [(4, 8, 16, 16, 16, 4), (2, 3, 32, 32, 16, 2), (2, 2, 8, 8, 64, 8), (1, 2, 4, 4, 12, 1), (2, 2, 16, 16, 64, 8),
+                (1, 2, 2, 2, 512, 64), (1, 1, 1, 1, 8, 2), (1, 3, 7, 9, 24, 3), (1, 2, 15, 17, 64, 16), (2, 40, 16, 16, 32, 4),
+                (3, 32, 32, 32, 16, 2), (2, 32, 8, 8, 64, 8), (1, 5, 3, 3, 256, 8)]
+
+
+def _ren_q8_check(case, ties, with_res, keep_y):
+    nodes, B, H, W, C, groups = case
+    x, P, dy = _ren_inputs(case, seed=21, ties=ties)
+    eps = 1e-5
+    v, g, b = P[:, :C], P[:, C:2 * C], P[:, 2 * C:3 * C]
+    res = np.random.default_rng(5).standard_normal(x.shape).astype(np.float32) if with_res else None
+    y32, mn, mx, amn, amx = oracle.range_evonorm_fwd(x, v, g, b, groups, eps, "f32")
+    want_y = oracle.residual_add(res, y32) if with_res else y32
+    n = B * H * W * C
+    q_ref, s_ref = oracle.quantize_sym_s8(want_y.reshape(nodes, n))
+    f = lambda *s: torch.empty(*s, dtype=torch.float32, device="cuda")
+    i = lambda *s: torch.empty(*s, dtype=torch.int32, device="cuda")
+    xd, Pd, stride = dev(x), dev(P), P.shape[1]
+    assert api.lpdt_range_evonorm_fwd_q8_fits(B, H, W, C, groups) == 1
+    assert api.lpdt_range_evonorm_bwd_q8_fits(B, H, W, C, groups) == 1
+    ctl = torch.zeros(api.lpdt_range_evonorm_q8_ctl_size(nodes), dtype=torch.uint8, device="cuda")
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    y = torch.full(x.shape, float("nan"), dtype=torch.float32, device="cuda") if keep_y else None
+    gmin, gmax, amin_, amax_ = f(nodes, B, groups), f(nodes, B, groups), i(nodes, B, groups), i(nodes, B, groups)
+    q = torch.full((nodes, n), 99, dtype=torch.int8, device="cuda")
+    sc = f(nodes)
+    rng_out = torch.full((nodes,), -1.0, device="cuda")
+    api.lpdt_range_evonorm_fwd_q8(nodes, B, H, W, C, groups, eps, xd, Pd, Pd[:, C:], Pd[:, 2 * C:], stride, y, gmin, gmax,
+                                  amin_, amax_, q, sc, ctl, amax_out=rng_out, res=None if res is None else dev(res),
+                                  dev_status=status)
+    assert not ctl.any() and int(status.item()) == 0           # the control block is left clean
+    assert np.array_equal(gmin.cpu().numpy(), mn) and np.array_equal(gmax.cpu().numpy(), mx)
+    assert np.array_equal(amin_.cpu().numpy(), amn) and np.array_equal(amax_.cpu().numpy(), amx)
+    if keep_y:
+        assert np.array_equal(y.cpu().numpy(), want_y)
+    assert np.array_equal(rng_out.cpu().numpy(), np.abs(want_y).reshape(nodes, -1).max(1))
+    assert np.array_equal(sc.cpu().numpy(), s_ref)
+    assert np.array_equal(q.cpu().numpy(), q_ref)            # the oracle's norm followed by the oracle's quantizer
+    # backward: the codes of dx.  dx itself matches the oracle to 1e-6 relative, not bit for bit, so the codes are
+    # pinned two ways: they equal the ORACLE's quantizer applied to the dx the plain backward call writes (same
+    # arithmetic inside the fused kernel), and dequantized they sit within half a step of the oracle's dx
+    dx32 = oracle.range_evonorm_bwd(dy, x, v, g, mn, mx, amn, amx, groups, eps, "f32")[0]
+    dx = f(*x.shape)
+    ws = ws_bytes(api.lpdt_range_evonorm_bwd_workspace_size(nodes, B, C))
+    G = torch.zeros(nodes, stride, device="cuda")
+    api.lpdt_range_evonorm_bwd(nodes, B, H, W, C, groups, eps, dev(dy), xd, Pd, Pd[:, C:], stride, gmin, gmax, amin_, amax_,
+                               dx, G, G[:, C:], G[:, 2 * C:], stride, ws)
+    qe_ref, se_ref = oracle.quantize_sym_s8(dx.cpu().numpy().reshape(nodes, n))
+    E = torch.full((nodes, n), 99, dtype=torch.int8, device="cuda")
+    sE = f(nodes)
+    G2 = torch.zeros_like(G)
+    ws2 = ws_bytes(api.lpdt_range_evonorm_bwd_workspace_size(nodes, B, C))
+    rng2 = torch.full((nodes,), -1.0, device="cuda")
+    api.lpdt_range_evonorm_bwd_q8(nodes, B, H, W, C, groups, eps, dev(dy), xd, Pd, Pd[:, C:], stride, gmin, gmax, amin_,
+                                  amax_, E, sE, G2, G2[:, C:], G2[:, 2 * C:], stride, ws2, ctl, amax_out=rng2,
+                                  dev_status=status)
+    assert not ctl.any() and int(status.item()) == 0
+    assert np.array_equal(sE.cpu().numpy(), se_ref)
+    assert np.array_equal(E.cpu().numpy(), qe_ref)
+    assert torch.equal(G2, G)
+    assert np.array_equal(rng2.cpu().numpy(), np.abs(dx.cpu().numpy()).reshape(nodes, -1).max(1))
+    deq = E.cpu().numpy().astype(np.float64) * se_ref[:, None].astype(np.float64)
+    err = np.abs(deq - dx32.reshape(nodes, n).astype(np.float64))
+    bar = 0.5 * se_ref[:, None].astype(np.float64) * (1 + 1e-5) + 1e-6 * np.abs(dx32.reshape(nodes, n)) + 1e-7
+    assert (err <= bar).all()
+    # deferred parameter sums: same partial sums in the workspace
+    G3 = torch.zeros_like(G)
+    api.lpdt_range_evonorm_bwd_q8(nodes, B, H, W, C, groups, eps, dev(dy), xd, Pd, Pd[:, C:], stride, gmin, gmax, amin_,
+                                  amax_, E, sE, None, None, None, stride, ws2, ctl, dev_status=status)
+    api.lpdt_range_evonorm_bwd_params(nodes, B, C, ws2, G3, G3[:, C:], G3[:, 2 * C:], stride)
+    assert torch.equal(G3, G) and np.array_equal(E.cpu().numpy(), qe_ref)
+    assert not ctl.any() and int(status.item()) == 0
+
+
+@pytest.mark.parametrize("case", REN_Q8_CASES)
+@pytest.mark.parametrize("ties", [False, True])
+def test_range_evonorm_q8(case, ties):
+    """Range-EvoNorm with the requantize step inside: codes, scales, statistics and parameter gradients equal
+    those of the norm call followed by the quantizer."""
+    _ren_q8_check(case, ties, with_res=False, keep_y=False)
+    _ren_q8_check(case, ties, with_res=True, keep_y=True)
+
+
+@pytest.mark.parametrize("env", [{"LPDT_REN_Q8_THREADS": "128"}, {"LPDT_REN_Q8_THREADS": "256", "LPDT_REN_Q8_DEPTH": "4"},
+                                 {"LPDT_REN_Q8_THREADS": "384"}])
+def test_range_evonorm_q8_on_every_launch_shape(env):
+    """The same cases in child processes with the CTA size and ring depth forced."""
+    import os, subprocess, sys
+    if os.environ.get("LPDT_CHILD") == "1":
+        pytest.skip("already inside a child run")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    child_env = dict(os.environ, LPDT_CHILD="1", **env)
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_ops.py"), "-m", "gpu",
+                        "-q", "-x", "-k", "test_range_evonorm_q8 and not launch_shape and not reports"], env=child_env,
+                       cwd=root, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0 and " passed" in r.stdout, r.stdout[-3000:] + r.stderr[-2000:]
+
+
+def test_range_evonorm_q8_reports_shapes_that_do_not_fit():
+    # a sample of 32x32x64 fp32 is 256 KB: beyond one CTA's shared memory
+    assert api.lpdt_range_evonorm_fwd_q8_fits(32, 32, 32, 64, 8) == 0
+    assert api.lpdt_range_evonorm_bwd_q8_fits(32, 32, 32, 64, 8) == 0
+    assert api.lpdt_range_evonorm_fwd_q8_fits(4, 4, 4, 6, 3) == 0          # 2 channels per group: no 4-wide columns
+    # more samples per node than half the CTAs the device can hold at once: the meeting could starve
+    assert api.lpdt_range_evonorm_bwd_q8_fits(4096, 32, 32, 16, 2) == 0
+    t = torch.zeros(2 * 32 * 32 * 64, device="cuda"); ti = torch.zeros(256, dtype=torch.int32, device="cuda")
+    q = torch.zeros(2 * 32 * 32 * 64, dtype=torch.int8, device="cuda")
+    ctl = torch.zeros(api.lpdt_range_evonorm_q8_ctl_size(1), dtype=torch.uint8, device="cuda")
+    with pytest.raises(api.LpdtError) as e:
+        api.lpdt_range_evonorm_fwd_q8(1, 2, 32, 32, 64, 8, 1e-5, t, t, t, t, 64, None, t, t, ti, ti, q, t, ctl)
+    assert e.value.code == 2
+    with pytest.raises(api.LpdtError) as e:      # no control block
+        api.lpdt_range_evonorm_fwd_q8(1, 2, 8, 8, 64, 8, 1e-5, t, t, t, t, 64, None, t, t, ti, ti, q, t, None)
+    assert e.value.code == 3
+
+
 def test_range_evonorm_errors():
     t = torch.zeros(64, device="cuda"); ti = torch.zeros(64, dtype=torch.int32, device="cuda")
     with pytest.raises(api.LpdtError) as e:      # one channel per group: the constant is infinite

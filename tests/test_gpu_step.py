@@ -271,3 +271,40 @@ def test_step_with_node_groups_on_separate_streams(name, nodes, batch, groups):
     torch.cuda.synchronize()
     for t in names:
         assert torch.equal(getattr(a, t), getattr(b, t)), t
+
+
+@pytest.mark.parametrize("name,nodes,batch,kw", [("resnet20", 3, 4, {}), ("vgg11", 2, 2, {}), ("resnet20_topk", 5, 2, {}),
+                                                 ("resnet20", 4, 32, dict(node_groups=2)),
+                                                 ("resnet20", 2, 4, dict(recompute_norm_input=True))])
+def test_step_with_requantize_inside_the_norm_layers(name, nodes, batch, kw):
+    """fuse_requantize: Range-EvoNorm layers in front of (behind, in the backward pass) a convolution write the
+    8-bit codes themselves.  Same codes, so every result equals the default step's bit for bit - eagerly and
+    as a graph replay - and the calls that disappear are quantizer launches."""
+    wl = wlmod.make_workload(name, nodes=nodes, batch=batch)
+    a = TrainStep.from_workload(wl, **kw)
+    b = TrainStep.from_workload(wl, fuse_requantize=True, **kw)
+    assert any(x.get("q8_fwd") for x in b.buf) and any(x.get("q8_bwd") for x in b.buf)
+    la = [c[0] for c in a.record()]
+    lb = [c[0] for c in b.record()]
+    fused = lb.count("lpdt_range_evonorm_fwd_q8") + lb.count("lpdt_range_evonorm_bwd_q8")
+    assert lb.count("lpdt_range_evonorm_fwd_q8") > 0 and lb.count("lpdt_range_evonorm_bwd_q8") > 0
+    assert la.count("lpdt_quantize_with_range") - lb.count("lpdt_quantize_with_range") == fused
+    a.load(wl); b.load(wl)
+    a.run(); b.run()
+    torch.cuda.synchronize()
+    assert int(b.dev_status.item()) == 0
+    names = ["grads", "x_half", "x_hat", "x_out"] + (["loss"] if "labels" in wl else [])
+    for t in names:
+        assert torch.equal(getattr(a, t), getattr(b, t)), t
+    for li, op in enumerate(wl["ops"]):
+        if op["op"] in ("conv", "linear"):
+            assert torch.equal(a.buf[li]["E"], b.buf[li]["E"]), f"E{li}"
+            assert torch.equal(a.buf[li]["qA"], b.buf[li]["qA"]), f"qA{li}"
+    b.capture()
+    a.params.copy_(a.x_out)
+    b.params.copy_(a.params); b.x_hat.copy_(a.x_hat)
+    a.run(); b.replay()
+    torch.cuda.synchronize()
+    assert int(b.dev_status.item()) == 0
+    for t in names:
+        assert torch.equal(getattr(a, t), getattr(b, t)), t
