@@ -53,7 +53,6 @@ struct HaloParams {
 
 struct HaloCtl {
     unsigned long long full[8], empty[8], tmem_full[8], tmem_empty[8], wfull;
-    unsigned long long out_full[2], out_free[2];      // result tiles in shared memory: written by the 4 epilogue warps / read by the store
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -96,7 +95,6 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
         for (int i = 0; i < p.stages; ++i) { mbar_init(smem_u32(&ctl->full[i]), 1); mbar_init(smem_u32(&ctl->empty[i]), 1); }
         for (int i = 0; i < 8; ++i) { mbar_init(smem_u32(&ctl->tmem_full[i]), 1); mbar_init(smem_u32(&ctl->tmem_empty[i]), 4); }
         mbar_init(smem_u32(&ctl->wfull), 1);
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&ctl->out_full[i]), 4); mbar_init(smem_u32(&ctl->out_free[i]), 1); }
         ctl->abort_flag = 0;
         mbar_fence_init();
     }
@@ -205,11 +203,10 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
         const int q = warp & 3;
         const int row = q * 32 + lane;
         const int pw = row % kTileW, phh = row / kTileW;
-        const bool issuer = (warp == 2 && lane == 0);        // issues and tracks the bulk stores
         uint32_t tcount = 0;
         HaloTile c = halo_decode(p, tile_lo);
         int sc_node = -1; float sc = 0.f;
-        if (p.tma_out && issuer) tma_prefetch_desc(&mapY);
+        if (p.tma_out && lane == 0) tma_prefetch_desc(&mapY);
         for (int tile = tile_lo; tile < tile_hi && !ctl->abort_flag; ++tile, ++tcount, halo_next(p, c)) {
             const int w = c.tw * kTileW + pw, h = c.th * kTileH + phh;
             const bool valid = (w < p.Wm) && (h < p.Hm);
@@ -221,13 +218,14 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
             const long long pix = (((long long)c.node * p.B + c.b) * p.Hm + h) * p.Wm + w;
             const uint32_t t_row = tmem_base + ((uint32_t)(q * 32) << 16) + acc * p.N;
             if (p.tma_out) {
-                // Result tile -> shared memory (pixel-major, the layout of the store's box) -> one bulk tensor
-                // store per tile; parts of the box outside the image are not written.  Two tile buffers: the
-                // store of the tile before last must have finished reading this one.
+                // Result rows -> shared memory (pixel-major, the layout of the store's box) -> bulk tensor stores.
+                // Every epilogue warp stores its own 32 pixels (4 rows of the tile) and tracks its own stores, so
+                // the four warps never wait for one another; parts of a box outside the image are not written.
+                // Two buffers per warp: the store issued two tiles ago must have finished reading this one.
                 const int ob = tcount & 1u;
-                const uint32_t use = tcount >> 1;
                 unsigned char *ot = out_tiles + (size_t)ob * 128 * p.N * 4;
-                if (use > 0 && !mbar_wait(smem_u32(&ctl->out_free[ob]), (use - 1) & 1, &ctl->abort_flag, p.dev_status)) break;
+                if (lane == 0) tma_store_wait_read<1>();
+                __syncwarp();
                 const int inner = p.out_inner;
                 const uint32_t sw = inner == 32 ? (uint32_t)(row & 7) : (uint32_t)((row >> 1) & 3);   // the box's swizzle
                 for (int cc = 0; cc < p.N; cc += 16) {
@@ -260,21 +258,12 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
                 if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
                 fence_proxy_async_smem();
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&ctl->out_full[ob]));
-                int ok = 1;
-                if (issuer) {
-                    ok = mbar_wait(smem_u32(&ctl->out_full[ob]), use & 1, &ctl->abort_flag, p.dev_status) ? 1 : 0;
-                    if (ok) {
-                        for (int g = 0; g * p.out_inner < p.N; ++g)
-                            tma_store_5d(&mapY, smem_u32(ot + (size_t)g * 128 * p.out_inner * 4), g * p.out_inner,
-                                         c.tw * kTileW, c.th * kTileH, c.b, c.node);
-                        tma_store_commit();
-                        // every store but this one has finished reading: the other buffer may be written again
-                        tma_store_wait_read<1>();
-                        if (tcount > 0) mbar_arrive(smem_u32(&ctl->out_free[ob ^ 1]));
-                    }
+                if (lane == 0) {
+                    for (int g = 0; g * inner < p.N; ++g)
+                        tma_store_5d(&mapY, smem_u32(ot + ((size_t)g * 128 + q * 32) * inner * 4), g * inner,
+                                     c.tw * kTileW, c.th * kTileH + q * (32 / kTileW), c.b, c.node);
+                    tma_store_commit();
                 }
-                if (warp == 2 && !__shfl_sync(0xffffffffu, ok, 0)) break;     // the whole warp leaves together
                 continue;
             }
             for (int cc = 0; cc < p.N; cc += 16) {
@@ -307,7 +296,7 @@ conv_halo16_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_consta
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&ctl->tmem_empty[acc]));
         }
-        if (p.tma_out && issuer) tma_store_wait_all();       // the tiles in shared memory have been read and written out
+        if (p.tma_out && lane == 0) tma_store_wait_all();    // this warp's rows in shared memory have been read and written out
     }
     tc_fence_before();
     __syncthreads();
@@ -405,7 +394,7 @@ lpdt_status tc_pix_halo(const lpdt_conv_desc &d, int mode, const int8_t *A, cons
     p.dev_status = dev_status;
     CUtensorMap mA, mW, mY;
     if (p.tma_out) {
-        if (!make_map_out_f32(&mY, Y, d.nodes, d.B, p.Hm, p.Wm, p.N, p.out_inner, kTileH, kTileW)) return LPDT_ERR_CUDA;
+        if (!make_map_out_f32(&mY, Y, d.nodes, d.B, p.Hm, p.Wm, p.N, p.out_inner, 32 / kTileW, kTileW)) return LPDT_ERR_CUDA;
     } else {
         mY = CUtensorMap{};
     }
