@@ -388,14 +388,45 @@ big_collect_kernel(const float *__restrict__ x_half, const float *__restrict__ x
 // some of the keys equal to it are taken, those at the lowest positions are: the cut follows the
 // need-th smallest position among them.
 __device__ void select_from_candidates(const Cand *__restrict__ list, int64_t n_cand, int64_t k, const uint32_t *h1,
-                                       int64_t lo, int64_t hi, SelectOut *o) {
+                                       int64_t lo, int64_t hi, SelectOut *o, uint32_t *s_keys, int key_cap) {
     // the collect pass left the exact histogram of the candidates' top 12 bits: the bucket of the k-th largest
-    // key comes from it without a scan, and only the 19 bits below are searched in the list
+    // key comes from it without a scan, and only the 19 bits below are searched
     int b1; long long need1, eq1;
     pick_bucket(h1, kTopBins, (long long)k, &b1, &need1, &eq1);
     long long need, eq;
-    const uint32_t thr = radix_select<false>(n_cand, [&](int64_t e) { return list[e].key; }, need1, kTopShift,
-                                             (uint32_t)b1 << kTopShift, &need, &eq);
+    uint32_t thr;
+    if (eq1 <= (long long)key_cap) {
+        // The bucket's keys (their exact number is known) fit the shared-memory buffer: one pass over the list
+        // copies them there, and the radix passes run over shared memory instead of re-reading the list.
+        __shared__ unsigned int s_n;
+        if (threadIdx.x == 0) s_n = 0;
+        __syncthreads();
+        const unsigned long long *l64 = reinterpret_cast<const unsigned long long *>(list);
+        for (int64_t base = 0; base < n_cand; base += 8 * (int64_t)blockDim.x) {
+            unsigned long long c[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int64_t eu = base + u * (int64_t)blockDim.x + threadIdx.x;
+                c[u] = eu < n_cand ? __ldg(l64 + eu) : 0ull;       // {key, pos}: the key is the low word
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int64_t eu = base + u * (int64_t)blockDim.x + threadIdx.x;
+                const uint32_t key = (uint32_t)c[u];
+                if (eu < n_cand && (int)(key >> kTopShift) == b1) {
+                    const unsigned slot = atomicAdd(&s_n, 1u);
+                    if (slot < (unsigned)key_cap) s_keys[slot] = key;
+                }
+            }
+        }
+        __syncthreads();
+        const int64_t n_in = s_n < (unsigned)key_cap ? s_n : key_cap;      // equals eq1
+        thr = radix_select<false>(n_in, [&](int64_t e) { return s_keys[e]; }, need1, kTopShift,
+                                  (uint32_t)b1 << kTopShift, &need, &eq);
+    } else {
+        thr = radix_select<false>(n_cand, [&](int64_t e) { return list[e].key; }, need1, kTopShift,
+                                  (uint32_t)b1 << kTopShift, &need, &eq);
+    }
     if (eq == need) {
         if (threadIdx.x == 0) { o->thr = thr; o->dense = 0; o->cut = hi; }
         return;
@@ -438,7 +469,40 @@ delta_amax_kernel(const float *__restrict__ x_half, const float *__restrict__ x_
     for (int s = a; s < seg.n_seg && seg.off[s] < c1; ++s) {
         const int64_t lo = seg.off[s] > c0 ? seg.off[s] : c0, hi = seg.off[s + 1] < c1 ? seg.off[s + 1] : c1;
         unsigned int m = 0;
-        for (int64_t e = lo + threadIdx.x; e < hi; e += blockDim.x) {
+        // 16-byte loads, four pairs in flight per thread, over the part of the span where both rows sit on
+        // 16-byte boundaries; scalar loads for the ragged ends (or the whole span)
+        int64_t v0 = lo, v1 = lo;
+        if ((((uintptr_t)(xh + lo) ^ (uintptr_t)(xq + lo)) & 15) == 0) {
+            v0 = lo + (int64_t)(((16 - ((uintptr_t)(xh + lo) & 15)) & 15) >> 2);
+            if (v0 > hi) v0 = hi;
+            v1 = v0 + ((hi - v0) & ~(int64_t)3);
+        }
+        for (int64_t e = lo + threadIdx.x; e < v0; e += blockDim.x) {
+            const unsigned int key = mag_bits(xh[e], xq[e], plus);
+            m = key > m ? key : m;
+        }
+        {
+            const float4 *h4 = reinterpret_cast<const float4 *>(xh + v0), *q4 = reinterpret_cast<const float4 *>(xq + v0);
+            const int64_t n4 = (v1 - v0) >> 2;
+            for (int64_t i = threadIdx.x; i < n4; i += 4 * (int64_t)blockDim.x) {
+                float4 a[4], b[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int64_t iu = i + u * (int64_t)blockDim.x;
+                    if (iu < n4) { a[u] = __ldg(h4 + iu); b[u] = __ldg(q4 + iu); }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    if (i + u * (int64_t)blockDim.x < n4) {
+                        unsigned int k0 = mag_bits(a[u].x, b[u].x, plus), k1 = mag_bits(a[u].y, b[u].y, plus);
+                        unsigned int k2 = mag_bits(a[u].z, b[u].z, plus), k3 = mag_bits(a[u].w, b[u].w, plus);
+                        k0 = k0 > k1 ? k0 : k1; k2 = k2 > k3 ? k2 : k3; k0 = k0 > k2 ? k0 : k2;
+                        m = k0 > m ? k0 : m;
+                    }
+                }
+            }
+        }
+        for (int64_t e = v1 + threadIdx.x; e < hi; e += blockDim.x) {
             const unsigned int key = mag_bits(xh[e], xq[e], plus);
             m = key > m ? key : m;
         }
@@ -470,7 +534,8 @@ select_and_rows_kernel(const float *__restrict__ x_half, const float *__restrict
                        SegTable seg, SelectOut *__restrict__ out, const float *__restrict__ Wmix, int nodes,
                        int32_t *__restrict__ tab, const unsigned int *__restrict__ amax_bits,
                        float *__restrict__ msg_scale, float *__restrict__ msg_inv, BigList big,
-                       const BigCtl *__restrict__ ctl, const Cand *__restrict__ cands, int64_t cand_per_node) {
+                       const BigCtl *__restrict__ ctl, const Cand *__restrict__ cands, int64_t cand_per_node,
+                       int key_cap /*keys the dynamic shared memory holds*/) {
     pdl_enter();
     if ((int)blockIdx.y == nodes) {
         if (blockIdx.x == 0) {
@@ -498,8 +563,9 @@ select_and_rows_kernel(const float *__restrict__ x_half, const float *__restrict
         // the k largest are among the candidates; otherwise the whole-segment path below decides
         const int64_t n_cand = (int64_t)ctl[(int64_t)node * big.n + bi].cand_count;
         if (n_cand >= k && n_cand <= cand_capacity(len)) {
+            extern __shared__ __align__(16) uint32_t s_sel_keys[];
             select_from_candidates(cands + (int64_t)node * cand_per_node + big.cand_base[bi], n_cand, k,
-                                   ctl[(int64_t)node * big.n + bi].h1, lo, hi, o);
+                                   ctl[(int64_t)node * big.n + bi].h1, lo, hi, o, s_sel_keys, key_cap);
             return;
         }
     }
@@ -557,6 +623,7 @@ gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float 
             for (int k = 0; k < V; ++k) hn[k] = 0.f;
             if (live) {
                 SelectOut so = sel[(int64_t)i * seg.n_seg + s0];
+                bool changed = DS;         // the public copy changes only where an entry is sent (top-k: 1 in 100)
                 float q_scale = 1.f, q_inv = 1.f;
                 if (Q8) { q_scale = msg_scale[(int64_t)i * seg.n_seg + s0]; q_inv = msg_inv[(int64_t)i * seg.n_seg + s0]; }
 #pragma unroll
@@ -570,6 +637,7 @@ gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float 
                     const float delta = DS ? __fadd_rn(xh[u][k], xq[u][k]) : __fsub_rn(xh[u][k], xq[u][k]);
                     const uint32_t key = __float_as_uint(delta) & 0x7fffffffu;
                     const bool keep = so.dense || key > so.thr || (key == so.thr && e0 + k < so.cut);
+                    changed |= keep;
                     float msg = delta;
                     if (Q8) {      // the message is the 8-bit code times the step; the state absorbs exactly that
                         const float code = fminf(fmaxf(rintf(__fmul_rn(delta, q_inv)), -127.f), 127.f);
@@ -583,7 +651,7 @@ gossip_mix_kernel(int nodes, int64_t d, const float *__restrict__ x_half, float 
                         st_new[k] = hn[k];
                     }
                 }
-                VecIO<V>::st(x_hat + (int64_t)i * d + e0, st_new);
+                if (changed) VecIO<V>::st(x_hat + (int64_t)i * d + e0, st_new);      // unchanged values are not rewritten
             }
             VecIO<V>::st(s_hat + ((size_t)i * TE + threadIdx.x) * V, hn);
         }
@@ -859,8 +927,22 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
         launch_k(delta_amax_kernel, dim3((unsigned)ceil_div(d, (int64_t)kChunk), nodes), 256, 0, st, x_half, x_hat, d, seg, amax_bits);
         LPDT_LAUNCH_CHECK();
     }
-    launch_k(select_and_rows_kernel, dim3(n_segments, nodes + 1), 1024, 0, st, x_half, x_hat, d, seg, sel, Wmix, nodes, tab,
-             amax_bits, msg_scale, msg_inv, big, ctl, cands, cand_per_node);
+    // Shared-memory buffer for the keys of the threshold's bucket of a long segment (1/16 of an octave of
+    // magnitudes: well under 1/64 of the segment unless the magnitudes are nearly constant; when they do not
+    // fit, the selection reads the candidate list again for every radix pass instead).
+    int key_cap = 0;
+    if (big.n > 0) {
+        int64_t want = longest / 64;
+        key_cap = (int)(want < 1024 ? 1024 : want > 40960 ? 40960 : want);
+        static PerDeviceOnce attr;
+        int dev;
+        if (attr.pending(&dev)) {
+            LPDT_CUDA(cudaFuncSetAttribute(select_and_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 40960 * 4));
+            attr.mark(dev);
+        }
+    }
+    launch_k(select_and_rows_kernel, dim3(n_segments, nodes + 1), 1024, (size_t)key_cap * sizeof(uint32_t), st, x_half, x_hat, d,
+             seg, sel, Wmix, nodes, tab, amax_bits, msg_scale, msg_inv, big, ctl, cands, cand_per_node, key_cap);
     LPDT_LAUNCH_CHECK();
     // parameters per thread: 16-byte accesses need every node's row on a 16-byte boundary (d a multiple of 4);
     // the networks' parameter counts are even but not multiples of 4, which still allows 8-byte accesses
