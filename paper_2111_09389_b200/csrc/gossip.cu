@@ -322,13 +322,14 @@ constexpr int kStage = 2048;
 __global__ void __launch_bounds__(256)
 big_collect_kernel(const float *__restrict__ x_half, const float *__restrict__ x_hat, int64_t d, SegTable seg,
                    BigList big, BigCtl *__restrict__ ctl, const BigState *__restrict__ state,
-                   Cand *__restrict__ cands, int64_t cand_per_node, unsigned int *__restrict__ amax_bits) {
+                   Cand *__restrict__ cands, int64_t cand_per_node, unsigned int *__restrict__ amax_bits,
+                   int chunk /*elements per CTA*/) {
     pdl_enter();
     const int bi = blockIdx.y, node = blockIdx.z, s = big.id[bi], plus = seg.plus;
     const int64_t lo = seg.off[s], hi = seg.off[s + 1];
-    const int64_t c0 = lo + (int64_t)blockIdx.x * kChunk;
+    const int64_t c0 = lo + (int64_t)blockIdx.x * chunk;
     if (c0 >= hi) return;
-    const int64_t c1 = (c0 + kChunk < hi) ? c0 + kChunk : hi;
+    const int64_t c1 = (c0 + chunk < hi) ? c0 + chunk : hi;
     const BigState stt = state[(int64_t)node * big.n + bi];
     const unsigned cap = (unsigned)cand_capacity(hi - lo);
     BigCtl *h = ctl + (int64_t)node * big.n + bi;
@@ -342,32 +343,51 @@ big_collect_kernel(const float *__restrict__ x_half, const float *__restrict__ x
     if (threadIdx.x == 0) s_cnt = 0;
     __syncthreads();
     uint32_t kmax = 0;          // largest magnitude of the chunk: the range of the segment's 8-bit message
-    for (int64_t e = c0 + threadIdx.x; e < c1; e += 4 * blockDim.x) {
-        float a[4], b[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int64_t eu = e + u * blockDim.x;
-            if (eu < c1) { a[u] = xh[eu]; b[u] = xq[eu]; }
+    auto consider = [&](float a, float b, int64_t eu) {
+        const uint32_t key = mag_bits(a, b, plus);
+        kmax = key > kmax ? key : kmax;
+        if ((key >> kTopShift) >= bucket) {
+            atomicAdd(&sh1[key >> kTopShift], 1u);
+            Cand c; c.key = key; c.pos = (uint32_t)(eu - lo);
+            const unsigned slot = atomicAdd(&s_cnt, 1u);
+            if (slot < kStage) stage[slot] = c;
+            else {                                             // a dense stretch: straight to the list
+                const unsigned at = atomicAdd(&h->cand_count, 1u);
+                if (at < cap) list[at] = c;
+            }
         }
+    };
+    // 16-byte loads, four pairs in flight per thread, where both rows sit on 16-byte boundaries; scalar loads
+    // for the ragged ends (or the whole chunk)
+    int64_t v0 = c0, v1 = c0;
+    if ((((uintptr_t)(xh + c0) ^ (uintptr_t)(xq + c0)) & 15) == 0) {
+        v0 = c0 + (int64_t)(((16 - ((uintptr_t)(xh + c0) & 15)) & 15) >> 2);
+        if (v0 > c1) v0 = c1;
+        v1 = v0 + ((c1 - v0) & ~(int64_t)3);
+    }
+    for (int64_t e = c0 + threadIdx.x; e < v0; e += blockDim.x) consider(xh[e], xq[e], e);
+    {
+        const float4 *h4 = reinterpret_cast<const float4 *>(xh + v0), *q4 = reinterpret_cast<const float4 *>(xq + v0);
+        const int64_t n4 = (v1 - v0) >> 2;
+        for (int64_t i = threadIdx.x; i < n4; i += 4 * (int64_t)blockDim.x) {
+            float4 a[4], b[4];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
-            const int64_t eu = e + u * blockDim.x;
-            if (eu < c1) {
-                const uint32_t key = mag_bits(a[u], b[u], plus);
-                kmax = key > kmax ? key : kmax;
-                if ((key >> kTopShift) >= bucket) {
-                    atomicAdd(&sh1[key >> kTopShift], 1u);
-                    Cand c; c.key = key; c.pos = (uint32_t)(eu - lo);
-                    const unsigned slot = atomicAdd(&s_cnt, 1u);
-                    if (slot < kStage) stage[slot] = c;
-                    else {                                             // a dense stretch: straight to the list
-                        const unsigned at = atomicAdd(&h->cand_count, 1u);
-                        if (at < cap) list[at] = c;
-                    }
+            for (int u = 0; u < 4; ++u) {
+                const int64_t iu = i + u * (int64_t)blockDim.x;
+                if (iu < n4) { a[u] = __ldg(h4 + iu); b[u] = __ldg(q4 + iu); }
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int64_t iu = i + u * (int64_t)blockDim.x;
+                if (iu < n4) {
+                    const int64_t e = v0 + 4 * iu;
+                    consider(a[u].x, b[u].x, e); consider(a[u].y, b[u].y, e + 1);
+                    consider(a[u].z, b[u].z, e + 2); consider(a[u].w, b[u].w, e + 3);
                 }
             }
         }
     }
+    for (int64_t e = v1 + threadIdx.x; e < c1; e += blockDim.x) consider(xh[e], xq[e], e);
     __syncthreads();
     if (amax_bits) {            // the same value the range pass of the 8-bit messages would find
         for (int o = 16; o > 0; o >>= 1) { const uint32_t t = __shfl_xor_sync(0xffffffffu, kmax, o); kmax = t > kmax ? t : kmax; }
@@ -915,12 +935,16 @@ static lpdt_status gossip_impl(int32_t nodes, int64_t d, const float *x_half, fl
     if (big.n > 0) {
         if (most_chunks > 0x7fffffff || nodes > 65535) return LPDT_ERR_UNSUPPORTED;
         LPDT_CUDA(cudaMemsetAsync(ctl, 0, (size_t)nodes * big.n * sizeof(BigCtl), st));
-        const dim3 g((unsigned)most_chunks, big.n, nodes);
+        // elements per CTA of the collect pass: every CTA clears and flushes a 4096-bin histogram, so chunks are as
+        // long as still leaves several CTAs per SM (16 K ... 64 K elements)
+        int chunk = kChunk;
+        while (chunk < 65536 && ceil_div(longest, (int64_t)chunk * 2) * big.n * nodes >= 4 * (int64_t)kNumSMs) chunk *= 2;
+        const dim3 g((unsigned)ceil_div(longest, (int64_t)chunk), big.n, nodes);
         const int64_t sample_ctas = ceil_div(longest, kSampleChunk);
         if (sample_ctas > 65535) return LPDT_ERR_UNSUPPORTED;
         launch_k(big_sample_kernel, dim3((unsigned)sample_ctas, big.n, nodes), 256, 0, st, x_half, x_hat, d, seg, big, ctl, state);
         LPDT_LAUNCH_CHECK();
-        launch_k(big_collect_kernel, g, 256, 0, st, x_half, x_hat, d, seg, big, ctl, state, cands, cand_per_node, amax_bits);
+        launch_k(big_collect_kernel, g, 256, 0, st, x_half, x_hat, d, seg, big, ctl, state, cands, cand_per_node, amax_bits, chunk);
         LPDT_LAUNCH_CHECK();
     }
     if (q8 && big.n < n_segments) {
