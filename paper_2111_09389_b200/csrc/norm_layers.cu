@@ -5,6 +5,7 @@
 // Sums that feed statistics or parameter gradients are accumulated in double.  All four
 // passes are HBM-bound streaming kernels.
 #include <math.h>
+#include <cooperative_groups.h>
 #include "common.cuh"
 
 namespace lpdt {
@@ -23,7 +24,11 @@ template <> struct NVec<1> {
     static __device__ __forceinline__ void st(float *p, const float (&o)[1]) { *p = o[0]; }
 };
 
-__device__ __forceinline__ float sigmoidf_acc(float u) { return 1.f / (1.f + expf(-u)); }
+// Logistic function from the hardware's base-2 exponential and reciprocal approximations: a few ulp of relative
+// error (the exponential's grows with |u|: about 1e-6 at |u| = 10), well inside the 1e-5 these layers are held
+// to.  The correctly rounded expf and IEEE division this replaces cost about 30 instructions per element and made
+// both EvoNorm-S0 kernels instruction-bound (38 / 40 % of the HBM copy peak).
+__device__ __forceinline__ float sigmoidf_acc(float u) { return __fdividef(1.f, 1.f + __expf(-u)); }
 
 // ------------------------------------------------------------------ EvoNorm-S0
 // One CTA per (node, sample).  Pass 1: per-thread sums of x and x*x in double, folded per group
@@ -168,6 +173,224 @@ evonorm_bwd_kernel(int HW, int C, int groups, float eps, const float *__restrict
             o[k] = tt * (sig + u * sig * (1.f - sig)) * invD - coef * (xv[k] - muf);
         }
         NVec<V>::st(dxs + (int64_t)p * C + c0, o);
+    }
+}
+
+// ---- EvoNorm-S0 with the sample held in shared memory ---------------------------------------------------
+// The two-pass kernels above read a sample twice; with one CTA per 256 KB sample the samples in flight exceed
+// the L2 and the second pass comes from DRAM again (measured: 2.6 % L2 hit rate, 20 B per element instead of
+// 12 in the backward kernel).  Here a cluster of R CTAs owns a sample: every CTA copies its share of the pixels
+// into shared memory with asynchronous 16-byte copies (all in flight at once), the group sums of the CTAs meet
+// through distributed shared memory (added in rank order by every CTA: the same result everywhere), and the
+// second pass reads shared memory.  Vector columns of 4 channels only.
+__device__ __forceinline__ void nl_cp_async16(void *smem_dst, const void *gsrc) {
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void nl_cp_async_commit_wait() {
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(256, 2)
+evonorm_fwd_cl_kernel(int HW, int C, int groups, float eps, const float *__restrict__ x, const float *__restrict__ v,
+                      const float *__restrict__ gamma, const float *__restrict__ beta, int64_t pstride, int B,
+                      float *__restrict__ y, float *__restrict__ gmean, float *__restrict__ gvar, int R, int ppc,
+                      unsigned hold_off) {
+    namespace cg = cooperative_groups;
+    constexpr int V = 4;
+    pdl_enter();
+    extern __shared__ double sm_d[];
+    const int T = blockDim.x, t = threadIdx.x;
+    double *s_sum = sm_d, *s_sq = sm_d + T, *part = sm_d + 2 * T;       // part: this CTA's [sum | sum of squares][groups]
+    double *g_mu = part + 2 * groups, *g_inv = g_mu + groups;
+    float *hold = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(sm_d) + hold_off);
+    const int CV = C / V, cpg = C / groups;
+    const int col = t % CV, row0 = t / CV, rstep = T / CV;
+    const int c0 = col * V, grp = c0 / cpg;
+    const int rank = (int)(blockIdx.x % R);
+    const int64_t sample = blockIdx.x / R;
+    const int node = (int)(sample / B);
+    const int p_lo = rank * ppc, p_end = (p_lo + ppc < HW) ? p_lo + ppc : HW;
+    const float *xs = x + sample * (int64_t)HW * C;
+    float *ys = y + sample * (int64_t)HW * C;
+    for (int p = p_lo + row0; p < p_end; p += rstep) nl_cp_async16(hold + (size_t)(p - p_lo) * C + c0, xs + (int64_t)p * C + c0);
+    float vc[V], gc[V], bc[V];
+#pragma unroll
+    for (int k = 0; k < V; ++k) {
+        vc[k] = v[(int64_t)node * pstride + c0 + k];
+        gc[k] = gamma[(int64_t)node * pstride + c0 + k];
+        bc[k] = beta[(int64_t)node * pstride + c0 + k];
+    }
+    nl_cp_async_commit_wait();           // every thread reads back only what its own copies brought
+    double sum = 0.0, sq = 0.0;
+    for (int p = p_lo + row0; p < p_end; p += rstep) {
+        const float4 a = *reinterpret_cast<const float4 *>(hold + (size_t)(p - p_lo) * C + c0);
+        const double d0 = a.x, d1 = a.y, d2 = a.z, d3 = a.w;
+        sum += d0; sq += d0 * d0; sum += d1; sq += d1 * d1; sum += d2; sq += d2 * d2; sum += d3; sq += d3 * d3;
+    }
+    s_sum[t] = sum; s_sq[t] = sq;
+    __syncthreads();
+    const int cols = cpg / V, members = cols * rstep;
+    for (int g = t; g < groups; g += T) {
+        double a = 0.0, b = 0.0;
+        for (int m = 0; m < members; ++m) {
+            const int th = (m / cols) * CV + g * cols + (m % cols);
+            a += s_sum[th]; b += s_sq[th];
+        }
+        part[g] = a; part[groups + g] = b;
+    }
+    cg::cluster_group cluster = cg::this_cluster();
+    if (R > 1) cluster.sync(); else __syncthreads();
+    for (int g = t; g < groups; g += T) {
+        double a = 0.0, b = 0.0;
+        for (int r = 0; r < R; ++r) {
+            const double *pr = R > 1 ? cluster.map_shared_rank(part, r) : part;
+            a += pr[g]; b += pr[groups + g];
+        }
+        const double cnt = (double)HW * cpg, mu = a / cnt;
+        double var = b / cnt - mu * mu;
+        if (var < 0.0) var = 0.0;
+        g_mu[g] = mu; g_inv[g] = 1.0 / sqrt(var + (double)eps);
+        if (rank == 0) { gmean[sample * groups + g] = (float)mu; gvar[sample * groups + g] = (float)var; }
+    }
+    __syncthreads();
+    if (R > 1) cluster.barrier_arrive();          // done reading the others' shared memory; waited for before exit
+    const float invD = (float)g_inv[grp];
+    for (int p = p_lo + row0; p < p_end; p += rstep) {
+        const float4 a = *reinterpret_cast<const float4 *>(hold + (size_t)(p - p_lo) * C + c0);
+        const float xv[V] = {a.x, a.y, a.z, a.w};
+        float yv[V];
+#pragma unroll
+        for (int k = 0; k < V; ++k) yv[k] = gc[k] * (xv[k] * sigmoidf_acc(vc[k] * xv[k])) * invD + bc[k];
+        NVec<V>::st(ys + (int64_t)p * C + c0, yv);
+    }
+    if (R > 1) cluster.barrier_wait();
+}
+
+__global__ void __launch_bounds__(256, 2)
+evonorm_bwd_cl_kernel(int HW, int C, int groups, float eps, const float *__restrict__ dy, const float *__restrict__ x,
+                      const float *__restrict__ v, const float *__restrict__ gamma, int64_t pstride, int B,
+                      const float *__restrict__ gmean, const float *__restrict__ gvar, float *__restrict__ dx,
+                      double *__restrict__ acc, int R, int ppc, unsigned hold_off) {
+    namespace cg = cooperative_groups;
+    constexpr int V = 4;
+    pdl_enter();
+    extern __shared__ double sm_d[];
+    const int T = blockDim.x, t = threadIdx.x;
+    double *s_S = sm_d, *part_S = sm_d + T, *g_S = part_S + groups, *s_ch = g_S + groups;      // s_ch: [3][V][T]
+    double *part_ch = s_ch + 3 * V * T;                                                       // [3][C] of this CTA
+    float *hx = reinterpret_cast<float *>(reinterpret_cast<unsigned char *>(sm_d) + hold_off);
+    float *hdy = hx + (size_t)ppc * C;
+    const int CV = C / V, cpg = C / groups;
+    const int col = t % CV, row0 = t / CV, rstep = T / CV;
+    const int c0 = col * V, grp = c0 / cpg;
+    const int rank = (int)(blockIdx.x % R);
+    const int64_t sample = blockIdx.x / R;
+    const int node = (int)(sample / B);
+    const int p_lo = rank * ppc, p_end = (p_lo + ppc < HW) ? p_lo + ppc : HW;
+    const float *xs = x + sample * (int64_t)HW * C;
+    const float *dys = dy + sample * (int64_t)HW * C;
+    float *dxs = dx + sample * (int64_t)HW * C;
+    for (int p = p_lo + row0; p < p_end; p += rstep) {
+        nl_cp_async16(hx + (size_t)(p - p_lo) * C + c0, xs + (int64_t)p * C + c0);
+        nl_cp_async16(hdy + (size_t)(p - p_lo) * C + c0, dys + (int64_t)p * C + c0);
+    }
+    const double mu = (double)gmean[sample * groups + grp];
+    const double Dd = sqrt((double)gvar[sample * groups + grp] + (double)eps);
+    const float invD = (float)(1.0 / Dd);
+    float vc[V], gc[V];
+#pragma unroll
+    for (int k = 0; k < V; ++k) {
+        vc[k] = v[(int64_t)node * pstride + c0 + k];
+        gc[k] = gamma[(int64_t)node * pstride + c0 + k];
+    }
+    nl_cp_async_commit_wait();
+    double S = 0.0, sv[V], sg[V], sb[V];
+#pragma unroll
+    for (int k = 0; k < V; ++k) { sv[k] = 0.0; sg[k] = 0.0; sb[k] = 0.0; }
+    for (int p = p_lo + row0; p < p_end; p += rstep) {
+        const float4 a = *reinterpret_cast<const float4 *>(hx + (size_t)(p - p_lo) * C + c0);
+        const float4 b = *reinterpret_cast<const float4 *>(hdy + (size_t)(p - p_lo) * C + c0);
+        const float xv[V] = {a.x, a.y, a.z, a.w}, dv_[V] = {b.x, b.y, b.z, b.w};
+        float loc[V];
+#pragma unroll
+        for (int k = 0; k < V; ++k) {
+            const float u = vc[k] * xv[k], sig = sigmoidf_acc(u);
+            const float m = xv[k] * sig, tt = dv_[k] * gc[k];
+            S += (double)(tt * m);
+            sb[k] += (double)dv_[k];
+            sg[k] += (double)(dv_[k] * m * invD);
+            sv[k] += (double)(tt * xv[k] * xv[k] * sig * (1.f - sig) * invD);
+            loc[k] = tt * (sig + u * sig * (1.f - sig)) * invD;      // the part of dx that needs no group sum
+        }
+        // dy is not needed again: its place takes the local term, so that the second pass has no logistic to redo
+        *reinterpret_cast<float4 *>(hdy + (size_t)(p - p_lo) * C + c0) = make_float4(loc[0], loc[1], loc[2], loc[3]);
+    }
+    s_S[t] = S;
+#pragma unroll
+    for (int k = 0; k < V; ++k) {
+        s_ch[(0 * V + k) * T + t] = sv[k]; s_ch[(1 * V + k) * T + t] = sg[k]; s_ch[(2 * V + k) * T + t] = sb[k];
+    }
+    __syncthreads();
+    const int cols = cpg / V, members = cols * rstep;
+    for (int g = t; g < groups; g += T) {
+        double a = 0.0;
+        for (int m = 0; m < members; ++m) a += s_S[(m / cols) * CV + g * cols + (m % cols)];
+        part_S[g] = a;
+    }
+    for (int i = t; i < 3 * C; i += T) {          // channel sums of this CTA's pixels: rows of the column in order
+        const int which = i / C, c = i % C, cl = c / V, k = c % V;
+        double a = 0.0;
+        for (int r = 0; r < rstep; ++r) a += s_ch[(which * V + k) * T + r * CV + cl];
+        part_ch[i] = a;
+    }
+    cg::cluster_group cluster = cg::this_cluster();
+    if (R > 1) cluster.sync(); else __syncthreads();
+    for (int g = t; g < groups; g += T) {
+        double a = 0.0;
+        for (int r = 0; r < R; ++r) a += (R > 1 ? cluster.map_shared_rank(part_S, r) : part_S)[g];
+        g_S[g] = a;
+    }
+    if (rank == 0) {
+        for (int i = t; i < 3 * C; i += T) {
+            double a = 0.0;
+            for (int r = 0; r < R; ++r) a += (R > 1 ? cluster.map_shared_rank(part_ch, r) : part_ch)[i];
+            acc[sample * 3 * C + i] = a;
+        }
+    }
+    __syncthreads();
+    if (R > 1) cluster.barrier_arrive();
+    const double cnt = (double)HW * cpg;
+    const float coef = (float)(g_S[grp] / (cnt * Dd * Dd * Dd));
+    const float muf = (float)mu;
+    for (int p = p_lo + row0; p < p_end; p += rstep) {
+        const float4 a = *reinterpret_cast<const float4 *>(hx + (size_t)(p - p_lo) * C + c0);
+        const float4 b = *reinterpret_cast<const float4 *>(hdy + (size_t)(p - p_lo) * C + c0);
+        const float xv[V] = {a.x, a.y, a.z, a.w}, loc[V] = {b.x, b.y, b.z, b.w};
+        float o[V];
+#pragma unroll
+        for (int k = 0; k < V; ++k) o[k] = loc[k] - coef * (xv[k] - muf);
+        NVec<V>::st(dxs + (int64_t)p * C + c0, o);
+    }
+    if (R > 1) cluster.barrier_wait();
+}
+
+// Cluster size and pixels per CTA for the kernels above: the smallest power of two (up to 8, and so that every
+// CTA keeps a thread row) whose share of `bytes_per_pixel` fits `target` bytes; 0 when even 8 CTAs would need
+// more than `limit`.
+static int evonorm_cluster(int HW, int rstep, size_t bytes_per_pixel, size_t target, size_t limit, int *ppc_out) {
+    const int rows = (int)ceil_div(HW, rstep);
+    int R = 1;
+    while (true) {
+        const int ppc = (int)ceil_div(ceil_div(HW, R), rstep) * rstep;
+        const size_t need = (size_t)ppc * bytes_per_pixel;
+        if (need <= target || R == 8 || R * 2 > rows) {
+            if (need > limit) return 0;
+            *ppc_out = ppc;
+            return R;
+        }
+        R *= 2;
     }
 }
 
@@ -415,6 +638,28 @@ extern "C" lpdt_status lpdt_evonorm_s0_fwd(int32_t nodes, int32_t B, int32_t H, 
     const size_t smem = (size_t)(2 * pl.threads + 2 * groups) * sizeof(double);
     if (smem > 48 * 1024) return LPDT_ERR_UNSUPPORTED;
     const dim3 grid((unsigned)((int64_t)nodes * B));
+    static int two_pass = -1;       // LPDT_EVONORM_TWO_PASS=1: the kernels that read a sample twice (A/B timing, parity tests)
+    if (two_pass < 0) { const char *e = getenv("LPDT_EVONORM_TWO_PASS"); two_pass = (e && e[0] == '1') ? 1 : 0; }
+    if (pl.V == 4 && !two_pass) {
+        const int rstep = pl.threads / (C / 4);
+        int ppc = 0;
+        // shares of up to 64 KB: measured best (clusters of 8 lose to cluster scheduling, 128 KB shares to occupancy)
+        const int R = evonorm_cluster(H * W, rstep, (size_t)C * 4, 64 * 1024, 160 * 1024, &ppc);
+        const size_t scratch = align_up((size_t)(2 * pl.threads + 4 * groups) * sizeof(double), 16);
+        if (R > 0 && scratch <= 32 * 1024 && (int64_t)nodes * B * R <= 0x7fffffff) {
+            static PerDeviceOnce attr;
+            int dev;
+            if (attr.pending(&dev)) {
+                LPDT_CUDA(cudaFuncSetAttribute(evonorm_fwd_cl_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024));
+                attr.mark(dev);
+            }
+            launch_k_cluster(evonorm_fwd_cl_kernel, dim3((unsigned)((int64_t)nodes * B * R)), pl.threads,
+                             scratch + (size_t)ppc * C * 4, as_stream(stream), R, H * W, C, groups, eps, x, v, gamma, beta,
+                             pstride, B, y, gmean, gvar, R, ppc, (unsigned)scratch);
+            LPDT_LAUNCH_CHECK();
+            return LPDT_OK;
+        }
+    }
     if (pl.V == 4) launch_k(evonorm_fwd_kernel<4>, grid, pl.threads, smem, as_stream(stream), H * W, C, groups, eps, x, v, gamma, beta, pstride, B, y, gmean, gvar);
     else launch_k(evonorm_fwd_kernel<1>, grid, pl.threads, smem, as_stream(stream), H * W, C, groups, eps, x, v, gamma, beta, pstride, B, y, gmean, gvar);
     LPDT_LAUNCH_CHECK();
@@ -443,8 +688,31 @@ extern "C" lpdt_status lpdt_evonorm_s0_bwd(int32_t nodes, int32_t B, int32_t H, 
     cudaStream_t st = as_stream(stream);
     double *acc = (double *)ws;
     const dim3 grid((unsigned)((int64_t)nodes * B));
-    if (pl.V == 4) launch_k(evonorm_bwd_kernel<4>, grid, pl.threads, smem, st, H * W, C, groups, eps, dy, x, v, gamma, pstride, B, gmean, gvar, dx, acc);
-    else launch_k(evonorm_bwd_kernel<1>, grid, pl.threads, smem, st, H * W, C, groups, eps, dy, x, v, gamma, pstride, B, gmean, gvar, dx, acc);
+    static int two_pass = -1;
+    if (two_pass < 0) { const char *e = getenv("LPDT_EVONORM_TWO_PASS"); two_pass = (e && e[0] == '1') ? 1 : 0; }
+    bool done = false;
+    if (pl.V == 4 && !two_pass) {
+        const int rstep = pl.threads / (C / 4);
+        int ppc = 0;
+        const int R = evonorm_cluster(H * W, rstep, (size_t)C * 8, 64 * 1024, 160 * 1024, &ppc);
+        const size_t scratch = align_up((size_t)(pl.threads + 2 * groups + 12 * pl.threads + 3 * C) * sizeof(double), 16);
+        if (R > 0 && scratch <= 48 * 1024 && (int64_t)nodes * B * R <= 0x7fffffff) {
+            static PerDeviceOnce attr;
+            int dev;
+            if (attr.pending(&dev)) {
+                LPDT_CUDA(cudaFuncSetAttribute(evonorm_bwd_cl_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 216 * 1024));
+                attr.mark(dev);
+            }
+            launch_k_cluster(evonorm_bwd_cl_kernel, dim3((unsigned)((int64_t)nodes * B * R)), pl.threads,
+                             scratch + (size_t)ppc * C * 8, st, R, H * W, C, groups, eps, dy, x, v, gamma, pstride, B, gmean,
+                             gvar, dx, acc, R, ppc, (unsigned)scratch);
+            done = true;
+        }
+    }
+    if (!done) {
+        if (pl.V == 4) launch_k(evonorm_bwd_kernel<4>, grid, pl.threads, smem, st, H * W, C, groups, eps, dy, x, v, gamma, pstride, B, gmean, gvar, dx, acc);
+        else launch_k(evonorm_bwd_kernel<1>, grid, pl.threads, smem, st, H * W, C, groups, eps, dy, x, v, gamma, pstride, B, gmean, gvar, dx, acc);
+    }
     LPDT_LAUNCH_CHECK();
     launch_k(norm_param_finalize, (nodes * 3 * C + 7) / 8, 256, 0, st, acc, nodes, B, C, 3, dv, dgamma, dbeta, gstride);
     LPDT_LAUNCH_CHECK();

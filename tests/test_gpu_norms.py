@@ -42,7 +42,11 @@ def _inputs(case, seed):
 
 EVO_CASES = [((4, 8, 16, 16, 16), 4), ((2, 3, 32, 32, 16), 2), ((2, 2, 8, 8, 64), 8), ((1, 3, 5, 7, 6), 3),
              ((1, 2, 4, 4, 12), 1), ((2, 2, 32, 32, 64), 8), ((1, 2, 2, 2, 512), 64), ((1, 1, 1, 1, 8), 2),
-             ((1, 2, 9, 9, 24), 3)]
+             ((1, 2, 9, 9, 24), 3),
+             # samples split over a cluster of 2, 4 or 8 CTAs (ragged last share), and one too large for the
+             # kernels that hold the sample in shared memory
+             ((1, 2, 31, 33, 64), 16), ((2, 2, 40, 40, 64), 8), ((1, 3, 64, 64, 32), 4), ((1, 1, 96, 96, 64), 8),
+             ((1, 1, 160, 160, 64), 8)]
 
 
 @pytest.mark.parametrize("case,groups", EVO_CASES)
@@ -125,3 +129,17 @@ def test_norm_layer_errors():
     with pytest.raises(api.LpdtError) as e:      # groups must divide C
         api.lpdt_evonorm_s0_fwd(1, 1, 2, 2, 6, 4, 1e-5, t, t, t, t, 6, t, t, t)
     assert e.value.code == 1
+
+
+def test_evonorm_s0_two_pass_kernels():
+    """The kernels that read a sample twice serve shapes the shared-memory kernels do not take; the cases are
+    re-run on them in a child process."""
+    import os, subprocess, sys
+    if os.environ.get("LPDT_CHILD") == "1":
+        pytest.skip("already inside a child run")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    child_env = dict(os.environ, LPDT_CHILD="1", LPDT_EVONORM_TWO_PASS="1")
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(root, "tests", "test_gpu_norms.py"), "-m", "gpu",
+                        "-q", "-x", "-k", "test_evonorm_s0_fwd_bwd"], env=child_env, cwd=root,
+                       capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0 and " passed" in r.stdout, r.stdout[-3000:] + r.stderr[-2000:]
