@@ -176,7 +176,10 @@ __device__ __forceinline__ TileCoord decode_raster(const PixParams &p, int tile)
     return c;
 }
 
-__global__ void __launch_bounds__(kPixThreads, 1)
+// MINB = 2: the register budget of two resident CTAs per SM, for layers whose K loop is a few stages long: a
+// CTA's fill and drain (first operand boxes, the last tile's epilogue) then overlap its neighbour's main loop.
+template <int MINB>
+__global__ void __launch_bounds__(kPixThreads, MINB)
 conv_pix_kernel(const __grid_constant__ CUtensorMap mapA, const __grid_constant__ CUtensorMap mapW,
                 const __grid_constant__ CUtensorMap mapY, const PixParams p) {
     extern __shared__ __align__(1024) unsigned char smem[];
@@ -661,6 +664,13 @@ static bool weight_map(CUtensorMap *m, const int8_t *base, int nodes, int Cout, 
 
 constexpr int kSmemBudget = 200 * 1024;
 constexpr int kMinSmem = 120 * 1024;      // keeps one CTA per SM, so TMEM allocation never waits
+constexpr int kMinSmemTwo = 78 * 1024;    // two-CTAs-per-SM launches: keeps a third one out
+// LPDT_PIX_TWO=0: one CTA per SM for every shape (A/B timing, parity tests)
+static bool pix_two_enabled() {
+    static int on = -1;
+    if (on < 0) { const char *e = getenv("LPDT_PIX_TWO"); on = (e && e[0] == '0') ? 0 : 1; }
+    return on == 1;
+}
 
 bool tc_supported(const lpdt_conv_desc &d) {
     if (d.stride != 1 && d.stride != 2) return false;
@@ -778,6 +788,19 @@ lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const flo
     if (p.stages > 8) p.stages = 8;
     if (p.stages < 2) return LPDT_ERR_UNSUPPORTED;
     p.tmem_cols = pow2_at_least(2 * p.BN);
+    const long long tiles = (long long)p.nodes * p.tilesB * p.tilesH * p.tilesW * p.tilesN * p.ncls;
+    if (tiles > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
+    // Two CTAs per SM for short K loops (at most four stages per tile) over more than one tile per SM: such
+    // a CTA spends most of its time filling and draining, which a neighbour on the same SM hides.  Needs two
+    // stages and the staging buffers inside half of the shared memory and both accumulator pairs in TMEM.
+    bool two = false;
+    {
+        int longest = 0;
+        for (int c = 0; c < p.ncls; ++c) longest = p.cls_iters[c] > longest ? p.cls_iters[c] : longest;
+        const int stages2 = (113 * 1024 - out_bytes - 1024) / stage_bytes;
+        two = pix_two_enabled() && longest <= 4 && tiles > kNumSMs && stages2 >= 2 && 2 * p.tmem_cols <= 512;
+        if (two) p.stages = stages2 > 8 ? 8 : stages2;
+    }
     p.w_rows_per_node = d.Cout;
     p.Y = Y; p.Yacc = Yacc; p.s1 = s1; p.s2 = s2; p.bias = bias; p.bias_stride = bias_stride;
     p.dev_status = dev_status; p.uns = uns ? 1 : 0;
@@ -801,19 +824,20 @@ lpdt_status tc_pix(const lpdt_conv_desc &d, int mode, const int8_t *A, const flo
         if (!make_map(&mY, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, Y, 5, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B))
             return LPDT_ERR_CUDA;
     }
-    if (smem < kMinSmem) smem = kMinSmem;
-    if (smem > 227 * 1024) return LPDT_ERR_UNSUPPORTED;
+    if (smem < (two ? kMinSmemTwo : kMinSmem)) smem = two ? kMinSmemTwo : kMinSmem;
+    if (smem > (two ? (size_t)113 * 1024 : (size_t)227 * 1024)) return LPDT_ERR_UNSUPPORTED;
     static PerDeviceOnce attr;
     int dev;
     if (attr.pending(&dev)) {
-        LPDT_CUDA(cudaFuncSetAttribute(conv_pix_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        LPDT_CUDA(cudaFuncSetAttribute(conv_pix_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        LPDT_CUDA(cudaFuncSetAttribute(conv_pix_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 113 * 1024));
         attr.mark(dev);
     }
-    const long long tiles = (long long)p.nodes * p.tilesB * p.tilesH * p.tilesW * p.tilesN * p.ncls;
-    if (tiles > 0x7fffffff) return LPDT_ERR_UNSUPPORTED;
-    const int grid = (int)(tiles < kNumSMs ? tiles : kNumSMs);
+    const int slots = two ? 2 * kNumSMs : kNumSMs;
+    const int grid = (int)(tiles < slots ? tiles : slots);
     g_last_kernel = "lpdt::tc::conv_pix_kernel";
-    launch_k(conv_pix_kernel, grid, kPixThreads, smem, st, mA, mW, mY, p);
+    if (two) launch_k(conv_pix_kernel<2>, grid, kPixThreads, smem, st, mA, mW, mY, p);
+    else launch_k(conv_pix_kernel<1>, grid, kPixThreads, smem, st, mA, mW, mY, p);
     LPDT_LAUNCH_CHECK();
     return LPDT_OK;
 }

@@ -1029,7 +1029,8 @@ def test_range_evonorm_cases_on_every_cluster_size(cluster):
 
 
 @pytest.mark.parametrize("env", [{"LPDT_FORCE_HALO": "1"}, {"LPDT_DISABLE_HALO": "1"}, {"LPDT_DISABLE_TC": "1"},
-                                 {"LPDT_AFFINE_SEPARATE": "1"}, {"LPDT_PIX_DIRECT_STORE": "1", "LPDT_DISABLE_HALO": "1"}])
+                                 {"LPDT_AFFINE_SEPARATE": "1"}, {"LPDT_PIX_DIRECT_STORE": "1", "LPDT_DISABLE_HALO": "1"},
+                                 {"LPDT_PIX_TWO": "0", "LPDT_DISABLE_HALO": "1"}])
 def test_qconv_cases_on_every_kernel_family(env):
     """The kernel choice is made once per process from the environment, so the contraction
     cases are re-run in child processes with the halo kernels forced, with the halo kernels
