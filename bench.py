@@ -433,7 +433,14 @@ def run_step_workload(name, rank, world, steps, warmup, graph=True, **step_optio
     # next batch runs on a copy stream while the current step computes, as a training loop would do it
     x_host = torch.from_numpy(wl["x"]).pin_memory()
     lab_host = torch.from_numpy(wl["labels"]).pin_memory() if "labels" in wl else None
-    loss_host = torch.empty(wl["nodes"], dtype=torch.float32).pin_memory()
+    # the loss of every step is copied to pinned host memory inside the timed region; the host waits for it one
+    # step late (two buffers), as a loop that logs the loss would, so that the next step is already queued
+    loss_host = [torch.empty(wl["nodes"], dtype=torch.float32).pin_memory() for _ in range(2)]
+    loss_there = [torch.cuda.Event() for _ in range(2)]
+    for _ in range(2):                       # untimed: the staging buffers and the copy stream are created here
+        st.upload(x_host, lab_host)
+        st.step_from_upload(step)
+    torch.cuda.synchronize()
     barrier(world)
     t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     t0.record()
@@ -442,8 +449,11 @@ def run_step_workload(name, rank, world, steps, warmup, graph=True, **step_optio
         st.step_from_upload(step)
         if i + 1 < steps:
             st.upload(x_host, lab_host)
-        loss_host.copy_(st.loss, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
+        loss_host[i % 2].copy_(st.loss, non_blocking=True)
+        loss_there[i % 2].record()
+        if i >= 1:
+            loss_there[(i - 1) % 2].synchronize()
+    loss_there[(steps - 1) % 2].synchronize()
     t1.record()
     torch.cuda.synchronize()
     barrier(world)
@@ -452,7 +462,7 @@ def run_step_workload(name, rank, world, steps, warmup, graph=True, **step_optio
     res = {"ms_per_step": ms_total / steps, "value": job_value(world, images, ms_total, steps),
            "e2e": {"value": world * images / (e2e_ms * 1e-3), "unit": UNIT,
                    "h2d_bytes_per_step": int(x_host.numel() * 4 + (lab_host.numel() * 4 if lab_host is not None else 0)),
-                   "d2h_bytes_per_step": int(loss_host.numel() * 4)},
+                   "d2h_bytes_per_step": int(loss_host[0].numel() * 4)},
            "int8_tops": 2 * macs * world / (ms_total / steps * 1e-3) / 1e12, "macs_per_step": macs,
            "launches": int(launches), "launches_per_step": int(launches) // max(1, steps),
            "nodes": wl["nodes"], "batch_per_node": wl["batch"], "params_per_node": wl["d"],
