@@ -593,6 +593,38 @@ def test_range_evonorm_q8_reports_shapes_that_do_not_fit():
     assert e.value.code == 3
 
 
+def test_range_evonorm_q8_with_a_control_block_that_was_not_cleared():
+    """The control block must be zero at launch.  When its ticket counter is not, the tickets name no sample of
+    the call: every CTA records LPDT_ERR_INVALID_ARG and returns without touching the tensors (no out-of-range
+    access), and the context stays usable."""
+    nodes, B, H, W, C, groups = 2, 4, 8, 8, 16, 2
+    x, P, dy = _ren_inputs((nodes, B, H, W, C, groups), seed=2)
+    f = lambda *s: torch.empty(*s, dtype=torch.float32, device="cuda")
+    i = lambda *s: torch.empty(*s, dtype=torch.int32, device="cuda")
+    Pd, stride = dev(P), P.shape[1]
+    n = B * H * W * C
+    ctl = torch.zeros(api.lpdt_range_evonorm_q8_ctl_size(nodes) // 4, dtype=torch.int32, device="cuda")
+    ctl[3 * nodes] = nodes * B                         # the ticket counter of a call that never finished
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    q = torch.full((nodes, n), 77, dtype=torch.int8, device="cuda")
+    sc = torch.full((nodes,), -1.0, device="cuda")
+    gmin, gmax, amin_, amax_ = f(nodes, B, groups), f(nodes, B, groups), i(nodes, B, groups), i(nodes, B, groups)
+    api.lpdt_range_evonorm_fwd_q8(nodes, B, H, W, C, groups, 1e-5, dev(x), Pd, Pd[:, C:], Pd[:, 2 * C:], stride, None, gmin,
+                                  gmax, amin_, amax_, q, sc, ctl.view(torch.uint8), dev_status=status)
+    torch.cuda.synchronize()
+    assert int(status.item()) == 1                     # LPDT_ERR_INVALID_ARG
+    assert (q == 77).all() and (sc == -1.0).all()
+    # cleared, the same buffers serve a correct call
+    ctl.zero_(); status.zero_()
+    api.lpdt_range_evonorm_fwd_q8(nodes, B, H, W, C, groups, 1e-5, dev(x), Pd, Pd[:, C:], Pd[:, 2 * C:], stride, None, gmin,
+                                  gmax, amin_, amax_, q, sc, ctl.view(torch.uint8), dev_status=status)
+    v, g, b = P[:, :C], P[:, C:2 * C], P[:, 2 * C:3 * C]
+    y32 = oracle.range_evonorm_fwd(x, v, g, b, groups, 1e-5, "f32")[0]
+    q_ref, s_ref = oracle.quantize_sym_s8(y32.reshape(nodes, n))
+    assert int(status.item()) == 0 and not ctl.any()
+    assert np.array_equal(q.cpu().numpy(), q_ref) and np.array_equal(sc.cpu().numpy(), s_ref)
+
+
 def test_range_evonorm_errors():
     t = torch.zeros(64, device="cuda"); ti = torch.zeros(64, dtype=torch.int32, device="cuda")
     with pytest.raises(api.LpdtError) as e:      # one channel per group: the constant is infinite
