@@ -428,7 +428,7 @@ __device__ __forceinline__ float from_ordered(uint32_t o) {
     return __uint_as_float((o & 0x80000000u) ? (o & 0x7fffffffu) : ~o);
 }
 
-constexpr int kRbnIters = 16;       // pixel rows per thread in one CTA
+constexpr int kRbnIters = 32;       // pixel rows per thread in one CTA
 
 template <int V>
 __global__ void __launch_bounds__(256)
@@ -445,21 +445,28 @@ rbn_stats_kernel(int64_t P, int C, const float *__restrict__ x, RbnStat *__restr
     double sum[V]; unsigned long long mx[V], mn[V];
 #pragma unroll
     for (int k = 0; k < V; ++k) { sum[k] = 0.0; mx[k] = 0ull; mn[k] = 0ull; }
-#pragma unroll 4
-    for (int it = 0; it < kRbnIters; ++it) {
-        const int64_t p = p0 + row0 + (int64_t)it * rstep;
-        if (p >= P) continue;
-        float xv[V];
-        NVec<V>::ld(xs + p * C + c0, xv);
-        const unsigned long long inv_pos = 0xFFFFFFFFull - (unsigned long long)p;
+    // four independent 16-byte loads are issued before any of them is used
+    for (int it0 = 0; it0 < kRbnIters; it0 += 4) {
+        float xb[4][V];
 #pragma unroll
-        for (int k = 0; k < V; ++k) {
-            sum[k] += (double)xv[k];
-            // + 0.f turns -0 into +0, so that equal zeros tie (and the lowest position wins) as in a float compare
-            const unsigned long long a = ((unsigned long long)ordered_bits(xv[k] + 0.f) << 32) | inv_pos;
-            const unsigned long long b = ((unsigned long long)ordered_bits(-xv[k] + 0.f) << 32) | inv_pos;
-            mx[k] = a > mx[k] ? a : mx[k];
-            mn[k] = b > mn[k] ? b : mn[k];
+        for (int u = 0; u < 4; ++u) {
+            const int64_t p = p0 + row0 + (int64_t)(it0 + u) * rstep;
+            if (p < P) NVec<V>::ld(xs + p * C + c0, xb[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int64_t p = p0 + row0 + (int64_t)(it0 + u) * rstep;
+            if (p >= P) continue;
+            const unsigned long long inv_pos = 0xFFFFFFFFull - (unsigned long long)p;
+#pragma unroll
+            for (int k = 0; k < V; ++k) {
+                sum[k] += (double)xb[u][k];
+                // + 0.f turns -0 into +0, so that equal zeros tie (and the lowest position wins) as in a float compare
+                const unsigned long long a = ((unsigned long long)ordered_bits(xb[u][k] + 0.f) << 32) | inv_pos;
+                const unsigned long long b = ((unsigned long long)ordered_bits(-xb[u][k] + 0.f) << 32) | inv_pos;
+                mx[k] = a > mx[k] ? a : mx[k];
+                mn[k] = b > mn[k] ? b : mn[k];
+            }
         }
     }
 #pragma unroll
@@ -511,15 +518,22 @@ rbn_apply_kernel(int64_t P, int C, float eps, float Cb, const float *__restrict_
         }
     }
     const int64_t p0 = (int64_t)blockIdx.x * rstep * kRbnIters;
-#pragma unroll 4
-    for (int it = 0; it < kRbnIters; ++it) {
-        const int64_t p = p0 + row0 + (int64_t)it * rstep;
-        if (p >= P) continue;
-        float xv[V], yv[V];
-        NVec<V>::ld(xs + p * C + c0, xv);
+    for (int it0 = 0; it0 < kRbnIters; it0 += 4) {
+        float xb[4][V];
 #pragma unroll
-        for (int k = 0; k < V; ++k) yv[k] = gc[k] * (xv[k] - mu[k]) * invD[k] + bc[k];
-        NVec<V>::st(ys + p * C + c0, yv);
+        for (int u = 0; u < 4; ++u) {
+            const int64_t p = p0 + row0 + (int64_t)(it0 + u) * rstep;
+            if (p < P) NVec<V>::ld(xs + p * C + c0, xb[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int64_t p = p0 + row0 + (int64_t)(it0 + u) * rstep;
+            if (p >= P) continue;
+            float yv[V];
+#pragma unroll
+            for (int k = 0; k < V; ++k) yv[k] = gc[k] * (xb[u][k] - mu[k]) * invD[k] + bc[k];
+            NVec<V>::st(ys + p * C + c0, yv);
+        }
     }
 }
 
@@ -539,15 +553,20 @@ rbn_bwd_sums_kernel(int64_t P, int C, const float *__restrict__ dy, const float 
 #pragma unroll
     for (int k = 0; k < V; ++k) { mu[k] = cmean[(int64_t)node * C + c0 + k]; a[k] = 0.0; b[k] = 0.0; }
     const int64_t p0 = (int64_t)blockIdx.x * rstep * kRbnIters;
-#pragma unroll 4
-    for (int it = 0; it < kRbnIters; ++it) {
-        const int64_t p = p0 + row0 + (int64_t)it * rstep;
-        if (p >= P) continue;
-        float xv[V], dv_[V];
-        NVec<V>::ld(xs + p * C + c0, xv);
-        NVec<V>::ld(dys + p * C + c0, dv_);
+    for (int it0 = 0; it0 < kRbnIters; it0 += 4) {
+        float xb[4][V], db[4][V];
 #pragma unroll
-        for (int k = 0; k < V; ++k) { a[k] += (double)dv_[k]; b[k] += (double)dv_[k] * (double)(xv[k] - mu[k]); }
+        for (int u = 0; u < 4; ++u) {
+            const int64_t p = p0 + row0 + (int64_t)(it0 + u) * rstep;
+            if (p < P) { NVec<V>::ld(xs + p * C + c0, xb[u]); NVec<V>::ld(dys + p * C + c0, db[u]); }
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int64_t p = p0 + row0 + (int64_t)(it0 + u) * rstep;
+            if (p >= P) continue;
+#pragma unroll
+            for (int k = 0; k < V; ++k) { a[k] += (double)db[u][k]; b[k] += (double)db[u][k] * (double)(xb[u][k] - mu[k]); }
+        }
     }
 #pragma unroll
     for (int k = 0; k < V; ++k) { s_a[k * T + t] = a[k]; s_b[k * T + t] = b[k]; }
@@ -593,19 +612,26 @@ rbn_bwd_apply_kernel(int64_t P, int C, float eps, float Cb, const float *__restr
         }
     }
     const int64_t p0 = (int64_t)blockIdx.x * rstep * kRbnIters;
-#pragma unroll 4
-    for (int it = 0; it < kRbnIters; ++it) {
-        const int64_t p = p0 + row0 + (int64_t)it * rstep;
-        if (p >= P) continue;
-        float dv_[V], o[V];
-        NVec<V>::ld(dys + p * C + c0, dv_);
+    for (int it0 = 0; it0 < kRbnIters; it0 += 4) {
+        float db[4][V];
 #pragma unroll
-        for (int k = 0; k < V; ++k) {
-            o[k] = dv_[k] * gD[k] - shift[k];
-            if (p == (int64_t)amx[k]) o[k] -= coef[k];
-            if (p == (int64_t)amn[k]) o[k] += coef[k];
+        for (int u = 0; u < 4; ++u) {
+            const int64_t p = p0 + row0 + (int64_t)(it0 + u) * rstep;
+            if (p < P) NVec<V>::ld(dys + p * C + c0, db[u]);
         }
-        NVec<V>::st(dxs + p * C + c0, o);
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const int64_t p = p0 + row0 + (int64_t)(it0 + u) * rstep;
+            if (p >= P) continue;
+            float o[V];
+#pragma unroll
+            for (int k = 0; k < V; ++k) {
+                o[k] = db[u][k] * gD[k] - shift[k];
+                if (p == (int64_t)amx[k]) o[k] -= coef[k];
+                if (p == (int64_t)amn[k]) o[k] += coef[k];
+            }
+            NVec<V>::st(dxs + p * C + c0, o);
+        }
     }
 }
 
