@@ -306,9 +306,11 @@ evonorm_bwd_cl_kernel(int HW, int C, int groups, float eps, const float *__restr
         gc[k] = gamma[(int64_t)node * pstride + c0 + k];
     }
     nl_cp_async_commit_wait();
-    double S = 0.0, sv[V], sg[V], sb[V];
+    // A thread owns at most a few dozen rows of its CTA's share (the share is bounded by the shared memory), so
+    // its own partial sums stay in fp32; every combination across threads, CTAs and samples is done in double.
+    float S = 0.f, sv[V], sg[V], sb[V];
 #pragma unroll
-    for (int k = 0; k < V; ++k) { sv[k] = 0.0; sg[k] = 0.0; sb[k] = 0.0; }
+    for (int k = 0; k < V; ++k) { sv[k] = 0.f; sg[k] = 0.f; sb[k] = 0.f; }
     for (int p = p_lo + row0; p < p_end; p += rstep) {
         const float4 a = *reinterpret_cast<const float4 *>(hx + (size_t)(p - p_lo) * C + c0);
         const float4 b = *reinterpret_cast<const float4 *>(hdy + (size_t)(p - p_lo) * C + c0);
@@ -318,19 +320,20 @@ evonorm_bwd_cl_kernel(int HW, int C, int groups, float eps, const float *__restr
         for (int k = 0; k < V; ++k) {
             const float u = vc[k] * xv[k], sig = sigmoidf_acc(u);
             const float m = xv[k] * sig, tt = dv_[k] * gc[k];
-            S += (double)(tt * m);
-            sb[k] += (double)dv_[k];
-            sg[k] += (double)(dv_[k] * m * invD);
-            sv[k] += (double)(tt * xv[k] * xv[k] * sig * (1.f - sig) * invD);
+            S += tt * m;
+            sb[k] += dv_[k];
+            sg[k] += dv_[k] * m * invD;
+            sv[k] += tt * xv[k] * xv[k] * sig * (1.f - sig) * invD;
             loc[k] = tt * (sig + u * sig * (1.f - sig)) * invD;      // the part of dx that needs no group sum
         }
         // dy is not needed again: its place takes the local term, so that the second pass has no logistic to redo
         *reinterpret_cast<float4 *>(hdy + (size_t)(p - p_lo) * C + c0) = make_float4(loc[0], loc[1], loc[2], loc[3]);
     }
-    s_S[t] = S;
+    s_S[t] = (double)S;
 #pragma unroll
     for (int k = 0; k < V; ++k) {
-        s_ch[(0 * V + k) * T + t] = sv[k]; s_ch[(1 * V + k) * T + t] = sg[k]; s_ch[(2 * V + k) * T + t] = sb[k];
+        s_ch[(0 * V + k) * T + t] = (double)sv[k]; s_ch[(1 * V + k) * T + t] = (double)sg[k];
+        s_ch[(2 * V + k) * T + t] = (double)sb[k];
     }
     __syncthreads();
     const int cols = cpg / V, members = cols * rstep;
